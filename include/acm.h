@@ -1,0 +1,203 @@
+/*
+ * acm.h -- C ABI of the B200 (sm_100a) AcceptMoE verifier-side MoE layer.
+ *
+ * One call processes ONE speculative-decoding verification block (T <= 64 draft-tree
+ * nodes, node 0 = root) through ONE MoE layer of the target model:
+ *
+ *   stage 1  router logits z_t = W_r x_t (+ bias), r_t = softmax(z_t), natural top-k K_t
+ *            (Section 3.1, Eq. 1)
+ *   stage 2  commitment-weighted demand u_e (Eq. 3, Eq. 4), root anchor A (Eq. 5),
+ *            self-sized eligible set S = A u Top_{n_er}(U_R) (Eq. 6), and under
+ *            offloading the residency-aware pruning S -> S' (Eq. 7)
+ *   stage 3  top-k routing restricted to S' (Eq. 2) with the target's own weighting
+ *   stage 4  grouped SwiGLU expert FFN over the activated experts + weighted combine
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer on the context's device unless marked "host".
+ *   - Matrices are row-major and dense.  dtype ACM_BF16: 2-byte bfloat16; ACM_F32: float.
+ *   - Expert e (0-based) is bit e%32 of word e/32 in every bitmask (uint32 words).
+ *   - All calls are asynchronous on `stream` and return after enqueueing; argument errors
+ *     are found on the host before anything is enqueued and leave outputs untouched.
+ *     Failures seen by device code (a bounded wait that ran out, a non-finite logit) are
+ *     sticky in a status word read by acm_device_status().  Nothing traps, aborts or prints.
+ *   - The caller owns every buffer it passes.  The context borrows weight pointers until
+ *     acm_destroy() or the next acm_set_layer_weights() for that layer, and owns its
+ *     workspace (allocated in acm_create with cudaMalloc on the current device).
+ *   - One context serves one stream at a time: calls on the same context that overlap on
+ *     the GPU race on its workspace.
+ *   - Limits (else ACM_ERR_UNSUPPORTED): n_experts <= 128, top_k <= 8, T <= 64;
+ *     bf16: hidden % 128 == 0, inter % 64 == 0; f32: hidden % 32 == 0.
+ *
+ * Numerical contract of stages 1-3.  Everything that decides a set member, a count or an
+ * index is IEEE binary32 in a fixed order: the logit dot product keeps 32 interleaved
+ * partial sums (partial l takes h = l, l+32, ... ascending, fused multiply-add) folded by a
+ * halving tree; sums over the expert axis use a 128-slot halving tree; exp/log are fixed
+ * polynomial recipes; demand accumulates with fused multiply-add over nodes in ascending
+ * order; every ranking is total, ties to the lower expert index.  Routing weights and FFN
+ * outputs carry no such contract (tensor-core accumulation order is unspecified).
+ */
+#ifndef ACM_H_
+#define ACM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct acm_ctx acm_ctx;          /* opaque */
+typedef void* acm_stream;                /* a cudaStream_t (NULL = default stream) */
+
+typedef enum {
+  ACM_OK = 0,
+  ACM_ERR_INVALID = 1,      /* bad argument */
+  ACM_ERR_UNSUPPORTED = 2,  /* outside the limits above */
+  ACM_ERR_CUDA = 3,         /* a CUDA runtime/driver call failed */
+  ACM_ERR_TIMEOUT = 4,      /* a bounded device-side wait ran out */
+  ACM_ERR_NOMEM = 5,
+  ACM_ERR_NONFINITE = 6     /* a router logit was NaN or infinite */
+} acm_status;
+
+typedef enum { ACM_F32 = 0, ACM_BF16 = 1 } acm_dtype;
+
+/* "preserves the target's native post-top-k weighting" (Section 3.1, below Eq. 2) */
+typedef enum {
+  ACM_W_RENORM_TOPK = 0,     /* w = r_e / sum of r over the k selected experts          */
+  ACM_W_SOFTMAX_RAW = 1,     /* w = r_e of the unmasked softmax (zero-probability mask) */
+  ACM_W_SOFTMAX_MASKED = 2   /* w = softmax over the eligible experts only (logit mask) */
+} acm_weighting;
+
+typedef enum {
+  ACM_DEMAND_TOPK_MASS = 0,  /* Eq. 4: router mass inside each node's natural top-k */
+  ACM_DEMAND_FULL_MASS = 1,  /* sum_t alpha_t r_{t,e} without the indicator (MoE-Spec aggregation) */
+  ACM_DEMAND_VOTES = 2       /* natural top-k vote counts */
+} acm_demand_mode;
+
+typedef struct {
+  int32_t hidden;        /* H */
+  int32_t n_experts;     /* E, routed experts */
+  int32_t top_k;         /* k */
+  int32_t inter;         /* I, per-expert SwiGLU intermediate size */
+  int32_t n_shared;      /* always-on shared experts (weight 1, outside selection), 0..4 */
+  int32_t max_nodes;     /* largest T that will be passed (<= 64) */
+  int32_t n_layers;      /* number of layer slots */
+  int32_t dtype;         /* acm_dtype of hidden states and all weights */
+  int32_t weighting;     /* acm_weighting */
+  float routed_scale;    /* multiplies every routed combine weight (1 = none) */
+} acm_model_desc;
+
+typedef struct {
+  int32_t demand;        /* acm_demand_mode; 0 = the paper's Eq. 4 */
+  int32_t use_anchors;   /* 1 = keep the anchor nodes' natural top-k (Eq. 5) */
+  int32_t fixed_budget;  /* 0 = self-sized (Eq. 6); B > 0 = hold the total set size at B */
+  float ceil_guard;      /* tau in n_er = ceil(exp(H) - tau); 2^-10 by default, 0 = literal */
+  int32_t residency;     /* 0 off; 1 = Eq. 7 pruning; 2 = (S intersect resident) union anchors */
+  int32_t max_remove;    /* optional cap on Eq. 7 removals; >= n_experts = nonbinding */
+} acm_select_params;
+
+/* Written by device code (all int32 so that it can live in device or pinned memory). */
+typedef struct {
+  int32_t n_anchor;           /* |A| */
+  int32_t n_er;               /* effective-rank cardinality of Eq. 6 (0 if unused) */
+  int32_t n_eligible;         /* |S| before pruning */
+  int32_t n_eligible_pruned;  /* |S'| */
+  int32_t n_activated;        /* eligible experts that received at least one node */
+  int32_t n_natural_union;    /* |U_nat| of Eq. 1 */
+  int32_t displaced_aS;       /* a(S): natural assignments displaced by restricting to S */
+  int32_t pruned_m;           /* m* of Eq. 7 */
+  int32_t n_staged;           /* activated experts that were not GPU-resident */
+  int32_t reserved[3];
+} acm_block_stats;
+
+/* Fills the paper's defaults: Eq. 4 demand, anchors on, self-sized, tau = 2^-10, no residency. */
+void acm_default_select_params(acm_select_params* p);
+
+/* Creates a context on the current CUDA device and allocates its workspace.  host pointers. */
+acm_status acm_create(const acm_model_desc* desc, acm_ctx** out);
+acm_status acm_destroy(acm_ctx* ctx);
+
+/* Registers (borrows) the device weights of one layer:
+ *   w_router [E,H]; router_bias [E] float or NULL; w_gate_up [E,2I,H] (rows 0..I-1 gate,
+ *   I..2I-1 up); w_down [E,H,I]; shared_gate_up [n_shared,2I,H] and shared_down
+ *   [n_shared,H,I] (NULL when n_shared == 0).  bf16 expert tensors must be 16-byte aligned. */
+acm_status acm_set_layer_weights(acm_ctx* ctx, int layer, const void* w_router,
+                                 const float* router_bias, const void* w_gate_up,
+                                 const void* w_down, const void* shared_gate_up,
+                                 const void* shared_down);
+
+/* Eq. 3 on the host: alpha_t = p_table[depth_t]^beta * N_{depth_t}^{-1/2} (width factor
+ * optional), evaluated in double and rounded once.  All pointers are HOST pointers.
+ * ACM_ERR_INVALID if a depth lies outside the table. */
+acm_status acm_node_weights(const int32_t* depth, int T, const float* p_table, int n_depths,
+                            float beta, int width_norm, float* alpha_out);
+
+/* Stage 1 (Section 3.1): x [T,H] -> logits [T,E], probs [T,E] (float), nat_idx [T,k]
+ * (int32, best first; ties to the lower index).  probs / nat_idx may be NULL. */
+acm_status acm_router(acm_ctx* ctx, int layer, const void* x, int T, float* logits,
+                      float* probs, int32_t* nat_idx, acm_stream stream);
+
+/* Stage 2 (Sections 3.2-3.4): probs [T,E], nat_idx [T,k], alpha [T] ->
+ * eligible_mask [ceil(E/32)] (= S', the set routing is restricted to), eligible_count [1].
+ * anchor_nodes: int32 node ids or NULL for {0}.  resident_mask: [ceil(E/32)] words, needed
+ * when params->residency != 0.  Optional outputs (may be NULL): demand [E] float,
+ * unpruned_mask [ceil(E/32)] (= S), stats [1]. */
+acm_status acm_select_eligible(acm_ctx* ctx, const float* probs, const int32_t* nat_idx, int T,
+                               const float* alpha, const int32_t* anchor_nodes,
+                               int n_anchor_nodes, const acm_select_params* params /*host*/,
+                               const uint32_t* resident_mask, uint32_t* eligible_mask,
+                               int32_t* eligible_count, float* demand, uint32_t* unpruned_mask,
+                               acm_block_stats* stats, acm_stream stream);
+
+/* Stage 3 (Eq. 2): logits [T,E], eligible_mask -> idx [T,k] (int32, best first, -1 where
+ * fewer than k experts are eligible), w [T,k] (float combine weights, 0 for empty slots). */
+acm_status acm_route_restricted(acm_ctx* ctx, const float* logits, const uint32_t* eligible_mask,
+                                int T, int32_t* idx, float* w, acm_stream stream);
+
+/* Stage 4 alone: y_t = sum_j w[t,j] * down_e( silu(gate_e x_t) * up_e x_t ), e = idx[t,j]
+ * (+ shared experts with weight 1).  x [T,H], idx/w [T,k] -> out [T,H] float (overwritten). */
+acm_status acm_expert_ffn(acm_ctx* ctx, int layer, const void* x, int T, const int32_t* idx,
+                          const float* w, float* out, acm_stream stream);
+
+/* Stages 1-4 for one block and layer.  alpha [T] device.  eligible_mask_override != NULL
+ * skips stage 2 and routes inside the given set (all ones = the natural-routing union path).
+ * Optional outputs (NULL to skip): idx_out [T,k], w_out [T,k], mask_out [ceil(E/32)],
+ * stats [1].  out [T,H] float is overwritten.
+ * With a residency registered for the layer (acm_set_resident) and params->residency != 0,
+ * activated experts that are not GPU-resident are copied from the registered pinned host
+ * tensors into the context's staging slots before their FFN runs; this needs one host
+ * synchronisation on `stream` inside the call. */
+acm_status acm_moe_verify(acm_ctx* ctx, int layer, const void* x, int T, const float* alpha,
+                          const acm_select_params* params /*host*/,
+                          const uint32_t* eligible_mask_override, float* out, int32_t* idx_out,
+                          float* w_out, uint32_t* mask_out, acm_block_stats* stats,
+                          acm_stream stream);
+
+/* Offload variant (Section 3.4): marks which experts of `layer` are GPU-resident
+ * (resident_mask: HOST words) and registers pinned HOST copies of the full expert tensors
+ * used to load non-resident experts on demand.  The device tensors registered with
+ * acm_set_layer_weights are then read only at resident experts.  NULL mask clears it. */
+acm_status acm_set_resident(acm_ctx* ctx, int layer, const uint32_t* resident_mask,
+                            const void* host_gate_up, const void* host_down);
+
+/* Host->device bytes copied for non-resident experts since the last call with reset != 0. */
+acm_status acm_h2d_bytes(acm_ctx* ctx, uint64_t* bytes_out /*host*/, int reset);
+
+/* Per-launch timing of the expert-FFN kernel with CUDA events on the launching stream.
+ * enable != 0 starts recording (at most `capacity` launches are kept); acm_ffn_time_ms
+ * synchronises those events and returns their summed duration and count (host pointers). */
+acm_status acm_ffn_timing(acm_ctx* ctx, int enable, int capacity);
+acm_status acm_ffn_time_ms(acm_ctx* ctx, float* total_ms, int32_t* launches);
+
+/* Number of kernel launches this context has enqueued since creation (host counter). */
+acm_status acm_launch_count(acm_ctx* ctx, uint64_t* launches_out /*host*/);
+
+/* Synchronises `stream` and returns the sticky device-side status (ACM_OK if none), then clears it. */
+acm_status acm_device_status(acm_ctx* ctx, acm_stream stream);
+
+const char* acm_status_string(acm_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* ACM_H_ */

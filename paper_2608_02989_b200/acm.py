@@ -1,0 +1,271 @@
+"""Python binding of libacm.so (the C ABI in include/acm.h): argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels; torch supplies device memory and
+streams.  There is no CPU fallback: importing works without a GPU (so that the exported
+symbols can be checked), but creating a context needs a B200 and a built library.
+"""
+from __future__ import annotations
+
+import ctypes
+from ctypes import POINTER, byref, c_float, c_int, c_int32, c_uint64, c_void_p
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libacm.so"
+
+OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM, ERR_NONFINITE = range(7)
+F32, BF16 = 0, 1
+W_RENORM_TOPK, W_SOFTMAX_RAW, W_SOFTMAX_MASKED = 0, 1, 2
+DEMAND_TOPK_MASS, DEMAND_FULL_MASS, DEMAND_VOTES = 0, 1, 2
+
+EXPORTS = [
+    "acm_default_select_params", "acm_create", "acm_destroy", "acm_set_layer_weights",
+    "acm_node_weights", "acm_router", "acm_select_eligible", "acm_route_restricted",
+    "acm_expert_ffn", "acm_moe_verify", "acm_set_resident", "acm_h2d_bytes", "acm_ffn_timing",
+    "acm_ffn_time_ms", "acm_launch_count", "acm_device_status", "acm_status_string",
+]
+
+
+class ModelDesc(ctypes.Structure):
+    _fields_ = [("hidden", c_int32), ("n_experts", c_int32), ("top_k", c_int32), ("inter", c_int32),
+                ("n_shared", c_int32), ("max_nodes", c_int32), ("n_layers", c_int32), ("dtype", c_int32),
+                ("weighting", c_int32), ("routed_scale", c_float)]
+
+
+class SelectParams(ctypes.Structure):
+    """acm_select_params; the defaults are the paper's (Eq. 4-6, anchors on, no residency)."""
+    _fields_ = [("demand", c_int32), ("use_anchors", c_int32), ("fixed_budget", c_int32),
+                ("ceil_guard", c_float), ("residency", c_int32), ("max_remove", c_int32)]
+
+    def __init__(self, demand=0, use_anchors=1, fixed_budget=0, ceil_guard=2.0 ** -10, residency=0,
+                 max_remove=128):
+        super().__init__(demand, use_anchors, fixed_budget, ceil_guard, residency, max_remove)
+
+
+class BlockStats(ctypes.Structure):
+    _fields_ = [("n_anchor", c_int32), ("n_er", c_int32), ("n_eligible", c_int32),
+                ("n_eligible_pruned", c_int32), ("n_activated", c_int32), ("n_natural_union", c_int32),
+                ("displaced_aS", c_int32), ("pruned_m", c_int32), ("n_staged", c_int32),
+                ("reserved", c_int32 * 3)]
+    NAMES = ["n_anchor", "n_er", "n_eligible", "n_eligible_pruned", "n_activated", "n_natural_union",
+             "displaced_aS", "pruned_m", "n_staged"]
+
+
+class AcmError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = int(code)
+        super().__init__(f"{where}: {status_string(code)} (acm_status {int(code)})")
+
+
+_lib = None
+
+
+def load_library():
+    """dlopen libacm.so (built in-tree by ``paper_2608_02989_b200.build``); fails loudly if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not LIB_PATH.exists():
+        raise FileNotFoundError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2608_02989_b200.build` "
+            "(there is no fallback path)")
+    lib = ctypes.CDLL(str(LIB_PATH))
+    lib.acm_status_string.restype = ctypes.c_char_p
+    lib.acm_status_string.argtypes = [c_int]
+    lib.acm_create.argtypes = [POINTER(ModelDesc), POINTER(c_void_p)]
+    lib.acm_destroy.argtypes = [c_void_p]
+    lib.acm_set_layer_weights.argtypes = [c_void_p, c_int] + [c_void_p] * 6
+    lib.acm_node_weights.argtypes = [c_void_p, c_int, c_void_p, c_int, c_float, c_int, c_void_p]
+    lib.acm_router.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.acm_select_eligible.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_int,
+                                        POINTER(SelectParams), c_void_p, c_void_p, c_void_p, c_void_p,
+                                        c_void_p, c_void_p, c_void_p]
+    lib.acm_route_restricted.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+    lib.acm_expert_ffn.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.acm_moe_verify.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, POINTER(SelectParams),
+                                   c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.acm_set_resident.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+    lib.acm_h2d_bytes.argtypes = [c_void_p, POINTER(c_uint64), c_int]
+    lib.acm_ffn_timing.argtypes = [c_void_p, c_int, c_int]
+    lib.acm_ffn_time_ms.argtypes = [c_void_p, POINTER(c_float), POINTER(c_int32)]
+    lib.acm_launch_count.argtypes = [c_void_p, POINTER(c_uint64)]
+    lib.acm_device_status.argtypes = [c_void_p, c_void_p]
+    lib.acm_default_select_params.argtypes = [POINTER(SelectParams)]
+    _lib = lib
+    return lib
+
+
+def status_string(code) -> str:
+    return load_library().acm_status_string(int(code)).decode()
+
+
+def _check(code, where):
+    if code != OK:
+        raise AcmError(code, where)
+
+
+def _p(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return c_void_p(stream.cuda_stream)
+
+
+def node_weights(depth, p_table, beta=0.5, width_norm=True) -> torch.Tensor:
+    """acm_node_weights (Eq. 3) on host tensors -> alpha [T] float32 (host)."""
+    depth = depth.to(torch.int32).contiguous().cpu()
+    p_table = p_table.to(torch.float32).contiguous().cpu()
+    alpha = torch.empty(depth.numel(), dtype=torch.float32)
+    _check(load_library().acm_node_weights(_p(depth), depth.numel(), _p(p_table), p_table.numel(),
+                                           float(beta), int(bool(width_norm)), _p(alpha)), "acm_node_weights")
+    return alpha
+
+
+class Context:
+    """Owns one acm_ctx.  Methods mirror the C entry points and take torch CUDA tensors."""
+
+    def __init__(self, hidden, n_experts, top_k, inter, n_shared=0, max_nodes=64, n_layers=1, dtype=BF16,
+                 weighting=W_RENORM_TOPK, routed_scale=1.0):
+        self.lib = load_library()
+        self.desc = ModelDesc(hidden, n_experts, top_k, inter, n_shared, max_nodes, n_layers, dtype, weighting,
+                              routed_scale)
+        self.handle = c_void_p()
+        _check(self.lib.acm_create(byref(self.desc), byref(self.handle)), "acm_create")
+        self._keep = {}
+        self.E, self.k, self.H, self.I = n_experts, top_k, hidden, inter
+        self.words = (n_experts + 31) // 32
+
+    @classmethod
+    def for_config(cls, cfg, n_layers=None, max_nodes=64):
+        return cls(cfg.hidden, cfg.n_experts, cfg.top_k, cfg.inter, cfg.n_shared, max_nodes,
+                   n_layers or cfg.n_layers, F32 if cfg.dtype == "f32" else BF16, cfg.weighting, 1.0)
+
+    def close(self):
+        if self.handle:
+            self.lib.acm_destroy(self.handle)
+            self.handle = c_void_p()
+            self._keep.clear()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ set-up
+    def set_layer_weights(self, layer, w_router, router_bias, gate_up, down, shared_gate_up=None, shared_down=None):
+        self._keep[("w", layer)] = (w_router, router_bias, gate_up, down, shared_gate_up, shared_down)
+        _check(self.lib.acm_set_layer_weights(self.handle, layer, _p(w_router), _p(router_bias), _p(gate_up),
+                                              _p(down), _p(shared_gate_up), _p(shared_down)),
+               "acm_set_layer_weights")
+
+    def set_resident(self, layer, resident_mask, host_gate_up, host_down):
+        """resident_mask: host int32/uint32 words (or None to clear); host_*: pinned host tensors."""
+        if resident_mask is None:
+            _check(self.lib.acm_set_resident(self.handle, layer, None, None, None), "acm_set_resident")
+            self._keep.pop(("r", layer), None)
+            return
+        m = resident_mask.contiguous().cpu()
+        self._keep[("r", layer)] = (m, host_gate_up, host_down)
+        _check(self.lib.acm_set_resident(self.handle, layer, _p(m), _p(host_gate_up), _p(host_down)),
+               "acm_set_resident")
+
+    # ------------------------------------------------------------------ stages
+    def router(self, layer, x, stream=None, want_probs=True, want_topk=True):
+        T = x.shape[0]
+        dev = x.device
+        logits = torch.empty(T, self.E, dtype=torch.float32, device=dev)
+        probs = torch.empty(T, self.E, dtype=torch.float32, device=dev) if want_probs else None
+        nat = torch.empty(T, self.k, dtype=torch.int32, device=dev) if want_topk else None
+        _check(self.lib.acm_router(self.handle, layer, _p(x), T, _p(logits), _p(probs), _p(nat), _stream(stream)),
+               "acm_router")
+        return logits, probs, nat
+
+    def select_eligible(self, probs, nat_idx, alpha, params=None, anchor_nodes=None, resident_mask=None,
+                        stream=None):
+        T = probs.shape[0]
+        dev = probs.device
+        params = params or SelectParams()
+        mask = torch.zeros(self.words, dtype=torch.int32, device=dev)
+        unpruned = torch.zeros(self.words, dtype=torch.int32, device=dev)
+        count = torch.zeros(1, dtype=torch.int32, device=dev)
+        demand = torch.zeros(self.E, dtype=torch.float32, device=dev)
+        stats = torch.zeros(12, dtype=torch.int32, device=dev)
+        n_anchor = 0 if anchor_nodes is None else anchor_nodes.numel()
+        _check(self.lib.acm_select_eligible(self.handle, _p(probs), _p(nat_idx), T, _p(alpha), _p(anchor_nodes),
+                                            n_anchor, byref(params), _p(resident_mask), _p(mask), _p(count),
+                                            _p(demand), _p(unpruned), _p(stats), _stream(stream)),
+               "acm_select_eligible")
+        return {"mask": mask, "unpruned_mask": unpruned, "count": count, "demand": demand, "stats": stats}
+
+    def route_restricted(self, logits, mask, stream=None):
+        T = logits.shape[0]
+        idx = torch.empty(T, self.k, dtype=torch.int32, device=logits.device)
+        w = torch.empty(T, self.k, dtype=torch.float32, device=logits.device)
+        _check(self.lib.acm_route_restricted(self.handle, _p(logits), _p(mask), T, _p(idx), _p(w), _stream(stream)),
+               "acm_route_restricted")
+        return idx, w
+
+    def expert_ffn(self, layer, x, idx, w, out=None, stream=None):
+        T = x.shape[0]
+        if out is None:
+            out = torch.empty(T, self.H, dtype=torch.float32, device=x.device)
+        _check(self.lib.acm_expert_ffn(self.handle, layer, _p(x), T, _p(idx), _p(w), _p(out), _stream(stream)),
+               "acm_expert_ffn")
+        return out
+
+    def moe_verify(self, layer, x, alpha, params=None, mask_override=None, out=None, want=False, stream=None):
+        """Stages 1-4.  want=True also returns idx, w, mask and stats (device tensors)."""
+        T = x.shape[0]
+        dev = x.device
+        if out is None:
+            out = torch.empty(T, self.H, dtype=torch.float32, device=dev)
+        if params is None and mask_override is None:
+            params = SelectParams()
+        idx = w = mask = stats = None
+        if want:
+            idx = torch.empty(T, self.k, dtype=torch.int32, device=dev)
+            w = torch.empty(T, self.k, dtype=torch.float32, device=dev)
+            mask = torch.zeros(self.words, dtype=torch.int32, device=dev)
+            stats = torch.zeros(12, dtype=torch.int32, device=dev)
+        _check(self.lib.acm_moe_verify(self.handle, layer, _p(x), T, _p(alpha),
+                                       byref(params) if params is not None else None, _p(mask_override), _p(out),
+                                       _p(idx), _p(w), _p(mask), _p(stats), _stream(stream)), "acm_moe_verify")
+        if want:
+            return out, idx, w, mask, stats
+        return out
+
+    # ------------------------------------------------------------------ bookkeeping
+    def h2d_bytes(self, reset=False) -> int:
+        v = c_uint64(0)
+        _check(self.lib.acm_h2d_bytes(self.handle, byref(v), int(reset)), "acm_h2d_bytes")
+        return v.value
+
+    def ffn_timing(self, enable, capacity=0):
+        _check(self.lib.acm_ffn_timing(self.handle, int(enable), int(capacity)), "acm_ffn_timing")
+
+    def ffn_time_ms(self):
+        ms, n = c_float(0), c_int32(0)
+        _check(self.lib.acm_ffn_time_ms(self.handle, byref(ms), byref(n)), "acm_ffn_time_ms")
+        return ms.value, n.value
+
+    def launch_count(self) -> int:
+        v = c_uint64(0)
+        _check(self.lib.acm_launch_count(self.handle, byref(v)), "acm_launch_count")
+        return v.value
+
+    def device_status(self, stream=None) -> int:
+        return int(self.lib.acm_device_status(self.handle, _stream(stream)))
+
+    def check_device_status(self, stream=None):
+        _check(self.device_status(stream), "device status")
+
+
+def stats_dict(stats_tensor) -> dict:
+    v = stats_tensor.cpu().tolist()
+    return dict(zip(BlockStats.NAMES, v))

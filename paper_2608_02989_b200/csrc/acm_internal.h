@@ -1,0 +1,135 @@
+// Internal declarations shared by the translation units of libacm (not part of the C ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/acm.h"
+
+namespace acm {
+
+constexpr int kMaxExperts = 128;   // E limit; also the padded length of expert-axis tree sums
+constexpr int kMaxTopK = 8;
+constexpr int kMaxNodes = 64;      // T limit = token columns of one FFN accumulator tile
+constexpr int kMaxShared = 4;
+constexpr int kMaxSlots = kMaxExperts + kMaxShared;   // activated-expert slots of one work list
+constexpr int kMaskWords = 4;
+
+// Work-list entry: which weight tensor an activated expert streams from, and its index there.
+constexpr int kSrcRouted = 0;   // the layer's device tensors, index = expert id
+constexpr int kSrcShared = 1;   // the layer's shared-expert tensors, index = shared id
+constexpr int kSrcStaged = 2;   // the context's staging slots (experts copied from the host)
+__host__ __device__ inline int32_t make_entry(int src, int idx) { return (src << 28) | idx; }
+__host__ __device__ inline int entry_src(int32_t e) { return (e >> 28) & 3; }
+__host__ __device__ inline int entry_idx(int32_t e) { return e & 0x0fffffff; }
+
+// A list of activated experts for the FFN kernel.  Slot a owns row a of `wdense`
+// (combine weight of every node, 0 where the node is not routed there).
+struct WorkList {
+  int32_t n;                      // number of activated experts in this list
+  int32_t n_stage;                // (list 1 only) experts that must be copied from the host first
+  int32_t pad[2];
+  int32_t entry[kMaxSlots];       // make_entry(src, idx)
+  int32_t expert[kMaxSlots];      // routed expert id (or -1 for shared)
+};
+
+// Device workspace of one context (one allocation, carved on the host).
+struct Workspace {
+  float* logits;        // [T,E]
+  float* probs;         // [T,E]
+  int32_t* nat_idx;     // [T,k]
+  int32_t* idx;         // [T,k]
+  float* w;             // [T,k]
+  uint32_t* mask;       // [4] eligible set S'
+  uint32_t* unpruned;   // [4] S
+  int32_t* count;       // [1]
+  float* demand;        // [E]
+  acm_block_stats* stats;
+  WorkList* lists;      // [2]: 0 = resident + shared, 1 = staged
+  float* wdense;        // [2][kMaxSlots][64]
+  void* hbuf;           // [2][kMaxSlots][64][I] bf16 (f32 path: [T][k+ns][I] float)
+  float* frag;          // [grid][128*64] split-K fragments
+  int32_t* frag_flag;   // [grid] epoch of the fragment stored there
+  int32_t* ready;       // [2][kMaxSlots] finished gate/up tiles per activated slot
+  int32_t* status;      // [1] sticky device-side status
+};
+
+struct SelectArgs {
+  const float* probs;
+  const int32_t* nat_idx;
+  const float* alpha;
+  const int32_t* anchor_nodes;
+  int n_anchor_nodes;
+  const uint32_t* resident;      // may be null
+  acm_select_params prm;
+  uint32_t* mask_out;
+  uint32_t* unpruned_out;        // may be null
+  int32_t* count_out;
+  float* demand_out;             // may be null
+  acm_block_stats* stats_out;    // may be null
+};
+
+struct RouteArgs {
+  const float* logits;
+  const uint32_t* mask;
+  int32_t* idx_out;
+  float* w_out;
+  int weighting;
+  float routed_scale;
+  // work-list construction (all null/0 when only the routes are wanted)
+  WorkList* lists;
+  float* wdense;
+  int32_t* ready;
+  const uint32_t* resident;      // non-null: experts outside it go to list 1 (staged)
+  int n_shared;
+  acm_block_stats* stats_out;    // n_activated / n_staged are filled in
+  int32_t* host_stage_list;      // mapped pinned memory: [0] = n_stage, [1..] = expert ids (may be null)
+};
+
+// ---- launchers (routing.cu) -------------------------------------------------------------
+cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
+                                 float* logits, int T, int H, int E, float* zero_buf,
+                                 size_t zero_floats, int32_t* status, cudaStream_t s);
+cudaError_t launch_softmax_topk(const float* logits, float* probs, int32_t* nat_idx, int T, int E,
+                                int k, int32_t* status, cudaStream_t s);
+cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s);
+cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s);
+// softmax/top-k + select (unless mask_override) + route + work lists in ONE single-CTA launch
+cudaError_t launch_fused_select_route(const float* logits, float* probs, int32_t* nat_idx,
+                                      const SelectArgs& sa, const RouteArgs& ra,
+                                      const uint32_t* mask_override, int T, int E, int k,
+                                      int32_t* status, cudaStream_t s);
+cudaError_t launch_routes_to_lists(const int32_t* idx, const float* w, WorkList* lists, float* wdense,
+                                   int32_t* ready, int n_shared, int T, int E, int k, cudaStream_t s);
+
+// ---- launchers (ffn.cu) -----------------------------------------------------------------
+struct FfnMaps {               // TMA descriptors of one layer (bf16 path)
+  CUtensorMap gate_up, down;               // routed experts  [E,2I,H] / [E,H,I]
+  CUtensorMap shared_gate_up, shared_down; // shared experts (copies of the above if none)
+  CUtensorMap staged_gate_up, staged_down; // staging slots   (copies of the above if none)
+};
+struct FfnLaunch {
+  int T, H, I, n_pad;
+  const WorkList* list;
+  const float* wdense;       // [kMaxSlots][64] of this list
+  void* hbuf;                // [kMaxSlots][64][I] bf16 of this list
+  int32_t* ready;            // [kMaxSlots] of this list (zero on entry)
+  float* frag;
+  int32_t* frag_flag;
+  int32_t epoch;
+  float* out;                // [T,H], accumulated into (zeroed by the caller)
+  int32_t* status;
+  int grid;
+  int phase_mask;            // 1 = gate/up, 2 = down, 3 = both in one launch
+};
+cudaError_t ffn_configure();   // one-time function attributes
+size_t ffn_smem_bytes();
+cudaError_t launch_ffn_bf16(const FfnLaunch& p, const FfnMaps& maps, const CUtensorMap& x_map,
+                            const CUtensorMap& h_map, cudaStream_t s);
+cudaError_t launch_ffn_f32(const float* x, const float* gate_up, const float* down,
+                           const float* shared_gate_up, const float* shared_down, int n_shared,
+                           const int32_t* idx, const float* w, float* hbuf, float* out, int T, int H,
+                           int I, int k, cudaStream_t s);
+
+}  // namespace acm

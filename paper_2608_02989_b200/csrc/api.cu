@@ -1,0 +1,620 @@
+// Host side of the C ABI declared in include/acm.h: context and workspace, argument checks,
+// TMA descriptors, launch sequencing, on-demand host->device staging of non-resident experts.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "acm_internal.h"
+
+using namespace acm;
+
+namespace {
+
+struct Layer {
+  const void* w_router = nullptr;
+  const float* bias = nullptr;
+  const void* gate_up = nullptr;
+  const void* down = nullptr;
+  const void* shared_gate_up = nullptr;
+  const void* shared_down = nullptr;
+  FfnMaps maps;
+  bool set = false;
+  bool has_resident = false;
+  const void* host_gate_up = nullptr;   // pinned host copies for on-demand loads
+  const void* host_down = nullptr;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+struct acm_ctx {
+  acm_model_desc desc;
+  int device = 0;
+  int sm_count = 0;
+  void* ws_base = nullptr;
+  Workspace ws;
+  uint32_t* resident_dev = nullptr;      // [n_layers][4]
+  std::vector<Layer> layers;
+  EncodeTiledFn encode = nullptr;
+  int32_t epoch = 0;
+  CUtensorMap h_map[2];
+  int h_map_npad = 0;
+  // staging of non-resident experts
+  void* stage_gate_up = nullptr;
+  void* stage_down = nullptr;
+  CUtensorMap stage_map_gu, stage_map_dn;
+  int32_t* host_stage_list = nullptr;    // pinned + mapped: [0] = count, [1..] = expert ids
+  int32_t* host_stage_list_dev = nullptr;
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_lists = nullptr, ev_copied = nullptr, ev_stage_free = nullptr;
+  bool stage_in_use = false;
+  uint64_t h2d_bytes = 0;
+  // per-launch FFN timing
+  bool timing = false;
+  std::vector<cudaEvent_t> ev_pool;
+  size_t ev_used = 0;
+  uint64_t launches = 0;
+  bool split_phases = false;             // ACM_FFN_SPLIT_PHASES=1 in the environment
+};
+
+namespace {
+
+#define ACM_CUDA(expr)                         \
+  do {                                         \
+    cudaError_t e__ = (expr);                  \
+    if (e__ != cudaSuccess) return ACM_ERR_CUDA; \
+  } while (0)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int mask_words(int E) { return (E + 31) / 32; }
+
+acm_status check_desc(const acm_model_desc& d) {
+  if (d.hidden <= 0 || d.n_experts <= 0 || d.top_k <= 0 || d.inter <= 0 || d.n_shared < 0 || d.max_nodes <= 0 ||
+      d.n_layers <= 0 || d.top_k > d.n_experts)
+    return ACM_ERR_INVALID;
+  if (d.dtype != ACM_F32 && d.dtype != ACM_BF16) return ACM_ERR_INVALID;
+  if (d.weighting < 0 || d.weighting > 2) return ACM_ERR_INVALID;
+  if (!std::isfinite(d.routed_scale)) return ACM_ERR_INVALID;
+  if (d.n_experts > kMaxExperts || d.top_k > kMaxTopK || d.max_nodes > kMaxNodes || d.n_shared > kMaxShared)
+    return ACM_ERR_UNSUPPORTED;
+  if (d.dtype == ACM_BF16 && (d.hidden % 128 != 0 || d.inter % 64 != 0)) return ACM_ERR_UNSUPPORTED;
+  if (d.dtype == ACM_F32 && d.hidden % 32 != 0) return ACM_ERR_UNSUPPORTED;
+  return ACM_OK;
+}
+
+acm_status check_params(const acm_select_params* p) {
+  if (!p) return ACM_ERR_INVALID;
+  if (p->demand < 0 || p->demand > 2 || p->fixed_budget < 0 || p->residency < 0 || p->residency > 2 ||
+      p->max_remove < 0 || !(p->ceil_guard >= 0.0f) || !(p->ceil_guard < 1.0f))
+    return ACM_ERR_INVALID;
+  return ACM_OK;
+}
+
+// 3-D bf16 tensor [d2][d1][d0] (d0 contiguous), box {64, box_rows, 1}, 128-byte swizzle.
+acm_status encode_3d(acm_ctx* c, CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
+                     uint32_t box_rows) {
+  if (reinterpret_cast<uintptr_t>(base) % 16 != 0) return ACM_ERR_INVALID;
+  const cuuint64_t dims[3] = {d0, d1, d2};
+  const cuuint64_t strides[2] = {d0 * 2, d0 * d1 * 2};
+  const cuuint32_t box[3] = {64, box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? ACM_OK : ACM_ERR_CUDA;
+}
+
+acm_status encode_2d(acm_ctx* c, CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint32_t box_rows) {
+  if (reinterpret_cast<uintptr_t>(base) % 16 != 0) return ACM_ERR_INVALID;
+  const cuuint64_t dims[2] = {d0, d1};
+  const cuuint64_t strides[1] = {d0 * 2};
+  const cuuint32_t box[2] = {64, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? ACM_OK : ACM_ERR_CUDA;
+}
+
+acm_status ensure_h_maps(acm_ctx* c, int n_pad) {
+  if (c->h_map_npad == n_pad) return ACM_OK;
+  const size_t list_bytes = static_cast<size_t>(kMaxSlots) * kMaxNodes * c->desc.inter * 2;
+  for (int l = 0; l < 2; ++l) {
+    acm_status st = encode_3d(c, &c->h_map[l], static_cast<char*>(c->ws.hbuf) + l * list_bytes, c->desc.inter,
+                              kMaxNodes, kMaxSlots, n_pad);
+    if (st != ACM_OK) return st;
+  }
+  c->h_map_npad = n_pad;
+  return ACM_OK;
+}
+
+acm_status check_block_args(const acm_ctx* c, int layer, int T, bool need_weights) {
+  if (!c) return ACM_ERR_INVALID;
+  if (layer < 0 || layer >= c->desc.n_layers) return ACM_ERR_INVALID;
+  if (T < 1 || T > c->desc.max_nodes) return ACM_ERR_INVALID;
+  if (need_weights && !c->layers[layer].set) return ACM_ERR_INVALID;
+  return ACM_OK;
+}
+
+// One FFN launch over work list `li` (0 = resident + shared, 1 = staged).
+acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li, float* out, cudaStream_t s) {
+  const acm_model_desc& d = c->desc;
+  const int n_pad = (T + 15) / 16 * 16;
+  acm_status st = ensure_h_maps(c, n_pad);
+  if (st != ACM_OK) return st;
+  CUtensorMap x_map;
+  st = encode_2d(c, &x_map, x, d.hidden, T, n_pad);
+  if (st != ACM_OK) return st;
+  FfnMaps maps = L.maps;
+  if (c->stage_gate_up) {
+    maps.staged_gate_up = c->stage_map_gu;
+    maps.staged_down = c->stage_map_dn;
+  }
+  FfnLaunch p;
+  p.T = T; p.H = d.hidden; p.I = d.inter; p.n_pad = n_pad;
+  p.list = c->ws.lists + li;
+  p.wdense = c->ws.wdense + static_cast<size_t>(li) * kMaxSlots * kMaxNodes;
+  p.hbuf = static_cast<char*>(c->ws.hbuf) + static_cast<size_t>(li) * kMaxSlots * kMaxNodes * d.inter * 2;
+  p.ready = c->ws.ready + li * kMaxSlots;
+  p.frag = c->ws.frag; p.frag_flag = c->ws.frag_flag;
+  p.epoch = ++c->epoch;
+  p.out = out; p.status = c->ws.status;
+  p.grid = c->sm_count;
+  p.phase_mask = 3;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  if (c->timing && c->ev_used + 2 <= c->ev_pool.size()) {
+    e0 = c->ev_pool[c->ev_used];
+    e1 = c->ev_pool[c->ev_used + 1];
+    c->ev_used += 2;
+    ACM_CUDA(cudaEventRecord(e0, s));
+  }
+  if (c->split_phases) {
+    // debugging aid: the two GEMM phases as separate launches (kernel boundary instead of flags)
+    p.phase_mask = 1;
+    ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], s));
+    p.phase_mask = 2;
+    p.epoch = ++c->epoch;
+    c->launches += 1;
+  }
+  ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], s));
+  c->launches += 1;
+  if (e1) ACM_CUDA(cudaEventRecord(e1, s));
+  return ACM_OK;
+}
+
+acm_status ensure_staging(acm_ctx* c) {
+  if (c->stage_gate_up) return ACM_OK;
+  const acm_model_desc& d = c->desc;
+  const size_t gu = static_cast<size_t>(d.n_experts) * 2 * d.inter * d.hidden * 2;
+  const size_t dn = static_cast<size_t>(d.n_experts) * d.hidden * d.inter * 2;
+  if (cudaMalloc(&c->stage_gate_up, gu) != cudaSuccess) return ACM_ERR_NOMEM;
+  if (cudaMalloc(&c->stage_down, dn) != cudaSuccess) return ACM_ERR_NOMEM;
+  acm_status st = encode_3d(c, &c->stage_map_gu, c->stage_gate_up, d.hidden, 2ull * d.inter, d.n_experts, 64);
+  if (st != ACM_OK) return st;
+  st = encode_3d(c, &c->stage_map_dn, c->stage_down, d.inter, d.hidden, d.n_experts, 128);
+  if (st != ACM_OK) return st;
+  ACM_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->host_stage_list), (kMaxExperts + 1) * sizeof(int32_t),
+                         cudaHostAllocMapped));
+  std::memset(c->host_stage_list, 0, (kMaxExperts + 1) * sizeof(int32_t));
+  ACM_CUDA(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->host_stage_list_dev), c->host_stage_list, 0));
+  ACM_CUDA(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+  ACM_CUDA(cudaEventCreateWithFlags(&c->ev_lists, cudaEventDisableTiming));
+  ACM_CUDA(cudaEventCreateWithFlags(&c->ev_copied, cudaEventDisableTiming));
+  ACM_CUDA(cudaEventCreateWithFlags(&c->ev_stage_free, cudaEventDisableTiming));
+  return ACM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+void acm_default_select_params(acm_select_params* p) {
+  if (!p) return;
+  p->demand = ACM_DEMAND_TOPK_MASS;
+  p->use_anchors = 1;
+  p->fixed_budget = 0;
+  p->ceil_guard = 0.0009765625f;
+  p->residency = 0;
+  p->max_remove = kMaxExperts;
+}
+
+const char* acm_status_string(acm_status s) {
+  switch (s) {
+    case ACM_OK: return "ok";
+    case ACM_ERR_INVALID: return "invalid argument";
+    case ACM_ERR_UNSUPPORTED: return "outside the supported limits";
+    case ACM_ERR_CUDA: return "CUDA call failed";
+    case ACM_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    case ACM_ERR_NOMEM: return "out of memory";
+    case ACM_ERR_NONFINITE: return "non-finite router logit";
+  }
+  return "unknown status";
+}
+
+acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
+  if (!desc || !out) return ACM_ERR_INVALID;
+  *out = nullptr;
+  acm_status st = check_desc(*desc);
+  if (st != ACM_OK) return st;
+  acm_ctx* c = new (std::nothrow) acm_ctx();
+  if (!c) return ACM_ERR_NOMEM;
+  c->desc = *desc;
+  c->layers.resize(desc->n_layers);
+  const char* split = std::getenv("ACM_FFN_SPLIT_PHASES");
+  c->split_phases = split && split[0] == '1';
+  auto fail = [&](acm_status s) {
+    acm_destroy(c);
+    return s;
+  };
+  if (cudaGetDevice(&c->device) != cudaSuccess) return fail(ACM_ERR_CUDA);
+  if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess)
+    return fail(ACM_ERR_CUDA);
+  if (desc->dtype == ACM_BF16) {
+    int major = 0;
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, c->device);
+    if (major != 10) return fail(ACM_ERR_UNSUPPORTED);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess)
+      return fail(ACM_ERR_CUDA);
+    c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    if (ffn_configure() != cudaSuccess) return fail(ACM_ERR_CUDA);
+  }
+
+  const int Tm = kMaxNodes, E = desc->n_experts, k = desc->top_k, I = desc->inter;
+  size_t off = 0;
+  auto carve = [&](size_t bytes) {
+    const size_t at = off;
+    off = align_up(off + bytes, 1024);
+    return at;
+  };
+  const size_t o_logits = carve(sizeof(float) * Tm * E), o_probs = carve(sizeof(float) * Tm * E);
+  const size_t o_nat = carve(sizeof(int32_t) * Tm * k), o_idx = carve(sizeof(int32_t) * Tm * k);
+  const size_t o_w = carve(sizeof(float) * Tm * k), o_mask = carve(16), o_unpr = carve(16), o_cnt = carve(16);
+  const size_t o_dem = carve(sizeof(float) * kMaxExperts), o_stats = carve(sizeof(acm_block_stats));
+  const size_t o_lists = carve(sizeof(WorkList) * 2);
+  const size_t o_wd = carve(sizeof(float) * 2 * kMaxSlots * kMaxNodes);
+  const size_t hbuf_bf16 = static_cast<size_t>(2) * kMaxSlots * kMaxNodes * I * 2;
+  const size_t hbuf_f32 = static_cast<size_t>(Tm) * (k + desc->n_shared) * I * 4;
+  const size_t o_h = carve(hbuf_bf16 > hbuf_f32 ? hbuf_bf16 : hbuf_f32);
+  const size_t o_frag = carve(sizeof(float) * static_cast<size_t>(c->sm_count) * 128 * kMaxNodes);
+  const size_t o_flag = carve(sizeof(int32_t) * c->sm_count);
+  const size_t o_ready = carve(sizeof(int32_t) * 2 * kMaxSlots);
+  const size_t o_status = carve(16);
+  const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
+  if (cudaMalloc(&c->ws_base, off) != cudaSuccess) return fail(ACM_ERR_NOMEM);
+  if (cudaMemset(c->ws_base, 0, off) != cudaSuccess) return fail(ACM_ERR_CUDA);
+  char* b = static_cast<char*>(c->ws_base);
+  c->ws.logits = reinterpret_cast<float*>(b + o_logits);
+  c->ws.probs = reinterpret_cast<float*>(b + o_probs);
+  c->ws.nat_idx = reinterpret_cast<int32_t*>(b + o_nat);
+  c->ws.idx = reinterpret_cast<int32_t*>(b + o_idx);
+  c->ws.w = reinterpret_cast<float*>(b + o_w);
+  c->ws.mask = reinterpret_cast<uint32_t*>(b + o_mask);
+  c->ws.unpruned = reinterpret_cast<uint32_t*>(b + o_unpr);
+  c->ws.count = reinterpret_cast<int32_t*>(b + o_cnt);
+  c->ws.demand = reinterpret_cast<float*>(b + o_dem);
+  c->ws.stats = reinterpret_cast<acm_block_stats*>(b + o_stats);
+  c->ws.lists = reinterpret_cast<WorkList*>(b + o_lists);
+  c->ws.wdense = reinterpret_cast<float*>(b + o_wd);
+  c->ws.hbuf = b + o_h;
+  c->ws.frag = reinterpret_cast<float*>(b + o_frag);
+  c->ws.frag_flag = reinterpret_cast<int32_t*>(b + o_flag);
+  c->ws.ready = reinterpret_cast<int32_t*>(b + o_ready);
+  c->ws.status = reinterpret_cast<int32_t*>(b + o_status);
+  c->resident_dev = reinterpret_cast<uint32_t*>(b + o_res);
+  *out = c;
+  return ACM_OK;
+}
+
+acm_status acm_destroy(acm_ctx* c) {
+  if (!c) return ACM_ERR_INVALID;
+  cudaDeviceSynchronize();
+  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
+  if (c->ev_lists) cudaEventDestroy(c->ev_lists);
+  if (c->ev_copied) cudaEventDestroy(c->ev_copied);
+  if (c->ev_stage_free) cudaEventDestroy(c->ev_stage_free);
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  if (c->host_stage_list) cudaFreeHost(c->host_stage_list);
+  if (c->stage_gate_up) cudaFree(c->stage_gate_up);
+  if (c->stage_down) cudaFree(c->stage_down);
+  if (c->ws_base) cudaFree(c->ws_base);
+  delete c;
+  return ACM_OK;
+}
+
+acm_status acm_set_layer_weights(acm_ctx* c, int layer, const void* w_router, const float* router_bias,
+                                 const void* w_gate_up, const void* w_down, const void* shared_gate_up,
+                                 const void* shared_down) {
+  if (!c || layer < 0 || layer >= c->desc.n_layers || !w_router) return ACM_ERR_INVALID;
+  const acm_model_desc& d = c->desc;
+  if ((w_gate_up == nullptr) != (w_down == nullptr)) return ACM_ERR_INVALID;
+  if (d.n_shared > 0 && w_gate_up && (!shared_gate_up || !shared_down)) return ACM_ERR_INVALID;
+  if (reinterpret_cast<uintptr_t>(w_router) % 16 != 0) return ACM_ERR_INVALID;
+  Layer L;
+  L.w_router = w_router; L.bias = router_bias; L.gate_up = w_gate_up; L.down = w_down;
+  L.shared_gate_up = d.n_shared ? shared_gate_up : nullptr;
+  L.shared_down = d.n_shared ? shared_down : nullptr;
+  if (d.dtype == ACM_BF16 && w_gate_up) {
+    acm_status st = encode_3d(c, &L.maps.gate_up, w_gate_up, d.hidden, 2ull * d.inter, d.n_experts, 64);
+    if (st != ACM_OK) return st;
+    st = encode_3d(c, &L.maps.down, w_down, d.inter, d.hidden, d.n_experts, 128);
+    if (st != ACM_OK) return st;
+    L.maps.shared_gate_up = L.maps.gate_up;
+    L.maps.shared_down = L.maps.down;
+    if (d.n_shared) {
+      st = encode_3d(c, &L.maps.shared_gate_up, shared_gate_up, d.hidden, 2ull * d.inter, d.n_shared, 64);
+      if (st != ACM_OK) return st;
+      st = encode_3d(c, &L.maps.shared_down, shared_down, d.inter, d.hidden, d.n_shared, 128);
+      if (st != ACM_OK) return st;
+    }
+    L.maps.staged_gate_up = L.maps.gate_up;
+    L.maps.staged_down = L.maps.down;
+  }
+  L.set = true;
+  c->layers[layer] = L;
+  return ACM_OK;
+}
+
+acm_status acm_node_weights(const int32_t* depth, int T, const float* p_table, int n_depths, float beta,
+                            int width_norm, float* alpha_out) {
+  if (!depth || !p_table || !alpha_out || T < 1 || n_depths < 1) return ACM_ERR_INVALID;
+  std::vector<int> width(n_depths, 0);
+  for (int t = 0; t < T; ++t) {
+    if (depth[t] < 0 || depth[t] >= n_depths) return ACM_ERR_INVALID;
+    ++width[depth[t]];
+  }
+  for (int t = 0; t < T; ++t) {
+    double a = std::pow(static_cast<double>(p_table[depth[t]]), static_cast<double>(beta));
+    if (width_norm) a /= std::sqrt(static_cast<double>(width[depth[t]]));
+    alpha_out[t] = static_cast<float>(a);
+  }
+  return ACM_OK;
+}
+
+acm_status acm_router(acm_ctx* c, int layer, const void* x, int T, float* logits, float* probs,
+                      int32_t* nat_idx, acm_stream stream) {
+  acm_status st = check_block_args(c, layer, T, true);
+  if (st != ACM_OK) return st;
+  if (!x || !logits || reinterpret_cast<uintptr_t>(x) % 16 != 0) return ACM_ERR_INVALID;
+  const acm_model_desc& d = c->desc;
+  const Layer& L = c->layers[layer];
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, logits, T, d.hidden, d.n_experts, nullptr, 0,
+                                c->ws.status, s));
+  c->launches += 1;
+  if (probs || nat_idx) {
+    ACM_CUDA(launch_softmax_topk(logits, probs, nat_idx, T, d.n_experts, d.top_k, c->ws.status, s));
+    c->launches += 1;
+  }
+  return ACM_OK;
+}
+
+acm_status acm_select_eligible(acm_ctx* c, const float* probs, const int32_t* nat_idx, int T, const float* alpha,
+                               const int32_t* anchor_nodes, int n_anchor_nodes, const acm_select_params* params,
+                               const uint32_t* resident_mask, uint32_t* eligible_mask, int32_t* eligible_count,
+                               float* demand, uint32_t* unpruned_mask, acm_block_stats* stats, acm_stream stream) {
+  if (!c || T < 1 || T > c->desc.max_nodes) return ACM_ERR_INVALID;
+  if (!probs || !nat_idx || !alpha || !eligible_mask || !eligible_count) return ACM_ERR_INVALID;
+  acm_status st = check_params(params);
+  if (st != ACM_OK) return st;
+  if (params->residency != 0 && !resident_mask) return ACM_ERR_INVALID;
+  if (anchor_nodes && (n_anchor_nodes < 1 || n_anchor_nodes > kMaxNodes)) return ACM_ERR_INVALID;
+  SelectArgs a;
+  a.probs = probs; a.nat_idx = nat_idx; a.alpha = alpha; a.anchor_nodes = anchor_nodes;
+  a.n_anchor_nodes = n_anchor_nodes; a.resident = params->residency ? resident_mask : nullptr; a.prm = *params;
+  a.mask_out = eligible_mask; a.unpruned_out = unpruned_mask; a.count_out = eligible_count;
+  a.demand_out = demand; a.stats_out = stats;
+  ACM_CUDA(launch_select(a, T, c->desc.n_experts, c->desc.top_k, static_cast<cudaStream_t>(stream)));
+  c->launches += 1;
+  return ACM_OK;
+}
+
+acm_status acm_route_restricted(acm_ctx* c, const float* logits, const uint32_t* eligible_mask, int T,
+                                int32_t* idx, float* w, acm_stream stream) {
+  if (!c || T < 1 || T > c->desc.max_nodes) return ACM_ERR_INVALID;
+  if (!logits || !eligible_mask || !idx || !w) return ACM_ERR_INVALID;
+  RouteArgs a = {};
+  a.logits = logits; a.mask = eligible_mask; a.idx_out = idx; a.w_out = w;
+  a.weighting = c->desc.weighting; a.routed_scale = c->desc.routed_scale;
+  ACM_CUDA(launch_route(a, T, c->desc.n_experts, c->desc.top_k, static_cast<cudaStream_t>(stream)));
+  c->launches += 1;
+  return ACM_OK;
+}
+
+acm_status acm_expert_ffn(acm_ctx* c, int layer, const void* x, int T, const int32_t* idx, const float* w,
+                          float* out, acm_stream stream) {
+  acm_status st = check_block_args(c, layer, T, true);
+  if (st != ACM_OK) return st;
+  const Layer& L = c->layers[layer];
+  if (!x || !idx || !w || !out || !L.gate_up) return ACM_ERR_INVALID;
+  if (reinterpret_cast<uintptr_t>(x) % 16 != 0 || reinterpret_cast<uintptr_t>(out) % 16 != 0) return ACM_ERR_INVALID;
+  if (L.has_resident) return ACM_ERR_UNSUPPORTED;   // staging is driven by acm_moe_verify
+  const acm_model_desc& d = c->desc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (d.dtype == ACM_F32) {
+    ACM_CUDA(launch_ffn_f32(static_cast<const float*>(x), static_cast<const float*>(L.gate_up),
+                            static_cast<const float*>(L.down), static_cast<const float*>(L.shared_gate_up),
+                            static_cast<const float*>(L.shared_down), d.n_shared, idx, w,
+                            static_cast<float*>(c->ws.hbuf), out, T, d.hidden, d.inter, d.top_k, s));
+    c->launches += 2;
+    return ACM_OK;
+  }
+  ACM_CUDA(cudaMemsetAsync(out, 0, sizeof(float) * static_cast<size_t>(T) * d.hidden, s));
+  ACM_CUDA(launch_routes_to_lists(idx, w, c->ws.lists, c->ws.wdense, c->ws.ready, d.n_shared, T, d.n_experts,
+                                  d.top_k, s));
+  c->launches += 1;
+  return run_ffn_list(c, L, x, T, 0, out, s);
+}
+
+acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const float* alpha,
+                          const acm_select_params* params, const uint32_t* eligible_mask_override, float* out,
+                          int32_t* idx_out, float* w_out, uint32_t* mask_out, acm_block_stats* stats,
+                          acm_stream stream) {
+  acm_status st = check_block_args(c, layer, T, true);
+  if (st != ACM_OK) return st;
+  const Layer& L = c->layers[layer];
+  if (!x || !out || !L.gate_up) return ACM_ERR_INVALID;
+  if (reinterpret_cast<uintptr_t>(x) % 16 != 0 || reinterpret_cast<uintptr_t>(out) % 16 != 0) return ACM_ERR_INVALID;
+  acm_select_params prm;
+  if (eligible_mask_override) {
+    acm_default_select_params(&prm);
+  } else {
+    if (!alpha) return ACM_ERR_INVALID;
+    st = check_params(params);
+    if (st != ACM_OK) return st;
+    prm = *params;
+    if (prm.residency != 0 && !L.has_resident) return ACM_ERR_INVALID;
+  }
+  const acm_model_desc& d = c->desc;
+  const int E = d.n_experts, k = d.top_k;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const bool f32 = d.dtype == ACM_F32;
+  uint32_t* res_dev = L.has_resident ? c->resident_dev + 4 * layer : nullptr;
+
+  // stage 1a (also clears the output the FFN accumulates into)
+  ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
+                                f32 ? 0 : static_cast<size_t>(T) * d.hidden, c->ws.status, s));
+  // stages 1b-3 and the FFN work lists, one single-CTA launch
+  SelectArgs sa;
+  sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
+  sa.n_anchor_nodes = 0; sa.resident = prm.residency ? res_dev : nullptr; sa.prm = prm;
+  sa.mask_out = c->ws.mask; sa.unpruned_out = c->ws.unpruned; sa.count_out = c->ws.count;
+  sa.demand_out = c->ws.demand; sa.stats_out = c->ws.stats;
+  RouteArgs ra = {};
+  ra.logits = c->ws.logits; ra.mask = c->ws.mask; ra.idx_out = c->ws.idx; ra.w_out = c->ws.w;
+  ra.weighting = d.weighting; ra.routed_scale = d.routed_scale;
+  ra.lists = c->ws.lists; ra.wdense = c->ws.wdense; ra.ready = c->ws.ready; ra.resident = res_dev;
+  ra.n_shared = d.n_shared; ra.host_stage_list = L.has_resident ? c->host_stage_list_dev : nullptr;
+  ra.stats_out = c->ws.stats;
+  ACM_CUDA(launch_fused_select_route(c->ws.logits, c->ws.probs, c->ws.nat_idx, sa, ra, eligible_mask_override, T, E,
+                                     k, c->ws.status, s));
+  c->launches += 2;
+
+  if (f32) {
+    ACM_CUDA(launch_ffn_f32(static_cast<const float*>(x), static_cast<const float*>(L.gate_up),
+                            static_cast<const float*>(L.down), static_cast<const float*>(L.shared_gate_up),
+                            static_cast<const float*>(L.shared_down), d.n_shared, c->ws.idx, c->ws.w,
+                            static_cast<float*>(c->ws.hbuf), out, T, d.hidden, d.inter, k, s));
+    c->launches += 2;
+  } else if (!L.has_resident) {
+    st = run_ffn_list(c, L, x, T, 0, out, s);
+    if (st != ACM_OK) return st;
+  } else {
+    // resident + shared experts run at once; the others are copied in from pinned host memory first
+    ACM_CUDA(cudaEventRecord(c->ev_lists, s));
+    st = run_ffn_list(c, L, x, T, 0, out, s);
+    if (st != ACM_OK) return st;
+    ACM_CUDA(cudaEventSynchronize(c->ev_lists));
+    const int n_stage = c->host_stage_list[0];
+    if (n_stage < 0 || n_stage > E) return ACM_ERR_CUDA;
+    if (n_stage > 0) {
+      const size_t gu = static_cast<size_t>(2) * d.inter * d.hidden * 2, dn = static_cast<size_t>(d.hidden) * d.inter * 2;
+      if (c->stage_in_use) ACM_CUDA(cudaStreamWaitEvent(c->copy_stream, c->ev_stage_free, 0));
+      for (int i = 0; i < n_stage; ++i) {
+        const int e = c->host_stage_list[1 + i];
+        if (e < 0 || e >= E) return ACM_ERR_CUDA;
+        ACM_CUDA(cudaMemcpyAsync(static_cast<char*>(c->stage_gate_up) + i * gu,
+                                 static_cast<const char*>(L.host_gate_up) + e * gu, gu, cudaMemcpyHostToDevice,
+                                 c->copy_stream));
+        ACM_CUDA(cudaMemcpyAsync(static_cast<char*>(c->stage_down) + i * dn,
+                                 static_cast<const char*>(L.host_down) + e * dn, dn, cudaMemcpyHostToDevice,
+                                 c->copy_stream));
+        c->h2d_bytes += gu + dn;
+      }
+      ACM_CUDA(cudaEventRecord(c->ev_copied, c->copy_stream));
+      ACM_CUDA(cudaStreamWaitEvent(s, c->ev_copied, 0));
+      st = run_ffn_list(c, L, x, T, 1, out, s);
+      if (st != ACM_OK) return st;
+      ACM_CUDA(cudaEventRecord(c->ev_stage_free, s));
+      c->stage_in_use = true;
+    }
+  }
+
+  const size_t tk = static_cast<size_t>(T) * k;
+  if (idx_out) ACM_CUDA(cudaMemcpyAsync(idx_out, c->ws.idx, sizeof(int32_t) * tk, cudaMemcpyDeviceToDevice, s));
+  if (w_out) ACM_CUDA(cudaMemcpyAsync(w_out, c->ws.w, sizeof(float) * tk, cudaMemcpyDeviceToDevice, s));
+  if (mask_out)
+    ACM_CUDA(cudaMemcpyAsync(mask_out, c->ws.mask, sizeof(uint32_t) * mask_words(E), cudaMemcpyDeviceToDevice, s));
+  if (stats) ACM_CUDA(cudaMemcpyAsync(stats, c->ws.stats, sizeof(acm_block_stats), cudaMemcpyDefault, s));
+  return ACM_OK;
+}
+
+acm_status acm_set_resident(acm_ctx* c, int layer, const uint32_t* resident_mask, const void* host_gate_up,
+                            const void* host_down) {
+  if (!c || layer < 0 || layer >= c->desc.n_layers) return ACM_ERR_INVALID;
+  Layer& L = c->layers[layer];
+  if (!resident_mask) {
+    L.has_resident = false;
+    L.host_gate_up = L.host_down = nullptr;
+    return ACM_OK;
+  }
+  if (c->desc.dtype != ACM_BF16) return ACM_ERR_UNSUPPORTED;
+  if (!host_gate_up || !host_down) return ACM_ERR_INVALID;
+  acm_status st = ensure_staging(c);
+  if (st != ACM_OK) return st;
+  uint32_t words[4] = {0, 0, 0, 0};
+  for (int w = 0; w < mask_words(c->desc.n_experts); ++w) words[w] = resident_mask[w];
+  ACM_CUDA(cudaMemcpy(c->resident_dev + 4 * layer, words, sizeof words, cudaMemcpyHostToDevice));
+  L.has_resident = true;
+  L.host_gate_up = host_gate_up;
+  L.host_down = host_down;
+  return ACM_OK;
+}
+
+acm_status acm_h2d_bytes(acm_ctx* c, uint64_t* bytes_out, int reset) {
+  if (!c || !bytes_out) return ACM_ERR_INVALID;
+  *bytes_out = c->h2d_bytes;
+  if (reset) c->h2d_bytes = 0;
+  return ACM_OK;
+}
+
+acm_status acm_ffn_timing(acm_ctx* c, int enable, int capacity) {
+  if (!c || capacity < 0) return ACM_ERR_INVALID;
+  c->timing = enable != 0;
+  c->ev_used = 0;
+  while (c->timing && c->ev_pool.size() < static_cast<size_t>(2) * capacity) {
+    cudaEvent_t e;
+    ACM_CUDA(cudaEventCreate(&e));
+    c->ev_pool.push_back(e);
+  }
+  return ACM_OK;
+}
+
+acm_status acm_ffn_time_ms(acm_ctx* c, float* total_ms, int32_t* launches) {
+  if (!c || !total_ms || !launches) return ACM_ERR_INVALID;
+  float total = 0.f;
+  for (size_t i = 0; i + 1 < c->ev_used; i += 2) {
+    ACM_CUDA(cudaEventSynchronize(c->ev_pool[i + 1]));
+    float ms = 0.f;
+    ACM_CUDA(cudaEventElapsedTime(&ms, c->ev_pool[i], c->ev_pool[i + 1]));
+    total += ms;
+  }
+  *total_ms = total;
+  *launches = static_cast<int32_t>(c->ev_used / 2);
+  return ACM_OK;
+}
+
+acm_status acm_launch_count(acm_ctx* c, uint64_t* launches_out) {
+  if (!c || !launches_out) return ACM_ERR_INVALID;
+  *launches_out = c->launches;
+  return ACM_OK;
+}
+
+acm_status acm_device_status(acm_ctx* c, acm_stream stream) {
+  if (!c) return ACM_ERR_INVALID;
+  ACM_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+  int32_t v = 0;
+  ACM_CUDA(cudaMemcpy(&v, c->ws.status, sizeof v, cudaMemcpyDeviceToHost));
+  if (v != 0) ACM_CUDA(cudaMemset(c->ws.status, 0, sizeof v));
+  return static_cast<acm_status>(v);
+}
+
+}  // extern "C"

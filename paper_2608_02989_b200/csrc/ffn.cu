@@ -1,0 +1,598 @@
+// Stage 4: grouped SwiGLU expert FFN over the activated experts with weighted combine,
+//   y_t = sum_e w_{t,e} * W_down_e ( silu(W_gate_e x_t) * (W_up_e x_t) ),
+// the step whose cost is the number of distinct expert weights touched (Section 1; Section 3.1).
+//
+// bf16 path (sm_100a): one persistent kernel, one CTA per SM, warp-specialised:
+//   warp 0      TMA producer: streams weight tiles (128 rows x 64 K, 128-byte swizzle) and the
+//               matching activation chunk into an 8-stage shared-memory ring
+//   warp 1      issues tcgen05.mma (M=128 weight rows, N=node columns, fp32 accumulators in TMEM)
+//   warps 2..5  epilogue: tcgen05.ld, SwiGLU / combine, stores
+// The weights are the M operand ("swap-AB"): every activated expert's weights are read from HBM
+// exactly once for all nodes of the block.  Both GEMMs are cut into equal contiguous ranges of
+// (tile, K-chunk) units, one range per CTA, so every SM streams the same number of bytes:
+//   phase 1  tile = 64 gate rows + the 64 matching up rows of one expert, K = hidden;
+//            a tile cut across CTAs is summed through a global fragment buffer by the CTA that
+//            owns its first chunk, which then applies w * silu(g) * u and writes the activation
+//   phase 2  tile = 128 output rows, K = (activated expert, intermediate) concatenated;
+//            partial tiles are accumulated into the output with reductions in L2.
+// Phase 2 reads the activations written by other CTAs in phase 1; per-expert completion counters
+// order the two.  Every wait is bounded; on expiry the kernel raises a status and drains.
+//
+// f32 path: plain FMA kernels (the fp32 toy configuration is a few MFLOP).
+#include <cuda_bf16.h>
+
+#include "acm_internal.h"
+
+namespace acm {
+namespace {
+
+constexpr int kStages = 8;
+constexpr int kBK = 64;                                  // K elements per stage (one 128-byte swizzle row)
+constexpr int kTileM = 128;
+constexpr int kABytes = kTileM * kBK * 2;                // 16 KB weight tile
+constexpr int kBBytesMax = kMaxNodes * kBK * 2;          // 8 KB activation chunk
+constexpr int kStageBytes = kABytes + kBBytesMax;
+constexpr int kExBytes = 64 * kMaxNodes * 4;             // up-projection exchange buffer
+constexpr int kAccCols = kMaxNodes;                      // TMEM columns per accumulator
+constexpr int kTmemCols = 128;                           // two accumulators
+constexpr int kThreads = 192;
+constexpr int kFragFloats = kTileM * kMaxNodes;
+constexpr unsigned long long kTimeoutNs = 1000ull * 1000ull * 1000ull;
+
+struct __align__(8) Barriers {
+  unsigned long long full[kStages];
+  unsigned long long empty[kStages];
+  unsigned long long tfull[2];
+  unsigned long long tempty[2];
+  unsigned long long drained;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + kExBytes + sizeof(Barriers);
+
+// ---------------------------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ unsigned long long global_timer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false (after raising the status once) if the limit ran out or the CTA
+// has already given up; callers then skip the rest of their work.
+__device__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (*abort_flag) return false;
+  for (int i = 0; i < 1024; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer();
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_timer() - t0 > kTimeoutNs) {
+      *abort_flag = 1;
+      atomicCAS(status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ int ld_acquire(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(int32_t* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// Bounded wait until *p >= target (p written by other CTAs with release semantics).
+__device__ bool flag_wait_ge(const int32_t* p, int target, volatile int* abort_flag, int32_t* status) {
+  if (*abort_flag) return false;
+  for (int i = 0; i < 256; ++i)
+    if (ld_acquire(p) >= target) return true;
+  const unsigned long long t0 = global_timer();
+  for (;;) {
+    for (int i = 0; i < 16; ++i) {
+      if (ld_acquire(p) >= target) return true;
+      __nanosleep(64);
+    }
+    if (*abort_flag) return false;
+    if (global_timer() - t0 > kTimeoutNs) {
+      *abort_flag = 1;
+      atomicCAS(status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// Barrier over the 128 epilogue threads that also ANDs a predicate, so that all of them take the
+// same decision after a bounded wait (a thread that left alone would strand the others at a barrier).
+__device__ __forceinline__ bool epi_vote_all(bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 p, %1, 0;\n\t"
+      "bar.red.and.pred q, 1, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}\n"
+      : "=r"(r) : "r"(static_cast<uint32_t>(pred)) : "memory");
+  return r != 0;
+}
+
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3, %4}], [%5], %6;"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, rows of 128 bytes, 128-byte swizzle, groups of
+// 8 rows 1024 bytes apart.  The tile base is 1024-byte aligned; stepping K by 16 elements adds 32 bytes.
+__device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);       // start address
+  d |= static_cast<uint64_t>(1) << 16;                           // leading byte offset (unused here)
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;                   // stride byte offset
+  d |= static_cast<uint64_t>(1) << 46;                           // descriptor version
+  d |= static_cast<uint64_t>(2) << 61;                           // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
+}
+
+// Equal contiguous ranges of (tile, K-chunk) units: CTA c owns [c*U/G, (c+1)*U/G).
+struct Sched {
+  long long u, u_end;
+  int kc;
+  __device__ Sched(int cta, int grid, long long tiles, int chunks_per_tile) : kc(chunks_per_tile) {
+    const long long total = tiles * chunks_per_tile;
+    u = total * cta / grid;
+    u_end = total * (cta + 1) / grid;
+  }
+  __device__ bool next(int& tile, int& k0, int& k1) {
+    if (u >= u_end) return false;
+    tile = static_cast<int>(u / kc);
+    k0 = static_cast<int>(u % kc);
+    const long long rem = u_end - u;
+    k1 = static_cast<int>(rem < kc - k0 ? k0 + rem : kc);
+    u += k1 - k0;
+    return true;
+  }
+};
+
+struct FfnArgs {
+  int T, H, I, n_pad;
+  const WorkList* list;
+  const float* wdense;
+  __nv_bfloat16* hbuf;
+  int32_t* ready;
+  float* frag;
+  int32_t* frag_flag;
+  int32_t epoch;
+  float* out;
+  int32_t* status;
+  int phase_mask;
+};
+
+__device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMap* routed, const CUtensorMap* shared,
+                                                       const CUtensorMap* staged) {
+  return src == kSrcRouted ? routed : src == kSrcShared ? shared : staged;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtensorMap x_map,
+           const __grid_constant__ CUtensorMap h_map, const FfnArgs p) {
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  unsigned char* stage_base = smem;
+  float* ex = reinterpret_cast<float*>(smem + static_cast<size_t>(kStages) * kStageBytes);
+  Barriers* bars = reinterpret_cast<Barriers*>(smem + static_cast<size_t>(kStages) * kStageBytes + kExBytes);
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cta = blockIdx.x, G = gridDim.x;
+  const int n_act = p.list->n;
+  const int tpe = p.I / 64;          // gate/up tiles per expert = K-chunks per expert in phase 2
+  const int kc1 = p.H / kBK;         // K-chunks of a phase-1 tile
+  const int h_tiles = p.H / kTileM;  // output tiles of phase 2
+  const int kc2 = n_act * tpe;       // K-chunks of a phase-2 tile
+  const uint32_t b_bytes = static_cast<uint32_t>(p.n_pad) * kBK * 2;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&bars->full[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->tfull[b]), 1);
+      mbar_init(smem_u32(&bars->tempty[b]), 128);
+    }
+    mbar_init(smem_u32(&bars->drained), 1);
+    bars->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 0 && lane == 0) {
+    prefetch_tensormap(&maps.gate_up);
+    prefetch_tensormap(&maps.down);
+    prefetch_tensormap(&x_map);
+    prefetch_tensormap(&h_map);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      uint32_t it = 0;
+      bool ok = true;
+      if (p.phase_mask & 1) {
+        Sched s1(cta, G, static_cast<long long>(n_act) * tpe, kc1);
+        int tile, k0, k1;
+        while (ok && s1.next(tile, k0, k1)) {
+          const int a = tile / tpe, ti = tile % tpe;
+          const int32_t ent = p.list->entry[a];
+          const CUtensorMap* gu = pick_map(entry_src(ent), &maps.gate_up, &maps.shared_gate_up, &maps.staged_gate_up);
+          const int eidx = entry_idx(ent);
+          for (int kc = k0; kc < k1; ++kc, ++it) {
+            const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+            if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
+            const uint32_t full = smem_u32(&bars->full[s]);
+            const uint32_t sa = smem_u32(stage_base + static_cast<size_t>(s) * kStageBytes);
+            mbar_expect_tx(full, kABytes + b_bytes);
+            tma_load_3d(sa, gu, full, kc * kBK, ti * 64, eidx, pol_w);                 // 64 gate rows
+            tma_load_3d(sa + kABytes / 2, gu, full, kc * kBK, p.I + ti * 64, eidx, pol_w);   // 64 up rows
+            tma_load_2d(sa + kABytes, &x_map, full, kc * kBK, 0, pol_x);
+          }
+        }
+      }
+      if (p.phase_mask & 2) {
+        Sched s2(cta, G, h_tiles, kc2);
+        int ht, k0, k1, ready_a = -1;
+        while (ok && s2.next(ht, k0, k1)) {
+          for (int kc = k0; kc < k1; ++kc, ++it) {
+            const int a = kc / tpe, ic = kc % tpe;
+            const int32_t ent = p.list->entry[a];
+            const CUtensorMap* dn = pick_map(entry_src(ent), &maps.down, &maps.shared_down, &maps.staged_down);
+            const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+            if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
+            const uint32_t full = smem_u32(&bars->full[s]);
+            const uint32_t sa = smem_u32(stage_base + static_cast<size_t>(s) * kStageBytes);
+            mbar_expect_tx(full, kABytes + b_bytes);
+            tma_load_3d(sa, dn, full, ic * kBK, ht * kTileM, entry_idx(ent), pol_w);
+            if (a != ready_a) {   // activations of expert slot a are complete once all its tiles are counted
+              if (!(ok = flag_wait_ge(&p.ready[a], tpe, abort_flag, p.status))) break;
+              fence_proxy_async();
+              ready_a = a;
+            }
+            tma_load_3d(sa + kABytes, &h_map, full, ic * kBK, 0, a, pol_x);
+          }
+        }
+      }
+      if (!ok) {
+        // giving up: let copies already in flight land before the CTA exits
+        const unsigned long long t0 = global_timer();
+        while (global_timer() - t0 < 200000ull) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc(p.n_pad);
+      uint32_t it = 0, f = 0;
+      bool ok = true;
+      for (int phase = 1; phase <= 2 && ok; ++phase) {
+        if (!(p.phase_mask & phase)) continue;
+        Sched sc = phase == 1 ? Sched(cta, G, static_cast<long long>(n_act) * tpe, kc1) : Sched(cta, G, h_tiles, kc2);
+        int tile, k0, k1;
+        while (ok && sc.next(tile, k0, k1)) {
+          const uint32_t b = f & 1u;
+          if (!(ok = mbar_wait(smem_u32(&bars->tempty[b]), ((f >> 1) & 1u) ^ 1u, abort_flag, p.status))) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + b * kAccCols;
+          for (int kc = k0; kc < k1; ++kc, ++it) {
+            const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+            if (!(ok = mbar_wait(smem_u32(&bars->full[s]), par, abort_flag, p.status))) break;
+            tc_fence_after();
+            const uint32_t sa = smem_u32(stage_base + static_cast<size_t>(s) * kStageBytes);
+            const uint64_t da = umma_smem_desc(sa), db = umma_smem_desc(sa + kABytes);
+#pragma unroll
+            for (int kk = 0; kk < kBK / 16; ++kk)
+              umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kc > k0 || kk > 0) ? 1u : 0u);
+            umma_commit(smem_u32(&bars->empty[s]));
+          }
+          if (!ok) break;
+          umma_commit(smem_u32(&bars->tfull[b]));
+          ++f;
+        }
+      }
+      if (!ok) {
+        // giving up: wait (bounded) for the MMAs already issued before TMEM is released
+        umma_commit(smem_u32(&bars->drained));
+        const unsigned long long t0 = global_timer();
+        while (!mbar_try_wait(smem_u32(&bars->drained), 0) && global_timer() - t0 < 1000000ull) {}
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (128 threads)
+    const int quarter = warp & 3;               // TMEM lanes this warp may read
+    const int row = quarter * 32 + lane;        // accumulator row = weight-tile row
+    const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+    uint32_t f = 0;
+    bool ok = true;
+    float v[kMaxNodes];
+    auto load_acc = [&](uint32_t b) {
+#pragma unroll
+      for (int c = 0; c < kMaxNodes; c += 16)
+        if (c < p.n_pad) tmem_ld16(tmem_base + lane_addr + b * kAccCols + c, v + c);
+      tmem_ld_wait();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&bars->tempty[b]));
+    };
+    if (p.phase_mask & 1) {
+      const long long U1 = static_cast<long long>(n_act) * tpe * kc1;
+      Sched s1(cta, G, static_cast<long long>(n_act) * tpe, kc1);
+      int tile, k0, k1;
+      while (s1.next(tile, k0, k1)) {
+        const uint32_t b = f & 1u;
+        ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f >> 1) & 1u, abort_flag, p.status));
+        if (!ok) break;
+        tc_fence_after();
+        load_acc(b);
+        ++f;
+        if (k0 > 0) {
+          // tail part of a tile whose first chunks belong to an earlier CTA: hand the fragment over
+          float* dst = p.frag + static_cast<size_t>(cta) * kFragFloats;
+#pragma unroll
+          for (int c = 0; c < kMaxNodes; ++c)
+            if (c < p.n_pad) dst[c * kTileM + row] = v[c];
+          __threadfence();
+          epi_bar_sync();
+          if (row == 0) st_release(&p.frag_flag[cta], p.epoch);
+          continue;
+        }
+        if (k1 < kc1) {
+          // head part: collect the fragments of the CTAs that own the rest of this tile
+          const long long tile_end = static_cast<long long>(tile + 1) * kc1;
+          for (int c2 = cta + 1; c2 < G; ++c2) {
+            const long long b2 = U1 * c2 / G, e2 = U1 * (c2 + 1) / G;
+            if (b2 >= tile_end) break;
+            if (e2 == b2) continue;
+            bool got = true;
+            if (row == 0) got = flag_wait_ge(&p.frag_flag[c2], p.epoch, abort_flag, p.status);
+            ok = epi_vote_all(got);
+            if (!ok) break;
+            const float* src = p.frag + static_cast<size_t>(c2) * kFragFloats;
+#pragma unroll
+            for (int c = 0; c < kMaxNodes; ++c)
+              if (c < p.n_pad) v[c] += __ldcg(src + c * kTileM + row);
+          }
+          if (!ok) break;
+        }
+        const int a = tile / tpe, ti = tile % tpe;
+        if (quarter >= 2) {
+#pragma unroll
+          for (int c = 0; c < kMaxNodes; ++c)
+            if (c < p.n_pad) ex[c * 64 + (row - 64)] = v[c];
+        }
+        epi_bar_sync();
+        if (quarter < 2) {
+          const float* wrow = p.wdense + static_cast<size_t>(a) * kMaxNodes;
+          __nv_bfloat16* hdst = p.hbuf + (static_cast<size_t>(a) * kMaxNodes) * p.I + ti * 64 + row;
+#pragma unroll
+          for (int c = 0; c < kMaxNodes; ++c) {
+            if (c < p.n_pad) {
+              const float g = v[c], u = ex[c * 64 + row];
+              const float h = wrow[c] * (g / (1.0f + __expf(-g))) * u;
+              hdst[static_cast<size_t>(c) * p.I] = __float2bfloat16_rn(h);
+            }
+          }
+          fence_proxy_async();
+          __threadfence();
+        }
+        epi_bar_sync();
+        if (row == 0) atomicAdd(&p.ready[a], 1);
+      }
+    }
+    if ((p.phase_mask & 2) && ok) {
+      Sched s2(cta, G, h_tiles, kc2);
+      int ht, k0, k1;
+      while (s2.next(ht, k0, k1)) {
+        const uint32_t b = f & 1u;
+        ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f >> 1) & 1u, abort_flag, p.status));
+        if (!ok) break;
+        tc_fence_after();
+        load_acc(b);
+        ++f;
+        float* dst = p.out + static_cast<size_t>(ht) * kTileM + row;
+#pragma unroll
+        for (int c = 0; c < kMaxNodes; ++c)
+          if (c < p.T) atomicAdd(dst + static_cast<size_t>(c) * p.H, v[c]);
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------- f32 path
+// h[t][j][i] = silu(g) * u for routed slot j < k (expert idx[t][j]) and shared slot j >= k.
+__global__ void k_ffn_f32_gate_up(const float* __restrict__ x, const float* __restrict__ gate_up,
+                                  const float* __restrict__ shared_gate_up, const int32_t* __restrict__ idx,
+                                  float* __restrict__ hbuf, int T, int H, int I, int k, int n_shared) {
+  const int slots = k + n_shared;
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= T * slots * I) return;
+  const int i = warp % I, j = (warp / I) % slots, t = warp / (I * slots);
+  const int e = j < k ? idx[t * k + j] : j - k;
+  const float* base = j < k ? gate_up : shared_gate_up;
+  float h = 0.0f;
+  if (e >= 0) {
+    const float* g_row = base + (static_cast<size_t>(e) * 2 * I + i) * H;
+    const float* u_row = g_row + static_cast<size_t>(I) * H;
+    const float* xr = x + static_cast<size_t>(t) * H;
+    float g = 0.f, u = 0.f;
+    for (int hh = lane; hh < H; hh += 32) {
+      g = fmaf(g_row[hh], xr[hh], g);
+      u = fmaf(u_row[hh], xr[hh], u);
+    }
+    for (int s = 16; s >= 1; s >>= 1) {
+      g += __shfl_xor_sync(0xffffffffu, g, s);
+      u += __shfl_xor_sync(0xffffffffu, u, s);
+    }
+    h = (g / (1.0f + expf(-g))) * u;
+  }
+  if (lane == 0) hbuf[(static_cast<size_t>(t) * slots + j) * I + i] = h;
+}
+
+__global__ void k_ffn_f32_down(const float* __restrict__ down, const float* __restrict__ shared_down,
+                               const int32_t* __restrict__ idx, const float* __restrict__ w,
+                               const float* __restrict__ hbuf, float* __restrict__ out, int T, int H, int I,
+                               int k, int n_shared) {
+  const int slots = k + n_shared;
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= T * H) return;
+  const int hh = warp % H, t = warp / H;
+  float y = 0.f;
+  for (int j = 0; j < slots; ++j) {
+    const int e = j < k ? idx[t * k + j] : j - k;
+    if (e < 0) continue;
+    const float* d_row = (j < k ? down : shared_down) + (static_cast<size_t>(e) * H + hh) * I;
+    const float* hr = hbuf + (static_cast<size_t>(t) * slots + j) * I;
+    float acc = 0.f;
+    for (int i = lane; i < I; i += 32) acc = fmaf(d_row[i], hr[i], acc);
+    for (int s = 16; s >= 1; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+    y += (j < k ? w[t * k + j] : 1.0f) * acc;
+  }
+  if (lane == 0) out[static_cast<size_t>(t) * H + hh] = y;
+}
+
+}  // namespace
+
+size_t ffn_smem_bytes() { return kSmemBytes; }
+
+cudaError_t ffn_configure() {
+  return cudaFuncSetAttribute(k_ffn_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+}
+
+cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
+                            const CUtensorMap& h_map, cudaStream_t s) {
+  FfnArgs a;
+  a.T = L.T; a.H = L.H; a.I = L.I; a.n_pad = L.n_pad;
+  a.list = L.list; a.wdense = L.wdense; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
+  a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag; a.epoch = L.epoch;
+  a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask;
+  void* args[] = {const_cast<FfnMaps*>(&maps), const_cast<CUtensorMap*>(&x_map), const_cast<CUtensorMap*>(&h_map), &a};
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(L.grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;   // CTAs wait on one another: all must be co-resident
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(k_ffn_bf16), args);
+}
+
+cudaError_t launch_ffn_f32(const float* x, const float* gate_up, const float* down,
+                           const float* shared_gate_up, const float* shared_down, int n_shared,
+                           const int32_t* idx, const float* w, float* hbuf, float* out, int T, int H,
+                           int I, int k, cudaStream_t s) {
+  const int slots = k + n_shared;
+  const long long warps1 = static_cast<long long>(T) * slots * I;
+  k_ffn_f32_gate_up<<<static_cast<unsigned>((warps1 * 32 + 255) / 256), 256, 0, s>>>(x, gate_up, shared_gate_up, idx, hbuf,
+                                                                                   T, H, I, k, n_shared);
+  cudaError_t err = cudaGetLastError();
+  if (err != cudaSuccess) return err;
+  const long long warps2 = static_cast<long long>(T) * H;
+  k_ffn_f32_down<<<static_cast<unsigned>((warps2 * 32 + 255) / 256), 256, 0, s>>>(down, shared_down, idx, w, hbuf, out, T,
+                                                                                H, I, k, n_shared);
+  return cudaGetLastError();
+}
+
+}  // namespace acm

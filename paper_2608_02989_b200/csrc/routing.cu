@@ -1,0 +1,689 @@
+// Stages 1-3 of the verifier-side MoE layer: router logits (Section 3.1), softmax and natural
+// top-k (Eq. 1), commitment-weighted demand (Eq. 4), anchors (Eq. 5), self-sized eligible set
+// (Eq. 6), residency-aware pruning (Eq. 7) and restricted top-k routing (Eq. 2), plus the
+// activated-expert work lists the FFN kernel consumes.
+//
+// Everything that decides a set member, a count or an index is binary32 in a fixed order
+// (explicit round-to-nearest intrinsics, so the compiler can neither contract nor reorder):
+// 32 interleaved partial sums + halving tree for the logit dot product, a 128-slot halving
+// tree for sums over the expert axis, fixed polynomial recipes for exp and log.
+#include <cuda_bf16.h>
+
+#include "acm_internal.h"
+
+namespace acm {
+namespace {
+
+__device__ __forceinline__ void raise_status(int32_t* status, int code) {
+  if (status) atomicCAS(status, 0, code);
+}
+
+// exp(x): x = n ln2 + r (two-term ln2), degree-7 Taylor polynomial, scale through the exponent field.
+__device__ __forceinline__ float exp_fixed(float x) {
+  x = fminf(fmaxf(x, -87.0f), 88.0f);
+  const float n = rintf(__fmul_rn(x, 1.44269502162933349609375f));
+  float r = __fmaf_rn(n, -0.693145751953125f, x);
+  r = __fmaf_rn(n, -1.428606765330187045037746429443359375e-06f, r);
+  float p = 1.98412701138295233249664306640625e-04f;
+  p = __fmaf_rn(p, r, 1.388888922519981861114501953125e-03f);
+  p = __fmaf_rn(p, r, 8.3333337679505348205566406250e-03f);
+  p = __fmaf_rn(p, r, 4.16666679084300994873046875e-02f);
+  p = __fmaf_rn(p, r, 0.16666667163372039794921875f);
+  p = __fmaf_rn(p, r, 0.5f);
+  p = __fmaf_rn(p, r, 1.0f);
+  p = __fmaf_rn(p, r, 1.0f);
+  const float scale = __int_as_float((static_cast<int>(n) + 127) << 23);
+  return __fmul_rn(p, scale);
+}
+
+// log(q), q positive and normal: q = m 2^e, m in (sqrt(1/2), sqrt(2)], log m = 2 atanh((m-1)/(m+1)).
+__device__ __forceinline__ float log_fixed(float q) {
+  const int bits = __float_as_int(q);
+  int e = ((bits >> 23) & 0xff) - 127;
+  float m = __int_as_float((bits & 0x007fffff) | 0x3f800000);
+  if (m > 1.41421353816986083984375f) {
+    m = __fmul_rn(m, 0.5f);
+    e += 1;
+  }
+  const float s = __fdiv_rn(__fsub_rn(m, 1.0f), __fadd_rn(m, 1.0f));
+  const float s2 = __fmul_rn(s, s);
+  float p = 9.0909093618392944335937500e-02f;
+  p = __fmaf_rn(p, s2, 0.111111111938953399658203125f);
+  p = __fmaf_rn(p, s2, 0.14285714924335479736328125f);
+  p = __fmaf_rn(p, s2, 0.20000000298023223876953125f);
+  p = __fmaf_rn(p, s2, 0.3333333432674407958984375f);
+  p = __fmaf_rn(p, s2, 1.0f);
+  const float lm = __fmul_rn(2.0f, __fmul_rn(s, p));
+  return __fmaf_rn(static_cast<float>(e), 0.693147182464599609375f, lm);
+}
+
+// Orderable key: larger logit first, then lower expert index.  0 is "no candidate".
+__device__ __forceinline__ unsigned long long rank_key(float z, int e) {
+  unsigned u = __float_as_uint(z);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return (static_cast<unsigned long long>(u) << 32) | static_cast<unsigned>(0xffffffffu - e);
+}
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) {
+    const unsigned long long o = __shfl_xor_sync(0xffffffffu, v, s);
+    v = o > v ? o : v;
+  }
+  return v;
+}
+__device__ __forceinline__ float warp_max_f(float v) {
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, s));
+  return v;
+}
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+  return v;
+}
+
+// Sum of a 128-slot array held as 4 values per lane (slot = lane + 32 c): the halving tree
+// a[i] += a[i+s], s = 64, 32, 16, ..., 1.  Result broadcast to the whole warp.
+__device__ __forceinline__ float warp_tree_sum_128(float a0, float a1, float a2, float a3) {
+  float v = __fadd_rn(__fadd_rn(a0, a2), __fadd_rn(a1, a3));
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) v = __fadd_rn(v, __shfl_down_sync(0xffffffffu, v, s));
+  return __shfl_sync(0xffffffffu, v, 0);
+}
+
+// ------------------------------------------------------------------------------------------
+// Stage 1a: router logits.  CTA tile = 8 nodes x 8 experts, rows staged in shared memory with
+// 16-byte async copies in 4 K-chunks.  A 16-byte load covers EPT consecutive h, i.e. EPT of
+// the 32 interleaved partial sums; Q = 32/EPT threads share one output.
+// ------------------------------------------------------------------------------------------
+constexpr int kRT = 8, kRE = 8;
+
+template <typename Elem>
+struct ElemTraits;
+template <>
+struct ElemTraits<float> {
+  static constexpr int EPT = 4;
+  __device__ static void unpack(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+    f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+  }
+};
+template <>
+struct ElemTraits<__nv_bfloat16> {
+  static constexpr int EPT = 8;
+  __device__ static void unpack(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+    f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
+    f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
+  }
+};
+
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {
+  const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+template <typename Elem>
+__global__ void __launch_bounds__(32 * (32 / ElemTraits<Elem>::EPT) * 1)
+k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const float* __restrict__ bias,
+                float* __restrict__ logits, int T, int H, int E, int n_chunks, float* zero_buf,
+                size_t zero_floats, int32_t* status) {
+  constexpr int EPT = ElemTraits<Elem>::EPT;
+  constexpr int Q = 32 / EPT;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int row_bytes = H * static_cast<int>(sizeof(Elem)) + 64;   // +64 B staggers rows over the banks
+  unsigned char* xs = smem_raw;
+  unsigned char* ws = smem_raw + static_cast<size_t>(kRT) * row_bytes;
+
+  const int tid = threadIdx.x;
+  const int e0 = blockIdx.x * kRE, t0 = blockIdx.y * kRT;
+
+  // zero the FFN output buffer (accumulated into by the FFN kernel), spread over the grid
+  if (zero_buf) {
+    const size_t nb = static_cast<size_t>(gridDim.x) * gridDim.y;
+    const size_t b = static_cast<size_t>(blockIdx.y) * gridDim.x + blockIdx.x;
+    const size_t n4 = zero_floats / 4;
+    float4* z4 = reinterpret_cast<float4*>(zero_buf);
+    for (size_t i = b * blockDim.x + tid; i < n4; i += nb * blockDim.x) z4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+
+  // async staging of 8 x-rows and 8 router rows, n_chunks commit groups along h
+  const int segs_per_row = H * static_cast<int>(sizeof(Elem)) / 16;
+  const int segs_per_chunk = segs_per_row / n_chunks;
+  for (int c = 0; c < n_chunks; ++c) {
+    for (int i = tid; i < (kRT + kRE) * segs_per_chunk; i += blockDim.x) {
+      const int row = i / segs_per_chunk, seg = c * segs_per_chunk + i % segs_per_chunk;
+      if (row < kRT) {
+        const int t = min(t0 + row, T - 1);
+        cp_async_16(xs + static_cast<size_t>(row) * row_bytes + seg * 16,
+                    reinterpret_cast<const unsigned char*>(x + static_cast<size_t>(t) * H) + seg * 16);
+      } else {
+        const int e = min(e0 + row - kRT, E - 1);
+        cp_async_16(ws + static_cast<size_t>(row - kRT) * row_bytes + seg * 16,
+                    reinterpret_cast<const unsigned char*>(wr + static_cast<size_t>(e) * H) + seg * 16);
+      }
+    }
+    cp_async_commit();
+  }
+
+  const int q = tid % Q;            // which EPT-wide group of the 32 partial sums
+  const int mt = tid / Q;           // micro tile: 2 nodes x 1 expert
+  const int el = mt % kRE, tp = mt / kRE;
+  float acc[2][EPT];
+#pragma unroll
+  for (int p = 0; p < EPT; ++p) acc[0][p] = acc[1][p] = 0.0f;
+
+  const unsigned char* xr0 = xs + static_cast<size_t>(2 * tp) * row_bytes + q * 16;
+  const unsigned char* xr1 = xr0 + row_bytes;
+  const unsigned char* wrow = ws + static_cast<size_t>(el) * row_bytes + q * 16;
+  const int steps_per_chunk = H / 32 / n_chunks;
+  const int step_bytes = 32 * static_cast<int>(sizeof(Elem));
+  for (int c = 0; c < n_chunks; ++c) {
+    // chunk c is complete once at most (n_chunks-1-c) groups are still pending
+    if (c == 0) { if (n_chunks == 4) cp_async_wait<3>(); else cp_async_wait<0>(); }
+    else if (c == 1) cp_async_wait<2>();
+    else if (c == 2) cp_async_wait<1>();
+    else cp_async_wait<0>();
+    __syncthreads();
+    const int j0 = c * steps_per_chunk;
+#pragma unroll 4
+    for (int j = j0; j < j0 + steps_per_chunk; ++j) {
+      float xa[EPT], xb[EPT], wv[EPT];
+      ElemTraits<Elem>::unpack(*reinterpret_cast<const uint4*>(xr0 + static_cast<size_t>(j) * step_bytes), xa);
+      ElemTraits<Elem>::unpack(*reinterpret_cast<const uint4*>(xr1 + static_cast<size_t>(j) * step_bytes), xb);
+      ElemTraits<Elem>::unpack(*reinterpret_cast<const uint4*>(wrow + static_cast<size_t>(j) * step_bytes), wv);
+#pragma unroll
+      for (int p = 0; p < EPT; ++p) {
+        acc[0][p] = __fmaf_rn(xa[p], wv[p], acc[0][p]);
+        acc[1][p] = __fmaf_rn(xb[p], wv[p], acc[1][p]);
+      }
+    }
+  }
+  // halving tree over the 32 partial sums: partial l = q*EPT + p
+#pragma unroll
+  for (int s = 16; s >= EPT; s >>= 1) {
+#pragma unroll
+    for (int p = 0; p < EPT; ++p) {
+      acc[0][p] = __fadd_rn(acc[0][p], __shfl_xor_sync(0xffffffffu, acc[0][p], s / EPT));
+      acc[1][p] = __fadd_rn(acc[1][p], __shfl_xor_sync(0xffffffffu, acc[1][p], s / EPT));
+    }
+  }
+#pragma unroll
+  for (int s = EPT / 2; s >= 1; s >>= 1) {
+#pragma unroll
+    for (int p = 0; p < s; ++p) {
+      acc[0][p] = __fadd_rn(acc[0][p], acc[0][p + s]);
+      acc[1][p] = __fadd_rn(acc[1][p], acc[1][p + s]);
+    }
+  }
+  if (q == 0 && e0 + el < E) {
+    const int e = e0 + el;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const int t = t0 + 2 * tp + r;
+      if (t < T) {
+        float z = acc[r][0];
+        if (bias) z = __fadd_rn(z, bias[e]);
+        logits[static_cast<size_t>(t) * E + e] = z;
+        if (!isfinite(z)) raise_status(status, ACM_ERR_NONFINITE);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Block-cooperative stages.  Each is called by every thread of the CTA (>= 128 threads, a
+// multiple of 32) and ends with __syncthreads().
+// ------------------------------------------------------------------------------------------
+struct StageSmem {
+  float alpha[kMaxNodes];
+  uint32_t natmask[kMaxNodes][kMaskWords];
+  int32_t votes[kMaxExperts];
+  float u[kMaxExperts];
+  float tree[kMaxExperts];
+  uint32_t A[kMaskWords], S[kMaskWords], Sp[kMaskWords], Hres[kMaskWords];
+  int32_t idx[kMaxNodes][kMaxTopK];
+  float w[kMaxNodes][kMaxTopK];
+  int32_t cnt[kMaxExperts];
+  int32_t slot_of[kMaxExperts];
+  int32_t list_of[kMaxExperts];
+  int32_t warp_tot[2][4];
+  int32_t scal[8];
+  float fscal[4];
+};
+
+// Stage 1b: softmax over the expert axis and natural top-k (ranked on the logits), one warp per node.
+__device__ void stage_softmax_topk(const float* __restrict__ logits, float* __restrict__ probs,
+                                   int32_t* __restrict__ nat_idx, int T, int E, int k) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  for (int t = warp; t < T; t += nwarps) {
+    float z[4], y[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int e = lane + 32 * c;
+      z[c] = e < E ? logits[static_cast<size_t>(t) * E + e] : -INFINITY;
+    }
+    const float zmax = warp_max_f(fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])));
+#pragma unroll
+    for (int c = 0; c < 4; ++c) y[c] = (lane + 32 * c < E) ? exp_fixed(__fsub_rn(z[c], zmax)) : 0.0f;
+    const float denom = warp_tree_sum_128(y[0], y[1], y[2], y[3]);
+    if (probs) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        if (lane + 32 * c < E) probs[static_cast<size_t>(t) * E + lane + 32 * c] = __fdiv_rn(y[c], denom);
+    }
+    if (nat_idx) {
+      unsigned taken = 0;
+      for (int j = 0; j < k; ++j) {
+        unsigned long long best = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int e = lane + 32 * c;
+          if (e < E && !((taken >> c) & 1u)) {
+            const unsigned long long key = rank_key(z[c], e);
+            best = key > best ? key : best;
+          }
+        }
+        best = warp_max_u64(best);
+        const int e = static_cast<int>(0xffffffffu - static_cast<unsigned>(best & 0xffffffffu));
+        if ((e & 31) == lane) taken |= 1u << (e >> 5);
+        if (lane == 0) nat_idx[static_cast<size_t>(t) * k + j] = e;
+      }
+    }
+  }
+  __syncthreads();
+}
+
+// 128-slot halving tree over shared memory (threads 0..127 hold one slot each).
+__device__ float block_tree_sum_128(float* tree, float mine) {
+  const int tid = threadIdx.x;
+  if (tid < kMaxExperts) tree[tid] = mine;
+  __syncthreads();
+#pragma unroll
+  for (int s = kMaxExperts / 2; s >= 1; s >>= 1) {
+    if (tid < s) tree[tid] = __fadd_rn(tree[tid], tree[tid + s]);
+    __syncthreads();
+  }
+  const float r = tree[0];
+  __syncthreads();
+  return r;
+}
+
+// Stage 2: demand, anchors, self-sizing, pruning.  Thread e < 128 owns expert e.
+__device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, int k) {
+  const int tid = threadIdx.x;
+  const int lane = tid & 31, warp = tid >> 5;
+  const bool owner = tid < kMaxExperts;
+  const bool live = tid < E;
+  for (int i = tid; i < kMaxNodes * kMaskWords; i += blockDim.x) (&sm.natmask[0][0])[i] = 0u;
+  if (tid < kMaskWords) {
+    sm.A[tid] = 0u;
+    sm.Hres[tid] = a.resident ? a.resident[tid < (E + 31) / 32 ? tid : 0] : 0xffffffffu;
+    if (tid >= (E + 31) / 32) sm.Hres[tid] = 0u;
+  }
+  if (tid < 8) sm.scal[tid] = 0;
+  for (int i = tid; i < T; i += blockDim.x) sm.alpha[i] = a.alpha[i];
+  __syncthreads();
+  for (int i = tid; i < T * k; i += blockDim.x) {
+    const int e = a.nat_idx[i];
+    if (e >= 0 && e < E) atomicOr(&sm.natmask[i / k][e >> 5], 1u << (e & 31));
+  }
+  if (a.prm.use_anchors) {
+    const int n_nodes = a.anchor_nodes ? a.n_anchor_nodes : 1;
+    for (int i = tid; i < n_nodes * k; i += blockDim.x) {
+      const int t = a.anchor_nodes ? a.anchor_nodes[i / k] : 0;
+      if (t >= 0 && t < T) {
+        const int e = a.nat_idx[static_cast<size_t>(t) * k + i % k];
+        if (e >= 0 && e < E) atomicOr(&sm.A[e >> 5], 1u << (e & 31));
+      }
+    }
+  }
+  __syncthreads();
+
+  // votes v_e and demand u_e (nodes ascending, fused multiply-add)
+  int votes = 0;
+  float u = 0.0f;
+  if (live) {
+    for (int t = 0; t < T; ++t) {
+      const bool in_topk = (sm.natmask[t][warp] >> lane) & 1u;
+      votes += in_topk ? 1 : 0;
+      if (a.prm.demand == ACM_DEMAND_FULL_MASS || (a.prm.demand == ACM_DEMAND_TOPK_MASS && in_topk))
+        u = __fmaf_rn(sm.alpha[t], a.probs[static_cast<size_t>(t) * E + tid], u);
+    }
+    if (a.prm.demand == ACM_DEMAND_VOTES) u = static_cast<float>(votes);
+  }
+  if (owner) {
+    sm.votes[tid] = votes;
+    sm.u[tid] = u;
+  }
+  const bool in_A = live && ((sm.A[warp] >> lane) & 1u);
+  const bool in_R = live && !in_A;
+  const int nA = __syncthreads_count(in_A);
+  const int nR = E - nA;
+  const int n_positive = __syncthreads_count(in_R && u > 0.0f);
+  const float upos = in_R ? fmaxf(u, 0.0f) : 0.0f;
+  const float Z = block_tree_sum_128(sm.tree, upos);
+
+  const int floor_keep = max(0, k - nA);
+  int n_er = 0, n_keep;
+  if (a.prm.fixed_budget > 0) {
+    n_keep = max(max(0, a.prm.fixed_budget - nA), floor_keep);
+  } else if (Z > 0.0f) {
+    const float qv = __fdiv_rn(upos, Z);
+    const float h = (qv >= 1.17549435e-38f) ? __fmul_rn(qv, log_fixed(qv)) : 0.0f;
+    const float entropy = -block_tree_sum_128(sm.tree, h);
+    const float perp = exp_fixed(entropy);
+    n_er = static_cast<int>(ceilf(__fsub_rn(perp, a.prm.ceil_guard)));
+    n_er = min(max(n_er, 1), n_positive);
+    n_keep = max(n_er, floor_keep);
+  } else {
+    n_keep = floor_keep;
+  }
+  n_keep = min(n_keep, nR);
+
+  // rank inside R by (u descending, index ascending)
+  bool in_S = in_A;
+  if (in_R) {
+    int rank = 0;
+    for (int j = 0; j < E; ++j) {
+      const bool j_in_R = !((sm.A[j >> 5] >> (j & 31)) & 1u);
+      const float uj = sm.u[j];
+      rank += (j_in_R && (uj > u || (uj == u && j < tid))) ? 1 : 0;
+    }
+    in_S = rank < n_keep;
+  }
+  const unsigned s_word = __ballot_sync(0xffffffffu, in_S);
+  if (owner && lane == 0) sm.S[warp] = s_word;
+  const int nS = __syncthreads_count(in_S);
+  const int n_union = __syncthreads_count(live && votes > 0);
+  if (live && votes > 0 && !in_S) atomicAdd(&sm.scal[0], votes);   // a(S)
+  __syncthreads();
+  const int aS = sm.scal[0];
+
+  bool in_Sp = in_S;
+  int m_star = 0;
+  const bool resident = live && ((sm.Hres[warp] >> lane) & 1u);
+  if (a.prm.residency == 1 && a.resident) {
+    const bool in_C = in_S && !resident;
+    bool removed = false;
+    if (in_C) {
+      int pos = 1, cum = votes;     // position in pi (1-based) and votes of the prefix ending here
+      for (int j = 0; j < E; ++j) {
+        if (j == tid) continue;
+        const bool j_in_C = ((sm.S[j >> 5] >> (j & 31)) & 1u) && !((sm.Hres[j >> 5] >> (j & 31)) & 1u);
+        const float uj = sm.u[j];
+        if (j_in_C && (uj < u || (uj == u && j < tid))) {
+          pos += 1;
+          cum += sm.votes[j];
+        }
+      }
+      removed = cum <= aS && nS - pos >= k && pos <= a.prm.max_remove;
+    }
+    in_Sp = in_S && !removed;
+    m_star = __syncthreads_count(removed);
+  } else if (a.prm.residency == 2 && a.resident) {
+    in_Sp = (in_S && resident) || in_A;
+  }
+  const unsigned sp_word = __ballot_sync(0xffffffffu, in_Sp);
+  if (owner && lane == 0) sm.Sp[warp] = sp_word;
+  const int nSp = __syncthreads_count(in_Sp);
+  if (a.prm.residency == 2 && a.resident) m_star = nS - nSp;
+
+  const int words = (E + 31) / 32;
+  if (tid < words) {
+    a.mask_out[tid] = sm.Sp[tid];
+    if (a.unpruned_out) a.unpruned_out[tid] = sm.S[tid];
+  }
+  if (live && a.demand_out) a.demand_out[tid] = u;
+  if (tid == 0) {
+    *a.count_out = nSp;
+    if (a.stats_out) {
+      acm_block_stats st;
+      st.n_anchor = nA; st.n_er = n_er; st.n_eligible = nS; st.n_eligible_pruned = nSp;
+      st.n_activated = 0; st.n_natural_union = n_union; st.displaced_aS = aS; st.pruned_m = m_star;
+      st.n_staged = 0; st.reserved[0] = st.reserved[1] = st.reserved[2] = 0;
+      *a.stats_out = st;
+    }
+  }
+  __syncthreads();
+}
+
+// Turns per-node routes (sm.idx / sm.w) into the FFN work lists: activated experts in ascending
+// id order, shared experts appended; combine weights scattered into the dense [slot][node] table.
+__device__ void stage_build_lists(const RouteArgs& a, StageSmem& sm, int T, int E, int k) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid < kMaxExperts) sm.cnt[tid] = 0;
+  for (int i = tid; i < 2 * kMaxSlots * kMaxNodes; i += blockDim.x) a.wdense[i] = 0.0f;
+  for (int i = tid; i < 2 * kMaxSlots; i += blockDim.x) a.ready[i] = 0;
+  if (tid < kMaskWords) sm.Hres[tid] = a.resident ? (tid < (E + 31) / 32 ? a.resident[tid] : 0u) : 0xffffffffu;
+  __syncthreads();
+  for (int i = tid; i < T * k; i += blockDim.x) {
+    const int e = sm.idx[i / k][i % k];
+    if (e >= 0) atomicAdd(&sm.cnt[e], 1);
+  }
+  __syncthreads();
+  // slots by ascending expert id: resident activated experts -> list 0, the others -> list 1
+  const bool active = tid < E && sm.cnt[tid] > 0;
+  const bool res = active && ((sm.Hres[warp & 3] >> lane) & 1u);
+  const bool stg = active && !res;
+  const unsigned b0 = __ballot_sync(0xffffffffu, res), b1 = __ballot_sync(0xffffffffu, stg);
+  if (tid < kMaxExperts && lane == 0) {
+    sm.warp_tot[0][warp] = __popc(b0);
+    sm.warp_tot[1][warp] = __popc(b1);
+  }
+  __syncthreads();
+  int base0 = 0, base1 = 0, n0 = 0, n1 = 0;
+#pragma unroll
+  for (int wv = 0; wv < 4; ++wv) {
+    if (wv < warp) { base0 += sm.warp_tot[0][wv]; base1 += sm.warp_tot[1][wv]; }
+    n0 += sm.warp_tot[0][wv];
+    n1 += sm.warp_tot[1][wv];
+  }
+  if (tid < kMaxExperts) {
+    const unsigned lower = (1u << lane) - 1u;
+    if (res) {
+      const int slot = base0 + __popc(b0 & lower);
+      sm.slot_of[tid] = slot; sm.list_of[tid] = 0;
+      a.lists[0].entry[slot] = make_entry(kSrcRouted, tid);
+      a.lists[0].expert[slot] = tid;
+    } else if (stg) {
+      const int slot = base1 + __popc(b1 & lower);
+      sm.slot_of[tid] = slot; sm.list_of[tid] = 1;
+      a.lists[1].entry[slot] = make_entry(kSrcStaged, slot);
+      a.lists[1].expert[slot] = tid;
+      if (a.host_stage_list) a.host_stage_list[1 + slot] = tid;
+    }
+  }
+  if (tid < a.n_shared) {
+    a.lists[0].entry[n0 + tid] = make_entry(kSrcShared, tid);
+    a.lists[0].expert[n0 + tid] = -1;
+  }
+  if (tid == 0) {
+    a.lists[0].n = n0 + a.n_shared; a.lists[0].n_stage = 0;
+    a.lists[1].n = n1; a.lists[1].n_stage = n1;
+    if (a.host_stage_list) a.host_stage_list[0] = n1;
+    if (a.stats_out) { a.stats_out->n_activated = n0 + n1; a.stats_out->n_staged = n1; }
+  }
+  __syncthreads();
+  for (int i = tid; i < T * k; i += blockDim.x) {
+    const int t = i / k, e = sm.idx[t][i % k];
+    if (e >= 0)
+      a.wdense[(static_cast<size_t>(sm.list_of[e]) * kMaxSlots + sm.slot_of[e]) * kMaxNodes + t] = sm.w[t][i % k];
+  }
+  for (int i = tid; i < a.n_shared * T; i += blockDim.x)
+    a.wdense[static_cast<size_t>(n0 + i / T) * kMaxNodes + i % T] = 1.0f;
+  __syncthreads();
+}
+
+// Stage 3: restricted top-k (Eq. 2) and combine weights, one warp per node.
+__device__ void stage_route(const RouteArgs& a, StageSmem& sm, int T, int E, int k) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  for (int t = warp; t < T; t += nwarps) {
+    float z[4], y[4];
+    bool elig[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int e = lane + 32 * c;
+      z[c] = e < E ? a.logits[static_cast<size_t>(t) * E + e] : -INFINITY;
+      elig[c] = e < E && ((a.mask[c] >> lane) & 1u);
+    }
+    const float zmax = warp_max_f(fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])));
+    float s_all = 0.f, s_elig = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      y[c] = (lane + 32 * c < E) ? expf(z[c] - zmax) : 0.0f;
+      s_all += y[c];
+      s_elig += elig[c] ? y[c] : 0.0f;
+    }
+    s_all = warp_sum_f(s_all);
+    s_elig = warp_sum_f(s_elig);
+    unsigned taken = 0;
+    float s_sel = 0.f, my_y = 0.f;
+    int my_e = -1;
+    for (int j = 0; j < k; ++j) {
+      unsigned long long best = 0;
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        if (elig[c] && !((taken >> c) & 1u)) {
+          const unsigned long long key = rank_key(z[c], lane + 32 * c);
+          best = key > best ? key : best;
+        }
+      best = warp_max_u64(best);
+      int e = -1;
+      float ye = 0.f;
+      if (best != 0ull) {
+        e = static_cast<int>(0xffffffffu - static_cast<unsigned>(best & 0xffffffffu));
+        const int c = e >> 5;
+        const float cand = c == 0 ? y[0] : c == 1 ? y[1] : c == 2 ? y[2] : y[3];
+        ye = __shfl_sync(0xffffffffu, cand, e & 31);
+        if ((e & 31) == lane) taken |= 1u << c;
+      }
+      s_sel += ye;
+      if (lane == j) { my_e = e; my_y = ye; }
+    }
+    if (lane < k) {
+      const float den = a.weighting == ACM_W_RENORM_TOPK ? s_sel : a.weighting == ACM_W_SOFTMAX_RAW ? s_all : s_elig;
+      const float wgt = my_e >= 0 ? a.routed_scale * my_y / den : 0.0f;
+      sm.idx[t][lane] = my_e;
+      sm.w[t][lane] = wgt;
+      if (a.idx_out) a.idx_out[static_cast<size_t>(t) * k + lane] = my_e;
+      if (a.w_out) a.w_out[static_cast<size_t>(t) * k + lane] = wgt;
+    }
+  }
+  __syncthreads();
+  if (a.lists) stage_build_lists(a, sm, T, E, k);
+}
+
+__global__ void __launch_bounds__(1024) k_softmax_topk(const float* logits, float* probs, int32_t* nat_idx,
+                                                       int T, int E, int k) {
+  stage_softmax_topk(logits, probs, nat_idx, T, E, k);
+}
+
+__global__ void __launch_bounds__(128) k_select(SelectArgs a, int T, int E, int k) {
+  __shared__ StageSmem sm;
+  stage_select(a, sm, T, E, k);
+}
+
+__global__ void __launch_bounds__(1024) k_route(RouteArgs a, int T, int E, int k) {
+  __shared__ StageSmem sm;
+  stage_route(a, sm, T, E, k);
+}
+
+__global__ void __launch_bounds__(1024) k_fused_select_route(const float* logits, float* probs, int32_t* nat_idx,
+                                                             SelectArgs sa, RouteArgs ra,
+                                                             const uint32_t* mask_override, int T, int E, int k) {
+  __shared__ StageSmem sm;
+  if (mask_override) {
+    if (threadIdx.x < (E + 31) / 32) sa.mask_out[threadIdx.x] = mask_override[threadIdx.x];
+    if (threadIdx.x == 0 && sa.stats_out) {
+      acm_block_stats st = {};
+      *sa.stats_out = st;
+    }
+    __syncthreads();
+  } else {
+    stage_softmax_topk(logits, probs, nat_idx, T, E, k);
+    stage_select(sa, sm, T, E, k);
+  }
+  stage_route(ra, sm, T, E, k);
+}
+
+__global__ void __launch_bounds__(512) k_routes_to_lists(const int32_t* idx, const float* w, RouteArgs a, int T,
+                                                         int E, int k) {
+  __shared__ StageSmem sm;
+  for (int i = threadIdx.x; i < T * k; i += blockDim.x) {
+    const int e = idx[i];
+    sm.idx[i / k][i % k] = (e >= 0 && e < E) ? e : -1;
+    sm.w[i / k][i % k] = w[i];
+  }
+  __syncthreads();
+  stage_build_lists(a, sm, T, E, k);
+}
+
+}  // namespace
+
+cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
+                                 float* logits, int T, int H, int E, float* zero_buf,
+                                 size_t zero_floats, int32_t* status, cudaStream_t s) {
+  const dim3 grid((E + kRE - 1) / kRE, (T + kRT - 1) / kRT);
+  const int elt = dtype == ACM_F32 ? 4 : 2;
+  const size_t smem = static_cast<size_t>(kRT + kRE) * (static_cast<size_t>(H) * elt + 64);
+  const int n_chunks = (H % 128 == 0) ? 4 : 1;
+  if (dtype == ACM_F32) {
+    auto kern = k_router_logits<float>;
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (err != cudaSuccess) return err;
+    kern<<<grid, 256, smem, s>>>(static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
+                                 logits, T, H, E, n_chunks, zero_buf, zero_floats, status);
+  } else {
+    auto kern = k_router_logits<__nv_bfloat16>;
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (err != cudaSuccess) return err;
+    kern<<<grid, 128, smem, s>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router),
+                                 bias, logits, T, H, E, n_chunks, zero_buf, zero_floats, status);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_softmax_topk(const float* logits, float* probs, int32_t* nat_idx, int T, int E,
+                                int k, int32_t* /*status*/, cudaStream_t s) {
+  const int threads = min(1024, 32 * T);
+  k_softmax_topk<<<1, max(threads, 32), 0, s>>>(logits, probs, nat_idx, T, E, k);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s) {
+  k_select<<<1, 128, 0, s>>>(a, T, E, k);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s) {
+  const int threads = max(128, min(1024, 32 * T));
+  k_route<<<1, threads, 0, s>>>(a, T, E, k);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fused_select_route(const float* logits, float* probs, int32_t* nat_idx,
+                                      const SelectArgs& sa, const RouteArgs& ra,
+                                      const uint32_t* mask_override, int T, int E, int k,
+                                      int32_t* /*status*/, cudaStream_t s) {
+  const int threads = max(128, min(1024, 32 * T));
+  k_fused_select_route<<<1, threads, 0, s>>>(logits, probs, nat_idx, sa, ra, mask_override, T, E, k);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_routes_to_lists(const int32_t* idx, const float* w, WorkList* lists, float* wdense,
+                                   int32_t* ready, int n_shared, int T, int E, int k, cudaStream_t s) {
+  RouteArgs a = {};
+  a.lists = lists;
+  a.wdense = wdense;
+  a.ready = ready;
+  a.n_shared = n_shared;
+  k_routes_to_lists<<<1, 512, 0, s>>>(idx, w, a, T, E, k);
+  return cudaGetLastError();
+}
+
+}  // namespace acm

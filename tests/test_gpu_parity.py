@@ -1,0 +1,351 @@
+"""GPU parity: every stage of the CUDA library, called through the C ABI, against the CPU oracle
+on the same seeded inputs.  Sets, counts, indices, logits, probabilities and demand are compared
+bit for bit; routing weights within 1e-5 relative; FFN outputs within 2e-2 x RMS(oracle output)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_02989_b200 import acm, workloads as wl
+from tests.helpers import full_mask, mask_to_set, set_to_mask
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+FFN_TOL = 2e-2
+
+
+def _u32(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def _take(t, rows):
+    return t[torch.as_tensor(np.asarray(rows), device=t.device, dtype=torch.long)]
+
+
+def _ctx(cfg, **kw):
+    return acm.Context.for_config(cfg, n_layers=kw.pop("n_layers", 1), **kw)
+
+
+def _block(cfg, layer=0, experts=True):
+    w = wl.layer_weights(cfg, layer, DEV, experts=experts)
+    x = wl.hidden_states(cfg, layer, DEV)
+    depth, p = wl.tree_depths(cfg), wl.commitment_table(cfg)
+    alpha = acm.node_weights(depth, p)
+    np.testing.assert_array_equal(alpha.numpy(), oracle.node_weights(depth.numpy(), p.numpy()))
+    return w, x, alpha
+
+
+def _set_weights(ctx, w, layer=0):
+    ctx.set_layer_weights(layer, w["w_router"], w["router_bias"], w["gate_up"], w["down"],
+                          w["shared_gate_up"], w["shared_down"])
+
+
+def _ffn_check(out, ref, what=""):
+    out = out.double().cpu().numpy()
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    err = float(np.abs(out - ref).max())
+    assert np.isfinite(out).all(), what
+    assert err <= FFN_TOL * rms, f"{what}: max|d|={err:.3e} > {FFN_TOL} * rms={rms:.3e}"
+    return err / rms
+
+
+ROUTER_SHAPES = [
+    # (dtype, T, H, E, k, bias)
+    ("f32", 8, 256, 16, 2, False),
+    ("f32", 5, 96, 13, 3, True),
+    ("bf16", 64, 2048, 128, 8, True),
+    ("bf16", 37, 1024, 60, 6, False),
+    ("bf16", 1, 256, 8, 1, False),
+    ("bf16", 64, 4096, 128, 8, False),
+    ("bf16", 33, 384, 100, 8, True),
+]
+
+
+@pytest.mark.parametrize("dtype,T,H,E,k,bias", ROUTER_SHAPES)
+def test_router_bit_exact(dtype, T, H, E, k, bias):
+    g = torch.Generator(device=DEV).manual_seed(T * 1000 + E)
+    td = torch.float32 if dtype == "f32" else torch.bfloat16
+    x = torch.randn(T, H, generator=g, device=DEV).to(td)
+    wr = (0.05 * torch.randn(E, H, generator=g, device=DEV)).to(td)
+    b = torch.randn(E, generator=g, device=DEV) if bias else None
+    ctx = acm.Context(H, E, k, 64, dtype=acm.F32 if dtype == "f32" else acm.BF16)
+    ctx.set_layer_weights(0, wr, b, None, None)
+    z, r, nat = ctx.router(0, x)
+    assert ctx.device_status() == acm.OK
+    zo, ro, nato = oracle.router(x, wr, b, k)
+    np.testing.assert_array_equal(z.cpu().numpy(), zo)
+    np.testing.assert_array_equal(r.cpu().numpy(), ro)
+    np.testing.assert_array_equal(nat.cpu().numpy(), nato)
+    ctx.close()
+
+
+def test_router_flags_non_finite_logits():
+    x = torch.randn(4, 256, device=DEV).to(torch.bfloat16)
+    wr = torch.randn(8, 256, device=DEV).to(torch.bfloat16)
+    b = torch.zeros(8, device=DEV)
+    b[3] = float("inf")
+    ctx = acm.Context(256, 8, 2, 64)
+    ctx.set_layer_weights(0, wr, b, None, None)
+    ctx.router(0, x)
+    assert ctx.device_status() == acm.ERR_NONFINITE
+    assert ctx.device_status() == acm.OK     # sticky until read, then cleared
+    ctx.close()
+
+
+def _random_routing_inputs(rng, T, E, k, scale):
+    z = (scale * rng.standard_normal((T, E))).astype(np.float32)
+    p = np.exp(z.astype(np.float64) - z.max(1, keepdims=True))
+    r = (p / p.sum(1, keepdims=True)).astype(np.float32)
+    nat = np.array([sorted(range(E), key=lambda e: (-float(row[e]), e))[:k] for row in z], dtype=np.int32)
+    return z, r, nat
+
+
+SELECT_MODES = [
+    dict(),
+    dict(demand=1),
+    dict(demand=2),
+    dict(use_anchors=0),
+    dict(fixed_budget=20),
+    dict(demand=1, use_anchors=0, fixed_budget=12),
+    dict(ceil_guard=0.0),
+    dict(residency=1),
+    dict(residency=1, max_remove=2),
+    dict(residency=2),
+]
+
+
+@pytest.mark.parametrize("mode_id", range(len(SELECT_MODES)))
+def test_select_eligible_bit_exact(mode_id):
+    mode = SELECT_MODES[mode_id]
+    rng = np.random.default_rng(100 + mode_id)
+    cases = [(64, 128, 8), (32, 64, 8), (48, 64, 6), (8, 16, 2), (1, 128, 8), (17, 33, 5), (64, 96, 1), (3, 8, 8)]
+    for T, E, k in cases:
+        ctx = acm.Context(256, E, k, 64)
+        for rep in range(6):
+            z, r, nat = _random_routing_inputs(rng, T, E, k, float(rng.choice([0.3, 1.0, 3.0])))
+            alpha = rng.uniform(0.05, 1.0, T).astype(np.float32)
+            if rep == 5:
+                alpha[:] = 1.0
+            resident = {e for e in range(E) if rng.random() < 0.4}
+            rmask = set_to_mask(resident, E)
+            anchors = None if rep % 3 else np.array(sorted(set([0, T // 2, T - 1])), dtype=np.int32)
+            po = oracle.SelectParams(**mode)
+            pg = acm.SelectParams(**mode)
+            want = oracle.select_eligible(r, nat, alpha, po, anchors, rmask if mode.get("residency") else None)
+            got = ctx.select_eligible(torch.tensor(r, device=DEV), torch.tensor(nat, device=DEV),
+                                      torch.tensor(alpha, device=DEV), pg,
+                                      None if anchors is None else torch.tensor(anchors, device=DEV),
+                                      torch.tensor(rmask.view(np.int32), device=DEV) if mode.get("residency") else None)
+            np.testing.assert_array_equal(_u32(got["mask"]), want["mask"])
+            np.testing.assert_array_equal(_u32(got["unpruned_mask"]), want["unpruned_mask"])
+            assert int(got["count"]) == want["count"]
+            np.testing.assert_array_equal(got["demand"].cpu().numpy(), want["demand"])
+            st = acm.stats_dict(got["stats"])
+            for key in ("n_anchor", "n_er", "n_eligible", "n_eligible_pruned", "n_natural_union", "displaced_aS",
+                        "pruned_m"):
+                assert st[key] == want["stats"][key], (key, T, E, k, rep)
+        ctx.close()
+
+
+def test_select_closed_forms_on_gpu():
+    # uniform residual demand over m experts -> n_er = m, for every m (Eq. 6 and the text below it)
+    E = 128
+    ctx = acm.Context(256, E, 1, 64)
+    for m in list(range(1, 20)) + [33, 64, 100, 120, 128]:
+        u = np.zeros((1, E), dtype=np.float32)
+        u[0, :m] = 0.37
+        got = ctx.select_eligible(torch.tensor(u, device=DEV), torch.zeros(1, 1, dtype=torch.int32, device=DEV),
+                                  torch.ones(1, device=DEV), acm.SelectParams(demand=1, use_anchors=0))
+        assert int(got["count"]) == m
+        assert mask_to_set(_u32(got["mask"]), E) == set(range(m))
+    ctx.close()
+
+
+@pytest.mark.parametrize("weighting", [0, 1, 2])
+def test_route_restricted(weighting):
+    rng = np.random.default_rng(weighting)
+    for T, E, k in [(64, 128, 8), (48, 64, 6), (8, 16, 2), (1, 8, 1), (19, 70, 7)]:
+        ctx = acm.Context(256, E, k, 64, weighting=weighting, routed_scale=1.5)
+        for rep in range(5):
+            z, _, nat = _random_routing_inputs(rng, T, E, k, 2.0)
+            if rep == 0:
+                S = set(range(E))
+            elif rep == 1:
+                S = set(range(max(1, k - 2)))           # fewer eligible experts than k
+            else:
+                S = {e for e in range(E) if rng.random() < 0.3} | {0}
+            mask = set_to_mask(S, E)
+            idx, w = ctx.route_restricted(torch.tensor(z, device=DEV), torch.tensor(mask.view(np.int32), device=DEV))
+            io, wo = oracle.route_restricted(z, mask, k, weighting, 1.5)
+            np.testing.assert_array_equal(idx.cpu().numpy(), io)
+            np.testing.assert_allclose(w.cpu().numpy(), wo, rtol=1e-5, atol=1e-7)
+            if rep == 0:
+                np.testing.assert_array_equal(idx.cpu().numpy(), nat)      # S = [E] is natural routing
+        ctx.close()
+
+
+FFN_SHAPES = [
+    # (T, H, I, E, k, n_shared)
+    (64, 256, 128, 8, 2, 0),
+    (16, 128, 64, 4, 1, 0),
+    (37, 512, 192, 12, 4, 0),       # ragged node count
+    (48, 256, 320, 16, 6, 2),       # shared experts, intermediate not a power of two
+    (1, 128, 64, 4, 2, 0),
+    (64, 2048, 768, 128, 8, 0),     # the Qwen3-30B-A3B layer shape
+]
+
+
+@pytest.mark.parametrize("T,H,I,E,k,ns", FFN_SHAPES)
+def test_expert_ffn_against_oracle(T, H, I, E, k, ns):
+    cfg = wl.scaled(wl.CONFIGS[3], hidden=H, inter=I, n_experts=E, top_k=k, n_shared=ns, n_nodes=T, zipf_bias=False)
+    w = wl.layer_weights(cfg, 7, DEV)
+    # larger weights than the recipe's so that outputs are O(1) and errors are visible
+    x = wl.hidden_states(cfg, 7, DEV)
+    rng = np.random.default_rng(T + E)
+    idx = np.array([rng.permutation(E)[:k] for _ in range(T)], dtype=np.int32)
+    if T > 2:
+        idx[1, -1] = -1                                # an empty slot
+    wt = rng.uniform(0.05, 1.0, (T, k)).astype(np.float32)
+    ctx = _ctx(cfg)
+    _set_weights(ctx, w)
+    out = ctx.expert_ffn(0, x, torch.tensor(idx, device=DEV), torch.tensor(wt, device=DEV))
+    assert ctx.device_status() == acm.OK
+    rows = np.arange(T) if T * E <= 2048 else np.array(sorted(rng.choice(T, 12, replace=False)))
+    ref = oracle.expert_ffn(_take(x, rows), idx[rows], wt[rows].astype(np.float64), w["gate_up"], w["down"],
+                            w["shared_gate_up"], w["shared_down"])
+    _ffn_check(_take(out, rows), ref, f"ffn {T}x{H}x{I}")
+    # twice in a row on the same context: workspace flags and counters are re-armed correctly
+    out2 = ctx.expert_ffn(0, x, torch.tensor(idx, device=DEV), torch.tensor(wt, device=DEV))
+    _ffn_check(_take(out2, rows), ref, "second call")
+    ctx.close()
+
+
+def test_expert_ffn_fp32_toy():
+    cfg = wl.CONFIGS[1]
+    w = wl.layer_weights(cfg, 0, DEV)
+    x = wl.hidden_states(cfg, 0, DEV)
+    rng = np.random.default_rng(0)
+    idx = np.array([rng.permutation(cfg.n_experts)[:2] for _ in range(cfg.n_nodes)], dtype=np.int32)
+    wt = rng.uniform(0.1, 1.0, idx.shape).astype(np.float32)
+    ctx = _ctx(cfg)
+    _set_weights(ctx, w)
+    out = ctx.expert_ffn(0, x, torch.tensor(idx, device=DEV), torch.tensor(wt, device=DEV))
+    ref = oracle.expert_ffn(x, idx, wt.astype(np.float64), w["gate_up"], w["down"])
+    assert _ffn_check(out, ref, "fp32 toy") < 1e-4
+    ctx.close()
+
+
+def _verify_layer(cfg, layer, ctx, slot, params_kw=None, rows=None, natural=False):
+    w, x, alpha = _block(cfg, layer)
+    _set_weights(ctx, w, slot)
+    E = cfg.n_experts
+    pk = params_kw or {}
+    if natural:
+        mo = torch.tensor(full_mask(E).view(np.int32), device=DEV)
+        out, idx, wt, mask, stats = ctx.moe_verify(slot, x, None, None, mask_override=mo, want=True)
+        ref = oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha.numpy(),
+                                cfg.top_k, weighting=cfg.weighting, shared_gate_up=w["shared_gate_up"],
+                                shared_down=w["shared_down"], mask_override=full_mask(E), with_ffn=False)
+    else:
+        out, idx, wt, mask, stats = ctx.moe_verify(slot, x, alpha.to(DEV), acm.SelectParams(**pk), want=True)
+        ref = oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha.numpy(),
+                                cfg.top_k, oracle.SelectParams(**pk), weighting=cfg.weighting,
+                                shared_gate_up=w["shared_gate_up"], shared_down=w["shared_down"], with_ffn=False)
+    assert ctx.device_status() == acm.OK
+    np.testing.assert_array_equal(_u32(mask), ref["mask"])
+    np.testing.assert_array_equal(idx.cpu().numpy(), ref["idx"])
+    np.testing.assert_allclose(wt.cpu().numpy(), ref["w"], rtol=1e-5, atol=1e-7)
+    st = acm.stats_dict(stats)
+    if not natural:
+        assert st["n_eligible_pruned"] == ref["count"]
+        for key in ("n_anchor", "n_er", "n_eligible", "n_natural_union", "displaced_aS"):
+            assert st[key] == ref["stats"][key]
+    assert st["n_activated"] == len(set(ref["idx"].ravel()) - {-1})
+    rows = np.arange(cfg.n_nodes) if rows is None else np.asarray(rows)
+    ffn = oracle.expert_ffn(_take(x, rows), ref["idx"][rows], ref["w"][rows], w["gate_up"], w["down"],
+                            w["shared_gate_up"], w["shared_down"])
+    rel = _ffn_check(_take(out, rows), ffn, f"C{cfg.index} layer {layer}")
+    return st, rel
+
+
+def test_config1_toy_fp32_end_to_end():
+    cfg = wl.CONFIGS[1]
+    ctx = _ctx(cfg)
+    st, rel = _verify_layer(cfg, 0, ctx, 0)
+    assert rel < 1e-4 and st["n_anchor"] == 2
+    _verify_layer(cfg, 0, ctx, 0, natural=True)
+    ctx.close()
+
+
+@pytest.mark.parametrize("c", [2, 3, 4])
+def test_full_size_configs_end_to_end(c):
+    """Full layer shapes of the OLMoE-, Qwen3-30B-A3B- and DeepSeek-V2-Lite-shaped configurations:
+    sets, routes and weights on every node; FFN outputs on sampled nodes the oracle computes one by one."""
+    cfg = wl.CONFIGS[c]
+    ctx = _ctx(cfg, n_layers=2)
+    sample = [0, 1, cfg.n_nodes // 2, cfg.n_nodes - 1]
+    sizes = []
+    for layer in (0, cfg.n_layers - 1):
+        st, _ = _verify_layer(cfg, layer, ctx, layer % 2, rows=sample)
+        sizes.append(st["n_eligible_pruned"])
+    _verify_layer(cfg, 1, ctx, 1, rows=sample, natural=True)
+    if c == 3:
+        assert all(10 <= s <= 45 for s in sizes), sizes     # skewed routing: the set is far below E
+    ctx.close()
+
+
+def test_selection_and_routing_on_every_layer_of_the_qwen3_30b_stack():
+    cfg = wl.CONFIGS[3]
+    ctx = _ctx(cfg)
+    depth, p = wl.tree_depths(cfg), wl.commitment_table(cfg)
+    alpha = acm.node_weights(depth, p)
+    alpha_dev = alpha.to(DEV)
+    for layer in range(cfg.n_layers):
+        w = wl.layer_weights(cfg, layer, DEV, experts=False)
+        x = wl.hidden_states(cfg, layer, DEV)
+        ctx.set_layer_weights(0, w["w_router"], w["router_bias"], None, None)
+        z, r, nat = ctx.router(0, x)
+        sel = ctx.select_eligible(r, nat, alpha_dev)
+        idx, wt = ctx.route_restricted(z, sel["mask"])
+        ref = oracle.moe_verify(x, w["w_router"], w["router_bias"], None, None, alpha.numpy(), cfg.top_k,
+                                weighting=cfg.weighting, with_ffn=False)
+        np.testing.assert_array_equal(z.cpu().numpy(), ref["logits"])
+        np.testing.assert_array_equal(_u32(sel["mask"]), ref["mask"])
+        np.testing.assert_array_equal(idx.cpu().numpy(), ref["idx"])
+    ctx.close()
+
+
+def test_invalid_arguments_are_rejected_on_the_host():
+    cfg = wl.scaled(wl.CONFIGS[3], hidden=256, inter=64, n_experts=8, top_k=2, n_nodes=8, zipf_bias=False)
+    w, x, alpha = _block(cfg)
+    ctx = _ctx(cfg)
+    out = torch.full((8, 256), 7.0, device=DEV)
+    with pytest.raises(acm.AcmError) as e:          # weights not registered yet
+        ctx.moe_verify(0, x, alpha.to(DEV), out=out)
+    assert e.value.code == acm.ERR_INVALID
+    _set_weights(ctx, w)
+    for bad in (lambda: ctx.moe_verify(3, x, alpha.to(DEV), out=out),                    # layer out of range
+                lambda: ctx.moe_verify(0, x[:0], alpha.to(DEV), out=out),                # T = 0
+                lambda: ctx.moe_verify(0, x, None, out=out),                             # alpha missing
+                lambda: ctx.moe_verify(0, x, alpha.to(DEV), acm.SelectParams(demand=5), out=out),
+                lambda: ctx.moe_verify(0, x, alpha.to(DEV), acm.SelectParams(residency=1), out=out),
+                lambda: ctx.moe_verify(0, x.view(-1)[1:1 + 7 * 256].view(7, 256), alpha.to(DEV), out=out)):  # misaligned x
+        with pytest.raises(acm.AcmError) as e:
+            bad()
+        assert e.value.code == acm.ERR_INVALID
+    torch.cuda.synchronize()
+    assert bool((out == 7.0).all())                  # outputs untouched by rejected calls
+    ctx.close()
+
+
+def test_deterministic_selection_and_routing_across_runs():
+    cfg = wl.CONFIGS[3]
+    w, x, alpha = _block(cfg, 5)
+    ctx = _ctx(cfg)
+    _set_weights(ctx, w)
+    a = ctx.moe_verify(0, x, alpha.to(DEV), want=True)
+    b = ctx.moe_verify(0, x, alpha.to(DEV), want=True)
+    torch.cuda.synchronize()
+    assert torch.equal(a[1], b[1]) and torch.equal(a[3], b[3]) and torch.equal(a[2], b[2])
+    assert float((a[0] - b[0]).abs().max()) <= 1e-3 * float(a[0].abs().max())
+    ctx.close()
