@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the verifier-side MoE layer (one JSON line on stdout).
+
+A step is one verification block through the whole hot path (router, selection, restricted
+routing, expert FFN) of every layer of the configuration's stack, layers back to back with
+distinct weights so that expert weights stream cold from HBM.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--layers L] [--impl reference]
+
+metric  verify-blocks/s per MoE layer = (layers x steps) / time, summed over replicas.
+N > 1   independent replicas (the path has no sharding and no collective): one rank per GPU
+        under torchrun, barrier + max-over-ranks timing.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "verify_blocks_per_s_per_moe_layer"
+UNIT = "layer-blocks/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=3, help="1..5; default 3 = Qwen3-30B-A3B-shaped stack")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of stacked layers (0 = the config's)")
+    ap.add_argument("--impl", default="acm", choices=["acm", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-natural", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def read_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            f = [v.strip() for v in s.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                smax = float(f[1])
+            except ValueError:
+                continue
+            for name, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        # the clock rises only under load: report the median of the upper half of the samples
+        busy = sm[len(sm) // 2:] if sm else []
+        med = busy[len(busy) // 2] if busy else None
+        return {"sm_mhz": med, "sm_max_mhz": smax, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def dist_setup(args):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return world, rank, local
+
+
+# ------------------------------------------------------------------------------------------
+def run_reference(args, world, rank):
+    """The CPU oracle as the reference arm: each step is a bounded sample of the workload."""
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    from paper_2608_02989_b200 import workloads as wl
+
+    cfg = wl.CONFIGS[args.config]
+    sample_layers = 1
+    sample_nodes = min(cfg.n_nodes, 16)
+    depth, p = wl.tree_depths(cfg), wl.commitment_table(cfg)
+    alpha = oracle.node_weights(depth.numpy(), p.numpy())
+    w = wl.layer_weights(cfg, 0, "cpu")
+    x = wl.hidden_states(cfg, 0, "cpu")
+    cores = os.cpu_count() or 1
+
+    def one_step():
+        res = oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha, cfg.top_k,
+                                weighting=cfg.weighting, shared_gate_up=w["shared_gate_up"],
+                                shared_down=w["shared_down"], with_ffn=False)
+        rows = np.arange(sample_nodes)
+        oracle.expert_ffn(x[:sample_nodes], res["idx"][rows], res["w"][rows], w["gate_up"], w["down"],
+                          w["shared_gate_up"], w["shared_down"])
+
+    for _ in range(max(args.warmup, 1)):
+        one_step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one_step()
+    dt = time.perf_counter() - t0
+    # a step covered sample_layers layers with sample_nodes of n_nodes nodes in the FFN: scale to whole blocks
+    frac = sample_nodes / cfg.n_nodes
+    value = sample_layers * args.steps * frac / dt
+    sample = (f"{sample_layers} layer of C{cfg.index}: router/selection/routing on all {cfg.n_nodes} nodes, expert FFN on "
+              f"the first {sample_nodes} nodes; layer-blocks/s scaled by {frac:.3f}")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": f"C{cfg.index} {cfg.name}-shaped", "hidden": cfg.hidden, "n_experts": cfg.n_experts,
+                   "top_k": cfg.top_k, "inter": cfg.inter, "n_nodes": cfg.n_nodes, "layers": sample_layers},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+def cpu_baseline(cfg, budget_s=20.0):
+    """Times the oracle, as it stands, on the host cores for a bounded sample of the workload."""
+    import numpy as np
+    import oracle
+    from paper_2608_02989_b200 import workloads as wl
+
+    depth, p = wl.tree_depths(cfg), wl.commitment_table(cfg)
+    alpha = oracle.node_weights(depth.numpy(), p.numpy())
+    w = wl.layer_weights(cfg, 0, "cpu")
+    x = wl.hidden_states(cfg, 0, "cpu")
+    nodes = min(cfg.n_nodes, 16)
+    t0 = time.perf_counter()
+    done = 0
+    while True:
+        res = oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha, cfg.top_k,
+                                weighting=cfg.weighting, shared_gate_up=w["shared_gate_up"],
+                                shared_down=w["shared_down"], with_ffn=False)
+        rows = np.arange(nodes)
+        oracle.expert_ffn(x[:nodes], res["idx"][rows], res["w"][rows], w["gate_up"], w["down"],
+                          w["shared_gate_up"], w["shared_down"])
+        done += 1
+        dt = time.perf_counter() - t0
+        if dt > budget_s / 2 or done >= 8:
+            break
+    frac = nodes / cfg.n_nodes
+    return {"value": done * frac / dt, "unit": UNIT, "cores": os.cpu_count() or 1, "kind": "oracle",
+            "sample": (f"{done} pass(es) over layer 0 of C{cfg.index}: router/selection/routing on all {cfg.n_nodes} "
+                       f"nodes + expert FFN on the first {nodes} nodes, scaled by {frac:.3f}; {dt:.1f} s wall")}
+
+
+def run_acm(args, world, rank, local):
+    import ctypes
+
+    import torch
+
+    from paper_2608_02989_b200 import acm, workloads as wl
+    from paper_2608_02989_b200 import build as acm_build
+
+    acm_build.build_library()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    cfg = wl.CONFIGS[args.config]
+    L = args.layers or cfg.n_layers
+    resident = cfg.resident_frac > 0
+    if resident:
+        # the full stack does not fit in HBM: as many physical layers as fit, reused cyclically
+        free, _ = torch.cuda.mem_get_info()
+        L_phys = max(1, min(L, int(0.6 * free // wl.weight_bytes_per_layer(cfg))))
+    else:
+        L_phys = L
+    T, H, E, k = cfg.n_nodes, cfg.hidden, cfg.n_experts, cfg.top_k
+
+    ctx = acm.Context.for_config(cfg, n_layers=L_phys)
+    keep = []
+    for l in range(L_phys):
+        w = wl.layer_weights(cfg, l + 1000 * rank, dev)
+        ctx.set_layer_weights(l, w["w_router"], w["router_bias"], w["gate_up"], w["down"], w["shared_gate_up"],
+                              w["shared_down"])
+        keep.append(w)
+    xs = torch.stack([wl.hidden_states(cfg, l + 1000 * rank, dev) for l in range(L)])       # [L,T,H]
+    depth, p = wl.tree_depths(cfg), wl.commitment_table(cfg)
+    alpha = acm.node_weights(depth, p)
+    alpha_dev = alpha.to(dev)
+    outs = torch.zeros(L, T, H, dtype=torch.float32, device=dev)
+    stats = torch.zeros(L, 12, dtype=torch.int32, device=dev)
+    full = torch.full((ctx.words,), -1, dtype=torch.int32, device=dev)
+    params = acm.SelectParams()
+    stream = torch.cuda.current_stream()
+    sp = ctypes.c_void_p(stream.cuda_stream)
+    lib, h = ctx.lib, ctx.handle
+
+    def vp(t):
+        return ctypes.c_void_p(t.data_ptr())
+
+    # argument tuples prepared once: the timed loop is C calls only
+    calls_sel = [(h, l % L_phys, vp(xs[l]), T, vp(alpha_dev), ctypes.byref(params), None, vp(outs[l]), None, None,
+                  None, vp(stats[l]), sp) for l in range(L)]
+    calls_nat = [(h, l % L_phys, vp(xs[l]), T, None, None, vp(full), vp(outs[l]), None, None, None, vp(stats[l]), sp)
+                 for l in range(L)]
+
+    def step(calls):
+        for a in calls:
+            rc = lib.acm_moe_verify(*a)
+            if rc:
+                raise acm.AcmError(rc, "acm_moe_verify")
+
+    def timed(calls, steps, warmup, with_roofline):
+        for _ in range(warmup):
+            step(calls)
+        barrier()
+        if with_roofline:
+            ctx.ffn_timing(True, steps * L * 2)
+        n0 = ctx.launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            step(calls)
+        e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        launches = ctx.launch_count() - n0
+        ffn_ms, ffn_n = (ctx.ffn_time_ms() if with_roofline else (0.0, 0))
+        ctx.ffn_timing(False)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t)
+        return ms, launches, ffn_ms, ffn_n
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms, launches, ffn_ms, ffn_n = timed(calls_sel, args.steps, max(args.warmup, 3), True)
+    clocks = sampler.stop() if rank == 0 else None
+    ctx.check_device_status()
+    st = stats.cpu().numpy()
+    n_act = st[:, 4].astype(float)
+    expert_bytes = cfg.expert_bytes
+    # algorithmic bytes of one FFN launch: the activated experts' weights (+ shared), x in, y out
+    alg_bytes = (n_act + cfg.n_shared) * expert_bytes + T * H * 2 + T * H * 4
+    alg_per_launch = float(alg_bytes.mean())
+    value = world * L * args.steps / (ms * 1e-3)
+
+    nat = None
+    if not args.no_natural:
+        ms_n, _, ffn_ms_n, ffn_n_n = timed(calls_nat, args.steps, 3, True)
+        st_n = stats.cpu().numpy()
+        nat_bytes = float(((st_n[:, 4] + cfg.n_shared) * expert_bytes + T * H * 6).mean())
+        nat = {"value": world * L * args.steps / (ms_n * 1e-3), "unit": UNIT, "ms_per_step": ms_n / args.steps,
+               "mean_activated_experts": float(st_n[:, 4].mean()),
+               "ffn_us_per_launch": 1e3 * ffn_ms_n / max(ffn_n_n, 1),
+               "ffn_gbs": nat_bytes / (1e6 * ffn_ms_n / max(ffn_n_n, 1)) if ffn_n_n else None}
+
+    e2e = None
+    if not args.no_e2e:
+        # the same calls with host buffers: pinned x in, pinned y out, copies inside the timed region
+        xs_host = xs.cpu().pin_memory()
+        alpha_host = alpha.pin_memory()
+        outs_host = torch.zeros(L, T, H, dtype=torch.float32).pin_memory()
+        x_dev = torch.empty_like(xs[0])
+        a_dev = torch.empty_like(alpha_dev)
+        o_dev = torch.empty_like(outs[0])
+
+        def e2e_step():
+            for l in range(L):
+                x_dev.copy_(xs_host[l], non_blocking=True)
+                a_dev.copy_(alpha_host, non_blocking=True)
+                rc = lib.acm_moe_verify(h, l % L_phys, vp(x_dev), T, vp(a_dev), ctypes.byref(params), None, vp(o_dev),
+                                        None, None, None, None, sp)
+                if rc:
+                    raise acm.AcmError(rc, "acm_moe_verify")
+                outs_host[l].copy_(o_dev, non_blocking=True)
+            stream.synchronize()      # the step's result is on the host
+
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            e2e_step()
+        barrier()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t)
+        e2e = {"value": world * L * args.steps / dt, "unit": UNIT,
+               "h2d_bytes_per_step": L * (T * H * cfg.elt_bytes + T * 4), "d2h_bytes_per_step": L * T * H * 4}
+
+    if rank != 0:
+        return
+    peak, peak_kind = read_peaks()
+    ffn_us = 1e3 * ffn_ms / max(ffn_n, 1)
+    achieved = alg_per_launch / (ffn_us * 1e-6) / 1e9 if ffn_n else None
+    traffic = None
+    prof = ROOT / "profiles" / "ffn_traffic.json"
+    if prof.exists():
+        try:
+            d = json.loads(prof.read_text())
+            # DRAM bytes per launch from an ncu capture, scaled by the activated experts of this run
+            traffic = d["dram_bytes_per_activated_expert"] * float(n_act.mean() + cfg.n_shared)
+        except (KeyError, ValueError):
+            traffic = None
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": f"C{cfg.index} {cfg.name}-shaped stack, restricted (AcceptMoE) routing",
+                   "hidden": H, "n_experts": E, "top_k": k, "inter": cfg.inter, "n_shared": cfg.n_shared,
+                   "n_nodes": T, "layers": L, "physical_layers": L_phys,
+                   "l2": f"inputs larger than L2: {L_phys} distinct layers, "
+                         f"{alg_per_launch * L_phys / 1e9:.1f} GB of expert weights streamed per step",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "us_per_layer": 1e3 * ms / (args.steps * L),
+        "mean_eligible": float(st[:, 3].mean()), "mean_activated": float(n_act.mean()),
+        "mean_natural_union": float(st[:, 5].mean()),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": (achieved / peak) if achieved else None, "traffic": traffic, "peak_kind": peak_kind,
+                     "kernel": "k_ffn_bf16", "us_per_launch": ffn_us, "launches_timed": ffn_n,
+                     "algorithmic_bytes_per_launch": alg_per_launch},
+        "natural_union_path": nat,
+        "e2e": e2e,
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(cfg)
+    print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    world, rank, local = dist_setup(args)
+    if args.impl == "reference":
+        run_reference(args, world, rank)
+        return
+    run_acm(args, world, rank, local)
+
+
+if __name__ == "__main__":
+    main()
