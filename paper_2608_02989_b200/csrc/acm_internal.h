@@ -49,8 +49,8 @@ struct Workspace {
   WorkList* lists;      // [2]: 0 = resident + shared, 1 = staged
   float* wdense;        // [2][kMaxSlots][64]
   void* hbuf;           // [2][kMaxSlots][64][I] bf16 (f32 path: [T][k+ns][I] float)
-  float* frag;          // [grid][128*64] split-K fragments
-  int32_t* frag_flag;   // [grid] epoch of the fragment stored there
+  float* frag;          // [2][grid][128*64] split-K fragments (one buffer per gate/up segment)
+  int32_t* frag_flag;   // [2][grid] epoch of the fragment stored there
   int32_t* ready;       // [2][kMaxSlots] finished gate/up tiles per activated slot
   int32_t* status;      // [1] sticky device-side status
 };
@@ -122,6 +122,7 @@ struct FfnLaunch {
   int32_t* status;
   int grid;
   int phase_mask;            // 1 = gate/up, 2 = down, 3 = both in one launch
+  unsigned long long* trace; // optional [grid][32] device timestamps (debugging aid) or null
 };
 cudaError_t ffn_configure();   // one-time function attributes
 size_t ffn_smem_bytes();

@@ -61,6 +61,7 @@ struct acm_ctx {
   size_t ev_used = 0;
   uint64_t launches = 0;
   bool split_phases = false;             // ACM_FFN_SPLIT_PHASES=1 in the environment
+  unsigned long long* trace = nullptr;   // ACM_FFN_TRACE=1: per-CTA timestamps of the last FFN launch
 };
 
 namespace {
@@ -167,6 +168,8 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   p.out = out; p.status = c->ws.status;
   p.grid = c->sm_count;
   p.phase_mask = 3;
+  p.trace = c->trace;
+  if (c->trace) ACM_CUDA(cudaMemsetAsync(c->trace, 0, sizeof(unsigned long long) * 32 * c->sm_count, s));
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   if (c->timing && c->ev_used + 2 <= c->ev_pool.size()) {
     e0 = c->ev_pool[c->ev_used];
@@ -224,6 +227,16 @@ void acm_default_select_params(acm_select_params* p) {
   p->max_remove = kMaxExperts;
 }
 
+// Debugging aid (not part of the public header): copies the per-CTA timestamps of the last FFN
+// launch to `host_out` ([sm_count][32] uint64).  Needs ACM_FFN_TRACE=1 at context creation.
+acm_status acm_debug_ffn_trace(acm_ctx* c, unsigned long long* host_out, int* n_ctas) {
+  if (!c || !host_out || !n_ctas || !c->trace) return ACM_ERR_INVALID;
+  ACM_CUDA(cudaDeviceSynchronize());
+  ACM_CUDA(cudaMemcpy(host_out, c->trace, sizeof(unsigned long long) * 32 * c->sm_count, cudaMemcpyDeviceToHost));
+  *n_ctas = c->sm_count;
+  return ACM_OK;
+}
+
 const char* acm_status_string(acm_status s) {
   switch (s) {
     case ACM_OK: return "ok";
@@ -248,6 +261,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->layers.resize(desc->n_layers);
   const char* split = std::getenv("ACM_FFN_SPLIT_PHASES");
   c->split_phases = split && split[0] == '1';
+  const char* trace = std::getenv("ACM_FFN_TRACE");
+  const bool want_trace = trace && trace[0] == '1';
   auto fail = [&](acm_status s) {
     acm_destroy(c);
     return s;
@@ -284,8 +299,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t hbuf_bf16 = static_cast<size_t>(2) * kMaxSlots * kMaxNodes * I * 2;
   const size_t hbuf_f32 = static_cast<size_t>(Tm) * (k + desc->n_shared) * I * 4;
   const size_t o_h = carve(hbuf_bf16 > hbuf_f32 ? hbuf_bf16 : hbuf_f32);
-  const size_t o_frag = carve(sizeof(float) * static_cast<size_t>(c->sm_count) * 128 * kMaxNodes);
-  const size_t o_flag = carve(sizeof(int32_t) * c->sm_count);
+  const size_t o_frag = carve(sizeof(float) * 2 * static_cast<size_t>(c->sm_count) * 128 * kMaxNodes);
+  const size_t o_flag = carve(sizeof(int32_t) * 2 * c->sm_count);
   const size_t o_ready = carve(sizeof(int32_t) * 2 * kMaxSlots);
   const size_t o_status = carve(16);
   const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
@@ -310,6 +325,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.ready = reinterpret_cast<int32_t*>(b + o_ready);
   c->ws.status = reinterpret_cast<int32_t*>(b + o_status);
   c->resident_dev = reinterpret_cast<uint32_t*>(b + o_res);
+  if (want_trace && cudaMalloc(&c->trace, sizeof(unsigned long long) * 32 * c->sm_count) != cudaSuccess)
+    return fail(ACM_ERR_NOMEM);
   *out = c;
   return ACM_OK;
 }
@@ -326,6 +343,7 @@ acm_status acm_destroy(acm_ctx* c) {
   if (c->stage_gate_up) cudaFree(c->stage_gate_up);
   if (c->stage_down) cudaFree(c->stage_down);
   if (c->ws_base) cudaFree(c->ws_base);
+  if (c->trace) cudaFree(c->trace);
   delete c;
   return ACM_OK;
 }

@@ -26,7 +26,14 @@
 namespace acm {
 namespace {
 
-constexpr int kStages = 8;
+#ifndef ACM_FFN_STAGES
+#define ACM_FFN_STAGES 7
+#endif
+#ifndef ACM_FFN_ACC
+#define ACM_FFN_ACC 4
+#endif
+constexpr int kStages = ACM_FFN_STAGES;
+constexpr int kAcc = ACM_FFN_ACC;                        // TMEM accumulators in flight (power of two)
 constexpr int kBK = 64;                                  // K elements per stage (one 128-byte swizzle row)
 constexpr int kTileM = 128;
 constexpr int kABytes = kTileM * kBK * 2;                // 16 KB weight tile
@@ -34,22 +41,29 @@ constexpr int kBBytesMax = kMaxNodes * kBK * 2;          // 8 KB activation chun
 constexpr int kStageBytes = kABytes + kBBytesMax;
 constexpr int kExBytes = 64 * kMaxNodes * 4;             // up-projection exchange buffer
 constexpr int kAccCols = kMaxNodes;                      // TMEM columns per accumulator
-constexpr int kTmemCols = 128;                           // two accumulators
-constexpr int kThreads = 192;
+constexpr int kTmemCols = kAcc * kAccCols;
+constexpr int kThreads = 224;                            // producer, MMA, 4 epilogue warps, helper warp
+constexpr int kFragBytes = kTileM * kMaxNodes * 4;       // contributor fragments pre-summed in shared memory
 constexpr int kFragFloats = kTileM * kMaxNodes;
 constexpr unsigned long long kTimeoutNs = 1000ull * 1000ull * 1000ull;
 
 struct __align__(8) Barriers {
   unsigned long long full[kStages];
   unsigned long long empty[kStages];
-  unsigned long long tfull[2];
-  unsigned long long tempty[2];
+  unsigned long long tfull[kAcc];
+  unsigned long long tempty[kAcc];
   unsigned long long drained;
+  unsigned long long frag_full[2];   // helper -> epilogue: pre-summed fragments of gate/up segment i are in smem
+  unsigned long long frag_free;      // epilogue -> helper: the fragment buffer may be overwritten
+  unsigned long long helper;         // completion of the helper warp's bulk copy
+  volatile uint32_t armed;           // stages whose barrier the weight producer has armed so far
   uint32_t tmem_base;
   int abort_flag;
+  float wd[kMaxNodes];          // combine weights of the expert being finalised
+  int32_t entry[kMaxSlots];     // this launch's work list (copied from global memory once)
 };
 
-constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + kExBytes + sizeof(Barriers);
+constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + kExBytes + kFragBytes + sizeof(Barriers);
 
 // ---------------------------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -72,6 +86,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {   // never blocks
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}\n"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
@@ -232,6 +255,9 @@ struct Sched {
   }
 };
 
+#define ACM_TRACE(slot) do { if (p.trace) p.trace[static_cast<size_t>(blockIdx.x) * 32 + (slot)] = global_timer(); } while (0)
+#define ACM_TRACE_ADD(slot, dt) do { if (p.trace) p.trace[static_cast<size_t>(blockIdx.x) * 32 + (slot)] += (dt); } while (0)
+
 struct FfnArgs {
   int T, H, I, n_pad;
   const WorkList* list;
@@ -244,11 +270,36 @@ struct FfnArgs {
   float* out;
   int32_t* status;
   int phase_mask;
+  unsigned long long* trace;   // optional [grid][32] timestamps (debugging aid), may be null
 };
 
 __device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMap* routed, const CUtensorMap* shared,
                                                        const CUtensorMap* staged) {
   return src == kSrcRouted ? routed : src == kSrcShared ? shared : staged;
+}
+
+// The stream of one launch is cut into up to four segments, executed in this order by every CTA:
+//   gate/up of expert group A, gate/up of group B, down of group A, down of group B
+// (A = first half of the activated experts).  While a CTA streams the second segment, the
+// epilogues of the first finish in the background, so the down projection of group A never
+// waits for its activations; likewise group B's are ready by the time group A's down is through.
+struct Segment {
+  int phase;      // 1 = gate/up, 2 = down
+  int a0, a1;     // activated-expert slots [a0, a1)
+  int p1_index;   // expert group: fragment buffer / completion counter of its gate/up segment (0 or 1)
+};
+__device__ __forceinline__ int make_segments(int n_act, int phase_mask, Segment* seg) {
+  const int nA = (n_act + 1) / 2;
+  int n = 0;
+  if (phase_mask & 1) {
+    if (nA > 0) seg[n++] = Segment{1, 0, nA, 0};
+    if (n_act > nA) seg[n++] = Segment{1, nA, n_act, 1};
+  }
+  if (phase_mask & 2) {
+    if (nA > 0) seg[n++] = Segment{2, 0, nA, 0};
+    if (n_act > nA) seg[n++] = Segment{2, nA, n_act, 1};
+  }
+  return n;
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -258,29 +309,38 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   unsigned char* stage_base = smem;
   float* ex = reinterpret_cast<float*>(smem + static_cast<size_t>(kStages) * kStageBytes);
-  Barriers* bars = reinterpret_cast<Barriers*>(smem + static_cast<size_t>(kStages) * kStageBytes + kExBytes);
+  float* sfrag = reinterpret_cast<float*>(smem + static_cast<size_t>(kStages) * kStageBytes + kExBytes);
+  Barriers* bars = reinterpret_cast<Barriers*>(smem + static_cast<size_t>(kStages) * kStageBytes + kExBytes + kFragBytes);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, G = gridDim.x;
   const int n_act = p.list->n;
-  const int tpe = p.I / 64;          // gate/up tiles per expert = K-chunks per expert in phase 2
-  const int kc1 = p.H / kBK;         // K-chunks of a phase-1 tile
-  const int h_tiles = p.H / kTileM;  // output tiles of phase 2
-  const int kc2 = n_act * tpe;       // K-chunks of a phase-2 tile
+  const int tpe = p.I / 64;          // gate/up tiles per expert = K-chunks per expert in the down phase
+  const int kc1 = p.H / kBK;         // K-chunks of a gate/up tile
+  const int h_tiles = p.H / kTileM;  // output tiles of the down phase
   const uint32_t b_bytes = static_cast<uint32_t>(p.n_pad) * kBK * 2;
+  Segment seg[4];
+  const int n_seg = make_segments(n_act, p.phase_mask, seg);
+  int32_t* s_entry = bars->entry;
+  for (int i = threadIdx.x; i < n_act; i += blockDim.x) s_entry[i] = p.list->entry[i];
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&bars->full[s]), 1);
       mbar_init(smem_u32(&bars->empty[s]), 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < kAcc; ++b) {
       mbar_init(smem_u32(&bars->tfull[b]), 1);
       mbar_init(smem_u32(&bars->tempty[b]), 128);
     }
     mbar_init(smem_u32(&bars->drained), 1);
+    mbar_init(smem_u32(&bars->frag_full[0]), 1);
+    mbar_init(smem_u32(&bars->frag_full[1]), 1);
+    mbar_init(smem_u32(&bars->frag_free), 128);
+    mbar_init(smem_u32(&bars->helper), 1);
     bars->abort_flag = 0;
+    bars->armed = 0;
     fence_barrier_init();
   }
   if (warp == 0 && lane == 0) {
@@ -297,54 +357,67 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
+  if (threadIdx.x == 0) ACM_TRACE(0);
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ weight producer
+    // Streams every weight tile of this CTA (and the x chunk of gate/up stages).  It arms each
+    // stage's barrier with the bytes of both operands; the activation chunk of a down stage is
+    // added by the helper warp once that expert group is complete, so this stream never stalls on
+    // it.  The loop is kept to a few instructions per stage: one thread pays every one of them.
     if (lane == 0) {
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
-      uint32_t it = 0;
-      bool ok = true;
-      if (p.phase_mask & 1) {
-        Sched s1(cta, G, static_cast<long long>(n_act) * tpe, kc1);
-        int tile, k0, k1;
-        while (ok && s1.next(tile, k0, k1)) {
-          const int a = tile / tpe, ti = tile % tpe;
-          const int32_t ent = p.list->entry[a];
-          const CUtensorMap* gu = pick_map(entry_src(ent), &maps.gate_up, &maps.shared_gate_up, &maps.staged_gate_up);
-          const int eidx = entry_idx(ent);
-          for (int kc = k0; kc < k1; ++kc, ++it) {
-            const uint32_t s = it % kStages, par = (it / kStages) & 1u;
-            if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
-            const uint32_t full = smem_u32(&bars->full[s]);
-            const uint32_t sa = smem_u32(stage_base + static_cast<size_t>(s) * kStageBytes);
-            mbar_expect_tx(full, kABytes + b_bytes);
-            tma_load_3d(sa, gu, full, kc * kBK, ti * 64, eidx, pol_w);                 // 64 gate rows
-            tma_load_3d(sa + kABytes / 2, gu, full, kc * kBK, p.I + ti * 64, eidx, pol_w);   // 64 up rows
-            tma_load_2d(sa + kABytes, &x_map, full, kc * kBK, 0, pol_x);
-          }
-        }
-      }
-      if (p.phase_mask & 2) {
-        Sched s2(cta, G, h_tiles, kc2);
-        int ht, k0, k1, ready_a = -1;
-        while (ok && s2.next(ht, k0, k1)) {
-          for (int kc = k0; kc < k1; ++kc, ++it) {
-            const int a = kc / tpe, ic = kc % tpe;
-            const int32_t ent = p.list->entry[a];
-            const CUtensorMap* dn = pick_map(entry_src(ent), &maps.down, &maps.shared_down, &maps.staged_down);
-            const uint32_t s = it % kStages, par = (it / kStages) & 1u;
-            if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
-            const uint32_t full = smem_u32(&bars->full[s]);
-            const uint32_t sa = smem_u32(stage_base + static_cast<size_t>(s) * kStageBytes);
-            mbar_expect_tx(full, kABytes + b_bytes);
-            tma_load_3d(sa, dn, full, ic * kBK, ht * kTileM, entry_idx(ent), pol_w);
-            if (a != ready_a) {   // activations of expert slot a are complete once all its tiles are counted
-              if (!(ok = flag_wait_ge(&p.ready[a], tpe, abort_flag, p.status))) break;
-              fence_proxy_async();
-              ready_a = a;
+      uint32_t s = 0, par = 0, n_armed = 0;
+      bool ok = true, traced_first = false;
+      for (int si = 0; si < n_seg && ok; ++si) {
+        const Segment sg = seg[si];
+        const int n_exp = sg.a1 - sg.a0;
+        if (sg.phase == 1) {
+          Sched sc(cta, G, static_cast<long long>(n_exp) * tpe, kc1);
+          int tile, k0, k1;
+          while (ok && sc.next(tile, k0, k1)) {
+            const int32_t ent = s_entry[sg.a0 + tile / tpe];
+            const int r0 = (tile % tpe) * 64, r1 = p.I + r0, eidx = entry_idx(ent);
+            const CUtensorMap* gu = pick_map(entry_src(ent), &maps.gate_up, &maps.shared_gate_up, &maps.staged_gate_up);
+            for (int kc = k0; kc < k1; ++kc) {
+              if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
+              const uint32_t full = smem_u32(&bars->full[s]);
+              const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
+              mbar_expect_tx(full, kABytes + b_bytes);
+              tma_load_3d(sa, gu, full, kc * kBK, r0, eidx, pol_w);                 // 64 gate rows
+              tma_load_3d(sa + kABytes / 2, gu, full, kc * kBK, r1, eidx, pol_w);   // 64 up rows
+              tma_load_2d(sa + kABytes, &x_map, full, kc * kBK, 0, pol_x);
+              if (!traced_first) { ACM_TRACE(1); traced_first = true; }
+              ++n_armed;
+              if (++s == kStages) { s = 0; par ^= 1u; }
             }
-            tma_load_3d(sa + kABytes, &h_map, full, ic * kBK, 0, a, pol_x);
           }
+          ACM_TRACE(sg.p1_index == 0 ? 13 : 2);
+        } else {
+          Sched sc(cta, G, h_tiles, n_exp * tpe);
+          int ht, k0, k1;
+          while (ok && sc.next(ht, k0, k1)) {
+            int a = sg.a0 + k0 / tpe, ic = k0 % tpe;
+            int32_t ent = s_entry[a];
+            const CUtensorMap* dn = pick_map(entry_src(ent), &maps.down, &maps.shared_down, &maps.staged_down);
+            int eidx = entry_idx(ent);
+            for (int kc = k0; kc < k1; ++kc) {
+              if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
+              const uint32_t full = smem_u32(&bars->full[s]);
+              const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
+              mbar_expect_tx(full, kABytes + b_bytes);
+              tma_load_3d(sa, dn, full, ic * kBK, ht * kTileM, eidx, pol_w);
+              bars->armed = ++n_armed;      // the helper warp may now add this stage's activation chunk
+              if (++s == kStages) { s = 0; par ^= 1u; }
+              if (++ic == tpe && kc + 1 < k1) {
+                ic = 0;
+                ent = s_entry[++a];
+                dn = pick_map(entry_src(ent), &maps.down, &maps.shared_down, &maps.staged_down);
+                eidx = entry_idx(ent);
+              }
+            }
+          }
+          ACM_TRACE(sg.p1_index == 0 ? 14 : 5);
         }
       }
       if (!ok) {
@@ -359,18 +432,22 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       const uint32_t idesc = umma_idesc(p.n_pad);
       uint32_t it = 0, f = 0;
       bool ok = true;
-      for (int phase = 1; phase <= 2 && ok; ++phase) {
-        if (!(p.phase_mask & phase)) continue;
-        Sched sc = phase == 1 ? Sched(cta, G, static_cast<long long>(n_act) * tpe, kc1) : Sched(cta, G, h_tiles, kc2);
+      unsigned long long acc_f[2] = {0, 0};
+      for (int si = 0; si < n_seg && ok; ++si) {
+        const Segment sg = seg[si];
+        const int n_exp = sg.a1 - sg.a0;
+        Sched sc = sg.phase == 1 ? Sched(cta, G, static_cast<long long>(n_exp) * tpe, kc1) : Sched(cta, G, h_tiles, n_exp * tpe);
         int tile, k0, k1;
         while (ok && sc.next(tile, k0, k1)) {
-          const uint32_t b = f & 1u;
-          if (!(ok = mbar_wait(smem_u32(&bars->tempty[b]), ((f >> 1) & 1u) ^ 1u, abort_flag, p.status))) break;
+          const uint32_t b = f % kAcc;
+          if (!(ok = mbar_wait(smem_u32(&bars->tempty[b]), ((f / kAcc) & 1u) ^ 1u, abort_flag, p.status))) break;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + b * kAccCols;
           for (int kc = k0; kc < k1; ++kc, ++it) {
             const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+            const unsigned long long tw = p.trace ? global_timer() : 0ull;
             if (!(ok = mbar_wait(smem_u32(&bars->full[s]), par, abort_flag, p.status))) break;
+            if (p.trace) { acc_f[sg.phase - 1] += global_timer() - tw; if (it == 0) ACM_TRACE(6); }
             tc_fence_after();
             const uint32_t sa = smem_u32(stage_base + static_cast<size_t>(s) * kStageBytes);
             const uint64_t da = umma_smem_desc(sa), db = umma_smem_desc(sa + kABytes);
@@ -383,12 +460,136 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           umma_commit(smem_u32(&bars->tfull[b]));
           ++f;
         }
+        ACM_TRACE(6 + sg.phase);
       }
+      ACM_TRACE_ADD(19, acc_f[0]); ACM_TRACE_ADD(20, acc_f[1]);
       if (!ok) {
         // giving up: wait (bounded) for the MMAs already issued before TMEM is released
         umma_commit(smem_u32(&bars->drained));
         const unsigned long long t0 = global_timer();
         while (!mbar_try_wait(smem_u32(&bars->drained), 0) && global_timer() - t0 < 1000000ull) {}
+      }
+    }
+  } else if (warp == 6) {
+    // ------------------------------------------------------------------ helper warp
+    // Keeps slow global round trips off the other roles' paths: (a) for each gate/up segment whose
+    // last fragment is the head of a tile shared with later CTAs, waits for their fragments and sums
+    // them into shared memory; (b) for each down segment, waits until every activation tile of its
+    // expert group has been stored, then tells the producer.
+    bool ok = true;
+    int frag_uses = 0;
+    uint32_t hs = 0, hidx = 0;   // ring slot and running index of the next stage, tracked through the gate/up stages too
+    for (int si = 0; si < n_seg && ok; ++si) {
+      const Segment sg = seg[si];
+      const int n_exp = sg.a1 - sg.a0;
+      if (sg.phase == 1) {
+        const long long tiles = static_cast<long long>(n_exp) * tpe;
+        const long long U1 = tiles * kc1;
+        const long long ub = U1 * cta / G, ue = U1 * (cta + 1) / G;
+        {
+          hidx += static_cast<uint32_t>(ue - ub);
+          hs = hidx % kStages;
+        }
+        if (ue <= ub) continue;
+        const long long last_tile = (ue - 1) / kc1;
+        const long long tile_end = (last_tile + 1) * kc1;
+        const bool head = (last_tile * kc1 >= ub) && (ue < tile_end);   // starts at chunk 0, ends before the tile does
+        if (!head) continue;
+        if (frag_uses > 0) {   // the buffer still holds the previous segment's sum until the epilogue has read it
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->frag_free), (frag_uses - 1) & 1u, abort_flag, p.status));
+          if (!ok) break;
+        }
+        const float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * kFragFloats;
+        const int32_t* frag_flag = p.frag_flag + sg.p1_index * G;
+        const int n_el = p.n_pad * kTileM;
+        bool first = true;
+        for (int c2 = cta + 1; c2 < G && ok; ++c2) {
+          const long long b2 = U1 * c2 / G, e2 = U1 * (c2 + 1) / G;
+          if (b2 >= tile_end) break;
+          if (e2 == b2) continue;
+          bool got = true;
+          if (lane == 0) got = flag_wait_ge(&frag_flag[c2], p.epoch, abort_flag, p.status);
+          ok = __all_sync(0xffffffffu, got);
+          if (!ok) break;
+          const float* src = frag + static_cast<size_t>(c2) * kFragFloats;
+          if (first) {
+            // first contributor: one bulk async copy into shared memory
+            if (lane == 0) {
+              fence_proxy_async();
+              const uint32_t hb = smem_u32(&bars->helper);
+              mbar_expect_tx(hb, static_cast<uint32_t>(n_el) * 4u);
+              asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                           ::"r"(smem_u32(sfrag)), "l"(src), "r"(static_cast<uint32_t>(n_el) * 4u), "r"(hb) : "memory");
+            }
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->helper), frag_uses & 1u, abort_flag, p.status));
+            if (!ok) break;
+            first = false;
+          } else {
+            // further contributors (a tile cut across three or more CTAs): batched loads, then add
+            const float4* src4 = reinterpret_cast<const float4*>(src);
+            float4* dst4 = reinterpret_cast<float4*>(sfrag);
+            for (int i0 = lane; i0 < n_el / 4; i0 += 32 * 8) {
+              float4 x4[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                if (i0 + 32 * j < n_el / 4) x4[j] = __ldcg(src4 + i0 + 32 * j);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                if (i0 + 32 * j < n_el / 4) {
+                  float4 o = dst4[i0 + 32 * j];
+                  o.x += x4[j].x; o.y += x4[j].y; o.z += x4[j].z; o.w += x4[j].w;
+                  dst4[i0 + 32 * j] = o;
+                }
+              }
+            }
+          }
+        }
+        if (!ok) break;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->frag_full[sg.p1_index]));
+        if (lane == 0) ACM_TRACE(sg.p1_index == 0 ? 9 : 15);
+        ++frag_uses;
+      } else {
+        // activation producer: once every activation tile of this expert group is stored, add the
+        // activation chunk of each down stage to the barrier the weight producer has armed (or will arm)
+        bool good = true;
+        if (lane == 0) {
+          const uint64_t pol_x = policy_evict_last();
+          Sched sc(cta, G, h_tiles, n_exp * tpe);
+          int ht, k0, k1;
+          bool polled = false;
+          while (good && sc.next(ht, k0, k1)) {
+            int a = sg.a0 + k0 / tpe, ic = k0 % tpe;
+            for (int kc = k0; kc < k1; ++kc) {
+              if (!polled) {
+                if (!(good = flag_wait_ge(&p.ready[sg.p1_index], n_exp * tpe, abort_flag, p.status))) break;
+                fence_proxy_async();
+                polled = true;
+                ACM_TRACE(sg.p1_index == 0 ? 17 : 18);
+              }
+              // never ahead of the weight producer: it has found the slot free and armed the barrier
+              if (bars->armed <= hidx) {
+                const unsigned long long t0 = global_timer();
+                while (bars->armed <= hidx) {
+                  if (*abort_flag) { good = false; break; }
+                  if (global_timer() - t0 > kTimeoutNs) {
+                    *abort_flag = 1;
+                    atomicCAS(p.status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+                    good = false;
+                    break;
+                  }
+                }
+                if (!good) break;
+              }
+              tma_load_3d(smem_u32(stage_base) + hs * kStageBytes + kABytes, &h_map, smem_u32(&bars->full[hs]),
+                          ic * kBK, 0, a, pol_x);
+              ++hidx;
+              if (++hs == kStages) hs = 0;
+              if (++ic == tpe) { ic = 0; ++a; }
+            }
+          }
+        }
+        ok = __all_sync(0xffffffffu, good);
       }
     }
   } else {
@@ -407,91 +608,123 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       tc_fence_before();
       mbar_arrive(smem_u32(&bars->tempty[b]));
     };
-    if (p.phase_mask & 1) {
-      const long long U1 = static_cast<long long>(n_act) * tpe * kc1;
-      Sched s1(cta, G, static_cast<long long>(n_act) * tpe, kc1);
-      int tile, k0, k1;
-      while (s1.next(tile, k0, k1)) {
-        const uint32_t b = f & 1u;
-        ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f >> 1) & 1u, abort_flag, p.status));
-        if (!ok) break;
-        tc_fence_after();
-        load_acc(b);
-        ++f;
-        if (k0 > 0) {
-          // tail part of a tile whose first chunks belong to an earlier CTA: hand the fragment over
-          float* dst = p.frag + static_cast<size_t>(cta) * kFragFloats;
-#pragma unroll
-          for (int c = 0; c < kMaxNodes; ++c)
-            if (c < p.n_pad) dst[c * kTileM + row] = v[c];
-          __threadfence();
-          epi_bar_sync();
-          if (row == 0) st_release(&p.frag_flag[cta], p.epoch);
-          continue;
-        }
-        if (k1 < kc1) {
-          // head part: collect the fragments of the CTAs that own the rest of this tile
-          const long long tile_end = static_cast<long long>(tile + 1) * kc1;
-          for (int c2 = cta + 1; c2 < G; ++c2) {
-            const long long b2 = U1 * c2 / G, e2 = U1 * (c2 + 1) / G;
-            if (b2 >= tile_end) break;
-            if (e2 == b2) continue;
-            bool got = true;
-            if (row == 0) got = flag_wait_ge(&p.frag_flag[c2], p.epoch, abort_flag, p.status);
-            ok = epi_vote_all(got);
-            if (!ok) break;
-            const float* src = p.frag + static_cast<size_t>(c2) * kFragFloats;
+    for (int si = 0; si < n_seg && ok; ++si) {
+      const Segment sg = seg[si];
+      const int n_exp = sg.a1 - sg.a0;
+      if (sg.phase == 1) {
+        const long long U1 = static_cast<long long>(n_exp) * tpe * kc1;
+        float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * kFragFloats;
+        int32_t* frag_flag = p.frag_flag + sg.p1_index * G;
+        Sched sc(cta, G, static_cast<long long>(n_exp) * tpe, kc1);
+        int tile, k0, k1;
+        while (sc.next(tile, k0, k1)) {
+          const uint32_t b = f % kAcc;
+          ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f / kAcc) & 1u, abort_flag, p.status));
+          if (!ok) break;
+          if (row == 0) ACM_TRACE(21);
+          tc_fence_after();
+          load_acc(b);
+          ++f;
+          if (row == 0) ACM_TRACE(22);
+          if (k0 > 0) {
+            // tail part of a tile whose first chunks belong to an earlier CTA: hand the fragment over
+            float* dst = frag + static_cast<size_t>(cta) * kFragFloats;
 #pragma unroll
             for (int c = 0; c < kMaxNodes; ++c)
-              if (c < p.n_pad) v[c] += __ldcg(src + c * kTileM + row);
+              if (c < p.n_pad) dst[c * kTileM + row] = v[c];
+            if (row == 0) ACM_TRACE(29);
+            fence_proxy_async();
+            __threadfence();
+            if (row == 0) ACM_TRACE(30);
+            epi_bar_sync();
+            if (row == 0) st_release(&frag_flag[cta], p.epoch);
+            continue;
           }
-          if (!ok) break;
+          const int a = sg.a0 + tile / tpe, ti = tile % tpe;
+          if (row < p.n_pad) bars->wd[row] = p.wdense[static_cast<size_t>(a) * kMaxNodes + row];
+          if (k1 < kc1) {
+            // head part: the helper warp has summed the other CTAs' fragments of this tile into smem
+            ok = epi_vote_all(mbar_wait(smem_u32(&bars->frag_full[sg.p1_index]), 0, abort_flag, p.status));
+            if (!ok) break;
+#pragma unroll
+            for (int c = 0; c < kMaxNodes; ++c)
+              if (c < p.n_pad) v[c] += sfrag[c * kTileM + row];
+            mbar_arrive(smem_u32(&bars->frag_free));
+          }
+          if (row == 0) ACM_TRACE(23);
+          // rows 0..63 hold gate, rows 64..127 the matching up projections.  Each pair of threads
+          // (i, i+64) splits the node columns: the gate thread finishes columns [0, 32), the up
+          // thread columns [32, 64); they swap the halves they do not finish through smem.
+          constexpr int kHalf = kMaxNodes / 2;
+          const int feat = row & 63;
+          if (quarter >= 2) {
+#pragma unroll
+            for (int c = 0; c < kHalf; ++c)
+              if (c < p.n_pad) ex[c * 64 + feat] = v[c];
+          } else {
+#pragma unroll
+            for (int c = kHalf; c < kMaxNodes; ++c)
+              if (c < p.n_pad) ex[c * 64 + feat] = v[c];
+          }
+          epi_bar_sync();
+          if (row == 0) ACM_TRACE(24);
+          {
+            __nv_bfloat16* __restrict__ hdst = p.hbuf + (static_cast<size_t>(a) * kMaxNodes) * p.I + ti * 64 + feat;
+            const int c0 = quarter < 2 ? 0 : kHalf;
+            float other[kHalf], wgt[kHalf];
+#pragma unroll
+            for (int j = 0; j < kHalf; ++j) {      // all shared-memory reads first: the stores below must not order them
+              other[j] = (c0 + j < p.n_pad) ? ex[(c0 + j) * 64 + feat] : 0.0f;
+              wgt[j] = (c0 + j < p.n_pad) ? bars->wd[c0 + j] : 0.0f;
+            }
+#pragma unroll
+            for (int j = 0; j < kHalf; ++j) {
+              if (c0 + j < p.n_pad) {
+                const float mine = quarter < 2 ? v[j] : v[kHalf + j];
+                const float g = quarter < 2 ? mine : other[j];
+                const float u = quarter < 2 ? other[j] : mine;
+                const float h = wgt[j] * u * __fdividef(g, 1.0f + __expf(-g));
+                hdst[static_cast<size_t>(c0 + j) * p.I] = __float2bfloat16_rn(h);
+              }
+            }
+            if (row == 0) ACM_TRACE(25);
+            fence_proxy_async();
+            if (row == 0) ACM_TRACE(26);
+            __threadfence();
+            if (row == 0) ACM_TRACE(27);
+          }
+          epi_bar_sync();
+          if (row == 0) atomicAdd(&p.ready[sg.p1_index], 1);
+          if (row == 0) ACM_TRACE(28);
         }
-        const int a = tile / tpe, ti = tile % tpe;
-        if (quarter >= 2) {
+        if (row == 0) ACM_TRACE(10);
+      } else {
+        Sched sc(cta, G, h_tiles, n_exp * tpe);
+        int ht, k0, k1;
+        while (sc.next(ht, k0, k1)) {
+          const uint32_t b = f % kAcc;
+          ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f / kAcc) & 1u, abort_flag, p.status));
+          if (!ok) break;
+          tc_fence_after();
+          load_acc(b);
+          ++f;
+          float* dst = p.out + static_cast<size_t>(ht) * kTileM + row;
+#ifndef ACM_EXP_NOATOMIC
 #pragma unroll
           for (int c = 0; c < kMaxNodes; ++c)
-            if (c < p.n_pad) ex[c * 64 + (row - 64)] = v[c];
+            if (c < p.T) atomicAdd(dst + static_cast<size_t>(c) * p.H, v[c]);
+#else
+          if (v[0] == 1234.5f) dst[0] = v[1];
+#endif
         }
-        epi_bar_sync();
-        if (quarter < 2) {
-          const float* wrow = p.wdense + static_cast<size_t>(a) * kMaxNodes;
-          __nv_bfloat16* hdst = p.hbuf + (static_cast<size_t>(a) * kMaxNodes) * p.I + ti * 64 + row;
-#pragma unroll
-          for (int c = 0; c < kMaxNodes; ++c) {
-            if (c < p.n_pad) {
-              const float g = v[c], u = ex[c * 64 + row];
-              const float h = wrow[c] * (g / (1.0f + __expf(-g))) * u;
-              hdst[static_cast<size_t>(c) * p.I] = __float2bfloat16_rn(h);
-            }
-          }
-          fence_proxy_async();
-          __threadfence();
-        }
-        epi_bar_sync();
-        if (row == 0) atomicAdd(&p.ready[a], 1);
-      }
-    }
-    if ((p.phase_mask & 2) && ok) {
-      Sched s2(cta, G, h_tiles, kc2);
-      int ht, k0, k1;
-      while (s2.next(ht, k0, k1)) {
-        const uint32_t b = f & 1u;
-        ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f >> 1) & 1u, abort_flag, p.status));
-        if (!ok) break;
-        tc_fence_after();
-        load_acc(b);
-        ++f;
-        float* dst = p.out + static_cast<size_t>(ht) * kTileM + row;
-#pragma unroll
-        for (int c = 0; c < kMaxNodes; ++c)
-          if (c < p.T) atomicAdd(dst + static_cast<size_t>(c) * p.H, v[c]);
+        if (row == 0) ACM_TRACE(11);
       }
     }
   }
 
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) ACM_TRACE(12);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
@@ -564,7 +797,7 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   a.T = L.T; a.H = L.H; a.I = L.I; a.n_pad = L.n_pad;
   a.list = L.list; a.wdense = L.wdense; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
   a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag; a.epoch = L.epoch;
-  a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask;
+  a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask; a.trace = L.trace;
   void* args[] = {const_cast<FfnMaps*>(&maps), const_cast<CUtensorMap*>(&x_map), const_cast<CUtensorMap*>(&h_map), &a};
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(L.grid);

@@ -254,11 +254,12 @@ struct StageSmem {
   int32_t warp_tot[2][4];
   int32_t scal[8];
   float fscal[4];
+  float probs[kMaxNodes * kMaxExperts];   // r[t][e], so that the demand loop never waits on global memory
 };
 
 // Stage 1b: softmax over the expert axis and natural top-k (ranked on the logits), one warp per node.
 __device__ void stage_softmax_topk(const float* __restrict__ logits, float* __restrict__ probs,
-                                   int32_t* __restrict__ nat_idx, int T, int E, int k) {
+                                   int32_t* __restrict__ nat_idx, float* probs_smem, int T, int E, int k) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   for (int t = warp; t < T; t += nwarps) {
     float z[4], y[4];
@@ -271,10 +272,13 @@ __device__ void stage_softmax_topk(const float* __restrict__ logits, float* __re
 #pragma unroll
     for (int c = 0; c < 4; ++c) y[c] = (lane + 32 * c < E) ? exp_fixed(__fsub_rn(z[c], zmax)) : 0.0f;
     const float denom = warp_tree_sum_128(y[0], y[1], y[2], y[3]);
-    if (probs) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c)
-        if (lane + 32 * c < E) probs[static_cast<size_t>(t) * E + lane + 32 * c] = __fdiv_rn(y[c], denom);
+    for (int c = 0; c < 4; ++c) {
+      if (lane + 32 * c < E) {
+        const float r = __fdiv_rn(y[c], denom);
+        if (probs) probs[static_cast<size_t>(t) * E + lane + 32 * c] = r;
+        if (probs_smem) probs_smem[t * E + lane + 32 * c] = r;
+      }
     }
     if (nat_idx) {
       unsigned taken = 0;
@@ -314,7 +318,8 @@ __device__ float block_tree_sum_128(float* tree, float mine) {
 }
 
 // Stage 2: demand, anchors, self-sizing, pruning.  Thread e < 128 owns expert e.
-__device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, int k) {
+// probs_ready: sm.probs already holds r (written by the softmax stage of the same CTA).
+__device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, int k, bool probs_ready) {
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   const bool owner = tid < kMaxExperts;
@@ -327,6 +332,8 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   }
   if (tid < 8) sm.scal[tid] = 0;
   for (int i = tid; i < T; i += blockDim.x) sm.alpha[i] = a.alpha[i];
+  if (!probs_ready)
+    for (int i = tid; i < T * E; i += blockDim.x) sm.probs[i] = a.probs[i];
   __syncthreads();
   for (int i = tid; i < T * k; i += blockDim.x) {
     const int e = a.nat_idx[i];
@@ -352,7 +359,7 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
       const bool in_topk = (sm.natmask[t][warp] >> lane) & 1u;
       votes += in_topk ? 1 : 0;
       if (a.prm.demand == ACM_DEMAND_FULL_MASS || (a.prm.demand == ACM_DEMAND_TOPK_MASS && in_topk))
-        u = __fmaf_rn(sm.alpha[t], a.probs[static_cast<size_t>(t) * E + tid], u);
+        u = __fmaf_rn(sm.alpha[t], sm.probs[t * E + tid], u);
     }
     if (a.prm.demand == ACM_DEMAND_VOTES) u = static_cast<float>(votes);
   }
@@ -580,12 +587,12 @@ __device__ void stage_route(const RouteArgs& a, StageSmem& sm, int T, int E, int
 
 __global__ void __launch_bounds__(1024) k_softmax_topk(const float* logits, float* probs, int32_t* nat_idx,
                                                        int T, int E, int k) {
-  stage_softmax_topk(logits, probs, nat_idx, T, E, k);
+  stage_softmax_topk(logits, probs, nat_idx, nullptr, T, E, k);
 }
 
 __global__ void __launch_bounds__(128) k_select(SelectArgs a, int T, int E, int k) {
   __shared__ StageSmem sm;
-  stage_select(a, sm, T, E, k);
+  stage_select(a, sm, T, E, k, false);
 }
 
 __global__ void __launch_bounds__(1024) k_route(RouteArgs a, int T, int E, int k) {
@@ -605,8 +612,8 @@ __global__ void __launch_bounds__(1024) k_fused_select_route(const float* logits
     }
     __syncthreads();
   } else {
-    stage_softmax_topk(logits, probs, nat_idx, T, E, k);
-    stage_select(sa, sm, T, E, k);
+    stage_softmax_topk(logits, probs, nat_idx, sm.probs, T, E, k);
+    stage_select(sa, sm, T, E, k, true);
   }
   stage_route(ra, sm, T, E, k);
 }
