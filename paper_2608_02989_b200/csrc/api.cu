@@ -97,38 +97,65 @@ acm_status check_params(const acm_select_params* p) {
   return ACM_OK;
 }
 
-// 3-D bf16 tensor [d2][d1][d0] (d0 contiguous), box {64, box_rows, 1}, 128-byte swizzle.
-acm_status encode_3d(acm_ctx* c, CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint64_t d2,
-                     uint32_t box_rows) {
+// bf16 tensor view for TMA with 128-byte swizzle.  Dimension 0 is always one 64-element (128-byte)
+// swizzle atom along K; the atom index is a dimension of its own, so that one copy can fetch
+// several atoms of the same rows and lay them out in shared memory atom after atom.
+acm_status encode_view(acm_ctx* c, CUtensorMap* m, const void* base, int rank, const uint64_t* dims,
+                       const uint64_t* strides_bytes /* rank-1 entries, for dims 1.. */, const uint32_t* box) {
   if (reinterpret_cast<uintptr_t>(base) % 16 != 0) return ACM_ERR_INVALID;
-  const cuuint64_t dims[3] = {d0, d1, d2};
-  const cuuint64_t strides[2] = {d0 * 2, d0 * d1 * 2};
-  const cuuint32_t box[3] = {64, box_rows, 1};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult r = c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+  cuuint64_t d[5], st[4];
+  cuuint32_t bx[5], es[5];
+  for (int i = 0; i < rank; ++i) {
+    d[i] = dims[i];
+    bx[i] = box[i];
+    es[i] = 1;
+    if (i > 0) st[i - 1] = strides_bytes[i - 1];
+  }
+  const CUresult r = c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), d, st, bx, es,
                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? ACM_OK : ACM_ERR_CUDA;
 }
 
-acm_status encode_2d(acm_ctx* c, CUtensorMap* m, const void* base, uint64_t d0, uint64_t d1, uint32_t box_rows) {
-  if (reinterpret_cast<uintptr_t>(base) % 16 != 0) return ACM_ERR_INVALID;
-  const cuuint64_t dims[2] = {d0, d1};
-  const cuuint64_t strides[1] = {d0 * 2};
-  const cuuint32_t box[2] = {64, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = c->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? ACM_OK : ACM_ERR_CUDA;
+// gate_up [n, 2I, H] as {k in atom, row in I, gate|up, atom of H, expert}; one box = 64 gate rows +
+// the 64 matching up rows x 2 atoms (32 KB), stored atom-major: [atom][gate rows, up rows][64].
+acm_status encode_gate_up(acm_ctx* c, CUtensorMap* m, const void* base, uint64_t n) {
+  const uint64_t H = c->desc.hidden, I = c->desc.inter;
+  const uint64_t dims[5] = {64, I, 2, H / 64, n};
+  const uint64_t strides[4] = {H * 2, I * H * 2, 128, 2 * I * H * 2};
+  const uint32_t box[5] = {64, 64, 2, 2, 1};
+  return encode_view(c, m, base, 5, dims, strides, box);
+}
+// down [n, H, I] as {k in atom, row in H, atom of I, expert}; one box = 128 rows x 2 atoms (32 KB).
+acm_status encode_down(acm_ctx* c, CUtensorMap* m, const void* base, uint64_t n) {
+  const uint64_t H = c->desc.hidden, I = c->desc.inter;
+  const uint64_t dims[4] = {64, H, I / 64, n};
+  const uint64_t strides[3] = {I * 2, 128, H * I * 2};
+  const uint32_t box[4] = {64, 128, 2, 1};
+  return encode_view(c, m, base, 4, dims, strides, box);
+}
+// x [T, H] as {k in atom, node, atom of H}; one box = n_pad nodes x 2 atoms.
+acm_status encode_x(acm_ctx* c, CUtensorMap* m, const void* x, int T, int n_pad) {
+  const uint64_t H = c->desc.hidden;
+  const uint64_t dims[3] = {64, static_cast<uint64_t>(T), H / 64};
+  const uint64_t strides[2] = {H * 2, 128};
+  const uint32_t box[3] = {64, static_cast<uint32_t>(n_pad), 2};
+  return encode_view(c, m, x, 3, dims, strides, box);
+}
+// activations [slots, 64, I] as {k in atom, node, atom of I, slot}; one box = n_pad nodes x 2 atoms.
+acm_status encode_h(acm_ctx* c, CUtensorMap* m, const void* base, int n_pad) {
+  const uint64_t I = c->desc.inter;
+  const uint64_t dims[4] = {64, kMaxNodes, I / 64, kMaxSlots};
+  const uint64_t strides[3] = {I * 2, 128, kMaxNodes * I * 2};
+  const uint32_t box[4] = {64, static_cast<uint32_t>(n_pad), 2, 1};
+  return encode_view(c, m, base, 4, dims, strides, box);
 }
 
 acm_status ensure_h_maps(acm_ctx* c, int n_pad) {
   if (c->h_map_npad == n_pad) return ACM_OK;
   const size_t list_bytes = static_cast<size_t>(kMaxSlots) * kMaxNodes * c->desc.inter * 2;
   for (int l = 0; l < 2; ++l) {
-    acm_status st = encode_3d(c, &c->h_map[l], static_cast<char*>(c->ws.hbuf) + l * list_bytes, c->desc.inter,
-                              kMaxNodes, kMaxSlots, n_pad);
+    acm_status st = encode_h(c, &c->h_map[l], static_cast<char*>(c->ws.hbuf) + l * list_bytes, n_pad);
     if (st != ACM_OK) return st;
   }
   c->h_map_npad = n_pad;
@@ -150,7 +177,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   acm_status st = ensure_h_maps(c, n_pad);
   if (st != ACM_OK) return st;
   CUtensorMap x_map;
-  st = encode_2d(c, &x_map, x, d.hidden, T, n_pad);
+  st = encode_x(c, &x_map, x, T, n_pad);
   if (st != ACM_OK) return st;
   FfnMaps maps = L.maps;
   if (c->stage_gate_up) {
@@ -198,9 +225,9 @@ acm_status ensure_staging(acm_ctx* c) {
   const size_t dn = static_cast<size_t>(d.n_experts) * d.hidden * d.inter * 2;
   if (cudaMalloc(&c->stage_gate_up, gu) != cudaSuccess) return ACM_ERR_NOMEM;
   if (cudaMalloc(&c->stage_down, dn) != cudaSuccess) return ACM_ERR_NOMEM;
-  acm_status st = encode_3d(c, &c->stage_map_gu, c->stage_gate_up, d.hidden, 2ull * d.inter, d.n_experts, 64);
+  acm_status st = encode_gate_up(c, &c->stage_map_gu, c->stage_gate_up, d.n_experts);
   if (st != ACM_OK) return st;
-  st = encode_3d(c, &c->stage_map_dn, c->stage_down, d.inter, d.hidden, d.n_experts, 128);
+  st = encode_down(c, &c->stage_map_dn, c->stage_down, d.n_experts);
   if (st != ACM_OK) return st;
   ACM_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->host_stage_list), (kMaxExperts + 1) * sizeof(int32_t),
                          cudaHostAllocMapped));
@@ -361,16 +388,16 @@ acm_status acm_set_layer_weights(acm_ctx* c, int layer, const void* w_router, co
   L.shared_gate_up = d.n_shared ? shared_gate_up : nullptr;
   L.shared_down = d.n_shared ? shared_down : nullptr;
   if (d.dtype == ACM_BF16 && w_gate_up) {
-    acm_status st = encode_3d(c, &L.maps.gate_up, w_gate_up, d.hidden, 2ull * d.inter, d.n_experts, 64);
+    acm_status st = encode_gate_up(c, &L.maps.gate_up, w_gate_up, d.n_experts);
     if (st != ACM_OK) return st;
-    st = encode_3d(c, &L.maps.down, w_down, d.inter, d.hidden, d.n_experts, 128);
+    st = encode_down(c, &L.maps.down, w_down, d.n_experts);
     if (st != ACM_OK) return st;
     L.maps.shared_gate_up = L.maps.gate_up;
     L.maps.shared_down = L.maps.down;
     if (d.n_shared) {
-      st = encode_3d(c, &L.maps.shared_gate_up, shared_gate_up, d.hidden, 2ull * d.inter, d.n_shared, 64);
+      st = encode_gate_up(c, &L.maps.shared_gate_up, shared_gate_up, d.n_shared);
       if (st != ACM_OK) return st;
-      st = encode_3d(c, &L.maps.shared_down, shared_down, d.inter, d.hidden, d.n_shared, 128);
+      st = encode_down(c, &L.maps.shared_down, shared_down, d.n_shared);
       if (st != ACM_OK) return st;
     }
     L.maps.staged_gate_up = L.maps.gate_up;

@@ -27,17 +27,19 @@ namespace acm {
 namespace {
 
 #ifndef ACM_FFN_STAGES
-#define ACM_FFN_STAGES 7
+#define ACM_FFN_STAGES 3
 #endif
 #ifndef ACM_FFN_ACC
 #define ACM_FFN_ACC 4
 #endif
 constexpr int kStages = ACM_FFN_STAGES;
 constexpr int kAcc = ACM_FFN_ACC;                        // TMEM accumulators in flight (power of two)
-constexpr int kBK = 64;                                  // K elements per stage (one 128-byte swizzle row)
+constexpr int kBK = 64;                                  // K elements of one 128-byte swizzle atom
+constexpr int kAtoms = 2;                                // atoms per pipeline stage: a stage covers 128 K
 constexpr int kTileM = 128;
-constexpr int kABytes = kTileM * kBK * 2;                // 16 KB weight tile
-constexpr int kBBytesMax = kMaxNodes * kBK * 2;          // 8 KB activation chunk
+constexpr int kAtomABytes = kTileM * kBK * 2;            // 16 KB: 128 weight rows x one atom
+constexpr int kABytes = kAtoms * kAtomABytes;            // 32 KB weight tile, one TMA copy
+constexpr int kBBytesMax = kAtoms * kMaxNodes * kBK * 2; // 16 KB activation chunk, one TMA copy
 constexpr int kStageBytes = kABytes + kBBytesMax;
 constexpr int kExBytes = 64 * kMaxNodes * 4;             // up-projection exchange buffer
 constexpr int kAccCols = kMaxNodes;                      // TMEM columns per accumulator
@@ -182,6 +184,20 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       " [%0], [%1, {%2, %3, %4}], [%5], %6;"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar), "l"(policy) : "memory");
 }
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3, int c4, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3, %4, %5, %6}], [%7], %8;"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -317,9 +333,11 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   const int cta = blockIdx.x, G = gridDim.x;
   const int n_act = p.list->n;
   const int tpe = p.I / 64;          // gate/up tiles per expert = K-chunks per expert in the down phase
-  const int kc1 = p.H / kBK;         // K-chunks of a gate/up tile
+  const int kc1 = p.H / (kBK * kAtoms);   // K-chunks (stages) of a gate/up tile
+  const int kpe = (tpe + kAtoms - 1) / kAtoms;   // K-chunks (stages) per expert in the down phase
   const int h_tiles = p.H / kTileM;  // output tiles of the down phase
-  const uint32_t b_bytes = static_cast<uint32_t>(p.n_pad) * kBK * 2;
+  const uint32_t b_atom_bytes = static_cast<uint32_t>(p.n_pad) * kBK * 2;   // one atom of the activation chunk
+  const uint32_t b_bytes = kAtoms * b_atom_bytes;
   Segment seg[4];
   const int n_seg = make_segments(n_act, p.phase_mask, seg);
   int32_t* s_entry = bars->entry;
@@ -377,16 +395,15 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           int tile, k0, k1;
           while (ok && sc.next(tile, k0, k1)) {
             const int32_t ent = s_entry[sg.a0 + tile / tpe];
-            const int r0 = (tile % tpe) * 64, r1 = p.I + r0, eidx = entry_idx(ent);
+            const int r0 = (tile % tpe) * 64, eidx = entry_idx(ent);
             const CUtensorMap* gu = pick_map(entry_src(ent), &maps.gate_up, &maps.shared_gate_up, &maps.staged_gate_up);
             for (int kc = k0; kc < k1; ++kc) {
               if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
               const uint32_t full = smem_u32(&bars->full[s]);
               const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
               mbar_expect_tx(full, kABytes + b_bytes);
-              tma_load_3d(sa, gu, full, kc * kBK, r0, eidx, pol_w);                 // 64 gate rows
-              tma_load_3d(sa + kABytes / 2, gu, full, kc * kBK, r1, eidx, pol_w);   // 64 up rows
-              tma_load_2d(sa + kABytes, &x_map, full, kc * kBK, 0, pol_x);
+              tma_load_5d(sa, gu, full, 0, r0, 0, kc * kAtoms, eidx, pol_w);   // 64 gate + 64 up rows, 2 atoms
+              tma_load_3d(sa + kABytes, &x_map, full, 0, 0, kc * kAtoms, pol_x);
               if (!traced_first) { ACM_TRACE(1); traced_first = true; }
               ++n_armed;
               if (++s == kStages) { s = 0; par ^= 1u; }
@@ -394,10 +411,10 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           }
           ACM_TRACE(sg.p1_index == 0 ? 13 : 2);
         } else {
-          Sched sc(cta, G, h_tiles, n_exp * tpe);
+          Sched sc(cta, G, h_tiles, n_exp * kpe);
           int ht, k0, k1;
           while (ok && sc.next(ht, k0, k1)) {
-            int a = sg.a0 + k0 / tpe, ic = k0 % tpe;
+            int a = sg.a0 + k0 / kpe, ic = k0 % kpe;
             int32_t ent = s_entry[a];
             const CUtensorMap* dn = pick_map(entry_src(ent), &maps.down, &maps.shared_down, &maps.staged_down);
             int eidx = entry_idx(ent);
@@ -406,10 +423,10 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
               const uint32_t full = smem_u32(&bars->full[s]);
               const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
               mbar_expect_tx(full, kABytes + b_bytes);
-              tma_load_3d(sa, dn, full, ic * kBK, ht * kTileM, eidx, pol_w);
+              tma_load_4d(sa, dn, full, 0, ht * kTileM, ic * kAtoms, eidx, pol_w);
               bars->armed = ++n_armed;      // the helper warp may now add this stage's activation chunk
               if (++s == kStages) { s = 0; par ^= 1u; }
-              if (++ic == tpe && kc + 1 < k1) {
+              if (++ic == kpe && kc + 1 < k1) {
                 ic = 0;
                 ent = s_entry[++a];
                 dn = pick_map(entry_src(ent), &maps.down, &maps.shared_down, &maps.staged_down);
@@ -436,7 +453,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       for (int si = 0; si < n_seg && ok; ++si) {
         const Segment sg = seg[si];
         const int n_exp = sg.a1 - sg.a0;
-        Sched sc = sg.phase == 1 ? Sched(cta, G, static_cast<long long>(n_exp) * tpe, kc1) : Sched(cta, G, h_tiles, n_exp * tpe);
+        Sched sc = sg.phase == 1 ? Sched(cta, G, static_cast<long long>(n_exp) * tpe, kc1) : Sched(cta, G, h_tiles, n_exp * kpe);
         int tile, k0, k1;
         while (ok && sc.next(tile, k0, k1)) {
           const uint32_t b = f % kAcc;
@@ -450,10 +467,14 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             if (p.trace) { acc_f[sg.phase - 1] += global_timer() - tw; if (it == 0) ACM_TRACE(6); }
             tc_fence_after();
             const uint32_t sa = smem_u32(stage_base + static_cast<size_t>(s) * kStageBytes);
-            const uint64_t da = umma_smem_desc(sa), db = umma_smem_desc(sa + kABytes);
 #pragma unroll
-            for (int kk = 0; kk < kBK / 16; ++kk)
-              umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kc > k0 || kk > 0) ? 1u : 0u);
+            for (int at = 0; at < kAtoms; ++at) {
+              const uint64_t da = umma_smem_desc(sa + at * kAtomABytes);
+              const uint64_t db = umma_smem_desc(sa + kABytes + at * b_atom_bytes);
+#pragma unroll
+              for (int kk = 0; kk < kBK / 16; ++kk)
+                umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kc > k0 || at > 0 || kk > 0) ? 1u : 0u);
+            }
             umma_commit(smem_u32(&bars->empty[s]));
           }
           if (!ok) break;
@@ -555,11 +576,11 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         bool good = true;
         if (lane == 0) {
           const uint64_t pol_x = policy_evict_last();
-          Sched sc(cta, G, h_tiles, n_exp * tpe);
+          Sched sc(cta, G, h_tiles, n_exp * kpe);
           int ht, k0, k1;
           bool polled = false;
           while (good && sc.next(ht, k0, k1)) {
-            int a = sg.a0 + k0 / tpe, ic = k0 % tpe;
+            int a = sg.a0 + k0 / kpe, ic = k0 % kpe;
             for (int kc = k0; kc < k1; ++kc) {
               if (!polled) {
                 if (!(good = flag_wait_ge(&p.ready[sg.p1_index], n_exp * tpe, abort_flag, p.status))) break;
@@ -581,11 +602,11 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
                 }
                 if (!good) break;
               }
-              tma_load_3d(smem_u32(stage_base) + hs * kStageBytes + kABytes, &h_map, smem_u32(&bars->full[hs]),
-                          ic * kBK, 0, a, pol_x);
+              tma_load_4d(smem_u32(stage_base) + hs * kStageBytes + kABytes, &h_map, smem_u32(&bars->full[hs]),
+                          0, 0, ic * kAtoms, a, pol_x);
               ++hidx;
               if (++hs == kStages) hs = 0;
-              if (++ic == tpe) { ic = 0; ++a; }
+              if (++ic == kpe) { ic = 0; ++a; }
             }
           }
         }
@@ -631,7 +652,11 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             float* dst = frag + static_cast<size_t>(cta) * kFragFloats;
 #pragma unroll
             for (int c = 0; c < kMaxNodes; ++c)
+#ifndef ACM_EXP_NOFRAG
               if (c < p.n_pad) dst[c * kTileM + row] = v[c];
+#else
+              if (v[c] == 1234.5f) dst[c * kTileM + row] = v[c];
+#endif
             if (row == 0) ACM_TRACE(29);
             fence_proxy_async();
             __threadfence();
@@ -684,7 +709,11 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
                 const float g = quarter < 2 ? mine : other[j];
                 const float u = quarter < 2 ? other[j] : mine;
                 const float h = wgt[j] * u * __fdividef(g, 1.0f + __expf(-g));
+#ifndef ACM_EXP_NOHST
                 hdst[static_cast<size_t>(c0 + j) * p.I] = __float2bfloat16_rn(h);
+#else
+                if (h == 1234.5f) hdst[0] = __float2bfloat16_rn(h);
+#endif
               }
             }
             if (row == 0) ACM_TRACE(25);
@@ -699,7 +728,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         }
         if (row == 0) ACM_TRACE(10);
       } else {
-        Sched sc(cta, G, h_tiles, n_exp * tpe);
+        Sched sc(cta, G, h_tiles, n_exp * kpe);
         int ht, k0, k1;
         while (sc.next(ht, k0, k1)) {
           const uint32_t b = f % kAcc;
