@@ -127,7 +127,7 @@ struct FfnLaunch {
 cudaError_t ffn_configure();   // one-time function attributes
 size_t ffn_smem_bytes();
 cudaError_t launch_ffn_bf16(const FfnLaunch& p, const FfnMaps& maps, const CUtensorMap& x_map,
-                            const CUtensorMap& h_map, cudaStream_t s);
+                            const CUtensorMap& h_map, const CUtensorMap& h_store_map, cudaStream_t s);
 cudaError_t launch_ffn_f32(const float* x, const float* gate_up, const float* down,
                            const float* shared_gate_up, const float* shared_down, int n_shared,
                            const int32_t* idx, const float* w, float* hbuf, float* out, int T, int H,

@@ -44,6 +44,7 @@ struct acm_ctx {
   EncodeTiledFn encode = nullptr;
   int32_t epoch = 0;
   CUtensorMap h_map[2];
+  CUtensorMap h_store_map[2];            // same buffers, one 64-feature tile per TMA store
   int h_map_npad = 0;
   // staging of non-resident experts
   void* stage_gate_up = nullptr;
@@ -143,11 +144,11 @@ acm_status encode_x(acm_ctx* c, CUtensorMap* m, const void* x, int T, int n_pad)
   return encode_view(c, m, x, 3, dims, strides, box);
 }
 // activations [slots, 64, I] as {k in atom, node, atom of I, slot}; one box = n_pad nodes x 2 atoms.
-acm_status encode_h(acm_ctx* c, CUtensorMap* m, const void* base, int n_pad) {
+acm_status encode_h(acm_ctx* c, CUtensorMap* m, const void* base, int n_pad, int atoms) {
   const uint64_t I = c->desc.inter;
   const uint64_t dims[4] = {64, kMaxNodes, I / 64, kMaxSlots};
   const uint64_t strides[3] = {I * 2, 128, kMaxNodes * I * 2};
-  const uint32_t box[4] = {64, static_cast<uint32_t>(n_pad), 2, 1};
+  const uint32_t box[4] = {64, static_cast<uint32_t>(n_pad), static_cast<uint32_t>(atoms), 1};
   return encode_view(c, m, base, 4, dims, strides, box);
 }
 
@@ -155,7 +156,9 @@ acm_status ensure_h_maps(acm_ctx* c, int n_pad) {
   if (c->h_map_npad == n_pad) return ACM_OK;
   const size_t list_bytes = static_cast<size_t>(kMaxSlots) * kMaxNodes * c->desc.inter * 2;
   for (int l = 0; l < 2; ++l) {
-    acm_status st = encode_h(c, &c->h_map[l], static_cast<char*>(c->ws.hbuf) + l * list_bytes, n_pad);
+    acm_status st = encode_h(c, &c->h_map[l], static_cast<char*>(c->ws.hbuf) + l * list_bytes, n_pad, 2);
+    if (st != ACM_OK) return st;
+    st = encode_h(c, &c->h_store_map[l], static_cast<char*>(c->ws.hbuf) + l * list_bytes, n_pad, 1);
     if (st != ACM_OK) return st;
   }
   c->h_map_npad = n_pad;
@@ -207,12 +210,12 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   if (c->split_phases) {
     // debugging aid: the two GEMM phases as separate launches (kernel boundary instead of flags)
     p.phase_mask = 1;
-    ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], s));
+    ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
     p.phase_mask = 2;
     p.epoch = ++c->epoch;
     c->launches += 1;
   }
-  ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], s));
+  ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
   c->launches += 1;
   if (e1) ACM_CUDA(cudaEventRecord(e1, s));
   return ACM_OK;

@@ -41,10 +41,11 @@ constexpr int kAtomABytes = kTileM * kBK * 2;            // 16 KB: 128 weight ro
 constexpr int kABytes = kAtoms * kAtomABytes;            // 32 KB weight tile, one TMA copy
 constexpr int kBBytesMax = kAtoms * kMaxNodes * kBK * 2; // 16 KB activation chunk, one TMA copy
 constexpr int kStageBytes = kABytes + kBBytesMax;
-constexpr int kExBytes = 64 * kMaxNodes * 4;             // up-projection exchange buffer
+constexpr int kOutStageBytes = kTileM * kMaxNodes * 4;   // 32 KB: outgoing fragment (also the gate/up exchange buffer)
+constexpr int kHStageBytes = kMaxNodes * 64 * 2;         // 8 KB: one finished activation tile (64 features x nodes)
 constexpr int kAccCols = kMaxNodes;                      // TMEM columns per accumulator
 constexpr int kTmemCols = kAcc * kAccCols;
-constexpr int kThreads = 224;                            // producer, MMA, 4 epilogue warps, helper warp
+constexpr int kThreads = 256;                            // producer, MMA, 4 epilogue warps, helper, publisher
 constexpr int kFragBytes = kTileM * kMaxNodes * 4;       // contributor fragments pre-summed in shared memory
 constexpr int kFragFloats = kTileM * kMaxNodes;
 constexpr unsigned long long kTimeoutNs = 1000ull * 1000ull * 1000ull;
@@ -58,6 +59,8 @@ struct __align__(8) Barriers {
   unsigned long long frag_full[2];   // helper -> epilogue: pre-summed fragments of gate/up segment i are in smem
   unsigned long long frag_free;      // epilogue -> helper: the fragment buffer may be overwritten
   unsigned long long helper;         // completion of the helper warp's bulk copy
+  unsigned long long ost_full, ost_free;   // epilogue <-> publisher: outgoing fragment staged / copied out
+  unsigned long long hst_full[2], hst_free[2];   // epilogue <-> publisher: activation tile staged / stored
   volatile uint32_t armed;           // stages whose barrier the weight producer has armed so far
   uint32_t tmem_base;
   int abort_flag;
@@ -65,7 +68,7 @@ struct __align__(8) Barriers {
   int32_t entry[kMaxSlots];     // this launch's work list (copied from global memory once)
 };
 
-constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + kExBytes + kFragBytes + sizeof(Barriers);
+constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + kOutStageBytes + kFragBytes + 2 * kHStageBytes + sizeof(Barriers);
 
 // ---------------------------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -147,6 +150,9 @@ __device__ bool flag_wait_ge(const int32_t* p, int target, volatile int* abort_f
   }
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 // Barrier over the 128 epilogue threads that also ANDs a predicate, so that all of them take the
@@ -320,13 +326,17 @@ __device__ __forceinline__ int make_segments(int n_act, int phase_mask, Segment*
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtensorMap x_map,
-           const __grid_constant__ CUtensorMap h_map, const FfnArgs p) {
+           const __grid_constant__ CUtensorMap h_map, const __grid_constant__ CUtensorMap hs_map,
+           const FfnArgs p) {
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   unsigned char* stage_base = smem;
-  float* ex = reinterpret_cast<float*>(smem + static_cast<size_t>(kStages) * kStageBytes);
-  float* sfrag = reinterpret_cast<float*>(smem + static_cast<size_t>(kStages) * kStageBytes + kExBytes);
-  Barriers* bars = reinterpret_cast<Barriers*>(smem + static_cast<size_t>(kStages) * kStageBytes + kExBytes + kFragBytes);
+  unsigned char* after_ring = smem + static_cast<size_t>(kStages) * kStageBytes;
+  float* ostage = reinterpret_cast<float*>(after_ring);           // outgoing fragment [node][128 rows]
+  float* ex = ostage;                                             // gate/up exchange aliases it (never used at once)
+  float* sfrag = reinterpret_cast<float*>(after_ring + kOutStageBytes);
+  unsigned char* hstage = after_ring + kOutStageBytes + kFragBytes;   // 2 x [node][64 features] bf16, swizzled
+  Barriers* bars = reinterpret_cast<Barriers*>(after_ring + kOutStageBytes + kFragBytes + 2 * kHStageBytes);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -357,6 +367,12 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     mbar_init(smem_u32(&bars->frag_full[1]), 1);
     mbar_init(smem_u32(&bars->frag_free), 128);
     mbar_init(smem_u32(&bars->helper), 1);
+    mbar_init(smem_u32(&bars->ost_full), 128);
+    mbar_init(smem_u32(&bars->ost_free), 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->hst_full[b]), 128);
+      mbar_init(smem_u32(&bars->hst_free[b]), 1);
+    }
     bars->abort_flag = 0;
     bars->armed = 0;
     fence_barrier_init();
@@ -613,12 +629,59 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         ok = __all_sync(0xffffffffu, good);
       }
     }
+  } else if (warp == 7) {
+    // ------------------------------------------------------------------ publisher
+    // Moves what the epilogue staged in shared memory to global memory with bulk copies, waits for
+    // them to complete and only then announces them (fragment flag / finished-tile counter).
+    if (lane == 0) {
+      uint32_t ost_n = 0, fin_n = 0;
+      bool ok = true;
+      for (int si = 0; si < n_seg && ok; ++si) {
+        const Segment sg = seg[si];
+        if (sg.phase != 1) continue;
+        const int n_exp = sg.a1 - sg.a0;
+        float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * kFragFloats;
+        int32_t* frag_flag = p.frag_flag + sg.p1_index * G;
+        Sched sc(cta, G, static_cast<long long>(n_exp) * tpe, kc1);
+        int tile, k0, k1;
+        while (ok && sc.next(tile, k0, k1)) {
+          if (k0 > 0) {
+            if (!(ok = mbar_wait(smem_u32(&bars->ost_full), ost_n & 1u, abort_flag, p.status))) break;
+            const uint32_t bytes = static_cast<uint32_t>(p.n_pad) * kTileM * 4u;
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                         ::"l"(frag + static_cast<size_t>(cta) * kFragFloats), "r"(smem_u32(ostage)), "r"(bytes) : "memory");
+            bulk_commit();
+            bulk_wait_all();
+            __threadfence();
+            st_release(&frag_flag[cta], p.epoch);
+            mbar_arrive(smem_u32(&bars->ost_free));
+            ++ost_n;
+          } else {
+            const uint32_t hb = fin_n & 1u;
+            if (!(ok = mbar_wait(smem_u32(&bars->hst_full[hb]), (fin_n >> 1) & 1u, abort_flag, p.status))) break;
+            const int a = sg.a0 + tile / tpe, ti = tile % tpe;
+            asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+                         ::"l"(&hs_map), "r"(0), "r"(0), "r"(ti), "r"(a), "r"(smem_u32(hstage + hb * kHStageBytes)) : "memory");
+            bulk_commit();
+            bulk_wait_all();
+            __threadfence();
+            atomicAdd(&p.ready[sg.p1_index], 1);
+            mbar_arrive(smem_u32(&bars->hst_free[hb]));
+            ++fin_n;
+            ACM_TRACE(28);
+          }
+        }
+      }
+    }
   } else {
     // ------------------------------------------------------------------ epilogue (128 threads)
+    // On-chip work only: accumulators -> registers -> shared memory.  Everything that has to reach
+    // global memory and be announced to other CTAs (fragments, activation tiles) is staged in shared
+    // memory and handed to the publisher warp, so these warps never sit in a memory fence.
     const int quarter = warp & 3;               // TMEM lanes this warp may read
     const int row = quarter * 32 + lane;        // accumulator row = weight-tile row
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-    uint32_t f = 0;
+    uint32_t f = 0, ost_uses = 0, fin_count = 0;
     bool ok = true;
     float v[kMaxNodes];
     auto load_acc = [&](uint32_t b) {
@@ -629,13 +692,16 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       tc_fence_before();
       mbar_arrive(smem_u32(&bars->tempty[b]));
     };
+    // the outgoing-fragment buffer (and the exchange buffer aliasing it) is free once the publisher
+    // has copied the previous fragment out
+    auto wait_ostage = [&]() -> bool {
+      if (ost_uses == 0) return true;
+      return epi_vote_all(mbar_wait(smem_u32(&bars->ost_free), (ost_uses - 1) & 1u, abort_flag, p.status));
+    };
     for (int si = 0; si < n_seg && ok; ++si) {
       const Segment sg = seg[si];
       const int n_exp = sg.a1 - sg.a0;
       if (sg.phase == 1) {
-        const long long U1 = static_cast<long long>(n_exp) * tpe * kc1;
-        float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * kFragFloats;
-        int32_t* frag_flag = p.frag_flag + sg.p1_index * G;
         Sched sc(cta, G, static_cast<long long>(n_exp) * tpe, kc1);
         int tile, k0, k1;
         while (sc.next(tile, k0, k1)) {
@@ -646,26 +712,18 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           tc_fence_after();
           load_acc(b);
           ++f;
-          if (row == 0) ACM_TRACE(22);
           if (k0 > 0) {
-            // tail part of a tile whose first chunks belong to an earlier CTA: hand the fragment over
-            float* dst = frag + static_cast<size_t>(cta) * kFragFloats;
+            // tail part of a tile whose first chunks belong to an earlier CTA: stage the fragment
+            if (!(ok = wait_ostage())) break;
 #pragma unroll
             for (int c = 0; c < kMaxNodes; ++c)
-#ifndef ACM_EXP_NOFRAG
-              if (c < p.n_pad) dst[c * kTileM + row] = v[c];
-#else
-              if (v[c] == 1234.5f) dst[c * kTileM + row] = v[c];
-#endif
-            if (row == 0) ACM_TRACE(29);
-            fence_proxy_async();
-            __threadfence();
-            if (row == 0) ACM_TRACE(30);
-            epi_bar_sync();
-            if (row == 0) st_release(&frag_flag[cta], p.epoch);
+              if (c < p.n_pad) ostage[c * kTileM + row] = v[c];
+            fence_proxy_async_smem();
+            mbar_arrive(smem_u32(&bars->ost_full));
+            ++ost_uses;
             continue;
           }
-          const int a = sg.a0 + tile / tpe, ti = tile % tpe;
+          const int a = sg.a0 + tile / tpe;
           if (row < p.n_pad) bars->wd[row] = p.wdense[static_cast<size_t>(a) * kMaxNodes + row];
           if (k1 < kc1) {
             // head part: the helper warp has summed the other CTAs' fragments of this tile into smem
@@ -682,6 +740,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           // thread columns [32, 64); they swap the halves they do not finish through smem.
           constexpr int kHalf = kMaxNodes / 2;
           const int feat = row & 63;
+          if (!(ok = wait_ostage())) break;
           if (quarter >= 2) {
 #pragma unroll
             for (int c = 0; c < kHalf; ++c)
@@ -691,14 +750,18 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             for (int c = kHalf; c < kMaxNodes; ++c)
               if (c < p.n_pad) ex[c * 64 + feat] = v[c];
           }
-          epi_bar_sync();
+          const uint32_t hb = fin_count & 1u;
+          bool hst_ok = true;
+          if (fin_count >= 2) hst_ok = mbar_wait(smem_u32(&bars->hst_free[hb]), ((fin_count >> 1) - 1) & 1u, abort_flag, p.status);
+          ok = epi_vote_all(hst_ok);      // also orders the exchange writes above before the reads below
+          if (!ok) break;
           if (row == 0) ACM_TRACE(24);
           {
-            __nv_bfloat16* __restrict__ hdst = p.hbuf + (static_cast<size_t>(a) * kMaxNodes) * p.I + ti * 64 + feat;
+            unsigned char* hs = hstage + hb * kHStageBytes;
             const int c0 = quarter < 2 ? 0 : kHalf;
             float other[kHalf], wgt[kHalf];
 #pragma unroll
-            for (int j = 0; j < kHalf; ++j) {      // all shared-memory reads first: the stores below must not order them
+            for (int j = 0; j < kHalf; ++j) {
               other[j] = (c0 + j < p.n_pad) ? ex[(c0 + j) * 64 + feat] : 0.0f;
               wgt[j] = (c0 + j < p.n_pad) ? bars->wd[c0 + j] : 0.0f;
             }
@@ -708,23 +771,23 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
                 const float mine = quarter < 2 ? v[j] : v[kHalf + j];
                 const float g = quarter < 2 ? mine : other[j];
                 const float u = quarter < 2 ? other[j] : mine;
-                const float h = wgt[j] * u * __fdividef(g, 1.0f + __expf(-g));
-#ifndef ACM_EXP_NOHST
-                hdst[static_cast<size_t>(c0 + j) * p.I] = __float2bfloat16_rn(h);
-#else
-                if (h == 1234.5f) hdst[0] = __float2bfloat16_rn(h);
-#endif
+                // w * u * silu(g), silu(g) = g/2 * (1 + tanh(g/2))
+                const float hg = 0.5f * g;
+                float th;
+                asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(hg));
+                const float q = wgt[j] * u * hg;
+                const float h = fmaf(q, th, q);
+                // activation tile [node][64 features] bf16 in the 128-byte-swizzled layout of its TMA store
+                const int t = c0 + j;
+                const int off = t * 128 + ((((feat >> 3) ^ (t & 7))) << 4) + ((feat & 7) << 1);
+                *reinterpret_cast<__nv_bfloat16*>(hs + off) = __float2bfloat16_rn(h);
               }
             }
+            fence_proxy_async_smem();
+            mbar_arrive(smem_u32(&bars->hst_full[hb]));
+            ++fin_count;
             if (row == 0) ACM_TRACE(25);
-            fence_proxy_async();
-            if (row == 0) ACM_TRACE(26);
-            __threadfence();
-            if (row == 0) ACM_TRACE(27);
           }
-          epi_bar_sync();
-          if (row == 0) atomicAdd(&p.ready[sg.p1_index], 1);
-          if (row == 0) ACM_TRACE(28);
         }
         if (row == 0) ACM_TRACE(10);
       } else {
@@ -738,13 +801,9 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           load_acc(b);
           ++f;
           float* dst = p.out + static_cast<size_t>(ht) * kTileM + row;
-#ifndef ACM_EXP_NOATOMIC
 #pragma unroll
           for (int c = 0; c < kMaxNodes; ++c)
             if (c < p.T) atomicAdd(dst + static_cast<size_t>(c) * p.H, v[c]);
-#else
-          if (v[0] == 1234.5f) dst[0] = v[1];
-#endif
         }
         if (row == 0) ACM_TRACE(11);
       }
@@ -821,13 +880,14 @@ cudaError_t ffn_configure() {
 }
 
 cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
-                            const CUtensorMap& h_map, cudaStream_t s) {
+                            const CUtensorMap& h_map, const CUtensorMap& hs_map, cudaStream_t s) {
   FfnArgs a;
   a.T = L.T; a.H = L.H; a.I = L.I; a.n_pad = L.n_pad;
   a.list = L.list; a.wdense = L.wdense; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
   a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag; a.epoch = L.epoch;
   a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask; a.trace = L.trace;
-  void* args[] = {const_cast<FfnMaps*>(&maps), const_cast<CUtensorMap*>(&x_map), const_cast<CUtensorMap*>(&h_map), &a};
+  void* args[] = {const_cast<FfnMaps*>(&maps), const_cast<CUtensorMap*>(&x_map), const_cast<CUtensorMap*>(&h_map),
+                  const_cast<CUtensorMap*>(&hs_map), &a};
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(L.grid);
   cfg.blockDim = dim3(kThreads);
