@@ -85,6 +85,7 @@ struct RouteArgs {
   int n_shared;
   acm_block_stats* stats_out;    // n_activated / n_staged are filled in
   int32_t* host_stage_list;      // mapped pinned memory: [0] = n_stage, [1..] = expert ids (may be null)
+  long long* dbg;                // optional clock stamps of the fused kernel's stages (debugging aid)
 };
 
 // ---- launchers (routing.cu) -------------------------------------------------------------

@@ -262,7 +262,7 @@ void acm_default_select_params(acm_select_params* p) {
 acm_status acm_debug_ffn_trace(acm_ctx* c, unsigned long long* host_out, int* n_ctas) {
   if (!c || !host_out || !n_ctas || !c->trace) return ACM_ERR_INVALID;
   ACM_CUDA(cudaDeviceSynchronize());
-  ACM_CUDA(cudaMemcpy(host_out, c->trace, sizeof(unsigned long long) * 32 * c->sm_count, cudaMemcpyDeviceToHost));
+  ACM_CUDA(cudaMemcpy(host_out, c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 16), cudaMemcpyDeviceToHost));
   *n_ctas = c->sm_count;
   return ACM_OK;
 }
@@ -355,7 +355,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.ready = reinterpret_cast<int32_t*>(b + o_ready);
   c->ws.status = reinterpret_cast<int32_t*>(b + o_status);
   c->resident_dev = reinterpret_cast<uint32_t*>(b + o_res);
-  if (want_trace && cudaMalloc(&c->trace, sizeof(unsigned long long) * 32 * c->sm_count) != cudaSuccess)
+  if (want_trace && cudaMalloc(&c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 16)) != cudaSuccess)
     return fail(ACM_ERR_NOMEM);
   *out = c;
   return ACM_OK;
@@ -542,6 +542,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   ra.lists = c->ws.lists; ra.wdense = c->ws.wdense; ra.ready = c->ws.ready; ra.resident = res_dev;
   ra.n_shared = d.n_shared; ra.host_stage_list = L.has_resident ? c->host_stage_list_dev : nullptr;
   ra.stats_out = c->ws.stats;
+  ra.dbg = c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr;
   ACM_CUDA(launch_fused_select_route(c->ws.logits, c->ws.probs, c->ws.nat_idx, sa, ra, eligible_mask_override, T, E,
                                      k, c->ws.status, s));
   c->launches += 2;

@@ -57,19 +57,26 @@ __device__ __forceinline__ float log_fixed(float q) {
   return __fmaf_rn(static_cast<float>(e), 0.693147182464599609375f, lm);
 }
 
-// Orderable key: larger logit first, then lower expert index.  0 is "no candidate".
-__device__ __forceinline__ unsigned long long rank_key(float z, int e) {
-  unsigned u = __float_as_uint(z);
-  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-  return (static_cast<unsigned long long>(u) << 32) | static_cast<unsigned>(0xffffffffu - e);
+// 32-bit orderable image of a float (larger float -> larger unsigned); 0 is below every real value.
+__device__ __forceinline__ unsigned order_key(float z) {
+  const unsigned u = __float_as_uint(z);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
-__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
-#pragma unroll
-  for (int s = 16; s >= 1; s >>= 1) {
-    const unsigned long long o = __shfl_xor_sync(0xffffffffu, v, s);
-    v = o > v ? o : v;
-  }
-  return v;
+// One round of a warp-wide top-k over 128 slots (slot e = lane + 32 c, key[c] == 0: not a candidate):
+// returns the slot with the largest key, ties to the lowest slot, or -1 if none is left; the
+// owning lane clears that key.  Two hardware warp reductions per round.
+__device__ __forceinline__ int warp_take_best(unsigned (&key)[4], int lane) {
+  const unsigned m01 = max(key[0], key[1]), m23 = max(key[2], key[3]);
+  const unsigned best = __reduce_max_sync(0xffffffffu, max(m01, m23));
+  if (best == 0u) return -1;
+  unsigned mine = 0xffffffffu;   // lowest slot of this lane that holds the best key
+  if (key[3] == best) mine = lane + 96;
+  if (key[2] == best) mine = lane + 64;
+  if (key[1] == best) mine = lane + 32;
+  if (key[0] == best) mine = lane;
+  const unsigned e = __reduce_min_sync(0xffffffffu, mine);
+  if ((e & 31u) == static_cast<unsigned>(lane)) key[e >> 5] = 0u;
+  return static_cast<int>(e);
 }
 __device__ __forceinline__ float warp_max_f(float v) {
 #pragma unroll
@@ -92,11 +99,12 @@ __device__ __forceinline__ float warp_tree_sum_128(float a0, float a1, float a2,
 }
 
 // ------------------------------------------------------------------------------------------
-// Stage 1a: router logits.  CTA tile = 8 nodes x 8 experts, rows staged in shared memory with
-// 16-byte async copies in 4 K-chunks.  A 16-byte load covers EPT consecutive h, i.e. EPT of
-// the 32 interleaved partial sums; Q = 32/EPT threads share one output.
+// Stage 1a: router logits.  CTA tile = 4 nodes x 8 experts (many small CTAs: the whole GPU works on
+// a 64 x 128 x 2048 product), rows staged in shared memory with 16-byte async copies in 4 K-chunks.
+// A 16-byte load covers EPT consecutive h, i.e. EPT of the 32 interleaved partial sums; Q = 32/EPT
+// threads share one output.
 // ------------------------------------------------------------------------------------------
-constexpr int kRT = 8, kRE = 8;
+constexpr int kRT = 4, kRE = 8;
 
 template <typename Elem>
 struct ElemTraits;
@@ -128,7 +136,7 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
 template <typename Elem>
-__global__ void __launch_bounds__(32 * (32 / ElemTraits<Elem>::EPT) * 1)
+__global__ void __launch_bounds__(kRT * kRE * (32 / ElemTraits<Elem>::EPT))
 k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const float* __restrict__ bias,
                 float* __restrict__ logits, int T, int H, int E, int n_chunks, float* zero_buf,
                 size_t zero_floats, int32_t* status) {
@@ -171,14 +179,13 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
   }
 
   const int q = tid % Q;            // which EPT-wide group of the 32 partial sums
-  const int mt = tid / Q;           // micro tile: 2 nodes x 1 expert
-  const int el = mt % kRE, tp = mt / kRE;
-  float acc[2][EPT];
+  const int mt = tid / Q;           // output of this thread group: one node x one expert
+  const int el = mt % kRE, tl = mt / kRE;
+  float acc[EPT];
 #pragma unroll
-  for (int p = 0; p < EPT; ++p) acc[0][p] = acc[1][p] = 0.0f;
+  for (int p = 0; p < EPT; ++p) acc[p] = 0.0f;
 
-  const unsigned char* xr0 = xs + static_cast<size_t>(2 * tp) * row_bytes + q * 16;
-  const unsigned char* xr1 = xr0 + row_bytes;
+  const unsigned char* xr0 = xs + static_cast<size_t>(tl) * row_bytes + q * 16;
   const unsigned char* wrow = ws + static_cast<size_t>(el) * row_bytes + q * 16;
   const int steps_per_chunk = H / 32 / n_chunks;
   const int step_bytes = 32 * static_cast<int>(sizeof(Elem));
@@ -192,46 +199,30 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
     const int j0 = c * steps_per_chunk;
 #pragma unroll 4
     for (int j = j0; j < j0 + steps_per_chunk; ++j) {
-      float xa[EPT], xb[EPT], wv[EPT];
+      float xa[EPT], wv[EPT];
       ElemTraits<Elem>::unpack(*reinterpret_cast<const uint4*>(xr0 + static_cast<size_t>(j) * step_bytes), xa);
-      ElemTraits<Elem>::unpack(*reinterpret_cast<const uint4*>(xr1 + static_cast<size_t>(j) * step_bytes), xb);
       ElemTraits<Elem>::unpack(*reinterpret_cast<const uint4*>(wrow + static_cast<size_t>(j) * step_bytes), wv);
 #pragma unroll
-      for (int p = 0; p < EPT; ++p) {
-        acc[0][p] = __fmaf_rn(xa[p], wv[p], acc[0][p]);
-        acc[1][p] = __fmaf_rn(xb[p], wv[p], acc[1][p]);
-      }
+      for (int p = 0; p < EPT; ++p) acc[p] = __fmaf_rn(xa[p], wv[p], acc[p]);
     }
   }
   // halving tree over the 32 partial sums: partial l = q*EPT + p
 #pragma unroll
   for (int s = 16; s >= EPT; s >>= 1) {
 #pragma unroll
-    for (int p = 0; p < EPT; ++p) {
-      acc[0][p] = __fadd_rn(acc[0][p], __shfl_xor_sync(0xffffffffu, acc[0][p], s / EPT));
-      acc[1][p] = __fadd_rn(acc[1][p], __shfl_xor_sync(0xffffffffu, acc[1][p], s / EPT));
-    }
+    for (int p = 0; p < EPT; ++p) acc[p] = __fadd_rn(acc[p], __shfl_xor_sync(0xffffffffu, acc[p], s / EPT));
   }
 #pragma unroll
   for (int s = EPT / 2; s >= 1; s >>= 1) {
 #pragma unroll
-    for (int p = 0; p < s; ++p) {
-      acc[0][p] = __fadd_rn(acc[0][p], acc[0][p + s]);
-      acc[1][p] = __fadd_rn(acc[1][p], acc[1][p + s]);
-    }
+    for (int p = 0; p < s; ++p) acc[p] = __fadd_rn(acc[p], acc[p + s]);
   }
-  if (q == 0 && e0 + el < E) {
-    const int e = e0 + el;
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-      const int t = t0 + 2 * tp + r;
-      if (t < T) {
-        float z = acc[r][0];
-        if (bias) z = __fadd_rn(z, bias[e]);
-        logits[static_cast<size_t>(t) * E + e] = z;
-        if (!isfinite(z)) raise_status(status, ACM_ERR_NONFINITE);
-      }
-    }
+  if (q == 0 && e0 + el < E && t0 + tl < T) {
+    const int e = e0 + el, t = t0 + tl;
+    float z = acc[0];
+    if (bias) z = __fadd_rn(z, bias[e]);
+    logits[static_cast<size_t>(t) * E + e] = z;
+    if (!isfinite(z)) raise_status(status, ACM_ERR_NONFINITE);
   }
 }
 
@@ -244,7 +235,8 @@ struct StageSmem {
   uint32_t natmask[kMaxNodes][kMaskWords];
   int32_t votes[kMaxExperts];
   float u[kMaxExperts];
-  float tree[kMaxExperts];
+  float tree[kMaxExperts + 4];
+  unsigned long long rkey[kMaxExperts];   // ranking keys of the experts (0 = not ranked)
   uint32_t A[kMaskWords], S[kMaskWords], Sp[kMaskWords], Hres[kMaskWords];
   int32_t idx[kMaxNodes][kMaxTopK];
   float w[kMaxNodes][kMaxTopK];
@@ -281,20 +273,11 @@ __device__ void stage_softmax_topk(const float* __restrict__ logits, float* __re
       }
     }
     if (nat_idx) {
-      unsigned taken = 0;
-      for (int j = 0; j < k; ++j) {
-        unsigned long long best = 0;
+      unsigned key[4];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int e = lane + 32 * c;
-          if (e < E && !((taken >> c) & 1u)) {
-            const unsigned long long key = rank_key(z[c], e);
-            best = key > best ? key : best;
-          }
-        }
-        best = warp_max_u64(best);
-        const int e = static_cast<int>(0xffffffffu - static_cast<unsigned>(best & 0xffffffffu));
-        if ((e & 31) == lane) taken |= 1u << (e >> 5);
+      for (int c = 0; c < 4; ++c) key[c] = (lane + 32 * c < E) ? order_key(z[c]) : 0u;
+      for (int j = 0; j < k; ++j) {
+        const int e = warp_take_best(key, lane);
         if (lane == 0) nat_idx[static_cast<size_t>(t) * k + j] = e;
       }
     }
@@ -302,19 +285,19 @@ __device__ void stage_softmax_topk(const float* __restrict__ logits, float* __re
   __syncthreads();
 }
 
-// 128-slot halving tree over shared memory (threads 0..127 hold one slot each).
+// 128-slot halving tree (threads 0..127 hold one slot each): levels 64 and 32 are formed by warp 0
+// from shared memory, the remaining levels with shuffles -- the same additions in the same order
+// as a[i] += a[i+s], s = 64, 32, ..., 1.
 __device__ float block_tree_sum_128(float* tree, float mine) {
   const int tid = threadIdx.x;
   if (tid < kMaxExperts) tree[tid] = mine;
   __syncthreads();
-#pragma unroll
-  for (int s = kMaxExperts / 2; s >= 1; s >>= 1) {
-    if (tid < s) tree[tid] = __fadd_rn(tree[tid], tree[tid + s]);
-    __syncthreads();
+  if (tid < 32) {
+    const float r = warp_tree_sum_128(tree[tid], tree[tid + 32], tree[tid + 64], tree[tid + 96]);
+    if (tid == 0) tree[kMaxExperts] = r;
   }
-  const float r = tree[0];
   __syncthreads();
-  return r;
+  return tree[kMaxExperts];
 }
 
 // Stage 2: demand, anchors, self-sizing, pruning.  Thread e < 128 owns expert e.
@@ -355,11 +338,24 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   int votes = 0;
   float u = 0.0f;
   if (live) {
-    for (int t = 0; t < T; ++t) {
-      const bool in_topk = (sm.natmask[t][warp] >> lane) & 1u;
-      votes += in_topk ? 1 : 0;
-      if (a.prm.demand == ACM_DEMAND_FULL_MASS || (a.prm.demand == ACM_DEMAND_TOPK_MASS && in_topk))
-        u = __fmaf_rn(sm.alpha[t], sm.probs[t * E + tid], u);
+    for (int t0 = 0; t0 < T; t0 += 16) {
+      float pr[16], al[16];
+      unsigned in_mask = 0;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {        // reads first, then the ordered chain of fused multiply-adds
+        const int t = t0 + j;
+        const bool valid = t < T;
+        pr[j] = valid ? sm.probs[t * E + tid] : 0.0f;
+        al[j] = valid ? sm.alpha[t] : 0.0f;
+        if (valid && ((sm.natmask[t][warp] >> lane) & 1u)) in_mask |= 1u << j;
+      }
+      votes += __popc(in_mask);
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const bool take = t0 + j < T && (a.prm.demand == ACM_DEMAND_FULL_MASS ||
+                                         (a.prm.demand == ACM_DEMAND_TOPK_MASS && ((in_mask >> j) & 1u)));
+        if (take) u = __fmaf_rn(al[j], pr[j], u);
+      }
     }
     if (a.prm.demand == ACM_DEMAND_VOTES) u = static_cast<float>(votes);
   }
@@ -392,17 +388,22 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   }
   n_keep = min(n_keep, nR);
 
-  // rank inside R by (u descending, index ascending)
-  bool in_S = in_A;
-  if (in_R) {
-    int rank = 0;
-    for (int j = 0; j < E; ++j) {
-      const bool j_in_R = !((sm.A[j >> 5] >> (j & 31)) & 1u);
-      const float uj = sm.u[j];
-      rank += (j_in_R && (uj > u || (uj == u && j < tid))) ? 1 : 0;
-    }
-    in_S = rank < n_keep;
+  // rank inside R by (u descending, index ascending): one 64-bit key per expert, counted by 4 threads each
+  if (owner) sm.rkey[tid] = in_R ? ((static_cast<unsigned long long>(order_key(u)) << 32) | (0xffffffffu - tid)) : 0ull;
+  __syncthreads();
+  if (tid < 4 * kMaxExperts) {
+    const int e = tid >> 2, part = tid & 3;
+    const unsigned long long mykey = sm.rkey[e];
+    int cnt = 0;
+#pragma unroll 8
+    for (int j = part * 32; j < part * 32 + 32; ++j) cnt += sm.rkey[j] > mykey ? 1 : 0;
+    cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
+    cnt += __shfl_xor_sync(0xffffffffu, cnt, 2);
+    if (part == 0) sm.cnt[e] = cnt;
   }
+  __syncthreads();
+  bool in_S = in_A;
+  if (in_R) in_S = sm.cnt[tid] < n_keep;
   const unsigned s_word = __ballot_sync(0xffffffffu, in_S);
   if (owner && lane == 0) sm.S[warp] = s_word;
   const int nS = __syncthreads_count(in_S);
@@ -548,26 +549,18 @@ __device__ void stage_route(const RouteArgs& a, StageSmem& sm, int T, int E, int
     }
     s_all = warp_sum_f(s_all);
     s_elig = warp_sum_f(s_elig);
-    unsigned taken = 0;
+    unsigned key[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) key[c] = elig[c] ? order_key(z[c]) : 0u;
     float s_sel = 0.f, my_y = 0.f;
     int my_e = -1;
     for (int j = 0; j < k; ++j) {
-      unsigned long long best = 0;
-#pragma unroll
-      for (int c = 0; c < 4; ++c)
-        if (elig[c] && !((taken >> c) & 1u)) {
-          const unsigned long long key = rank_key(z[c], lane + 32 * c);
-          best = key > best ? key : best;
-        }
-      best = warp_max_u64(best);
-      int e = -1;
+      const int e = warp_take_best(key, lane);
       float ye = 0.f;
-      if (best != 0ull) {
-        e = static_cast<int>(0xffffffffu - static_cast<unsigned>(best & 0xffffffffu));
+      if (e >= 0) {
         const int c = e >> 5;
         const float cand = c == 0 ? y[0] : c == 1 ? y[1] : c == 2 ? y[2] : y[3];
         ye = __shfl_sync(0xffffffffu, cand, e & 31);
-        if ((e & 31) == lane) taken |= 1u << c;
       }
       s_sel += ye;
       if (lane == j) { my_e = e; my_y = ye; }
@@ -582,6 +575,7 @@ __device__ void stage_route(const RouteArgs& a, StageSmem& sm, int T, int E, int
     }
   }
   __syncthreads();
+  if (a.dbg && threadIdx.x == 0) a.dbg[3] = clock64();
   if (a.lists) stage_build_lists(a, sm, T, E, k);
 }
 
@@ -590,7 +584,7 @@ __global__ void __launch_bounds__(1024) k_softmax_topk(const float* logits, floa
   stage_softmax_topk(logits, probs, nat_idx, nullptr, T, E, k);
 }
 
-__global__ void __launch_bounds__(128) k_select(SelectArgs a, int T, int E, int k) {
+__global__ void __launch_bounds__(512) k_select(SelectArgs a, int T, int E, int k) {
   __shared__ StageSmem sm;
   stage_select(a, sm, T, E, k, false);
 }
@@ -600,10 +594,12 @@ __global__ void __launch_bounds__(1024) k_route(RouteArgs a, int T, int E, int k
   stage_route(a, sm, T, E, k);
 }
 
+#define ACM_RT(slot) do { if (ra.dbg && threadIdx.x == 0) ra.dbg[slot] = clock64(); } while (0)
 __global__ void __launch_bounds__(1024) k_fused_select_route(const float* logits, float* probs, int32_t* nat_idx,
                                                              SelectArgs sa, RouteArgs ra,
                                                              const uint32_t* mask_override, int T, int E, int k) {
   __shared__ StageSmem sm;
+  ACM_RT(0);
   if (mask_override) {
     if (threadIdx.x < (E + 31) / 32) sa.mask_out[threadIdx.x] = mask_override[threadIdx.x];
     if (threadIdx.x == 0 && sa.stats_out) {
@@ -613,9 +609,12 @@ __global__ void __launch_bounds__(1024) k_fused_select_route(const float* logits
     __syncthreads();
   } else {
     stage_softmax_topk(logits, probs, nat_idx, sm.probs, T, E, k);
+    ACM_RT(1);
     stage_select(sa, sm, T, E, k, true);
+    ACM_RT(2);
   }
   stage_route(ra, sm, T, E, k);
+  ACM_RT(4);
 }
 
 __global__ void __launch_bounds__(512) k_routes_to_lists(const int32_t* idx, const float* w, RouteArgs a, int T,
@@ -643,13 +642,13 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     auto kern = k_router_logits<float>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (err != cudaSuccess) return err;
-    kern<<<grid, 256, smem, s>>>(static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
+    kern<<<grid, kRT * kRE * 8, smem, s>>>(static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
                                  logits, T, H, E, n_chunks, zero_buf, zero_floats, status);
   } else {
     auto kern = k_router_logits<__nv_bfloat16>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (err != cudaSuccess) return err;
-    kern<<<grid, 128, smem, s>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router),
+    kern<<<grid, kRT * kRE * 4, smem, s>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router),
                                  bias, logits, T, H, E, n_chunks, zero_buf, zero_floats, status);
   }
   return cudaGetLastError();
@@ -663,7 +662,7 @@ cudaError_t launch_softmax_topk(const float* logits, float* probs, int32_t* nat_
 }
 
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s) {
-  k_select<<<1, 128, 0, s>>>(a, T, E, k);
+  k_select<<<1, 512, 0, s>>>(a, T, E, k);
   return cudaGetLastError();
 }
 
@@ -677,7 +676,7 @@ cudaError_t launch_fused_select_route(const float* logits, float* probs, int32_t
                                       const SelectArgs& sa, const RouteArgs& ra,
                                       const uint32_t* mask_override, int T, int E, int k,
                                       int32_t* /*status*/, cudaStream_t s) {
-  const int threads = max(128, min(1024, 32 * T));
+  const int threads = max(512, min(1024, 32 * T));
   k_fused_select_route<<<1, threads, 0, s>>>(logits, probs, nat_idx, sa, ra, mask_override, T, E, k);
   return cudaGetLastError();
 }
