@@ -21,6 +21,8 @@
 // f32 path: plain FMA kernels (the fp32 toy configuration is a few MFLOP).
 #include <cuda_bf16.h>
 
+#include <cstdlib>
+
 #include "acm_internal.h"
 
 namespace acm {
@@ -261,12 +263,35 @@ __device__ __forceinline__ uint32_t umma_idesc(int n) {
 struct Sched {
   long long u, u_end;
   int kc;
-  __device__ Sched(int cta, int grid, long long tiles, int chunks_per_tile) : kc(chunks_per_tile) {
+  int rr_next, rr_end, rr_stride;   // whole tiles dealt round-robin (rr_stride > 0) instead of a cut range
+  // equal contiguous ranges of (tile, K-chunk) units: CTA c owns [c*U/G, (c+1)*U/G)
+  __device__ Sched(int cta, int grid, long long tiles, int chunks_per_tile)
+      : kc(chunks_per_tile), rr_next(0), rr_end(0), rr_stride(0) {
     const long long total = tiles * chunks_per_tile;
     u = total * cta / grid;
     u_end = total * (cta + 1) / grid;
   }
+  // whole tiles: CTA c owns tiles c, c+G, c+2G, ... < tiles (tiles is a multiple of G here)
+  __device__ static Sched whole_tiles(int cta, int grid, int tiles, int chunks_per_tile) {
+    Sched s(0, 1, 0, chunks_per_tile);
+    s.rr_next = cta;
+    s.rr_end = tiles;
+    s.rr_stride = grid;
+    return s;
+  }
+  __device__ long long stages() const {
+    if (rr_stride > 0) return rr_next < rr_end ? static_cast<long long>((rr_end - rr_next + rr_stride - 1) / rr_stride) * kc : 0;
+    return u_end - u;
+  }
   __device__ bool next(int& tile, int& k0, int& k1) {
+    if (rr_stride > 0) {
+      if (rr_next >= rr_end) return false;
+      tile = rr_next;
+      k0 = 0;
+      k1 = kc;
+      rr_next += rr_stride;
+      return true;
+    }
     if (u >= u_end) return false;
     tile = static_cast<int>(u / kc);
     k0 = static_cast<int>(u % kc);
@@ -300,28 +325,59 @@ __device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMa
   return src == kSrcRouted ? routed : src == kSrcShared ? shared : staged;
 }
 
-// The stream of one launch is cut into up to four segments, executed in this order by every CTA:
-//   gate/up of expert group A, gate/up of group B, down of group A, down of group B
-// (A = first half of the activated experts).  While a CTA streams the second segment, the
-// epilogues of the first finish in the background, so the down projection of group A never
-// waits for its activations; likewise group B's are ready by the time group A's down is through.
+// The stream of one launch is cut into up to four segments, executed in this order by every CTA.
+// A gate/up tile (64 gate + 64 up rows over the whole hidden dimension) needs the complete sum before
+// its activation can be formed, so wherever possible a tile is given whole to one CTA:
+//   with at least one tile per CTA:
+//     1. the n_tiles mod G tiles that do not fill a round, cut evenly over all CTAs (their
+//        cross-CTA fragment exchange then hides behind the next segment)
+//     2. whole tiles, one per CTA and round
+//     3. down projection of the experts that were complete before the last round
+//     4. down projection of the rest -- by then their activations have been stored
+//   with fewer tiles than CTAs: gate/up of the first half of the experts, gate/up of the second
+//   half (both cut evenly), then down of the first half, down of the second half.
+// Down-projection work is linear in K and is always cut evenly.
 struct Segment {
   int phase;      // 1 = gate/up, 2 = down
-  int a0, a1;     // activated-expert slots [a0, a1)
-  int p1_index;   // expert group: fragment buffer / completion counter of its gate/up segment (0 or 1)
+  int whole;      // gate/up only: 1 = whole tiles dealt round-robin, 0 = tiles cut evenly over the CTAs
+  int t0, nt;     // gate/up: first tile and number of tiles (tile = slot * tiles_per_expert + sub-tile)
+  int a0, a1;     // down: activated-expert slots [a0, a1)
+  int p1_index;   // gate/up: which fragment buffer a cut segment uses; down: expert group it waits for
 };
-__device__ __forceinline__ int make_segments(int n_act, int phase_mask, Segment* seg) {
-  const int nA = (n_act + 1) / 2;
+struct Plan {
+  Segment seg[4];
+  int n_seg;
+  int a_split;    // experts [0, a_split) form group 0 (complete early), the rest group 1
+};
+__device__ __forceinline__ Plan make_plan(int n_act, int tpe, int grid, int phase_mask) {
+  Plan pl;
+  pl.n_seg = 0;
+  const int n_t = n_act * tpe;
+  const int rounds = n_t / grid, rem = n_t % grid;
   int n = 0;
-  if (phase_mask & 1) {
-    if (nA > 0) seg[n++] = Segment{1, 0, nA, 0};
-    if (n_act > nA) seg[n++] = Segment{1, nA, n_act, 1};
+  if (rounds == 0) {
+    const int nA = (n_act + 1) / 2;
+    pl.a_split = nA;
+    if (phase_mask & 1) {
+      if (nA > 0) pl.seg[n++] = Segment{1, 0, 0, nA * tpe, 0, 0, 0};
+      if (n_act > nA) pl.seg[n++] = Segment{1, 0, nA * tpe, (n_act - nA) * tpe, 0, 0, 1};
+    }
+  } else {
+    pl.a_split = (rem + (rounds - 1) * grid) / tpe;
+    if (phase_mask & 1) {
+      if (rem > 0) pl.seg[n++] = Segment{1, 0, 0, rem, 0, 0, 0};
+      pl.seg[n++] = Segment{1, 1, rem, rounds * grid, 0, 0, 1};
+    }
   }
   if (phase_mask & 2) {
-    if (nA > 0) seg[n++] = Segment{2, 0, nA, 0};
-    if (n_act > nA) seg[n++] = Segment{2, nA, n_act, 1};
+    if (pl.a_split > 0) pl.seg[n++] = Segment{2, 0, 0, 0, 0, pl.a_split, 0};
+    if (n_act > pl.a_split) pl.seg[n++] = Segment{2, 0, 0, 0, pl.a_split, n_act, 1};
   }
-  return n;
+  pl.n_seg = n;
+  return pl;
+}
+__device__ __forceinline__ Sched p1_sched(const Segment& sg, int cta, int grid, int kc1) {
+  return sg.whole ? Sched::whole_tiles(cta, grid, sg.nt, kc1) : Sched(cta, grid, sg.nt, kc1);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -348,8 +404,10 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   const int h_tiles = p.H / kTileM;  // output tiles of the down phase
   const uint32_t b_atom_bytes = static_cast<uint32_t>(p.n_pad) * kBK * 2;   // one atom of the activation chunk
   const uint32_t b_bytes = kAtoms * b_atom_bytes;
-  Segment seg[4];
-  const int n_seg = make_segments(n_act, p.phase_mask, seg);
+  const Plan plan = make_plan(n_act, tpe, G, p.phase_mask);
+  const Segment* seg = plan.seg;
+  const int n_seg = plan.n_seg;
+  const int a_split = plan.a_split;
   int32_t* s_entry = bars->entry;
   for (int i = threadIdx.x; i < n_act; i += blockDim.x) s_entry[i] = p.list->entry[i];
 
@@ -407,11 +465,11 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         const Segment sg = seg[si];
         const int n_exp = sg.a1 - sg.a0;
         if (sg.phase == 1) {
-          Sched sc(cta, G, static_cast<long long>(n_exp) * tpe, kc1);
+          Sched sc = p1_sched(sg, cta, G, kc1);
           int tile, k0, k1;
           while (ok && sc.next(tile, k0, k1)) {
-            const int32_t ent = s_entry[sg.a0 + tile / tpe];
-            const int r0 = (tile % tpe) * 64, eidx = entry_idx(ent);
+            const int32_t ent = s_entry[(sg.t0 + tile) / tpe];
+            const int r0 = ((sg.t0 + tile) % tpe) * 64, eidx = entry_idx(ent);
             const CUtensorMap* gu = pick_map(entry_src(ent), &maps.gate_up, &maps.shared_gate_up, &maps.staged_gate_up);
             for (int kc = k0; kc < k1; ++kc) {
               if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
@@ -469,7 +527,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       for (int si = 0; si < n_seg && ok; ++si) {
         const Segment sg = seg[si];
         const int n_exp = sg.a1 - sg.a0;
-        Sched sc = sg.phase == 1 ? Sched(cta, G, static_cast<long long>(n_exp) * tpe, kc1) : Sched(cta, G, h_tiles, n_exp * kpe);
+        Sched sc = sg.phase == 1 ? p1_sched(sg, cta, G, kc1) : Sched(cta, G, h_tiles, n_exp * kpe);
         int tile, k0, k1;
         while (ok && sc.next(tile, k0, k1)) {
           const uint32_t b = f % kAcc;
@@ -520,13 +578,12 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       const Segment sg = seg[si];
       const int n_exp = sg.a1 - sg.a0;
       if (sg.phase == 1) {
-        const long long tiles = static_cast<long long>(n_exp) * tpe;
+        hidx += static_cast<uint32_t>(p1_sched(sg, cta, G, kc1).stages());
+        hs = hidx % kStages;
+        if (sg.whole) continue;          // whole tiles: nothing to exchange
+        const long long tiles = sg.nt;
         const long long U1 = tiles * kc1;
         const long long ub = U1 * cta / G, ue = U1 * (cta + 1) / G;
-        {
-          hidx += static_cast<uint32_t>(ue - ub);
-          hs = hidx % kStages;
-        }
         if (ue <= ub) continue;
         const long long last_tile = (ue - 1) / kc1;
         const long long tile_end = (last_tile + 1) * kc1;
@@ -539,47 +596,28 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         const float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * kFragFloats;
         const int32_t* frag_flag = p.frag_flag + sg.p1_index * G;
         const int n_el = p.n_pad * kTileM;
-        bool first = true;
+        int c_first = -1;
         for (int c2 = cta + 1; c2 < G && ok; ++c2) {
           const long long b2 = U1 * c2 / G, e2 = U1 * (c2 + 1) / G;
           if (b2 >= tile_end) break;
           if (e2 == b2) continue;
+          if (c_first < 0) c_first = c2;
           bool got = true;
           if (lane == 0) got = flag_wait_ge(&frag_flag[c2], p.epoch, abort_flag, p.status);
           ok = __all_sync(0xffffffffu, got);
-          if (!ok) break;
-          const float* src = frag + static_cast<size_t>(c2) * kFragFloats;
-          if (first) {
-            // first contributor: one bulk async copy into shared memory
-            if (lane == 0) {
-              fence_proxy_async();
-              const uint32_t hb = smem_u32(&bars->helper);
-              mbar_expect_tx(hb, static_cast<uint32_t>(n_el) * 4u);
-              asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                           ::"r"(smem_u32(sfrag)), "l"(src), "r"(static_cast<uint32_t>(n_el) * 4u), "r"(hb) : "memory");
-            }
-            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->helper), frag_uses & 1u, abort_flag, p.status));
-            if (!ok) break;
-            first = false;
-          } else {
-            // further contributors (a tile cut across three or more CTAs): batched loads, then add
-            const float4* src4 = reinterpret_cast<const float4*>(src);
-            float4* dst4 = reinterpret_cast<float4*>(sfrag);
-            for (int i0 = lane; i0 < n_el / 4; i0 += 32 * 8) {
-              float4 x4[8];
-#pragma unroll
-              for (int j = 0; j < 8; ++j)
-                if (i0 + 32 * j < n_el / 4) x4[j] = __ldcg(src4 + i0 + 32 * j);
-#pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                if (i0 + 32 * j < n_el / 4) {
-                  float4 o = dst4[i0 + 32 * j];
-                  o.x += x4[j].x; o.y += x4[j].y; o.z += x4[j].z; o.w += x4[j].w;
-                  dst4[i0 + 32 * j] = o;
-                }
-              }
-            }
+        }
+        if (!ok) break;
+        if (c_first >= 0) {
+          // every contributor has added its part to the first contributor's buffer: one bulk copy
+          if (lane == 0) {
+            fence_proxy_async();
+            const uint32_t hb = smem_u32(&bars->helper);
+            mbar_expect_tx(hb, static_cast<uint32_t>(n_el) * 4u);
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_u32(sfrag)), "l"(frag + static_cast<size_t>(c_first) * kFragFloats),
+                           "r"(static_cast<uint32_t>(n_el) * 4u), "r"(hb) : "memory");
           }
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->helper), frag_uses & 1u, abort_flag, p.status));
         }
         if (!ok) break;
         __syncwarp();
@@ -599,7 +637,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             int a = sg.a0 + k0 / kpe, ic = k0 % kpe;
             for (int kc = k0; kc < k1; ++kc) {
               if (!polled) {
-                if (!(good = flag_wait_ge(&p.ready[sg.p1_index], n_exp * tpe, abort_flag, p.status))) break;
+                if (!(good = flag_wait_ge(&p.ready[sg.p1_index], n_exp * tpe, abort_flag, p.status))) break;   // n_exp = size of the group
                 fence_proxy_async();
                 polled = true;
                 ACM_TRACE(sg.p1_index == 0 ? 17 : 18);
@@ -639,17 +677,32 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       for (int si = 0; si < n_seg && ok; ++si) {
         const Segment sg = seg[si];
         if (sg.phase != 1) continue;
-        const int n_exp = sg.a1 - sg.a0;
         float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * kFragFloats;
         int32_t* frag_flag = p.frag_flag + sg.p1_index * G;
-        Sched sc(cta, G, static_cast<long long>(n_exp) * tpe, kc1);
+        Sched sc = p1_sched(sg, cta, G, kc1);
         int tile, k0, k1;
         while (ok && sc.next(tile, k0, k1)) {
           if (k0 > 0) {
             if (!(ok = mbar_wait(smem_u32(&bars->ost_full), ost_n & 1u, abort_flag, p.status))) break;
             const uint32_t bytes = static_cast<uint32_t>(p.n_pad) * kTileM * 4u;
-            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                         ::"l"(frag + static_cast<size_t>(cta) * kFragFloats), "r"(smem_u32(ostage)), "r"(bytes) : "memory");
+            // All CTAs that hold a tail part of this tile add into ONE global buffer, the one of the
+            // first of them: it copies, the others wait for that copy and then reduce-add on top.
+            const long long U1 = static_cast<long long>(sg.nt) * kc1;
+            const long long tile_begin = static_cast<long long>(tile) * kc1;
+            int c_head = cta - 1;
+            while (c_head > 0 && U1 * c_head / G > tile_begin) --c_head;       // owner of the tile's first chunk
+            int c_first = c_head + 1;
+            while (c_first < cta && U1 * (c_first + 1) / G == U1 * c_first / G) ++c_first;   // skip empty ranges
+            float* dst = frag + static_cast<size_t>(c_first) * kFragFloats;
+            if (c_first == cta) {
+              asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                           ::"l"(dst), "r"(smem_u32(ostage)), "r"(bytes) : "memory");
+            } else {
+              if (!(ok = flag_wait_ge(&frag_flag[c_first], p.epoch, abort_flag, p.status))) break;
+              fence_proxy_async();
+              asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
+                           ::"l"(dst), "r"(smem_u32(ostage)), "r"(bytes) : "memory");
+            }
             bulk_commit();
             bulk_wait_all();
             __threadfence();
@@ -659,13 +712,13 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           } else {
             const uint32_t hb = fin_n & 1u;
             if (!(ok = mbar_wait(smem_u32(&bars->hst_full[hb]), (fin_n >> 1) & 1u, abort_flag, p.status))) break;
-            const int a = sg.a0 + tile / tpe, ti = tile % tpe;
+            const int a = (sg.t0 + tile) / tpe, ti = (sg.t0 + tile) % tpe;
             asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
                          ::"l"(&hs_map), "r"(0), "r"(0), "r"(ti), "r"(a), "r"(smem_u32(hstage + hb * kHStageBytes)) : "memory");
             bulk_commit();
             bulk_wait_all();
             __threadfence();
-            atomicAdd(&p.ready[sg.p1_index], 1);
+            atomicAdd(&p.ready[a >= a_split ? 1 : 0], 1);
             mbar_arrive(smem_u32(&bars->hst_free[hb]));
             ++fin_n;
             ACM_TRACE(28);
@@ -702,7 +755,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       const Segment sg = seg[si];
       const int n_exp = sg.a1 - sg.a0;
       if (sg.phase == 1) {
-        Sched sc(cta, G, static_cast<long long>(n_exp) * tpe, kc1);
+        Sched sc = p1_sched(sg, cta, G, kc1);
         int tile, k0, k1;
         while (sc.next(tile, k0, k1)) {
           const uint32_t b = f % kAcc;
@@ -723,7 +776,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             ++ost_uses;
             continue;
           }
-          const int a = sg.a0 + tile / tpe;
+          const int a = (sg.t0 + tile) / tpe;
           if (row < p.n_pad) bars->wd[row] = p.wdense[static_cast<size_t>(a) * kMaxNodes + row];
           if (k1 < kc1) {
             // head part: the helper warp has summed the other CTAs' fragments of this tile into smem
@@ -759,28 +812,34 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           {
             unsigned char* hs = hstage + hb * kHStageBytes;
             const int c0 = quarter < 2 ? 0 : kHalf;
-            float other[kHalf], wgt[kHalf];
 #pragma unroll
-            for (int j = 0; j < kHalf; ++j) {
-              other[j] = (c0 + j < p.n_pad) ? ex[(c0 + j) * 64 + feat] : 0.0f;
-              wgt[j] = (c0 + j < p.n_pad) ? bars->wd[c0 + j] : 0.0f;
-            }
+            for (int j0 = 0; j0 < kHalf; j0 += 8) {
+              if (c0 + j0 < p.n_pad) {           // n_pad is a multiple of 16: a block of 8 columns is all in or all out
+                float other[8], wgt[8], hval[8];
 #pragma unroll
-            for (int j = 0; j < kHalf; ++j) {
-              if (c0 + j < p.n_pad) {
-                const float mine = quarter < 2 ? v[j] : v[kHalf + j];
-                const float g = quarter < 2 ? mine : other[j];
-                const float u = quarter < 2 ? other[j] : mine;
-                // w * u * silu(g), silu(g) = g/2 * (1 + tanh(g/2))
-                const float hg = 0.5f * g;
-                float th;
-                asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(hg));
-                const float q = wgt[j] * u * hg;
-                const float h = fmaf(q, th, q);
+                for (int j = 0; j < 8; ++j) {
+                  other[j] = ex[(c0 + j0 + j) * 64 + feat];
+                  wgt[j] = bars->wd[c0 + j0 + j];
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const float mine = quarter < 2 ? v[j0 + j] : v[kHalf + j0 + j];
+                  const float g = quarter < 2 ? mine : other[j];
+                  const float u = quarter < 2 ? other[j] : mine;
+                  // w * u * silu(g), silu(g) = g/2 * (1 + tanh(g/2))
+                  const float hg = 0.5f * g;
+                  float th;
+                  asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(hg));
+                  const float q = wgt[j] * u * hg;
+                  hval[j] = fmaf(q, th, q);
+                }
                 // activation tile [node][64 features] bf16 in the 128-byte-swizzled layout of its TMA store
-                const int t = c0 + j;
-                const int off = t * 128 + ((((feat >> 3) ^ (t & 7))) << 4) + ((feat & 7) << 1);
-                *reinterpret_cast<__nv_bfloat16*>(hs + off) = __float2bfloat16_rn(h);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                  const int t = c0 + j0 + j;
+                  const int off = t * 128 + ((((feat >> 3) ^ (t & 7))) << 4) + ((feat & 7) << 1);
+                  *reinterpret_cast<__nv_bfloat16*>(hs + off) = __float2bfloat16_rn(hval[j]);
+                }
               }
             }
             fence_proxy_async_smem();
@@ -897,7 +956,8 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   attr[0].id = cudaLaunchAttributeCooperative;   // CTAs wait on one another: all must be co-resident
   attr[0].val.cooperative = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  static const bool plain = [] { const char* e = std::getenv("ACM_FFN_PLAIN_LAUNCH"); return e && e[0] == '1'; }();
+  cfg.numAttrs = plain ? 0 : 1;
   return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(k_ffn_bf16), args);
 }
 
