@@ -192,6 +192,30 @@ acm_status acm_ffn_time_ms(acm_ctx* ctx, float* total_ms, int32_t* launches);
 /* Number of kernel launches this context has enqueued since creation (host counter). */
 acm_status acm_launch_count(acm_ctx* ctx, uint64_t* launches_out /*host*/);
 
+/* Allocation-free expert FFN for fp32 layers (the paper has no counterpart: this exists for
+ * callers that must not allocate device memory when they call -- code running inside a memory
+ * pool it does not own, under an allocator that is frozen, or where cudaMalloc's implicit
+ * device synchronisation is not acceptable).  Same computation as acm_expert_ffn on an ACM_F32
+ * layer without shared experts: y_t = sum_j w[t,j] * down_e( silu(gate_e x_t) * up_e x_t ),
+ * e = idx[t,j] (-1 = empty slot).  All pointers are device pointers: x [T,hidden], idx/w
+ * [T,top_k], w_gate_up [n_experts,2*inter,hidden], w_down [n_experts,hidden,inter], out
+ * [T,hidden] (overwritten).  It needs no context and calls no allocator: the intermediate
+ * activations go to a fixed 4 MiB array inside the library image, which every GPU that loads
+ * the library holds until the process exits.
+ *   - Limit: T * top_k * inter <= ACM_NOALLOC_MAX_FLOATS (2^20), T <= 64, top_k <= 8,
+ *     n_experts <= 128; anything larger returns ACM_ERR_UNSUPPORTED and launches nothing.
+ *   - The first call on each device looks up that device's address of the array (one
+ *     cudaGetSymbolAddress, with that device current); make that first call before starting
+ *     any stream capture.
+ *   - Every call uses the same array and leaves its contents behind.  Nothing in it has to be
+ *     zero on entry (each element is written before it is read), but two calls that overlap on
+ *     the GPU -- different streams, or different threads -- race on it: serialise them. */
+#define ACM_NOALLOC_MAX_FLOATS (1u << 20)
+acm_status acm_expert_ffn_f32_noalloc(const float* x, int T, int hidden, int inter, int n_experts,
+                                      int top_k, const int32_t* idx, const float* w,
+                                      const float* w_gate_up, const float* w_down, float* out,
+                                      acm_stream stream);
+
 /* Synchronises `stream` and returns the sticky device-side status (ACM_OK if none), then clears it. */
 acm_status acm_device_status(acm_ctx* ctx, acm_stream stream);
 

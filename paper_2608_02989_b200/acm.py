@@ -25,7 +25,9 @@ EXPORTS = [
     "acm_node_weights", "acm_router", "acm_select_eligible", "acm_route_restricted",
     "acm_expert_ffn", "acm_moe_verify", "acm_set_resident", "acm_h2d_bytes", "acm_ffn_timing",
     "acm_ffn_time_ms", "acm_launch_count", "acm_device_status", "acm_status_string",
+    "acm_expert_ffn_f32_noalloc",
 ]
+NOALLOC_MAX_FLOATS = 1 << 20
 
 
 class ModelDesc(ctypes.Structure):
@@ -93,6 +95,8 @@ def load_library():
     lib.acm_launch_count.argtypes = [c_void_p, POINTER(c_uint64)]
     lib.acm_device_status.argtypes = [c_void_p, c_void_p]
     lib.acm_default_select_params.argtypes = [POINTER(SelectParams)]
+    lib.acm_expert_ffn_f32_noalloc.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p,
+                                               c_void_p, c_void_p, c_void_p, c_void_p]
     _lib = lib
     return lib
 
@@ -124,6 +128,18 @@ def node_weights(depth, p_table, beta=0.5, width_norm=True) -> torch.Tensor:
     _check(load_library().acm_node_weights(_p(depth), depth.numel(), _p(p_table), p_table.numel(),
                                            float(beta), int(bool(width_norm)), _p(alpha)), "acm_node_weights")
     return alpha
+
+
+def expert_ffn_f32_noalloc(x, idx, w, gate_up, down, out, stream=None):
+    """acm_expert_ffn_f32_noalloc: the fp32 expert FFN for callers that may not allocate device memory at
+    call time.  Every tensor, `out` included, is the caller's; nothing is allocated here or in the library
+    (its scratch is a fixed array in the library image, shared by all calls: do not overlap calls)."""
+    T, H = x.shape
+    E, _, I = down.shape
+    k = idx.shape[1]
+    _check(load_library().acm_expert_ffn_f32_noalloc(_p(x), T, H, I, E, k, _p(idx), _p(w), _p(gate_up), _p(down),
+                                                     _p(out), _stream(stream)), "acm_expert_ffn_f32_noalloc")
+    return out
 
 
 class Context:

@@ -22,6 +22,7 @@
 #include <cuda_bf16.h>
 
 #include <cstdlib>
+#include <mutex>
 
 #include "acm_internal.h"
 
@@ -963,3 +964,44 @@ cudaError_t launch_ffn_f32(const float* x, const float* gate_up, const float* do
 
 }  // namespace acm
 
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant of the f32 expert FFN.  The per-(node, slot) intermediate activations that
+// the context-based call keeps in its cudaMalloc'ed workspace live here in a fixed array that is part
+// of the library image, so the call never allocates.
+// ------------------------------------------------------------------------------------------------
+namespace {
+constexpr size_t kNoAllocScratchFloats = ACM_NOALLOC_MAX_FLOATS;
+static __device__ __align__(256) float g_noalloc_scratch[kNoAllocScratchFloats];
+
+constexpr int kNoAllocMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+float* g_noalloc_ptr[kNoAllocMaxDevices];   // device address of the array above, per device (0 = not looked up yet)
+}  // namespace
+
+extern "C" acm_status acm_expert_ffn_f32_noalloc(const float* x, int T, int hidden, int inter, int n_experts, int top_k,
+                                                 const int32_t* idx, const float* w, const float* w_gate_up,
+                                                 const float* w_down, float* out, acm_stream stream) {
+  if (!x || !idx || !w || !w_gate_up || !w_down || !out) return ACM_ERR_INVALID;
+  if (T < 1 || hidden < 1 || inter < 1 || n_experts < 1 || top_k < 1 || top_k > n_experts) return ACM_ERR_INVALID;
+  if (T > acm::kMaxNodes || top_k > acm::kMaxTopK || n_experts > acm::kMaxExperts) return ACM_ERR_UNSUPPORTED;
+  // the scratch holds one float per (node, slot, intermediate feature): refuse what does not fit
+  if (static_cast<size_t>(T) * top_k * inter > kNoAllocScratchFloats) return ACM_ERR_UNSUPPORTED;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return ACM_ERR_CUDA;
+  if (dev < 0 || dev >= kNoAllocMaxDevices) return ACM_ERR_UNSUPPORTED;
+  float* scratch = nullptr;
+  {
+    // First call on this device: ask the runtime where this device's copy of the array lives.  In host
+    // code the array's name is only a handle; a kernel must be given the address obtained here.
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return ACM_ERR_CUDA;
+      g_noalloc_ptr[dev] = static_cast<float*>(p);
+    }
+    scratch = g_noalloc_ptr[dev];
+  }
+  const cudaError_t err = acm::launch_ffn_f32(x, w_gate_up, w_down, nullptr, nullptr, 0, idx, w, scratch, out, T, hidden,
+                                              inter, top_k, static_cast<cudaStream_t>(stream));
+  return err == cudaSuccess ? ACM_OK : ACM_ERR_CUDA;
+}
