@@ -33,7 +33,7 @@ UNIT = "layer-blocks/s"
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=3, help="1..5; default 3 = Qwen3-30B-A3B-shaped stack")
     ap.add_argument("--layers", type=int, default=0, help="override the number of stacked layers (0 = the config's)")
@@ -69,7 +69,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -110,6 +110,19 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": smax, "reasons": sorted(reasons), "samples": len(sm)}
 
 
+def aggregate_over_ranks(local_ms: float, local_units: float, dist=None, device="cpu"):
+    """Replicas only: every rank runs the same independent workload.  Returns (max time over ranks in ms,
+    units summed over ranks); the job's throughput is their ratio."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return local_ms, local_units
+    import torch
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([local_units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t), float(u)
+
+
 def dist_setup(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -127,39 +140,34 @@ def run_reference(args, world, rank):
     from paper_2608_02989_b200 import workloads as wl
 
     cfg = wl.CONFIGS[args.config]
-    sample_layers = 1
-    sample_nodes = min(cfg.n_nodes, 16)
+    blocks_per_step = 4                      # bounded sample: a step is 4 whole layer-blocks, not the whole stack
     depth, p = wl.tree_depths(cfg), wl.commitment_table(cfg)
     alpha = oracle.node_weights(depth.numpy(), p.numpy())
-    w = wl.layer_weights(cfg, 0, "cpu")
-    x = wl.hidden_states(cfg, 0, "cpu")
+    layers = [(wl.layer_weights(cfg, l, "cpu"), wl.hidden_states(cfg, l, "cpu")) for l in range(min(2, cfg.n_layers))]
     cores = os.cpu_count() or 1
 
     def one_step():
-        res = oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha, cfg.top_k,
-                                weighting=cfg.weighting, shared_gate_up=w["shared_gate_up"],
-                                shared_down=w["shared_down"], with_ffn=False)
-        rows = np.arange(sample_nodes)
-        oracle.expert_ffn(x[:sample_nodes], res["idx"][rows], res["w"][rows], w["gate_up"], w["down"],
-                          w["shared_gate_up"], w["shared_down"])
+        for i in range(blocks_per_step):
+            w, x = layers[i % len(layers)]
+            oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha, cfg.top_k,
+                              weighting=cfg.weighting, shared_gate_up=w["shared_gate_up"],
+                              shared_down=w["shared_down"])
 
-    for _ in range(max(args.warmup, 1)):
+    for _ in range(min(max(args.warmup, 1), 3)):
         one_step()
     t0 = time.perf_counter()
     for _ in range(args.steps):
         one_step()
     dt = time.perf_counter() - t0
-    # a step covered sample_layers layers with sample_nodes of n_nodes nodes in the FFN: scale to whole blocks
-    frac = sample_nodes / cfg.n_nodes
-    value = sample_layers * args.steps * frac / dt
-    sample = (f"{sample_layers} layer of C{cfg.index}: router/selection/routing on all {cfg.n_nodes} nodes, expert FFN on "
-              f"the first {sample_nodes} nodes; layer-blocks/s scaled by {frac:.3f}")
+    value = blocks_per_step * args.steps / dt
+    sample = (f"each step = {blocks_per_step} whole layer-blocks of C{cfg.index} (all stages, all {cfg.n_nodes} nodes) "
+              f"instead of the {cfg.n_layers}-layer stack")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": f"C{cfg.index} {cfg.name}-shaped", "hidden": cfg.hidden, "n_experts": cfg.n_experts,
-                   "top_k": cfg.top_k, "inter": cfg.inter, "n_nodes": cfg.n_nodes, "layers": sample_layers},
+                   "top_k": cfg.top_k, "inter": cfg.inter, "n_nodes": cfg.n_nodes, "layers": blocks_per_step},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -168,34 +176,28 @@ def run_reference(args, world, rank):
 
 
 # ------------------------------------------------------------------------------------------
-def cpu_baseline(cfg, budget_s=20.0):
-    """Times the oracle, as it stands, on the host cores for a bounded sample of the workload."""
-    import numpy as np
+def cpu_baseline(cfg, budget_s=15.0):
+    """Times the oracle, as it stands, on the host cores for a bounded sample of the workload:
+    whole layer-blocks (every stage, every node) over the first layers until the budget is spent."""
     import oracle
     from paper_2608_02989_b200 import workloads as wl
 
     depth, p = wl.tree_depths(cfg), wl.commitment_table(cfg)
     alpha = oracle.node_weights(depth.numpy(), p.numpy())
-    w = wl.layer_weights(cfg, 0, "cpu")
-    x = wl.hidden_states(cfg, 0, "cpu")
-    nodes = min(cfg.n_nodes, 16)
+    layers = [(wl.layer_weights(cfg, l, "cpu"), wl.hidden_states(cfg, l, "cpu")) for l in range(min(2, cfg.n_layers))]
     t0 = time.perf_counter()
     done = 0
     while True:
-        res = oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha, cfg.top_k,
-                                weighting=cfg.weighting, shared_gate_up=w["shared_gate_up"],
-                                shared_down=w["shared_down"], with_ffn=False)
-        rows = np.arange(nodes)
-        oracle.expert_ffn(x[:nodes], res["idx"][rows], res["w"][rows], w["gate_up"], w["down"],
-                          w["shared_gate_up"], w["shared_down"])
+        w, x = layers[done % len(layers)]
+        oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha, cfg.top_k,
+                          weighting=cfg.weighting, shared_gate_up=w["shared_gate_up"], shared_down=w["shared_down"])
         done += 1
         dt = time.perf_counter() - t0
-        if dt > budget_s / 2 or done >= 8:
+        if dt > budget_s or done >= 400:
             break
-    frac = nodes / cfg.n_nodes
-    return {"value": done * frac / dt, "unit": UNIT, "cores": os.cpu_count() or 1, "kind": "oracle",
-            "sample": (f"{done} pass(es) over layer 0 of C{cfg.index}: router/selection/routing on all {cfg.n_nodes} "
-                       f"nodes + expert FFN on the first {nodes} nodes, scaled by {frac:.3f}; {dt:.1f} s wall")}
+    return {"value": done / dt, "unit": UNIT, "cores": os.cpu_count() or 1, "kind": "oracle",
+            "sample": (f"{done} whole layer-blocks of C{cfg.index} (all stages, all {cfg.n_nodes} nodes) cycling over "
+                       f"{len(layers)} layers; {dt:.1f} s wall")}
 
 
 def run_acm(args, world, rank, local):
@@ -281,9 +283,7 @@ def run_acm(args, world, rank, local):
         ffn_ms, ffn_n = (ctx.ffn_time_ms() if with_roofline else (0.0, 0))
         ctx.ffn_timing(False)
         if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t)
+            ms, _ = aggregate_over_ranks(ms, float(L * steps), dist, dev)
         return ms, launches, ffn_ms, ffn_n
 
     sampler = ClockSampler(local)
@@ -340,9 +340,7 @@ def run_acm(args, world, rank, local):
         barrier()
         dt = time.perf_counter() - t0
         if world > 1:
-            t = torch.tensor([dt], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t)
+            dt, _ = aggregate_over_ranks(dt, float(L * args.steps), dist, dev)
         e2e = {"value": world * L * args.steps / dt, "unit": UNIT,
                "h2d_bytes_per_step": L * (T * H * cfg.elt_bytes + T * 4), "d2h_bytes_per_step": L * T * H * 4}
 

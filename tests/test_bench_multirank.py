@@ -1,0 +1,42 @@
+"""N > 1 in the benchmark means independent replicas: the only cross-rank step is aggregating the timing
+(max over ranks) and the work (sum over ranks).  Covered with two gloo ranks on CPU."""
+import os
+import subprocess
+import sys
+import textwrap
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent.parent
+
+WORKER = textwrap.dedent("""
+    import os, sys, json
+    sys.path.insert(0, {root!r})
+    import torch.distributed as dist
+    import bench
+    dist.init_process_group("gloo")
+    rank = dist.get_rank()
+    ms, units = bench.aggregate_over_ranks(10.0 + 5.0 * rank, 48.0 * 20, dist, "cpu")
+    if rank == 0:
+        print(json.dumps({{"ms": ms, "units": units, "world": dist.get_world_size()}}))
+    dist.destroy_process_group()
+""")
+
+
+def test_two_rank_aggregation_is_max_time_and_summed_work(tmp_path):
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER.format(root=str(ROOT)))
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT="29541")
+    out = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+                          "--master-addr", "127.0.0.1", "--master-port", "29541", str(script)],
+                         capture_output=True, text=True, env=env, timeout=240)
+    assert out.returncode == 0, out.stderr[-2000:]
+    import json
+    line = [l for l in out.stdout.splitlines() if l.startswith("{")][-1]
+    res = json.loads(line)
+    assert res == {"ms": 15.0, "units": 1920.0, "world": 2}
+
+
+def test_single_process_aggregation_is_identity():
+    sys.path.insert(0, str(ROOT))
+    import bench
+    assert bench.aggregate_over_ranks(3.5, 7.0) == (3.5, 7.0)

@@ -349,3 +349,65 @@ def test_deterministic_selection_and_routing_across_runs():
     assert torch.equal(a[1], b[1]) and torch.equal(a[3], b[3]) and torch.equal(a[2], b[2])
     assert float((a[0] - b[0]).abs().max()) <= 1e-3 * float(a[0].abs().max())
     ctx.close()
+
+
+@pytest.mark.parametrize("mode", [1, 2])
+def test_offload_variant_residency_and_on_demand_loads(mode):
+    """Config-5 mechanism on a reduced layer: a seeded 40 % of the experts is GPU-resident, eligibility is
+    conditioned on residency (Eq. 7, or the strict resident-plus-anchors variant), and activated non-resident
+    experts are copied from pinned host memory.  The device copies of non-resident experts are poisoned with NaN:
+    a correct result proves they were never read."""
+    cfg = wl.scaled(wl.CONFIGS[5], hidden=512, inter=256, n_experts=32, top_k=4, n_nodes=32, max_depth=5, n_layers=1)
+    w, x, alpha = _block(cfg, 2)
+    E = cfg.n_experts
+    rmask = wl.resident_mask(cfg, 2)
+    resident = mask_to_set(rmask.numpy().view(np.uint32), E)
+    assert len(resident) == round(0.4 * E)
+    host_gu = w["gate_up"].cpu().pin_memory()
+    host_dn = w["down"].cpu().pin_memory()
+    dev_gu, dev_dn = w["gate_up"].clone(), w["down"].clone()
+    for e in range(E):
+        if e not in resident:
+            dev_gu[e] = float("nan")
+            dev_dn[e] = float("nan")
+    ctx = _ctx(cfg)
+    ctx.set_layer_weights(0, w["w_router"], w["router_bias"], dev_gu, dev_dn)
+    ctx.set_resident(0, rmask, host_gu, host_dn)
+    for rep in range(2):          # twice: staging slots and events are reused correctly
+        ctx.h2d_bytes(reset=True)
+        out, idx, wt, mask, stats = ctx.moe_verify(0, x, alpha.to(DEV), acm.SelectParams(residency=mode), want=True)
+        assert ctx.device_status() == acm.OK
+        ref = oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha.numpy(), cfg.top_k,
+                                oracle.SelectParams(residency=mode), weighting=cfg.weighting,
+                                resident_mask=rmask.numpy().view(np.uint32))
+        np.testing.assert_array_equal(_u32(mask), ref["mask"])
+        np.testing.assert_array_equal(idx.cpu().numpy(), ref["idx"])
+        _ffn_check(out, ref["out"], f"offload mode {mode}")
+        st = acm.stats_dict(stats)
+        activated = set(ref["idx"].ravel()) - {-1}
+        staged = activated - resident
+        assert st["n_activated"] == len(activated) and st["n_staged"] == len(staged)
+        assert st["pruned_m"] == ref["stats"]["pruned_m"]
+        assert ctx.h2d_bytes() == len(staged) * cfg.expert_bytes
+        if mode == 2:
+            assert staged <= set(ref["nat_idx"][0])       # only the root's anchors can be non-resident
+    # natural routing on the same offloaded layer: every activated non-resident expert is loaded
+    ctx.h2d_bytes(reset=True)
+    full = torch.tensor(full_mask(E).view(np.int32), device=DEV)
+    out, idx, wt, mask, stats = ctx.moe_verify(0, x, None, None, mask_override=full, want=True)
+    ref = oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha.numpy(), cfg.top_k,
+                            weighting=cfg.weighting, mask_override=full_mask(E))
+    _ffn_check(out, ref["out"], "offload natural")
+    nat_staged = (set(ref["idx"].ravel()) - {-1}) - resident
+    assert ctx.h2d_bytes() == len(nat_staged) * cfg.expert_bytes
+    assert acm.stats_dict(stats)["n_staged"] == len(nat_staged)
+    ctx.close()
+
+
+def test_config5_shape_one_layer():
+    """The Qwen3-235B-A22B-shaped layer at full size (4.8 GB of weights), restricted routing, all resident."""
+    cfg = wl.CONFIGS[5]
+    ctx = _ctx(cfg)
+    st, _ = _verify_layer(cfg, 0, ctx, 0, rows=[0, 31, 63])
+    assert st["n_activated"] > cfg.top_k
+    ctx.close()
