@@ -26,6 +26,7 @@ ROOT = Path(__file__).resolve().parent
 if str(ROOT) not in sys.path:
     sys.path.insert(0, str(ROOT))
 
+DRAM_BYTES_PER_ACTIVATED_EXPERT = {3: (272407296 + 196981760 + 197342976) / 68.0}   # config -> bytes
 METRIC = "verify_blocks_per_s_per_moe_layer"
 UNIT = "layer-blocks/s"
 
@@ -349,15 +350,10 @@ def run_acm(args, world, rank, local):
     peak, peak_kind = read_peaks()
     ffn_us = 1e3 * ffn_ms / max(ffn_n, 1)
     achieved = alg_per_launch / (ffn_us * 1e-6) / 1e9 if ffn_n else None
-    traffic = None
-    prof = ROOT / "profiles" / "ffn_traffic.json"
-    if prof.exists():
-        try:
-            d = json.loads(prof.read_text())
-            # DRAM bytes per launch from an ncu capture, scaled by the activated experts of this run
-            traffic = d["dram_bytes_per_activated_expert"] * float(n_act.mean() + cfg.n_shared)
-        except (KeyError, ValueError):
-            traffic = None
+    # DRAM bytes (read + write) of k_ffn_bf16 per activated expert, from the ncu capture summarised in
+    # profiles/k_ffn_bf16_c3_layer.txt (4-layer case; traffic is proportional to the activated experts)
+    per_expert = DRAM_BYTES_PER_ACTIVATED_EXPERT.get(cfg.index)
+    traffic = per_expert * float(n_act.mean() + cfg.n_shared) if per_expert else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
