@@ -68,6 +68,7 @@ struct SelectArgs {
   int32_t* count_out;
   float* demand_out;             // may be null
   acm_block_stats* stats_out;    // may be null
+  long long* dbg;                // optional clock stamps (debugging aid)
 };
 
 struct RouteArgs {

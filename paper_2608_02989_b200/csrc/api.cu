@@ -459,7 +459,7 @@ acm_status acm_select_eligible(acm_ctx* c, const float* probs, const int32_t* na
   a.probs = probs; a.nat_idx = nat_idx; a.alpha = alpha; a.anchor_nodes = anchor_nodes;
   a.n_anchor_nodes = n_anchor_nodes; a.resident = params->residency ? resident_mask : nullptr; a.prm = *params;
   a.mask_out = eligible_mask; a.unpruned_out = unpruned_mask; a.count_out = eligible_count;
-  a.demand_out = demand; a.stats_out = stats;
+  a.demand_out = demand; a.stats_out = stats; a.dbg = nullptr;
   ACM_CUDA(launch_select(a, T, c->desc.n_experts, c->desc.top_k, static_cast<cudaStream_t>(stream)));
   c->launches += 1;
   return ACM_OK;
@@ -536,6 +536,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   sa.n_anchor_nodes = 0; sa.resident = prm.residency ? res_dev : nullptr; sa.prm = prm;
   sa.mask_out = c->ws.mask; sa.unpruned_out = c->ws.unpruned; sa.count_out = c->ws.count;
   sa.demand_out = c->ws.demand; sa.stats_out = c->ws.stats;
+  sa.dbg = c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr;
   RouteArgs ra = {};
   ra.logits = c->ws.logits; ra.mask = c->ws.mask; ra.idx_out = c->ws.idx; ra.w_out = c->ws.w;
   ra.weighting = d.weighting; ra.routed_scale = d.routed_scale;

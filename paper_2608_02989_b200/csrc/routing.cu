@@ -78,16 +78,6 @@ __device__ __forceinline__ int warp_take_best(unsigned (&key)[4], int lane) {
   if ((e & 31u) == static_cast<unsigned>(lane)) key[e >> 5] = 0u;
   return static_cast<int>(e);
 }
-__device__ __forceinline__ float warp_max_f(float v) {
-#pragma unroll
-  for (int s = 16; s >= 1; s >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, s));
-  return v;
-}
-__device__ __forceinline__ float warp_sum_f(float v) {
-#pragma unroll
-  for (int s = 16; s >= 1; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
-  return v;
-}
 
 // Sum of a 128-slot array held as 4 values per lane (slot = lane + 32 c): the halving tree
 // a[i] += a[i+s], s = 64, 32, 16, ..., 1.  Result broadcast to the whole warp.
@@ -246,130 +236,184 @@ struct StageSmem {
   int32_t warp_tot[2][4];
   int32_t scal[8];
   float fscal[4];
+  int32_t nat[kMaxNodes][kMaxTopK];       // natural top-k of every node
   float probs[kMaxNodes * kMaxExperts];   // r[t][e], so that the demand loop never waits on global memory
+  float logits[kMaxNodes * kMaxExperts];  // z[t][e] (fused kernel only)
 };
 
-// Stage 1b: softmax over the expert axis and natural top-k (ranked on the logits), one warp per node.
+// Stage 1b: softmax over the expert axis and natural top-k (ranked on the logits).  One warp works on
+// two nodes at a time, interleaved, so that the warp-wide reductions of one overlap the other's.
 __device__ void stage_softmax_topk(const float* __restrict__ logits, float* __restrict__ probs,
-                                   int32_t* __restrict__ nat_idx, float* probs_smem, int T, int E, int k) {
+                                   int32_t* __restrict__ nat_idx, float* probs_smem, int32_t (*nat_smem)[kMaxTopK], int T,
+                                   int E, int k) {
+  constexpr int R = 2;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  for (int t = warp; t < T; t += nwarps) {
-    float z[4], y[4];
+  for (int t0 = warp * R; t0 < T; t0 += nwarps * R) {
+    float z[R][4], y[R][4], zmax[R], denom[R];
+    unsigned key[R][4];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const int e = lane + 32 * c;
-      z[c] = e < E ? logits[static_cast<size_t>(t) * E + e] : -INFINITY;
-    }
-    const float zmax = warp_max_f(fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])));
+    for (int r = 0; r < R; ++r) {
+      const int t = min(t0 + r, T - 1);      // a duplicate of the last node where the pair is incomplete
 #pragma unroll
-    for (int c = 0; c < 4; ++c) y[c] = (lane + 32 * c < E) ? exp_fixed(__fsub_rn(z[c], zmax)) : 0.0f;
-    const float denom = warp_tree_sum_128(y[0], y[1], y[2], y[3]);
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      if (lane + 32 * c < E) {
-        const float r = __fdiv_rn(y[c], denom);
-        if (probs) probs[static_cast<size_t>(t) * E + lane + 32 * c] = r;
-        if (probs_smem) probs_smem[t * E + lane + 32 * c] = r;
+      for (int c = 0; c < 4; ++c) {
+        const int e = lane + 32 * c;
+        const float v = logits[static_cast<size_t>(t) * E + min(e, E - 1)];   // unconditional load, clamped index
+        z[r][c] = e < E ? v : -INFINITY;
       }
     }
-    if (nat_idx) {
-      unsigned key[4];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) key[c] = (lane + 32 * c < E) ? order_key(z[c]) : 0u;
+    for (int r = 0; r < R; ++r) zmax[r] = fmaxf(fmaxf(z[r][0], z[r][1]), fmaxf(z[r][2], z[r][3]));
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) zmax[r] = fmaxf(zmax[r], __shfl_xor_sync(0xffffffffu, zmax[r], s));
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const float ex = exp_fixed(__fsub_rn(z[r][c], zmax[r]));
+        y[r][c] = (lane + 32 * c < E) ? ex : 0.0f;
+        key[r][c] = (lane + 32 * c < E) ? order_key(z[r][c]) : 0u;
+      }
+      denom[r] = __fadd_rn(__fadd_rn(y[r][0], y[r][2]), __fadd_rn(y[r][1], y[r][3]));
+    }
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) denom[r] = __fadd_rn(denom[r], __shfl_down_sync(0xffffffffu, denom[r], s));
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      denom[r] = __shfl_sync(0xffffffffu, denom[r], 0);
+      const int t = t0 + r;
+      if (t < T) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (lane + 32 * c < E) {
+            const float pr = __fdiv_rn(y[r][c], denom[r]);
+            if (probs) probs[static_cast<size_t>(t) * E + lane + 32 * c] = pr;
+            if (probs_smem) probs_smem[t * E + lane + 32 * c] = pr;
+          }
+        }
+      }
+    }
+    if (nat_idx || nat_smem) {
       for (int j = 0; j < k; ++j) {
-        const int e = warp_take_best(key, lane);
-        if (lane == 0) nat_idx[static_cast<size_t>(t) * k + j] = e;
+        int e[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) e[r] = warp_take_best(key[r], lane);
+        if (lane == 0) {
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            if (t0 + r < T) {
+              if (nat_idx) nat_idx[static_cast<size_t>(t0 + r) * k + j] = e[r];
+              if (nat_smem) nat_smem[t0 + r][j] = e[r];
+            }
+          }
+        }
       }
     }
   }
   __syncthreads();
 }
 
+// The selection stage runs on threads 0..127 only (one per expert slot) and synchronises them
+// with a named barrier, so the other warps of a larger CTA do not take part in its many barriers.
+__device__ __forceinline__ void sel_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+__device__ __forceinline__ int sel_count(bool pred) {
+  int n;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %1, 0;\n\tbar.red.popc.u32 %0, 2, 128, p;\n\t}\n"
+      : "=r"(n) : "r"(static_cast<unsigned>(pred)) : "memory");
+  return n;
+}
 // 128-slot halving tree (threads 0..127 hold one slot each): levels 64 and 32 are formed by warp 0
 // from shared memory, the remaining levels with shuffles -- the same additions in the same order
 // as a[i] += a[i+s], s = 64, 32, ..., 1.
-__device__ float block_tree_sum_128(float* tree, float mine) {
+__device__ float sel_tree_sum_128(float* tree, float mine) {
   const int tid = threadIdx.x;
-  if (tid < kMaxExperts) tree[tid] = mine;
-  __syncthreads();
+  tree[tid] = mine;
+  sel_sync();
   if (tid < 32) {
     const float r = warp_tree_sum_128(tree[tid], tree[tid + 32], tree[tid + 64], tree[tid + 96]);
     if (tid == 0) tree[kMaxExperts] = r;
   }
-  __syncthreads();
+  sel_sync();
   return tree[kMaxExperts];
 }
 
-// Stage 2: demand, anchors, self-sizing, pruning.  Thread e < 128 owns expert e.
-// probs_ready: sm.probs already holds r (written by the softmax stage of the same CTA).
-__device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, int k, bool probs_ready) {
+// Stage 2: demand, anchors, self-sizing, pruning.  Called by threads 0..127 only; thread e owns expert e.
+// Reads r from sm.probs and the natural top-k from sm.nat (the caller fills both).
+#define ACM_ST(slot) do { if (a.dbg && threadIdx.x == 0) a.dbg[slot] = clock64(); } while (0)
+__device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, int k) {
   const int tid = threadIdx.x;
+  ACM_ST(5);
   const int lane = tid & 31, warp = tid >> 5;
-  const bool owner = tid < kMaxExperts;
   const bool live = tid < E;
-  for (int i = tid; i < kMaxNodes * kMaskWords; i += blockDim.x) (&sm.natmask[0][0])[i] = 0u;
+  for (int i = tid; i < kMaxNodes * kMaskWords; i += kMaxExperts) (&sm.natmask[0][0])[i] = 0u;
   if (tid < kMaskWords) {
     sm.A[tid] = 0u;
-    sm.Hres[tid] = a.resident ? a.resident[tid < (E + 31) / 32 ? tid : 0] : 0xffffffffu;
-    if (tid >= (E + 31) / 32) sm.Hres[tid] = 0u;
+    sm.Hres[tid] = (tid < (E + 31) / 32) ? (a.resident ? a.resident[tid] : 0xffffffffu) : 0u;
   }
   if (tid < 8) sm.scal[tid] = 0;
-  for (int i = tid; i < T; i += blockDim.x) sm.alpha[i] = a.alpha[i];
-  if (!probs_ready)
-    for (int i = tid; i < T * E; i += blockDim.x) sm.probs[i] = a.probs[i];
-  __syncthreads();
-  for (int i = tid; i < T * k; i += blockDim.x) {
-    const int e = a.nat_idx[i];
+  for (int i = tid; i < T; i += kMaxExperts) sm.alpha[i] = a.alpha[i];
+  sel_sync();
+  for (int i = tid; i < T * k; i += kMaxExperts) {
+    const int e = sm.nat[i / k][i % k];
     if (e >= 0 && e < E) atomicOr(&sm.natmask[i / k][e >> 5], 1u << (e & 31));
   }
   if (a.prm.use_anchors) {
     const int n_nodes = a.anchor_nodes ? a.n_anchor_nodes : 1;
-    for (int i = tid; i < n_nodes * k; i += blockDim.x) {
+    for (int i = tid; i < n_nodes * k; i += kMaxExperts) {
       const int t = a.anchor_nodes ? a.anchor_nodes[i / k] : 0;
       if (t >= 0 && t < T) {
-        const int e = a.nat_idx[static_cast<size_t>(t) * k + i % k];
+        const int e = sm.nat[t][i % k];
         if (e >= 0 && e < E) atomicOr(&sm.A[e >> 5], 1u << (e & 31));
       }
     }
   }
-  __syncthreads();
+  sel_sync();
+  ACM_ST(6);
 
   // votes v_e and demand u_e (nodes ascending, fused multiply-add)
   int votes = 0;
   float u = 0.0f;
+  const int demand_mode = a.prm.demand;
   if (live) {
     for (int t0 = 0; t0 < T; t0 += 16) {
       float pr[16], al[16];
       unsigned in_mask = 0;
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {        // reads first, then the ordered chain of fused multiply-adds
-        const int t = t0 + j;
-        const bool valid = t < T;
-        pr[j] = valid ? sm.probs[t * E + tid] : 0.0f;
-        al[j] = valid ? sm.alpha[t] : 0.0f;
-        if (valid && ((sm.natmask[t][warp] >> lane) & 1u)) in_mask |= 1u << j;
+      for (int j = 0; j < 16; ++j) {        // unconditional reads first (clamped index), then the ordered chain
+        const int t = min(t0 + j, T - 1);
+        pr[j] = sm.probs[t * E + tid];
+        al[j] = sm.alpha[t];
+        in_mask |= ((sm.natmask[t][warp] >> lane) & 1u) << j;
       }
+      if (t0 + 16 > T) in_mask &= (1u << (T - t0)) - 1u;
       votes += __popc(in_mask);
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const bool take = t0 + j < T && (a.prm.demand == ACM_DEMAND_FULL_MASS ||
-                                         (a.prm.demand == ACM_DEMAND_TOPK_MASS && ((in_mask >> j) & 1u)));
+        const bool take = t0 + j < T && (demand_mode == ACM_DEMAND_FULL_MASS ||
+                                         (demand_mode == ACM_DEMAND_TOPK_MASS && ((in_mask >> j) & 1u)));
         if (take) u = __fmaf_rn(al[j], pr[j], u);
       }
+      if (a.dbg && threadIdx.x == 0) a.dbg[13 + (t0 >> 4)] = clock64() + __float_as_int(u) * 0;
     }
     if (a.prm.demand == ACM_DEMAND_VOTES) u = static_cast<float>(votes);
   }
-  if (owner) {
-    sm.votes[tid] = votes;
-    sm.u[tid] = u;
-  }
+  ACM_ST(7);
+  sm.votes[tid] = votes;
+  sm.u[tid] = u;
   const bool in_A = live && ((sm.A[warp] >> lane) & 1u);
   const bool in_R = live && !in_A;
-  const int nA = __syncthreads_count(in_A);
+  const int nA = sel_count(in_A);
   const int nR = E - nA;
-  const int n_positive = __syncthreads_count(in_R && u > 0.0f);
+  const int n_positive = sel_count(in_R && u > 0.0f);
   const float upos = in_R ? fmaxf(u, 0.0f) : 0.0f;
-  const float Z = block_tree_sum_128(sm.tree, upos);
+  const float Z = sel_tree_sum_128(sm.tree, upos);
+  ACM_ST(8);
 
   const int floor_keep = max(0, k - nA);
   int n_er = 0, n_keep;
@@ -378,7 +422,7 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   } else if (Z > 0.0f) {
     const float qv = __fdiv_rn(upos, Z);
     const float h = (qv >= 1.17549435e-38f) ? __fmul_rn(qv, log_fixed(qv)) : 0.0f;
-    const float entropy = -block_tree_sum_128(sm.tree, h);
+    const float entropy = -sel_tree_sum_128(sm.tree, h);
     const float perp = exp_fixed(entropy);
     n_er = static_cast<int>(ceilf(__fsub_rn(perp, a.prm.ceil_guard)));
     n_er = min(max(n_er, 1), n_positive);
@@ -387,30 +431,29 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
     n_keep = floor_keep;
   }
   n_keep = min(n_keep, nR);
+  ACM_ST(9);
 
-  // rank inside R by (u descending, index ascending): one 64-bit key per expert, counted by 4 threads each
-  if (owner) sm.rkey[tid] = in_R ? ((static_cast<unsigned long long>(order_key(u)) << 32) | (0xffffffffu - tid)) : 0ull;
-  __syncthreads();
-  if (tid < 4 * kMaxExperts) {
-    const int e = tid >> 2, part = tid & 3;
-    const unsigned long long mykey = sm.rkey[e];
-    int cnt = 0;
-#pragma unroll 8
-    for (int j = part * 32; j < part * 32 + 32; ++j) cnt += sm.rkey[j] > mykey ? 1 : 0;
-    cnt += __shfl_xor_sync(0xffffffffu, cnt, 1);
-    cnt += __shfl_xor_sync(0xffffffffu, cnt, 2);
-    if (part == 0) sm.cnt[e] = cnt;
-  }
-  __syncthreads();
+  // rank inside R by (u descending, index ascending): one 64-bit key per expert
+  const unsigned long long mykey =
+      in_R ? ((static_cast<unsigned long long>(order_key(u)) << 32) | (0xffffffffu - tid)) : 0ull;
+  sm.rkey[tid] = mykey;
+  sel_sync();
   bool in_S = in_A;
-  if (in_R) in_S = sm.cnt[tid] < n_keep;
+  if (in_R) {
+    int rank = 0;
+#pragma unroll 16
+    for (int j = 0; j < kMaxExperts; ++j) rank += sm.rkey[j] > mykey ? 1 : 0;
+    in_S = rank < n_keep;
+  }
+  ACM_ST(10);
   const unsigned s_word = __ballot_sync(0xffffffffu, in_S);
-  if (owner && lane == 0) sm.S[warp] = s_word;
-  const int nS = __syncthreads_count(in_S);
-  const int n_union = __syncthreads_count(live && votes > 0);
+  if (lane == 0) sm.S[warp] = s_word;
+  const int nS = sel_count(in_S);
+  const int n_union = sel_count(live && votes > 0);
   if (live && votes > 0 && !in_S) atomicAdd(&sm.scal[0], votes);   // a(S)
-  __syncthreads();
+  sel_sync();
   const int aS = sm.scal[0];
+  ACM_ST(11);
 
   bool in_Sp = in_S;
   int m_star = 0;
@@ -432,15 +475,16 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
       removed = cum <= aS && nS - pos >= k && pos <= a.prm.max_remove;
     }
     in_Sp = in_S && !removed;
-    m_star = __syncthreads_count(removed);
+    m_star = sel_count(removed);
   } else if (a.prm.residency == 2 && a.resident) {
     in_Sp = (in_S && resident) || in_A;
   }
   const unsigned sp_word = __ballot_sync(0xffffffffu, in_Sp);
-  if (owner && lane == 0) sm.Sp[warp] = sp_word;
-  const int nSp = __syncthreads_count(in_Sp);
+  if (lane == 0) sm.Sp[warp] = sp_word;
+  const int nSp = sel_count(in_Sp);
   if (a.prm.residency == 2 && a.resident) m_star = nS - nSp;
 
+  ACM_ST(12);
   const int words = (E + 31) / 32;
   if (tid < words) {
     a.mask_out[tid] = sm.Sp[tid];
@@ -457,7 +501,7 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
       *a.stats_out = st;
     }
   }
-  __syncthreads();
+  sel_sync();
 }
 
 // Turns per-node routes (sm.idx / sm.w) into the FFN work lists: activated experts in ascending
@@ -465,7 +509,13 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
 __device__ void stage_build_lists(const RouteArgs& a, StageSmem& sm, int T, int E, int k) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid < kMaxExperts) sm.cnt[tid] = 0;
-  for (int i = tid; i < 2 * kMaxSlots * kMaxNodes; i += blockDim.x) a.wdense[i] = 0.0f;
+  {
+    const int rows = E + a.n_shared;     // slots that can be occupied in a list
+    for (int i = tid; i < rows * kMaxNodes; i += blockDim.x) {
+      a.wdense[i] = 0.0f;
+      if (a.resident) a.wdense[kMaxSlots * kMaxNodes + i] = 0.0f;
+    }
+  }
   for (int i = tid; i < 2 * kMaxSlots; i += blockDim.x) a.ready[i] = 0;
   if (tid < kMaskWords) sm.Hres[tid] = a.resident ? (tid < (E + 31) / 32 ? a.resident[tid] : 0u) : 0xffffffffu;
   __syncthreads();
@@ -529,49 +579,77 @@ __device__ void stage_build_lists(const RouteArgs& a, StageSmem& sm, int T, int 
 
 // Stage 3: restricted top-k (Eq. 2) and combine weights, one warp per node.
 __device__ void stage_route(const RouteArgs& a, StageSmem& sm, int T, int E, int k) {
+  constexpr int R = 2;                       // two nodes per warp at a time, interleaved
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  for (int t = warp; t < T; t += nwarps) {
-    float z[4], y[4];
-    bool elig[4];
+  uint32_t mask_w[4];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const int e = lane + 32 * c;
-      z[c] = e < E ? a.logits[static_cast<size_t>(t) * E + e] : -INFINITY;
-      elig[c] = e < E && ((a.mask[c] >> lane) & 1u);
-    }
-    const float zmax = warp_max_f(fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3])));
-    float s_all = 0.f, s_elig = 0.f;
+  for (int c = 0; c < 4; ++c) mask_w[c] = a.mask[min(c, (E + 31) / 32 - 1)];
+  for (int t0 = warp * R; t0 < T; t0 += nwarps * R) {
+    float z[R][4], y[R][4], zmax[R], s_all[R], s_elig[R], s_sel[R], my_y[R];
+    unsigned key[R][4];
+    int my_e[R];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      y[c] = (lane + 32 * c < E) ? expf(z[c] - zmax) : 0.0f;
-      s_all += y[c];
-      s_elig += elig[c] ? y[c] : 0.0f;
-    }
-    s_all = warp_sum_f(s_all);
-    s_elig = warp_sum_f(s_elig);
-    unsigned key[4];
+    for (int r = 0; r < R; ++r) {
+      const int t = min(t0 + r, T - 1);
 #pragma unroll
-    for (int c = 0; c < 4; ++c) key[c] = elig[c] ? order_key(z[c]) : 0u;
-    float s_sel = 0.f, my_y = 0.f;
-    int my_e = -1;
-    for (int j = 0; j < k; ++j) {
-      const int e = warp_take_best(key, lane);
-      float ye = 0.f;
-      if (e >= 0) {
-        const int c = e >> 5;
-        const float cand = c == 0 ? y[0] : c == 1 ? y[1] : c == 2 ? y[2] : y[3];
-        ye = __shfl_sync(0xffffffffu, cand, e & 31);
+      for (int c = 0; c < 4; ++c) {
+        const int e = lane + 32 * c;
+        const float v = a.logits[static_cast<size_t>(t) * E + min(e, E - 1)];
+        z[r][c] = e < E ? v : -INFINITY;
       }
-      s_sel += ye;
-      if (lane == j) { my_e = e; my_y = ye; }
+      zmax[r] = fmaxf(fmaxf(z[r][0], z[r][1]), fmaxf(z[r][2], z[r][3]));
+    }
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) zmax[r] = fmaxf(zmax[r], __shfl_xor_sync(0xffffffffu, zmax[r], s));
+    }
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      s_all[r] = 0.f; s_elig[r] = 0.f; s_sel[r] = 0.f; my_y[r] = 0.f; my_e[r] = -1;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const bool in_e = lane + 32 * c < E;
+        const bool elig = in_e && ((mask_w[c] >> lane) & 1u);
+        y[r][c] = in_e ? __expf(z[r][c] - zmax[r]) : 0.0f;
+        s_all[r] += y[r][c];
+        s_elig[r] += elig ? y[r][c] : 0.0f;
+        key[r][c] = elig ? order_key(z[r][c]) : 0u;
+      }
+    }
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        s_all[r] += __shfl_xor_sync(0xffffffffu, s_all[r], s);
+        s_elig[r] += __shfl_xor_sync(0xffffffffu, s_elig[r], s);
+      }
+    }
+    for (int j = 0; j < k; ++j) {
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const int e = warp_take_best(key[r], lane);
+        const int c = (e >= 0 ? e : 0) >> 5;
+        const float cand = c == 0 ? y[r][0] : c == 1 ? y[r][1] : c == 2 ? y[r][2] : y[r][3];
+        const float got = __shfl_sync(0xffffffffu, cand, (e >= 0 ? e : 0) & 31);
+        const float ye = e >= 0 ? got : 0.f;
+        s_sel[r] += ye;
+        if (lane == j) { my_e[r] = e; my_y[r] = ye; }
+      }
     }
     if (lane < k) {
-      const float den = a.weighting == ACM_W_RENORM_TOPK ? s_sel : a.weighting == ACM_W_SOFTMAX_RAW ? s_all : s_elig;
-      const float wgt = my_e >= 0 ? a.routed_scale * my_y / den : 0.0f;
-      sm.idx[t][lane] = my_e;
-      sm.w[t][lane] = wgt;
-      if (a.idx_out) a.idx_out[static_cast<size_t>(t) * k + lane] = my_e;
-      if (a.w_out) a.w_out[static_cast<size_t>(t) * k + lane] = wgt;
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const int t = t0 + r;
+        if (t < T) {
+          const float den = a.weighting == ACM_W_RENORM_TOPK ? s_sel[r] : a.weighting == ACM_W_SOFTMAX_RAW ? s_all[r] : s_elig[r];
+          const float wgt = my_e[r] >= 0 ? a.routed_scale * my_y[r] / den : 0.0f;
+          sm.idx[t][lane] = my_e[r];
+          sm.w[t][lane] = wgt;
+          if (a.idx_out) a.idx_out[static_cast<size_t>(t) * k + lane] = my_e[r];
+          if (a.w_out) a.w_out[static_cast<size_t>(t) * k + lane] = wgt;
+        }
+      }
     }
   }
   __syncthreads();
@@ -581,45 +659,66 @@ __device__ void stage_route(const RouteArgs& a, StageSmem& sm, int T, int E, int
 
 __global__ void __launch_bounds__(1024) k_softmax_topk(const float* logits, float* probs, int32_t* nat_idx,
                                                        int T, int E, int k) {
-  stage_softmax_topk(logits, probs, nat_idx, nullptr, T, E, k);
+  stage_softmax_topk(logits, probs, nat_idx, nullptr, nullptr, T, E, k);
 }
 
-__global__ void __launch_bounds__(512) k_select(SelectArgs a, int T, int E, int k) {
-  __shared__ StageSmem sm;
-  stage_select(a, sm, T, E, k, false);
+extern __shared__ __align__(16) unsigned char routing_smem[];
+
+__global__ void __launch_bounds__(128) k_select(SelectArgs a, int T, int E, int k) {
+  StageSmem& sm = *reinterpret_cast<StageSmem*>(routing_smem);
+  for (int i = threadIdx.x; i < T * E; i += blockDim.x) sm.probs[i] = a.probs[i];
+  for (int i = threadIdx.x; i < T * k; i += blockDim.x) sm.nat[i / k][i % k] = a.nat_idx[i];
+  __syncthreads();
+  stage_select(a, sm, T, E, k);
 }
 
 __global__ void __launch_bounds__(1024) k_route(RouteArgs a, int T, int E, int k) {
-  __shared__ StageSmem sm;
+  StageSmem& sm = *reinterpret_cast<StageSmem*>(routing_smem);
   stage_route(a, sm, T, E, k);
 }
 
 #define ACM_RT(slot) do { if (ra.dbg && threadIdx.x == 0) ra.dbg[slot] = clock64(); } while (0)
+// Stages 1b-3 in one CTA.  The logits are staged in shared memory once; every later stage reads
+// shared memory only, and the selection stage runs on four warps while the others wait.
 __global__ void __launch_bounds__(1024) k_fused_select_route(const float* logits, float* probs, int32_t* nat_idx,
                                                              SelectArgs sa, RouteArgs ra,
                                                              const uint32_t* mask_override, int T, int E, int k) {
-  __shared__ StageSmem sm;
+  StageSmem& sm = *reinterpret_cast<StageSmem*>(routing_smem);
   ACM_RT(0);
+  {
+    const float4* src = reinterpret_cast<const float4*>(logits);
+    float4* dst = reinterpret_cast<float4*>(sm.logits);
+    for (int i = threadIdx.x; i < T * E / 4; i += blockDim.x) dst[i] = __ldcg(src + i);
+    for (int i = (T * E / 4) * 4 + threadIdx.x; i < T * E; i += blockDim.x) sm.logits[i] = logits[i];
+  }
+  __syncthreads();
   if (mask_override) {
-    if (threadIdx.x < (E + 31) / 32) sa.mask_out[threadIdx.x] = mask_override[threadIdx.x];
+    if (threadIdx.x < kMaskWords) {
+      const uint32_t m = threadIdx.x < (E + 31) / 32 ? mask_override[threadIdx.x] : 0u;
+      sm.Sp[threadIdx.x] = m;
+      if (threadIdx.x < (E + 31) / 32) sa.mask_out[threadIdx.x] = m;
+    }
     if (threadIdx.x == 0 && sa.stats_out) {
       acm_block_stats st = {};
       *sa.stats_out = st;
     }
     __syncthreads();
   } else {
-    stage_softmax_topk(logits, probs, nat_idx, sm.probs, T, E, k);
+    stage_softmax_topk(sm.logits, probs, nat_idx, sm.probs, sm.nat, T, E, k);
     ACM_RT(1);
-    stage_select(sa, sm, T, E, k, true);
+    if (threadIdx.x < kMaxExperts) stage_select(sa, sm, T, E, k);
+    __syncthreads();
     ACM_RT(2);
   }
+  ra.logits = sm.logits;
+  ra.mask = sm.Sp;
   stage_route(ra, sm, T, E, k);
   ACM_RT(4);
 }
 
 __global__ void __launch_bounds__(512) k_routes_to_lists(const int32_t* idx, const float* w, RouteArgs a, int T,
                                                          int E, int k) {
-  __shared__ StageSmem sm;
+  StageSmem& sm = *reinterpret_cast<StageSmem*>(routing_smem);
   for (int i = threadIdx.x; i < T * k; i += blockDim.x) {
     const int e = idx[i];
     sm.idx[i / k][i % k] = (e >= 0 && e < E) ? e : -1;
@@ -662,13 +761,17 @@ cudaError_t launch_softmax_topk(const float* logits, float* probs, int32_t* nat_
 }
 
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s) {
-  k_select<<<1, 512, 0, s>>>(a, T, E, k);
+  cudaError_t err = cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(StageSmem)));
+  if (err != cudaSuccess) return err;
+  k_select<<<1, 128, sizeof(StageSmem), s>>>(a, T, E, k);
   return cudaGetLastError();
 }
 
 cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s) {
   const int threads = max(128, min(1024, 32 * T));
-  k_route<<<1, threads, 0, s>>>(a, T, E, k);
+  cudaError_t err = cudaFuncSetAttribute(k_route, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(StageSmem)));
+  if (err != cudaSuccess) return err;
+  k_route<<<1, threads, sizeof(StageSmem), s>>>(a, T, E, k);
   return cudaGetLastError();
 }
 
@@ -676,8 +779,10 @@ cudaError_t launch_fused_select_route(const float* logits, float* probs, int32_t
                                       const SelectArgs& sa, const RouteArgs& ra,
                                       const uint32_t* mask_override, int T, int E, int k,
                                       int32_t* /*status*/, cudaStream_t s) {
-  const int threads = max(512, min(1024, 32 * T));
-  k_fused_select_route<<<1, threads, 0, s>>>(logits, probs, nat_idx, sa, ra, mask_override, T, E, k);
+  const int threads = max(128, min(1024, 32 * ((T + 1) / 2)));     // two nodes per warp in the per-node stages
+  cudaError_t err = cudaFuncSetAttribute(k_fused_select_route, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(StageSmem)));
+  if (err != cudaSuccess) return err;
+  k_fused_select_route<<<1, threads, sizeof(StageSmem), s>>>(logits, probs, nat_idx, sa, ra, mask_override, T, E, k);
   return cudaGetLastError();
 }
 
@@ -688,7 +793,9 @@ cudaError_t launch_routes_to_lists(const int32_t* idx, const float* w, WorkList*
   a.wdense = wdense;
   a.ready = ready;
   a.n_shared = n_shared;
-  k_routes_to_lists<<<1, 512, 0, s>>>(idx, w, a, T, E, k);
+  cudaError_t err = cudaFuncSetAttribute(k_routes_to_lists, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(StageSmem)));
+  if (err != cudaSuccess) return err;
+  k_routes_to_lists<<<1, 512, sizeof(StageSmem), s>>>(idx, w, a, T, E, k);
   return cudaGetLastError();
 }
 
