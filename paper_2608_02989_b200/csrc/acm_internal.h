@@ -53,6 +53,7 @@ struct Workspace {
   int32_t* frag_flag;   // [2][grid] epoch of the fragment stored there
   int32_t* ready;       // [2][kMaxSlots] finished gate/up tiles per activated slot
   int32_t* status;      // [1] sticky device-side status
+  int32_t* tile_done;   // [64] router kernel: expert tiles finished per node tile (self-resetting)
 };
 
 struct SelectArgs {
@@ -92,9 +93,8 @@ struct RouteArgs {
 // ---- launchers (routing.cu) -------------------------------------------------------------
 cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
                                  float* logits, int T, int H, int E, float* zero_buf,
-                                 size_t zero_floats, int32_t* status, cudaStream_t s);
-cudaError_t launch_softmax_topk(const float* logits, float* probs, int32_t* nat_idx, int T, int E,
-                                int k, int32_t* status, cudaStream_t s);
+                                 size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx, int k,
+                                 int32_t* tile_done, cudaStream_t s);
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s);
 // softmax/top-k + select (unless mask_override) + route + work lists in ONE single-CTA launch

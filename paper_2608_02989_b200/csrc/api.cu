@@ -333,6 +333,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_flag = carve(sizeof(int32_t) * 2 * c->sm_count);
   const size_t o_ready = carve(sizeof(int32_t) * 2 * kMaxSlots);
   const size_t o_status = carve(16);
+  const size_t o_tile = carve(sizeof(int32_t) * kMaxNodes);
   const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
   if (cudaMalloc(&c->ws_base, off) != cudaSuccess) return fail(ACM_ERR_NOMEM);
   if (cudaMemset(c->ws_base, 0, off) != cudaSuccess) return fail(ACM_ERR_CUDA);
@@ -354,6 +355,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.frag_flag = reinterpret_cast<int32_t*>(b + o_flag);
   c->ws.ready = reinterpret_cast<int32_t*>(b + o_ready);
   c->ws.status = reinterpret_cast<int32_t*>(b + o_status);
+  c->ws.tile_done = reinterpret_cast<int32_t*>(b + o_tile);
   c->resident_dev = reinterpret_cast<uint32_t*>(b + o_res);
   if (want_trace && cudaMalloc(&c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 16)) != cudaSuccess)
     return fail(ACM_ERR_NOMEM);
@@ -435,13 +437,10 @@ acm_status acm_router(acm_ctx* c, int layer, const void* x, int T, float* logits
   const acm_model_desc& d = c->desc;
   const Layer& L = c->layers[layer];
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // softmax and natural top-k are finished inside the same launch (last CTA of each node tile)
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, logits, T, d.hidden, d.n_experts, nullptr, 0,
-                                c->ws.status, s));
+                                c->ws.status, probs, nat_idx, d.top_k, c->ws.tile_done, s));
   c->launches += 1;
-  if (probs || nat_idx) {
-    ACM_CUDA(launch_softmax_topk(logits, probs, nat_idx, T, d.n_experts, d.top_k, c->ws.status, s));
-    c->launches += 1;
-  }
   return ACM_OK;
 }
 
@@ -528,8 +527,11 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   uint32_t* res_dev = L.has_resident ? c->resident_dev + 4 * layer : nullptr;
 
   // stage 1a (also clears the output the FFN accumulates into)
+  const bool need_probs = eligible_mask_override == nullptr;
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
-                                f32 ? 0 : static_cast<size_t>(T) * d.hidden, c->ws.status, s));
+                                f32 ? 0 : static_cast<size_t>(T) * d.hidden, c->ws.status,
+                                need_probs ? c->ws.probs : nullptr, need_probs ? c->ws.nat_idx : nullptr, k,
+                                c->ws.tile_done, s));
   // stages 1b-3 and the FFN work lists, one single-CTA launch
   SelectArgs sa;
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;

@@ -88,6 +88,40 @@ __device__ __forceinline__ float warp_tree_sum_128(float a0, float a1, float a2,
   return __shfl_sync(0xffffffffu, v, 0);
 }
 
+// Stage 1b for ONE node, by one warp: softmax over the expert axis (fixed recipe) and natural
+// top-k ranked on the logits.  `z_row` may have been written by other CTAs: read through L2.
+__device__ void softmax_topk_row(const float* z_row, float* probs_row, int32_t* nat_row, int E, int k, int lane) {
+  float z[4], y[4];
+  unsigned key[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const int e = lane + 32 * c;
+    const float v = __ldcg(z_row + min(e, E - 1));
+    z[c] = e < E ? v : -INFINITY;
+  }
+  float zmax = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, s));
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const float ex = exp_fixed(__fsub_rn(z[c], zmax));
+    y[c] = (lane + 32 * c < E) ? ex : 0.0f;
+    key[c] = (lane + 32 * c < E) ? order_key(z[c]) : 0u;
+  }
+  const float denom = warp_tree_sum_128(y[0], y[1], y[2], y[3]);
+  if (probs_row) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      if (lane + 32 * c < E) probs_row[lane + 32 * c] = __fdiv_rn(y[c], denom);
+  }
+  if (nat_row) {
+    for (int j = 0; j < k; ++j) {
+      const int e = warp_take_best(key, lane);
+      if (lane == 0) nat_row[j] = e;
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // Stage 1a: router logits.  CTA tile = 4 nodes x 8 experts (many small CTAs: the whole GPU works on
 // a 64 x 128 x 2048 product), rows staged in shared memory with 16-byte async copies in 4 K-chunks.
@@ -128,8 +162,8 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 template <typename Elem>
 __global__ void __launch_bounds__(kRT * kRE * (32 / ElemTraits<Elem>::EPT))
 k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const float* __restrict__ bias,
-                float* __restrict__ logits, int T, int H, int E, int n_chunks, float* zero_buf,
-                size_t zero_floats, int32_t* status) {
+                float* logits, int T, int H, int E, int n_chunks, float* zero_buf,
+                size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx, int k, int32_t* tile_done) {
   constexpr int EPT = ElemTraits<Elem>::EPT;
   constexpr int Q = 32 / EPT;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -214,6 +248,29 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
     logits[static_cast<size_t>(t) * E + e] = z;
     if (!isfinite(z)) raise_status(status, ACM_ERR_NONFINITE);
   }
+  // The CTA that completes a tile of nodes last (all expert tiles written) finishes those nodes:
+  // softmax and natural top-k, one warp per node -- spread over as many SMs as there are node tiles.
+  if (tile_done) {
+    __shared__ int s_last;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+      const int prev = atomicAdd(&tile_done[blockIdx.y], 1);
+      s_last = prev == static_cast<int>(gridDim.x) - 1;
+      if (s_last) tile_done[blockIdx.y] = 0;          // re-armed for the next call
+    }
+    __syncthreads();
+    if (s_last) {
+      __threadfence();
+      const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
+      for (int r = warp; r < kRT; r += nwarps) {
+        const int t = t0 + r;
+        if (t < T)
+          softmax_topk_row(logits + static_cast<size_t>(t) * E, probs ? probs + static_cast<size_t>(t) * E : nullptr,
+                           nat_idx ? nat_idx + static_cast<size_t>(t) * k : nullptr, E, k, lane);
+      }
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -240,83 +297,6 @@ struct StageSmem {
   float probs[kMaxNodes * kMaxExperts];   // r[t][e], so that the demand loop never waits on global memory
   float logits[kMaxNodes * kMaxExperts];  // z[t][e] (fused kernel only)
 };
-
-// Stage 1b: softmax over the expert axis and natural top-k (ranked on the logits).  One warp works on
-// two nodes at a time, interleaved, so that the warp-wide reductions of one overlap the other's.
-__device__ void stage_softmax_topk(const float* __restrict__ logits, float* __restrict__ probs,
-                                   int32_t* __restrict__ nat_idx, float* probs_smem, int32_t (*nat_smem)[kMaxTopK], int T,
-                                   int E, int k) {
-  constexpr int R = 2;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  for (int t0 = warp * R; t0 < T; t0 += nwarps * R) {
-    float z[R][4], y[R][4], zmax[R], denom[R];
-    unsigned key[R][4];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const int t = min(t0 + r, T - 1);      // a duplicate of the last node where the pair is incomplete
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int e = lane + 32 * c;
-        const float v = logits[static_cast<size_t>(t) * E + min(e, E - 1)];   // unconditional load, clamped index
-        z[r][c] = e < E ? v : -INFINITY;
-      }
-    }
-#pragma unroll
-    for (int r = 0; r < R; ++r) zmax[r] = fmaxf(fmaxf(z[r][0], z[r][1]), fmaxf(z[r][2], z[r][3]));
-#pragma unroll
-    for (int s = 16; s >= 1; s >>= 1) {
-#pragma unroll
-      for (int r = 0; r < R; ++r) zmax[r] = fmaxf(zmax[r], __shfl_xor_sync(0xffffffffu, zmax[r], s));
-    }
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const float ex = exp_fixed(__fsub_rn(z[r][c], zmax[r]));
-        y[r][c] = (lane + 32 * c < E) ? ex : 0.0f;
-        key[r][c] = (lane + 32 * c < E) ? order_key(z[r][c]) : 0u;
-      }
-      denom[r] = __fadd_rn(__fadd_rn(y[r][0], y[r][2]), __fadd_rn(y[r][1], y[r][3]));
-    }
-#pragma unroll
-    for (int s = 16; s >= 1; s >>= 1) {
-#pragma unroll
-      for (int r = 0; r < R; ++r) denom[r] = __fadd_rn(denom[r], __shfl_down_sync(0xffffffffu, denom[r], s));
-    }
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      denom[r] = __shfl_sync(0xffffffffu, denom[r], 0);
-      const int t = t0 + r;
-      if (t < T) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          if (lane + 32 * c < E) {
-            const float pr = __fdiv_rn(y[r][c], denom[r]);
-            if (probs) probs[static_cast<size_t>(t) * E + lane + 32 * c] = pr;
-            if (probs_smem) probs_smem[t * E + lane + 32 * c] = pr;
-          }
-        }
-      }
-    }
-    if (nat_idx || nat_smem) {
-      for (int j = 0; j < k; ++j) {
-        int e[R];
-#pragma unroll
-        for (int r = 0; r < R; ++r) e[r] = warp_take_best(key[r], lane);
-        if (lane == 0) {
-#pragma unroll
-          for (int r = 0; r < R; ++r) {
-            if (t0 + r < T) {
-              if (nat_idx) nat_idx[static_cast<size_t>(t0 + r) * k + j] = e[r];
-              if (nat_smem) nat_smem[t0 + r][j] = e[r];
-            }
-          }
-        }
-      }
-    }
-  }
-  __syncthreads();
-}
 
 // The selection stage runs on threads 0..127 only (one per expert slot) and synchronises them
 // with a named barrier, so the other warps of a larger CTA do not take part in its many barriers.
@@ -657,11 +637,6 @@ __device__ void stage_route(const RouteArgs& a, StageSmem& sm, int T, int E, int
   if (a.lists) stage_build_lists(a, sm, T, E, k);
 }
 
-__global__ void __launch_bounds__(1024) k_softmax_topk(const float* logits, float* probs, int32_t* nat_idx,
-                                                       int T, int E, int k) {
-  stage_softmax_topk(logits, probs, nat_idx, nullptr, nullptr, T, E, k);
-}
-
 extern __shared__ __align__(16) unsigned char routing_smem[];
 
 __global__ void __launch_bounds__(128) k_select(SelectArgs a, int T, int E, int k) {
@@ -704,7 +679,15 @@ __global__ void __launch_bounds__(1024) k_fused_select_route(const float* logits
     }
     __syncthreads();
   } else {
-    stage_softmax_topk(sm.logits, probs, nat_idx, sm.probs, sm.nat, T, E, k);
+    // probabilities and natural top-k were finished by the router kernel: bring them on chip
+    {
+      const float4* src = reinterpret_cast<const float4*>(probs);
+      float4* dst = reinterpret_cast<float4*>(sm.probs);
+      for (int i = threadIdx.x; i < T * E / 4; i += blockDim.x) dst[i] = __ldcg(src + i);
+      for (int i = (T * E / 4) * 4 + threadIdx.x; i < T * E; i += blockDim.x) sm.probs[i] = probs[i];
+      for (int i = threadIdx.x; i < T * k; i += blockDim.x) sm.nat[i / k][i % k] = nat_idx[i];
+    }
+    __syncthreads();
     ACM_RT(1);
     if (threadIdx.x < kMaxExperts) stage_select(sa, sm, T, E, k);
     __syncthreads();
@@ -732,7 +715,9 @@ __global__ void __launch_bounds__(512) k_routes_to_lists(const int32_t* idx, con
 
 cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
                                  float* logits, int T, int H, int E, float* zero_buf,
-                                 size_t zero_floats, int32_t* status, cudaStream_t s) {
+                                 size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx, int k,
+                                 int32_t* tile_done, cudaStream_t s) {
+  if (!probs && !nat_idx) tile_done = nullptr;
   const dim3 grid((E + kRE - 1) / kRE, (T + kRT - 1) / kRT);
   const int elt = dtype == ACM_F32 ? 4 : 2;
   const size_t smem = static_cast<size_t>(kRT + kRE) * (static_cast<size_t>(H) * elt + 64);
@@ -742,21 +727,14 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (err != cudaSuccess) return err;
     kern<<<grid, kRT * kRE * 8, smem, s>>>(static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
-                                 logits, T, H, E, n_chunks, zero_buf, zero_floats, status);
+                                 logits, T, H, E, n_chunks, zero_buf, zero_floats, status, probs, nat_idx, k, tile_done);
   } else {
     auto kern = k_router_logits<__nv_bfloat16>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (err != cudaSuccess) return err;
     kern<<<grid, kRT * kRE * 4, smem, s>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router),
-                                 bias, logits, T, H, E, n_chunks, zero_buf, zero_floats, status);
+                                 bias, logits, T, H, E, n_chunks, zero_buf, zero_floats, status, probs, nat_idx, k, tile_done);
   }
-  return cudaGetLastError();
-}
-
-cudaError_t launch_softmax_topk(const float* logits, float* probs, int32_t* nat_idx, int T, int E,
-                                int k, int32_t* /*status*/, cudaStream_t s) {
-  const int threads = min(1024, 32 * T);
-  k_softmax_topk<<<1, max(threads, 32), 0, s>>>(logits, probs, nat_idx, T, E, k);
   return cudaGetLastError();
 }
 
