@@ -49,8 +49,8 @@ struct Workspace {
   WorkList* lists;      // [2]: 0 = resident + shared, 1 = staged
   float* wdense;        // [2][kMaxSlots][64]
   void* hbuf;           // [2][kMaxSlots][64][I] bf16 (f32 path: [T][k+ns][I] float)
-  float* frag;          // [2][grid][128*64] split-K fragments (one buffer per gate/up segment)
-  int32_t* frag_flag;   // [2][grid] epoch of the fragment stored there
+  float* frag;          // [2][grid][128*64] split-K partial sums, accumulated into the finishing CTA's buffer; zero between launches
+  int32_t* frag_flag;   // [2][grid] how many CTAs have added to that buffer; zero between launches
   int32_t* ready;       // [2][kMaxSlots] finished gate/up tiles per activated slot
   int32_t* status;      // [1] sticky device-side status
   int32_t* tile_done;   // [64] router kernel: expert tiles finished per node tile (self-resetting)

@@ -43,6 +43,7 @@ struct acm_ctx {
   std::vector<Layer> layers;
   EncodeTiledFn encode = nullptr;
   int32_t epoch = 0;
+  size_t frag_bytes = 0, flag_bytes = 0;   // fragment buffers and arrival counters (zero between launches)
   CUtensorMap h_map[2];
   CUtensorMap h_store_map[2];            // same buffers, one 64-feature tile per TMA store
   int h_map_npad = 0;
@@ -352,6 +353,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.wdense = reinterpret_cast<float*>(b + o_wd);
   c->ws.hbuf = b + o_h;
   c->ws.frag = reinterpret_cast<float*>(b + o_frag);
+  c->frag_bytes = sizeof(float) * 2 * static_cast<size_t>(c->sm_count) * 128 * kMaxNodes;
+  c->flag_bytes = sizeof(int32_t) * 2 * c->sm_count;
   c->ws.frag_flag = reinterpret_cast<int32_t*>(b + o_flag);
   c->ws.ready = reinterpret_cast<int32_t*>(b + o_ready);
   c->ws.status = reinterpret_cast<int32_t*>(b + o_status);
@@ -665,7 +668,12 @@ acm_status acm_device_status(acm_ctx* c, acm_stream stream) {
   ACM_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
   int32_t v = 0;
   ACM_CUDA(cudaMemcpy(&v, c->ws.status, sizeof v, cudaMemcpyDeviceToHost));
-  if (v != 0) ACM_CUDA(cudaMemset(c->ws.status, 0, sizeof v));
+  if (v != 0) {
+    // a launch that gave up may have left partial sums behind: restore the all-zero state the FFN kernel expects
+    ACM_CUDA(cudaMemset(c->ws.status, 0, sizeof v));
+    ACM_CUDA(cudaMemset(c->ws.frag, 0, c->frag_bytes));
+    ACM_CUDA(cudaMemset(c->ws.frag_flag, 0, c->flag_bytes));
+  }
   return static_cast<acm_status>(v);
 }
 

@@ -124,6 +124,9 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
 __device__ __forceinline__ void st_release(int32_t* p, int v) {
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ void red_release_add(int32_t* p, int v) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
 // Bounded wait until *p >= target (p written by other CTAs with release semantics).
 __device__ bool flag_wait_ge(const int32_t* p, int target, volatile int* abort_flag, int32_t* status) {
   if (*abort_flag) return false;
@@ -578,36 +581,37 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->frag_free), (frag_uses - 1) & 1u, abort_flag, p.status));
           if (!ok) break;
         }
-        const float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * kFragFloats;
-        const int32_t* frag_flag = p.frag_flag + sg.p1_index * G;
+        float* frag = p.frag + (static_cast<size_t>(sg.p1_index) * G + cta) * kFragFloats;   // this CTA's buffer
+        int32_t* arrived = p.frag_flag + sg.p1_index * G + cta;
         const int n_el = p.n_pad * kTileM;
-        int c_first = -1;
-        for (int c2 = cta + 1; c2 < G && ok; ++c2) {
+        int n_contrib = 0;
+        for (int c2 = cta + 1; c2 < G; ++c2) {
           const long long b2 = U1 * c2 / G, e2 = U1 * (c2 + 1) / G;
           if (b2 >= tile_end) break;
-          if (e2 == b2) continue;
-          if (c_first < 0) c_first = c2;
-          bool got = true;
-          if (lane == 0) got = flag_wait_ge(&frag_flag[c2], p.epoch, abort_flag, p.status);
-          ok = __all_sync(0xffffffffu, got);
+          if (e2 > b2) ++n_contrib;
         }
-        if (!ok) break;
-        if (c_first >= 0) {
-          // every contributor has added its part to the first contributor's buffer: one bulk copy
+        {
+          // every CTA holding a later part of the tile has reduce-added its fragment: one bulk copy
+          bool got = true;
+          if (lane == 0) got = flag_wait_ge(arrived, n_contrib, abort_flag, p.status);
+          ok = __all_sync(0xffffffffu, got);
+          if (!ok) break;
           if (lane == 0) {
             fence_proxy_async();
             const uint32_t hb = smem_u32(&bars->helper);
             mbar_expect_tx(hb, static_cast<uint32_t>(n_el) * 4u);
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         ::"r"(smem_u32(sfrag)), "l"(frag + static_cast<size_t>(c_first) * kFragFloats),
-                           "r"(static_cast<uint32_t>(n_el) * 4u), "r"(hb) : "memory");
+                         ::"r"(smem_u32(sfrag)), "l"(frag), "r"(static_cast<uint32_t>(n_el) * 4u), "r"(hb) : "memory");
           }
           ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->helper), frag_uses & 1u, abort_flag, p.status));
+          if (!ok) break;
+          if (lane == 0) mbar_arrive(smem_u32(&bars->frag_full[sg.p1_index]));
+          if (lane == 0) ACM_TRACE(sg.p1_index == 0 ? 9 : 15);
+          // leave the buffer and its counter zero for the next launch
+          float4* z4 = reinterpret_cast<float4*>(frag);
+          for (int i = lane; i < n_el / 4; i += 32) z4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (lane == 0) *arrived = 0;
         }
-        if (!ok) break;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars->frag_full[sg.p1_index]));
-        if (lane == 0) ACM_TRACE(sg.p1_index == 0 ? 9 : 15);
         ++frag_uses;
       } else {
         // activation producer: once every activation tile of this expert group is stored, add the
@@ -670,28 +674,18 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           if (k0 > 0) {
             if (!(ok = mbar_wait(smem_u32(&bars->ost_full), ost_n & 1u, abort_flag, p.status))) break;
             const uint32_t bytes = static_cast<uint32_t>(p.n_pad) * kTileM * 4u;
-            // All CTAs that hold a tail part of this tile add into ONE global buffer, the one of the
-            // first of them: it copies, the others wait for that copy and then reduce-add on top.
+            // All CTAs that hold a tail part of this tile add into ONE global buffer, that of the CTA
+            // which owns the tile's first chunks and will finish it.  The buffers are zero between
+            // launches (the finishing CTA clears its own after reading), so nobody waits for anybody.
             const long long U1 = static_cast<long long>(sg.nt) * kc1;
             const long long tile_begin = static_cast<long long>(tile) * kc1;
             int c_head = cta - 1;
             while (c_head > 0 && U1 * c_head / G > tile_begin) --c_head;       // owner of the tile's first chunk
-            int c_first = c_head + 1;
-            while (c_first < cta && U1 * (c_first + 1) / G == U1 * c_first / G) ++c_first;   // skip empty ranges
-            float* dst = frag + static_cast<size_t>(c_first) * kFragFloats;
-            if (c_first == cta) {
-              asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                           ::"l"(dst), "r"(smem_u32(ostage)), "r"(bytes) : "memory");
-            } else {
-              if (!(ok = flag_wait_ge(&frag_flag[c_first], p.epoch, abort_flag, p.status))) break;
-              fence_proxy_async();
-              asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
-                           ::"l"(dst), "r"(smem_u32(ostage)), "r"(bytes) : "memory");
-            }
+            asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
+                         ::"l"(frag + static_cast<size_t>(c_head) * kFragFloats), "r"(smem_u32(ostage)), "r"(bytes) : "memory");
             bulk_commit();
             bulk_wait_all();
-            __threadfence();
-            st_release(&frag_flag[cta], p.epoch);
+            red_release_add(&frag_flag[c_head], 1);
             mbar_arrive(smem_u32(&bars->ost_free));
             ++ost_n;
           } else {
@@ -702,8 +696,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
                          ::"l"(&hs_map), "r"(0), "r"(0), "r"(ti), "r"(a), "r"(smem_u32(hstage + hb * kHStageBytes)) : "memory");
             bulk_commit();
             bulk_wait_all();
-            __threadfence();
-            atomicAdd(&p.ready[a >= a_split ? 1 : 0], 1);
+            red_release_add(&p.ready[a >= a_split ? 1 : 0], 1);
             mbar_arrive(smem_u32(&bars->hst_free[hb]));
             ++fin_n;
             ACM_TRACE(28);
