@@ -39,6 +39,7 @@ struct Workspace {
   float* logits;        // [T,E]
   float* probs;         // [T,E]
   int32_t* nat_idx;     // [T,k]
+  uint32_t* nat_mask;   // [T,4] the same sets as bit masks
   int32_t* idx;         // [T,k]
   float* w;             // [T,k]
   uint32_t* mask;       // [4] eligible set S'
@@ -54,6 +55,7 @@ struct Workspace {
   int32_t* ready;       // [2][kMaxSlots] finished gate/up tiles per activated slot
   int32_t* status;      // [1] sticky device-side status
   int32_t* tile_done;   // [64] router kernel: expert tiles finished per node tile (self-resetting)
+  int32_t* ticket;      // [1] select/route kernel: finished CTAs (self-resetting)
 };
 
 struct SelectArgs {
@@ -69,7 +71,7 @@ struct SelectArgs {
   int32_t* count_out;
   float* demand_out;             // may be null
   acm_block_stats* stats_out;    // may be null
-  long long* dbg;                // optional clock stamps (debugging aid)
+  long long* dbg;                // optional time stamps in ns (debugging aid)
 };
 
 struct RouteArgs {
@@ -87,21 +89,22 @@ struct RouteArgs {
   int n_shared;
   acm_block_stats* stats_out;    // n_activated / n_staged are filled in
   int32_t* host_stage_list;      // mapped pinned memory: [0] = n_stage, [1..] = expert ids (may be null)
-  long long* dbg;                // optional clock stamps of the fused kernel's stages (debugging aid)
+  long long* dbg;                // optional time stamps in ns of the select/route kernel's stages (debugging aid)
 };
 
 // ---- launchers (routing.cu) -------------------------------------------------------------
 cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
                                  float* logits, int T, int H, int E, float* zero_buf,
-                                 size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx, int k,
-                                 int32_t* tile_done, cudaStream_t s);
+                                 size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx,
+                                 uint32_t* nat_mask, int k, int32_t* tile_done, cudaStream_t s);
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s);
-// softmax/top-k + select (unless mask_override) + route + work lists in ONE single-CTA launch
-cudaError_t launch_fused_select_route(const float* logits, float* probs, int32_t* nat_idx,
-                                      const SelectArgs& sa, const RouteArgs& ra,
-                                      const uint32_t* mask_override, int T, int E, int k,
-                                      int32_t* status, cudaStream_t s);
+// select (unless mask_override) + route + work lists in ONE launch of ceil(T/4) small CTAs;
+// `nat_mask` = the natural top-k sets as bit masks [T][4] (from launch_router_logits), `ticket` = one
+// zero-initialised counter the kernel leaves at zero
+cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
+                                const uint32_t* mask_override, int T, int E, int k, int32_t* ticket,
+                                cudaStream_t s);
 cudaError_t launch_routes_to_lists(const int32_t* idx, const float* w, WorkList* lists, float* wdense,
                                    int32_t* ready, int n_shared, int T, int E, int k, cudaStream_t s);
 

@@ -335,6 +335,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_ready = carve(sizeof(int32_t) * 2 * kMaxSlots);
   const size_t o_status = carve(16);
   const size_t o_tile = carve(sizeof(int32_t) * kMaxNodes);
+  const size_t o_ticket = carve(16);
+  const size_t o_natmask = carve(sizeof(uint32_t) * Tm * kMaskWords);
   const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
   if (cudaMalloc(&c->ws_base, off) != cudaSuccess) return fail(ACM_ERR_NOMEM);
   if (cudaMemset(c->ws_base, 0, off) != cudaSuccess) return fail(ACM_ERR_CUDA);
@@ -359,6 +361,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.ready = reinterpret_cast<int32_t*>(b + o_ready);
   c->ws.status = reinterpret_cast<int32_t*>(b + o_status);
   c->ws.tile_done = reinterpret_cast<int32_t*>(b + o_tile);
+  c->ws.ticket = reinterpret_cast<int32_t*>(b + o_ticket);
+  c->ws.nat_mask = reinterpret_cast<uint32_t*>(b + o_natmask);
   c->resident_dev = reinterpret_cast<uint32_t*>(b + o_res);
   if (want_trace && cudaMalloc(&c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 16)) != cudaSuccess)
     return fail(ACM_ERR_NOMEM);
@@ -442,7 +446,7 @@ acm_status acm_router(acm_ctx* c, int layer, const void* x, int T, float* logits
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // softmax and natural top-k are finished inside the same launch (last CTA of each node tile)
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, logits, T, d.hidden, d.n_experts, nullptr, 0,
-                                c->ws.status, probs, nat_idx, d.top_k, c->ws.tile_done, s));
+                                c->ws.status, probs, nat_idx, nullptr, d.top_k, c->ws.tile_done, s));
   c->launches += 1;
   return ACM_OK;
 }
@@ -533,9 +537,9 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   const bool need_probs = eligible_mask_override == nullptr;
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
                                 f32 ? 0 : static_cast<size_t>(T) * d.hidden, c->ws.status,
-                                need_probs ? c->ws.probs : nullptr, need_probs ? c->ws.nat_idx : nullptr, k,
-                                c->ws.tile_done, s));
-  // stages 1b-3 and the FFN work lists, one single-CTA launch
+                                need_probs ? c->ws.probs : nullptr, need_probs ? c->ws.nat_idx : nullptr,
+                                need_probs ? c->ws.nat_mask : nullptr, k, c->ws.tile_done, s));
+  // stages 2-3 and the FFN work lists: one launch of a few small CTAs
   SelectArgs sa;
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
   sa.n_anchor_nodes = 0; sa.resident = prm.residency ? res_dev : nullptr; sa.prm = prm;
@@ -549,8 +553,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   ra.n_shared = d.n_shared; ra.host_stage_list = L.has_resident ? c->host_stage_list_dev : nullptr;
   ra.stats_out = c->ws.stats;
   ra.dbg = c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr;
-  ACM_CUDA(launch_fused_select_route(c->ws.logits, c->ws.probs, c->ws.nat_idx, sa, ra, eligible_mask_override, T, E,
-                                     k, c->ws.status, s));
+  ACM_CUDA(launch_select_route(c->ws.nat_mask, sa, ra, eligible_mask_override, T, E, k, c->ws.ticket, s));
   c->launches += 2;
 
   if (f32) {

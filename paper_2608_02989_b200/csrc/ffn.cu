@@ -121,9 +121,6 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void st_release(int32_t* p, int v) {
-  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
 __device__ __forceinline__ void red_release_add(int32_t* p, int v) {
   asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -385,6 +382,8 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, G = gridDim.x;
+  // the entries are fetched without waiting for the count: one global round trip, not two
+  const int32_t my_entry = threadIdx.x < kMaxSlots ? p.list->entry[threadIdx.x] : 0;
   const int n_act = p.list->n;
   const int tpe = p.I / 64;          // gate/up tiles per expert = K-chunks per expert in the down phase
   const int kc1 = p.H / (kBK * kAtoms);   // K-chunks (stages) of a gate/up tile
@@ -397,7 +396,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   const int n_seg = plan.n_seg;
   const int a_split = plan.a_split;
   int32_t* s_entry = bars->entry;
-  for (int i = threadIdx.x; i < n_act; i += blockDim.x) s_entry[i] = p.list->entry[i];
+  if (threadIdx.x < kMaxSlots) s_entry[threadIdx.x] = my_entry;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {

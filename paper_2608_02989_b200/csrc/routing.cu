@@ -14,6 +14,11 @@
 namespace acm {
 namespace {
 
+__device__ __forceinline__ long long time_ns() {     // one clock for every SM (debug stamps)
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return static_cast<long long>(t);
+}
 __device__ __forceinline__ void raise_status(int32_t* status, int code) {
   if (status) atomicCAS(status, 0, code);
 }
@@ -90,7 +95,8 @@ __device__ __forceinline__ float warp_tree_sum_128(float a0, float a1, float a2,
 
 // Stage 1b for ONE node, by one warp: softmax over the expert axis (fixed recipe) and natural
 // top-k ranked on the logits.  `z_row` may have been written by other CTAs: read through L2.
-__device__ void softmax_topk_row(const float* z_row, float* probs_row, int32_t* nat_row, int E, int k, int lane) {
+__device__ void softmax_topk_row(const float* z_row, float* probs_row, int32_t* nat_row, uint32_t* natmask_row,
+                                 int E, int k, int lane) {
   float z[4], y[4];
   unsigned key[4];
 #pragma unroll
@@ -115,10 +121,17 @@ __device__ void softmax_topk_row(const float* z_row, float* probs_row, int32_t* 
       if (lane + 32 * c < E) probs_row[lane + 32 * c] = __fdiv_rn(y[c], denom);
   }
   if (nat_row) {
+    uint32_t b0 = 0u, b1 = 0u, b2 = 0u, b3 = 0u;      // the same set as a bit mask (warp-uniform)
     for (int j = 0; j < k; ++j) {
       const int e = warp_take_best(key, lane);
       if (lane == 0) nat_row[j] = e;
+      if (e >= 0) {
+        const uint32_t bit = 1u << (e & 31);
+        const int wd = e >> 5;
+        b0 |= wd == 0 ? bit : 0u; b1 |= wd == 1 ? bit : 0u; b2 |= wd == 2 ? bit : 0u; b3 |= wd == 3 ? bit : 0u;
+      }
     }
+    if (natmask_row && lane < kMaskWords) natmask_row[lane] = lane == 0 ? b0 : lane == 1 ? b1 : lane == 2 ? b2 : b3;
   }
 }
 
@@ -163,7 +176,8 @@ template <typename Elem>
 __global__ void __launch_bounds__(kRT * kRE * (32 / ElemTraits<Elem>::EPT))
 k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const float* __restrict__ bias,
                 float* logits, int T, int H, int E, int n_chunks, float* zero_buf,
-                size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx, int k, int32_t* tile_done) {
+                size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k,
+                int32_t* tile_done) {
   constexpr int EPT = ElemTraits<Elem>::EPT;
   constexpr int Q = 32 / EPT;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -267,23 +281,30 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
         const int t = t0 + r;
         if (t < T)
           softmax_topk_row(logits + static_cast<size_t>(t) * E, probs ? probs + static_cast<size_t>(t) * E : nullptr,
-                           nat_idx ? nat_idx + static_cast<size_t>(t) * k : nullptr, E, k, lane);
+                           nat_idx ? nat_idx + static_cast<size_t>(t) * k : nullptr,
+                           nat_mask ? nat_mask + static_cast<size_t>(t) * kMaskWords : nullptr, E, k, lane);
       }
     }
   }
 }
 
 // ------------------------------------------------------------------------------------------
-// Block-cooperative stages.  Each is called by every thread of the CTA (>= 128 threads, a
-// multiple of 32) and ends with __syncthreads().
+// Stages 2 and 3.  The selection is a decision over the whole block (the demand sums over every
+// node), the routing is per node.  Rather than one CTA doing both for 64 nodes, a small grid runs
+// them: EVERY CTA repeats the selection on its 128 threads (it is deterministic, so all of them
+// hold the same S'), then routes its own four nodes, one warp each; the CTA that finishes last
+// gathers the routes into the FFN work lists.
 // ------------------------------------------------------------------------------------------
+constexpr int kNodesPerCta = 4;
+constexpr int kSelThreads = 128;
+
 struct StageSmem {
   float alpha[kMaxNodes];
   uint32_t natmask[kMaxNodes][kMaskWords];
   int32_t votes[kMaxExperts];
   float u[kMaxExperts];
   float tree[kMaxExperts + 4];
-  unsigned long long rkey[kMaxExperts];   // ranking keys of the experts (0 = not ranked)
+  alignas(16) unsigned long long rkey[kMaxExperts];   // ranking keys of the experts (0 = not ranked)
   uint32_t A[kMaskWords], S[kMaskWords], Sp[kMaskWords], Hres[kMaskWords];
   int32_t idx[kMaxNodes][kMaxTopK];
   float w[kMaxNodes][kMaxTopK];
@@ -292,14 +313,10 @@ struct StageSmem {
   int32_t list_of[kMaxExperts];
   int32_t warp_tot[2][4];
   int32_t scal[8];
-  float fscal[4];
-  int32_t nat[kMaxNodes][kMaxTopK];       // natural top-k of every node
-  float probs[kMaxNodes * kMaxExperts];   // r[t][e], so that the demand loop never waits on global memory
-  float logits[kMaxNodes * kMaxExperts];  // z[t][e] (fused kernel only)
 };
 
 // The selection stage runs on threads 0..127 only (one per expert slot) and synchronises them
-// with a named barrier, so the other warps of a larger CTA do not take part in its many barriers.
+// with a named barrier, so further warps of a larger CTA would not take part in its barriers.
 __device__ __forceinline__ void sel_sync() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 __device__ __forceinline__ int sel_count(bool pred) {
   int n;
@@ -323,69 +340,92 @@ __device__ float sel_tree_sum_128(float* tree, float mine) {
   return tree[kMaxExperts];
 }
 
-// Stage 2: demand, anchors, self-sizing, pruning.  Called by threads 0..127 only; thread e owns expert e.
-// Reads r from sm.probs and the natural top-k from sm.nat (the caller fills both).
-#define ACM_ST(slot) do { if (a.dbg && threadIdx.x == 0) a.dbg[slot] = clock64(); } while (0)
-__device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, int k) {
+// Stage 2: demand, anchors, self-sizing, pruning.  Called by threads 0..127; thread e owns expert e.
+// r comes straight from global memory (every load is issued before the first wait); the natural
+// top-k sets come as bit masks from `natmask_g` ([T][4], written by the router kernel) or, if that
+// is null, are built here from a.nat_idx.  Global results are written only if `write_out`.
+#define ACM_ST(slot) do { if (a.dbg && write_out && threadIdx.x == 0) a.dbg[slot] = time_ns(); } while (0)
+__device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, int k, const uint32_t* natmask_g,
+                             bool write_out) {
   const int tid = threadIdx.x;
   ACM_ST(5);
   const int lane = tid & 31, warp = tid >> 5;
   const bool live = tid < E;
-  for (int i = tid; i < kMaxNodes * kMaskWords; i += kMaxExperts) (&sm.natmask[0][0])[i] = 0u;
-  if (tid < kMaskWords) {
-    sm.A[tid] = 0u;
-    sm.Hres[tid] = (tid < (E + 31) / 32) ? (a.resident ? a.resident[tid] : 0xffffffffu) : 0u;
+  // small loads first (they gate the first barrier), then the 64 probabilities of this expert's column
+  const float my_alpha = tid < kMaxNodes ? a.alpha[min(tid, T - 1)] : 0.0f;
+  uint32_t my_nm[2] = {0u, 0u};
+  if (natmask_g) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) my_nm[i] = __ldcg(natmask_g + min(tid + i * kSelThreads, T * kMaskWords - 1));
   }
+  float pr[kMaxNodes];
+  {
+    const float* col = a.probs + min(tid, E - 1);
+#pragma unroll
+    for (int t = 0; t < kMaxNodes; ++t) pr[t] = __ldcg(col + static_cast<size_t>(min(t, T - 1)) * E);
+  }
+  if (tid < kMaxNodes) sm.alpha[tid] = my_alpha;
+  if (tid < kMaskWords) sm.Hres[tid] = (tid < (E + 31) / 32) ? (a.resident ? a.resident[tid] : 0xffffffffu) : 0u;
   if (tid < 8) sm.scal[tid] = 0;
-  for (int i = tid; i < T; i += kMaxExperts) sm.alpha[i] = a.alpha[i];
-  sel_sync();
-  for (int i = tid; i < T * k; i += kMaxExperts) {
-    const int e = sm.nat[i / k][i % k];
-    if (e >= 0 && e < E) atomicOr(&sm.natmask[i / k][e >> 5], 1u << (e & 31));
-  }
-  if (a.prm.use_anchors) {
-    const int n_nodes = a.anchor_nodes ? a.n_anchor_nodes : 1;
-    for (int i = tid; i < n_nodes * k; i += kMaxExperts) {
-      const int t = a.anchor_nodes ? a.anchor_nodes[i / k] : 0;
-      if (t >= 0 && t < T) {
-        const int e = sm.nat[t][i % k];
-        if (e >= 0 && e < E) atomicOr(&sm.A[e >> 5], 1u << (e & 31));
-      }
+  if (natmask_g) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) (&sm.natmask[0][0])[tid + i * kSelThreads] = my_nm[i];
+  } else {
+    for (int i = tid; i < kMaxNodes * kMaskWords; i += kSelThreads) (&sm.natmask[0][0])[i] = 0u;
+    sel_sync();
+    for (int i = tid; i < T * k; i += kSelThreads) {
+      const int e = a.nat_idx[i];
+      if (e >= 0 && e < E) atomicOr(&sm.natmask[i / k][e >> 5], 1u << (e & 31));
     }
   }
   sel_sync();
+  if (tid < kMaskWords) {           // anchors (Eq. 5): union of the anchor nodes' natural sets
+    uint32_t A = 0u;
+    if (a.prm.use_anchors) {
+      const int n_nodes = a.anchor_nodes ? a.n_anchor_nodes : 1;
+      for (int i = 0; i < n_nodes; ++i) {
+        const int t = a.anchor_nodes ? a.anchor_nodes[i] : 0;
+        if (t >= 0 && t < T) A |= sm.natmask[t][tid];
+      }
+    }
+    sm.A[tid] = A;
+  }
   ACM_ST(6);
 
   // votes v_e and demand u_e (nodes ascending, fused multiply-add)
   int votes = 0;
   float u = 0.0f;
   const int demand_mode = a.prm.demand;
-  if (live) {
-    for (int t0 = 0; t0 < T; t0 += 16) {
-      float pr[16], al[16];
+#pragma unroll
+  for (int t0 = 0; t0 < kMaxNodes; t0 += 16) {
+    if (t0 < T) {
+      float al[16];
       unsigned in_mask = 0;
 #pragma unroll
-      for (int j = 0; j < 16; ++j) {        // unconditional reads first (clamped index), then the ordered chain
+      for (int j = 0; j < 16; ++j) {
         const int t = min(t0 + j, T - 1);
-        pr[j] = sm.probs[t * E + tid];
         al[j] = sm.alpha[t];
         in_mask |= ((sm.natmask[t][warp] >> lane) & 1u) << j;
       }
-      if (t0 + 16 > T) in_mask &= (1u << (T - t0)) - 1u;
+      const unsigned valid = t0 + 16 > T ? (1u << (T - t0)) - 1u : 0xffffu;
+      in_mask &= valid;
       votes += __popc(in_mask);
+      // which nodes enter the chain; the chain itself is branch-free (multiply-add, then select)
+      const unsigned take = demand_mode == ACM_DEMAND_FULL_MASS ? valid
+                          : demand_mode == ACM_DEMAND_TOPK_MASS ? in_mask : 0u;
 #pragma unroll
       for (int j = 0; j < 16; ++j) {
-        const bool take = t0 + j < T && (demand_mode == ACM_DEMAND_FULL_MASS ||
-                                         (demand_mode == ACM_DEMAND_TOPK_MASS && ((in_mask >> j) & 1u)));
-        if (take) u = __fmaf_rn(al[j], pr[j], u);
+        const float nu = __fmaf_rn(al[j], pr[t0 + j], u);
+        u = ((take >> j) & 1u) ? nu : u;
       }
-      if (a.dbg && threadIdx.x == 0) a.dbg[13 + (t0 >> 4)] = clock64() + __float_as_int(u) * 0;
     }
-    if (a.prm.demand == ACM_DEMAND_VOTES) u = static_cast<float>(votes);
   }
+  if (!live) { votes = 0; u = 0.0f; }
+  if (a.prm.demand == ACM_DEMAND_VOTES) u = static_cast<float>(votes);
   ACM_ST(7);
   sm.votes[tid] = votes;
   sm.u[tid] = u;
+  sel_sync();                       // sm.A
   const bool in_A = live && ((sm.A[warp] >> lane) & 1u);
   const bool in_R = live && !in_A;
   const int nA = sel_count(in_A);
@@ -421,8 +461,12 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   bool in_S = in_A;
   if (in_R) {
     int rank = 0;
-#pragma unroll 16
-    for (int j = 0; j < kMaxExperts; ++j) rank += sm.rkey[j] > mykey ? 1 : 0;
+    const ulonglong2* keys2 = reinterpret_cast<const ulonglong2*>(sm.rkey);
+#pragma unroll 8
+    for (int j = 0; j < kMaxExperts / 2; ++j) {
+      const ulonglong2 kk = keys2[j];
+      rank += (kk.x > mykey ? 1 : 0) + (kk.y > mykey ? 1 : 0);
+    }
     in_S = rank < n_keep;
   }
   ACM_ST(10);
@@ -465,20 +509,22 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   if (a.prm.residency == 2 && a.resident) m_star = nS - nSp;
 
   ACM_ST(12);
-  const int words = (E + 31) / 32;
-  if (tid < words) {
-    a.mask_out[tid] = sm.Sp[tid];
-    if (a.unpruned_out) a.unpruned_out[tid] = sm.S[tid];
-  }
-  if (live && a.demand_out) a.demand_out[tid] = u;
-  if (tid == 0) {
-    *a.count_out = nSp;
-    if (a.stats_out) {
-      acm_block_stats st;
-      st.n_anchor = nA; st.n_er = n_er; st.n_eligible = nS; st.n_eligible_pruned = nSp;
-      st.n_activated = 0; st.n_natural_union = n_union; st.displaced_aS = aS; st.pruned_m = m_star;
-      st.n_staged = 0; st.reserved[0] = st.reserved[1] = st.reserved[2] = 0;
-      *a.stats_out = st;
+  if (write_out) {
+    const int words = (E + 31) / 32;
+    if (tid < words) {
+      a.mask_out[tid] = sm.Sp[tid];
+      if (a.unpruned_out) a.unpruned_out[tid] = sm.S[tid];
+    }
+    if (live && a.demand_out) a.demand_out[tid] = u;
+    if (tid == 0) {
+      *a.count_out = nSp;
+      if (a.stats_out) {
+        acm_block_stats st;
+        st.n_anchor = nA; st.n_er = n_er; st.n_eligible = nS; st.n_eligible_pruned = nSp;
+        st.n_activated = 0; st.n_natural_union = n_union; st.displaced_aS = aS; st.pruned_m = m_star;
+        st.n_staged = 0; st.reserved[0] = st.reserved[1] = st.reserved[2] = 0;
+        *a.stats_out = st;
+      }
     }
   }
   sel_sync();
@@ -486,17 +532,18 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
 
 // Turns per-node routes (sm.idx / sm.w) into the FFN work lists: activated experts in ascending
 // id order, shared experts appended; combine weights scattered into the dense [slot][node] table.
-__device__ void stage_build_lists(const RouteArgs& a, StageSmem& sm, int T, int E, int k) {
+// `zero`: also clear the dense tables and the finished-tile counters here (otherwise the caller has).
+__device__ void stage_build_lists(const RouteArgs& a, StageSmem& sm, int T, int E, int k, bool zero) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid < kMaxExperts) sm.cnt[tid] = 0;
-  {
+  if (zero) {
     const int rows = E + a.n_shared;     // slots that can be occupied in a list
     for (int i = tid; i < rows * kMaxNodes; i += blockDim.x) {
       a.wdense[i] = 0.0f;
       if (a.resident) a.wdense[kMaxSlots * kMaxNodes + i] = 0.0f;
     }
+    for (int i = tid; i < 2 * kMaxSlots; i += blockDim.x) a.ready[i] = 0;
   }
-  for (int i = tid; i < 2 * kMaxSlots; i += blockDim.x) a.ready[i] = 0;
   if (tid < kMaskWords) sm.Hres[tid] = a.resident ? (tid < (E + 31) / 32 ? a.resident[tid] : 0u) : 0xffffffffu;
   __syncthreads();
   for (int i = tid; i < T * k; i += blockDim.x) {
@@ -557,166 +604,170 @@ __device__ void stage_build_lists(const RouteArgs& a, StageSmem& sm, int T, int 
   __syncthreads();
 }
 
-// Stage 3: restricted top-k (Eq. 2) and combine weights, one warp per node.
-__device__ void stage_route(const RouteArgs& a, StageSmem& sm, int T, int E, int k) {
-  constexpr int R = 2;                       // two nodes per warp at a time, interleaved
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+// Stage 3 for ONE node, by one warp: restricted top-k (Eq. 2) ranked on the logits, and the
+// combine weights.  Lane j < k returns the j-th choice (expert id or -1) and its weight.
+__device__ __forceinline__ void route_node(const float (&z)[4], const uint32_t (&mask_w)[4], int E, int k, int lane,
+                                           int weighting, float routed_scale, int& e_out, float& w_out) {
+  float y[4];
+  unsigned key[4];
+  float zmax = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
+#pragma unroll
+  for (int s = 16; s >= 1; s >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, s));
+  float s_all = 0.f, s_elig = 0.f, s_sel = 0.f, my_y = 0.f;
+  int my_e = -1;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const bool in_e = lane + 32 * c < E;
+    const bool elig = in_e && ((mask_w[c] >> lane) & 1u);
+    y[c] = in_e ? __expf(z[c] - zmax) : 0.0f;
+    s_all += y[c];
+    s_elig += elig ? y[c] : 0.0f;
+    key[c] = elig ? order_key(z[c]) : 0u;
+  }
+  if (weighting != ACM_W_RENORM_TOPK) {      // warp-uniform: only the denominator that is used
+    float other = weighting == ACM_W_SOFTMAX_RAW ? s_all : s_elig;
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) other += __shfl_xor_sync(0xffffffffu, other, s);
+    s_all = s_elig = other;
+  }
+  for (int j = 0; j < k; ++j) {
+    const int e = warp_take_best(key, lane);
+    const int c = (e >= 0 ? e : 0) >> 5;
+    const float cand = c == 0 ? y[0] : c == 1 ? y[1] : c == 2 ? y[2] : y[3];
+    const float got = __shfl_sync(0xffffffffu, cand, (e >= 0 ? e : 0) & 31);
+    const float ye = e >= 0 ? got : 0.f;
+    s_sel += ye;
+    if (lane == j) { my_e = e; my_y = ye; }
+  }
+  const float den = weighting == ACM_W_RENORM_TOPK ? s_sel : weighting == ACM_W_SOFTMAX_RAW ? s_all : s_elig;
+  e_out = my_e;
+  w_out = my_e >= 0 ? routed_scale * my_y / den : 0.0f;
+}
+
+__device__ __forceinline__ void load_logit_row(const float* logits, int t, int E, int lane, float (&z)[4]) {
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const int e = lane + 32 * c;
+    const float v = __ldcg(logits + static_cast<size_t>(t) * E + min(e, E - 1));
+    z[c] = e < E ? v : -INFINITY;
+  }
+}
+
+__global__ void __launch_bounds__(kSelThreads) k_select(SelectArgs a, int T, int E, int k) {
+  __shared__ StageSmem sm;
+  stage_select(a, sm, T, E, k, nullptr, true);
+}
+
+// grid = ceil(T / 4) CTAs of four warps, one node per warp
+__global__ void __launch_bounds__(kSelThreads) k_route(RouteArgs a, int T, int E, int k) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = blockIdx.x * kNodesPerCta + warp;
+  if (t >= T) return;
+  float z[4];
   uint32_t mask_w[4];
+  load_logit_row(a.logits, t, E, lane, z);
 #pragma unroll
   for (int c = 0; c < 4; ++c) mask_w[c] = a.mask[min(c, (E + 31) / 32 - 1)];
-  for (int t0 = warp * R; t0 < T; t0 += nwarps * R) {
-    float z[R][4], y[R][4], zmax[R], s_all[R], s_elig[R], s_sel[R], my_y[R];
-    unsigned key[R][4];
-    int my_e[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      const int t = min(t0 + r, T - 1);
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int e = lane + 32 * c;
-        const float v = a.logits[static_cast<size_t>(t) * E + min(e, E - 1)];
-        z[r][c] = e < E ? v : -INFINITY;
-      }
-      zmax[r] = fmaxf(fmaxf(z[r][0], z[r][1]), fmaxf(z[r][2], z[r][3]));
-    }
-#pragma unroll
-    for (int s = 16; s >= 1; s >>= 1) {
-#pragma unroll
-      for (int r = 0; r < R; ++r) zmax[r] = fmaxf(zmax[r], __shfl_xor_sync(0xffffffffu, zmax[r], s));
-    }
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-      s_all[r] = 0.f; s_elig[r] = 0.f; s_sel[r] = 0.f; my_y[r] = 0.f; my_e[r] = -1;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const bool in_e = lane + 32 * c < E;
-        const bool elig = in_e && ((mask_w[c] >> lane) & 1u);
-        y[r][c] = in_e ? __expf(z[r][c] - zmax[r]) : 0.0f;
-        s_all[r] += y[r][c];
-        s_elig[r] += elig ? y[r][c] : 0.0f;
-        key[r][c] = elig ? order_key(z[r][c]) : 0u;
-      }
-    }
-#pragma unroll
-    for (int s = 16; s >= 1; s >>= 1) {
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-        s_all[r] += __shfl_xor_sync(0xffffffffu, s_all[r], s);
-        s_elig[r] += __shfl_xor_sync(0xffffffffu, s_elig[r], s);
-      }
-    }
-    for (int j = 0; j < k; ++j) {
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-        const int e = warp_take_best(key[r], lane);
-        const int c = (e >= 0 ? e : 0) >> 5;
-        const float cand = c == 0 ? y[r][0] : c == 1 ? y[r][1] : c == 2 ? y[r][2] : y[r][3];
-        const float got = __shfl_sync(0xffffffffu, cand, (e >= 0 ? e : 0) & 31);
-        const float ye = e >= 0 ? got : 0.f;
-        s_sel[r] += ye;
-        if (lane == j) { my_e[r] = e; my_y[r] = ye; }
-      }
-    }
-    if (lane < k) {
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-        const int t = t0 + r;
-        if (t < T) {
-          const float den = a.weighting == ACM_W_RENORM_TOPK ? s_sel[r] : a.weighting == ACM_W_SOFTMAX_RAW ? s_all[r] : s_elig[r];
-          const float wgt = my_e[r] >= 0 ? a.routed_scale * my_y[r] / den : 0.0f;
-          sm.idx[t][lane] = my_e[r];
-          sm.w[t][lane] = wgt;
-          if (a.idx_out) a.idx_out[static_cast<size_t>(t) * k + lane] = my_e[r];
-          if (a.w_out) a.w_out[static_cast<size_t>(t) * k + lane] = wgt;
-        }
-      }
-    }
+  int e;
+  float w;
+  route_node(z, mask_w, E, k, lane, a.weighting, a.routed_scale, e, w);
+  if (lane < k) {
+    a.idx_out[static_cast<size_t>(t) * k + lane] = e;
+    a.w_out[static_cast<size_t>(t) * k + lane] = w;
   }
-  __syncthreads();
-  if (a.dbg && threadIdx.x == 0) a.dbg[3] = clock64();
-  if (a.lists) stage_build_lists(a, sm, T, E, k);
 }
 
-extern __shared__ __align__(16) unsigned char routing_smem[];
-
-__global__ void __launch_bounds__(128) k_select(SelectArgs a, int T, int E, int k) {
-  StageSmem& sm = *reinterpret_cast<StageSmem*>(routing_smem);
-  for (int i = threadIdx.x; i < T * E; i += blockDim.x) sm.probs[i] = a.probs[i];
-  for (int i = threadIdx.x; i < T * k; i += blockDim.x) sm.nat[i / k][i % k] = a.nat_idx[i];
-  __syncthreads();
-  stage_select(a, sm, T, E, k);
-}
-
-__global__ void __launch_bounds__(1024) k_route(RouteArgs a, int T, int E, int k) {
-  StageSmem& sm = *reinterpret_cast<StageSmem*>(routing_smem);
-  stage_route(a, sm, T, E, k);
-}
-
-#define ACM_RT(slot) do { if (ra.dbg && threadIdx.x == 0) ra.dbg[slot] = clock64(); } while (0)
-// Stages 1b-3 in one CTA.  The logits are staged in shared memory once; every later stage reads
-// shared memory only, and the selection stage runs on four warps while the others wait.
-__global__ void __launch_bounds__(1024) k_fused_select_route(const float* logits, float* probs, int32_t* nat_idx,
-                                                             SelectArgs sa, RouteArgs ra,
-                                                             const uint32_t* mask_override, int T, int E, int k) {
-  StageSmem& sm = *reinterpret_cast<StageSmem*>(routing_smem);
+#define ACM_RT(slot) do { if (ra.dbg && blockIdx.x == 0 && threadIdx.x == 0) ra.dbg[slot] = time_ns(); } while (0)
+// Stages 2-3 and the FFN work lists in one launch of ceil(T / 4) CTAs (see the note above).
+// `ticket` counts finished CTAs (zero on entry, reset by the last one).
+__global__ void __launch_bounds__(kSelThreads)
+k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uint32_t* mask_override, int T, int E,
+               int k, int32_t* ticket) {
+  __shared__ StageSmem sm;
+  __shared__ int s_last;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int t_mine = blockIdx.x * kNodesPerCta + warp;
   ACM_RT(0);
+  float z[4];
+  load_logit_row(ra.logits, min(t_mine, T - 1), E, lane, z);      // in flight during the selection
   {
-    const float4* src = reinterpret_cast<const float4*>(logits);
-    float4* dst = reinterpret_cast<float4*>(sm.logits);
-    for (int i = threadIdx.x; i < T * E / 4; i += blockDim.x) dst[i] = __ldcg(src + i);
-    for (int i = (T * E / 4) * 4 + threadIdx.x; i < T * E; i += blockDim.x) sm.logits[i] = logits[i];
-  }
-  __syncthreads();
-  if (mask_override) {
-    if (threadIdx.x < kMaskWords) {
-      const uint32_t m = threadIdx.x < (E + 31) / 32 ? mask_override[threadIdx.x] : 0u;
-      sm.Sp[threadIdx.x] = m;
-      if (threadIdx.x < (E + 31) / 32) sa.mask_out[threadIdx.x] = m;
+    // clear this CTA's share of the dense combine-weight tables and (CTA 0) the finished-tile counters
+    const int n4 = (E + ra.n_shared) * kMaxNodes / 4;
+    float4* wd = reinterpret_cast<float4*>(ra.wdense);
+    for (int i = blockIdx.x * kSelThreads + tid; i < n4; i += gridDim.x * kSelThreads) {
+      wd[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (ra.resident) wd[kMaxSlots * kMaxNodes / 4 + i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    if (threadIdx.x == 0 && sa.stats_out) {
+    if (blockIdx.x == 0)
+      for (int i = tid; i < 2 * kMaxSlots; i += kSelThreads) ra.ready[i] = 0;
+  }
+  if (mask_override) {
+    if (tid < kMaskWords) {
+      const uint32_t m = tid < (E + 31) / 32 ? mask_override[tid] : 0u;
+      sm.Sp[tid] = m;
+      if (blockIdx.x == 0 && tid < (E + 31) / 32) sa.mask_out[tid] = m;
+    }
+    if (blockIdx.x == 0 && tid == 0 && sa.stats_out) {
       acm_block_stats st = {};
       *sa.stats_out = st;
     }
     __syncthreads();
   } else {
-    // probabilities and natural top-k were finished by the router kernel: bring them on chip
-    {
-      const float4* src = reinterpret_cast<const float4*>(probs);
-      float4* dst = reinterpret_cast<float4*>(sm.probs);
-      for (int i = threadIdx.x; i < T * E / 4; i += blockDim.x) dst[i] = __ldcg(src + i);
-      for (int i = (T * E / 4) * 4 + threadIdx.x; i < T * E; i += blockDim.x) sm.probs[i] = probs[i];
-      for (int i = threadIdx.x; i < T * k; i += blockDim.x) sm.nat[i / k][i % k] = nat_idx[i];
-    }
-    __syncthreads();
-    ACM_RT(1);
-    if (threadIdx.x < kMaxExperts) stage_select(sa, sm, T, E, k);
-    __syncthreads();
-    ACM_RT(2);
+    stage_select(sa, sm, T, E, k, natmask_g, blockIdx.x == 0);
   }
-  ra.logits = sm.logits;
-  ra.mask = sm.Sp;
-  stage_route(ra, sm, T, E, k);
-  ACM_RT(4);
+  ACM_RT(2);
+  {
+    uint32_t mask_w[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) mask_w[c] = sm.Sp[c];
+    int e;
+    float w;
+    route_node(z, mask_w, E, k, lane, ra.weighting, ra.routed_scale, e, w);
+    if (t_mine < T && lane < k) {
+      ra.idx_out[static_cast<size_t>(t_mine) * k + lane] = e;
+      ra.w_out[static_cast<size_t>(t_mine) * k + lane] = w;
+    }
+  }
+  ACM_RT(3);
+  // the CTA that finishes last sees every route and builds the lists
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int prev = atomicAdd(ticket, 1);
+    s_last = prev == static_cast<int>(gridDim.x) - 1;
+    if (s_last) *ticket = 0;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  for (int i = tid; i < T * k; i += kSelThreads) {
+    sm.idx[i / k][i % k] = __ldcg(ra.idx_out + i);
+    sm.w[i / k][i % k] = __ldcg(ra.w_out + i);
+  }
+  __syncthreads();
+  if (ra.dbg && tid == 0) ra.dbg[1] = time_ns();
+  stage_build_lists(ra, sm, T, E, k, false);
+  if (ra.dbg && tid == 0) ra.dbg[4] = time_ns();
 }
 
 __global__ void __launch_bounds__(512) k_routes_to_lists(const int32_t* idx, const float* w, RouteArgs a, int T,
                                                          int E, int k) {
-  StageSmem& sm = *reinterpret_cast<StageSmem*>(routing_smem);
+  __shared__ StageSmem sm;
   for (int i = threadIdx.x; i < T * k; i += blockDim.x) {
     const int e = idx[i];
     sm.idx[i / k][i % k] = (e >= 0 && e < E) ? e : -1;
     sm.w[i / k][i % k] = w[i];
   }
   __syncthreads();
-  stage_build_lists(a, sm, T, E, k);
+  stage_build_lists(a, sm, T, E, k, true);
 }
 
 }  // namespace
 
 cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
                                  float* logits, int T, int H, int E, float* zero_buf,
-                                 size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx, int k,
-                                 int32_t* tile_done, cudaStream_t s) {
+                                 size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx,
+                                 uint32_t* nat_mask, int k, int32_t* tile_done, cudaStream_t s) {
   if (!probs && !nat_idx) tile_done = nullptr;
   const dim3 grid((E + kRE - 1) / kRE, (T + kRT - 1) / kRT);
   const int elt = dtype == ACM_F32 ? 4 : 2;
@@ -727,40 +778,35 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (err != cudaSuccess) return err;
     kern<<<grid, kRT * kRE * 8, smem, s>>>(static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
-                                 logits, T, H, E, n_chunks, zero_buf, zero_floats, status, probs, nat_idx, k, tile_done);
+                                           logits, T, H, E, n_chunks, zero_buf, zero_floats, status, probs, nat_idx,
+                                           nat_mask, k, tile_done);
   } else {
     auto kern = k_router_logits<__nv_bfloat16>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (err != cudaSuccess) return err;
-    kern<<<grid, kRT * kRE * 4, smem, s>>>(static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w_router),
-                                 bias, logits, T, H, E, n_chunks, zero_buf, zero_floats, status, probs, nat_idx, k, tile_done);
+    kern<<<grid, kRT * kRE * 4, smem, s>>>(static_cast<const __nv_bfloat16*>(x),
+                                           static_cast<const __nv_bfloat16*>(w_router), bias, logits, T, H, E,
+                                           n_chunks, zero_buf, zero_floats, status, probs, nat_idx, nat_mask, k,
+                                           tile_done);
   }
   return cudaGetLastError();
 }
 
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s) {
-  cudaError_t err = cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(StageSmem)));
-  if (err != cudaSuccess) return err;
-  k_select<<<1, 128, sizeof(StageSmem), s>>>(a, T, E, k);
+  k_select<<<1, kSelThreads, 0, s>>>(a, T, E, k);
   return cudaGetLastError();
 }
 
 cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s) {
-  const int threads = max(128, min(1024, 32 * T));
-  cudaError_t err = cudaFuncSetAttribute(k_route, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(StageSmem)));
-  if (err != cudaSuccess) return err;
-  k_route<<<1, threads, sizeof(StageSmem), s>>>(a, T, E, k);
+  k_route<<<(T + kNodesPerCta - 1) / kNodesPerCta, kSelThreads, 0, s>>>(a, T, E, k);
   return cudaGetLastError();
 }
 
-cudaError_t launch_fused_select_route(const float* logits, float* probs, int32_t* nat_idx,
-                                      const SelectArgs& sa, const RouteArgs& ra,
-                                      const uint32_t* mask_override, int T, int E, int k,
-                                      int32_t* /*status*/, cudaStream_t s) {
-  const int threads = max(128, min(1024, 32 * ((T + 1) / 2)));     // two nodes per warp in the per-node stages
-  cudaError_t err = cudaFuncSetAttribute(k_fused_select_route, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(StageSmem)));
-  if (err != cudaSuccess) return err;
-  k_fused_select_route<<<1, threads, sizeof(StageSmem), s>>>(logits, probs, nat_idx, sa, ra, mask_override, T, E, k);
+cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
+                                const uint32_t* mask_override, int T, int E, int k, int32_t* ticket,
+                                cudaStream_t s) {
+  k_select_route<<<(T + kNodesPerCta - 1) / kNodesPerCta, kSelThreads, 0, s>>>(nat_mask, sa, ra, mask_override, T, E,
+                                                                              k, ticket);
   return cudaGetLastError();
 }
 
@@ -771,9 +817,7 @@ cudaError_t launch_routes_to_lists(const int32_t* idx, const float* w, WorkList*
   a.wdense = wdense;
   a.ready = ready;
   a.n_shared = n_shared;
-  cudaError_t err = cudaFuncSetAttribute(k_routes_to_lists, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(sizeof(StageSmem)));
-  if (err != cudaSuccess) return err;
-  k_routes_to_lists<<<1, 512, sizeof(StageSmem), s>>>(idx, w, a, T, E, k);
+  k_routes_to_lists<<<1, 512, 0, s>>>(idx, w, a, T, E, k);
   return cudaGetLastError();
 }
 
