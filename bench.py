@@ -15,6 +15,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import subprocess
 import sys
@@ -204,6 +205,7 @@ def cpu_baseline(cfg, budget_s=15.0):
 def run_acm(args, world, rank, local):
     import ctypes
 
+    import numpy as np
     import torch
 
     from paper_2608_02989_b200 import acm, workloads as wl
@@ -266,12 +268,24 @@ def run_acm(args, world, rank, local):
             if rc:
                 raise acm.AcmError(rc, "acm_moe_verify")
 
+    # Every `period`-th launch of the FFN kernel is bracketed by events (a bracketed launch cannot
+    # overlap its set-up with the kernel before it, so bracketing all of them would slow the step it
+    # measures).  The period is coprime with the layer count: over the steps every layer is sampled.
+    period = 1
+    if not resident:
+        period = 5
+        while math.gcd(period, L) != 1:
+            period += 1
+
+    def sampled_layers(steps):
+        return np.arange(0, steps * L, period) % L
+
     def timed(calls, steps, warmup, with_roofline):
         for _ in range(warmup):
             step(calls)
         barrier()
         if with_roofline:
-            ctx.ffn_timing(True, steps * L * 2)
+            ctx.ffn_timing(period, steps * L * 2)
         n0 = ctx.launch_count()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
@@ -298,14 +312,15 @@ def run_acm(args, world, rank, local):
     expert_bytes = cfg.expert_bytes
     # algorithmic bytes of one FFN launch: the activated experts' weights (+ shared), x in, y out
     alg_bytes = (n_act + cfg.n_shared) * expert_bytes + T * H * 2 + T * H * 4
-    alg_per_launch = float(alg_bytes.mean())
+    alg_per_launch = float(alg_bytes[sampled_layers(args.steps)].mean()) if not resident else float(alg_bytes.mean())
     value = world * L * args.steps / (ms * 1e-3)
 
     nat = None
     if not args.no_natural:
         ms_n, _, ffn_ms_n, ffn_n_n = timed(calls_nat, args.steps, 3, True)
         st_n = stats.cpu().numpy()
-        nat_bytes = float(((st_n[:, 4] + cfg.n_shared) * expert_bytes + T * H * 6).mean())
+        nat_bytes = (st_n[:, 4] + cfg.n_shared) * expert_bytes + T * H * 6
+        nat_bytes = float(nat_bytes[sampled_layers(args.steps)].mean()) if not resident else float(nat_bytes.mean())
         nat = {"value": world * L * args.steps / (ms_n * 1e-3), "unit": UNIT, "ms_per_step": ms_n / args.steps,
                "mean_activated_experts": float(st_n[:, 4].mean()),
                "ffn_us_per_launch": 1e3 * ffn_ms_n / max(ffn_n_n, 1),
@@ -353,7 +368,7 @@ def run_acm(args, world, rank, local):
     # DRAM bytes (read + write) of k_ffn_bf16 per activated expert, from the ncu capture summarised in
     # profiles/k_ffn_bf16_c3_layer.txt (4-layer case; traffic is proportional to the activated experts)
     per_expert = DRAM_BYTES_PER_ACTIVATED_EXPERT.get(cfg.index)
-    traffic = per_expert * float(n_act.mean() + cfg.n_shared) if per_expert else None
+    traffic = per_expert * (alg_per_launch - T * H * 6) / expert_bytes if per_expert else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -370,6 +385,7 @@ def run_acm(args, world, rank, local):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": (achieved / peak) if achieved else None, "traffic": traffic, "peak_kind": peak_kind,
                      "kernel": "k_ffn_bf16", "us_per_launch": ffn_us, "launches_timed": ffn_n,
+                     "timed_every": period,
                      "algorithmic_bytes_per_launch": alg_per_launch},
         "natural_union_path": nat,
         "e2e": e2e,

@@ -184,8 +184,11 @@ acm_status acm_set_resident(acm_ctx* ctx, int layer, const uint32_t* resident_ma
 acm_status acm_h2d_bytes(acm_ctx* ctx, uint64_t* bytes_out /*host*/, int reset);
 
 /* Per-launch timing of the expert-FFN kernel with CUDA events on the launching stream.
- * enable != 0 starts recording (at most `capacity` launches are kept); acm_ffn_time_ms
- * synchronises those events and returns their summed duration and count (host pointers). */
+ * enable = n > 0 starts recording every n-th launch of that kernel, counted from this call (n = 1:
+ * every launch; at most `capacity` launches are kept); enable = 0 stops.  A bracketed launch is
+ * ordered strictly after the kernel before it (no dependent-launch overlap), so its duration is the
+ * kernel's own.  acm_ffn_time_ms synchronises the events and returns their summed duration and
+ * count (host pointers). */
 acm_status acm_ffn_timing(acm_ctx* ctx, int enable, int capacity);
 acm_status acm_ffn_time_ms(acm_ctx* ctx, float* total_ms, int32_t* launches);
 

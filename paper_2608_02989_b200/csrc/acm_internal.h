@@ -92,11 +92,22 @@ struct RouteArgs {
   long long* dbg;                // optional time stamps in ns of the select/route kernel's stages (debugging aid)
 };
 
+// Programmatic dependent launch: a kernel launched with `pdl` may start while the kernel before it
+// in the stream is still running; it runs its set-up, then waits (griddepcontrol.wait) for that
+// kernel to complete before it touches global memory.  Every kernel of the hot path signals its
+// dependents at once and waits before its first global access, so completion stays transitive.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+inline void set_pdl_attr(cudaLaunchAttribute* attr) {
+  attr->id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr->val.programmaticStreamSerializationAllowed = 1;
+}
+
 // ---- launchers (routing.cu) -------------------------------------------------------------
 cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
                                  float* logits, int T, int H, int E, float* zero_buf,
                                  size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx,
-                                 uint32_t* nat_mask, int k, int32_t* tile_done, cudaStream_t s);
+                                 uint32_t* nat_mask, int k, int32_t* tile_done, bool pdl, cudaStream_t s);
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s);
 // select (unless mask_override) + route + work lists in ONE launch of ceil(T/4) small CTAs;
@@ -104,7 +115,7 @@ cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s
 // zero-initialised counter the kernel leaves at zero
 cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
                                 const uint32_t* mask_override, int T, int E, int k, int32_t* ticket,
-                                cudaStream_t s);
+                                bool pdl, cudaStream_t s);
 cudaError_t launch_routes_to_lists(const int32_t* idx, const float* w, WorkList* lists, float* wdense,
                                    int32_t* ready, int n_shared, int T, int E, int k, cudaStream_t s);
 
@@ -127,6 +138,7 @@ struct FfnLaunch {
   int32_t* status;
   int grid;
   int phase_mask;            // 1 = gate/up, 2 = down, 3 = both in one launch
+  bool pdl;                  // launch with programmatic stream serialization
   unsigned long long* trace; // optional [grid][32] device timestamps (debugging aid) or null
 };
 cudaError_t ffn_configure();   // one-time function attributes

@@ -59,6 +59,9 @@ struct acm_ctx {
   uint64_t h2d_bytes = 0;
   // per-launch FFN timing
   bool timing = false;
+  int timing_period = 1;        // every n-th FFN launch is bracketed by events
+  long long timing_seen = 0;
+  bool pdl = true;              // programmatic dependent launches between the kernels of the hot path
   std::vector<cudaEvent_t> ev_pool;
   size_t ev_used = 0;
   uint64_t launches = 0;
@@ -175,7 +178,8 @@ acm_status check_block_args(const acm_ctx* c, int layer, int T, bool need_weight
 }
 
 // One FFN launch over work list `li` (0 = resident + shared, 1 = staged).
-acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li, float* out, cudaStream_t s) {
+acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li, float* out, cudaStream_t s,
+                        bool pdl_ok = false) {
   const acm_model_desc& d = c->desc;
   const int n_pad = (T + 15) / 16 * 16;
   acm_status st = ensure_h_maps(c, n_pad);
@@ -200,9 +204,10 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   p.grid = c->sm_count;
   p.phase_mask = 3;
   p.trace = c->trace;
+  p.pdl = false;
   if (c->trace) ACM_CUDA(cudaMemsetAsync(c->trace, 0, sizeof(unsigned long long) * 32 * c->sm_count, s));
   cudaEvent_t e0 = nullptr, e1 = nullptr;
-  if (c->timing && c->ev_used + 2 <= c->ev_pool.size()) {
+  if (c->timing && (c->timing_seen++ % c->timing_period) == 0 && c->ev_used + 2 <= c->ev_pool.size()) {
     e0 = c->ev_pool[c->ev_used];
     e1 = c->ev_pool[c->ev_used + 1];
     c->ev_used += 2;
@@ -216,6 +221,8 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
     p.epoch = ++c->epoch;
     c->launches += 1;
   }
+  // dependent launch only straight after the select/route kernel (no event, memset or copy between)
+  p.pdl = pdl_ok && c->pdl && !e0 && !c->trace && !c->split_phases;
   ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
   c->launches += 1;
   if (e1) ACM_CUDA(cudaEventRecord(e1, s));
@@ -292,6 +299,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->layers.resize(desc->n_layers);
   const char* split = std::getenv("ACM_FFN_SPLIT_PHASES");
   c->split_phases = split && split[0] == '1';
+  const char* no_pdl = std::getenv("ACM_NO_PDL");
+  c->pdl = !(no_pdl && no_pdl[0] == '1');
   const char* trace = std::getenv("ACM_FFN_TRACE");
   const bool want_trace = trace && trace[0] == '1';
   auto fail = [&](acm_status s) {
@@ -446,7 +455,7 @@ acm_status acm_router(acm_ctx* c, int layer, const void* x, int T, float* logits
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // softmax and natural top-k are finished inside the same launch (last CTA of each node tile)
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, logits, T, d.hidden, d.n_experts, nullptr, 0,
-                                c->ws.status, probs, nat_idx, nullptr, d.top_k, c->ws.tile_done, s));
+                                c->ws.status, probs, nat_idx, nullptr, d.top_k, c->ws.tile_done, false, s));
   c->launches += 1;
   return ACM_OK;
 }
@@ -538,7 +547,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
                                 f32 ? 0 : static_cast<size_t>(T) * d.hidden, c->ws.status,
                                 need_probs ? c->ws.probs : nullptr, need_probs ? c->ws.nat_idx : nullptr,
-                                need_probs ? c->ws.nat_mask : nullptr, k, c->ws.tile_done, s));
+                                need_probs ? c->ws.nat_mask : nullptr, k, c->ws.tile_done, c->pdl, s));
   // stages 2-3 and the FFN work lists: one launch of a few small CTAs
   SelectArgs sa;
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
@@ -553,7 +562,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   ra.n_shared = d.n_shared; ra.host_stage_list = L.has_resident ? c->host_stage_list_dev : nullptr;
   ra.stats_out = c->ws.stats;
   ra.dbg = c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr;
-  ACM_CUDA(launch_select_route(c->ws.nat_mask, sa, ra, eligible_mask_override, T, E, k, c->ws.ticket, s));
+  ACM_CUDA(launch_select_route(c->ws.nat_mask, sa, ra, eligible_mask_override, T, E, k, c->ws.ticket, c->pdl, s));
   c->launches += 2;
 
   if (f32) {
@@ -563,7 +572,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
                             static_cast<float*>(c->ws.hbuf), out, T, d.hidden, d.inter, k, s));
     c->launches += 2;
   } else if (!L.has_resident) {
-    st = run_ffn_list(c, L, x, T, 0, out, s);
+    st = run_ffn_list(c, L, x, T, 0, out, s, true);
     if (st != ACM_OK) return st;
   } else {
     // resident + shared experts run at once; the others are copied in from pinned host memory first
@@ -636,7 +645,10 @@ acm_status acm_h2d_bytes(acm_ctx* c, uint64_t* bytes_out, int reset) {
 
 acm_status acm_ffn_timing(acm_ctx* c, int enable, int capacity) {
   if (!c || capacity < 0) return ACM_ERR_INVALID;
+  if (enable < 0) return ACM_ERR_INVALID;
   c->timing = enable != 0;
+  c->timing_period = enable > 0 ? enable : 1;
+  c->timing_seen = 0;
   c->ev_used = 0;
   while (c->timing && c->ev_pool.size() < static_cast<size_t>(2) * capacity) {
     cudaEvent_t e;

@@ -382,22 +382,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, G = gridDim.x;
-  // the entries are fetched without waiting for the count: one global round trip, not two
-  const int32_t my_entry = threadIdx.x < kMaxSlots ? p.list->entry[threadIdx.x] : 0;
-  const int n_act = p.list->n;
-  const int tpe = p.I / 64;          // gate/up tiles per expert = K-chunks per expert in the down phase
-  const int kc1 = p.H / (kBK * kAtoms);   // K-chunks (stages) of a gate/up tile
-  const int kpe = (tpe + kAtoms - 1) / kAtoms;   // K-chunks (stages) per expert in the down phase
-  const int h_tiles = p.H / kTileM;  // output tiles of the down phase
-  const uint32_t b_atom_bytes = static_cast<uint32_t>(p.n_pad) * kBK * 2;   // one atom of the activation chunk
-  const uint32_t b_bytes = kAtoms * b_atom_bytes;
-  const Plan plan = make_plan(n_act, tpe, G, p.phase_mask);
-  const Segment* seg = plan.seg;
-  const int n_seg = plan.n_seg;
-  const int a_split = plan.a_split;
-  int32_t* s_entry = bars->entry;
-  if (threadIdx.x < kMaxSlots) s_entry[threadIdx.x] = my_entry;
-
+  griddep_launch_dependents();
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&bars->full[s]), 1);
@@ -432,6 +417,25 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
     tmem_relinquish();
   }
+  // Everything above touched only this CTA's own resources; global memory written by the kernels
+  // before this one (the work list above all) is read only from here on.
+  griddep_wait();
+  // the entries are fetched without waiting for the count: one global round trip, not two
+  const int32_t my_entry = threadIdx.x < kMaxSlots ? p.list->entry[threadIdx.x] : 0;
+  const int n_act = p.list->n;
+  const int tpe = p.I / 64;          // gate/up tiles per expert = K-chunks per expert in the down phase
+  const int kc1 = p.H / (kBK * kAtoms);   // K-chunks (stages) of a gate/up tile
+  const int kpe = (tpe + kAtoms - 1) / kAtoms;   // K-chunks (stages) per expert in the down phase
+  const int h_tiles = p.H / kTileM;  // output tiles of the down phase
+  const uint32_t b_atom_bytes = static_cast<uint32_t>(p.n_pad) * kBK * 2;   // one atom of the activation chunk
+  const uint32_t b_bytes = kAtoms * b_atom_bytes;
+  const Plan plan = make_plan(n_act, tpe, G, p.phase_mask);
+  const Segment* seg = plan.seg;
+  const int n_seg = plan.n_seg;
+  const int a_split = plan.a_split;
+  int32_t* s_entry = bars->entry;
+  if (threadIdx.x < kMaxSlots) s_entry[threadIdx.x] = my_entry;
+
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -929,12 +933,20 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   cfg.blockDim = dim3(kThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = s;
+  // The CTAs wait on one another, so all of them must be resident: one CTA per SM on an otherwise
+  // idle GPU is, and a cooperative launch makes the driver check it.  A dependent launch cannot be
+  // cooperative (its CTAs trickle in behind the previous kernel's); there the waits' limits, which
+  // end in an error status instead of a hang, are the guard.
   cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeCooperative;   // CTAs wait on one another: all must be co-resident
-  attr[0].val.cooperative = 1;
+  if (L.pdl) {
+    set_pdl_attr(&attr[0]);
+  } else {
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+  }
   cfg.attrs = attr;
   static const bool plain = [] { const char* e = std::getenv("ACM_FFN_PLAIN_LAUNCH"); return e && e[0] == '1'; }();
-  cfg.numAttrs = plain ? 0 : 1;
+  cfg.numAttrs = (plain && !L.pdl) ? 0 : 1;
   return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(k_ffn_bf16), args);
 }
 

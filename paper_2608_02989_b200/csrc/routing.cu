@@ -187,6 +187,8 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
 
   const int tid = threadIdx.x;
   const int e0 = blockIdx.x * kRE, t0 = blockIdx.y * kRT;
+  griddep_launch_dependents();
+  griddep_wait();
 
   // zero the FFN output buffer (accumulated into by the FFN kernel), spread over the grid
   if (zero_buf) {
@@ -687,6 +689,8 @@ k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uin
   __shared__ int s_last;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int t_mine = blockIdx.x * kNodesPerCta + warp;
+  griddep_launch_dependents();
+  griddep_wait();
   ACM_RT(0);
   float z[4];
   load_logit_row(ra.logits, min(t_mine, T - 1), E, lane, z);      // in flight during the selection
@@ -767,8 +771,14 @@ __global__ void __launch_bounds__(512) k_routes_to_lists(const int32_t* idx, con
 cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
                                  float* logits, int T, int H, int E, float* zero_buf,
                                  size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx,
-                                 uint32_t* nat_mask, int k, int32_t* tile_done, cudaStream_t s) {
+                                 uint32_t* nat_mask, int k, int32_t* tile_done, bool pdl, cudaStream_t s) {
   if (!probs && !nat_idx) tile_done = nullptr;
+  cudaLaunchAttribute attr[1];
+  set_pdl_attr(attr);
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
   const dim3 grid((E + kRE - 1) / kRE, (T + kRT - 1) / kRT);
   const int elt = dtype == ACM_F32 ? 4 : 2;
   const size_t smem = static_cast<size_t>(kRT + kRE) * (static_cast<size_t>(H) * elt + 64);
@@ -777,19 +787,19 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     auto kern = k_router_logits<float>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (err != cudaSuccess) return err;
-    kern<<<grid, kRT * kRE * 8, smem, s>>>(static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
-                                           logits, T, H, E, n_chunks, zero_buf, zero_floats, status, probs, nat_idx,
-                                           nat_mask, k, tile_done);
+    cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * 8); cfg.dynamicSmemBytes = smem;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
+                              logits, T, H, E, n_chunks, zero_buf, zero_floats, status, probs, nat_idx, nat_mask, k,
+                              tile_done);
   } else {
     auto kern = k_router_logits<__nv_bfloat16>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (err != cudaSuccess) return err;
-    kern<<<grid, kRT * kRE * 4, smem, s>>>(static_cast<const __nv_bfloat16*>(x),
-                                           static_cast<const __nv_bfloat16*>(w_router), bias, logits, T, H, E,
-                                           n_chunks, zero_buf, zero_floats, status, probs, nat_idx, nat_mask, k,
-                                           tile_done);
+    cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * 4); cfg.dynamicSmemBytes = smem;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x),
+                              static_cast<const __nv_bfloat16*>(w_router), bias, logits, T, H, E, n_chunks, zero_buf,
+                              zero_floats, status, probs, nat_idx, nat_mask, k, tile_done);
   }
-  return cudaGetLastError();
 }
 
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s) {
@@ -804,10 +814,16 @@ cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s
 
 cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
                                 const uint32_t* mask_override, int T, int E, int k, int32_t* ticket,
-                                cudaStream_t s) {
-  k_select_route<<<(T + kNodesPerCta - 1) / kNodesPerCta, kSelThreads, 0, s>>>(nat_mask, sa, ra, mask_override, T, E,
-                                                                              k, ticket);
-  return cudaGetLastError();
+                                bool pdl, cudaStream_t s) {
+  cudaLaunchAttribute attr[1];
+  set_pdl_attr(attr);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((T + kNodesPerCta - 1) / kNodesPerCta);
+  cfg.blockDim = dim3(kSelThreads);
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, k_select_route, nat_mask, sa, ra, mask_override, T, E, k, ticket);
 }
 
 cudaError_t launch_routes_to_lists(const int32_t* idx, const float* w, WorkList* lists, float* wdense,
