@@ -107,7 +107,8 @@ inline void set_pdl_attr(cudaLaunchAttribute* attr) {
 cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
                                  float* logits, int T, int H, int E, float* zero_buf,
                                  size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx,
-                                 uint32_t* nat_mask, int k, int32_t* tile_done, bool pdl, cudaStream_t s);
+                                 uint32_t* nat_mask, int k, int32_t* tile_done, bool pdl, cudaStream_t s,
+                                 long long* dbg = nullptr);
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s);
 // select (unless mask_override) + route + work lists in ONE launch of ceil(T/4) small CTAs;

@@ -66,7 +66,8 @@ struct acm_ctx {
   size_t ev_used = 0;
   uint64_t launches = 0;
   bool split_phases = false;             // ACM_FFN_SPLIT_PHASES=1 in the environment
-  unsigned long long* trace = nullptr;   // ACM_FFN_TRACE=1: per-CTA timestamps of the last FFN launch
+  unsigned long long* trace = nullptr;   // ACM_FFN_TRACE=1|2: per-CTA timestamps of the last FFN launch
+  bool trace_light = false;              // =2: leave the launch sequence as it is (stale slots are not cleared)
 };
 
 namespace {
@@ -205,7 +206,8 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   p.phase_mask = 3;
   p.trace = c->trace;
   p.pdl = false;
-  if (c->trace) ACM_CUDA(cudaMemsetAsync(c->trace, 0, sizeof(unsigned long long) * 32 * c->sm_count, s));
+  if (c->trace && !c->trace_light)
+    ACM_CUDA(cudaMemsetAsync(c->trace, 0, sizeof(unsigned long long) * 32 * c->sm_count, s));
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   if (c->timing && (c->timing_seen++ % c->timing_period) == 0 && c->ev_used + 2 <= c->ev_pool.size()) {
     e0 = c->ev_pool[c->ev_used];
@@ -222,7 +224,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
     c->launches += 1;
   }
   // dependent launch only straight after the select/route kernel (no event, memset or copy between)
-  p.pdl = pdl_ok && c->pdl && !e0 && !c->trace && !c->split_phases;
+  p.pdl = pdl_ok && c->pdl && !e0 && (!c->trace || c->trace_light) && !c->split_phases;
   ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
   c->launches += 1;
   if (e1) ACM_CUDA(cudaEventRecord(e1, s));
@@ -302,7 +304,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const char* no_pdl = std::getenv("ACM_NO_PDL");
   c->pdl = !(no_pdl && no_pdl[0] == '1');
   const char* trace = std::getenv("ACM_FFN_TRACE");
-  const bool want_trace = trace && trace[0] == '1';
+  const bool want_trace = trace && (trace[0] == '1' || trace[0] == '2');
+  c->trace_light = trace && trace[0] == '2';
   auto fail = [&](acm_status s) {
     acm_destroy(c);
     return s;
@@ -455,7 +458,8 @@ acm_status acm_router(acm_ctx* c, int layer, const void* x, int T, float* logits
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // softmax and natural top-k are finished inside the same launch (last CTA of each node tile)
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, logits, T, d.hidden, d.n_experts, nullptr, 0,
-                                c->ws.status, probs, nat_idx, nullptr, d.top_k, c->ws.tile_done, false, s));
+                                c->ws.status, probs, nat_idx, nullptr, d.top_k, c->ws.tile_done, false, s,
+                                c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr));
   c->launches += 1;
   return ACM_OK;
 }
@@ -547,7 +551,8 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
                                 f32 ? 0 : static_cast<size_t>(T) * d.hidden, c->ws.status,
                                 need_probs ? c->ws.probs : nullptr, need_probs ? c->ws.nat_idx : nullptr,
-                                need_probs ? c->ws.nat_mask : nullptr, k, c->ws.tile_done, c->pdl, s));
+                                need_probs ? c->ws.nat_mask : nullptr, k, c->ws.tile_done, c->pdl, s,
+                                c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr));
   // stages 2-3 and the FFN work lists: one launch of a few small CTAs
   SelectArgs sa;
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
@@ -688,6 +693,8 @@ acm_status acm_device_status(acm_ctx* c, acm_stream stream) {
     ACM_CUDA(cudaMemset(c->ws.status, 0, sizeof v));
     ACM_CUDA(cudaMemset(c->ws.frag, 0, c->frag_bytes));
     ACM_CUDA(cudaMemset(c->ws.frag_flag, 0, c->flag_bytes));
+    ACM_CUDA(cudaMemset(c->ws.ticket, 0, 16));
+    ACM_CUDA(cudaMemset(c->ws.tile_done, 0, sizeof(int32_t) * kMaxNodes));
   }
   return static_cast<acm_status>(v);
 }

@@ -138,7 +138,7 @@ __device__ void softmax_topk_row(const float* z_row, float* probs_row, int32_t* 
 // ------------------------------------------------------------------------------------------
 // Stage 1a: router logits.  CTA tile = 4 nodes x 8 experts (many small CTAs: the whole GPU works on
 // a 64 x 128 x 2048 product), rows staged in shared memory with 16-byte async copies in 4 K-chunks.
-// A 16-byte load covers EPT consecutive h, i.e. EPT of the 32 interleaved partial sums; Q = 32/EPT
+// One vector load covers EPT consecutive h, i.e. EPT of the 32 interleaved partial sums; Q = 32/EPT
 // threads share one output.
 // ------------------------------------------------------------------------------------------
 constexpr int kRT = 4, kRE = 8;
@@ -148,6 +148,7 @@ struct ElemTraits;
 template <>
 struct ElemTraits<float> {
   static constexpr int EPT = 4;
+  using Vec = uint4;
   __device__ static void unpack(const uint4& v, float* f) {
     f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
     f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
@@ -155,29 +156,58 @@ struct ElemTraits<float> {
 };
 template <>
 struct ElemTraits<__nv_bfloat16> {
-  static constexpr int EPT = 8;
+#ifndef ACM_ROUTER_BF16_EPT
+#define ACM_ROUTER_BF16_EPT 4
+#endif
+  static constexpr int EPT = ACM_ROUTER_BF16_EPT;
+#if ACM_ROUTER_BF16_EPT == 8
+  using Vec = uint4;
   __device__ static void unpack(const uint4& v, float* f) {
     f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
     f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
     f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
     f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
   }
+#else
+  using Vec = uint2;        // 8-byte loads, 8 threads per output: twice the warps to hide latency with
+  __device__ static void unpack(const uint2& v, float* f) {
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+  }
+#endif
 };
 
-__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {
-  const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(d), "l"(gmem_src) : "memory");
+// ---- bulk asynchronous copies (global -> shared) completing on an mbarrier ----
+__device__ __forceinline__ unsigned smem_addr(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, unsigned bytes, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_addr(smem_dst)), "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+// Waits for phase `parity` of the barrier; gives up after a bounded number of polls (false).
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsigned parity) {
+  const unsigned a = smem_addr(bar);
+  for (int it = 0; it < (1 << 22); ++it) {
+    unsigned done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+        : "=r"(done) : "r"(a), "r"(parity) : "memory");
+    if (done) return true;
+  }
+  return false;
+}
 
 template <typename Elem>
 __global__ void __launch_bounds__(kRT * kRE * (32 / ElemTraits<Elem>::EPT))
 k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const float* __restrict__ bias,
                 float* logits, int T, int H, int E, int n_chunks, float* zero_buf,
                 size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k,
-                int32_t* tile_done) {
+                int32_t* tile_done, long long* dbg) {
   constexpr int EPT = ElemTraits<Elem>::EPT;
   constexpr int Q = 32 / EPT;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -189,6 +219,7 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
   const int e0 = blockIdx.x * kRE, t0 = blockIdx.y * kRT;
   griddep_launch_dependents();
   griddep_wait();
+  if (dbg && tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) dbg[13] = time_ns();
 
   // zero the FFN output buffer (accumulated into by the FFN kernel), spread over the grid
   if (zero_buf) {
@@ -199,23 +230,31 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
     for (size_t i = b * blockDim.x + tid; i < n4; i += nb * blockDim.x) z4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
 
-  // async staging of 8 x-rows and 8 router rows, n_chunks commit groups along h
-  const int segs_per_row = H * static_cast<int>(sizeof(Elem)) / 16;
-  const int segs_per_chunk = segs_per_row / n_chunks;
-  for (int c = 0; c < n_chunks; ++c) {
-    for (int i = tid; i < (kRT + kRE) * segs_per_chunk; i += blockDim.x) {
-      const int row = i / segs_per_chunk, seg = c * segs_per_chunk + i % segs_per_chunk;
-      if (row < kRT) {
-        const int t = min(t0 + row, T - 1);
-        cp_async_16(xs + static_cast<size_t>(row) * row_bytes + seg * 16,
-                    reinterpret_cast<const unsigned char*>(x + static_cast<size_t>(t) * H) + seg * 16);
-      } else {
-        const int e = min(e0 + row - kRT, E - 1);
-        cp_async_16(ws + static_cast<size_t>(row - kRT) * row_bytes + seg * 16,
-                    reinterpret_cast<const unsigned char*>(wr + static_cast<size_t>(e) * H) + seg * 16);
-      }
+  // Staging: the 4 x-rows and 8 router rows of this tile, in n_chunks pieces along h.  One thread
+  // per row issues its pieces as bulk copies; piece c of all rows completes on barrier c.
+  __shared__ __align__(8) unsigned long long chunk_bar[4];
+  const unsigned chunk_bytes = static_cast<unsigned>(H * sizeof(Elem)) / n_chunks;
+  if (tid == 0) {
+    for (int c = 0; c < n_chunks; ++c) mbar_init(&chunk_bar[c], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (tid == 0)
+    for (int c = 0; c < n_chunks; ++c) mbar_arrive_expect_tx(&chunk_bar[c], (kRT + kRE) * chunk_bytes);
+  if (tid < kRT + kRE) {
+    const int row = tid;
+    const unsigned char* src;
+    unsigned char* dst;
+    if (row < kRT) {
+      src = reinterpret_cast<const unsigned char*>(x + static_cast<size_t>(min(t0 + row, T - 1)) * H);
+      dst = xs + static_cast<size_t>(row) * row_bytes;
+    } else {
+      src = reinterpret_cast<const unsigned char*>(wr + static_cast<size_t>(min(e0 + row - kRT, E - 1)) * H);
+      dst = ws + static_cast<size_t>(row - kRT) * row_bytes;
     }
-    cp_async_commit();
+    for (int c = 0; c < n_chunks; ++c)
+      bulk_load(dst + static_cast<size_t>(c) * chunk_bytes, src + static_cast<size_t>(c) * chunk_bytes, chunk_bytes,
+                &chunk_bar[c]);
   }
 
   const int q = tid % Q;            // which EPT-wide group of the 32 partial sums
@@ -225,23 +264,19 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
 #pragma unroll
   for (int p = 0; p < EPT; ++p) acc[p] = 0.0f;
 
-  const unsigned char* xr0 = xs + static_cast<size_t>(tl) * row_bytes + q * 16;
-  const unsigned char* wrow = ws + static_cast<size_t>(el) * row_bytes + q * 16;
+  using Vec = typename ElemTraits<Elem>::Vec;
+  const unsigned char* xr0 = xs + static_cast<size_t>(tl) * row_bytes + q * sizeof(Vec);
+  const unsigned char* wrow = ws + static_cast<size_t>(el) * row_bytes + q * sizeof(Vec);
   const int steps_per_chunk = H / 32 / n_chunks;
   const int step_bytes = 32 * static_cast<int>(sizeof(Elem));
   for (int c = 0; c < n_chunks; ++c) {
-    // chunk c is complete once at most (n_chunks-1-c) groups are still pending
-    if (c == 0) { if (n_chunks == 4) cp_async_wait<3>(); else cp_async_wait<0>(); }
-    else if (c == 1) cp_async_wait<2>();
-    else if (c == 2) cp_async_wait<1>();
-    else cp_async_wait<0>();
-    __syncthreads();
+    if (!mbar_wait_bounded(&chunk_bar[c], 0u)) raise_status(status, ACM_ERR_TIMEOUT);
     const int j0 = c * steps_per_chunk;
 #pragma unroll 4
     for (int j = j0; j < j0 + steps_per_chunk; ++j) {
       float xa[EPT], wv[EPT];
-      ElemTraits<Elem>::unpack(*reinterpret_cast<const uint4*>(xr0 + static_cast<size_t>(j) * step_bytes), xa);
-      ElemTraits<Elem>::unpack(*reinterpret_cast<const uint4*>(wrow + static_cast<size_t>(j) * step_bytes), wv);
+      ElemTraits<Elem>::unpack(*reinterpret_cast<const Vec*>(xr0 + static_cast<size_t>(j) * step_bytes), xa);
+      ElemTraits<Elem>::unpack(*reinterpret_cast<const Vec*>(wrow + static_cast<size_t>(j) * step_bytes), wv);
 #pragma unroll
       for (int p = 0; p < EPT; ++p) acc[p] = __fmaf_rn(xa[p], wv[p], acc[p]);
     }
@@ -264,6 +299,7 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
     logits[static_cast<size_t>(t) * E + e] = z;
     if (!isfinite(z)) raise_status(status, ACM_ERR_NONFINITE);
   }
+  if (dbg && tid == 0) atomicMax(reinterpret_cast<unsigned long long*>(dbg + 14), static_cast<unsigned long long>(time_ns()));
   // The CTA that completes a tile of nodes last (all expert tiles written) finishes those nodes:
   // softmax and natural top-k, one warp per node -- spread over as many SMs as there are node tiles.
   if (tile_done) {
@@ -286,6 +322,7 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
                            nat_idx ? nat_idx + static_cast<size_t>(t) * k : nullptr,
                            nat_mask ? nat_mask + static_cast<size_t>(t) * kMaskWords : nullptr, E, k, lane);
       }
+      if (dbg && tid == 0) atomicMax(reinterpret_cast<unsigned long long*>(dbg + 15), static_cast<unsigned long long>(time_ns()));
     }
   }
 }
@@ -771,7 +808,8 @@ __global__ void __launch_bounds__(512) k_routes_to_lists(const int32_t* idx, con
 cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
                                  float* logits, int T, int H, int E, float* zero_buf,
                                  size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx,
-                                 uint32_t* nat_mask, int k, int32_t* tile_done, bool pdl, cudaStream_t s) {
+                                 uint32_t* nat_mask, int k, int32_t* tile_done, bool pdl, cudaStream_t s,
+                                 long long* dbg) {
   if (!probs && !nat_idx) tile_done = nullptr;
   cudaLaunchAttribute attr[1];
   set_pdl_attr(attr);
@@ -782,7 +820,10 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
   const dim3 grid((E + kRE - 1) / kRE, (T + kRT - 1) / kRT);
   const int elt = dtype == ACM_F32 ? 4 : 2;
   const size_t smem = static_cast<size_t>(kRT + kRE) * (static_cast<size_t>(H) * elt + 64);
-  const int n_chunks = (H % 128 == 0) ? 4 : 1;
+  // pieces of at least 4 KB per row: every bulk copy has a fixed cost, and few large ones land sooner
+  const size_t row = static_cast<size_t>(H) * elt;
+  const int n_chunks = (row >= 16384 && H % 128 == 0) ? 4 : (row >= 8192 && H % 64 == 0) ? 2 : 1;
+  if ((static_cast<size_t>(H) * elt) % 16 != 0) return cudaErrorInvalidValue;   // rows are copied in 16-byte units
   if (dtype == ACM_F32) {
     auto kern = k_router_logits<float>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
@@ -790,15 +831,15 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * 8); cfg.dynamicSmemBytes = smem;
     return cudaLaunchKernelEx(&cfg, kern, static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
                               logits, T, H, E, n_chunks, zero_buf, zero_floats, status, probs, nat_idx, nat_mask, k,
-                              tile_done);
+                              tile_done, dbg);
   } else {
     auto kern = k_router_logits<__nv_bfloat16>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
     if (err != cudaSuccess) return err;
-    cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * 4); cfg.dynamicSmemBytes = smem;
+    cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * (32 / ElemTraits<__nv_bfloat16>::EPT)); cfg.dynamicSmemBytes = smem;
     return cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x),
                               static_cast<const __nv_bfloat16*>(w_router), bias, logits, T, H, E, n_chunks, zero_buf,
-                              zero_floats, status, probs, nat_idx, nat_mask, k, tile_done);
+                              zero_floats, status, probs, nat_idx, nat_mask, k, tile_done, dbg);
   }
 }
 
