@@ -24,16 +24,10 @@ __host__ __device__ inline int32_t make_entry(int src, int idx) { return (src <<
 __host__ __device__ inline int entry_src(int32_t e) { return (e >> 28) & 3; }
 __host__ __device__ inline int entry_idx(int32_t e) { return e & 0x0fffffff; }
 
-// A list of activated experts for the FFN kernel.  Slot a owns row a of `wdense`
-// (combine weight of every node, 0 where the node is not routed there).
-struct WorkList {
-  int32_t n;                      // number of activated experts in this list
-  int32_t n_stage;                // (list 1 only) experts that must be copied from the host first
-  int32_t pad[2];
-  int32_t entry[kMaxSlots];       // make_entry(src, idx)
-  int32_t expert[kMaxSlots];      // routed expert id (or -1 for shared)
-};
-
+// The FFN kernel takes its activated experts from a bit mask over the routed experts (slot a = the
+// a-th set bit, i.e. ascending expert id; shared experts are appended) and the combine weights from a
+// dense table indexed [expert][node] (0 where the node is not routed there).  Both are filled
+// straight by the routing warps, so nothing has to gather the routes into lists first.
 // Device workspace of one context (one allocation, carved on the host).
 struct Workspace {
   float* logits;        // [T,E]
@@ -47,8 +41,8 @@ struct Workspace {
   int32_t* count;       // [1]
   float* demand;        // [E]
   acm_block_stats* stats;
-  WorkList* lists;      // [2]: 0 = resident + shared, 1 = staged
-  float* wdense;        // [2][kMaxSlots][64]
+  uint32_t* act_mask;   // [4] activated routed experts of the current block
+  float* wtab;          // [kMaxExperts][64] combine weight of (expert, node)
   void* hbuf;           // [2][kMaxSlots][64][I] bf16 (f32 path: [T][k+ns][I] float)
   float* frag;          // [2][grid][128*64] split-K partial sums, accumulated into the finishing CTA's buffer; zero between launches
   int32_t* frag_flag;   // [2][grid] how many CTAs have added to that buffer; zero between launches
@@ -81,14 +75,14 @@ struct RouteArgs {
   float* w_out;
   int weighting;
   float routed_scale;
-  // work-list construction (all null/0 when only the routes are wanted)
-  WorkList* lists;
-  float* wdense;
-  int32_t* ready;
-  const uint32_t* resident;      // non-null: experts outside it go to list 1 (staged)
-  int n_shared;
+  // inputs of the FFN kernel (all null when only the routes are wanted); zero on entry
+  uint32_t* act_mask;            // [4] activated experts, OR-ed into
+  float* wtab;                   // [kMaxExperts][64] combine weights by (expert, node)
+  // The CTA that finishes last can also report on the whole block (it needs a ticket, so only when asked):
+  int32_t* ticket;               // zero-initialised counter, left at zero; null: no report
+  const uint32_t* resident;      // non-null: activated experts outside it are "staged"
   acm_block_stats* stats_out;    // n_activated / n_staged are filled in
-  int32_t* host_stage_list;      // mapped pinned memory: [0] = n_stage, [1..] = expert ids (may be null)
+  int32_t* host_stage_list;      // mapped pinned memory: [0] = n_stage, [1..] = staged expert ids (may be null)
   long long* dbg;                // optional time stamps in ns of the select/route kernel's stages (debugging aid)
 };
 
@@ -106,19 +100,18 @@ inline void set_pdl_attr(cudaLaunchAttribute* attr) {
 // ---- launchers (routing.cu) -------------------------------------------------------------
 cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
                                  float* logits, int T, int H, int E, float* zero_buf,
-                                 size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx,
-                                 uint32_t* nat_mask, int k, int32_t* tile_done, bool pdl, cudaStream_t s,
-                                 long long* dbg = nullptr);
+                                 size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status,
+                                 float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k, int32_t* tile_done,
+                                 bool pdl, cudaStream_t s, long long* dbg = nullptr);
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s);
-// select (unless mask_override) + route + work lists in ONE launch of ceil(T/4) small CTAs;
-// `nat_mask` = the natural top-k sets as bit masks [T][4] (from launch_router_logits), `ticket` = one
-// zero-initialised counter the kernel leaves at zero
+// select (unless mask_override) + route + the FFN kernel's routing inputs in ONE launch of ceil(T/4)
+// small CTAs; `nat_mask` = the natural top-k sets as bit masks [T][4] (from launch_router_logits)
 cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
-                                const uint32_t* mask_override, int T, int E, int k, int32_t* ticket,
-                                bool pdl, cudaStream_t s);
-cudaError_t launch_routes_to_lists(const int32_t* idx, const float* w, WorkList* lists, float* wdense,
-                                   int32_t* ready, int n_shared, int T, int E, int k, cudaStream_t s);
+                                const uint32_t* mask_override, int T, int E, int k, bool pdl, cudaStream_t s);
+// routes given by the caller -> activated mask, weight table (both cleared first) and cleared `ready`
+cudaError_t launch_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask, float* wtab,
+                                   int32_t* ready, int T, int E, int k, cudaStream_t s);
 
 // ---- launchers (ffn.cu) -----------------------------------------------------------------
 struct FfnMaps {               // TMA descriptors of one layer (bf16 path)
@@ -128,8 +121,12 @@ struct FfnMaps {               // TMA descriptors of one layer (bf16 path)
 };
 struct FfnLaunch {
   int T, H, I, n_pad;
-  const WorkList* list;
-  const float* wdense;       // [kMaxSlots][64] of this list
+  const uint32_t* act_mask;  // [4] activated routed experts
+  const uint32_t* resident;  // [4] or null (all resident)
+  int li;                    // 0: resident activated experts + shared experts; 1: the staged (non-resident) ones
+  int n_shared;
+  const float* wtab;         // [kMaxExperts][64] combine weights by (expert, node)
+  acm_block_stats* stats;    // list 0 fills n_activated / n_staged (may be null)
   void* hbuf;                // [kMaxSlots][64][I] bf16 of this list
   int32_t* ready;            // [kMaxSlots] of this list (zero on entry)
   float* frag;

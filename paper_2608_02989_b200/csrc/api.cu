@@ -58,6 +58,7 @@ struct acm_ctx {
   bool stage_in_use = false;
   uint64_t h2d_bytes = 0;
   // per-launch FFN timing
+  size_t ffn_in_floats = 0;     // length of the block wtab | ready | act_mask, in floats
   bool timing = false;
   int timing_period = 1;        // every n-th FFN launch is bracketed by events
   long long timing_seen = 0;
@@ -180,7 +181,7 @@ acm_status check_block_args(const acm_ctx* c, int layer, int T, bool need_weight
 
 // One FFN launch over work list `li` (0 = resident + shared, 1 = staged).
 acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li, float* out, cudaStream_t s,
-                        bool pdl_ok = false) {
+                        const uint32_t* res_dev = nullptr, acm_block_stats* stats_dev = nullptr, bool pdl_ok = false) {
   const acm_model_desc& d = c->desc;
   const int n_pad = (T + 15) / 16 * 16;
   acm_status st = ensure_h_maps(c, n_pad);
@@ -195,8 +196,12 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   }
   FfnLaunch p;
   p.T = T; p.H = d.hidden; p.I = d.inter; p.n_pad = n_pad;
-  p.list = c->ws.lists + li;
-  p.wdense = c->ws.wdense + static_cast<size_t>(li) * kMaxSlots * kMaxNodes;
+  p.act_mask = c->ws.act_mask;
+  p.resident = res_dev;
+  p.li = li;
+  p.n_shared = d.n_shared;
+  p.wtab = c->ws.wtab;
+  p.stats = stats_dev;
   p.hbuf = static_cast<char*>(c->ws.hbuf) + static_cast<size_t>(li) * kMaxSlots * kMaxNodes * d.inter * 2;
   p.ready = c->ws.ready + li * kMaxSlots;
   p.frag = c->ws.frag; p.frag_flag = c->ws.frag_flag;
@@ -337,14 +342,15 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_nat = carve(sizeof(int32_t) * Tm * k), o_idx = carve(sizeof(int32_t) * Tm * k);
   const size_t o_w = carve(sizeof(float) * Tm * k), o_mask = carve(16), o_unpr = carve(16), o_cnt = carve(16);
   const size_t o_dem = carve(sizeof(float) * kMaxExperts), o_stats = carve(sizeof(acm_block_stats));
-  const size_t o_lists = carve(sizeof(WorkList) * 2);
-  const size_t o_wd = carve(sizeof(float) * 2 * kMaxSlots * kMaxNodes);
+  // the FFN kernel's routing inputs, contiguous so that one pass clears them: weight table, finished-tile
+  // counters, activated mask
+  const size_t ffn_in_bytes = sizeof(float) * kMaxExperts * kMaxNodes + sizeof(int32_t) * 2 * kMaxSlots + 16;
+  const size_t o_ffn_in = carve(align_up(ffn_in_bytes, 16));
   const size_t hbuf_bf16 = static_cast<size_t>(2) * kMaxSlots * kMaxNodes * I * 2;
   const size_t hbuf_f32 = static_cast<size_t>(Tm) * (k + desc->n_shared) * I * 4;
   const size_t o_h = carve(hbuf_bf16 > hbuf_f32 ? hbuf_bf16 : hbuf_f32);
   const size_t o_frag = carve(sizeof(float) * 2 * static_cast<size_t>(c->sm_count) * 128 * kMaxNodes);
   const size_t o_flag = carve(sizeof(int32_t) * 2 * c->sm_count);
-  const size_t o_ready = carve(sizeof(int32_t) * 2 * kMaxSlots);
   const size_t o_status = carve(16);
   const size_t o_tile = carve(sizeof(int32_t) * kMaxNodes);
   const size_t o_ticket = carve(16);
@@ -363,14 +369,16 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.count = reinterpret_cast<int32_t*>(b + o_cnt);
   c->ws.demand = reinterpret_cast<float*>(b + o_dem);
   c->ws.stats = reinterpret_cast<acm_block_stats*>(b + o_stats);
-  c->ws.lists = reinterpret_cast<WorkList*>(b + o_lists);
-  c->ws.wdense = reinterpret_cast<float*>(b + o_wd);
+  c->ws.wtab = reinterpret_cast<float*>(b + o_ffn_in);
+  c->ws.ready = reinterpret_cast<int32_t*>(b + o_ffn_in + sizeof(float) * kMaxExperts * kMaxNodes);
+  c->ws.act_mask = reinterpret_cast<uint32_t*>(b + o_ffn_in + sizeof(float) * kMaxExperts * kMaxNodes +
+                                               sizeof(int32_t) * 2 * kMaxSlots);
+  c->ffn_in_floats = align_up(ffn_in_bytes, 16) / sizeof(float);
   c->ws.hbuf = b + o_h;
   c->ws.frag = reinterpret_cast<float*>(b + o_frag);
   c->frag_bytes = sizeof(float) * 2 * static_cast<size_t>(c->sm_count) * 128 * kMaxNodes;
   c->flag_bytes = sizeof(int32_t) * 2 * c->sm_count;
   c->ws.frag_flag = reinterpret_cast<int32_t*>(b + o_flag);
-  c->ws.ready = reinterpret_cast<int32_t*>(b + o_ready);
   c->ws.status = reinterpret_cast<int32_t*>(b + o_status);
   c->ws.tile_done = reinterpret_cast<int32_t*>(b + o_tile);
   c->ws.ticket = reinterpret_cast<int32_t*>(b + o_ticket);
@@ -458,7 +466,7 @@ acm_status acm_router(acm_ctx* c, int layer, const void* x, int T, float* logits
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // softmax and natural top-k are finished inside the same launch (last CTA of each node tile)
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, logits, T, d.hidden, d.n_experts, nullptr, 0,
-                                c->ws.status, probs, nat_idx, nullptr, d.top_k, c->ws.tile_done, false, s,
+                                nullptr, 0, c->ws.status, probs, nat_idx, nullptr, d.top_k, c->ws.tile_done, false, s,
                                 c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr));
   c->launches += 1;
   return ACM_OK;
@@ -515,8 +523,7 @@ acm_status acm_expert_ffn(acm_ctx* c, int layer, const void* x, int T, const int
     return ACM_OK;
   }
   ACM_CUDA(cudaMemsetAsync(out, 0, sizeof(float) * static_cast<size_t>(T) * d.hidden, s));
-  ACM_CUDA(launch_routes_to_lists(idx, w, c->ws.lists, c->ws.wdense, c->ws.ready, d.n_shared, T, d.n_experts,
-                                  d.top_k, s));
+  ACM_CUDA(launch_routes_to_table(idx, w, c->ws.act_mask, c->ws.wtab, c->ws.ready, T, d.n_experts, d.top_k, s));
   c->launches += 1;
   return run_ffn_list(c, L, x, T, 0, out, s);
 }
@@ -546,14 +553,15 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   const bool f32 = d.dtype == ACM_F32;
   uint32_t* res_dev = L.has_resident ? c->resident_dev + 4 * layer : nullptr;
 
-  // stage 1a (also clears the output the FFN accumulates into)
+  // stage 1 (also clears the output the FFN accumulates into and the FFN kernel's routing inputs)
   const bool need_probs = eligible_mask_override == nullptr;
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
-                                f32 ? 0 : static_cast<size_t>(T) * d.hidden, c->ws.status,
+                                f32 ? 0 : static_cast<size_t>(T) * d.hidden, c->ws.wtab, c->ffn_in_floats,
+                                c->ws.status,
                                 need_probs ? c->ws.probs : nullptr, need_probs ? c->ws.nat_idx : nullptr,
                                 need_probs ? c->ws.nat_mask : nullptr, k, c->ws.tile_done, c->pdl, s,
                                 c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr));
-  // stages 2-3 and the FFN work lists: one launch of a few small CTAs
+  // stages 2-3: one launch of a few small CTAs, which also fill the FFN kernel's routing inputs
   SelectArgs sa;
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
   sa.n_anchor_nodes = 0; sa.resident = prm.residency ? res_dev : nullptr; sa.prm = prm;
@@ -563,11 +571,13 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   RouteArgs ra = {};
   ra.logits = c->ws.logits; ra.mask = c->ws.mask; ra.idx_out = c->ws.idx; ra.w_out = c->ws.w;
   ra.weighting = d.weighting; ra.routed_scale = d.routed_scale;
-  ra.lists = c->ws.lists; ra.wdense = c->ws.wdense; ra.ready = c->ws.ready; ra.resident = res_dev;
-  ra.n_shared = d.n_shared; ra.host_stage_list = L.has_resident ? c->host_stage_list_dev : nullptr;
+  ra.act_mask = c->ws.act_mask; ra.wtab = c->ws.wtab; ra.resident = res_dev;
+  ra.host_stage_list = L.has_resident ? c->host_stage_list_dev : nullptr;
   ra.stats_out = c->ws.stats;
+  // the bf16 FFN kernel counts the activated experts itself; otherwise the routing kernel's last CTA does
+  ra.ticket = (f32 || L.has_resident) ? c->ws.ticket : nullptr;
   ra.dbg = c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr;
-  ACM_CUDA(launch_select_route(c->ws.nat_mask, sa, ra, eligible_mask_override, T, E, k, c->ws.ticket, c->pdl, s));
+  ACM_CUDA(launch_select_route(c->ws.nat_mask, sa, ra, eligible_mask_override, T, E, k, c->pdl, s));
   c->launches += 2;
 
   if (f32) {
@@ -577,12 +587,12 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
                             static_cast<float*>(c->ws.hbuf), out, T, d.hidden, d.inter, k, s));
     c->launches += 2;
   } else if (!L.has_resident) {
-    st = run_ffn_list(c, L, x, T, 0, out, s, true);
+    st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, c->ws.stats, true);
     if (st != ACM_OK) return st;
   } else {
     // resident + shared experts run at once; the others are copied in from pinned host memory first
     ACM_CUDA(cudaEventRecord(c->ev_lists, s));
-    st = run_ffn_list(c, L, x, T, 0, out, s);
+    st = run_ffn_list(c, L, x, T, 0, out, s, res_dev, c->ws.stats);
     if (st != ACM_OK) return st;
     ACM_CUDA(cudaEventSynchronize(c->ev_lists));
     const int n_stage = c->host_stage_list[0];
@@ -603,7 +613,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
       }
       ACM_CUDA(cudaEventRecord(c->ev_copied, c->copy_stream));
       ACM_CUDA(cudaStreamWaitEvent(s, c->ev_copied, 0));
-      st = run_ffn_list(c, L, x, T, 1, out, s);
+      st = run_ffn_list(c, L, x, T, 1, out, s, res_dev, nullptr);
       if (st != ACM_OK) return st;
       ACM_CUDA(cudaEventRecord(c->ev_stage_free, s));
       c->stage_in_use = true;

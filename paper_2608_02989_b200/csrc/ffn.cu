@@ -68,7 +68,8 @@ struct __align__(8) Barriers {
   uint32_t tmem_base;
   int abort_flag;
   float wd[kMaxNodes];          // combine weights of the expert being finalised
-  int32_t entry[kMaxSlots];     // this launch's work list (copied from global memory once)
+  int32_t entry[kMaxSlots];     // this launch's work list: make_entry(source, index) of every activated slot
+  int32_t expert[kMaxSlots];    // routed expert id of the slot (-1: shared expert)
 };
 
 constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + kOutStageBytes + kFragBytes + 2 * kHStageBytes + sizeof(Barriers);
@@ -246,15 +247,16 @@ __device__ __forceinline__ uint32_t umma_idesc(int n) {
 
 // Equal contiguous ranges of (tile, K-chunk) units: CTA c owns [c*U/G, (c+1)*U/G).
 struct Sched {
-  long long u, u_end;
+  unsigned u, u_end;   // 32-bit on purpose: one thread per role walks this, and 64-bit division costs it microseconds
   int kc;
   int rr_next, rr_end, rr_stride;   // whole tiles dealt round-robin (rr_stride > 0) instead of a cut range
   // equal contiguous ranges of (tile, K-chunk) units: CTA c owns [c*U/G, (c+1)*U/G)
-  __device__ Sched(int cta, int grid, long long tiles, int chunks_per_tile)
+  // (the launcher checks that tiles * chunks_per_tile * grid fits in 32 bits)
+  __device__ Sched(int cta, int grid, int tiles, int chunks_per_tile)
       : kc(chunks_per_tile), rr_next(0), rr_end(0), rr_stride(0) {
-    const long long total = tiles * chunks_per_tile;
-    u = total * cta / grid;
-    u_end = total * (cta + 1) / grid;
+    const unsigned total = static_cast<unsigned>(tiles) * static_cast<unsigned>(chunks_per_tile);
+    u = total * static_cast<unsigned>(cta) / static_cast<unsigned>(grid);
+    u_end = total * static_cast<unsigned>(cta + 1) / static_cast<unsigned>(grid);
   }
   // whole tiles: CTA c owns tiles c, c+G, c+2G, ... < tiles (tiles is a multiple of G here)
   __device__ static Sched whole_tiles(int cta, int grid, int tiles, int chunks_per_tile) {
@@ -266,7 +268,7 @@ struct Sched {
   }
   __device__ long long stages() const {
     if (rr_stride > 0) return rr_next < rr_end ? static_cast<long long>((rr_end - rr_next + rr_stride - 1) / rr_stride) * kc : 0;
-    return u_end - u;
+    return static_cast<long long>(u_end - u);
   }
   __device__ bool next(int& tile, int& k0, int& k1) {
     if (rr_stride > 0) {
@@ -278,11 +280,11 @@ struct Sched {
       return true;
     }
     if (u >= u_end) return false;
-    tile = static_cast<int>(u / kc);
-    k0 = static_cast<int>(u % kc);
-    const long long rem = u_end - u;
-    k1 = static_cast<int>(rem < kc - k0 ? k0 + rem : kc);
-    u += k1 - k0;
+    tile = static_cast<int>(u / static_cast<unsigned>(kc));
+    k0 = static_cast<int>(u - static_cast<unsigned>(tile) * static_cast<unsigned>(kc));
+    const int rem = static_cast<int>(u_end - u);
+    k1 = rem < kc - k0 ? k0 + rem : kc;
+    u += static_cast<unsigned>(k1 - k0);
     return true;
   }
 };
@@ -292,8 +294,11 @@ struct Sched {
 
 struct FfnArgs {
   int T, H, I, n_pad;
-  const WorkList* list;
-  const float* wdense;
+  const uint32_t* act_mask;
+  const uint32_t* resident;
+  int li, n_shared;
+  const float* wtab;
+  acm_block_stats* stats;
   __nv_bfloat16* hbuf;
   int32_t* ready;
   float* frag;
@@ -420,9 +425,19 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   // Everything above touched only this CTA's own resources; global memory written by the kernels
   // before this one (the work list above all) is read only from here on.
   griddep_wait();
-  // the entries are fetched without waiting for the count: one global round trip, not two
-  const int32_t my_entry = threadIdx.x < kMaxSlots ? p.list->entry[threadIdx.x] : 0;
-  const int n_act = p.list->n;
+  // The work list of this launch: slot a = the a-th activated expert of this list in ascending id
+  // order (list 0: the resident ones, then the shared experts; list 1: the non-resident ones, which
+  // the host has copied into staging slot a).
+  uint32_t am[kMaskWords];
+  int n_routed = 0;
+#pragma unroll
+  for (int wd = 0; wd < kMaskWords; ++wd) {
+    const uint32_t act = p.act_mask[wd];
+    const uint32_t res = p.resident ? p.resident[wd] : 0xffffffffu;
+    am[wd] = p.li == 0 ? act & res : act & ~res;
+    n_routed += __popc(am[wd]);
+  }
+  const int n_act = n_routed + (p.li == 0 ? p.n_shared : 0);
   const int tpe = p.I / 64;          // gate/up tiles per expert = K-chunks per expert in the down phase
   const int kc1 = p.H / (kBK * kAtoms);   // K-chunks (stages) of a gate/up tile
   const int kpe = (tpe + kAtoms - 1) / kAtoms;   // K-chunks (stages) per expert in the down phase
@@ -434,7 +449,31 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   const int n_seg = plan.n_seg;
   const int a_split = plan.a_split;
   int32_t* s_entry = bars->entry;
-  if (threadIdx.x < kMaxSlots) s_entry[threadIdx.x] = my_entry;
+  if (threadIdx.x < kMaxExperts) {
+    const int e = threadIdx.x, wd = e >> 5;
+    if ((am[wd] >> (e & 31)) & 1u) {
+      int slot = __popc(am[wd] & ((1u << (e & 31)) - 1u));
+#pragma unroll
+      for (int v = 0; v < kMaskWords; ++v) slot += v < wd ? __popc(am[v]) : 0;
+      s_entry[slot] = p.li == 0 ? make_entry(kSrcRouted, e) : make_entry(kSrcStaged, slot);
+      bars->expert[slot] = e;
+    }
+  } else if (p.li == 0 && threadIdx.x - kMaxExperts < p.n_shared) {
+    const int i = threadIdx.x - kMaxExperts;
+    s_entry[n_routed + i] = make_entry(kSrcShared, i);
+    bars->expert[n_routed + i] = -1;
+  }
+  if (p.stats && p.li == 0 && blockIdx.x == 0 && threadIdx.x == 0) {
+    int n_all = 0, n_stg = 0;
+#pragma unroll
+    for (int wd = 0; wd < kMaskWords; ++wd) {
+      const uint32_t act = p.act_mask[wd];
+      n_all += __popc(act);
+      n_stg += p.resident ? __popc(act & ~p.resident[wd]) : 0;
+    }
+    p.stats->n_activated = n_all;
+    p.stats->n_staged = n_stg;
+  }
 
   tc_fence_before();
   __syncthreads();
@@ -758,7 +797,10 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             continue;
           }
           const int a = (sg.t0 + tile) / tpe;
-          if (row < p.n_pad) bars->wd[row] = p.wdense[static_cast<size_t>(a) * kMaxNodes + row];
+          if (row < p.n_pad) {
+            const int ex_id = bars->expert[a];      // combine weights: the table row of a routed expert, 1 for a shared one
+            bars->wd[row] = ex_id >= 0 ? p.wtab[static_cast<size_t>(ex_id) * kMaxNodes + row] : (row < p.T ? 1.0f : 0.0f);
+          }
           if (k1 < kc1) {
             // head part: the helper warp has summed the other CTAs' fragments of this tile into smem
             ok = epi_vote_all(mbar_wait(smem_u32(&bars->frag_full[sg.p1_index]), 0, abort_flag, p.status));
@@ -921,9 +963,16 @@ cudaError_t ffn_configure() {
 
 cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
                             const CUtensorMap& h_map, const CUtensorMap& hs_map, cudaStream_t s) {
+  {
+    // the schedules count (tile, K-chunk) units times the grid in 32 bits
+    const unsigned long long u1 = static_cast<unsigned long long>(kMaxSlots) * (L.I / 64) * (L.H / (kBK * kAtoms));
+    const unsigned long long u2 = static_cast<unsigned long long>(L.H / kTileM) * kMaxSlots * ((L.I / 64 + kAtoms - 1) / kAtoms);
+    if ((u1 > u2 ? u1 : u2) * (static_cast<unsigned long long>(L.grid) + 1) >= (1ull << 32)) return cudaErrorInvalidValue;
+  }
   FfnArgs a;
   a.T = L.T; a.H = L.H; a.I = L.I; a.n_pad = L.n_pad;
-  a.list = L.list; a.wdense = L.wdense; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
+  a.act_mask = L.act_mask; a.resident = L.resident; a.li = L.li; a.n_shared = L.n_shared; a.wtab = L.wtab;
+  a.stats = L.stats; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
   a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag; a.epoch = L.epoch;
   a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask; a.trace = L.trace;
   void* args[] = {const_cast<FfnMaps*>(&maps), const_cast<CUtensorMap*>(&x_map), const_cast<CUtensorMap*>(&h_map),

@@ -206,7 +206,7 @@ template <typename Elem>
 __global__ void __launch_bounds__(kRT * kRE * (32 / ElemTraits<Elem>::EPT))
 k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const float* __restrict__ bias,
                 float* logits, int T, int H, int E, int n_chunks, float* zero_buf,
-                size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k,
+                size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status, float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k,
                 int32_t* tile_done, long long* dbg) {
   constexpr int EPT = ElemTraits<Elem>::EPT;
   constexpr int Q = 32 / EPT;
@@ -221,13 +221,19 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
   griddep_wait();
   if (dbg && tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) dbg[13] = time_ns();
 
-  // zero the FFN output buffer (accumulated into by the FFN kernel), spread over the grid
-  if (zero_buf) {
+  // zero the FFN output buffer (accumulated into by the FFN kernel) and the FFN kernel's routing
+  // inputs (activated mask, weight table, finished-tile counters), spread over the grid
+  {
     const size_t nb = static_cast<size_t>(gridDim.x) * gridDim.y;
     const size_t b = static_cast<size_t>(blockIdx.y) * gridDim.x + blockIdx.x;
-    const size_t n4 = zero_floats / 4;
-    float4* z4 = reinterpret_cast<float4*>(zero_buf);
-    for (size_t i = b * blockDim.x + tid; i < n4; i += nb * blockDim.x) z4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (zero_buf) {
+      float4* z4 = reinterpret_cast<float4*>(zero_buf);
+      for (size_t i = b * blockDim.x + tid; i < zero_floats / 4; i += nb * blockDim.x) z4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (zero_buf2) {
+      float4* z4 = reinterpret_cast<float4*>(zero_buf2);
+      for (size_t i = b * blockDim.x + tid; i < zero_floats2 / 4; i += nb * blockDim.x) z4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
   }
 
   // Staging: the 4 x-rows and 8 router rows of this tile, in n_chunks pieces along h.  One thread
@@ -345,12 +351,6 @@ struct StageSmem {
   float tree[kMaxExperts + 4];
   alignas(16) unsigned long long rkey[kMaxExperts];   // ranking keys of the experts (0 = not ranked)
   uint32_t A[kMaskWords], S[kMaskWords], Sp[kMaskWords], Hres[kMaskWords];
-  int32_t idx[kMaxNodes][kMaxTopK];
-  float w[kMaxNodes][kMaxTopK];
-  int32_t cnt[kMaxExperts];
-  int32_t slot_of[kMaxExperts];
-  int32_t list_of[kMaxExperts];
-  int32_t warp_tot[2][4];
   int32_t scal[8];
 };
 
@@ -569,80 +569,6 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   sel_sync();
 }
 
-// Turns per-node routes (sm.idx / sm.w) into the FFN work lists: activated experts in ascending
-// id order, shared experts appended; combine weights scattered into the dense [slot][node] table.
-// `zero`: also clear the dense tables and the finished-tile counters here (otherwise the caller has).
-__device__ void stage_build_lists(const RouteArgs& a, StageSmem& sm, int T, int E, int k, bool zero) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid < kMaxExperts) sm.cnt[tid] = 0;
-  if (zero) {
-    const int rows = E + a.n_shared;     // slots that can be occupied in a list
-    for (int i = tid; i < rows * kMaxNodes; i += blockDim.x) {
-      a.wdense[i] = 0.0f;
-      if (a.resident) a.wdense[kMaxSlots * kMaxNodes + i] = 0.0f;
-    }
-    for (int i = tid; i < 2 * kMaxSlots; i += blockDim.x) a.ready[i] = 0;
-  }
-  if (tid < kMaskWords) sm.Hres[tid] = a.resident ? (tid < (E + 31) / 32 ? a.resident[tid] : 0u) : 0xffffffffu;
-  __syncthreads();
-  for (int i = tid; i < T * k; i += blockDim.x) {
-    const int e = sm.idx[i / k][i % k];
-    if (e >= 0) atomicAdd(&sm.cnt[e], 1);
-  }
-  __syncthreads();
-  // slots by ascending expert id: resident activated experts -> list 0, the others -> list 1
-  const bool active = tid < E && sm.cnt[tid] > 0;
-  const bool res = active && ((sm.Hres[warp & 3] >> lane) & 1u);
-  const bool stg = active && !res;
-  const unsigned b0 = __ballot_sync(0xffffffffu, res), b1 = __ballot_sync(0xffffffffu, stg);
-  if (tid < kMaxExperts && lane == 0) {
-    sm.warp_tot[0][warp] = __popc(b0);
-    sm.warp_tot[1][warp] = __popc(b1);
-  }
-  __syncthreads();
-  int base0 = 0, base1 = 0, n0 = 0, n1 = 0;
-#pragma unroll
-  for (int wv = 0; wv < 4; ++wv) {
-    if (wv < warp) { base0 += sm.warp_tot[0][wv]; base1 += sm.warp_tot[1][wv]; }
-    n0 += sm.warp_tot[0][wv];
-    n1 += sm.warp_tot[1][wv];
-  }
-  if (tid < kMaxExperts) {
-    const unsigned lower = (1u << lane) - 1u;
-    if (res) {
-      const int slot = base0 + __popc(b0 & lower);
-      sm.slot_of[tid] = slot; sm.list_of[tid] = 0;
-      a.lists[0].entry[slot] = make_entry(kSrcRouted, tid);
-      a.lists[0].expert[slot] = tid;
-    } else if (stg) {
-      const int slot = base1 + __popc(b1 & lower);
-      sm.slot_of[tid] = slot; sm.list_of[tid] = 1;
-      a.lists[1].entry[slot] = make_entry(kSrcStaged, slot);
-      a.lists[1].expert[slot] = tid;
-      if (a.host_stage_list) a.host_stage_list[1 + slot] = tid;
-    }
-  }
-  if (tid < a.n_shared) {
-    a.lists[0].entry[n0 + tid] = make_entry(kSrcShared, tid);
-    a.lists[0].expert[n0 + tid] = -1;
-  }
-  if (tid == 0) {
-    a.lists[0].n = n0 + a.n_shared; a.lists[0].n_stage = 0;
-    a.lists[1].n = n1; a.lists[1].n_stage = n1;
-    if (a.host_stage_list) a.host_stage_list[0] = n1;
-    if (a.stats_out) { a.stats_out->n_activated = n0 + n1; a.stats_out->n_staged = n1; }
-  }
-  __syncthreads();
-  for (int i = tid; i < T * k; i += blockDim.x) {
-    const int t = i / k, e = sm.idx[t][i % k];
-    if (e >= 0)
-      a.wdense[(static_cast<size_t>(sm.list_of[e]) * kMaxSlots + sm.slot_of[e]) * kMaxNodes + t] = sm.w[t][i % k];
-  }
-  for (int i = tid; i < a.n_shared * T; i += blockDim.x)
-    a.wdense[static_cast<size_t>(n0 + i / T) * kMaxNodes + i % T] = 1.0f;
-  __syncthreads();
-}
-
 // Stage 3 for ONE node, by one warp: restricted top-k (Eq. 2) ranked on the logits, and the
 // combine weights.  Lane j < k returns the j-th choice (expert id or -1) and its weight.
 __device__ __forceinline__ void route_node(const float (&z)[4], const uint32_t (&mask_w)[4], int E, int k, int lane,
@@ -692,6 +618,18 @@ __device__ __forceinline__ void load_logit_row(const float* logits, int t, int E
   }
 }
 
+// Publishes one node's routes (lane j < k holds choice j) to the FFN kernel's inputs: the activated
+// mask (one OR per touched word) and the weight table.
+__device__ __forceinline__ void publish_routes(uint32_t* act_mask, float* wtab, int t, int k, int lane, int e, float w) {
+  const bool has = lane < k && e >= 0;
+#pragma unroll
+  for (int wd = 0; wd < kMaskWords; ++wd) {
+    const unsigned bits = __reduce_or_sync(0xffffffffu, (has && (e >> 5) == wd) ? 1u << (e & 31) : 0u);
+    if (lane == wd && bits) atomicOr(act_mask + wd, bits);
+  }
+  if (has) wtab[static_cast<size_t>(e) * kMaxNodes + t] = w;
+}
+
 __global__ void __launch_bounds__(kSelThreads) k_select(SelectArgs a, int T, int E, int k) {
   __shared__ StageSmem sm;
   stage_select(a, sm, T, E, k, nullptr, true);
@@ -721,7 +659,7 @@ __global__ void __launch_bounds__(kSelThreads) k_route(RouteArgs a, int T, int E
 // `ticket` counts finished CTAs (zero on entry, reset by the last one).
 __global__ void __launch_bounds__(kSelThreads)
 k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uint32_t* mask_override, int T, int E,
-               int k, int32_t* ticket) {
+               int k) {
   __shared__ StageSmem sm;
   __shared__ int s_last;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -731,17 +669,6 @@ k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uin
   ACM_RT(0);
   float z[4];
   load_logit_row(ra.logits, min(t_mine, T - 1), E, lane, z);      // in flight during the selection
-  {
-    // clear this CTA's share of the dense combine-weight tables and (CTA 0) the finished-tile counters
-    const int n4 = (E + ra.n_shared) * kMaxNodes / 4;
-    float4* wd = reinterpret_cast<float4*>(ra.wdense);
-    for (int i = blockIdx.x * kSelThreads + tid; i < n4; i += gridDim.x * kSelThreads) {
-      wd[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (ra.resident) wd[kMaxSlots * kMaxNodes / 4 + i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    if (blockIdx.x == 0)
-      for (int i = tid; i < 2 * kMaxSlots; i += kSelThreads) ra.ready[i] = 0;
-  }
   if (mask_override) {
     if (tid < kMaskWords) {
       const uint32_t m = tid < (E + 31) / 32 ? mask_override[tid] : 0u;
@@ -768,48 +695,74 @@ k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uin
       ra.idx_out[static_cast<size_t>(t_mine) * k + lane] = e;
       ra.w_out[static_cast<size_t>(t_mine) * k + lane] = w;
     }
+    if (ra.act_mask && t_mine < T) publish_routes(ra.act_mask, ra.wtab, t_mine, k, lane, e, w);
   }
   ACM_RT(3);
-  // the CTA that finishes last sees every route and builds the lists
+  if (!ra.ticket) return;
+  // Asked for a report on the whole block: the CTA that finishes last sees the complete mask.
   __threadfence();
   __syncthreads();
   if (tid == 0) {
-    const int prev = atomicAdd(ticket, 1);
+    const int prev = atomicAdd(ra.ticket, 1);
     s_last = prev == static_cast<int>(gridDim.x) - 1;
-    if (s_last) *ticket = 0;
+    if (s_last) *ra.ticket = 0;
   }
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  for (int i = tid; i < T * k; i += kSelThreads) {
-    sm.idx[i / k][i % k] = __ldcg(ra.idx_out + i);
-    sm.w[i / k][i % k] = __ldcg(ra.w_out + i);
+  if (warp == 0) {
+    const int words = (E + 31) / 32;
+    const uint32_t act = lane < words ? __ldcg(ra.act_mask + lane) : 0u;
+    const uint32_t res = lane < words ? (ra.resident ? ra.resident[lane] : 0xffffffffu) : 0u;
+    const uint32_t stg = act & ~res;
+    int n_act = __popc(act), n_stg = __popc(stg), before = 0;
+#pragma unroll
+    for (int s = 1; s < 32; s <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, n_stg, s);      // inclusive scan of the staged counts
+      n_stg += lane >= s ? up : 0;
+    }
+    before = n_stg - __popc(stg);
+    const int tot_stg = __shfl_sync(0xffffffffu, n_stg, 31);
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) n_act += __shfl_xor_sync(0xffffffffu, n_act, s);
+    if (ra.host_stage_list) {
+      uint32_t m = stg;
+      int pos = before;
+      while (m) {                        // staged experts in ascending id order = their staging slots
+        const int b = __ffs(m) - 1;
+        m &= m - 1;
+        ra.host_stage_list[1 + pos++] = lane * 32 + b;
+      }
+      if (lane == 0) ra.host_stage_list[0] = tot_stg;
+    }
+    if (lane == 0 && ra.stats_out) { ra.stats_out->n_activated = n_act; ra.stats_out->n_staged = tot_stg; }
   }
-  __syncthreads();
-  if (ra.dbg && tid == 0) ra.dbg[1] = time_ns();
-  stage_build_lists(ra, sm, T, E, k, false);
   if (ra.dbg && tid == 0) ra.dbg[4] = time_ns();
 }
 
-__global__ void __launch_bounds__(512) k_routes_to_lists(const int32_t* idx, const float* w, RouteArgs a, int T,
-                                                         int E, int k) {
-  __shared__ StageSmem sm;
+// Routes given by the caller (acm_expert_ffn) -> the FFN kernel's inputs.  One CTA.
+__global__ void __launch_bounds__(512) k_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask,
+                                                         float* wtab, int32_t* ready, int T, int E, int k) {
+  for (int i = threadIdx.x; i < kMaxExperts * kMaxNodes; i += blockDim.x) wtab[i] = 0.0f;
+  for (int i = threadIdx.x; i < 2 * kMaxSlots; i += blockDim.x) ready[i] = 0;
+  if (threadIdx.x < kMaskWords) act_mask[threadIdx.x] = 0u;
+  __syncthreads();
   for (int i = threadIdx.x; i < T * k; i += blockDim.x) {
     const int e = idx[i];
-    sm.idx[i / k][i % k] = (e >= 0 && e < E) ? e : -1;
-    sm.w[i / k][i % k] = w[i];
+    if (e >= 0 && e < E) {
+      atomicOr(act_mask + (e >> 5), 1u << (e & 31));
+      wtab[static_cast<size_t>(e) * kMaxNodes + i / k] = w[i];
+    }
   }
-  __syncthreads();
-  stage_build_lists(a, sm, T, E, k, true);
 }
 
 }  // namespace
 
 cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router, const float* bias,
                                  float* logits, int T, int H, int E, float* zero_buf,
-                                 size_t zero_floats, int32_t* status, float* probs, int32_t* nat_idx,
-                                 uint32_t* nat_mask, int k, int32_t* tile_done, bool pdl, cudaStream_t s,
-                                 long long* dbg) {
+                                 size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status,
+                                 float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k, int32_t* tile_done,
+                                 bool pdl, cudaStream_t s, long long* dbg) {
   if (!probs && !nat_idx) tile_done = nullptr;
   cudaLaunchAttribute attr[1];
   set_pdl_attr(attr);
@@ -830,7 +783,7 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     if (err != cudaSuccess) return err;
     cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * 8); cfg.dynamicSmemBytes = smem;
     return cudaLaunchKernelEx(&cfg, kern, static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
-                              logits, T, H, E, n_chunks, zero_buf, zero_floats, status, probs, nat_idx, nat_mask, k,
+                              logits, T, H, E, n_chunks, zero_buf, zero_floats, zero_buf2, zero_floats2, status, probs, nat_idx, nat_mask, k,
                               tile_done, dbg);
   } else {
     auto kern = k_router_logits<__nv_bfloat16>;
@@ -839,7 +792,7 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * (32 / ElemTraits<__nv_bfloat16>::EPT)); cfg.dynamicSmemBytes = smem;
     return cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x),
                               static_cast<const __nv_bfloat16*>(w_router), bias, logits, T, H, E, n_chunks, zero_buf,
-                              zero_floats, status, probs, nat_idx, nat_mask, k, tile_done, dbg);
+                              zero_floats, zero_buf2, zero_floats2, status, probs, nat_idx, nat_mask, k, tile_done, dbg);
   }
 }
 
@@ -854,8 +807,7 @@ cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s
 }
 
 cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
-                                const uint32_t* mask_override, int T, int E, int k, int32_t* ticket,
-                                bool pdl, cudaStream_t s) {
+                                const uint32_t* mask_override, int T, int E, int k, bool pdl, cudaStream_t s) {
   cudaLaunchAttribute attr[1];
   set_pdl_attr(attr);
   cudaLaunchConfig_t cfg = {};
@@ -864,17 +816,12 @@ cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, 
   cfg.stream = s;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, k_select_route, nat_mask, sa, ra, mask_override, T, E, k, ticket);
+  return cudaLaunchKernelEx(&cfg, k_select_route, nat_mask, sa, ra, mask_override, T, E, k);
 }
 
-cudaError_t launch_routes_to_lists(const int32_t* idx, const float* w, WorkList* lists, float* wdense,
-                                   int32_t* ready, int n_shared, int T, int E, int k, cudaStream_t s) {
-  RouteArgs a = {};
-  a.lists = lists;
-  a.wdense = wdense;
-  a.ready = ready;
-  a.n_shared = n_shared;
-  k_routes_to_lists<<<1, 512, 0, s>>>(idx, w, a, T, E, k);
+cudaError_t launch_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask, float* wtab,
+                                   int32_t* ready, int T, int E, int k, cudaStream_t s) {
+  k_routes_to_table<<<1, 512, 0, s>>>(idx, w, act_mask, wtab, ready, T, E, k);
   return cudaGetLastError();
 }
 
