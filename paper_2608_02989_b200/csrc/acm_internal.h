@@ -50,6 +50,7 @@ struct Workspace {
   int32_t* status;      // [1] sticky device-side status
   int32_t* tile_done;   // [64] router kernel: expert tiles finished per node tile (self-resetting)
   int32_t* ticket;      // [1] select/route kernel: finished CTAs (self-resetting)
+  uint32_t* sel_words;  // [8] the eligible mask as tagged 16-bit pieces (early start of the FFN kernel)
 };
 
 struct SelectArgs {
@@ -83,6 +84,8 @@ struct RouteArgs {
   const uint32_t* resident;      // non-null: activated experts outside it are "staged"
   acm_block_stats* stats_out;    // n_activated / n_staged are filled in
   int32_t* host_stage_list;      // mapped pinned memory: [0] = n_stage, [1..] = staged expert ids (may be null)
+  uint32_t* sel_flag;            // non-null: [8] words, the eligible mask in 16-bit pieces tagged with sel_epoch
+  int32_t sel_epoch;
   long long* dbg;                // optional time stamps in ns of the select/route kernel's stages (debugging aid)
 };
 
@@ -109,6 +112,7 @@ cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s
 // small CTAs; `nat_mask` = the natural top-k sets as bit masks [T][4] (from launch_router_logits)
 cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
                                 const uint32_t* mask_override, int T, int E, int k, bool pdl, cudaStream_t s);
+int route_ctas(int T);   // grid size of launch_select_route
 // routes given by the caller -> activated mask, weight table (both cleared first) and cleared `ready`
 cudaError_t launch_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask, float* wtab,
                                    int32_t* ready, int T, int E, int k, cudaStream_t s);
@@ -131,7 +135,13 @@ struct FfnLaunch {
   int32_t* ready;            // [kMaxSlots] of this list (zero on entry)
   float* frag;
   int32_t* frag_flag;
-  int32_t epoch;
+  // Early start: if sel_flag is given the kernel does not wait for the routing kernel to complete.  It
+  // polls the eight tagged words at sel_flag (16 bits of the ELIGIBLE mask under the low 16 bits of
+  // sel_epoch each) and takes the eligible set as its work list -- an eligible expert no node chose
+  // has zero combine weights and contributes nothing.  The combine weights are read only when the
+  // first tile is finalised, after a full dependency wait.
+  const uint32_t* sel_flag;
+  int32_t sel_epoch;
   float* out;                // [T,H], accumulated into (zeroed by the caller)
   int32_t* status;
   int grid;

@@ -63,6 +63,7 @@ struct acm_ctx {
   int timing_period = 1;        // every n-th FFN launch is bracketed by events
   long long timing_seen = 0;
   bool pdl = true;              // programmatic dependent launches between the kernels of the hot path
+  bool early_start = true;      // the FFN kernel starts on the eligible set, before the routes are final
   std::vector<cudaEvent_t> ev_pool;
   size_t ev_used = 0;
   uint64_t launches = 0;
@@ -181,7 +182,8 @@ acm_status check_block_args(const acm_ctx* c, int layer, int T, bool need_weight
 
 // One FFN launch over work list `li` (0 = resident + shared, 1 = staged).
 acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li, float* out, cudaStream_t s,
-                        const uint32_t* res_dev = nullptr, acm_block_stats* stats_dev = nullptr, bool pdl_ok = false) {
+                        const uint32_t* res_dev = nullptr, acm_block_stats* stats_dev = nullptr, bool pdl_ok = false,
+                        int32_t early_epoch = 0) {
   const acm_model_desc& d = c->desc;
   const int n_pad = (T + 15) / 16 * 16;
   acm_status st = ensure_h_maps(c, n_pad);
@@ -205,9 +207,16 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   p.hbuf = static_cast<char*>(c->ws.hbuf) + static_cast<size_t>(li) * kMaxSlots * kMaxNodes * d.inter * 2;
   p.ready = c->ws.ready + li * kMaxSlots;
   p.frag = c->ws.frag; p.frag_flag = c->ws.frag_flag;
-  p.epoch = ++c->epoch;
+  p.sel_flag = nullptr; p.sel_epoch = 0;
+  if (early_epoch != 0) {
+    p.sel_flag = c->ws.sel_words;
+    p.sel_epoch = early_epoch;
+  }
   p.out = out; p.status = c->ws.status;
-  p.grid = c->sm_count;
+  // Early start: the routing kernel still holds a few SMs when this kernel's CTAs are placed, and an SM
+  // changes hands slowly; leave those SMs out so that every CTA starts at once.
+  p.grid = early_epoch != 0 ? c->sm_count - route_ctas(T) : c->sm_count;
+  if (p.grid < 1) p.grid = 1;
   p.phase_mask = 3;
   p.trace = c->trace;
   p.pdl = false;
@@ -225,7 +234,6 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
     p.phase_mask = 1;
     ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
     p.phase_mask = 2;
-    p.epoch = ++c->epoch;
     c->launches += 1;
   }
   // dependent launch only straight after the select/route kernel (no event, memset or copy between)
@@ -308,6 +316,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->split_phases = split && split[0] == '1';
   const char* no_pdl = std::getenv("ACM_NO_PDL");
   c->pdl = !(no_pdl && no_pdl[0] == '1');
+  const char* no_early = std::getenv("ACM_NO_EARLY_START");
+  c->early_start = !(no_early && no_early[0] == '1');
   const char* trace = std::getenv("ACM_FFN_TRACE");
   const bool want_trace = trace && (trace[0] == '1' || trace[0] == '2');
   c->trace_light = trace && trace[0] == '2';
@@ -354,6 +364,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_status = carve(16);
   const size_t o_tile = carve(sizeof(int32_t) * kMaxNodes);
   const size_t o_ticket = carve(16);
+  const size_t o_selw = carve(32);
   const size_t o_natmask = carve(sizeof(uint32_t) * Tm * kMaskWords);
   const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
   if (cudaMalloc(&c->ws_base, off) != cudaSuccess) return fail(ACM_ERR_NOMEM);
@@ -382,6 +393,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.status = reinterpret_cast<int32_t*>(b + o_status);
   c->ws.tile_done = reinterpret_cast<int32_t*>(b + o_tile);
   c->ws.ticket = reinterpret_cast<int32_t*>(b + o_ticket);
+  c->ws.sel_words = reinterpret_cast<uint32_t*>(b + o_selw);
   c->ws.nat_mask = reinterpret_cast<uint32_t*>(b + o_natmask);
   c->resident_dev = reinterpret_cast<uint32_t*>(b + o_res);
   if (want_trace && cudaMalloc(&c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 16)) != cudaSuccess)
@@ -576,6 +588,17 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   ra.stats_out = c->ws.stats;
   // the bf16 FFN kernel counts the activated experts itself; otherwise the routing kernel's last CTA does
   ra.ticket = (f32 || L.has_resident) ? c->ws.ticket : nullptr;
+  // Early start of the FFN kernel on the eligible set: when a selection runs (the eligible experts are
+  // then nearly always all activated; with an override mask they need not be) and every expert is resident.
+  const bool early = !f32 && !L.has_resident && !eligible_mask_override && !c->split_phases && c->early_start;
+  int32_t early_epoch = 0;
+  if (early) {
+    early_epoch = ++c->epoch;            // its low 16 bits tag the published words; 0 is never a valid tag
+    if ((early_epoch & 0xffff) == 0) early_epoch = ++c->epoch;
+    if (early_epoch <= 0) early_epoch = c->epoch = 1;
+    ra.sel_flag = c->ws.sel_words;
+    ra.sel_epoch = early_epoch;
+  }
   ra.dbg = c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr;
   ACM_CUDA(launch_select_route(c->ws.nat_mask, sa, ra, eligible_mask_override, T, E, k, c->pdl, s));
   c->launches += 2;
@@ -587,7 +610,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
                             static_cast<float*>(c->ws.hbuf), out, T, d.hidden, d.inter, k, s));
     c->launches += 2;
   } else if (!L.has_resident) {
-    st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, c->ws.stats, true);
+    st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, c->ws.stats, true, early_epoch);
     if (st != ACM_OK) return st;
   } else {
     // resident + shared experts run at once; the others are copied in from pinned host memory first
@@ -704,6 +727,8 @@ acm_status acm_device_status(acm_ctx* c, acm_stream stream) {
     ACM_CUDA(cudaMemset(c->ws.frag, 0, c->frag_bytes));
     ACM_CUDA(cudaMemset(c->ws.frag_flag, 0, c->flag_bytes));
     ACM_CUDA(cudaMemset(c->ws.ticket, 0, 16));
+    ACM_CUDA(cudaMemset(c->ws.sel_words, 0, 32));
+    c->epoch = 0;
     ACM_CUDA(cudaMemset(c->ws.tile_done, 0, sizeof(int32_t) * kMaxNodes));
   }
   return static_cast<acm_status>(v);

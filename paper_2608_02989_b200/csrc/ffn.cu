@@ -70,6 +70,7 @@ struct __align__(8) Barriers {
   float wd[kMaxNodes];          // combine weights of the expert being finalised
   int32_t entry[kMaxSlots];     // this launch's work list: make_entry(source, index) of every activated slot
   int32_t expert[kMaxSlots];    // routed expert id of the slot (-1: shared expert)
+  uint32_t sel_half[2 * kMaskWords];   // early start: the eligible mask in 16-bit pieces
 };
 
 constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + kOutStageBytes + kFragBytes + 2 * kHStageBytes + sizeof(Barriers);
@@ -303,7 +304,8 @@ struct FfnArgs {
   int32_t* ready;
   float* frag;
   int32_t* frag_flag;
-  int32_t epoch;
+  const uint32_t* sel_flag;
+  int32_t sel_epoch;
   float* out;
   int32_t* status;
   int phase_mask;
@@ -388,6 +390,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, G = gridDim.x;
   griddep_launch_dependents();
+  if (threadIdx.x == 0) ACM_TRACE(12);     // kernel entry
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&bars->full[s]), 1);
@@ -423,8 +426,30 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     tmem_relinquish();
   }
   // Everything above touched only this CTA's own resources; global memory written by the kernels
-  // before this one (the work list above all) is read only from here on.
-  griddep_wait();
+  // before this one is read only from here on.  Early start: wait for the eligible set only.
+  const bool early = p.sel_flag != nullptr;
+  if (early) {
+    // eight tagged words (16 mask bits under the 16-bit tag of this call), each polled by its own thread
+    if (threadIdx.x < 2 * kMaskWords) {
+      bool seen = false;
+      uint32_t v = 0;
+      const uint32_t tag = static_cast<uint32_t>(p.sel_epoch) & 0xffffu;
+      const unsigned long long t0 = global_timer();
+      do {
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.sel_flag + threadIdx.x) : "memory");
+        seen = (v >> 16) == tag;
+      } while (!seen && global_timer() - t0 < kTimeoutNs);
+      if (!seen) {
+        bars->abort_flag = 1;
+        atomicCAS(p.status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+        v = 0;
+      }
+      bars->sel_half[threadIdx.x] = v & 0xffffu;
+    }
+    __syncthreads();
+  } else {
+    griddep_wait();
+  }
   // The work list of this launch: slot a = the a-th activated expert of this list in ascending id
   // order (list 0: the resident ones, then the shared experts; list 1: the non-resident ones, which
   // the host has copied into staging slot a).
@@ -432,7 +457,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   int n_routed = 0;
 #pragma unroll
   for (int wd = 0; wd < kMaskWords; ++wd) {
-    const uint32_t act = p.act_mask[wd];
+    const uint32_t act = early ? (bars->sel_half[2 * wd] | (bars->sel_half[2 * wd + 1] << 16)) : p.act_mask[wd];
     const uint32_t res = p.resident ? p.resident[wd] : 0xffffffffu;
     am[wd] = p.li == 0 ? act & res : act & ~res;
     n_routed += __popc(am[wd]);
@@ -463,18 +488,6 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     s_entry[n_routed + i] = make_entry(kSrcShared, i);
     bars->expert[n_routed + i] = -1;
   }
-  if (p.stats && p.li == 0 && blockIdx.x == 0 && threadIdx.x == 0) {
-    int n_all = 0, n_stg = 0;
-#pragma unroll
-    for (int wd = 0; wd < kMaskWords; ++wd) {
-      const uint32_t act = p.act_mask[wd];
-      n_all += __popc(act);
-      n_stg += p.resident ? __popc(act & ~p.resident[wd]) : 0;
-    }
-    p.stats->n_activated = n_all;
-    p.stats->n_staged = n_stg;
-  }
-
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -489,6 +502,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     // it.  The loop is kept to a few instructions per stage: one thread pays every one of them.
     if (lane == 0) {
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      ACM_TRACE(3);
       uint32_t s = 0, par = 0, n_armed = 0;
       bool ok = true, traced_first = false;
       for (int si = 0; si < n_seg && ok; ++si) {
@@ -502,7 +516,9 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             const int r0 = ((sg.t0 + tile) % tpe) * 64, eidx = entry_idx(ent);
             const CUtensorMap* gu = pick_map(entry_src(ent), &maps.gate_up, &maps.shared_gate_up, &maps.staged_gate_up);
             for (int kc = k0; kc < k1; ++kc) {
+              if (!traced_first) ACM_TRACE(4);
               if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
+              if (!traced_first) ACM_TRACE(16);
               const uint32_t full = smem_u32(&bars->full[s]);
               const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
               mbar_expect_tx(full, kABytes + b_bytes);
@@ -755,7 +771,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     const int row = quarter * 32 + lane;        // accumulator row = weight-tile row
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
     uint32_t f = 0, ost_uses = 0, fin_count = 0;
-    bool ok = true;
+    bool ok = true, waited = !early;
     float v[kMaxNodes];
     auto load_acc = [&](uint32_t b) {
 #pragma unroll
@@ -797,9 +813,13 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             continue;
           }
           const int a = (sg.t0 + tile) / tpe;
+          if (!waited) {          // the combine weights are the routing kernel's last output
+            griddep_wait();
+            waited = true;
+          }
           if (row < p.n_pad) {
             const int ex_id = bars->expert[a];      // combine weights: the table row of a routed expert, 1 for a shared one
-            bars->wd[row] = ex_id >= 0 ? p.wtab[static_cast<size_t>(ex_id) * kMaxNodes + row] : (row < p.T ? 1.0f : 0.0f);
+            bars->wd[row] = ex_id >= 0 ? __ldcg(p.wtab + static_cast<size_t>(ex_id) * kMaxNodes + row) : (row < p.T ? 1.0f : 0.0f);
           }
           if (k1 < kc1) {
             // head part: the helper warp has summed the other CTAs' fragments of this tile into smem
@@ -894,7 +914,18 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
 
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0) ACM_TRACE(12);
+  if (p.stats && p.li == 0 && blockIdx.x == 0 && threadIdx.x == 0) {
+    griddep_wait();                       // early start: the routing kernel is long complete
+    int n_all = 0, n_stg = 0;
+#pragma unroll
+    for (int wd = 0; wd < kMaskWords; ++wd) {
+      const uint32_t act = __ldcg(p.act_mask + wd);
+      n_all += __popc(act);
+      n_stg += p.resident ? __popc(act & ~p.resident[wd]) : 0;
+    }
+    p.stats->n_activated = n_all;
+    p.stats->n_staged = n_stg;
+  }
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
@@ -973,7 +1004,8 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   a.T = L.T; a.H = L.H; a.I = L.I; a.n_pad = L.n_pad;
   a.act_mask = L.act_mask; a.resident = L.resident; a.li = L.li; a.n_shared = L.n_shared; a.wtab = L.wtab;
   a.stats = L.stats; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
-  a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag; a.epoch = L.epoch;
+  a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag;
+  a.sel_flag = L.sel_flag; a.sel_epoch = L.sel_epoch;
   a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask; a.trace = L.trace;
   void* args[] = {const_cast<FfnMaps*>(&maps), const_cast<CUtensorMap*>(&x_map), const_cast<CUtensorMap*>(&h_map),
                   const_cast<CUtensorMap*>(&hs_map), &a};

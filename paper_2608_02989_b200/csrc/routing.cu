@@ -654,16 +654,28 @@ __global__ void __launch_bounds__(kSelThreads) k_route(RouteArgs a, int T, int E
   }
 }
 
+// The FFN kernel may start on the eligible set while the routes are made.  The set is published as
+// eight self-validating words, 16 mask bits under a 16-bit tag of this call each: a reader needs no
+// second load to know that what it read is current.  (Relaxed stores: everything else the reader
+// depends on was complete before this kernel passed its dependency wait.)
+__device__ __forceinline__ void publish_eligible(const RouteArgs& ra, const StageSmem& sm, int i) {
+  const uint32_t bits = (sm.Sp[i >> 1] >> (16 * (i & 1))) & 0xffffu;
+  const uint32_t word = bits | (static_cast<uint32_t>(ra.sel_epoch) << 16);
+  asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(ra.sel_flag + i), "r"(word) : "memory");
+}
+
 #define ACM_RT(slot) do { if (ra.dbg && blockIdx.x == 0 && threadIdx.x == 0) ra.dbg[slot] = time_ns(); } while (0)
-// Stages 2-3 and the FFN work lists in one launch of ceil(T / 4) CTAs (see the note above).
-// `ticket` counts finished CTAs (zero on entry, reset by the last one).
-__global__ void __launch_bounds__(kSelThreads)
+// Stages 2-3 and the FFN kernel's routing inputs in one launch of a few CTAs (see the note above):
+// one warp per node, up to 16 nodes per CTA; warps 0-3 of every CTA run the selection.  Few CTAs on
+// purpose: the FFN kernel, launched as a dependent, can take over an SM only once this kernel has left it.
+constexpr int kRouteNodesPerCta = 16;
+__global__ void __launch_bounds__(32 * kRouteNodesPerCta)
 k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uint32_t* mask_override, int T, int E,
                int k) {
   __shared__ StageSmem sm;
   __shared__ int s_last;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int t_mine = blockIdx.x * kNodesPerCta + warp;
+  const int t_mine = blockIdx.x * (blockDim.x >> 5) + warp;
   griddep_launch_dependents();
   griddep_wait();
   ACM_RT(0);
@@ -681,8 +693,13 @@ k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uin
     }
     __syncthreads();
   } else {
-    stage_select(sa, sm, T, E, k, natmask_g, blockIdx.x == 0);
+    if (tid < kSelThreads) {
+      stage_select(sa, sm, T, E, k, natmask_g, blockIdx.x == 0);
+      if (ra.sel_flag && blockIdx.x == 0 && tid < 2 * kMaskWords) publish_eligible(ra, sm, tid);
+    }
+    __syncthreads();
   }
+  if (mask_override && ra.sel_flag && blockIdx.x == 0 && tid < 2 * kMaskWords) publish_eligible(ra, sm, tid);
   ACM_RT(2);
   {
     uint32_t mask_w[4];
@@ -772,7 +789,10 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
   cfg.numAttrs = pdl ? 1 : 0;
   const dim3 grid((E + kRE - 1) / kRE, (T + kRT - 1) / kRT);
   const int elt = dtype == ACM_F32 ? 4 : 2;
-  const size_t smem = static_cast<size_t>(kRT + kRE) * (static_cast<size_t>(H) * elt + 64);
+  size_t smem = static_cast<size_t>(kRT + kRE) * (static_cast<size_t>(H) * elt + 64);
+  // At most two CTAs per SM (by asking for more shared memory than the tile needs): the grid then
+  // spreads over the whole GPU instead of piling four deep onto the SMs that happen to be free first.
+  if (smem < (104u << 10)) smem = 104u << 10;
   // pieces of at least 4 KB per row: every bulk copy has a fixed cost, and few large ones land sooner
   const size_t row = static_cast<size_t>(H) * elt;
   const int n_chunks = (row >= 16384 && H % 128 == 0) ? 4 : (row >= 8192 && H % 64 == 0) ? 2 : 1;
@@ -796,6 +816,11 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
   }
 }
 
+int route_ctas(int T) {
+  const int npc = T < kRouteNodesPerCta ? (T < 4 ? 4 : T) : kRouteNodesPerCta;
+  return (T + npc - 1) / npc;
+}
+
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s) {
   k_select<<<1, kSelThreads, 0, s>>>(a, T, E, k);
   return cudaGetLastError();
@@ -811,8 +836,9 @@ cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, 
   cudaLaunchAttribute attr[1];
   set_pdl_attr(attr);
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((T + kNodesPerCta - 1) / kNodesPerCta);
-  cfg.blockDim = dim3(kSelThreads);
+  const int npc = T < kRouteNodesPerCta ? (T < 4 ? 4 : T) : kRouteNodesPerCta;     // at least the four selection warps
+  cfg.gridDim = dim3(route_ctas(T));
+  cfg.blockDim = dim3(32 * npc);
   cfg.stream = s;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
