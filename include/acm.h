@@ -173,6 +173,21 @@ acm_status acm_moe_verify(acm_ctx* ctx, int layer, const void* x, int T, const f
                           float* w_out, uint32_t* mask_out, acm_block_stats* stats,
                           acm_stream stream);
 
+/* The same call for HOST buffers (Section 3.1's per-layer step as a serving loop sees it): x_host
+ * [T,H] and alpha_host [T] are read from, and out_host [T,H] float is written to, PINNED host
+ * memory.  The copies run on the context's own copy streams through two alternating sets of device
+ * buffers, so the upload of the next block and the download of the previous one overlap this block's
+ * kernels; the kernels run on `stream`.  The call returns once everything is enqueued.  out_host and
+ * stats_host (optional, host) are valid after acm_host_synchronize(); x_host and alpha_host must stay
+ * unchanged until then (or until two later calls of this function have returned and `stream` has
+ * passed them).  Not available with a residency registered for the layer. */
+acm_status acm_moe_verify_host(acm_ctx* ctx, int layer, const void* x_host, int T,
+                               const float* alpha_host, const acm_select_params* params /*host*/,
+                               float* out_host, acm_block_stats* stats_host, acm_stream stream);
+
+/* Waits until every copy enqueued by acm_moe_verify_host has completed. */
+acm_status acm_host_synchronize(acm_ctx* ctx);
+
 /* Offload variant (Section 3.4): marks which experts of `layer` are GPU-resident
  * (resident_mask: HOST words) and registers pinned HOST copies of the full expert tensors
  * used to load non-resident experts on demand.  The device tensors registered with

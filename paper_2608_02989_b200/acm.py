@@ -23,8 +23,8 @@ DEMAND_TOPK_MASS, DEMAND_FULL_MASS, DEMAND_VOTES = 0, 1, 2
 EXPORTS = [
     "acm_default_select_params", "acm_create", "acm_destroy", "acm_set_layer_weights",
     "acm_node_weights", "acm_router", "acm_select_eligible", "acm_route_restricted",
-    "acm_expert_ffn", "acm_moe_verify", "acm_set_resident", "acm_h2d_bytes", "acm_ffn_timing",
-    "acm_ffn_time_ms", "acm_launch_count", "acm_device_status", "acm_status_string",
+    "acm_expert_ffn", "acm_moe_verify", "acm_moe_verify_host", "acm_host_synchronize", "acm_set_resident",
+    "acm_h2d_bytes", "acm_ffn_timing", "acm_ffn_time_ms", "acm_launch_count", "acm_device_status", "acm_status_string",
     "acm_expert_ffn_f32_noalloc",
 ]
 NOALLOC_MAX_FLOATS = 1 << 20
@@ -88,6 +88,9 @@ def load_library():
     lib.acm_expert_ffn.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.acm_moe_verify.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, POINTER(SelectParams),
                                    c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.acm_moe_verify_host.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, POINTER(SelectParams),
+                                        c_void_p, c_void_p, c_void_p]
+    lib.acm_host_synchronize.argtypes = [c_void_p]
     lib.acm_set_resident.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p]
     lib.acm_h2d_bytes.argtypes = [c_void_p, POINTER(c_uint64), c_int]
     lib.acm_ffn_timing.argtypes = [c_void_p, c_int, c_int]
@@ -255,6 +258,20 @@ class Context:
         if want:
             return out, idx, w, mask, stats
         return out
+
+    def moe_verify_host(self, layer, x_host, alpha_host, out_host, params=None, stats_host=None, stream=None):
+        """Stages 1-4 on PINNED host tensors (x, alpha in; out, optional stats [12] int32 out).  Asynchronous:
+        call host_synchronize() before reading out_host."""
+        for t in (x_host, alpha_host, out_host):
+            if t.is_cuda or not t.is_pinned():
+                raise ValueError("moe_verify_host takes pinned host tensors")
+        params = params or SelectParams()
+        _check(self.lib.acm_moe_verify_host(self.handle, layer, _p(x_host), x_host.shape[0], _p(alpha_host),
+                                            byref(params), _p(out_host), _p(stats_host), _stream(stream)),
+               "acm_moe_verify_host")
+
+    def host_synchronize(self):
+        _check(self.lib.acm_host_synchronize(self.handle), "acm_host_synchronize")
 
     # ------------------------------------------------------------------ bookkeeping
     def h2d_bytes(self, reset=False) -> int:

@@ -57,6 +57,15 @@ struct acm_ctx {
   cudaEvent_t ev_lists = nullptr, ev_copied = nullptr, ev_stage_free = nullptr;
   bool stage_in_use = false;
   uint64_t h2d_bytes = 0;
+  // host-buffer path (acm_moe_verify_host): two alternating sets of device buffers and copy streams
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  void* hx_dev[2] = {nullptr, nullptr};
+  float* halpha_dev[2] = {nullptr, nullptr};
+  float* hout_dev[2] = {nullptr, nullptr};
+  acm_block_stats* hstats_dev[2] = {nullptr, nullptr};
+  cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+  unsigned long long host_calls = 0;
+  size_t host_h2d = 0, host_d2h = 0;   // bytes copied by that path
   // per-launch FFN timing
   size_t ffn_in_floats = 0;     // length of the block wtab | ready | act_mask, in floats
   bool timing = false;
@@ -285,7 +294,7 @@ void acm_default_select_params(acm_select_params* p) {
 acm_status acm_debug_ffn_trace(acm_ctx* c, unsigned long long* host_out, int* n_ctas) {
   if (!c || !host_out || !n_ctas || !c->trace) return ACM_ERR_INVALID;
   ACM_CUDA(cudaDeviceSynchronize());
-  ACM_CUDA(cudaMemcpy(host_out, c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 16), cudaMemcpyDeviceToHost));
+  ACM_CUDA(cudaMemcpy(host_out, c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 32), cudaMemcpyDeviceToHost));
   *n_ctas = c->sm_count;
   return ACM_OK;
 }
@@ -396,7 +405,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.sel_words = reinterpret_cast<uint32_t*>(b + o_selw);
   c->ws.nat_mask = reinterpret_cast<uint32_t*>(b + o_natmask);
   c->resident_dev = reinterpret_cast<uint32_t*>(b + o_res);
-  if (want_trace && cudaMalloc(&c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 16)) != cudaSuccess)
+  if (want_trace && cudaMalloc(&c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 32)) != cudaSuccess)
     return fail(ACM_ERR_NOMEM);
   *out = c;
   return ACM_OK;
@@ -410,6 +419,17 @@ acm_status acm_destroy(acm_ctx* c) {
   if (c->ev_copied) cudaEventDestroy(c->ev_copied);
   if (c->ev_stage_free) cudaEventDestroy(c->ev_stage_free);
   if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  if (c->h2d_stream) cudaStreamDestroy(c->h2d_stream);
+  if (c->d2h_stream) cudaStreamDestroy(c->d2h_stream);
+  for (int b = 0; b < 2; ++b) {
+    if (c->hx_dev[b]) cudaFree(c->hx_dev[b]);
+    if (c->halpha_dev[b]) cudaFree(c->halpha_dev[b]);
+    if (c->hout_dev[b]) cudaFree(c->hout_dev[b]);
+    if (c->hstats_dev[b]) cudaFree(c->hstats_dev[b]);
+    if (c->ev_in[b]) cudaEventDestroy(c->ev_in[b]);
+    if (c->ev_done[b]) cudaEventDestroy(c->ev_done[b]);
+    if (c->ev_out[b]) cudaEventDestroy(c->ev_out[b]);
+  }
   if (c->host_stage_list) cudaFreeHost(c->host_stage_list);
   if (c->stage_gate_up) cudaFree(c->stage_gate_up);
   if (c->stage_down) cudaFree(c->stage_down);
@@ -651,6 +671,76 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   if (stats) ACM_CUDA(cudaMemcpyAsync(stats, c->ws.stats, sizeof(acm_block_stats), cudaMemcpyDefault, s));
   return ACM_OK;
 }
+
+namespace {
+acm_status ensure_host_path(acm_ctx* c) {
+  if (c->h2d_stream) return ACM_OK;
+  const acm_model_desc& d = c->desc;
+  const size_t elt = d.dtype == ACM_F32 ? 4 : 2;
+  ACM_CUDA(cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking));
+  ACM_CUDA(cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking));
+  for (int b = 0; b < 2; ++b) {
+    ACM_CUDA(cudaMalloc(&c->hx_dev[b], static_cast<size_t>(kMaxNodes) * d.hidden * elt));
+    ACM_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->halpha_dev[b]), kMaxNodes * sizeof(float)));
+    ACM_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->hout_dev[b]), static_cast<size_t>(kMaxNodes) * d.hidden * sizeof(float)));
+    ACM_CUDA(cudaMalloc(reinterpret_cast<void**>(&c->hstats_dev[b]), sizeof(acm_block_stats)));
+    ACM_CUDA(cudaEventCreateWithFlags(&c->ev_in[b], cudaEventDisableTiming));
+    ACM_CUDA(cudaEventCreateWithFlags(&c->ev_done[b], cudaEventDisableTiming));
+    ACM_CUDA(cudaEventCreateWithFlags(&c->ev_out[b], cudaEventDisableTiming));
+  }
+  return ACM_OK;
+}
+}  // namespace
+
+acm_status acm_moe_verify_host(acm_ctx* c, int layer, const void* x_host, int T, const float* alpha_host,
+                               const acm_select_params* params, float* out_host, acm_block_stats* stats_host,
+                               acm_stream stream) {
+  acm_status st = check_block_args(c, layer, T, true);
+  if (st != ACM_OK) return st;
+  if (!x_host || !alpha_host || !out_host || !params) return ACM_ERR_INVALID;
+  if (c->layers[layer].has_resident) return ACM_ERR_UNSUPPORTED;
+  st = ensure_host_path(c);
+  if (st != ACM_OK) return st;
+  const acm_model_desc& d = c->desc;
+  const size_t elt = d.dtype == ACM_F32 ? 4 : 2;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int b = static_cast<int>(c->host_calls & 1ull);
+  const bool reused = c->host_calls >= 2;
+  // upload into set b once the kernels of the call before last (its previous user) are done with it
+  if (reused) ACM_CUDA(cudaStreamWaitEvent(c->h2d_stream, c->ev_done[b], 0));
+  ACM_CUDA(cudaMemcpyAsync(c->hx_dev[b], x_host, static_cast<size_t>(T) * d.hidden * elt, cudaMemcpyHostToDevice,
+                           c->h2d_stream));
+  ACM_CUDA(cudaMemcpyAsync(c->halpha_dev[b], alpha_host, static_cast<size_t>(T) * sizeof(float),
+                           cudaMemcpyHostToDevice, c->h2d_stream));
+  ACM_CUDA(cudaEventRecord(c->ev_in[b], c->h2d_stream));
+  // kernels: after the upload, and after the download that last read this set's output buffer
+  ACM_CUDA(cudaStreamWaitEvent(s, c->ev_in[b], 0));
+  if (reused) ACM_CUDA(cudaStreamWaitEvent(s, c->ev_out[b], 0));
+  st = acm_moe_verify(c, layer, c->hx_dev[b], T, c->halpha_dev[b], params, nullptr, c->hout_dev[b], nullptr, nullptr,
+                      nullptr, stats_host ? c->hstats_dev[b] : nullptr, stream);
+  if (st != ACM_OK) return st;
+  ACM_CUDA(cudaEventRecord(c->ev_done[b], s));
+  // download
+  ACM_CUDA(cudaStreamWaitEvent(c->d2h_stream, c->ev_done[b], 0));
+  ACM_CUDA(cudaMemcpyAsync(out_host, c->hout_dev[b], static_cast<size_t>(T) * d.hidden * sizeof(float),
+                           cudaMemcpyDeviceToHost, c->d2h_stream));
+  if (stats_host)
+    ACM_CUDA(cudaMemcpyAsync(stats_host, c->hstats_dev[b], sizeof(acm_block_stats), cudaMemcpyDeviceToHost,
+                             c->d2h_stream));
+  ACM_CUDA(cudaEventRecord(c->ev_out[b], c->d2h_stream));
+  c->host_calls += 1;
+  c->host_h2d += static_cast<size_t>(T) * d.hidden * elt + static_cast<size_t>(T) * sizeof(float);
+  c->host_d2h += static_cast<size_t>(T) * d.hidden * sizeof(float) + (stats_host ? sizeof(acm_block_stats) : 0);
+  return ACM_OK;
+}
+
+acm_status acm_host_synchronize(acm_ctx* c) {
+  if (!c) return ACM_ERR_INVALID;
+  if (!c->d2h_stream) return ACM_OK;
+  ACM_CUDA(cudaStreamSynchronize(c->d2h_stream));
+  return ACM_OK;
+}
+
 
 acm_status acm_set_resident(acm_ctx* c, int layer, const uint32_t* resident_mask, const void* host_gate_up,
                             const void* host_down) {

@@ -218,6 +218,8 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
   const int tid = threadIdx.x;
   const int e0 = blockIdx.x * kRE, t0 = blockIdx.y * kRT;
   griddep_launch_dependents();
+  if (dbg && tid == 0) atomicMax(reinterpret_cast<unsigned long long*>(dbg + 17), static_cast<unsigned long long>(time_ns()));
+  if (dbg && tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) dbg[16] = time_ns();
   griddep_wait();
   if (dbg && tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) dbg[13] = time_ns();
 

@@ -411,3 +411,44 @@ def test_config5_shape_one_layer():
     st, _ = _verify_layer(cfg, 0, ctx, 0, rows=[0, 31, 63])
     assert st["n_activated"] > cfg.top_k
     ctx.close()
+
+
+def test_eligible_but_unchosen_experts_contribute_nothing():
+    """The FFN kernel starts on the ELIGIBLE set before the routes exist.  With few nodes and a large fixed
+    budget most eligible experts are chosen by no node: they must add nothing to the output, and the
+    activated count must still be that of the routes."""
+    cfg = wl.scaled(wl.CONFIGS[3], n_nodes=5)
+    ctx = _ctx(cfg)
+    st, _ = _verify_layer(cfg, 0, ctx, 0, params_kw={"fixed_budget": 96})
+    assert st["n_eligible_pruned"] == 96 and st["n_activated"] <= 5 * cfg.top_k < st["n_eligible_pruned"]
+    ctx.close()
+
+
+def test_host_buffer_call_matches_the_device_call():
+    """acm_moe_verify_host: pinned host x / alpha in, pinned host out back, through the two alternating
+    buffer sets (five calls, so both sets are reused), against the device-pointer call on the same blocks."""
+    cfg = wl.CONFIGS[3]
+    ctx = _ctx(cfg, n_layers=2)
+    depth, p = wl.tree_depths(cfg), wl.commitment_table(cfg)
+    alpha = acm.node_weights(depth, p)
+    alpha_pin = alpha.pin_memory()
+    blocks = []
+    for layer in range(2):
+        w = wl.layer_weights(cfg, layer, DEV)
+        _set_weights(ctx, w, layer)
+        blocks.append(w)
+    calls = [0, 1, 1, 0, 1]
+    xs = [wl.hidden_states(cfg, 10 + i, DEV) for i in range(len(calls))]
+    xs_pin = [x.cpu().pin_memory() for x in xs]
+    outs_pin = [torch.full((cfg.n_nodes, cfg.hidden), float("nan")).pin_memory() for _ in calls]
+    stats_pin = [torch.zeros(12, dtype=torch.int32).pin_memory() for _ in calls]
+    for i, layer in enumerate(calls):
+        ctx.moe_verify_host(layer, xs_pin[i], alpha_pin, outs_pin[i], stats_host=stats_pin[i])
+    ctx.host_synchronize()
+    assert ctx.device_status() == acm.OK
+    for i, layer in enumerate(calls):
+        out, idx, wt, mask, stats = ctx.moe_verify(layer, xs[i], alpha.to(DEV), acm.SelectParams(), want=True)
+        ref = out.double().cpu().numpy()
+        _ffn_check(outs_pin[i].to(DEV), ref, f"host call {i}")
+        assert acm.stats_dict(stats_pin[i]) == acm.stats_dict(stats)
+    ctx.close()
