@@ -2,21 +2,27 @@
 //   y_t = sum_e w_{t,e} * W_down_e ( silu(W_gate_e x_t) * (W_up_e x_t) ),
 // the step whose cost is the number of distinct expert weights touched (Section 1; Section 3.1).
 //
-// bf16 path (sm_100a): one persistent kernel, one CTA per SM, warp-specialised:
-//   warp 0      TMA producer: streams weight tiles (128 rows x 64 K, 128-byte swizzle) and the
-//               matching activation chunk into an 8-stage shared-memory ring
+// bf16 path (sm_100a): one persistent kernel, one CTA per SM, eight specialised warps:
+//   warp 0      weight producer: one TMA copy per operand and stage (32 KB of weights = 128 rows x 128 K
+//               in two 128-byte-swizzled atoms, plus the x chunk of gate/up stages) into a 3-stage ring
 //   warp 1      issues tcgen05.mma (M=128 weight rows, N=node columns, fp32 accumulators in TMEM)
-//   warps 2..5  epilogue: tcgen05.ld, SwiGLU / combine, stores
+//   warps 2..5  epilogue: tcgen05.ld, SwiGLU / combine; only TMEM and shared memory are touched here
+//   warp 6      helper: waits for other CTAs' partial sums and copies them into shared memory ahead of
+//               need; adds the activation chunk to down stages once their expert group is complete
+//   warp 7      publisher: moves staged fragments / activation tiles to global memory (bulk reduce-add,
+//               TMA store), waits for completion, then raises the counter other CTAs wait on
 // The weights are the M operand ("swap-AB"): every activated expert's weights are read from HBM
-// exactly once for all nodes of the block.  Both GEMMs are cut into equal contiguous ranges of
-// (tile, K-chunk) units, one range per CTA, so every SM streams the same number of bytes:
-//   phase 1  tile = 64 gate rows + the 64 matching up rows of one expert, K = hidden;
-//            a tile cut across CTAs is summed through a global fragment buffer by the CTA that
-//            owns its first chunk, which then applies w * silu(g) * u and writes the activation
-//   phase 2  tile = 128 output rows, K = (activated expert, intermediate) concatenated;
-//            partial tiles are accumulated into the output with reductions in L2.
-// Phase 2 reads the activations written by other CTAs in phase 1; per-expert completion counters
-// order the two.  Every wait is bounded; on expiry the kernel raises a status and drains.
+// exactly once for all nodes of the block.  Work plan of a launch (make_plan):
+//   gate/up  tile = 64 gate rows + the 64 matching up rows of one expert, K = hidden.  The
+//            n_tiles mod grid leftover tiles come first, cut into equal contiguous ranges of (tile,
+//            K-chunk) units over all CTAs; the CTA that owns a tile's last chunk receives the others'
+//            partial sums (added into its pre-zeroed global buffer), applies w * silu(g) * u and
+//            stores the activation tile.  Then whole tiles, one per CTA and round.
+//   down     tile = 128 output rows, K = (activated expert, intermediate) concatenated, cut evenly;
+//            experts complete early first.  Partial tiles are added to the output with fp32
+//            reductions in L2 (the caller zeroes the output).
+// The down phase reads activations written by other CTAs in the gate/up phase; two group counters
+// order them.  Every wait is bounded; on expiry the kernel raises a status and drains.
 //
 // f32 path: plain FMA kernels (the fp32 toy configuration is a few MFLOP).
 #include <cuda_bf16.h>

@@ -1,7 +1,7 @@
 // Stages 1-3 of the verifier-side MoE layer: router logits (Section 3.1), softmax and natural
 // top-k (Eq. 1), commitment-weighted demand (Eq. 4), anchors (Eq. 5), self-sized eligible set
 // (Eq. 6), residency-aware pruning (Eq. 7) and restricted top-k routing (Eq. 2), plus the
-// activated-expert work lists the FFN kernel consumes.
+// routing inputs the FFN kernel consumes (activated-expert mask, combine-weight table).
 //
 // Everything that decides a set member, a count or an index is binary32 in a fixed order
 // (explicit round-to-nearest intrinsics, so the compiler can neither contract nor reorder):
