@@ -222,10 +222,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
     p.sel_epoch = early_epoch;
   }
   p.out = out; p.status = c->ws.status;
-  // Early start: the routing kernel still holds a few SMs when this kernel's CTAs are placed, and an SM
-  // changes hands slowly; leave those SMs out so that every CTA starts at once.
-  p.grid = early_epoch != 0 ? c->sm_count - route_ctas(T) : c->sm_count;
-  if (p.grid < 1) p.grid = 1;
+  p.grid = c->sm_count;
   p.phase_mask = 3;
   p.trace = c->trace;
   p.pdl = false;
@@ -247,6 +244,10 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   }
   // dependent launch only straight after the select/route kernel (no event, memset or copy between)
   p.pdl = pdl_ok && c->pdl && !e0 && (!c->trace || c->trace_light) && !c->split_phases;
+  // Straight after the routing kernel: the few SMs it ran on (or still holds, in an early start) take
+  // microseconds longer to accept a CTA of this kernel -- an SM changes hands slowly when the shared-memory
+  // split changes -- and one late CTA delays every CTA that exchanges fragments with it.  Leave them out.
+  if (pdl_ok && c->sm_count > route_ctas(T)) p.grid = c->sm_count - route_ctas(T);
   ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
   c->launches += 1;
   if (e1) ACM_CUDA(cudaEventRecord(e1, s));

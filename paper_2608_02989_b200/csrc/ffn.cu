@@ -59,6 +59,56 @@ constexpr int kFragBytes = kTileM * kMaxNodes * 4;       // contributor fragment
 constexpr int kFragFloats = kTileM * kMaxNodes;
 constexpr unsigned long long kTimeoutNs = 1000ull * 1000ull * 1000ull;
 
+// Division by a launch constant through a precomputed 64-bit reciprocal (exact for n < 2^32): the
+// schedules below are walked by ONE thread per role, for which a hardware-less integer division is
+// a chain of dozens of dependent instructions.
+struct FastDiv {
+  unsigned long long M;   // ceil(2^64 / d) for d >= 2
+  unsigned d;
+};
+inline FastDiv make_fastdiv(unsigned d) {
+  FastDiv f;
+  f.d = d;
+  f.M = d > 1 ? 0xffffffffffffffffull / d + 1ull : 0ull;
+  return f;
+}
+// a divisor only known on the device (used a handful of times): M = 0 means "divide the plain way"
+__device__ __forceinline__ FastDiv plain_div(unsigned d) {
+  FastDiv f;
+  f.d = d;
+  f.M = 0ull;
+  return f;
+}
+__device__ __forceinline__ unsigned fdiv(unsigned n, const FastDiv& f) {
+  return f.M == 0ull ? (f.d == 1 ? n : n / f.d) : static_cast<unsigned>(__umul64hi(static_cast<unsigned long long>(n), f.M));
+}
+
+// The stream of one launch is cut into up to four segments, executed in this order by every CTA.
+// A gate/up tile (64 gate + 64 up rows over the whole hidden dimension) needs the complete sum before
+// its activation can be formed, so wherever possible a tile is given whole to one CTA:
+//   with at least one tile per CTA:
+//     1. the n_tiles mod G tiles that do not fill a round, cut evenly over all CTAs (their
+//        cross-CTA fragment exchange then hides behind the next segment)
+//     2. whole tiles, one per CTA and round
+//     3. down projection of the experts that were complete before the last round
+//     4. down projection of the rest -- by then their activations have been stored
+//   with fewer tiles than CTAs: gate/up of the first half of the experts, gate/up of the second
+//   half (both cut evenly), then down of the first half, down of the second half.
+// Down-projection work is linear in K and is always cut evenly.
+struct Segment {
+  int phase;      // 1 = gate/up, 2 = down
+  int whole;      // gate/up only: 1 = whole tiles dealt round-robin, 0 = tiles cut evenly over the CTAs
+  int t0, nt;     // gate/up: first tile and number of tiles (tile = slot * tiles_per_expert + sub-tile)
+  int a0, a1;     // down: activated-expert slots [a0, a1)
+  int p1_index;   // gate/up: which fragment buffer a cut segment uses; down: expert group it waits for
+  FastDiv chunks; // K-chunks per tile: the per-tile constant for gate/up, (a1 - a0) * chunks per expert for down
+};
+struct Plan {
+  Segment seg[4];
+  int n_seg;
+  int a_split;    // experts [0, a_split) form group 0 (complete early), the rest group 1
+};
+
 struct __align__(8) Barriers {
   unsigned long long full[kStages];
   unsigned long long empty[kStages];
@@ -77,6 +127,7 @@ struct __align__(8) Barriers {
   int32_t entry[kMaxSlots];     // this launch's work list: make_entry(source, index) of every activated slot
   int32_t expert[kMaxSlots];    // routed expert id of the slot (-1: shared expert)
   uint32_t sel_half[2 * kMaskWords];   // early start: the eligible mask in 16-bit pieces
+  Plan plan;                    // this launch's work plan
 };
 
 constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + kOutStageBytes + kFragBytes + 2 * kHStageBytes + sizeof(Barriers);
@@ -97,13 +148,17 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// With the suspend-time hint the hardware parks the thread until the phase completes (or the hint
+// runs out) instead of returning at once: a role that polls in a tight loop takes issue slots and
+// shared-memory bandwidth from the single-thread roles (producer, MMA issuer) it waits for.
+constexpr uint32_t kSuspendHintNs = 100000u;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}\n"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
   return ok != 0;
 }
 // Bounded wait.  Returns false (after raising the status once) if the limit ran out or the CTA
@@ -254,27 +309,28 @@ __device__ __forceinline__ uint32_t umma_idesc(int n) {
 
 // Equal contiguous ranges of (tile, K-chunk) units: CTA c owns [c*U/G, (c+1)*U/G).
 struct Sched {
-  unsigned u, u_end;   // 32-bit on purpose: one thread per role walks this, and 64-bit division costs it microseconds
+  unsigned u, u_end;   // 32-bit on purpose (the launcher checks that the products fit)
+  FastDiv kcd;
   int kc;
   int rr_next, rr_end, rr_stride;   // whole tiles dealt round-robin (rr_stride > 0) instead of a cut range
   // equal contiguous ranges of (tile, K-chunk) units: CTA c owns [c*U/G, (c+1)*U/G)
   // (the launcher checks that tiles * chunks_per_tile * grid fits in 32 bits)
-  __device__ Sched(int cta, int grid, int tiles, int chunks_per_tile)
-      : kc(chunks_per_tile), rr_next(0), rr_end(0), rr_stride(0) {
-    const unsigned total = static_cast<unsigned>(tiles) * static_cast<unsigned>(chunks_per_tile);
-    u = total * static_cast<unsigned>(cta) / static_cast<unsigned>(grid);
-    u_end = total * static_cast<unsigned>(cta + 1) / static_cast<unsigned>(grid);
+  __device__ Sched(int cta, const FastDiv& grid, int tiles, const FastDiv& chunks_per_tile)
+      : kcd(chunks_per_tile), kc(static_cast<int>(chunks_per_tile.d)), rr_next(0), rr_end(0), rr_stride(0) {
+    const unsigned total = static_cast<unsigned>(tiles) * chunks_per_tile.d;
+    u = fdiv(total * static_cast<unsigned>(cta), grid);
+    u_end = fdiv(total * static_cast<unsigned>(cta + 1), grid);
   }
   // whole tiles: CTA c owns tiles c, c+G, c+2G, ... < tiles (tiles is a multiple of G here)
-  __device__ static Sched whole_tiles(int cta, int grid, int tiles, int chunks_per_tile) {
-    Sched s(0, 1, 0, chunks_per_tile);
+  __device__ static Sched whole_tiles(int cta, const FastDiv& grid, int tiles, const FastDiv& chunks_per_tile) {
+    Sched s(0, grid, 0, chunks_per_tile);
     s.rr_next = cta;
     s.rr_end = tiles;
-    s.rr_stride = grid;
+    s.rr_stride = static_cast<int>(grid.d);
     return s;
   }
   __device__ long long stages() const {
-    if (rr_stride > 0) return rr_next < rr_end ? static_cast<long long>((rr_end - rr_next + rr_stride - 1) / rr_stride) * kc : 0;
+    if (rr_stride > 0) return rr_next < rr_end ? static_cast<long long>((rr_end - rr_next + rr_stride - 1) / rr_stride) * kc : 0;   // (helper warp only)
     return static_cast<long long>(u_end - u);
   }
   __device__ bool next(int& tile, int& k0, int& k1) {
@@ -287,7 +343,7 @@ struct Sched {
       return true;
     }
     if (u >= u_end) return false;
-    tile = static_cast<int>(u / static_cast<unsigned>(kc));
+    tile = static_cast<int>(fdiv(u, kcd));
     k0 = static_cast<int>(u - static_cast<unsigned>(tile) * static_cast<unsigned>(kc));
     const int rem = static_cast<int>(u_end - u);
     k1 = rem < kc - k0 ? k0 + rem : kc;
@@ -301,6 +357,7 @@ struct Sched {
 
 struct FfnArgs {
   int T, H, I, n_pad;
+  FastDiv d_grid, d_kc1, d_tpe, d_kpe;   // reciprocals of the grid size and of the per-tile / per-expert chunk counts
   const uint32_t* act_mask;
   const uint32_t* resident;
   int li, n_shared;
@@ -323,32 +380,9 @@ __device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMa
   return src == kSrcRouted ? routed : src == kSrcShared ? shared : staged;
 }
 
-// The stream of one launch is cut into up to four segments, executed in this order by every CTA.
-// A gate/up tile (64 gate + 64 up rows over the whole hidden dimension) needs the complete sum before
-// its activation can be formed, so wherever possible a tile is given whole to one CTA:
-//   with at least one tile per CTA:
-//     1. the n_tiles mod G tiles that do not fill a round, cut evenly over all CTAs (their
-//        cross-CTA fragment exchange then hides behind the next segment)
-//     2. whole tiles, one per CTA and round
-//     3. down projection of the experts that were complete before the last round
-//     4. down projection of the rest -- by then their activations have been stored
-//   with fewer tiles than CTAs: gate/up of the first half of the experts, gate/up of the second
-//   half (both cut evenly), then down of the first half, down of the second half.
-// Down-projection work is linear in K and is always cut evenly.
-struct Segment {
-  int phase;      // 1 = gate/up, 2 = down
-  int whole;      // gate/up only: 1 = whole tiles dealt round-robin, 0 = tiles cut evenly over the CTAs
-  int t0, nt;     // gate/up: first tile and number of tiles (tile = slot * tiles_per_expert + sub-tile)
-  int a0, a1;     // down: activated-expert slots [a0, a1)
-  int p1_index;   // gate/up: which fragment buffer a cut segment uses; down: expert group it waits for
-};
-struct Plan {
-  Segment seg[4];
-  int n_seg;
-  int a_split;    // experts [0, a_split) form group 0 (complete early), the rest group 1
-};
-__device__ __forceinline__ Plan make_plan(int n_act, int tpe, int grid, int phase_mask) {
-  Plan pl;
+// (filled in place, in shared memory: a private copy indexed at run time would live in local memory,
+// whose first touch costs every role a trip to DRAM at the start of the kernel)
+__device__ __forceinline__ void make_plan(Plan& pl, int n_act, int tpe, int grid, int phase_mask, const FastDiv& d_kc1, int kpe) {
   pl.n_seg = 0;
   const int n_t = n_act * tpe;
   const int rounds = n_t / grid, rem = n_t % grid;
@@ -357,24 +391,23 @@ __device__ __forceinline__ Plan make_plan(int n_act, int tpe, int grid, int phas
     const int nA = (n_act + 1) / 2;
     pl.a_split = nA;
     if (phase_mask & 1) {
-      if (nA > 0) pl.seg[n++] = Segment{1, 0, 0, nA * tpe, 0, 0, 0};
-      if (n_act > nA) pl.seg[n++] = Segment{1, 0, nA * tpe, (n_act - nA) * tpe, 0, 0, 1};
+      if (nA > 0) pl.seg[n++] = Segment{1, 0, 0, nA * tpe, 0, 0, 0, d_kc1};
+      if (n_act > nA) pl.seg[n++] = Segment{1, 0, nA * tpe, (n_act - nA) * tpe, 0, 0, 1, d_kc1};
     }
   } else {
     pl.a_split = (rem + (rounds - 1) * grid) / tpe;
     if (phase_mask & 1) {
-      if (rem > 0) pl.seg[n++] = Segment{1, 0, 0, rem, 0, 0, 0};
-      pl.seg[n++] = Segment{1, 1, rem, rounds * grid, 0, 0, 1};
+      if (rem > 0) pl.seg[n++] = Segment{1, 0, 0, rem, 0, 0, 0, d_kc1};
+      pl.seg[n++] = Segment{1, 1, rem, rounds * grid, 0, 0, 1, d_kc1};
     }
   }
   if (phase_mask & 2) {
-    if (pl.a_split > 0) pl.seg[n++] = Segment{2, 0, 0, 0, 0, pl.a_split, 0};
-    if (n_act > pl.a_split) pl.seg[n++] = Segment{2, 0, 0, 0, pl.a_split, n_act, 1};
+    if (pl.a_split > 0) pl.seg[n++] = Segment{2, 0, 0, 0, 0, pl.a_split, 0, plain_div(static_cast<unsigned>(pl.a_split * kpe))};
+    if (n_act > pl.a_split) pl.seg[n++] = Segment{2, 0, 0, 0, pl.a_split, n_act, 1, plain_div(static_cast<unsigned>((n_act - pl.a_split) * kpe))};
   }
   pl.n_seg = n;
-  return pl;
 }
-__device__ __forceinline__ Sched p1_sched(const Segment& sg, int cta, int grid, int kc1) {
+__device__ __forceinline__ Sched p1_sched(const Segment& sg, int cta, const FastDiv& grid, const FastDiv& kc1) {
   return sg.whole ? Sched::whole_tiles(cta, grid, sg.nt, kc1) : Sched(cta, grid, sg.nt, kc1);
 }
 
@@ -434,6 +467,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   // Everything above touched only this CTA's own resources; global memory written by the kernels
   // before this one is read only from here on.  Early start: wait for the eligible set only.
   const bool early = p.sel_flag != nullptr;
+  if (threadIdx.x == 0) ACM_TRACE(29);
   if (early) {
     // eight tagged words (16 mask bits under the 16-bit tag of this call), each polled by its own thread
     if (threadIdx.x < 2 * kMaskWords) {
@@ -456,6 +490,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   } else {
     griddep_wait();
   }
+  if (threadIdx.x == 0) ACM_TRACE(30);
   // The work list of this launch: slot a = the a-th activated expert of this list in ascending id
   // order (list 0: the resident ones, then the shared experts; list 1: the non-resident ones, which
   // the host has copied into staging slot a).
@@ -475,15 +510,13 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   const int h_tiles = p.H / kTileM;  // output tiles of the down phase
   const uint32_t b_atom_bytes = static_cast<uint32_t>(p.n_pad) * kBK * 2;   // one atom of the activation chunk
   const uint32_t b_bytes = kAtoms * b_atom_bytes;
-  const Plan plan = make_plan(n_act, tpe, G, p.phase_mask);
-  const Segment* seg = plan.seg;
-  const int n_seg = plan.n_seg;
-  const int a_split = plan.a_split;
+  if (threadIdx.x == kThreads - 1) make_plan(bars->plan, n_act, tpe, G, p.phase_mask, p.d_kc1, kpe);
   int32_t* s_entry = bars->entry;
   if (threadIdx.x < kMaxExperts) {
     const int e = threadIdx.x, wd = e >> 5;
-    if ((am[wd] >> (e & 31)) & 1u) {
-      int slot = __popc(am[wd] & ((1u << (e & 31)) - 1u));
+    const uint32_t mine = wd == 0 ? am[0] : wd == 1 ? am[1] : wd == 2 ? am[2] : am[3];
+    if ((mine >> (e & 31)) & 1u) {
+      int slot = __popc(mine & ((1u << (e & 31)) - 1u));
 #pragma unroll
       for (int v = 0; v < kMaskWords; ++v) slot += v < wd ? __popc(am[v]) : 0;
       s_entry[slot] = p.li == 0 ? make_entry(kSrcRouted, e) : make_entry(kSrcStaged, slot);
@@ -494,9 +527,13 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     s_entry[n_routed + i] = make_entry(kSrcShared, i);
     bars->expert[n_routed + i] = -1;
   }
+  if (threadIdx.x == 0) ACM_TRACE(31);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  const Segment* seg = bars->plan.seg;
+  const int n_seg = bars->plan.n_seg;
+  const int a_split = bars->plan.a_split;
   const uint32_t tmem_base = bars->tmem_base;
   if (threadIdx.x == 0) ACM_TRACE(0);
 
@@ -508,23 +545,20 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     // it.  The loop is kept to a few instructions per stage: one thread pays every one of them.
     if (lane == 0) {
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
-      ACM_TRACE(3);
       uint32_t s = 0, par = 0, n_armed = 0;
       bool ok = true, traced_first = false;
       for (int si = 0; si < n_seg && ok; ++si) {
         const Segment sg = seg[si];
-        const int n_exp = sg.a1 - sg.a0;
         if (sg.phase == 1) {
-          Sched sc = p1_sched(sg, cta, G, kc1);
+          Sched sc = p1_sched(sg, cta, p.d_grid, p.d_kc1);
           int tile, k0, k1;
           while (ok && sc.next(tile, k0, k1)) {
-            const int32_t ent = s_entry[(sg.t0 + tile) / tpe];
-            const int r0 = ((sg.t0 + tile) % tpe) * 64, eidx = entry_idx(ent);
+            const int a_of = static_cast<int>(fdiv(static_cast<unsigned>(sg.t0 + tile), p.d_tpe));
+            const int32_t ent = s_entry[a_of];
+            const int r0 = (sg.t0 + tile - a_of * tpe) * 64, eidx = entry_idx(ent);
             const CUtensorMap* gu = pick_map(entry_src(ent), &maps.gate_up, &maps.shared_gate_up, &maps.staged_gate_up);
             for (int kc = k0; kc < k1; ++kc) {
-              if (!traced_first) ACM_TRACE(4);
               if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
-              if (!traced_first) ACM_TRACE(16);
               const uint32_t full = smem_u32(&bars->full[s]);
               const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
               mbar_expect_tx(full, kABytes + b_bytes);
@@ -537,10 +571,11 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           }
           ACM_TRACE(sg.p1_index == 0 ? 13 : 2);
         } else {
-          Sched sc(cta, G, h_tiles, n_exp * kpe);
+          Sched sc(cta, p.d_grid, h_tiles, sg.chunks);
           int ht, k0, k1;
           while (ok && sc.next(ht, k0, k1)) {
-            int a = sg.a0 + k0 / kpe, ic = k0 % kpe;
+            const int q0 = static_cast<int>(fdiv(static_cast<unsigned>(k0), p.d_kpe));
+            int a = sg.a0 + q0, ic = k0 - q0 * kpe;
             int32_t ent = s_entry[a];
             const CUtensorMap* dn = pick_map(entry_src(ent), &maps.down, &maps.shared_down, &maps.staged_down);
             int eidx = entry_idx(ent);
@@ -578,8 +613,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       unsigned long long acc_f[2] = {0, 0};
       for (int si = 0; si < n_seg && ok; ++si) {
         const Segment sg = seg[si];
-        const int n_exp = sg.a1 - sg.a0;
-        Sched sc = sg.phase == 1 ? p1_sched(sg, cta, G, kc1) : Sched(cta, G, h_tiles, n_exp * kpe);
+        Sched sc = sg.phase == 1 ? p1_sched(sg, cta, p.d_grid, p.d_kc1) : Sched(cta, p.d_grid, h_tiles, sg.chunks);
         int tile, k0, k1;
         while (ok && sc.next(tile, k0, k1)) {
           const uint32_t b = f % kAcc;
@@ -630,15 +664,14 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       const Segment sg = seg[si];
       const int n_exp = sg.a1 - sg.a0;
       if (sg.phase == 1) {
-        hidx += static_cast<uint32_t>(p1_sched(sg, cta, G, kc1).stages());
+        hidx += static_cast<uint32_t>(p1_sched(sg, cta, p.d_grid, p.d_kc1).stages());
         hs = hidx % kStages;
         if (sg.whole) continue;          // whole tiles: nothing to exchange
-        const long long tiles = sg.nt;
-        const long long U1 = tiles * kc1;
-        const long long ub = U1 * cta / G, ue = U1 * (cta + 1) / G;
+        const unsigned U1 = static_cast<unsigned>(sg.nt) * kc1;
+        const unsigned ub = fdiv(U1 * cta, p.d_grid), ue = fdiv(U1 * (cta + 1), p.d_grid);
         if (ue <= ub) continue;
-        const long long last_tile = (ue - 1) / kc1;
-        const long long tile_end = (last_tile + 1) * kc1;
+        const unsigned last_tile = fdiv(ue - 1, p.d_kc1);
+        const unsigned tile_end = (last_tile + 1) * kc1;
         const bool head = (last_tile * kc1 >= ub) && (ue < tile_end);   // starts at chunk 0, ends before the tile does
         if (!head) continue;
         if (frag_uses > 0) {   // the buffer still holds the previous segment's sum until the epilogue has read it
@@ -650,7 +683,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         const int n_el = p.n_pad * kTileM;
         int n_contrib = 0;
         for (int c2 = cta + 1; c2 < G; ++c2) {
-          const long long b2 = U1 * c2 / G, e2 = U1 * (c2 + 1) / G;
+          const unsigned b2 = fdiv(U1 * c2, p.d_grid), e2 = fdiv(U1 * (c2 + 1), p.d_grid);
           if (b2 >= tile_end) break;
           if (e2 > b2) ++n_contrib;
         }
@@ -683,11 +716,12 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         bool good = true;
         if (lane == 0) {
           const uint64_t pol_x = policy_evict_last();
-          Sched sc(cta, G, h_tiles, n_exp * kpe);
+          Sched sc(cta, p.d_grid, h_tiles, sg.chunks);
           int ht, k0, k1;
           bool polled = false;
           while (good && sc.next(ht, k0, k1)) {
-            int a = sg.a0 + k0 / kpe, ic = k0 % kpe;
+            const int q0 = static_cast<int>(fdiv(static_cast<unsigned>(k0), p.d_kpe));
+            int a = sg.a0 + q0, ic = k0 - q0 * kpe;
             for (int kc = k0; kc < k1; ++kc) {
               if (!polled) {
                 if (!(good = flag_wait_ge(&p.ready[sg.p1_index], n_exp * tpe, abort_flag, p.status))) break;   // n_exp = size of the group
@@ -732,7 +766,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         if (sg.phase != 1) continue;
         float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * kFragFloats;
         int32_t* frag_flag = p.frag_flag + sg.p1_index * G;
-        Sched sc = p1_sched(sg, cta, G, kc1);
+        Sched sc = p1_sched(sg, cta, p.d_grid, p.d_kc1);
         int tile, k0, k1;
         while (ok && sc.next(tile, k0, k1)) {
           if (k0 > 0) {
@@ -741,10 +775,10 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             // All CTAs that hold a tail part of this tile add into ONE global buffer, that of the CTA
             // which owns the tile's first chunks and will finish it.  The buffers are zero between
             // launches (the finishing CTA clears its own after reading), so nobody waits for anybody.
-            const long long U1 = static_cast<long long>(sg.nt) * kc1;
-            const long long tile_begin = static_cast<long long>(tile) * kc1;
+            const unsigned U1 = static_cast<unsigned>(sg.nt) * kc1;            // (fits 32 bits: see the launcher)
+            const unsigned tile_begin = static_cast<unsigned>(tile) * kc1;
             int c_head = cta - 1;
-            while (c_head > 0 && U1 * c_head / G > tile_begin) --c_head;       // owner of the tile's first chunk
+            while (c_head > 0 && fdiv(U1 * c_head, p.d_grid) > tile_begin) --c_head;       // owner of the tile's first chunk
             asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
                          ::"l"(frag + static_cast<size_t>(c_head) * kFragFloats), "r"(smem_u32(ostage)), "r"(bytes) : "memory");
             bulk_commit();
@@ -755,7 +789,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           } else {
             const uint32_t hb = fin_n & 1u;
             if (!(ok = mbar_wait(smem_u32(&bars->hst_full[hb]), (fin_n >> 1) & 1u, abort_flag, p.status))) break;
-            const int a = (sg.t0 + tile) / tpe, ti = (sg.t0 + tile) % tpe;
+            const int a = static_cast<int>(fdiv(static_cast<unsigned>(sg.t0 + tile), p.d_tpe)), ti = sg.t0 + tile - a * tpe;
             asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
                          ::"l"(&hs_map), "r"(0), "r"(0), "r"(ti), "r"(a), "r"(smem_u32(hstage + hb * kHStageBytes)) : "memory");
             bulk_commit();
@@ -763,6 +797,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             red_release_add(&p.ready[a >= a_split ? 1 : 0], 1);
             mbar_arrive(smem_u32(&bars->hst_free[hb]));
             ++fin_n;
+            if (fin_n == 1) ACM_TRACE(16);
             ACM_TRACE(28);
           }
         }
@@ -795,9 +830,8 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     };
     for (int si = 0; si < n_seg && ok; ++si) {
       const Segment sg = seg[si];
-      const int n_exp = sg.a1 - sg.a0;
       if (sg.phase == 1) {
-        Sched sc = p1_sched(sg, cta, G, kc1);
+        Sched sc = p1_sched(sg, cta, p.d_grid, p.d_kc1);
         int tile, k0, k1;
         while (sc.next(tile, k0, k1)) {
           const uint32_t b = f % kAcc;
@@ -818,7 +852,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             ++ost_uses;
             continue;
           }
-          const int a = (sg.t0 + tile) / tpe;
+          const int a = static_cast<int>(fdiv(static_cast<unsigned>(sg.t0 + tile), p.d_tpe));
           if (!waited) {          // the combine weights are the routing kernel's last output
             griddep_wait();
             waited = true;
@@ -899,7 +933,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         }
         if (row == 0) ACM_TRACE(10);
       } else {
-        Sched sc(cta, G, h_tiles, n_exp * kpe);
+        Sched sc(cta, p.d_grid, h_tiles, sg.chunks);
         int ht, k0, k1;
         while (sc.next(ht, k0, k1)) {
           const uint32_t b = f % kAcc;
@@ -1007,6 +1041,13 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
     if ((u1 > u2 ? u1 : u2) * (static_cast<unsigned long long>(L.grid) + 1) >= (1ull << 32)) return cudaErrorInvalidValue;
   }
   FfnArgs a;
+  {
+    const int tpe = L.I / 64;
+    a.d_grid = make_fastdiv(static_cast<unsigned>(L.grid));
+    a.d_kc1 = make_fastdiv(static_cast<unsigned>(L.H / (kBK * kAtoms)));
+    a.d_tpe = make_fastdiv(static_cast<unsigned>(tpe));
+    a.d_kpe = make_fastdiv(static_cast<unsigned>((tpe + kAtoms - 1) / kAtoms));
+  }
   a.T = L.T; a.H = L.H; a.I = L.I; a.n_pad = L.n_pad;
   a.act_mask = L.act_mask; a.resident = L.resident; a.li = L.li; a.n_shared = L.n_shared; a.wtab = L.wtab;
   a.stats = L.stats; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
