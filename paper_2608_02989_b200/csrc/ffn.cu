@@ -103,8 +103,20 @@ struct Segment {
   int p1_index;   // gate/up: which fragment buffer a cut segment uses; down: expert group it waits for
   FastDiv chunks; // K-chunks per tile: the per-tile constant for gate/up, (a1 - a0) * chunks per expert for down
 };
+// This CTA's share of one segment of the plan.  Cut segments: equal contiguous ranges of (tile,
+// K-chunk) units, CTA c owns [c*U/G, (c+1)*U/G); whole-tile segments: tiles c, c+G, c+2G, ...
+// The divisions are done once per launch, by four lanes in parallel (fill_ranges), and every role
+// then walks its share with additions only: each role is a single thread that runs this code alone.
+struct SegRange {
+  unsigned u, u_end;     // cut: the CTA's unit range; whole: first tile and tile count of the segment
+  int tile0, k00;        // cut: tile and chunk of unit u
+  int kc;                // chunks per tile
+  int stride;            // whole: the grid size (tile step); 0 for a cut segment
+  unsigned n_stages;     // pipeline stages this CTA runs in the segment
+};
 struct Plan {
   Segment seg[4];
+  SegRange range[4];   // this CTA's share of each segment
   int n_seg;
   int a_split;    // experts [0, a_split) form group 0 (complete early), the rest group 1
 };
@@ -307,47 +319,27 @@ __device__ __forceinline__ uint32_t umma_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
 }
 
-// Equal contiguous ranges of (tile, K-chunk) units: CTA c owns [c*U/G, (c+1)*U/G).
 struct Sched {
-  unsigned u, u_end;   // 32-bit on purpose (the launcher checks that the products fit)
-  FastDiv kcd;
-  int kc;
-  int rr_next, rr_end, rr_stride;   // whole tiles dealt round-robin (rr_stride > 0) instead of a cut range
-  // equal contiguous ranges of (tile, K-chunk) units: CTA c owns [c*U/G, (c+1)*U/G)
-  // (the launcher checks that tiles * chunks_per_tile * grid fits in 32 bits)
-  __device__ Sched(int cta, const FastDiv& grid, int tiles, const FastDiv& chunks_per_tile)
-      : kcd(chunks_per_tile), kc(static_cast<int>(chunks_per_tile.d)), rr_next(0), rr_end(0), rr_stride(0) {
-    const unsigned total = static_cast<unsigned>(tiles) * chunks_per_tile.d;
-    u = fdiv(total * static_cast<unsigned>(cta), grid);
-    u_end = fdiv(total * static_cast<unsigned>(cta + 1), grid);
-  }
-  // whole tiles: CTA c owns tiles c, c+G, c+2G, ... < tiles (tiles is a multiple of G here)
-  __device__ static Sched whole_tiles(int cta, const FastDiv& grid, int tiles, const FastDiv& chunks_per_tile) {
-    Sched s(0, grid, 0, chunks_per_tile);
-    s.rr_next = cta;
-    s.rr_end = tiles;
-    s.rr_stride = static_cast<int>(grid.d);
-    return s;
-  }
-  __device__ long long stages() const {
-    if (rr_stride > 0) return rr_next < rr_end ? static_cast<long long>((rr_end - rr_next + rr_stride - 1) / rr_stride) * kc : 0;   // (helper warp only)
-    return static_cast<long long>(u_end - u);
-  }
-  __device__ bool next(int& tile, int& k0, int& k1) {
-    if (rr_stride > 0) {
-      if (rr_next >= rr_end) return false;
-      tile = rr_next;
+  unsigned u, u_end;
+  int tile, k0n, kc, stride;
+  __device__ explicit Sched(const SegRange& r) : u(r.u), u_end(r.u_end), tile(r.tile0), k0n(r.k00), kc(r.kc), stride(r.stride) {}
+  __device__ bool next(int& t, int& k0, int& k1) {
+    if (stride > 0) {            // whole tiles: u counts tiles
+      if (u >= u_end) return false;
+      t = static_cast<int>(u);
       k0 = 0;
       k1 = kc;
-      rr_next += rr_stride;
+      u += static_cast<unsigned>(stride);
       return true;
     }
     if (u >= u_end) return false;
-    tile = static_cast<int>(fdiv(u, kcd));
-    k0 = static_cast<int>(u - static_cast<unsigned>(tile) * static_cast<unsigned>(kc));
+    t = tile;
+    k0 = k0n;
     const int rem = static_cast<int>(u_end - u);
     k1 = rem < kc - k0 ? k0 + rem : kc;
     u += static_cast<unsigned>(k1 - k0);
+    ++tile;
+    k0n = 0;
     return true;
   }
 };
@@ -382,10 +374,11 @@ __device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMa
 
 // (filled in place, in shared memory: a private copy indexed at run time would live in local memory,
 // whose first touch costs every role a trip to DRAM at the start of the kernel)
-__device__ __forceinline__ void make_plan(Plan& pl, int n_act, int tpe, int grid, int phase_mask, const FastDiv& d_kc1, int kpe) {
+__device__ __forceinline__ void make_plan(Plan& pl, int n_act, int tpe, int grid, int phase_mask, const FastDiv& d_kc1, int kpe,
+                                          const FastDiv& d_grid, const FastDiv& d_tpe) {
   pl.n_seg = 0;
   const int n_t = n_act * tpe;
-  const int rounds = n_t / grid, rem = n_t % grid;
+  const int rounds = static_cast<int>(fdiv(static_cast<unsigned>(n_t), d_grid)), rem = n_t - rounds * grid;
   int n = 0;
   if (rounds == 0) {
     const int nA = (n_act + 1) / 2;
@@ -395,7 +388,7 @@ __device__ __forceinline__ void make_plan(Plan& pl, int n_act, int tpe, int grid
       if (n_act > nA) pl.seg[n++] = Segment{1, 0, nA * tpe, (n_act - nA) * tpe, 0, 0, 1, d_kc1};
     }
   } else {
-    pl.a_split = (rem + (rounds - 1) * grid) / tpe;
+    pl.a_split = static_cast<int>(fdiv(static_cast<unsigned>(rem + (rounds - 1) * grid), d_tpe));
     if (phase_mask & 1) {
       if (rem > 0) pl.seg[n++] = Segment{1, 0, 0, rem, 0, 0, 0, d_kc1};
       pl.seg[n++] = Segment{1, 1, rem, rounds * grid, 0, 0, 1, d_kc1};
@@ -407,8 +400,28 @@ __device__ __forceinline__ void make_plan(Plan& pl, int n_act, int tpe, int grid
   }
   pl.n_seg = n;
 }
-__device__ __forceinline__ Sched p1_sched(const Segment& sg, int cta, const FastDiv& grid, const FastDiv& kc1) {
-  return sg.whole ? Sched::whole_tiles(cta, grid, sg.nt, kc1) : Sched(cta, grid, sg.nt, kc1);
+
+// Range of segment `si` for CTA `cta` (see SegRange).  (tiles * chunks * grid fits 32 bits: launcher.)
+__device__ __forceinline__ SegRange make_range(const Segment& sg, int cta, const FastDiv& d_grid, int h_tiles) {
+  SegRange r;
+  r.kc = static_cast<int>(sg.chunks.d);
+  if (sg.phase == 1 && sg.whole) {
+    r.u = static_cast<unsigned>(cta);
+    r.u_end = static_cast<unsigned>(sg.nt);
+    r.tile0 = 0; r.k00 = 0;
+    r.stride = static_cast<int>(d_grid.d);
+    r.n_stages = cta < sg.nt ? fdiv(static_cast<unsigned>(sg.nt - cta) + d_grid.d - 1u, d_grid) * sg.chunks.d : 0u;
+    return r;
+  }
+  const unsigned tiles = sg.phase == 1 ? static_cast<unsigned>(sg.nt) : static_cast<unsigned>(h_tiles);
+  const unsigned total = tiles * sg.chunks.d;
+  r.u = fdiv(total * static_cast<unsigned>(cta), d_grid);
+  r.u_end = fdiv(total * static_cast<unsigned>(cta + 1), d_grid);
+  r.tile0 = static_cast<int>(fdiv(r.u, sg.chunks));
+  r.k00 = static_cast<int>(r.u - static_cast<unsigned>(r.tile0) * sg.chunks.d);
+  r.stride = 0;
+  r.n_stages = r.u_end - r.u;
+  return r;
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -510,7 +523,11 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   const int h_tiles = p.H / kTileM;  // output tiles of the down phase
   const uint32_t b_atom_bytes = static_cast<uint32_t>(p.n_pad) * kBK * 2;   // one atom of the activation chunk
   const uint32_t b_bytes = kAtoms * b_atom_bytes;
-  if (threadIdx.x == kThreads - 1) make_plan(bars->plan, n_act, tpe, G, p.phase_mask, p.d_kc1, kpe);
+  if (warp == kThreads / 32 - 1) {      // the publisher warp has nothing else to do yet
+    if (lane == 31) make_plan(bars->plan, n_act, tpe, G, p.phase_mask, p.d_kc1, kpe, p.d_grid, p.d_tpe);
+    __syncwarp();
+    if (lane < bars->plan.n_seg) bars->plan.range[lane] = make_range(bars->plan.seg[lane], cta, p.d_grid, h_tiles);
+  }
   int32_t* s_entry = bars->entry;
   if (threadIdx.x < kMaxExperts) {
     const int e = threadIdx.x, wd = e >> 5;
@@ -550,7 +567,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       for (int si = 0; si < n_seg && ok; ++si) {
         const Segment sg = seg[si];
         if (sg.phase == 1) {
-          Sched sc = p1_sched(sg, cta, p.d_grid, p.d_kc1);
+          Sched sc(bars->plan.range[si]);
           int tile, k0, k1;
           while (ok && sc.next(tile, k0, k1)) {
             const int a_of = static_cast<int>(fdiv(static_cast<unsigned>(sg.t0 + tile), p.d_tpe));
@@ -571,7 +588,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           }
           ACM_TRACE(sg.p1_index == 0 ? 13 : 2);
         } else {
-          Sched sc(cta, p.d_grid, h_tiles, sg.chunks);
+          Sched sc(bars->plan.range[si]);
           int ht, k0, k1;
           while (ok && sc.next(ht, k0, k1)) {
             const int q0 = static_cast<int>(fdiv(static_cast<unsigned>(k0), p.d_kpe));
@@ -613,7 +630,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       unsigned long long acc_f[2] = {0, 0};
       for (int si = 0; si < n_seg && ok; ++si) {
         const Segment sg = seg[si];
-        Sched sc = sg.phase == 1 ? p1_sched(sg, cta, p.d_grid, p.d_kc1) : Sched(cta, p.d_grid, h_tiles, sg.chunks);
+        Sched sc(bars->plan.range[si]);
         int tile, k0, k1;
         while (ok && sc.next(tile, k0, k1)) {
           const uint32_t b = f % kAcc;
@@ -664,7 +681,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       const Segment sg = seg[si];
       const int n_exp = sg.a1 - sg.a0;
       if (sg.phase == 1) {
-        hidx += static_cast<uint32_t>(p1_sched(sg, cta, p.d_grid, p.d_kc1).stages());
+        hidx += bars->plan.range[si].n_stages;
         hs = hidx % kStages;
         if (sg.whole) continue;          // whole tiles: nothing to exchange
         const unsigned U1 = static_cast<unsigned>(sg.nt) * kc1;
@@ -716,7 +733,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         bool good = true;
         if (lane == 0) {
           const uint64_t pol_x = policy_evict_last();
-          Sched sc(cta, p.d_grid, h_tiles, sg.chunks);
+          Sched sc(bars->plan.range[si]);
           int ht, k0, k1;
           bool polled = false;
           while (good && sc.next(ht, k0, k1)) {
@@ -766,7 +783,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         if (sg.phase != 1) continue;
         float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * kFragFloats;
         int32_t* frag_flag = p.frag_flag + sg.p1_index * G;
-        Sched sc = p1_sched(sg, cta, p.d_grid, p.d_kc1);
+        Sched sc(bars->plan.range[si]);
         int tile, k0, k1;
         while (ok && sc.next(tile, k0, k1)) {
           if (k0 > 0) {
@@ -831,7 +848,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     for (int si = 0; si < n_seg && ok; ++si) {
       const Segment sg = seg[si];
       if (sg.phase == 1) {
-        Sched sc = p1_sched(sg, cta, p.d_grid, p.d_kc1);
+        Sched sc(bars->plan.range[si]);
         int tile, k0, k1;
         while (sc.next(tile, k0, k1)) {
           const uint32_t b = f % kAcc;
@@ -933,7 +950,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         }
         if (row == 0) ACM_TRACE(10);
       } else {
-        Sched sc(cta, p.d_grid, h_tiles, sg.chunks);
+        Sched sc(bars->plan.range[si]);
         int ht, k0, k1;
         while (sc.next(ht, k0, k1)) {
           const uint32_t b = f % kAcc;
