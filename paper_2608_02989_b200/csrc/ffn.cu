@@ -852,6 +852,20 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         int tile, k0, k1;
         while (sc.next(tile, k0, k1)) {
           const uint32_t b = f % kAcc;
+          // A tile this CTA will finish needs its expert's combine weights: fetch them (one L2 round
+          // trip) while the tile's MMAs run, not after them.  They are the routing kernel's last output.
+          float wd_mine = 0.0f;
+          const int a = static_cast<int>(fdiv(static_cast<unsigned>(sg.t0 + tile), p.d_tpe));
+          if (k0 == 0) {
+            if (!waited) {
+              griddep_wait();
+              waited = true;
+            }
+            if (row < p.n_pad) {
+              const int ex_id = bars->expert[a];      // the table row of a routed expert, 1 for a shared one
+              wd_mine = ex_id >= 0 ? __ldcg(p.wtab + static_cast<size_t>(ex_id) * kMaxNodes + row) : (row < p.T ? 1.0f : 0.0f);
+            }
+          }
           ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f / kAcc) & 1u, abort_flag, p.status));
           if (!ok) break;
           if (row == 0) ACM_TRACE(21);
@@ -869,15 +883,8 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             ++ost_uses;
             continue;
           }
-          const int a = static_cast<int>(fdiv(static_cast<unsigned>(sg.t0 + tile), p.d_tpe));
-          if (!waited) {          // the combine weights are the routing kernel's last output
-            griddep_wait();
-            waited = true;
-          }
-          if (row < p.n_pad) {
-            const int ex_id = bars->expert[a];      // combine weights: the table row of a routed expert, 1 for a shared one
-            bars->wd[row] = ex_id >= 0 ? __ldcg(p.wtab + static_cast<size_t>(ex_id) * kMaxNodes + row) : (row < p.T ? 1.0f : 0.0f);
-          }
+          if (row < p.n_pad) bars->wd[row] = wd_mine;
+          if (row == 0 && fin_count == 0) ACM_TRACE(3);
           if (k1 < kc1) {
             // head part: the helper warp has summed the other CTAs' fragments of this tile into smem
             ok = epi_vote_all(mbar_wait(smem_u32(&bars->frag_full[sg.p1_index]), 0, abort_flag, p.status));
@@ -945,6 +952,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             fence_proxy_async_smem();
             mbar_arrive(smem_u32(&bars->hst_full[hb]));
             ++fin_count;
+            if (row == 0 && fin_count == 1) ACM_TRACE(4);
             if (row == 0) ACM_TRACE(25);
           }
         }
