@@ -142,6 +142,8 @@ struct __align__(8) Barriers {
   Plan plan;                    // this launch's work plan
 };
 
+static_assert(sizeof(Barriers) <= 232448 - 1024 - kStages * kStageBytes - kOutStageBytes - kFragBytes - 2 * kHStageBytes,
+              "shared memory: ring + staging buffers + control block exceed 227 KB");
 constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + kOutStageBytes + kFragBytes + 2 * kHStageBytes + sizeof(Barriers);
 
 // ---------------------------------------------------------------------------------- PTX helpers
@@ -160,17 +162,13 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// With the suspend-time hint the hardware parks the thread until the phase completes (or the hint
-// runs out) instead of returning at once: a role that polls in a tight loop takes issue slots and
-// shared-memory bandwidth from the single-thread roles (producer, MMA issuer) it waits for.
-constexpr uint32_t kSuspendHintNs = 100000u;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}\n"
-      : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
 // Bounded wait.  Returns false (after raising the status once) if the limit ran out or the CTA
