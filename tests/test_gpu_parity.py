@@ -452,3 +452,51 @@ def test_host_buffer_call_matches_the_device_call():
         _ffn_check(outs_pin[i].to(DEV), ref, f"host call {i}")
         assert acm.stats_dict(stats_pin[i]) == acm.stats_dict(stats)
     ctx.close()
+
+
+@pytest.mark.parametrize("env", [{"ACM_NO_PDL": "1"}, {"ACM_NO_EARLY_START": "1"},
+                                 {"ACM_NO_PDL": "1", "ACM_NO_EARLY_START": "1"}])
+def test_launch_modes_agree_with_the_oracle(env, monkeypatch):
+    """The fused call has three launch modes (dependent launches + early start on the eligible set, dependent
+    launches only, plain stream order); each is read from the environment when a context is created and each
+    must give the oracle's sets, routes and outputs."""
+    for key, val in env.items():
+        monkeypatch.setenv(key, val)
+    cfg = wl.CONFIGS[3]
+    ctx = _ctx(cfg, n_layers=2)
+    for layer in (0, 1):
+        _verify_layer(cfg, layer, ctx, layer, rows=[0, 7, 63])
+    ctx.close()
+
+
+def test_back_to_back_layers_without_host_synchronisation():
+    """Sixteen layer calls enqueued without a host synchronisation in between (dependent launches overlap each
+    kernel's set-up with the kernel before it; the per-call tags of the published eligible set must never be
+    mistaken for the previous call's), with a changing number of nodes; every call's routes against the oracle."""
+    cfg = wl.CONFIGS[3]
+    ctx = _ctx(cfg, n_layers=4)
+    depth, p = wl.tree_depths(cfg), wl.commitment_table(cfg)
+    alpha_full = acm.node_weights(depth, p)
+    ws, refs, outs = [], [], []
+    for layer in range(4):
+        w = wl.layer_weights(cfg, layer, DEV)
+        _set_weights(ctx, w, layer)
+        ws.append(w)
+    calls = [(i % 4, [64, 33, 17, 64, 5, 48][i % 6]) for i in range(16)]
+    xs = [wl.hidden_states(cfg, 20 + i, DEV)[:T].contiguous() for i, (_, T) in enumerate(calls)]
+    res = []
+    for (layer, T), x in zip(calls, xs):
+        res.append(ctx.moe_verify(layer, x, alpha_full[:T].to(DEV), acm.SelectParams(), want=True))
+    torch.cuda.synchronize()
+    assert ctx.device_status() == acm.OK
+    for (layer, T), x, (out, idx, wt, mask, stats) in zip(calls, xs, res):
+        w = ws[layer]
+        ref = oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha_full[:T].numpy(),
+                                cfg.top_k, oracle.SelectParams(), weighting=cfg.weighting, with_ffn=False)
+        np.testing.assert_array_equal(_u32(mask), ref["mask"])
+        np.testing.assert_array_equal(idx.cpu().numpy(), ref["idx"])
+        assert acm.stats_dict(stats)["n_activated"] == len(set(ref["idx"].ravel()) - {-1})
+        rows = [0, T - 1]
+        ffn = oracle.expert_ffn(_take(x, rows), ref["idx"][rows], ref["w"][rows], w["gate_up"], w["down"])
+        _ffn_check(_take(out, rows), ffn, f"call layer {layer} T {T}")
+    ctx.close()
