@@ -480,24 +480,27 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   const bool early = p.sel_flag != nullptr;
   if (threadIdx.x == 0) ACM_TRACE(29);
   if (early) {
-    // eight tagged words (16 mask bits under the 16-bit tag of this call), each polled by its own thread
-    if (threadIdx.x < 2 * kMaskWords) {
+    // eight tagged words (16 mask bits under the 16-bit tag of this call), each polled by its own thread --
+    // of warp 2, which has nothing else to do yet, so that the poll runs beside the set-up above
+    bool timed_out = false;
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + 2 * kMaskWords) {
+      const int i = threadIdx.x - 64;
       bool seen = false;
       uint32_t v = 0;
       const uint32_t tag = static_cast<uint32_t>(p.sel_epoch) & 0xffffu;
       const unsigned long long t0 = global_timer();
       do {
-        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.sel_flag + threadIdx.x) : "memory");
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.sel_flag + i) : "memory");
         seen = (v >> 16) == tag;
       } while (!seen && global_timer() - t0 < kTimeoutNs);
-      if (!seen) {
-        bars->abort_flag = 1;
-        atomicCAS(p.status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
-        v = 0;
-      }
-      bars->sel_half[threadIdx.x] = v & 0xffffu;
+      timed_out = !seen;
+      bars->sel_half[i] = seen ? (v & 0xffffu) : 0u;
     }
     __syncthreads();
+    if (timed_out) {
+      bars->abort_flag = 1;
+      atomicCAS(p.status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+    }
   } else {
     griddep_wait();
   }
