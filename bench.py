@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-natural", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--pool", type=int, default=0,
+                    help="supplementary run: config-5-shaped layers (Zipf-biased routing) behind an LRU expert pool "
+                         "of this many slots per layer; reports hit rate and host-to-device MiB per block")
     return ap.parse_args()
 
 
@@ -133,6 +136,82 @@ def dist_setup(args):
 
 
 # ------------------------------------------------------------------------------------------
+def run_pool(args):
+    """Offload variant (Section 3.4): every layer's experts live in an X-slot LRU pool on the GPU, the full
+    weights in pinned host memory.  A 'step' is one verification block through the stacked layers; the blocks
+    differ (new hidden states each step), so the pools see a changing demand."""
+    import ctypes
+
+    import numpy as np
+    import torch
+
+    from paper_2608_02989_b200 import acm, workloads as wl
+    from paper_2608_02989_b200 import build as acm_build
+
+    acm_build.build_library()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    cfg = wl.scaled(wl.CONFIGS[5], zipf_bias=True)
+    L = args.layers or 4
+    X = args.pool
+    T, H, E = cfg.n_nodes, cfg.hidden, cfg.n_experts
+    ctx = acm.Context.for_config(cfg, n_layers=L)
+    keep = []
+    for l in range(L):
+        w = wl.layer_weights(cfg, l, dev)
+        host_gu, host_dn = w["gate_up"].cpu().pin_memory(), w["down"].cpu().pin_memory()
+        pool_gu = torch.empty((X,) + tuple(w["gate_up"].shape[1:]), dtype=w["gate_up"].dtype, device=dev)
+        pool_dn = torch.empty((X,) + tuple(w["down"].shape[1:]), dtype=w["down"].dtype, device=dev)
+        ctx.set_layer_weights(l, w["w_router"], w["router_bias"], None, None)
+        ctx.set_slot_pool(l, pool_gu, pool_dn, host_gu, host_dn, list(range(X)))     # starts full: experts 0..X-1
+        keep.append((w["w_router"], w["router_bias"], host_gu, host_dn, pool_gu, pool_dn))
+        del w
+        torch.cuda.empty_cache()
+    n_blocks = max(args.steps, 8)
+    xs = [[wl.hidden_states(cfg, 100 * b + l, dev) for l in range(L)] for b in range(n_blocks)]
+    alpha = acm.node_weights(wl.tree_depths(cfg), wl.commitment_table(cfg)).to(dev)
+    out = torch.zeros(T, H, dtype=torch.float32, device=dev)
+    stats = torch.zeros(12, dtype=torch.int32, device=dev)
+    full = torch.full((ctx.words,), -1, dtype=torch.int32, device=dev)
+    res = {}
+    for name, kw in (("restricted_eq7", dict(params=acm.SelectParams(residency=1))),
+                     ("restricted_no_pruning", dict(params=acm.SelectParams(residency=0))),
+                     ("natural", dict(params=None, mask_override=full))):
+        for l in range(L):      # same starting pool for every policy
+            ctx.set_slot_pool(l, keep[l][4], keep[l][5], keep[l][2], keep[l][3], list(range(X)))
+        n_act = []
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        try:
+            for b in range(n_blocks):
+                for l in range(L):
+                    ctx.moe_verify(l, xs[b][l], alpha if kw.get("params") is not None else None, kw.get("params"),
+                                   mask_override=kw.get("mask_override"), out=out)
+        except acm.AcmError as err:
+            torch.cuda.synchronize()
+            if err.code != acm.ERR_UNSUPPORTED:
+                raise
+            res[name] = {"unsupported": "a block activated more experts than the pool has slots: needs the paper's waves"}
+            continue
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        ctx.check_device_status()
+        hits = misses = h2d = 0
+        for l in range(L):
+            ps = ctx.pool_stats(l, reset=True)
+            hits += ps["hits"]; misses += ps["misses"]; h2d += ps["h2d_bytes"]
+        res[name] = {"layer_blocks_per_s": n_blocks * L / dt, "hit_rate": hits / max(hits + misses, 1),
+                     "activated_per_layer_block": (hits + misses) / (n_blocks * L),
+                     "h2d_mib_per_layer_block": h2d / 2 ** 20 / (n_blocks * L)}
+    line = {"metric": METRIC, "value": res["restricted_eq7"]["layer_blocks_per_s"], "unit": UNIT, "n_gpus": 1,
+            "steps": n_blocks, "warmup": 0, "higher_is_better": True, "dtype": cfg.dtype, "data": "synthetic",
+            "config": {"workload": f"C5 {cfg.name}-shaped layers with Zipf-biased routing behind an LRU pool of {X} "
+                                   f"expert slots per layer (offload variant); {L} layers, {n_blocks} distinct blocks",
+                       "hidden": H, "n_experts": E, "top_k": cfg.top_k, "inter": cfg.inter, "n_nodes": T},
+            "policies": res}
+    print(json.dumps(line))
+
+
 def run_reference(args, world, rank):
     """The CPU oracle as the reference arm: each step is a bounded sample of the workload."""
     if rank != 0:
@@ -399,6 +478,10 @@ def run_acm(args, world, rank, local):
 def main():
     args = parse_args()
     world, rank, local = dist_setup(args)
+    if args.pool and args.impl == "acm":
+        if rank == 0:
+            run_pool(args)
+        return
     if args.impl == "reference":
         run_reference(args, world, rank)
         return

@@ -195,6 +195,25 @@ acm_status acm_host_synchronize(acm_ctx* ctx);
 acm_status acm_set_resident(acm_ctx* ctx, int layer, const uint32_t* resident_mask,
                             const void* host_gate_up, const void* host_down);
 
+/* Offload variant with the paper's per-layer expert pool (Section 3.4: "an X-slot expert pool in GPU
+ * memory", LRU): the layer's routed experts live in `n_slots` slots of the caller's device tensors
+ * pool_gate_up [n_slots,2I,H] / pool_down [n_slots,H,I] (128-byte aligned; the tensors given to
+ * acm_set_layer_weights may then be NULL), the full weights in PINNED host tensors [E,...].  The first
+ * n_initial slots are filled with initial_experts (host ids; copied synchronously).  From then on, with
+ * params->residency != 0, acm_moe_verify takes the pool's current contents as the resident set H of
+ * Eq. 7; an activated expert that is not in the pool is copied into the least recently used slot this
+ * block does not use before its FFN runs, and stays for later blocks.  A block whose activated experts
+ * outnumber the slots would need the paper's waves: ACM_ERR_UNSUPPORTED.  One host synchronisation on
+ * `stream` per call, as with acm_set_resident.  acm_set_resident(layer, NULL, ...) removes the pool. */
+acm_status acm_set_slot_pool(acm_ctx* ctx, int layer, int n_slots, void* pool_gate_up, void* pool_down,
+                             const void* host_gate_up, const void* host_down,
+                             const int32_t* initial_experts /*host*/, int n_initial);
+
+/* Pool counters since the last reset (host pointers, any may be NULL): activated experts found in the
+ * pool, activated experts loaded, bytes loaded; slot_expert [n_slots] = expert id in each slot or -1. */
+acm_status acm_pool_stats(acm_ctx* ctx, int layer, uint64_t* hits, uint64_t* misses, uint64_t* h2d_bytes,
+                          int32_t* slot_expert, int reset);
+
 /* Host->device bytes copied for non-resident experts since the last call with reset != 0. */
 acm_status acm_h2d_bytes(acm_ctx* ctx, uint64_t* bytes_out /*host*/, int reset);
 

@@ -24,6 +24,7 @@ EXPORTS = [
     "acm_default_select_params", "acm_create", "acm_destroy", "acm_set_layer_weights",
     "acm_node_weights", "acm_router", "acm_select_eligible", "acm_route_restricted",
     "acm_expert_ffn", "acm_moe_verify", "acm_moe_verify_host", "acm_host_synchronize", "acm_set_resident",
+    "acm_set_slot_pool", "acm_pool_stats",
     "acm_h2d_bytes", "acm_ffn_timing", "acm_ffn_time_ms", "acm_launch_count", "acm_device_status", "acm_status_string",
     "acm_expert_ffn_f32_noalloc",
 ]
@@ -92,6 +93,9 @@ def load_library():
                                         c_void_p, c_void_p, c_void_p]
     lib.acm_host_synchronize.argtypes = [c_void_p]
     lib.acm_set_resident.argtypes = [c_void_p, c_int, c_void_p, c_void_p, c_void_p]
+    lib.acm_set_slot_pool.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int]
+    lib.acm_pool_stats.argtypes = [c_void_p, c_int, POINTER(c_uint64), POINTER(c_uint64), POINTER(c_uint64),
+                                   c_void_p, c_int]
     lib.acm_h2d_bytes.argtypes = [c_void_p, POINTER(c_uint64), c_int]
     lib.acm_ffn_timing.argtypes = [c_void_p, c_int, c_int]
     lib.acm_ffn_time_ms.argtypes = [c_void_p, POINTER(c_float), POINTER(c_int32)]
@@ -193,6 +197,23 @@ class Context:
         self._keep[("r", layer)] = (m, host_gate_up, host_down)
         _check(self.lib.acm_set_resident(self.handle, layer, _p(m), _p(host_gate_up), _p(host_down)),
                "acm_set_resident")
+
+    def set_slot_pool(self, layer, pool_gate_up, pool_down, host_gate_up, host_down, initial_experts=()):
+        """LRU expert pool: pool_* device tensors [n_slots, ...], host_* pinned tensors [E, ...]."""
+        init = torch.tensor(list(initial_experts), dtype=torch.int32)
+        self._keep[("p", layer)] = (pool_gate_up, pool_down, host_gate_up, host_down)
+        _check(self.lib.acm_set_slot_pool(self.handle, layer, pool_gate_up.shape[0], _p(pool_gate_up), _p(pool_down),
+                                          _p(host_gate_up), _p(host_down), _p(init) if init.numel() else None,
+                                          init.numel()), "acm_set_slot_pool")
+
+    def pool_stats(self, layer, reset=False):
+        """-> dict(hits, misses, h2d_bytes, slot_expert [n_slots] list)."""
+        h, m, b = c_uint64(0), c_uint64(0), c_uint64(0)
+        n_slots = self._keep[("p", layer)][0].shape[0]
+        slots = torch.full((n_slots,), -2, dtype=torch.int32)
+        _check(self.lib.acm_pool_stats(self.handle, layer, byref(h), byref(m), byref(b), _p(slots), int(reset)),
+               "acm_pool_stats")
+        return {"hits": h.value, "misses": m.value, "h2d_bytes": b.value, "slot_expert": slots.tolist()}
 
     # ------------------------------------------------------------------ stages
     def router(self, layer, x, stream=None, want_probs=True, want_topk=True):

@@ -83,7 +83,8 @@ struct RouteArgs {
   int32_t* ticket;               // zero-initialised counter, left at zero; null: no report
   const uint32_t* resident;      // non-null: activated experts outside it are "staged"
   acm_block_stats* stats_out;    // n_activated / n_staged are filled in
-  int32_t* host_stage_list;      // mapped pinned memory: [0] = n_stage, [1..] = staged expert ids (may be null)
+  int32_t* host_stage_list;      // mapped pinned memory (may be null): [0] = n_stage, [1..] = staged expert ids,
+                                 // [1 + kMaxExperts ..] = the activated mask (4 words)
   uint32_t* sel_flag;            // non-null: [8] words, the eligible mask in 16-bit pieces tagged with sel_epoch
   int32_t sel_epoch;
   long long* dbg;                // optional time stamps in ns of the select/route kernel's stages (debugging aid)
@@ -129,6 +130,7 @@ struct FfnLaunch {
   const uint32_t* resident;  // [4] or null (all resident)
   int li;                    // 0: resident activated experts + shared experts; 1: the staged (non-resident) ones
   int n_shared;
+  const int32_t* slot_of;    // non-null: expert id -> slot of the layer's expert pool (the `staged` tensor maps)
   const float* wtab;         // [kMaxExperts][64] combine weights by (expert, node)
   acm_block_stats* stats;    // list 0 fills n_activated / n_staged (may be null)
   void* hbuf;                // [kMaxSlots][64][I] bf16 of this list

@@ -25,6 +25,19 @@ struct Layer {
   bool has_resident = false;
   const void* host_gate_up = nullptr;   // pinned host copies for on-demand loads
   const void* host_down = nullptr;
+  // LRU expert pool (acm_set_slot_pool): the layer's experts live in n_slots device slots
+  bool has_pool = false;
+  int n_slots = 0;
+  void* pool_gate_up = nullptr;         // device [n_slots, 2I, H]
+  void* pool_down = nullptr;            // device [n_slots, H, I]
+  CUtensorMap pool_map_gu, pool_map_dn;
+  std::vector<int32_t> slot_expert;     // slot -> expert id or -1
+  std::vector<int32_t> expert_slot;     // expert id -> slot or -1
+  std::vector<uint64_t> last_use;       // slot -> tick of its last use
+  uint64_t tick = 0;
+  int32_t* slot_of_dev[2] = {nullptr, nullptr};   // device copies of expert_slot, alternating (see acm_moe_verify)
+  int slot_of_cur = 0;
+  uint64_t pool_hits = 0, pool_misses = 0, pool_h2d = 0;
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -53,6 +66,8 @@ struct acm_ctx {
   CUtensorMap stage_map_gu, stage_map_dn;
   int32_t* host_stage_list = nullptr;    // pinned + mapped: [0] = count, [1..] = expert ids
   int32_t* host_stage_list_dev = nullptr;
+  uint32_t* resident_words_pinned = nullptr;   // pinned ring of resident-mask updates in flight (64 x 4 words)
+  unsigned long long resident_words_next = 0;
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_lists = nullptr, ev_copied = nullptr, ev_stage_free = nullptr;
   bool stage_in_use = false;
@@ -201,7 +216,10 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   st = encode_x(c, &x_map, x, T, n_pad);
   if (st != ACM_OK) return st;
   FfnMaps maps = L.maps;
-  if (c->stage_gate_up) {
+  if (L.has_pool) {
+    maps.staged_gate_up = L.pool_map_gu;
+    maps.staged_down = L.pool_map_dn;
+  } else if (c->stage_gate_up) {
     maps.staged_gate_up = c->stage_map_gu;
     maps.staged_down = c->stage_map_dn;
   }
@@ -211,6 +229,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   p.resident = res_dev;
   p.li = li;
   p.n_shared = d.n_shared;
+  p.slot_of = L.has_pool ? L.slot_of_dev[L.slot_of_cur] : nullptr;
   p.wtab = c->ws.wtab;
   p.stats = stats_dev;
   p.hbuf = static_cast<char*>(c->ws.hbuf) + static_cast<size_t>(li) * kMaxSlots * kMaxNodes * d.inter * 2;
@@ -254,8 +273,26 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   return ACM_OK;
 }
 
+// what both offload variants need: the pinned report buffer, the copy stream and its events
+acm_status ensure_offload_common(acm_ctx* c) {
+  if (c->host_stage_list) return ACM_OK;
+  const size_t n = (kMaxExperts + 1 + kMaskWords) * sizeof(int32_t);
+  ACM_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->host_stage_list), n, cudaHostAllocMapped));
+  std::memset(c->host_stage_list, 0, n);
+  ACM_CUDA(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->host_stage_list_dev), c->host_stage_list, 0));
+  ACM_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->resident_words_pinned), 64 * kMaskWords * sizeof(uint32_t),
+                         cudaHostAllocDefault));
+  ACM_CUDA(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+  ACM_CUDA(cudaEventCreateWithFlags(&c->ev_lists, cudaEventDisableTiming));
+  ACM_CUDA(cudaEventCreateWithFlags(&c->ev_copied, cudaEventDisableTiming));
+  ACM_CUDA(cudaEventCreateWithFlags(&c->ev_stage_free, cudaEventDisableTiming));
+  return ACM_OK;
+}
+
 acm_status ensure_staging(acm_ctx* c) {
   if (c->stage_gate_up) return ACM_OK;
+  acm_status st0 = ensure_offload_common(c);
+  if (st0 != ACM_OK) return st0;
   const acm_model_desc& d = c->desc;
   const size_t gu = static_cast<size_t>(d.n_experts) * 2 * d.inter * d.hidden * 2;
   const size_t dn = static_cast<size_t>(d.n_experts) * d.hidden * d.inter * 2;
@@ -265,14 +302,6 @@ acm_status ensure_staging(acm_ctx* c) {
   if (st != ACM_OK) return st;
   st = encode_down(c, &c->stage_map_dn, c->stage_down, d.n_experts);
   if (st != ACM_OK) return st;
-  ACM_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->host_stage_list), (kMaxExperts + 1) * sizeof(int32_t),
-                         cudaHostAllocMapped));
-  std::memset(c->host_stage_list, 0, (kMaxExperts + 1) * sizeof(int32_t));
-  ACM_CUDA(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->host_stage_list_dev), c->host_stage_list, 0));
-  ACM_CUDA(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
-  ACM_CUDA(cudaEventCreateWithFlags(&c->ev_lists, cudaEventDisableTiming));
-  ACM_CUDA(cudaEventCreateWithFlags(&c->ev_copied, cudaEventDisableTiming));
-  ACM_CUDA(cudaEventCreateWithFlags(&c->ev_stage_free, cudaEventDisableTiming));
   return ACM_OK;
 }
 
@@ -432,6 +461,10 @@ acm_status acm_destroy(acm_ctx* c) {
     if (c->ev_out[b]) cudaEventDestroy(c->ev_out[b]);
   }
   if (c->host_stage_list) cudaFreeHost(c->host_stage_list);
+  if (c->resident_words_pinned) cudaFreeHost(c->resident_words_pinned);
+  for (Layer& L : c->layers)
+    for (int b = 0; b < 2; ++b)
+      if (L.slot_of_dev[b]) cudaFree(L.slot_of_dev[b]);
   if (c->stage_gate_up) cudaFree(c->stage_gate_up);
   if (c->stage_down) cudaFree(c->stage_down);
   if (c->ws_base) cudaFree(c->ws_base);
@@ -568,7 +601,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   acm_status st = check_block_args(c, layer, T, true);
   if (st != ACM_OK) return st;
   const Layer& L = c->layers[layer];
-  if (!x || !out || !L.gate_up) return ACM_ERR_INVALID;
+  if (!x || !out || (!L.gate_up && !L.has_pool)) return ACM_ERR_INVALID;
   if (reinterpret_cast<uintptr_t>(x) % 16 != 0 || reinterpret_cast<uintptr_t>(out) % 16 != 0) return ACM_ERR_INVALID;
   acm_select_params prm;
   if (eligible_mask_override) {
@@ -641,8 +674,67 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
     ACM_CUDA(cudaEventSynchronize(c->ev_lists));
     const int n_stage = c->host_stage_list[0];
     if (n_stage < 0 || n_stage > E) return ACM_ERR_CUDA;
-    if (n_stage > 0) {
-      const size_t gu = static_cast<size_t>(2) * d.inter * d.hidden * 2, dn = static_cast<size_t>(d.hidden) * d.inter * 2;
+    const size_t gu = static_cast<size_t>(2) * d.inter * d.hidden * 2, dn = static_cast<size_t>(d.hidden) * d.inter * 2;
+    if (L.has_pool) {
+      // LRU expert pool: the experts activated by this block that were resident are touched; the others
+      // are loaded, synchronously with respect to their FFN, into the least recently used slots that this
+      // block does not use, and stay resident for later blocks.
+      Layer& P = c->layers[layer];
+      uint32_t act[kMaskWords];
+      for (int w = 0; w < kMaskWords; ++w) act[w] = static_cast<uint32_t>(c->host_stage_list[1 + kMaxExperts + w]);
+      int n_act = 0;
+      for (int w = 0; w < kMaskWords; ++w) n_act += __builtin_popcount(act[w]);
+      if (n_act > P.n_slots) return ACM_ERR_UNSUPPORTED;      // would need several waves over the pool
+      P.tick += 1;
+      for (int e = 0; e < E; ++e)
+        if (((act[e >> 5] >> (e & 31)) & 1u) && P.expert_slot[e] >= 0) {
+          P.last_use[P.expert_slot[e]] = P.tick;
+          P.pool_hits += 1;
+        }
+      if (n_stage > 0) {
+        for (int i = 0; i < n_stage; ++i) {
+          const int e = c->host_stage_list[1 + i];
+          if (e < 0 || e >= E || P.expert_slot[e] >= 0) return ACM_ERR_CUDA;
+          int victim = -1;
+          for (int sl = 0; sl < P.n_slots; ++sl) {           // free slots first, then the oldest one not used now
+            if (P.last_use[sl] == P.tick) continue;
+            if (victim < 0 || P.last_use[sl] < P.last_use[victim]) victim = sl;
+          }
+          if (victim < 0) return ACM_ERR_UNSUPPORTED;
+          if (P.slot_expert[victim] >= 0) P.expert_slot[P.slot_expert[victim]] = -1;
+          P.slot_expert[victim] = e;
+          P.expert_slot[e] = victim;
+          P.last_use[victim] = P.tick;
+          ACM_CUDA(cudaMemcpyAsync(static_cast<char*>(P.pool_gate_up) + victim * gu,
+                                   static_cast<const char*>(P.host_gate_up) + e * gu, gu, cudaMemcpyHostToDevice,
+                                   c->copy_stream));
+          ACM_CUDA(cudaMemcpyAsync(static_cast<char*>(P.pool_down) + victim * dn,
+                                   static_cast<const char*>(P.host_down) + e * dn, dn, cudaMemcpyHostToDevice,
+                                   c->copy_stream));
+          P.pool_misses += 1;
+          P.pool_h2d += gu + dn;
+          c->h2d_bytes += gu + dn;
+        }
+        // the new expert -> slot table goes into the other device copy (the running kernel reads this one)
+        const int nxt = P.slot_of_cur ^ 1;
+        ACM_CUDA(cudaMemcpyAsync(P.slot_of_dev[nxt], P.expert_slot.data(), sizeof(int32_t) * E, cudaMemcpyHostToDevice,
+                                 c->copy_stream));
+        ACM_CUDA(cudaEventRecord(c->ev_copied, c->copy_stream));
+        ACM_CUDA(cudaStreamWaitEvent(s, c->ev_copied, 0));
+        P.slot_of_cur = nxt;
+        st = run_ffn_list(c, P, x, T, 1, out, s, res_dev, nullptr);
+        if (st != ACM_OK) return st;
+        // the resident set of the next block (this block's kernels still read the old one: stream order)
+        uint32_t words[kMaskWords] = {0, 0, 0, 0};
+        for (int e = 0; e < E; ++e)
+          if (P.expert_slot[e] >= 0) words[e >> 5] |= 1u << (e & 31);
+        std::memcpy(c->resident_words_pinned + kMaskWords * (c->resident_words_next % 64), words, sizeof words);
+        ACM_CUDA(cudaMemcpyAsync(c->resident_dev + 4 * layer,
+                                 c->resident_words_pinned + kMaskWords * (c->resident_words_next % 64), sizeof words,
+                                 cudaMemcpyHostToDevice, s));
+        c->resident_words_next += 1;
+      }
+    } else if (n_stage > 0) {
       if (c->stage_in_use) ACM_CUDA(cudaStreamWaitEvent(c->copy_stream, c->ev_stage_free, 0));
       for (int i = 0; i < n_stage; ++i) {
         const int e = c->host_stage_list[1 + i];
@@ -749,9 +841,11 @@ acm_status acm_set_resident(acm_ctx* c, int layer, const uint32_t* resident_mask
   Layer& L = c->layers[layer];
   if (!resident_mask) {
     L.has_resident = false;
+    L.has_pool = false;
     L.host_gate_up = L.host_down = nullptr;
     return ACM_OK;
   }
+  if (L.has_pool) return ACM_ERR_INVALID;      // clear the pool first (NULL mask)
   if (c->desc.dtype != ACM_BF16) return ACM_ERR_UNSUPPORTED;
   if (!host_gate_up || !host_down) return ACM_ERR_INVALID;
   acm_status st = ensure_staging(c);
@@ -762,6 +856,83 @@ acm_status acm_set_resident(acm_ctx* c, int layer, const uint32_t* resident_mask
   L.has_resident = true;
   L.host_gate_up = host_gate_up;
   L.host_down = host_down;
+  return ACM_OK;
+}
+
+acm_status acm_set_slot_pool(acm_ctx* c, int layer, int n_slots, void* pool_gate_up, void* pool_down,
+                             const void* host_gate_up, const void* host_down, const int32_t* initial_experts,
+                             int n_initial) {
+  if (!c || layer < 0 || layer >= c->desc.n_layers) return ACM_ERR_INVALID;
+  const acm_model_desc& d = c->desc;
+  if (d.dtype != ACM_BF16) return ACM_ERR_UNSUPPORTED;
+  Layer& L = c->layers[layer];
+  if (!L.set) return ACM_ERR_INVALID;
+  if (n_slots < d.top_k || n_slots > kMaxSlots || !pool_gate_up || !pool_down || !host_gate_up || !host_down)
+    return ACM_ERR_INVALID;
+  if (n_initial < 0 || n_initial > n_slots || (n_initial > 0 && !initial_experts)) return ACM_ERR_INVALID;
+  if (reinterpret_cast<uintptr_t>(pool_gate_up) % 128 != 0 || reinterpret_cast<uintptr_t>(pool_down) % 128 != 0)
+    return ACM_ERR_INVALID;
+  acm_status st = ensure_offload_common(c);
+  if (st != ACM_OK) return st;
+  st = encode_gate_up(c, &L.pool_map_gu, pool_gate_up, n_slots);
+  if (st != ACM_OK) return st;
+  st = encode_down(c, &L.pool_map_dn, pool_down, n_slots);
+  if (st != ACM_OK) return st;
+  if (!L.gate_up) {          // no full device tensors: every descriptor the kernel is handed must still be valid
+    L.maps.gate_up = L.pool_map_gu;
+    L.maps.down = L.pool_map_dn;
+    if (d.n_shared == 0) {
+      L.maps.shared_gate_up = L.pool_map_gu;
+      L.maps.shared_down = L.pool_map_dn;
+    }
+  }
+  const int E = d.n_experts;
+  L.n_slots = n_slots;
+  L.pool_gate_up = pool_gate_up;
+  L.pool_down = pool_down;
+  L.host_gate_up = host_gate_up;
+  L.host_down = host_down;
+  L.slot_expert.assign(n_slots, -1);
+  L.expert_slot.assign(E, -1);
+  L.last_use.assign(n_slots, 0);
+  L.tick = 0;
+  L.pool_hits = L.pool_misses = L.pool_h2d = 0;
+  const size_t gu = static_cast<size_t>(2) * d.inter * d.hidden * 2, dn = static_cast<size_t>(d.hidden) * d.inter * 2;
+  for (int i = 0; i < n_initial; ++i) {
+    const int e = initial_experts[i];
+    if (e < 0 || e >= E || L.expert_slot[e] >= 0) return ACM_ERR_INVALID;
+    ACM_CUDA(cudaMemcpy(static_cast<char*>(pool_gate_up) + i * gu, static_cast<const char*>(host_gate_up) + e * gu, gu,
+                        cudaMemcpyHostToDevice));
+    ACM_CUDA(cudaMemcpy(static_cast<char*>(pool_down) + i * dn, static_cast<const char*>(host_down) + e * dn, dn,
+                        cudaMemcpyHostToDevice));
+    L.slot_expert[i] = e;
+    L.expert_slot[e] = i;
+  }
+  for (int b = 0; b < 2; ++b) {
+    if (!L.slot_of_dev[b]) ACM_CUDA(cudaMalloc(reinterpret_cast<void**>(&L.slot_of_dev[b]), sizeof(int32_t) * kMaxExperts));
+    ACM_CUDA(cudaMemcpy(L.slot_of_dev[b], L.expert_slot.data(), sizeof(int32_t) * E, cudaMemcpyHostToDevice));
+  }
+  L.slot_of_cur = 0;
+  uint32_t words[kMaskWords] = {0, 0, 0, 0};
+  for (int e = 0; e < E; ++e)
+    if (L.expert_slot[e] >= 0) words[e >> 5] |= 1u << (e & 31);
+  ACM_CUDA(cudaMemcpy(c->resident_dev + 4 * layer, words, sizeof words, cudaMemcpyHostToDevice));
+  L.has_resident = true;
+  L.has_pool = true;
+  return ACM_OK;
+}
+
+acm_status acm_pool_stats(acm_ctx* c, int layer, uint64_t* hits, uint64_t* misses, uint64_t* h2d_bytes,
+                          int32_t* slot_expert, int reset) {
+  if (!c || layer < 0 || layer >= c->desc.n_layers) return ACM_ERR_INVALID;
+  Layer& L = c->layers[layer];
+  if (!L.has_pool) return ACM_ERR_INVALID;
+  if (hits) *hits = L.pool_hits;
+  if (misses) *misses = L.pool_misses;
+  if (h2d_bytes) *h2d_bytes = L.pool_h2d;
+  if (slot_expert)
+    for (int i = 0; i < L.n_slots; ++i) slot_expert[i] = L.slot_expert[i];
+  if (reset) L.pool_hits = L.pool_misses = L.pool_h2d = 0;
   return ACM_OK;
 }
 

@@ -351,6 +351,7 @@ struct FfnArgs {
   const uint32_t* act_mask;
   const uint32_t* resident;
   int li, n_shared;
+  const int32_t* slot_of;
   const float* wtab;
   acm_block_stats* stats;
   __nv_bfloat16* hbuf;
@@ -537,7 +538,10 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
       int slot = __popc(mine & ((1u << (e & 31)) - 1u));
 #pragma unroll
       for (int v = 0; v < kMaskWords; ++v) slot += v < wd ? __popc(am[v]) : 0;
-      s_entry[slot] = p.li == 0 ? make_entry(kSrcRouted, e) : make_entry(kSrcStaged, slot);
+      // where the expert's weights are: the layer's own tensors (resident), staging slot `slot` (copied in
+      // for this block), or -- with an expert pool -- whichever pool slot holds it
+      s_entry[slot] = p.slot_of ? make_entry(kSrcStaged, p.slot_of[e])
+                                : p.li == 0 ? make_entry(kSrcRouted, e) : make_entry(kSrcStaged, slot);
       bars->expert[slot] = e;
     }
   } else if (p.li == 0 && threadIdx.x - kMaxExperts < p.n_shared) {
@@ -1075,7 +1079,7 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
     a.d_kpe = make_fastdiv(static_cast<unsigned>((tpe + kAtoms - 1) / kAtoms));
   }
   a.T = L.T; a.H = L.H; a.I = L.I; a.n_pad = L.n_pad;
-  a.act_mask = L.act_mask; a.resident = L.resident; a.li = L.li; a.n_shared = L.n_shared; a.wtab = L.wtab;
+  a.act_mask = L.act_mask; a.resident = L.resident; a.li = L.li; a.n_shared = L.n_shared; a.slot_of = L.slot_of; a.wtab = L.wtab;
   a.stats = L.stats; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
   a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag;
   a.sel_flag = L.sel_flag; a.sel_epoch = L.sel_epoch;

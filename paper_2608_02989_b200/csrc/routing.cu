@@ -753,6 +753,7 @@ k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uin
         ra.host_stage_list[1 + pos++] = lane * 32 + b;
       }
       if (lane == 0) ra.host_stage_list[0] = tot_stg;
+      if (lane < kMaskWords) ra.host_stage_list[1 + kMaxExperts + lane] = static_cast<int32_t>(act);   // the activated set
     }
     if (lane == 0 && ra.stats_out) { ra.stats_out->n_activated = n_act; ra.stats_out->n_staged = tot_stg; }
   }

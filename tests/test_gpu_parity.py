@@ -500,3 +500,78 @@ def test_back_to_back_layers_without_host_synchronisation():
         ffn = oracle.expert_ffn(_take(x, rows), ref["idx"][rows], ref["w"][rows], w["gate_up"], w["down"])
         _ffn_check(_take(out, rows), ffn, f"call layer {layer} T {T}")
     ctx.close()
+
+
+class _LruModel:
+    """The pool policy restated for the test: free slots first (lowest index), else the least recently used
+    slot among those the current block does not use; ties to the lower slot index."""
+
+    def __init__(self, n_slots, initial):
+        self.slot_expert = [-1] * n_slots
+        self.last_use = [0] * n_slots
+        self.tick = 0
+        for i, e in enumerate(initial):
+            self.slot_expert[i] = e
+
+    def resident(self):
+        return {e for e in self.slot_expert if e >= 0}
+
+    def block(self, activated):
+        self.tick += 1
+        hits = misses = 0
+        for s, e in enumerate(self.slot_expert):
+            if e in activated:
+                self.last_use[s] = self.tick
+                hits += 1
+        for e in sorted(activated - self.resident()):
+            cand = [s for s in range(len(self.slot_expert)) if self.last_use[s] != self.tick]
+            victim = min(cand, key=lambda s: (self.last_use[s], s))
+            self.slot_expert[victim] = e
+            self.last_use[victim] = self.tick
+            misses += 1
+        return hits, misses
+
+
+@pytest.mark.parametrize("mode", [1, 0])
+def test_lru_expert_pool_over_a_sequence_of_blocks(mode):
+    """Section 3.4's X-slot pool on a reduced config-5 layer: the expert tensors exist on the device only as pool
+    slots; eight blocks in a row, each against the oracle run with the resident set an LRU model predicts, plus the
+    model's hit / miss counts, loaded bytes and final slot contents."""
+    cfg = wl.scaled(wl.CONFIGS[5], hidden=512, inter=256, n_experts=64, top_k=4, n_nodes=24, max_depth=5, n_layers=1,
+                    zipf_bias=True)            # skewed expert popularity: the activated set stays below the pool size
+    w, _, alpha = _block(cfg, 3)
+    E, X = cfg.n_experts, 24
+    host_gu, host_dn = w["gate_up"].cpu().pin_memory(), w["down"].cpu().pin_memory()
+    pool_gu = torch.full((X,) + tuple(w["gate_up"].shape[1:]), float("nan"), dtype=w["gate_up"].dtype, device=DEV)
+    pool_dn = torch.full((X,) + tuple(w["down"].shape[1:]), float("nan"), dtype=w["down"].dtype, device=DEV)
+    initial = list(range(0, 24, 2))                 # 12 of the 20 slots start occupied
+    ctx = _ctx(cfg)
+    ctx.set_layer_weights(0, w["w_router"], w["router_bias"], None, None)
+    ctx.set_slot_pool(0, pool_gu, pool_dn, host_gu, host_dn, initial)
+    model = _LruModel(X, initial)
+    tot_hits = tot_misses = 0
+    for blk in range(8):
+        x = wl.hidden_states(cfg, 40 + blk, DEV)
+        rset = model.resident()
+        rmask = np.zeros(2, dtype=np.uint32)
+        for e in rset:
+            rmask[e >> 5] |= np.uint32(1) << np.uint32(e & 31)
+        out, idx, wt, mask, stats = ctx.moe_verify(0, x, alpha.to(DEV), acm.SelectParams(residency=mode), want=True)
+        assert ctx.device_status() == acm.OK
+        ref = oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha.numpy(), cfg.top_k,
+                                oracle.SelectParams(residency=mode), weighting=cfg.weighting, resident_mask=rmask)
+        np.testing.assert_array_equal(_u32(mask), ref["mask"])
+        np.testing.assert_array_equal(idx.cpu().numpy(), ref["idx"])
+        _ffn_check(out, ref["out"], f"pool block {blk}")
+        activated = {int(e) for e in set(ref["idx"].ravel()) - {-1}}
+        hits, misses = model.block(activated)
+        tot_hits += hits
+        tot_misses += misses
+        st = acm.stats_dict(stats)
+        assert st["n_activated"] == len(activated) and st["n_staged"] == misses
+    ps = ctx.pool_stats(0)
+    assert (ps["hits"], ps["misses"]) == (tot_hits, tot_misses)
+    assert ps["h2d_bytes"] == tot_misses * cfg.expert_bytes
+    assert ps["slot_expert"] == model.slot_expert
+    assert tot_misses > 0 and tot_hits > 0
+    ctx.close()
