@@ -202,9 +202,11 @@ acm_status acm_set_resident(acm_ctx* ctx, int layer, const uint32_t* resident_ma
  * n_initial slots are filled with initial_experts (host ids; copied synchronously).  From then on, with
  * params->residency != 0, acm_moe_verify takes the pool's current contents as the resident set H of
  * Eq. 7; an activated expert that is not in the pool is copied into the least recently used slot this
- * block does not use before its FFN runs, and stays for later blocks.  A block whose activated experts
- * outnumber the slots would need the paper's waves: ACM_ERR_UNSUPPORTED.  One host synchronisation on
- * `stream` per call, as with acm_set_resident.  acm_set_resident(layer, NULL, ...) removes the pool. */
+ * block does not use before its FFN runs, and stays for later blocks.  When the activated experts
+ * outnumber the free slots the loads go in waves (each wave: copies, then one FFN launch over the experts
+ * just loaded; a later wave waits for the launch before it and may replace any slot).  One host
+ * synchronisation on `stream` per call, as with acm_set_resident.  acm_set_resident(layer, NULL, ...)
+ * removes the pool. */
 acm_status acm_set_slot_pool(acm_ctx* ctx, int layer, int n_slots, void* pool_gate_up, void* pool_down,
                              const void* host_gate_up, const void* host_down,
                              const int32_t* initial_experts /*host*/, int n_initial);

@@ -129,6 +129,7 @@ struct FfnLaunch {
   const uint32_t* act_mask;  // [4] activated routed experts
   const uint32_t* resident;  // [4] or null (all resident)
   int li;                    // 0: resident activated experts + shared experts; 1: the staged (non-resident) ones
+  uint32_t only[4];          // further restriction of this launch's experts (all ones: none); one wave of list 1
   int n_shared;
   const int32_t* slot_of;    // non-null: expert id -> slot of the layer's expert pool (the `staged` tensor maps)
   const float* wtab;         // [kMaxExperts][64] combine weights by (expert, node)

@@ -37,7 +37,7 @@ struct Layer {
   uint64_t tick = 0;
   int32_t* slot_of_dev[2] = {nullptr, nullptr};   // device copies of expert_slot, alternating (see acm_moe_verify)
   int slot_of_cur = 0;
-  uint64_t pool_hits = 0, pool_misses = 0, pool_h2d = 0;
+  uint64_t pool_hits = 0, pool_misses = 0, pool_h2d = 0, pool_waves = 0;
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -68,6 +68,7 @@ struct acm_ctx {
   int32_t* host_stage_list_dev = nullptr;
   uint32_t* resident_words_pinned = nullptr;   // pinned ring of resident-mask updates in flight (64 x 4 words)
   unsigned long long resident_words_next = 0;
+  bool pool_waves_list1_used = false;   // within one call: the second work list has been used by an earlier wave
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_lists = nullptr, ev_copied = nullptr, ev_stage_free = nullptr;
   bool stage_in_use = false;
@@ -207,7 +208,7 @@ acm_status check_block_args(const acm_ctx* c, int layer, int T, bool need_weight
 // One FFN launch over work list `li` (0 = resident + shared, 1 = staged).
 acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li, float* out, cudaStream_t s,
                         const uint32_t* res_dev = nullptr, acm_block_stats* stats_dev = nullptr, bool pdl_ok = false,
-                        int32_t early_epoch = 0) {
+                        int32_t early_epoch = 0, const uint32_t* only = nullptr) {
   const acm_model_desc& d = c->desc;
   const int n_pad = (T + 15) / 16 * 16;
   acm_status st = ensure_h_maps(c, n_pad);
@@ -228,6 +229,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   p.act_mask = c->ws.act_mask;
   p.resident = res_dev;
   p.li = li;
+  for (int w = 0; w < 4; ++w) p.only[w] = only ? only[w] : 0xffffffffu;
   p.n_shared = d.n_shared;
   p.slot_of = L.has_pool ? L.slot_of_dev[L.slot_of_cur] : nullptr;
   p.wtab = c->ws.wtab;
@@ -684,27 +686,44 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
       for (int w = 0; w < kMaskWords; ++w) act[w] = static_cast<uint32_t>(c->host_stage_list[1 + kMaxExperts + w]);
       int n_act = 0;
       for (int w = 0; w < kMaskWords; ++w) n_act += __builtin_popcount(act[w]);
-      if (n_act > P.n_slots) return ACM_ERR_UNSUPPORTED;      // would need several waves over the pool
+      if (n_act - n_stage > P.n_slots) return ACM_ERR_CUDA;   // more resident experts than slots: cannot be
       P.tick += 1;
       for (int e = 0; e < E; ++e)
         if (((act[e >> 5] >> (e & 31)) & 1u) && P.expert_slot[e] >= 0) {
           P.last_use[P.expert_slot[e]] = P.tick;
           P.pool_hits += 1;
         }
-      if (n_stage > 0) {
-        for (int i = 0; i < n_stage; ++i) {
-          const int e = c->host_stage_list[1 + i];
-          if (e < 0 || e >= E || P.expert_slot[e] >= 0) return ACM_ERR_CUDA;
+      // The activated experts that are not in the pool are loaded in WAVES (Section 3.4: a routed union
+      // larger than the pool is processed in several waves that each fit).  The first wave may only take
+      // slots this block does not use -- the FFN over the resident experts is running -- so it needs no wait;
+      // every later wave first waits for the FFN launched before it and may then replace any slot.  The
+      // expert FFN is a sum over experts, so a wave is a subset of experts over all nodes: each expert is
+      // loaded once.
+      std::vector<int32_t> wave_of(P.n_slots, -1);
+      int done = 0, wave = 0;
+      while (done < n_stage) {
+        if (wave > 0) {
+          ACM_CUDA(cudaEventRecord(c->ev_stage_free, s));
+          ACM_CUDA(cudaStreamWaitEvent(c->copy_stream, c->ev_stage_free, 0));
+        }
+        uint32_t only[kMaskWords] = {0, 0, 0, 0};
+        int loaded = 0;
+        while (done < n_stage) {
           int victim = -1;
-          for (int sl = 0; sl < P.n_slots; ++sl) {           // free slots first, then the oldest one not used now
-            if (P.last_use[sl] == P.tick) continue;
+          for (int sl = 0; sl < P.n_slots; ++sl) {           // free slots first, then the least recently used
+            if (wave_of[sl] == wave) continue;               // just loaded for this wave
+            if (wave == 0 && P.last_use[sl] == P.tick) continue;
             if (victim < 0 || P.last_use[sl] < P.last_use[victim]) victim = sl;
           }
-          if (victim < 0) return ACM_ERR_UNSUPPORTED;
+          if (victim < 0) break;                             // this wave is full
+          const int e = c->host_stage_list[1 + done];
+          if (e < 0 || e >= E || P.expert_slot[e] >= 0) return ACM_ERR_CUDA;
           if (P.slot_expert[victim] >= 0) P.expert_slot[P.slot_expert[victim]] = -1;
           P.slot_expert[victim] = e;
           P.expert_slot[e] = victim;
           P.last_use[victim] = P.tick;
+          wave_of[victim] = wave;
+          only[e >> 5] |= 1u << (e & 31);
           ACM_CUDA(cudaMemcpyAsync(static_cast<char*>(P.pool_gate_up) + victim * gu,
                                    static_cast<const char*>(P.host_gate_up) + e * gu, gu, cudaMemcpyHostToDevice,
                                    c->copy_stream));
@@ -714,16 +733,29 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
           P.pool_misses += 1;
           P.pool_h2d += gu + dn;
           c->h2d_bytes += gu + dn;
+          ++done;
+          ++loaded;
         }
-        // the new expert -> slot table goes into the other device copy (the running kernel reads this one)
-        const int nxt = P.slot_of_cur ^ 1;
-        ACM_CUDA(cudaMemcpyAsync(P.slot_of_dev[nxt], P.expert_slot.data(), sizeof(int32_t) * E, cudaMemcpyHostToDevice,
-                                 c->copy_stream));
-        ACM_CUDA(cudaEventRecord(c->ev_copied, c->copy_stream));
-        ACM_CUDA(cudaStreamWaitEvent(s, c->ev_copied, 0));
-        P.slot_of_cur = nxt;
-        st = run_ffn_list(c, P, x, T, 1, out, s, res_dev, nullptr);
-        if (st != ACM_OK) return st;
+        if (loaded > 0) {
+          // the new expert -> slot table goes into the other device copy (a running kernel may read this one)
+          const int nxt = P.slot_of_cur ^ 1;
+          ACM_CUDA(cudaMemcpyAsync(P.slot_of_dev[nxt], P.expert_slot.data(), sizeof(int32_t) * E,
+                                   cudaMemcpyHostToDevice, c->copy_stream));
+          ACM_CUDA(cudaEventRecord(c->ev_copied, c->copy_stream));
+          ACM_CUDA(cudaStreamWaitEvent(s, c->ev_copied, 0));
+          P.slot_of_cur = nxt;
+          if (c->pool_waves_list1_used)      // the second work list's counters are cleared once per block by the router kernel
+            ACM_CUDA(cudaMemsetAsync(c->ws.ready + kMaxSlots, 0, sizeof(int32_t) * kMaxSlots, s));
+          c->pool_waves_list1_used = true;
+          st = run_ffn_list(c, P, x, T, 1, out, s, res_dev, nullptr, false, 0, only);
+          if (st != ACM_OK) return st;
+          P.pool_waves += 1;
+        }
+        ++wave;
+        if (wave > n_stage + 1) return ACM_ERR_CUDA;       // cannot happen: every wave after the first has room
+      }
+      c->pool_waves_list1_used = false;
+      if (n_stage > 0) {
         // the resident set of the next block (this block's kernels still read the old one: stream order)
         uint32_t words[kMaskWords] = {0, 0, 0, 0};
         for (int e = 0; e < E; ++e)

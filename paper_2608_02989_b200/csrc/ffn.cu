@@ -351,6 +351,7 @@ struct FfnArgs {
   const uint32_t* act_mask;
   const uint32_t* resident;
   int li, n_shared;
+  uint32_t only[4];
   const int32_t* slot_of;
   const float* wtab;
   acm_block_stats* stats;
@@ -515,7 +516,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   for (int wd = 0; wd < kMaskWords; ++wd) {
     const uint32_t act = early ? (bars->sel_half[2 * wd] | (bars->sel_half[2 * wd + 1] << 16)) : p.act_mask[wd];
     const uint32_t res = p.resident ? p.resident[wd] : 0xffffffffu;
-    am[wd] = p.li == 0 ? act & res : act & ~res;
+    am[wd] = (p.li == 0 ? act & res : act & ~res) & p.only[wd];
     n_routed += __popc(am[wd]);
   }
   const int n_act = n_routed + (p.li == 0 ? p.n_shared : 0);
@@ -1080,6 +1081,7 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   }
   a.T = L.T; a.H = L.H; a.I = L.I; a.n_pad = L.n_pad;
   a.act_mask = L.act_mask; a.resident = L.resident; a.li = L.li; a.n_shared = L.n_shared; a.slot_of = L.slot_of; a.wtab = L.wtab;
+  for (int w = 0; w < 4; ++w) a.only[w] = L.only[w];
   a.stats = L.stats; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
   a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag;
   a.sel_flag = L.sel_flag; a.sel_epoch = L.sel_epoch;

@@ -517,18 +517,28 @@ class _LruModel:
         return {e for e in self.slot_expert if e >= 0}
 
     def block(self, activated):
+        """One block: hits are touched; misses are loaded in ascending id order, in waves -- the first wave may
+        only replace slots this block does not use, every later wave any slot it has not just filled."""
         self.tick += 1
+        n = len(self.slot_expert)
         hits = misses = 0
         for s, e in enumerate(self.slot_expert):
             if e in activated:
                 self.last_use[s] = self.tick
                 hits += 1
-        for e in sorted(activated - self.resident()):
-            cand = [s for s in range(len(self.slot_expert)) if self.last_use[s] != self.tick]
-            victim = min(cand, key=lambda s: (self.last_use[s], s))
-            self.slot_expert[victim] = e
-            self.last_use[victim] = self.tick
-            misses += 1
+        todo = sorted(activated - self.resident())
+        wave, wave_of = 0, [-1] * n
+        while todo:
+            while todo:
+                cand = [s for s in range(n) if wave_of[s] != wave and not (wave == 0 and self.last_use[s] == self.tick)]
+                if not cand:
+                    break
+                victim = min(cand, key=lambda s: (self.last_use[s], s))
+                self.slot_expert[victim] = todo.pop(0)
+                self.last_use[victim] = self.tick
+                wave_of[victim] = wave
+                misses += 1
+            wave += 1
         return hits, misses
 
 
@@ -574,4 +584,39 @@ def test_lru_expert_pool_over_a_sequence_of_blocks(mode):
     assert ps["h2d_bytes"] == tot_misses * cfg.expert_bytes
     assert ps["slot_expert"] == model.slot_expert
     assert tot_misses > 0 and tot_hits > 0
+    ctx.close()
+
+
+def test_expert_pool_smaller_than_the_routed_union_runs_in_waves():
+    """Natural routing activates more experts than the pool has slots: the loads and their FFN launches go in
+    several waves; the output is still the oracle's and every activated expert outside the pool is loaded once."""
+    cfg = wl.scaled(wl.CONFIGS[5], hidden=512, inter=256, n_experts=64, top_k=4, n_nodes=24, max_depth=5, n_layers=1)
+    w, _, alpha = _block(cfg, 4)
+    E, X = cfg.n_experts, 10
+    host_gu, host_dn = w["gate_up"].cpu().pin_memory(), w["down"].cpu().pin_memory()
+    pool_gu = torch.full((X,) + tuple(w["gate_up"].shape[1:]), float("nan"), dtype=w["gate_up"].dtype, device=DEV)
+    pool_dn = torch.full((X,) + tuple(w["down"].shape[1:]), float("nan"), dtype=w["down"].dtype, device=DEV)
+    initial = [1, 5, 9, 13, 17, 21, 25]
+    ctx = _ctx(cfg)
+    ctx.set_layer_weights(0, w["w_router"], w["router_bias"], None, None)
+    ctx.set_slot_pool(0, pool_gu, pool_dn, host_gu, host_dn, initial)
+    model = _LruModel(X, initial)
+    full = torch.tensor(full_mask(E).view(np.int32), device=DEV)
+    tot_hits = tot_misses = 0
+    for blk in range(3):
+        x = wl.hidden_states(cfg, 60 + blk, DEV)
+        out, idx, wt, mask, stats = ctx.moe_verify(0, x, None, None, mask_override=full, want=True)
+        assert ctx.device_status() == acm.OK
+        ref = oracle.moe_verify(x, w["w_router"], w["router_bias"], w["gate_up"], w["down"], alpha.numpy(), cfg.top_k,
+                                weighting=cfg.weighting, mask_override=full_mask(E))
+        np.testing.assert_array_equal(idx.cpu().numpy(), ref["idx"])
+        _ffn_check(out, ref["out"], f"waves block {blk}")
+        activated = {int(e) for e in set(ref["idx"].ravel()) - {-1}}
+        assert len(activated) > X
+        hits, misses = model.block(activated)
+        tot_hits += hits
+        tot_misses += misses
+    ps = ctx.pool_stats(0)
+    assert (ps["hits"], ps["misses"]) == (tot_hits, tot_misses)
+    assert ps["slot_expert"] == model.slot_expert
     ctx.close()
