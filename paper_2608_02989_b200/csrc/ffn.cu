@@ -173,7 +173,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false (after raising the status once) if the limit ran out or the CTA
 // has already given up; callers then skip the rest of their work.
-__device__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
   if (*abort_flag) return false;
   for (int i = 0; i < 1024; ++i)
     if (mbar_try_wait(bar, parity)) return true;
@@ -188,6 +188,12 @@ __device__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_fla
       return false;
     }
   }
+}
+// Bounded wait: one inlined poll for the common case (the phase is already complete), the bounded loop
+// out of line.  The single-thread roles pay every instruction of their per-stage loop.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status);
 }
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
   int v;
@@ -631,6 +637,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = umma_idesc(p.n_pad);
+      const uint64_t desc_hi = umma_smem_desc(0);
       uint32_t it = 0, f = 0;
       bool ok = true;
       unsigned long long acc_f[2] = {0, 0};
@@ -649,14 +656,15 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
             if (!(ok = mbar_wait(smem_u32(&bars->full[s]), par, abort_flag, p.status))) break;
             if (p.trace) { acc_f[sg.phase - 1] += global_timer() - tw; if (it == 0) ACM_TRACE(6); }
             tc_fence_after();
-            const uint32_t sa = smem_u32(stage_base + static_cast<size_t>(s) * kStageBytes);
+            // descriptors: only the address field changes from stage to stage and atom to atom
+            const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
+            const uint64_t da0 = desc_hi | ((sa & 0x3ffffu) >> 4), db0 = desc_hi | (((sa + kABytes) & 0x3ffffu) >> 4);
 #pragma unroll
             for (int at = 0; at < kAtoms; ++at) {
-              const uint64_t da = umma_smem_desc(sa + at * kAtomABytes);
-              const uint64_t db = umma_smem_desc(sa + kABytes + at * b_atom_bytes);
 #pragma unroll
               for (int kk = 0; kk < kBK / 16; ++kk)
-                umma_bf16(d_tmem, da + 2 * kk, db + 2 * kk, idesc, (kc > k0 || at > 0 || kk > 0) ? 1u : 0u);
+                umma_bf16(d_tmem, da0 + (at * (kAtomABytes >> 4) + 2 * kk), db0 + (at * (b_atom_bytes >> 4) + 2 * kk), idesc,
+                          (kc > k0 || at > 0 || kk > 0) ? 1u : 0u);
             }
             umma_commit(smem_u32(&bars->empty[s]));
           }

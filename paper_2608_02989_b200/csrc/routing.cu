@@ -387,7 +387,7 @@ __device__ float sel_tree_sum_128(float* tree, float mine) {
 // is null, are built here from a.nat_idx.  Global results are written only if `write_out`.
 #define ACM_ST(slot) do { if (a.dbg && write_out && threadIdx.x == 0) a.dbg[slot] = time_ns(); } while (0)
 __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, int k, const uint32_t* natmask_g,
-                             bool write_out) {
+                             bool write_out, uint32_t* publish_words = nullptr, uint32_t publish_tag = 0) {
   const int tid = threadIdx.x;
   ACM_ST(5);
   const int lane = tid & 31, warp = tid >> 5;
@@ -546,7 +546,13 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   }
   const unsigned sp_word = __ballot_sync(0xffffffffu, in_Sp);
   if (lane == 0) sm.Sp[warp] = sp_word;
-  const int nSp = sel_count(in_Sp);
+  const int nSp = sel_count(in_Sp);          // (a barrier: sm.Sp is complete)
+  if (publish_words && tid < 2 * kMaskWords) {
+    // The FFN kernel may start on the eligible set now, before the outputs below are written and while the
+    // routes are made: eight self-validating words, 16 mask bits under a 16-bit tag of this call each.
+    const uint32_t bits = (sm.Sp[tid >> 1] >> (16 * (tid & 1))) & 0xffffu;
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(publish_words + tid), "r"(bits | (publish_tag << 16)) : "memory");
+  }
   if (a.prm.residency == 2 && a.resident) m_star = nS - nSp;
 
   ACM_ST(12);
@@ -696,8 +702,8 @@ k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uin
     __syncthreads();
   } else {
     if (tid < kSelThreads) {
-      stage_select(sa, sm, T, E, k, natmask_g, blockIdx.x == 0);
-      if (ra.sel_flag && blockIdx.x == 0 && tid < 2 * kMaskWords) publish_eligible(ra, sm, tid);
+      stage_select(sa, sm, T, E, k, natmask_g, blockIdx.x == 0, blockIdx.x == 0 ? ra.sel_flag : nullptr,
+                   static_cast<uint32_t>(ra.sel_epoch) & 0xffffu);
     }
     __syncthreads();
   }
