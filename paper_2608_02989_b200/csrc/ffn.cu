@@ -12,7 +12,7 @@
 //   warp 7      publisher: moves staged fragments / activation tiles to global memory (bulk reduce-add,
 //               TMA store), waits for completion, then raises the counter other CTAs wait on
 // The weights are the M operand ("swap-AB"): every activated expert's weights are read from HBM
-// exactly once for all nodes of the block.  Work plan of a launch (make_plan):
+// exactly once for all nodes of the block.  Work plan of a launch (plan_lane):
 //   gate/up  tile = 64 gate rows + the 64 matching up rows of one expert, K = hidden.  The
 //            n_tiles mod grid leftover tiles come first, cut into equal contiguous ranges of (tile,
 //            K-chunk) units over all CTAs; the CTA that owns a tile's last chunk receives the others'
@@ -378,35 +378,13 @@ __device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMa
   return src == kSrcRouted ? routed : src == kSrcShared ? shared : staged;
 }
 
-// (filled in place, in shared memory: a private copy indexed at run time would live in local memory,
-// whose first touch costs every role a trip to DRAM at the start of the kernel)
-__device__ __forceinline__ void make_plan(Plan& pl, int n_act, int tpe, int grid, int phase_mask, const FastDiv& d_kc1, int kpe,
-                                          const FastDiv& d_grid, const FastDiv& d_tpe) {
-  pl.n_seg = 0;
-  const int n_t = n_act * tpe;
-  const int rounds = static_cast<int>(fdiv(static_cast<unsigned>(n_t), d_grid)), rem = n_t - rounds * grid;
-  int n = 0;
-  if (rounds == 0) {
-    const int nA = (n_act + 1) / 2;
-    pl.a_split = nA;
-    if (phase_mask & 1) {
-      if (nA > 0) pl.seg[n++] = Segment{1, 0, 0, nA * tpe, 0, 0, 0, d_kc1};
-      if (n_act > nA) pl.seg[n++] = Segment{1, 0, nA * tpe, (n_act - nA) * tpe, 0, 0, 1, d_kc1};
-    }
-  } else {
-    pl.a_split = static_cast<int>(fdiv(static_cast<unsigned>(rem + (rounds - 1) * grid), d_tpe));
-    if (phase_mask & 1) {
-      if (rem > 0) pl.seg[n++] = Segment{1, 0, 0, rem, 0, 0, 0, d_kc1};
-      pl.seg[n++] = Segment{1, 1, rem, rounds * grid, 0, 0, 1, d_kc1};
-    }
-  }
-  if (phase_mask & 2) {
-    if (pl.a_split > 0) pl.seg[n++] = Segment{2, 0, 0, 0, 0, pl.a_split, 0, plain_div(static_cast<unsigned>(pl.a_split * kpe))};
-    if (n_act > pl.a_split) pl.seg[n++] = Segment{2, 0, 0, 0, pl.a_split, n_act, 1, plain_div(static_cast<unsigned>((n_act - pl.a_split) * kpe))};
-  }
-  pl.n_seg = n;
-}
-
+// The plan lives in shared memory (a private copy indexed at run time would live in local memory, whose
+// first touch costs every role a trip to DRAM at the start of the kernel).  It has at most four
+// segments; lane i of one warp works out the i-th one by itself -- the four candidates in order, each
+// present or not -- and its own range in it, so nothing waits for a serial pass.
+__device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act, int tpe, int grid, int phase_mask,
+                                          const FastDiv& d_kc1, int kpe, const FastDiv& d_grid, const FastDiv& d_tpe,
+                                          int h_tiles);
 // Range of segment `si` for CTA `cta` (see SegRange).  (tiles * chunks * grid fits 32 bits: launcher.)
 __device__ __forceinline__ SegRange make_range(const Segment& sg, int cta, const FastDiv& d_grid, int h_tiles) {
   SegRange r;
@@ -423,11 +401,50 @@ __device__ __forceinline__ SegRange make_range(const Segment& sg, int cta, const
   const unsigned total = tiles * sg.chunks.d;
   r.u = fdiv(total * static_cast<unsigned>(cta), d_grid);
   r.u_end = fdiv(total * static_cast<unsigned>(cta + 1), d_grid);
-  r.tile0 = static_cast<int>(fdiv(r.u, sg.chunks));
+  r.tile0 = static_cast<int>(fdiv(tiles * static_cast<unsigned>(cta), d_grid));   // = floor(u / chunks): floors nest
   r.k00 = static_cast<int>(r.u - static_cast<unsigned>(r.tile0) * sg.chunks.d);
   r.stride = 0;
   r.n_stages = r.u_end - r.u;
   return r;
+}
+
+__device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act, int tpe, int grid, int phase_mask,
+                                          const FastDiv& d_kc1, int kpe, const FastDiv& d_grid, const FastDiv& d_tpe,
+                                          int h_tiles) {
+  const int n_t = n_act * tpe;
+  const int rounds = static_cast<int>(fdiv(static_cast<unsigned>(n_t), d_grid)), rem = n_t - rounds * grid;
+  const bool p1 = (phase_mask & 1) != 0, p2 = (phase_mask & 2) != 0;
+  // candidates in execution order: two gate/up segments, two down segments
+  Segment c0, c1, c2, c3;
+  bool h0, h1, h2, h3;
+  int a_split;
+  if (rounds == 0) {
+    const int nA = (n_act + 1) / 2;
+    a_split = nA;
+    c0 = Segment{1, 0, 0, nA * tpe, 0, 0, 0, d_kc1};                          h0 = p1 && nA > 0;
+    c1 = Segment{1, 0, nA * tpe, (n_act - nA) * tpe, 0, 0, 1, d_kc1};         h1 = p1 && n_act > nA;
+  } else {
+    a_split = static_cast<int>(fdiv(static_cast<unsigned>(rem + (rounds - 1) * grid), d_tpe));
+    c0 = Segment{1, 0, 0, rem, 0, 0, 0, d_kc1};                               h0 = p1 && rem > 0;
+    c1 = Segment{1, 1, rem, rounds * grid, 0, 0, 1, d_kc1};                   h1 = p1;
+  }
+  c2 = Segment{2, 0, 0, 0, 0, a_split, 0, plain_div(static_cast<unsigned>(a_split * kpe))};                 h2 = p2 && a_split > 0;
+  c3 = Segment{2, 0, 0, 0, a_split, n_act, 1, plain_div(static_cast<unsigned>((n_act - a_split) * kpe))};   h3 = p2 && n_act > a_split;
+  const int i0 = 0, i1 = i0 + h0, i2 = i1 + h1, i3 = i2 + h2, n = i3 + h3;
+  Segment mine = c0;
+  bool have = false;
+  if (h0 && i0 == lane) { mine = c0; have = true; }
+  if (h1 && i1 == lane) { mine = c1; have = true; }
+  if (h2 && i2 == lane) { mine = c2; have = true; }
+  if (h3 && i3 == lane) { mine = c3; have = true; }
+  if (have) {
+    pl.seg[lane] = mine;
+    pl.range[lane] = make_range(mine, cta, d_grid, h_tiles);
+  }
+  if (lane == 0) {
+    pl.n_seg = n;
+    pl.a_split = a_split;
+  }
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -532,11 +549,8 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   const int h_tiles = p.H / kTileM;  // output tiles of the down phase
   const uint32_t b_atom_bytes = static_cast<uint32_t>(p.n_pad) * kBK * 2;   // one atom of the activation chunk
   const uint32_t b_bytes = kAtoms * b_atom_bytes;
-  if (warp == kThreads / 32 - 1) {      // the publisher warp has nothing else to do yet
-    if (lane == 31) make_plan(bars->plan, n_act, tpe, G, p.phase_mask, p.d_kc1, kpe, p.d_grid, p.d_tpe);
-    __syncwarp();
-    if (lane < bars->plan.n_seg) bars->plan.range[lane] = make_range(bars->plan.seg[lane], cta, p.d_grid, h_tiles);
-  }
+  if (warp == kThreads / 32 - 1 && lane < 4)      // (the publisher warp has nothing else to do yet)
+    plan_lane(bars->plan, lane, cta, n_act, tpe, G, p.phase_mask, p.d_kc1, kpe, p.d_grid, p.d_tpe, h_tiles);
   int32_t* s_entry = bars->entry;
   if (threadIdx.x < kMaxExperts) {
     const int e = threadIdx.x, wd = e >> 5;
