@@ -641,6 +641,20 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
           ACM_TRACE(sg.p1_index == 0 ? 14 : 5);
         }
       }
+      // The block's activated-expert counts, by the thread that is done first (its copies are all issued
+      // microseconds before the last epilogue): off the kernel's tail.
+      if (p.stats && p.li == 0 && blockIdx.x == 0) {
+        griddep_wait();                       // early start: the routing kernel is long complete
+        int n_all = 0, n_stg = 0;
+#pragma unroll
+        for (int wd = 0; wd < kMaskWords; ++wd) {
+          const uint32_t act = __ldcg(p.act_mask + wd);
+          n_all += __popc(act);
+          n_stg += p.resident ? __popc(act & ~p.resident[wd]) : 0;
+        }
+        p.stats->n_activated = n_all;
+        p.stats->n_staged = n_stg;
+      }
       if (!ok) {
         // giving up: let copies already in flight land before the CTA exits
         const unsigned long long t0 = global_timer();
@@ -1007,18 +1021,6 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
 
   tc_fence_before();
   __syncthreads();
-  if (p.stats && p.li == 0 && blockIdx.x == 0 && threadIdx.x == 0) {
-    griddep_wait();                       // early start: the routing kernel is long complete
-    int n_all = 0, n_stg = 0;
-#pragma unroll
-    for (int wd = 0; wd < kMaskWords; ++wd) {
-      const uint32_t act = __ldcg(p.act_mask + wd);
-      n_all += __popc(act);
-      n_stg += p.resident ? __popc(act & ~p.resident[wd]) : 0;
-    }
-    p.stats->n_activated = n_all;
-    p.stats->n_staged = n_stg;
-  }
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
