@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-natural", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="supplementary run: B > 1 verification blocks per call (they share the config's nodes and "
+                         "one pass over the expert weights) against the same blocks verified one call each")
     ap.add_argument("--pool", type=int, default=0,
                     help="supplementary run: config-5-shaped layers (Zipf-biased routing) behind an LRU expert pool "
                          "of this many slots per layer; reports hit rate and host-to-device MiB per block")
@@ -475,12 +478,98 @@ def run_acm(args, world, rank, local):
         dist.destroy_process_group()
 
 
+def run_batch(args):
+    """Multi-block batches: the configuration's T nodes are B verification blocks (trees of their own).  One
+    call per layer verifies them together -- every activated expert is streamed once for all blocks -- and is
+    compared with the same blocks verified one call each.  A 'step' is the B blocks through the stacked
+    layers; the metric counts blocks, so one batch call of B blocks is B layer-blocks."""
+    import ctypes
+
+    import torch
+
+    from paper_2608_02989_b200 import acm, workloads as wl
+    from paper_2608_02989_b200 import build as acm_build
+
+    acm_build.build_library()
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    cfg = wl.CONFIGS[args.config]
+    L, B = args.layers or cfg.n_layers, args.batch
+    T, H, E, k = cfg.n_nodes, cfg.hidden, cfg.n_experts, cfg.top_k
+    ctx = acm.Context.for_config(cfg, n_layers=L)
+    keep = []
+    for l in range(L):
+        w = wl.layer_weights(cfg, l, dev)
+        ctx.set_layer_weights(l, w["w_router"], w["router_bias"], w["gate_up"], w["down"], w["shared_gate_up"],
+                              w["shared_down"])
+        keep.append(w)
+    xs = torch.stack([wl.hidden_states(cfg, l, dev) for l in range(L)])
+    offsets, depths = wl.batch_tree_depths(cfg, B)
+    p = wl.commitment_table(cfg)
+    alpha = torch.cat([acm.node_weights(depths[offsets[b]:offsets[b + 1]], p) for b in range(B)]).to(dev)
+    outs = torch.zeros(L, T, H, dtype=torch.float32, device=dev)
+    stats = torch.zeros(L, B, 12, dtype=torch.int32, device=dev)
+    act = torch.zeros(L, ctx.words, dtype=torch.int32, device=dev)
+    params = acm.SelectParams()
+    sp = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    lib, h = ctx.lib, ctx.handle
+    offs_c = (ctypes.c_int32 * (B + 1))(*offsets)
+
+    def vp(t):
+        return ctypes.c_void_p(t.data_ptr())
+
+    calls_batch = [(h, l, vp(xs[l]), B, offs_c, vp(alpha), ctypes.byref(params), vp(outs[l]), None, None, None,
+                    vp(act[l]), vp(stats[l]), sp) for l in range(L)]
+    calls_single = [(h, l, vp(xs[l][offsets[b]:]), offsets[b + 1] - offsets[b], vp(alpha[offsets[b]:]),
+                     ctypes.byref(params), None, vp(outs[l][offsets[b]:]), None, None, None, vp(stats[l][b]), sp)
+                    for l in range(L) for b in range(B)]
+
+    def run(fn, calls, name):
+        for a in calls:
+            rc = fn(*a)
+            if rc:
+                raise acm.AcmError(rc, name)
+
+    res = {}
+    for name, fn, calls in (("batched", lib.acm_moe_verify_batch, calls_batch),
+                            ("one_call_per_block", lib.acm_moe_verify, calls_single)):
+        for _ in range(max(args.warmup, 3)):
+            run(fn, calls, name)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            run(fn, calls, name)
+        e1.record()
+        torch.cuda.synchronize()
+        ctx.check_device_status()
+        ms = e0.elapsed_time(e1) / args.steps
+        streamed = float(stats[:, :, 4].sum().item()) if name == "one_call_per_block" else \
+            float(sum(bin(int(v) & 0xffffffff).count("1") for v in act.flatten().tolist()))
+        res[name] = {"layer_blocks_per_s": B * L / (ms * 1e-3), "ms_per_step": ms,
+                     "us_per_layer": ms * 1e3 / L, "experts_streamed_per_layer": streamed / L,
+                     "expert_weight_mb_per_block_per_layer": streamed / L * cfg.expert_bytes / 1e6 / B}
+    line = {"metric": METRIC, "value": res["batched"]["layer_blocks_per_s"], "unit": UNIT, "n_gpus": 1,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "higher_is_better": True, "dtype": cfg.dtype,
+            "data": "synthetic",
+            "config": {"workload": f"C{cfg.index} {cfg.name}-shaped stack, {B} verification blocks per call "
+                                   f"({T} nodes in all, block sizes {offsets[1]}..{offsets[-1] - offsets[-2]})",
+                       "hidden": H, "n_experts": E, "top_k": k, "inter": cfg.inter, "n_nodes": T, "blocks": B,
+                       "layers": L, "l2": "inputs larger than L2: distinct layers streamed per step"},
+            "variants": res}
+    print(json.dumps(line))
+
+
 def main():
     args = parse_args()
     world, rank, local = dist_setup(args)
     if args.pool and args.impl == "acm":
         if rank == 0:
             run_pool(args)
+        return
+    if args.batch > 1 and args.impl == "acm":
+        if rank == 0:
+            run_batch(args)
         return
     if args.impl == "reference":
         run_reference(args, world, rank)

@@ -173,6 +173,25 @@ acm_status acm_moe_verify(acm_ctx* ctx, int layer, const void* x, int T, const f
                           float* w_out, uint32_t* mask_out, acm_block_stats* stats,
                           acm_stream stream);
 
+/* Multi-block batch (the paper verifies one block at a time, Section 4.1 "batch size one"; this is the
+ * same layer step for several verification blocks that share one pass over the expert weights).  The
+ * blocks' nodes are stacked along the node axis: block b owns rows block_offsets[b] ..
+ * block_offsets[b+1]-1 of x [T,hidden], alpha [T], out, idx_out, w_out (T = block_offsets[n_blocks] <=
+ * 64; block_offsets is a HOST array of n_blocks+1 ascending entries starting at 0; every block has at
+ * least one node and its first row is its root).  Stages 1-3 run per block exactly as in
+ * acm_moe_verify: block b's eligible set comes from its own nodes (Eq. 3-7) and its nodes are routed
+ * inside it (Eq. 2), so every per-block result equals that of a single-block call on the block's rows.
+ * Stage 4 runs once over all rows: an expert activated by several blocks is streamed from HBM once.
+ * mask_out [n_blocks][ceil(E/32)] = the blocks' eligible sets; activated_out [ceil(E/32)] = the union of
+ * activated experts (what was streamed); stats [n_blocks] (n_activated = experts activated by that
+ * block's own nodes).  All optional, device (stats: device or pinned).  bf16 layers without a
+ * residency only (ACM_ERR_UNSUPPORTED otherwise). */
+acm_status acm_moe_verify_batch(acm_ctx* ctx, int layer, const void* x, int n_blocks,
+                                const int32_t* block_offsets /*host*/, const float* alpha,
+                                const acm_select_params* params /*host*/, float* out, int32_t* idx_out,
+                                float* w_out, uint32_t* mask_out, uint32_t* activated_out,
+                                acm_block_stats* stats, acm_stream stream);
+
 /* The same call for HOST buffers (Section 3.1's per-layer step as a serving loop sees it): x_host
  * [T,H] and alpha_host [T] are read from, and out_host [T,H] float is written to, PINNED host
  * memory.  The copies run on the context's own copy streams through two alternating sets of device

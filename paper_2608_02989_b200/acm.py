@@ -23,7 +23,7 @@ DEMAND_TOPK_MASS, DEMAND_FULL_MASS, DEMAND_VOTES = 0, 1, 2
 EXPORTS = [
     "acm_default_select_params", "acm_create", "acm_destroy", "acm_set_layer_weights",
     "acm_node_weights", "acm_router", "acm_select_eligible", "acm_route_restricted",
-    "acm_expert_ffn", "acm_moe_verify", "acm_moe_verify_host", "acm_host_synchronize", "acm_set_resident",
+    "acm_expert_ffn", "acm_moe_verify", "acm_moe_verify_batch", "acm_moe_verify_host", "acm_host_synchronize", "acm_set_resident",
     "acm_set_slot_pool", "acm_pool_stats",
     "acm_h2d_bytes", "acm_ffn_timing", "acm_ffn_time_ms", "acm_launch_count", "acm_device_status", "acm_status_string",
     "acm_expert_ffn_f32_noalloc",
@@ -89,6 +89,8 @@ def load_library():
     lib.acm_expert_ffn.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.acm_moe_verify.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, POINTER(SelectParams),
                                    c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
+    lib.acm_moe_verify_batch.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p, POINTER(SelectParams),
+                                         c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.acm_moe_verify_host.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, POINTER(SelectParams),
                                         c_void_p, c_void_p, c_void_p]
     lib.acm_host_synchronize.argtypes = [c_void_p]
@@ -278,6 +280,31 @@ class Context:
                                        _p(idx), _p(w), _p(mask), _p(stats), _stream(stream)), "acm_moe_verify")
         if want:
             return out, idx, w, mask, stats
+        return out
+
+    def moe_verify_batch(self, layer, x, block_offsets, alpha, params=None, out=None, want=False, stream=None):
+        """Stages 1-4 for several blocks stacked along the node axis (block b = rows block_offsets[b] ..
+        block_offsets[b+1]-1).  want=True also returns idx, w, the blocks' masks [n_blocks, words], the
+        union of activated experts [words] and the blocks' stats [n_blocks, 12]."""
+        T = x.shape[0]
+        dev = x.device
+        offs = (c_int32 * len(block_offsets))(*[int(v) for v in block_offsets])
+        nb = len(block_offsets) - 1
+        if out is None:
+            out = torch.empty(T, self.H, dtype=torch.float32, device=dev)
+        params = params or SelectParams()
+        idx = w = mask = act = stats = None
+        if want:
+            idx = torch.empty(T, self.k, dtype=torch.int32, device=dev)
+            w = torch.empty(T, self.k, dtype=torch.float32, device=dev)
+            mask = torch.zeros(max(nb, 1), self.words, dtype=torch.int32, device=dev)
+            act = torch.zeros(self.words, dtype=torch.int32, device=dev)
+            stats = torch.zeros(max(nb, 1), 12, dtype=torch.int32, device=dev)
+        _check(self.lib.acm_moe_verify_batch(self.handle, layer, _p(x), nb, offs, _p(alpha), byref(params), _p(out),
+                                             _p(idx), _p(w), _p(mask), _p(act), _p(stats), _stream(stream)),
+               "acm_moe_verify_batch")
+        if want:
+            return out, idx, w, mask, act, stats
         return out
 
     def moe_verify_host(self, layer, x_host, alpha_host, out_host, params=None, stats_host=None, stream=None):

@@ -36,11 +36,12 @@ struct Workspace {
   uint32_t* nat_mask;   // [T,4] the same sets as bit masks
   int32_t* idx;         // [T,k]
   float* w;             // [T,k]
-  uint32_t* mask;       // [4] eligible set S'
-  uint32_t* unpruned;   // [4] S
-  int32_t* count;       // [1]
-  float* demand;        // [E]
-  acm_block_stats* stats;
+  // per block of a batch (a single block uses entry 0)
+  uint32_t* mask;       // [64][4] eligible set S'
+  uint32_t* unpruned;   // [64][4] S
+  int32_t* count;       // [64]
+  float* demand;        // [64][kMaxExperts]
+  acm_block_stats* stats;   // [64]
   uint32_t* act_mask;   // [4] activated routed experts of the current block
   float* wtab;          // [kMaxExperts][64] combine weight of (expert, node)
   void* hbuf;           // [2][kMaxSlots][64][I] bf16 (f32 path: [T][k+ns][I] float)
@@ -50,7 +51,7 @@ struct Workspace {
   int32_t* status;      // [1] sticky device-side status
   int32_t* tile_done;   // [64] router kernel: expert tiles finished per node tile (self-resetting)
   int32_t* ticket;      // [1] select/route kernel: finished CTAs (self-resetting)
-  uint32_t* sel_words;  // [8] the eligible mask as tagged 16-bit pieces (early start of the FFN kernel)
+  uint32_t* sel_words;  // [kMaxEarlyBlocks][8] the eligible masks as tagged 16-bit pieces (early start of the FFN kernel)
 };
 
 struct SelectArgs {
@@ -68,6 +69,13 @@ struct SelectArgs {
   acm_block_stats* stats_out;    // may be null
   long long* dbg;                // optional time stamps in ns (debugging aid)
 };
+
+// A batch of verification blocks stacked along the node axis: block b owns rows off[b] .. off[b+1]-1.
+struct BatchDesc {
+  int n_blocks;
+  int off[kMaxNodes + 1];
+};
+constexpr int kMaxEarlyBlocks = 8;   // blocks whose eligible sets the FFN kernel can poll for (8 tagged words each)
 
 struct RouteArgs {
   const float* logits;
@@ -114,6 +122,10 @@ cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s
 cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
                                 const uint32_t* mask_override, int T, int E, int k, bool pdl, cudaStream_t s);
 int route_ctas(int T);   // grid size of launch_select_route
+// the same for a batch of blocks: one CTA per block; the per-block outputs of `sa` (mask, unpruned, count,
+// demand [kMaxExperts each], stats) are arrays over the blocks, ra.sel_flag holds 8 words per block
+cudaError_t launch_select_route_batch(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
+                                      const BatchDesc& bd, int E, int k, bool pdl, cudaStream_t s);
 // routes given by the caller -> activated mask, weight table (both cleared first) and cleared `ready`
 cudaError_t launch_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask, float* wtab,
                                    int32_t* ready, int T, int E, int k, cudaStream_t s);
@@ -145,6 +157,7 @@ struct FfnLaunch {
   // first tile is finalised, after a full dependency wait.
   const uint32_t* sel_flag;
   int32_t sel_epoch;
+  int sel_blocks;            // blocks of a batch (1..kMaxEarlyBlocks): eight words each, the work list is their union
   float* out;                // [T,H], accumulated into (zeroed by the caller)
   int32_t* status;
   int grid;

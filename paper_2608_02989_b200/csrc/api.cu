@@ -208,7 +208,7 @@ acm_status check_block_args(const acm_ctx* c, int layer, int T, bool need_weight
 // One FFN launch over work list `li` (0 = resident + shared, 1 = staged).
 acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li, float* out, cudaStream_t s,
                         const uint32_t* res_dev = nullptr, acm_block_stats* stats_dev = nullptr, bool pdl_ok = false,
-                        int32_t early_epoch = 0, const uint32_t* only = nullptr) {
+                        int32_t early_epoch = 0, const uint32_t* only = nullptr, int n_blocks = 0) {
   const acm_model_desc& d = c->desc;
   const int n_pad = (T + 15) / 16 * 16;
   acm_status st = ensure_h_maps(c, n_pad);
@@ -237,7 +237,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   p.hbuf = static_cast<char*>(c->ws.hbuf) + static_cast<size_t>(li) * kMaxSlots * kMaxNodes * d.inter * 2;
   p.ready = c->ws.ready + li * kMaxSlots;
   p.frag = c->ws.frag; p.frag_flag = c->ws.frag_flag;
-  p.sel_flag = nullptr; p.sel_epoch = 0;
+  p.sel_flag = nullptr; p.sel_epoch = 0; p.sel_blocks = n_blocks > 0 ? n_blocks : 1;
   if (early_epoch != 0) {
     p.sel_flag = c->ws.sel_words;
     p.sel_epoch = early_epoch;
@@ -268,7 +268,8 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   // Straight after the routing kernel: the few SMs it ran on (or still holds, in an early start) take
   // microseconds longer to accept a CTA of this kernel -- an SM changes hands slowly when the shared-memory
   // split changes -- and one late CTA delays every CTA that exchanges fragments with it.  Leave them out.
-  if (pdl_ok && c->sm_count > route_ctas(T)) p.grid = c->sm_count - route_ctas(T);
+  const int routing_ctas = n_blocks > 0 ? n_blocks : route_ctas(T);   // a batch: one CTA per block
+  if (pdl_ok && c->sm_count > 2 * routing_ctas) p.grid = c->sm_count - routing_ctas;
   ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
   c->launches += 1;
   if (e1) ACM_CUDA(cudaEventRecord(e1, s));
@@ -391,8 +392,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   };
   const size_t o_logits = carve(sizeof(float) * Tm * E), o_probs = carve(sizeof(float) * Tm * E);
   const size_t o_nat = carve(sizeof(int32_t) * Tm * k), o_idx = carve(sizeof(int32_t) * Tm * k);
-  const size_t o_w = carve(sizeof(float) * Tm * k), o_mask = carve(16), o_unpr = carve(16), o_cnt = carve(16);
-  const size_t o_dem = carve(sizeof(float) * kMaxExperts), o_stats = carve(sizeof(acm_block_stats));
+  const size_t o_w = carve(sizeof(float) * Tm * k), o_mask = carve(16 * Tm), o_unpr = carve(16 * Tm), o_cnt = carve(4 * Tm);
+  const size_t o_dem = carve(sizeof(float) * kMaxExperts * Tm), o_stats = carve(sizeof(acm_block_stats) * Tm);
   // the FFN kernel's routing inputs, contiguous so that one pass clears them: weight table, finished-tile
   // counters, activated mask
   const size_t ffn_in_bytes = sizeof(float) * kMaxExperts * kMaxNodes + sizeof(int32_t) * 2 * kMaxSlots + 16;
@@ -405,7 +406,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_status = carve(16);
   const size_t o_tile = carve(sizeof(int32_t) * kMaxNodes);
   const size_t o_ticket = carve(16);
-  const size_t o_selw = carve(32);
+  const size_t o_selw = carve(32 * kMaxEarlyBlocks);
   const size_t o_natmask = carve(sizeof(uint32_t) * Tm * kMaskWords);
   const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
   if (cudaMalloc(&c->ws_base, off) != cudaSuccess) return fail(ACM_ERR_NOMEM);
@@ -797,6 +798,80 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   return ACM_OK;
 }
 
+acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_blocks, const int32_t* block_offsets,
+                                const float* alpha, const acm_select_params* params, float* out, int32_t* idx_out,
+                                float* w_out, uint32_t* mask_out, uint32_t* activated_out, acm_block_stats* stats,
+                                acm_stream stream) {
+  if (!c || !block_offsets || n_blocks < 1 || n_blocks > kMaxNodes) return ACM_ERR_INVALID;
+  BatchDesc bd;
+  bd.n_blocks = n_blocks;
+  if (block_offsets[0] != 0) return ACM_ERR_INVALID;
+  for (int b = 0; b <= n_blocks; ++b) {
+    if (b > 0 && block_offsets[b] <= block_offsets[b - 1]) return ACM_ERR_INVALID;     // every block has a node
+    if (block_offsets[b] > kMaxNodes) return ACM_ERR_INVALID;
+    bd.off[b] = block_offsets[b];
+  }
+  const int T = block_offsets[n_blocks];
+  acm_status st = check_block_args(c, layer, T, true);
+  if (st != ACM_OK) return st;
+  const Layer& L = c->layers[layer];
+  if (!x || !out || !alpha || !L.gate_up) return ACM_ERR_INVALID;
+  if (reinterpret_cast<uintptr_t>(x) % 16 != 0 || reinterpret_cast<uintptr_t>(out) % 16 != 0) return ACM_ERR_INVALID;
+  st = check_params(params);
+  if (st != ACM_OK) return st;
+  const acm_model_desc& d = c->desc;
+  if (d.dtype != ACM_BF16 || L.has_resident || params->residency != 0) return ACM_ERR_UNSUPPORTED;
+  const int E = d.n_experts, k = d.top_k;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+  // stage 1 over all rows at once (it is per node); also clears `out` and the FFN kernel's routing inputs
+  ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, out,
+                                static_cast<size_t>(T) * d.hidden, c->ws.wtab, c->ffn_in_floats, c->ws.status,
+                                c->ws.probs, c->ws.nat_idx, c->ws.nat_mask, k, c->ws.tile_done, c->pdl, s, nullptr));
+  // stages 2-3: one CTA per block
+  SelectArgs sa;
+  sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
+  sa.n_anchor_nodes = 0; sa.resident = nullptr; sa.prm = *params;
+  sa.mask_out = c->ws.mask; sa.unpruned_out = c->ws.unpruned; sa.count_out = c->ws.count;
+  sa.demand_out = c->ws.demand; sa.stats_out = c->ws.stats;
+  sa.dbg = nullptr;
+  RouteArgs ra = {};
+  ra.logits = c->ws.logits; ra.mask = c->ws.mask; ra.idx_out = c->ws.idx; ra.w_out = c->ws.w;
+  ra.weighting = d.weighting; ra.routed_scale = d.routed_scale;
+  ra.act_mask = c->ws.act_mask; ra.wtab = c->ws.wtab;
+  // early start of the FFN kernel on the union of the blocks' eligible sets (it polls eight words per block)
+  const bool early = n_blocks <= kMaxEarlyBlocks && !c->split_phases && c->early_start;
+  int32_t early_epoch = 0;
+  if (early) {
+    early_epoch = ++c->epoch;
+    if ((early_epoch & 0xffff) == 0) early_epoch = ++c->epoch;
+    if (early_epoch <= 0) early_epoch = c->epoch = 1;
+    ra.sel_flag = c->ws.sel_words;
+    ra.sel_epoch = early_epoch;
+  }
+  ACM_CUDA(launch_select_route_batch(c->ws.nat_mask, sa, ra, bd, E, k, c->pdl, s));
+  c->launches += 2;
+  // stage 4 once over all rows: an expert activated by several blocks is streamed once
+  st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, nullptr, true, early_epoch, nullptr, n_blocks);
+  if (st != ACM_OK) return st;
+
+  const size_t tk = static_cast<size_t>(T) * k;
+  if (idx_out) ACM_CUDA(cudaMemcpyAsync(idx_out, c->ws.idx, sizeof(int32_t) * tk, cudaMemcpyDeviceToDevice, s));
+  if (w_out) ACM_CUDA(cudaMemcpyAsync(w_out, c->ws.w, sizeof(float) * tk, cudaMemcpyDeviceToDevice, s));
+  if (mask_out) {
+    if (mask_words(E) == kMaskWords) {
+      ACM_CUDA(cudaMemcpyAsync(mask_out, c->ws.mask, sizeof(uint32_t) * kMaskWords * n_blocks, cudaMemcpyDeviceToDevice, s));
+    } else {
+      ACM_CUDA(cudaMemcpy2DAsync(mask_out, sizeof(uint32_t) * mask_words(E), c->ws.mask, sizeof(uint32_t) * kMaskWords,
+                                 sizeof(uint32_t) * mask_words(E), n_blocks, cudaMemcpyDeviceToDevice, s));
+    }
+  }
+  if (activated_out)
+    ACM_CUDA(cudaMemcpyAsync(activated_out, c->ws.act_mask, sizeof(uint32_t) * mask_words(E), cudaMemcpyDeviceToDevice, s));
+  if (stats) ACM_CUDA(cudaMemcpyAsync(stats, c->ws.stats, sizeof(acm_block_stats) * n_blocks, cudaMemcpyDefault, s));
+  return ACM_OK;
+}
+
 namespace {
 acm_status ensure_host_path(acm_ctx* c) {
   if (c->h2d_stream) return ACM_OK;
@@ -1021,7 +1096,7 @@ acm_status acm_device_status(acm_ctx* c, acm_stream stream) {
     ACM_CUDA(cudaMemset(c->ws.frag, 0, c->frag_bytes));
     ACM_CUDA(cudaMemset(c->ws.frag_flag, 0, c->flag_bytes));
     ACM_CUDA(cudaMemset(c->ws.ticket, 0, 16));
-    ACM_CUDA(cudaMemset(c->ws.sel_words, 0, 32));
+    ACM_CUDA(cudaMemset(c->ws.sel_words, 0, 32 * kMaxEarlyBlocks));
     c->epoch = 0;
     ACM_CUDA(cudaMemset(c->ws.tile_done, 0, sizeof(int32_t) * kMaxNodes));
   }

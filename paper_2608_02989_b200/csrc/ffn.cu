@@ -138,7 +138,7 @@ struct __align__(8) Barriers {
   float wd[kMaxNodes];          // combine weights of the expert being finalised
   int32_t entry[kMaxSlots];     // this launch's work list: make_entry(source, index) of every activated slot
   int32_t expert[kMaxSlots];    // routed expert id of the slot (-1: shared expert)
-  uint32_t sel_half[2 * kMaskWords];   // early start: the eligible mask in 16-bit pieces
+  uint32_t sel_half[4 * kMaskWords];   // early start: the eligible mask in 16-bit pieces (second half: blocks 4..7 of a batch)
   Plan plan;                    // this launch's work plan
 };
 
@@ -367,6 +367,7 @@ struct FfnArgs {
   int32_t* frag_flag;
   const uint32_t* sel_flag;
   int32_t sel_epoch;
+  int sel_blocks;
   float* out;
   int32_t* status;
   int phase_mask;
@@ -508,7 +509,29 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     // eight tagged words (16 mask bits under the 16-bit tag of this call), each polled by its own thread --
     // of warp 2, which has nothing else to do yet, so that the poll runs beside the set-up above
     bool timed_out = false;
-    if (threadIdx.x >= 64 && threadIdx.x < 64 + 2 * kMaskWords) {
+    if (p.sel_blocks > 1) {
+      // a batch of blocks: eight words per block, one thread each (warps 2 and 3: four blocks per warp); the
+      // work list is the union of the blocks' sets
+      if (threadIdx.x >= 64 && threadIdx.x < 128) {
+        const int j = threadIdx.x - 64;
+        const bool mine = j < 2 * kMaskWords * p.sel_blocks;
+        bool seen = true;
+        uint32_t v = 0;
+        if (mine) {
+          const uint32_t tag = static_cast<uint32_t>(p.sel_epoch) & 0xffffu;
+          const unsigned long long t0 = global_timer();
+          do {
+            asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.sel_flag + j) : "memory");
+            seen = (v >> 16) == tag;
+          } while (!seen && global_timer() - t0 < kTimeoutNs);
+        }
+        timed_out = !seen;
+        uint32_t bits = (mine && seen) ? (v & 0xffffu) : 0u;
+        bits |= __shfl_xor_sync(0xffffffffu, bits, 8);
+        bits |= __shfl_xor_sync(0xffffffffu, bits, 16);
+        if (lane < 2 * kMaskWords) bars->sel_half[(j >> 5) * 2 * kMaskWords + lane] = bits;
+      }
+    } else if (threadIdx.x >= 64 && threadIdx.x < 64 + 2 * kMaskWords) {
       const int i = threadIdx.x - 64;
       bool seen = false;
       uint32_t v = 0;
@@ -537,7 +560,13 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   int n_routed = 0;
 #pragma unroll
   for (int wd = 0; wd < kMaskWords; ++wd) {
-    const uint32_t act = early ? (bars->sel_half[2 * wd] | (bars->sel_half[2 * wd + 1] << 16)) : p.act_mask[wd];
+    uint32_t act;
+    if (early) {
+      act = bars->sel_half[2 * wd] | (bars->sel_half[2 * wd + 1] << 16);
+      if (p.sel_blocks > 1) act |= bars->sel_half[2 * kMaskWords + 2 * wd] | (bars->sel_half[2 * kMaskWords + 2 * wd + 1] << 16);
+    } else {
+      act = p.act_mask[wd];
+    }
     const uint32_t res = p.resident ? p.resident[wd] : 0xffffffffu;
     am[wd] = (p.li == 0 ? act & res : act & ~res) & p.only[wd];
     n_routed += __popc(am[wd]);
@@ -1108,7 +1137,7 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   for (int w = 0; w < 4; ++w) a.only[w] = L.only[w];
   a.stats = L.stats; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
   a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag;
-  a.sel_flag = L.sel_flag; a.sel_epoch = L.sel_epoch;
+  a.sel_flag = L.sel_flag; a.sel_epoch = L.sel_epoch; a.sel_blocks = L.sel_blocks;
   a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask; a.trace = L.trace;
   void* args[] = {const_cast<FfnMaps*>(&maps), const_cast<CUtensorMap*>(&x_map), const_cast<CUtensorMap*>(&h_map),
                   const_cast<CUtensorMap*>(&hs_map), &a};

@@ -638,6 +638,16 @@ __device__ __forceinline__ void publish_routes(uint32_t* act_mask, float* wtab, 
   if (has) wtab[static_cast<size_t>(e) * kMaxNodes + t] = w;
 }
 
+// the same sets OR-ed into a mask in shared memory (what one block of a batch activates by itself)
+__device__ __forceinline__ void publish_routes_local(uint32_t* s_act, int k, int lane, int e) {
+  const bool has = lane < k && e >= 0;
+#pragma unroll
+  for (int wd = 0; wd < kMaskWords; ++wd) {
+    const unsigned bits = __reduce_or_sync(0xffffffffu, (has && (e >> 5) == wd) ? 1u << (e & 31) : 0u);
+    if (lane == wd && bits) atomicOr(s_act + wd, bits);
+  }
+}
+
 __global__ void __launch_bounds__(kSelThreads) k_select(SelectArgs a, int T, int E, int k) {
   __shared__ StageSmem sm;
   stage_select(a, sm, T, E, k, nullptr, true);
@@ -766,6 +776,61 @@ k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uin
   if (ra.dbg && tid == 0) ra.dbg[4] = time_ns();
 }
 
+// Several verification blocks in one launch: CTA b owns block b (the rows bd.off[b] .. bd.off[b+1]-1 of
+// every per-node array).  Its warps 0-3 run the selection on the block's own nodes (Eq. 3-7 see nothing
+// of the other blocks; the block's first row is its root), then all of its warps route the block's
+// nodes inside that set (Eq. 2).  The FFN kernel's inputs are shared by all blocks: the activated mask
+// is OR-ed into by everyone, the weight table is indexed by the row in the stacked batch.  Block b's
+// eligible set is published in its own eight tagged words, ra.sel_flag + 8 b.
+__global__ void __launch_bounds__(32 * kRouteNodesPerCta)
+k_select_route_batch(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, BatchDesc bd, int E, int k) {
+  __shared__ StageSmem sm;
+  __shared__ uint32_t s_act[kMaskWords];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
+  const int b = blockIdx.x;
+  const int t_lo = bd.off[b], T = bd.off[b + 1] - t_lo;
+  griddep_launch_dependents();
+  griddep_wait();
+  if (tid < kMaskWords) s_act[tid] = 0u;
+  SelectArgs mine = sa;
+  mine.probs += static_cast<size_t>(t_lo) * E;
+  mine.alpha += t_lo;
+  mine.anchor_nodes = nullptr;
+  mine.n_anchor_nodes = 0;
+  mine.mask_out += b * kMaskWords;
+  if (mine.unpruned_out) mine.unpruned_out += b * kMaskWords;
+  mine.count_out += b;
+  if (mine.demand_out) mine.demand_out += static_cast<size_t>(b) * kMaxExperts;
+  if (mine.stats_out) mine.stats_out += b;
+  mine.dbg = nullptr;
+  if (tid < kSelThreads)
+    stage_select(mine, sm, T, E, k, natmask_g + static_cast<size_t>(t_lo) * kMaskWords, true,
+                 ra.sel_flag ? ra.sel_flag + 2 * kMaskWords * b : nullptr, static_cast<uint32_t>(ra.sel_epoch) & 0xffffu);
+  __syncthreads();
+  uint32_t mask_w[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) mask_w[c] = sm.Sp[c];
+  for (int t = t_lo + warp; t < t_lo + T; t += n_warps) {
+    float z[4];
+    load_logit_row(ra.logits, t, E, lane, z);
+    int e;
+    float w;
+    route_node(z, mask_w, E, k, lane, ra.weighting, ra.routed_scale, e, w);
+    if (lane < k) {
+      ra.idx_out[static_cast<size_t>(t) * k + lane] = e;
+      ra.w_out[static_cast<size_t>(t) * k + lane] = w;
+    }
+    publish_routes(ra.act_mask, ra.wtab, t, k, lane, e, w);
+    publish_routes_local(s_act, k, lane, e);
+  }
+  __syncthreads();
+  if (tid == 0 && mine.stats_out) {      // this block's own activated experts (the batch's union is the mask)
+    int n = 0;
+    for (int wd = 0; wd < kMaskWords; ++wd) n += __popc(s_act[wd]);
+    mine.stats_out->n_activated = n;
+  }
+}
+
 // Routes given by the caller (acm_expert_ffn) -> the FFN kernel's inputs.  One CTA.
 __global__ void __launch_bounds__(512) k_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask,
                                                          float* wtab, int32_t* ready, int T, int E, int k) {
@@ -852,6 +917,22 @@ cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, 
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, k_select_route, nat_mask, sa, ra, mask_override, T, E, k);
+}
+
+cudaError_t launch_select_route_batch(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
+                                      const BatchDesc& bd, int E, int k, bool pdl, cudaStream_t s) {
+  cudaLaunchAttribute attr[1];
+  set_pdl_attr(attr);
+  cudaLaunchConfig_t cfg = {};
+  int widest = 1;
+  for (int b = 0; b < bd.n_blocks; ++b) widest = bd.off[b + 1] - bd.off[b] > widest ? bd.off[b + 1] - bd.off[b] : widest;
+  const int warps = widest < 4 ? 4 : widest > kRouteNodesPerCta ? kRouteNodesPerCta : widest;   // at least the four selection warps
+  cfg.gridDim = dim3(bd.n_blocks);
+  cfg.blockDim = dim3(32 * warps);
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, k_select_route_batch, nat_mask, sa, ra, bd, E, k);
 }
 
 cudaError_t launch_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask, float* wtab,

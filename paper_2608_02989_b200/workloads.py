@@ -101,6 +101,26 @@ def tree_depths(cfg: BlockConfig, layer: int = 0) -> torch.Tensor:
     return torch.sort(d).values.to(torch.int32)
 
 
+def batch_tree_depths(cfg: BlockConfig, n_blocks: int):
+    """A batch of `n_blocks` verification blocks that together hold cfg.n_nodes nodes (sizes differ by at
+    most one node, larger blocks first): returns (offsets [n_blocks+1], depths [T] int32).  Every block is
+    a tree of its own, built like tree_depths: root first, every level 1..min(D, size-1) occupied, the
+    rest uniform over the levels (seeded per block), sorted by depth."""
+    T = cfg.n_nodes
+    if not 1 <= n_blocks <= T:
+        raise ValueError("n_blocks must be between 1 and the number of nodes")
+    sizes = [T // n_blocks + (1 if b < T % n_blocks else 0) for b in range(n_blocks)]
+    offsets, depths = [0], []
+    for b, n in enumerate(sizes):
+        D = min(cfg.max_depth, n - 1)
+        g = _gen(cfg.seed(0) + 600_000 + b, "cpu")
+        extra = torch.randint(1, D + 1, (n - 1 - D,), generator=g) if n - 1 - D > 0 else torch.zeros(0, dtype=torch.long)
+        d = torch.cat([torch.zeros(1, dtype=torch.long), torch.arange(1, D + 1), extra])
+        depths.append(torch.sort(d).values.to(torch.int32))
+        offsets.append(offsets[-1] + n)
+    return offsets, torch.cat(depths)
+
+
 def hidden_states(cfg: BlockConfig, layer: int, device="cpu") -> torch.Tensor:
     """x [T, H], N(0, 1), independent per layer."""
     g = _gen(cfg.seed(layer) + 100_000, device)

@@ -620,3 +620,76 @@ def test_expert_pool_smaller_than_the_routed_union_runs_in_waves():
     assert (ps["hits"], ps["misses"]) == (tot_hits, tot_misses)
     assert ps["slot_expert"] == model.slot_expert
     ctx.close()
+
+
+def _batch_reference(cfg, w, x, offsets, depths, params_kw):
+    """The oracle knows single blocks only: a batch is, by definition, every block verified by itself."""
+    p = wl.commitment_table(cfg)
+    alphas, refs = [], []
+    for b in range(len(offsets) - 1):
+        lo, hi = offsets[b], offsets[b + 1]
+        a = oracle.node_weights(depths[lo:hi].numpy(), p.numpy())
+        refs.append(oracle.moe_verify(x[lo:hi], w["w_router"], w["router_bias"], w["gate_up"], w["down"], a,
+                                      cfg.top_k, oracle.SelectParams(**params_kw), weighting=cfg.weighting,
+                                      shared_gate_up=w["shared_gate_up"], shared_down=w["shared_down"],
+                                      with_ffn=False))
+        alphas.append(a)
+    return np.concatenate(alphas), refs
+
+
+@pytest.mark.parametrize("c,n_blocks,params_kw", [(3, 4, {}), (3, 7, {}), (3, 2, {"fixed_budget": 12}), (4, 3, {}),
+                                                  (3, 12, {}), (2, 32, {}), (3, 1, {})])
+def test_multi_block_batch_equals_every_block_verified_alone(c, n_blocks, params_kw):
+    """Several verification blocks in one call: each block's eligible set, routes and statistics are those of
+    the oracle run on that block alone (ragged block sizes, 1 to 32 blocks, with and without the FFN
+    kernel's early start, shared experts), the FFN output rows match the oracle's, and the activated mask is
+    the union over the blocks."""
+    cfg = wl.CONFIGS[c]
+    ctx = _ctx(cfg)
+    w = wl.layer_weights(cfg, 0, DEV)
+    _set_weights(ctx, w, 0)
+    x = wl.hidden_states(cfg, 0, DEV)
+    offsets, depths = wl.batch_tree_depths(cfg, n_blocks)
+    assert offsets[-1] == cfg.n_nodes and len(set(np.diff(offsets))) <= 2
+    alpha_ref, refs = _batch_reference(cfg, w, x, offsets, depths, params_kw)
+    p = wl.commitment_table(cfg)
+    alpha = torch.cat([acm.node_weights(depths[offsets[b]:offsets[b + 1]], p) for b in range(n_blocks)])
+    np.testing.assert_array_equal(alpha.numpy(), alpha_ref)
+    for rep in range(2):                  # the second call runs on the workspace the first one left behind
+        out, idx, wt, mask, act, stats = ctx.moe_verify_batch(0, x, offsets, alpha.to(DEV),
+                                                              acm.SelectParams(**params_kw), want=True)
+        assert ctx.device_status() == acm.OK
+        union = set()
+        for b, ref in enumerate(refs):
+            lo, hi = offsets[b], offsets[b + 1]
+            np.testing.assert_array_equal(_u32(mask[b]), ref["mask"])
+            np.testing.assert_array_equal(idx[lo:hi].cpu().numpy(), ref["idx"])
+            np.testing.assert_allclose(wt[lo:hi].cpu().numpy(), ref["w"], rtol=1e-5, atol=1e-7)
+            st = acm.stats_dict(stats[b])
+            assert st["n_eligible_pruned"] == ref["count"]
+            for key in ("n_anchor", "n_er", "n_eligible", "n_natural_union", "displaced_aS"):
+                assert st[key] == ref["stats"][key]
+            mine = set(ref["idx"].ravel().tolist()) - {-1}
+            assert st["n_activated"] == len(mine)
+            union |= mine
+        assert mask_to_set(_u32(act), cfg.n_experts) == union
+        rows = sorted({0, offsets[1] - 1, offsets[min(1, n_blocks - 1)], cfg.n_nodes // 2, cfg.n_nodes - 1})
+        ref_idx = np.concatenate([r["idx"] for r in refs])
+        ref_w = np.concatenate([r["w"] for r in refs])
+        ffn = oracle.expert_ffn(_take(x, rows), ref_idx[rows], ref_w[rows], w["gate_up"], w["down"],
+                                w["shared_gate_up"], w["shared_down"])
+        _ffn_check(_take(out, rows), ffn, f"C{c} batch of {n_blocks}")
+    ctx.close()
+
+
+def test_multi_block_batch_rejects_bad_descriptions():
+    cfg = wl.scaled(wl.CONFIGS[3], inter=128)
+    ctx = _ctx(cfg)
+    w = wl.layer_weights(cfg, 0, DEV)
+    _set_weights(ctx, w, 0)
+    x = wl.hidden_states(cfg, 0, DEV)
+    alpha = torch.ones(cfg.n_nodes, device=DEV)
+    for offs in ([0, 0, 64], [1, 64], [0, 40, 30, 64], [0, 65], [0]):
+        with pytest.raises(acm.AcmError):
+            ctx.moe_verify_batch(0, x[: max(1, min(offs[-1], 64))], offs, alpha)
+    ctx.close()
