@@ -43,6 +43,10 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-natural", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--selector", default="acceptmoe", choices=["acceptmoe", "acceptmoe-b", "count-b", "moe-spec"],
+                    help="eligible-set policy of the restricted path: the paper's self-sizing selector (default), its "
+                         "fixed-budget variant, or the fixed-budget baselines of Section 4.1 (votes / summed router mass)")
+    ap.add_argument("--budget", type=int, default=22, help="B0 of the fixed-budget selectors")
     ap.add_argument("--batch", type=int, default=0,
                     help="supplementary run: B > 1 verification blocks per call (they share the config's nodes and "
                          "one pass over the expert weights) against the same blocks verified one call each")
@@ -326,11 +330,20 @@ def run_acm(args, world, rank, local):
     xs = torch.stack([wl.hidden_states(cfg, l + 1000 * rank, dev) for l in range(L)])       # [L,T,H]
     depth, p = wl.tree_depths(cfg), wl.commitment_table(cfg)
     alpha = acm.node_weights(depth, p)
+    if args.selector in ("count-b", "moe-spec"):
+        alpha = torch.ones_like(alpha)           # the baselines weigh every node alike
     alpha_dev = alpha.to(dev)
     outs = torch.zeros(L, T, H, dtype=torch.float32, device=dev)
     stats = torch.zeros(L, 12, dtype=torch.int32, device=dev)
     full = torch.full((ctx.words,), -1, dtype=torch.int32, device=dev)
-    params = acm.SelectParams()
+    params = {"acceptmoe": acm.SelectParams(),
+              "acceptmoe-b": acm.SelectParams(fixed_budget=args.budget),
+              "count-b": acm.SelectParams(demand=2, use_anchors=0, fixed_budget=args.budget),
+              "moe-spec": acm.SelectParams(demand=1, use_anchors=0, fixed_budget=args.budget)}[args.selector]
+    selector_name = {"acceptmoe": "restricted (AcceptMoE) routing",
+                     "acceptmoe-b": f"restricted routing, AcceptMoE-B with B0={args.budget}",
+                     "count-b": f"restricted routing, Count-B baseline with B0={args.budget}",
+                     "moe-spec": f"restricted routing, MoE-Spec baseline with B0={args.budget}"}[args.selector]
     stream = torch.cuda.current_stream()
     sp = ctypes.c_void_p(stream.cuda_stream)
     lib, h = ctx.lib, ctx.handle
@@ -451,7 +464,7 @@ def run_acm(args, world, rank, local):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": f"C{cfg.index} {cfg.name}-shaped stack, restricted (AcceptMoE) routing",
+        "config": {"workload": f"C{cfg.index} {cfg.name}-shaped stack, {selector_name}",
                    "hidden": H, "n_experts": E, "top_k": k, "inter": cfg.inter, "n_shared": cfg.n_shared,
                    "n_nodes": T, "layers": L, "physical_layers": L_phys,
                    "l2": f"inputs larger than L2: {L_phys} distinct layers, "

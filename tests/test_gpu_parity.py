@@ -106,7 +106,8 @@ SELECT_MODES = [
     dict(demand=2),
     dict(use_anchors=0),
     dict(fixed_budget=20),
-    dict(demand=1, use_anchors=0, fixed_budget=12),
+    dict(demand=1, use_anchors=0, fixed_budget=12),     # MoE-Spec (with uniform node weights, rep 5)
+    dict(demand=2, use_anchors=0, fixed_budget=16),     # Count-B
     dict(ceil_guard=0.0),
     dict(residency=1),
     dict(residency=1, max_remove=2),
