@@ -120,7 +120,11 @@ acm_status acm_destroy(acm_ctx* ctx);
 /* Registers (borrows) the device weights of one layer:
  *   w_router [E,H]; router_bias [E] float or NULL; w_gate_up [E,2I,H] (rows 0..I-1 gate,
  *   I..2I-1 up); w_down [E,H,I]; shared_gate_up [n_shared,2I,H] and shared_down
- *   [n_shared,H,I] (NULL when n_shared == 0).  bf16 expert tensors must be 16-byte aligned. */
+ *   [n_shared,H,I] (NULL when n_shared == 0).  bf16 expert tensors must be 16-byte aligned.
+ *   The weights are constants to the library: their contents must be complete on the device
+ *   when this call is made and must not be written while a call that uses the layer is enqueued or
+ *   running (the router rows are fetched ahead of stream order, while the kernel before is still
+ *   draining).  To change them, synchronise the stream, write, and register them again. */
 acm_status acm_set_layer_weights(acm_ctx* ctx, int layer, const void* w_router,
                                  const float* router_bias, const void* w_gate_up,
                                  const void* w_down, const void* shared_gate_up,

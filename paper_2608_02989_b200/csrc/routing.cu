@@ -220,8 +220,39 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
   griddep_launch_dependents();
   if (dbg && tid == 0) atomicMax(reinterpret_cast<unsigned long long*>(dbg + 17), static_cast<unsigned long long>(time_ns()));
   if (dbg && tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) dbg[16] = time_ns();
+
+  // Staging: the 4 x-rows and 8 router rows of this tile, in n_chunks pieces along h.  One thread
+  // per row issues its pieces as bulk copies; piece c of all rows completes on barrier c.  The
+  // router rows are requested BEFORE the dependency wait: the weights are constants of the layer
+  // (nothing enqueued after they were registered may write them), so a CTA that is resident while the
+  // kernel before it drains already has them on the way.  The x rows follow the wait.
+  __shared__ __align__(8) unsigned long long chunk_bar[4];
+  const unsigned chunk_bytes = static_cast<unsigned>(H * sizeof(Elem)) / n_chunks;
+  if (tid == 0) {
+    for (int c = 0; c < n_chunks; ++c) mbar_init(&chunk_bar[c], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (tid == 0)
+    for (int c = 0; c < n_chunks; ++c) mbar_arrive_expect_tx(&chunk_bar[c], (kRT + kRE) * chunk_bytes);
+  if (tid >= kRT && tid < kRT + kRE) {
+    const int row = tid - kRT;
+    const unsigned char* src = reinterpret_cast<const unsigned char*>(wr + static_cast<size_t>(min(e0 + row, E - 1)) * H);
+    unsigned char* dst = ws + static_cast<size_t>(row) * row_bytes;
+    for (int c = 0; c < n_chunks; ++c)
+      bulk_load(dst + static_cast<size_t>(c) * chunk_bytes, src + static_cast<size_t>(c) * chunk_bytes, chunk_bytes,
+                &chunk_bar[c]);
+  }
   griddep_wait();
   if (dbg && tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) dbg[13] = time_ns();
+  if (tid < kRT) {
+    const int row = tid;
+    const unsigned char* src = reinterpret_cast<const unsigned char*>(x + static_cast<size_t>(min(t0 + row, T - 1)) * H);
+    unsigned char* dst = xs + static_cast<size_t>(row) * row_bytes;
+    for (int c = 0; c < n_chunks; ++c)
+      bulk_load(dst + static_cast<size_t>(c) * chunk_bytes, src + static_cast<size_t>(c) * chunk_bytes, chunk_bytes,
+                &chunk_bar[c]);
+  }
 
   // zero the FFN output buffer (accumulated into by the FFN kernel) and the FFN kernel's routing
   // inputs (activated mask, weight table, finished-tile counters), spread over the grid
@@ -236,33 +267,6 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
       float4* z4 = reinterpret_cast<float4*>(zero_buf2);
       for (size_t i = b * blockDim.x + tid; i < zero_floats2 / 4; i += nb * blockDim.x) z4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
-  }
-
-  // Staging: the 4 x-rows and 8 router rows of this tile, in n_chunks pieces along h.  One thread
-  // per row issues its pieces as bulk copies; piece c of all rows completes on barrier c.
-  __shared__ __align__(8) unsigned long long chunk_bar[4];
-  const unsigned chunk_bytes = static_cast<unsigned>(H * sizeof(Elem)) / n_chunks;
-  if (tid == 0) {
-    for (int c = 0; c < n_chunks; ++c) mbar_init(&chunk_bar[c], 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
-  if (tid == 0)
-    for (int c = 0; c < n_chunks; ++c) mbar_arrive_expect_tx(&chunk_bar[c], (kRT + kRE) * chunk_bytes);
-  if (tid < kRT + kRE) {
-    const int row = tid;
-    const unsigned char* src;
-    unsigned char* dst;
-    if (row < kRT) {
-      src = reinterpret_cast<const unsigned char*>(x + static_cast<size_t>(min(t0 + row, T - 1)) * H);
-      dst = xs + static_cast<size_t>(row) * row_bytes;
-    } else {
-      src = reinterpret_cast<const unsigned char*>(wr + static_cast<size_t>(min(e0 + row - kRT, E - 1)) * H);
-      dst = ws + static_cast<size_t>(row - kRT) * row_bytes;
-    }
-    for (int c = 0; c < n_chunks; ++c)
-      bulk_load(dst + static_cast<size_t>(c) * chunk_bytes, src + static_cast<size_t>(c) * chunk_bytes, chunk_bytes,
-                &chunk_bar[c]);
   }
 
   const int q = tid % Q;            // which EPT-wide group of the 32 partial sums
