@@ -451,6 +451,29 @@ def run_acm(args, world, rank, local):
         e2e = {"value": world * L * args.steps / dt, "unit": UNIT,
                "h2d_bytes_per_step": L * (T * H * cfg.elt_bytes + T * 4), "d2h_bytes_per_step": L * T * H * 4}
 
+    # Per-stage device times (an instrumented pass after the timed ones): the kernels stamp a global clock,
+    # the launch sequence and its overlaps stay as they are.  One sample per layer, each taken with that
+    # layer as the last call of a pass over the whole stack (so it runs behind its usual predecessor).
+    stage_us = None
+    if rank == 0 and not resident and cfg.dtype == "bf16":
+        ctx.stage_timing(True)
+        acc = {}
+        n_samples = min(L, 16)
+        for j in np.linspace(0, L - 1, n_samples).astype(int):
+            order = list(range(j + 1, L)) + list(range(0, j + 1))
+            for _ in range(2):
+                for l in order:
+                    rc = lib.acm_moe_verify(*calls_sel[l])
+                    if rc:
+                        raise acm.AcmError(rc, "acm_moe_verify")
+            for key, v in ctx.stage_times().items():
+                acc[key] = acc.get(key, 0.0) + v / n_samples
+        ctx.stage_timing(False)
+        stage_us = {key: round(v, 2) for key, v in acc.items()}
+        stage_us["note"] = ("in-kernel stamps, mean over %d layers: router = dependency release to selection start; "
+                            "select; route; ffn = first role start to last tile (it starts on the eligible set while "
+                            "the routes are made); whole = start of router to end of ffn" % n_samples)
+
     if rank != 0:
         return
     peak, peak_kind = read_peaks()
@@ -478,6 +501,7 @@ def run_acm(args, world, rank, local):
                      "kernel": "k_ffn_bf16", "us_per_launch": ffn_us, "launches_timed": ffn_n,
                      "timed_every": period,
                      "algorithmic_bytes_per_launch": alg_per_launch},
+        "stage_us": stage_us,
         "natural_union_path": nat,
         "e2e": e2e,
         "gpu_launches": int(launches),

@@ -251,6 +251,22 @@ acm_status acm_h2d_bytes(acm_ctx* ctx, uint64_t* bytes_out /*host*/, int reset);
 acm_status acm_ffn_timing(acm_ctx* ctx, int enable, int capacity);
 acm_status acm_ffn_time_ms(acm_ctx* ctx, float* total_ms, int32_t* launches);
 
+/* Per-stage device times of the fused call, from time stamps the kernels themselves take (one global
+ * nanosecond clock) -- the launch sequence, its overlaps included, stays as it is.  acm_stage_timing
+ * switches the stamps on or off (it synchronises the device; on costs a few stores per CTA).
+ * acm_stage_times synchronises and reports, for the LAST acm_moe_verify call on a bf16 layer without a
+ * residency, us_out [5] (host, microseconds):
+ *   [0] stage 1: from the router kernel passing its dependency wait (everything before it in the
+ *       stream is complete) to the start of the selection -- logits, softmax, natural top-k;
+ *   [1] stage 2: the selection (Eq. 4-7), until the eligible set is published;
+ *   [2] stage 3: the routes (Eq. 2) and the FFN kernel's routing inputs;
+ *   [3] stage 4: the FFN kernel from its first CTA's roles starting to its last tile finished -- it
+ *       starts on the eligible set while stage 3 runs, so [0..3] overlap and do not add up to
+ *   [4] the whole: from the start of [0] to the end of [3].
+ * ACM_ERR_INVALID when the stamps are off or no such call has run. */
+acm_status acm_stage_timing(acm_ctx* ctx, int enable);
+acm_status acm_stage_times(acm_ctx* ctx, double* us_out /*host [5]*/);
+
 /* Number of kernel launches this context has enqueued since creation (host counter). */
 acm_status acm_launch_count(acm_ctx* ctx, uint64_t* launches_out /*host*/);
 

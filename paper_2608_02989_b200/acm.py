@@ -25,7 +25,7 @@ EXPORTS = [
     "acm_node_weights", "acm_router", "acm_select_eligible", "acm_route_restricted",
     "acm_expert_ffn", "acm_moe_verify", "acm_moe_verify_batch", "acm_moe_verify_host", "acm_host_synchronize", "acm_set_resident",
     "acm_set_slot_pool", "acm_pool_stats",
-    "acm_h2d_bytes", "acm_ffn_timing", "acm_ffn_time_ms", "acm_launch_count", "acm_device_status", "acm_status_string",
+    "acm_h2d_bytes", "acm_ffn_timing", "acm_ffn_time_ms", "acm_stage_timing", "acm_stage_times", "acm_launch_count", "acm_device_status", "acm_status_string",
     "acm_expert_ffn_f32_noalloc",
 ]
 NOALLOC_MAX_FLOATS = 1 << 20
@@ -100,6 +100,8 @@ def load_library():
                                    c_void_p, c_int]
     lib.acm_h2d_bytes.argtypes = [c_void_p, POINTER(c_uint64), c_int]
     lib.acm_ffn_timing.argtypes = [c_void_p, c_int, c_int]
+    lib.acm_stage_timing.argtypes = [c_void_p, c_int]
+    lib.acm_stage_times.argtypes = [c_void_p, POINTER(ctypes.c_double)]
     lib.acm_ffn_time_ms.argtypes = [c_void_p, POINTER(c_float), POINTER(c_int32)]
     lib.acm_launch_count.argtypes = [c_void_p, POINTER(c_uint64)]
     lib.acm_device_status.argtypes = [c_void_p, c_void_p]
@@ -334,6 +336,15 @@ class Context:
         ms, n = c_float(0), c_int32(0)
         _check(self.lib.acm_ffn_time_ms(self.handle, byref(ms), byref(n)), "acm_ffn_time_ms")
         return ms.value, n.value
+
+    def stage_timing(self, enable):
+        _check(self.lib.acm_stage_timing(self.handle, int(bool(enable))), "acm_stage_timing")
+
+    def stage_times(self) -> dict:
+        """Device microseconds of the last fused call's stages (they overlap; see acm_stage_times)."""
+        us = (ctypes.c_double * 5)()
+        _check(self.lib.acm_stage_times(self.handle, us), "acm_stage_times")
+        return dict(zip(("router", "select", "route", "ffn", "whole"), [float(v) for v in us]))
 
     def launch_count(self) -> int:
         v = c_uint64(0)

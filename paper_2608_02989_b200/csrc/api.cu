@@ -1079,6 +1079,48 @@ acm_status acm_ffn_time_ms(acm_ctx* c, float* total_ms, int32_t* launches) {
   return ACM_OK;
 }
 
+acm_status acm_stage_timing(acm_ctx* c, int enable) {
+  if (!c) return ACM_ERR_INVALID;
+  ACM_CUDA(cudaDeviceSynchronize());
+  if (enable) {
+    if (!c->trace) {
+      const size_t bytes = sizeof(unsigned long long) * (32 * c->sm_count + 32);
+      if (cudaMalloc(&c->trace, bytes) != cudaSuccess) return ACM_ERR_NOMEM;
+      ACM_CUDA(cudaMemset(c->trace, 0, bytes));
+      c->trace_light = true;       // stamps only: the launch sequence stays exactly as it is
+    }
+  } else if (c->trace) {
+    ACM_CUDA(cudaFree(c->trace));
+    c->trace = nullptr;
+    c->trace_light = false;
+  }
+  return ACM_OK;
+}
+
+acm_status acm_stage_times(acm_ctx* c, double* us_out) {
+  if (!c || !us_out || !c->trace) return ACM_ERR_INVALID;
+  ACM_CUDA(cudaDeviceSynchronize());
+  std::vector<unsigned long long> buf(32 * static_cast<size_t>(c->sm_count) + 32);
+  ACM_CUDA(cudaMemcpy(buf.data(), c->trace, sizeof(unsigned long long) * buf.size(), cudaMemcpyDeviceToHost));
+  const unsigned long long* rt = buf.data() + 32 * static_cast<size_t>(c->sm_count);
+  const unsigned long long t_in = rt[13], t_sel0 = rt[0], t_sel1 = rt[2], t_route = rt[3];
+  if (t_in == 0 || t_sel0 < t_in || t_sel1 < t_sel0 || t_route < t_sel1) return ACM_ERR_INVALID;   // no fused call seen yet
+  unsigned long long ffn0 = ~0ull, ffn1 = 0;
+  for (int cta = 0; cta < c->sm_count; ++cta) {
+    const unsigned long long* row = buf.data() + 32 * static_cast<size_t>(cta);
+    if (row[0] >= t_in && row[0] < ffn0) ffn0 = row[0];          // (older stamps belong to earlier calls)
+    for (int slot = 10; slot <= 11; ++slot)
+      if (row[slot] >= t_in && row[slot] > ffn1) ffn1 = row[slot];
+  }
+  if (ffn1 == 0 || ffn0 == ~0ull || ffn1 < ffn0) return ACM_ERR_INVALID;
+  us_out[0] = 1e-3 * static_cast<double>(t_sel0 - t_in);
+  us_out[1] = 1e-3 * static_cast<double>(t_sel1 - t_sel0);
+  us_out[2] = 1e-3 * static_cast<double>(t_route - t_sel1);
+  us_out[3] = 1e-3 * static_cast<double>(ffn1 - ffn0);
+  us_out[4] = 1e-3 * static_cast<double>(ffn1 - t_in);
+  return ACM_OK;
+}
+
 acm_status acm_launch_count(acm_ctx* c, uint64_t* launches_out) {
   if (!c || !launches_out) return ACM_ERR_INVALID;
   *launches_out = c->launches;

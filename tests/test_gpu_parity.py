@@ -694,3 +694,33 @@ def test_multi_block_batch_rejects_bad_descriptions():
         with pytest.raises(acm.AcmError):
             ctx.moe_verify_batch(0, x[: max(1, min(offs[-1], 64))], offs, alpha)
     ctx.close()
+
+
+def test_stage_times_come_from_device_stamps():
+    cfg = wl.scaled(wl.CONFIGS[3], inter=256)
+    ctx = _ctx(cfg, n_layers=2)
+    with pytest.raises(acm.AcmError):
+        ctx.stage_times()                       # stamps are off
+    ctx.stage_timing(True)
+    with pytest.raises(acm.AcmError):
+        ctx.stage_times()                       # no call yet
+    outs = []
+    for layer in (0, 1):
+        w, x, alpha = _block(cfg, layer)
+        _set_weights(ctx, w, layer)
+        outs.append((x, alpha.to(DEV)))
+    for _ in range(3):
+        for layer in (0, 1):
+            out = ctx.moe_verify(layer, outs[layer][0], outs[layer][1])
+    st = ctx.stage_times()
+    assert ctx.device_status() == acm.OK
+    assert all(v > 0.0 for v in st.values()), st
+    assert st["whole"] >= st["ffn"] and st["whole"] >= st["router"] + st["select"]
+    assert st["whole"] < 1000.0, st
+    ref = ctx.moe_verify(1, outs[1][0], outs[1][1])
+    ctx.stage_timing(False)
+    again = ctx.moe_verify(1, outs[1][0], outs[1][1])
+    np.testing.assert_allclose(again.cpu().numpy(), ref.cpu().numpy(), rtol=1e-3, atol=1e-4)    # same result with stamps on and off
+    with pytest.raises(acm.AcmError):
+        ctx.stage_times()
+    ctx.close()
