@@ -20,6 +20,10 @@
  *     are found on the host before anything is enqueued and leave outputs untouched.
  *     Failures seen by device code (a bounded wait that ran out, a non-finite logit) are
  *     sticky in a status word read by acm_device_status().  Nothing traps, aborts or prints.
+ *   - A context serves one stream at a time (its workspace is shared by its calls), and its calls
+ *     must not be captured into a CUDA graph: every fused call carries a host-side sequence number
+ *     that tags what its kernels hand to one another, so a replay would meet the tags of the run
+ *     before it.
  *   - The caller owns every buffer it passes.  The context borrows weight pointers until
  *     acm_destroy() or the next acm_set_layer_weights() for that layer, and owns its
  *     workspace (allocated in acm_create with cudaMalloc on the current device).
