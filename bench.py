@@ -27,7 +27,7 @@ ROOT = Path(__file__).resolve().parent
 if str(ROOT) not in sys.path:
     sys.path.insert(0, str(ROOT))
 
-DRAM_BYTES_PER_ACTIVATED_EXPERT = {3: (271194112 + 197305344 + 196898304) / 68.0}   # config -> bytes
+DRAM_BYTES_PER_ACTIVATED_EXPERT = {3: (271304192 + 197928448 + 197003776) / 68.0}   # config -> bytes
 METRIC = "verify_blocks_per_s_per_moe_layer"
 UNIT = "layer-blocks/s"
 
