@@ -414,7 +414,7 @@ def run_acm(args, world, rank, local):
     if not args.no_natural:
         ms_n, _, ffn_ms_n, ffn_n_n = timed(calls_nat, args.steps, 3, True)
         st_n = stats.cpu().numpy()
-        nat_bytes = (st_n[:, 4] + cfg.n_shared) * expert_bytes + T * H * 6
+        nat_bytes = (st_n[:, 4].astype(float) + cfg.n_shared) * expert_bytes + T * H * 6
         nat_bytes = float(nat_bytes[sampled_layers(args.steps)].mean()) if not resident else float(nat_bytes.mean())
         nat = {"value": world * L * args.steps / (ms_n * 1e-3), "unit": UNIT, "ms_per_step": ms_n / args.steps,
                "mean_activated_experts": float(st_n[:, 4].mean()),
