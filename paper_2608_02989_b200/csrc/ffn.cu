@@ -802,21 +802,33 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         // activation producer: once every activation tile of this expert group is stored, add the
         // activation chunk of each down stage to the barrier the weight producer has armed (or will arm)
         bool good = true;
-        if (lane == 0) {
+        {
+          // The experts whose activation tiles this CTA's share of the segment reads (one finished-tile counter
+          // per expert), polled side by side, one lane each: from the first to the last K-chunk of the share, or
+          // the whole group if the share runs on into the next output tile.
+          const SegRange& rg = bars->plan.range[si];
+          const unsigned n_units = rg.u_end - rg.u;
+          if (n_units > 0) {
+            int q_lo = 0, q_hi = n_exp - 1;
+            if (static_cast<unsigned>(rg.k00) + n_units <= static_cast<unsigned>(rg.kc)) {
+              q_lo = static_cast<int>(fdiv(static_cast<unsigned>(rg.k00), p.d_kpe));
+              q_hi = static_cast<int>(fdiv(static_cast<unsigned>(rg.k00) + n_units - 1u, p.d_kpe));
+            }
+            for (int q = q_lo + lane; q <= q_hi && good; q += 32)
+              good = flag_wait_ge(&p.ready[sg.a0 + q], tpe, abort_flag, p.status);
+          }
+          good = __all_sync(0xffffffffu, good);
+          if (lane == 0) ACM_TRACE(sg.p1_index == 0 ? 17 : 18);
+        }
+        if (good && lane == 0) {
           const uint64_t pol_x = policy_evict_last();
           Sched sc(bars->plan.range[si]);
           int ht, k0, k1;
-          bool polled = false;
+          fence_proxy_async();
           while (good && sc.next(ht, k0, k1)) {
             const int q0 = static_cast<int>(fdiv(static_cast<unsigned>(k0), p.d_kpe));
             int a = sg.a0 + q0, ic = k0 - q0 * kpe;
             for (int kc = k0; kc < k1; ++kc) {
-              if (!polled) {
-                if (!(good = flag_wait_ge(&p.ready[sg.p1_index], n_exp * tpe, abort_flag, p.status))) break;   // n_exp = size of the group
-                fence_proxy_async();
-                polled = true;
-                ACM_TRACE(sg.p1_index == 0 ? 17 : 18);
-              }
               // never ahead of the weight producer: it has found the slot free and armed the barrier
               if (bars->armed <= hidx) {
                 const unsigned long long t0 = global_timer();
@@ -882,7 +894,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
                          ::"l"(&hs_map), "r"(0), "r"(0), "r"(ti), "r"(a), "r"(smem_u32(hstage + hb * kHStageBytes)) : "memory");
             bulk_commit();
             bulk_wait_all();
-            red_release_add(&p.ready[a >= a_split ? 1 : 0], 1);
+            red_release_add(&p.ready[a], 1);
             mbar_arrive(smem_u32(&bars->hst_free[hb]));
             ++fin_n;
             if (fin_n == 1) ACM_TRACE(16);
