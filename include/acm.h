@@ -243,6 +243,18 @@ acm_status acm_set_slot_pool(acm_ctx* ctx, int layer, int n_slots, void* pool_ga
 acm_status acm_pool_stats(acm_ctx* ctx, int layer, uint64_t* hits, uint64_t* misses, uint64_t* h2d_bytes,
                           int32_t* slot_expert, int reset);
 
+/* The pool's replacement policy by itself (pure host code, no GPU; what acm_moe_verify runs for a layer with
+ * a pool).  One block: the activated experts (mask words, host) found in the pool are hits and count as used
+ * now; the others are loaded in ascending id, wave by wave.  Wave 0 runs beside the FFN over the hits and may
+ * only take slots this block does not use; every later wave may replace any slot not loaded in the same wave.
+ * Inside a wave the victim is the least recently used slot it may take (empty slots first, ties to the lower
+ * slot).  In-out (host): slot_expert [n_slots] (expert id or -1), last_use [n_slots], *tick (advanced by one).
+ * Out (host, room for n_experts entries each): load i puts load_expert[i] into load_slot[i] in wave
+ * load_wave[i]; *n_loads, *n_hits. */
+acm_status acm_pool_plan(int n_experts, int n_slots, int32_t* slot_expert, uint64_t* last_use, uint64_t* tick,
+                         const uint32_t* activated_mask, int32_t* load_expert, int32_t* load_slot,
+                         int32_t* load_wave, int32_t* n_loads, int32_t* n_hits);
+
 /* Host->device bytes copied for non-resident experts since the last call with reset != 0. */
 acm_status acm_h2d_bytes(acm_ctx* ctx, uint64_t* bytes_out /*host*/, int reset);
 

@@ -24,7 +24,7 @@ EXPORTS = [
     "acm_default_select_params", "acm_create", "acm_destroy", "acm_set_layer_weights",
     "acm_node_weights", "acm_router", "acm_select_eligible", "acm_route_restricted",
     "acm_expert_ffn", "acm_moe_verify", "acm_moe_verify_batch", "acm_moe_verify_host", "acm_host_synchronize", "acm_set_resident",
-    "acm_set_slot_pool", "acm_pool_stats",
+    "acm_set_slot_pool", "acm_pool_stats", "acm_pool_plan",
     "acm_h2d_bytes", "acm_ffn_timing", "acm_ffn_time_ms", "acm_stage_timing", "acm_stage_times", "acm_launch_count", "acm_device_status", "acm_status_string",
     "acm_expert_ffn_f32_noalloc",
 ]
@@ -98,6 +98,8 @@ def load_library():
     lib.acm_set_slot_pool.argtypes = [c_void_p, c_int, c_int, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_int]
     lib.acm_pool_stats.argtypes = [c_void_p, c_int, POINTER(c_uint64), POINTER(c_uint64), POINTER(c_uint64),
                                    c_void_p, c_int]
+    lib.acm_pool_plan.argtypes = [c_int, c_int, c_void_p, c_void_p, POINTER(c_uint64), c_void_p, c_void_p, c_void_p,
+                                  c_void_p, POINTER(c_int32), POINTER(c_int32)]
     lib.acm_h2d_bytes.argtypes = [c_void_p, POINTER(c_uint64), c_int]
     lib.acm_ffn_timing.argtypes = [c_void_p, c_int, c_int]
     lib.acm_stage_timing.argtypes = [c_void_p, c_int]
@@ -139,6 +141,26 @@ def node_weights(depth, p_table, beta=0.5, width_norm=True) -> torch.Tensor:
     _check(load_library().acm_node_weights(_p(depth), depth.numel(), _p(p_table), p_table.numel(),
                                            float(beta), int(bool(width_norm)), _p(alpha)), "acm_node_weights")
     return alpha
+
+
+def pool_plan(n_experts, slot_expert, last_use, tick, activated):
+    """acm_pool_plan on host data: slot_expert / last_use are lists (updated copies are returned), `activated`
+    a set of expert ids.  Returns (slot_expert, last_use, tick, loads [(expert, slot, wave)], n_hits)."""
+    import numpy as np
+    n_slots = len(slot_expert)
+    se = np.asarray(slot_expert, dtype=np.int32).copy()
+    lu = np.asarray(last_use, dtype=np.uint64).copy()
+    words = (n_experts + 31) // 32
+    mask = np.zeros(words, dtype=np.uint32)
+    for e in activated:
+        mask[e // 32] |= np.uint32(1 << (e % 32))
+    le, ls, lw = (np.zeros(n_experts, dtype=np.int32) for _ in range(3))
+    t, n_loads, n_hits = c_uint64(int(tick)), c_int32(0), c_int32(0)
+    vp = lambda a: a.ctypes.data_as(c_void_p)
+    _check(load_library().acm_pool_plan(n_experts, n_slots, vp(se), vp(lu), byref(t), vp(mask), vp(le), vp(ls), vp(lw),
+                                        byref(n_loads), byref(n_hits)), "acm_pool_plan")
+    n = n_loads.value
+    return se.tolist(), lu.tolist(), t.value, list(zip(le[:n].tolist(), ls[:n].tolist(), lw[:n].tolist())), n_hits.value
 
 
 def expert_ffn_f32_noalloc(x, idx, w, gate_up, down, out, stream=None):

@@ -40,6 +40,60 @@ struct Layer {
   uint64_t pool_hits = 0, pool_misses = 0, pool_h2d = 0, pool_waves = 0;
 };
 
+// The pool's replacement policy for ONE block, pure host logic (no CUDA): given the pool's state and the
+// block's activated experts, marks the hits as used now and plans the loads of the misses, in ascending expert
+// id, wave by wave.  Wave 0 runs beside the FFN over the hits, so it may only take slots this block does not
+// use; every later wave starts after the FFN launched before it and may replace any slot not loaded in the
+// same wave.  Within a wave the victim is the least recently used eligible slot (empty slots count as never
+// used; ties go to the lower slot).  Returns false on an inconsistent state.
+constexpr int kSlotTableRing = 32;
+struct PoolLoad {
+  int32_t expert, slot, wave;
+};
+bool plan_pool_block(int E, int n_slots, std::vector<int32_t>& slot_expert, std::vector<int32_t>& expert_slot,
+                     std::vector<uint64_t>& last_use, uint64_t& tick, const uint32_t* act, std::vector<PoolLoad>& loads,
+                     int& n_hits) {
+  loads.clear();
+  n_hits = 0;
+  tick += 1;
+  std::vector<int32_t> misses;
+  for (int e = 0; e < E; ++e) {
+    if (!((act[e >> 5] >> (e & 31)) & 1u)) continue;
+    if (expert_slot[e] >= 0) {
+      last_use[expert_slot[e]] = tick;
+      n_hits += 1;
+    } else {
+      misses.push_back(e);
+    }
+  }
+  if (n_hits > n_slots) return false;
+  std::vector<int32_t> wave_of(n_slots, -1);
+  size_t done = 0;
+  int wave = 0;
+  while (done < misses.size()) {
+    while (done < misses.size()) {
+      int victim = -1;
+      for (int sl = 0; sl < n_slots; ++sl) {
+        if (wave_of[sl] == wave) continue;                  // just loaded for this wave
+        if (wave == 0 && last_use[sl] == tick) continue;    // in use by the FFN over the hits
+        if (victim < 0 || last_use[sl] < last_use[victim]) victim = sl;
+      }
+      if (victim < 0) break;                                // this wave is full
+      const int e = misses[done];
+      if (slot_expert[victim] >= 0) expert_slot[slot_expert[victim]] = -1;
+      slot_expert[victim] = e;
+      expert_slot[e] = victim;
+      last_use[victim] = tick;
+      wave_of[victim] = wave;
+      loads.push_back(PoolLoad{e, victim, wave});
+      ++done;
+    }
+    ++wave;
+    if (wave > static_cast<int>(misses.size()) + 1) return false;   // cannot happen: every wave after the first has room
+  }
+  return true;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -66,6 +120,8 @@ struct acm_ctx {
   CUtensorMap stage_map_gu, stage_map_dn;
   int32_t* host_stage_list = nullptr;    // pinned + mapped: [0] = count, [1..] = expert ids
   int32_t* host_stage_list_dev = nullptr;
+  int32_t* slot_table_pinned = nullptr;        // pinned ring of expert -> slot tables in flight (kSlotTableRing x kMaxExperts)
+  uint64_t slot_table_next = 0;
   uint32_t* resident_words_pinned = nullptr;   // pinned ring of resident-mask updates in flight (64 x 4 words)
   unsigned long long resident_words_next = 0;
   bool pool_waves_list1_used = false;   // within one call: the second work list has been used by an earlier wave
@@ -285,6 +341,8 @@ acm_status ensure_offload_common(acm_ctx* c) {
   ACM_CUDA(cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->host_stage_list_dev), c->host_stage_list, 0));
   ACM_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->resident_words_pinned), 64 * kMaskWords * sizeof(uint32_t),
                          cudaHostAllocDefault));
+  ACM_CUDA(cudaHostAlloc(reinterpret_cast<void**>(&c->slot_table_pinned),
+                         static_cast<size_t>(kSlotTableRing) * kMaxExperts * sizeof(int32_t), cudaHostAllocDefault));
   ACM_CUDA(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
   ACM_CUDA(cudaEventCreateWithFlags(&c->ev_lists, cudaEventDisableTiming));
   ACM_CUDA(cudaEventCreateWithFlags(&c->ev_copied, cudaEventDisableTiming));
@@ -465,6 +523,7 @@ acm_status acm_destroy(acm_ctx* c) {
   }
   if (c->host_stage_list) cudaFreeHost(c->host_stage_list);
   if (c->resident_words_pinned) cudaFreeHost(c->resident_words_pinned);
+  if (c->slot_table_pinned) cudaFreeHost(c->slot_table_pinned);
   for (Layer& L : c->layers)
     for (int b = 0; b < 2; ++b)
       if (L.slot_of_dev[b]) cudaFree(L.slot_of_dev[b]);
@@ -685,75 +744,59 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
       Layer& P = c->layers[layer];
       uint32_t act[kMaskWords];
       for (int w = 0; w < kMaskWords; ++w) act[w] = static_cast<uint32_t>(c->host_stage_list[1 + kMaxExperts + w]);
-      int n_act = 0;
-      for (int w = 0; w < kMaskWords; ++w) n_act += __builtin_popcount(act[w]);
-      if (n_act - n_stage > P.n_slots) return ACM_ERR_CUDA;   // more resident experts than slots: cannot be
-      P.tick += 1;
-      for (int e = 0; e < E; ++e)
-        if (((act[e >> 5] >> (e & 31)) & 1u) && P.expert_slot[e] >= 0) {
-          P.last_use[P.expert_slot[e]] = P.tick;
-          P.pool_hits += 1;
-        }
       // The activated experts that are not in the pool are loaded in WAVES (Section 3.4: a routed union
-      // larger than the pool is processed in several waves that each fit).  The first wave may only take
-      // slots this block does not use -- the FFN over the resident experts is running -- so it needs no wait;
-      // every later wave first waits for the FFN launched before it and may then replace any slot.  The
-      // expert FFN is a sum over experts, so a wave is a subset of experts over all nodes: each expert is
-      // loaded once.
-      std::vector<int32_t> wave_of(P.n_slots, -1);
-      int done = 0, wave = 0;
-      while (done < n_stage) {
+      // larger than the pool is processed in several waves that each fit).  The first wave needs no wait -- it
+      // only takes slots this block does not use, while the FFN over the resident experts is running; every
+      // later wave first waits for the FFN launched before it.  The expert FFN is a sum over experts, so a
+      // wave is a subset of experts over all nodes: each expert is loaded once.
+      std::vector<PoolLoad> loads;
+      int n_hits = 0;
+      if (!plan_pool_block(E, P.n_slots, P.slot_expert, P.expert_slot, P.last_use, P.tick, act, loads, n_hits))
+        return ACM_ERR_CUDA;
+      if (static_cast<int>(loads.size()) != n_stage) return ACM_ERR_CUDA;     // the kernel's report and the host's view agree
+      P.pool_hits += n_hits;
+      size_t at = 0;
+      for (int wave = 0; at < loads.size(); ++wave) {
         if (wave > 0) {
           ACM_CUDA(cudaEventRecord(c->ev_stage_free, s));
           ACM_CUDA(cudaStreamWaitEvent(c->copy_stream, c->ev_stage_free, 0));
         }
         uint32_t only[kMaskWords] = {0, 0, 0, 0};
-        int loaded = 0;
-        while (done < n_stage) {
-          int victim = -1;
-          for (int sl = 0; sl < P.n_slots; ++sl) {           // free slots first, then the least recently used
-            if (wave_of[sl] == wave) continue;               // just loaded for this wave
-            if (wave == 0 && P.last_use[sl] == P.tick) continue;
-            if (victim < 0 || P.last_use[sl] < P.last_use[victim]) victim = sl;
-          }
-          if (victim < 0) break;                             // this wave is full
-          const int e = c->host_stage_list[1 + done];
-          if (e < 0 || e >= E || P.expert_slot[e] >= 0) return ACM_ERR_CUDA;
-          if (P.slot_expert[victim] >= 0) P.expert_slot[P.slot_expert[victim]] = -1;
-          P.slot_expert[victim] = e;
-          P.expert_slot[e] = victim;
-          P.last_use[victim] = P.tick;
-          wave_of[victim] = wave;
+        // the expert -> slot table this wave's launch reads: where its own experts are (the planner has already
+        // applied later waves too, which may have moved other experts on; after the last wave it is exact)
+        std::vector<int32_t> table(P.expert_slot);
+        for (; at < loads.size() && loads[at].wave == wave; ++at) {
+          const int e = loads[at].expert, sl = loads[at].slot;
           only[e >> 5] |= 1u << (e & 31);
-          ACM_CUDA(cudaMemcpyAsync(static_cast<char*>(P.pool_gate_up) + victim * gu,
+          table[e] = sl;
+          ACM_CUDA(cudaMemcpyAsync(static_cast<char*>(P.pool_gate_up) + sl * gu,
                                    static_cast<const char*>(P.host_gate_up) + e * gu, gu, cudaMemcpyHostToDevice,
                                    c->copy_stream));
-          ACM_CUDA(cudaMemcpyAsync(static_cast<char*>(P.pool_down) + victim * dn,
+          ACM_CUDA(cudaMemcpyAsync(static_cast<char*>(P.pool_down) + sl * dn,
                                    static_cast<const char*>(P.host_down) + e * dn, dn, cudaMemcpyHostToDevice,
                                    c->copy_stream));
           P.pool_misses += 1;
           P.pool_h2d += gu + dn;
           c->h2d_bytes += gu + dn;
-          ++done;
-          ++loaded;
         }
-        if (loaded > 0) {
-          // the new expert -> slot table goes into the other device copy (a running kernel may read this one)
-          const int nxt = P.slot_of_cur ^ 1;
-          ACM_CUDA(cudaMemcpyAsync(P.slot_of_dev[nxt], P.expert_slot.data(), sizeof(int32_t) * E,
-                                   cudaMemcpyHostToDevice, c->copy_stream));
-          ACM_CUDA(cudaEventRecord(c->ev_copied, c->copy_stream));
-          ACM_CUDA(cudaStreamWaitEvent(s, c->ev_copied, 0));
-          P.slot_of_cur = nxt;
-          if (c->pool_waves_list1_used)      // the second work list's counters are cleared once per block by the router kernel
-            ACM_CUDA(cudaMemsetAsync(c->ws.ready + kMaxSlots, 0, sizeof(int32_t) * kMaxSlots, s));
-          c->pool_waves_list1_used = true;
-          st = run_ffn_list(c, P, x, T, 1, out, s, res_dev, nullptr, false, 0, only);
-          if (st != ACM_OK) return st;
-          P.pool_waves += 1;
-        }
-        ++wave;
-        if (wave > n_stage + 1) return ACM_ERR_CUDA;       // cannot happen: every wave after the first has room
+        // the new expert -> slot table goes into the other device copy (a running kernel may read this one)
+        const int nxt = P.slot_of_cur ^ 1;
+        if (c->slot_table_next % kSlotTableRing == kSlotTableRing - 1)
+          ACM_CUDA(cudaStreamSynchronize(c->copy_stream));       // the ring of pinned tables is about to wrap
+        int32_t* staged_table = c->slot_table_pinned + static_cast<size_t>(kMaxExperts) * (c->slot_table_next % kSlotTableRing);
+        std::memcpy(staged_table, table.data(), sizeof(int32_t) * E);
+        ACM_CUDA(cudaMemcpyAsync(P.slot_of_dev[nxt], staged_table, sizeof(int32_t) * E, cudaMemcpyHostToDevice,
+                                 c->copy_stream));
+        c->slot_table_next += 1;
+        ACM_CUDA(cudaEventRecord(c->ev_copied, c->copy_stream));
+        ACM_CUDA(cudaStreamWaitEvent(s, c->ev_copied, 0));
+        P.slot_of_cur = nxt;
+        if (c->pool_waves_list1_used)      // the second work list's counters are cleared once per block by the router kernel
+          ACM_CUDA(cudaMemsetAsync(c->ws.ready + kMaxSlots, 0, sizeof(int32_t) * kMaxSlots, s));
+        c->pool_waves_list1_used = true;
+        st = run_ffn_list(c, P, x, T, 1, out, s, res_dev, nullptr, false, 0, only);
+        if (st != ACM_OK) return st;
+        P.pool_waves += 1;
       }
       c->pool_waves_list1_used = false;
       if (n_stage > 0) {
@@ -1040,6 +1083,40 @@ acm_status acm_pool_stats(acm_ctx* c, int layer, uint64_t* hits, uint64_t* misse
   if (slot_expert)
     for (int i = 0; i < L.n_slots; ++i) slot_expert[i] = L.slot_expert[i];
   if (reset) L.pool_hits = L.pool_misses = L.pool_h2d = 0;
+  return ACM_OK;
+}
+
+acm_status acm_pool_plan(int n_experts, int n_slots, int32_t* slot_expert, uint64_t* last_use, uint64_t* tick,
+                         const uint32_t* activated_mask, int32_t* load_expert, int32_t* load_slot, int32_t* load_wave,
+                         int32_t* n_loads, int32_t* n_hits) {
+  if (n_experts < 1 || n_experts > kMaxExperts || n_slots < 1 || n_slots > kMaxExperts || !slot_expert || !last_use ||
+      !tick || !activated_mask || !load_expert || !load_slot || !load_wave || !n_loads || !n_hits)
+    return ACM_ERR_INVALID;
+  std::vector<int32_t> se(slot_expert, slot_expert + n_slots), es(n_experts, -1);
+  std::vector<uint64_t> lu(last_use, last_use + n_slots);
+  for (int sl = 0; sl < n_slots; ++sl) {
+    if (se[sl] < -1 || se[sl] >= n_experts) return ACM_ERR_INVALID;
+    if (se[sl] >= 0) {
+      if (es[se[sl]] >= 0) return ACM_ERR_INVALID;      // an expert in two slots
+      es[se[sl]] = sl;
+    }
+  }
+  uint32_t act[kMaskWords] = {0, 0, 0, 0};
+  for (int w = 0; w < mask_words(n_experts); ++w) act[w] = activated_mask[w];
+  std::vector<PoolLoad> loads;
+  int hits = 0;
+  if (!plan_pool_block(n_experts, n_slots, se, es, lu, *tick, act, loads, hits)) return ACM_ERR_INVALID;
+  for (size_t i = 0; i < loads.size(); ++i) {
+    load_expert[i] = loads[i].expert;
+    load_slot[i] = loads[i].slot;
+    load_wave[i] = loads[i].wave;
+  }
+  *n_loads = static_cast<int32_t>(loads.size());
+  *n_hits = hits;
+  for (int sl = 0; sl < n_slots; ++sl) {
+    slot_expert[sl] = se[sl];
+    last_use[sl] = lu[sl];
+  }
   return ACM_OK;
 }
 

@@ -7,7 +7,7 @@ import torch
 
 import oracle
 from paper_2608_02989_b200 import acm, workloads as wl
-from tests.helpers import full_mask, mask_to_set, set_to_mask
+from tests.helpers import LruModel as _LruModel, full_mask, mask_to_set, set_to_mask
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -501,46 +501,6 @@ def test_back_to_back_layers_without_host_synchronisation():
         ffn = oracle.expert_ffn(_take(x, rows), ref["idx"][rows], ref["w"][rows], w["gate_up"], w["down"])
         _ffn_check(_take(out, rows), ffn, f"call layer {layer} T {T}")
     ctx.close()
-
-
-class _LruModel:
-    """The pool policy restated for the test: free slots first (lowest index), else the least recently used
-    slot among those the current block does not use; ties to the lower slot index."""
-
-    def __init__(self, n_slots, initial):
-        self.slot_expert = [-1] * n_slots
-        self.last_use = [0] * n_slots
-        self.tick = 0
-        for i, e in enumerate(initial):
-            self.slot_expert[i] = e
-
-    def resident(self):
-        return {e for e in self.slot_expert if e >= 0}
-
-    def block(self, activated):
-        """One block: hits are touched; misses are loaded in ascending id order, in waves -- the first wave may
-        only replace slots this block does not use, every later wave any slot it has not just filled."""
-        self.tick += 1
-        n = len(self.slot_expert)
-        hits = misses = 0
-        for s, e in enumerate(self.slot_expert):
-            if e in activated:
-                self.last_use[s] = self.tick
-                hits += 1
-        todo = sorted(activated - self.resident())
-        wave, wave_of = 0, [-1] * n
-        while todo:
-            while todo:
-                cand = [s for s in range(n) if wave_of[s] != wave and not (wave == 0 and self.last_use[s] == self.tick)]
-                if not cand:
-                    break
-                victim = min(cand, key=lambda s: (self.last_use[s], s))
-                self.slot_expert[victim] = todo.pop(0)
-                self.last_use[victim] = self.tick
-                wave_of[victim] = wave
-                misses += 1
-            wave += 1
-        return hits, misses
 
 
 @pytest.mark.parametrize("mode", [1, 0])
