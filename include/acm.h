@@ -170,7 +170,10 @@ acm_status acm_expert_ffn(acm_ctx* ctx, int layer, const void* x, int T, const i
 /* Stages 1-4 for one block and layer.  alpha [T] device.  eligible_mask_override != NULL
  * skips stage 2 and routes inside the given set (all ones = the natural-routing union path).
  * Optional outputs (NULL to skip): idx_out [T,k], w_out [T,k], mask_out [ceil(E/32)],
- * stats [1].  out [T,H] float is overwritten.
+ * stats [1].  out [T,H] float is overwritten.  stats in memory of the context's device is written
+ * by the kernels themselves; anywhere else (pinned host memory) it is copied at the end of the
+ * call, and so are idx_out, w_out and mask_out -- a copy between this call's last kernel and the
+ * next call's first ends the overlap of the two, so ask only for what is needed in a tight loop.
  * With a residency registered for the layer (acm_set_resident) and params->residency != 0,
  * activated experts that are not GPU-resident are copied from the registered pinned host
  * tensors into the context's staging slots before their FFN runs; this needs one host

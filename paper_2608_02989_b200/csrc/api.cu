@@ -261,6 +261,21 @@ acm_status check_block_args(const acm_ctx* c, int layer, int T, bool need_weight
   return ACM_OK;
 }
 
+// Where the kernels write a call's statistics: straight into the caller's buffer when that is memory of this
+// device (no copy node then sits between this call's last kernel and the next call's first, which would end the
+// overlap of the two), else into the workspace, copied out at the end of the call.
+acm_block_stats* stats_target(acm_ctx* c, acm_block_stats* user, bool* direct) {
+  *direct = false;
+  if (!user) return c->ws.stats;
+  cudaPointerAttributes attr;
+  if (cudaPointerGetAttributes(&attr, user) == cudaSuccess && attr.type == cudaMemoryTypeDevice && attr.device == c->device) {
+    *direct = true;
+    return user;
+  }
+  cudaGetLastError();      // (an unregistered host pointer sets an error on some drivers)
+  return c->ws.stats;
+}
+
 // One FFN launch over work list `li` (0 = resident + shared, 1 = staged).
 acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li, float* out, cudaStream_t s,
                         const uint32_t* res_dev = nullptr, acm_block_stats* stats_dev = nullptr, bool pdl_ok = false,
@@ -694,14 +709,16 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
   sa.n_anchor_nodes = 0; sa.resident = prm.residency ? res_dev : nullptr; sa.prm = prm;
   sa.mask_out = c->ws.mask; sa.unpruned_out = c->ws.unpruned; sa.count_out = c->ws.count;
-  sa.demand_out = c->ws.demand; sa.stats_out = c->ws.stats;
+  bool stats_direct = false;
+  acm_block_stats* stats_dev = stats_target(c, stats, &stats_direct);
+  sa.demand_out = c->ws.demand; sa.stats_out = stats_dev;
   sa.dbg = c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr;
   RouteArgs ra = {};
   ra.logits = c->ws.logits; ra.mask = c->ws.mask; ra.idx_out = c->ws.idx; ra.w_out = c->ws.w;
   ra.weighting = d.weighting; ra.routed_scale = d.routed_scale;
   ra.act_mask = c->ws.act_mask; ra.wtab = c->ws.wtab; ra.resident = res_dev;
   ra.host_stage_list = L.has_resident ? c->host_stage_list_dev : nullptr;
-  ra.stats_out = c->ws.stats;
+  ra.stats_out = stats_dev;
   // the bf16 FFN kernel counts the activated experts itself; otherwise the routing kernel's last CTA does
   ra.ticket = (f32 || L.has_resident) ? c->ws.ticket : nullptr;
   // Early start of the FFN kernel on the eligible set: when a selection runs (the eligible experts are
@@ -726,12 +743,12 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
                             static_cast<float*>(c->ws.hbuf), out, T, d.hidden, d.inter, k, s));
     c->launches += 2;
   } else if (!L.has_resident) {
-    st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, c->ws.stats, true, early_epoch);
+    st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, stats_dev, true, early_epoch);
     if (st != ACM_OK) return st;
   } else {
     // resident + shared experts run at once; the others are copied in from pinned host memory first
     ACM_CUDA(cudaEventRecord(c->ev_lists, s));
-    st = run_ffn_list(c, L, x, T, 0, out, s, res_dev, c->ws.stats);
+    st = run_ffn_list(c, L, x, T, 0, out, s, res_dev, stats_dev);
     if (st != ACM_OK) return st;
     ACM_CUDA(cudaEventSynchronize(c->ev_lists));
     const int n_stage = c->host_stage_list[0];
@@ -837,7 +854,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   if (w_out) ACM_CUDA(cudaMemcpyAsync(w_out, c->ws.w, sizeof(float) * tk, cudaMemcpyDeviceToDevice, s));
   if (mask_out)
     ACM_CUDA(cudaMemcpyAsync(mask_out, c->ws.mask, sizeof(uint32_t) * mask_words(E), cudaMemcpyDeviceToDevice, s));
-  if (stats) ACM_CUDA(cudaMemcpyAsync(stats, c->ws.stats, sizeof(acm_block_stats), cudaMemcpyDefault, s));
+  if (stats && !stats_direct) ACM_CUDA(cudaMemcpyAsync(stats, c->ws.stats, sizeof(acm_block_stats), cudaMemcpyDefault, s));
   return ACM_OK;
 }
 
@@ -876,7 +893,9 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
   sa.n_anchor_nodes = 0; sa.resident = nullptr; sa.prm = *params;
   sa.mask_out = c->ws.mask; sa.unpruned_out = c->ws.unpruned; sa.count_out = c->ws.count;
-  sa.demand_out = c->ws.demand; sa.stats_out = c->ws.stats;
+  bool stats_direct = false;
+  acm_block_stats* stats_dev = stats_target(c, stats, &stats_direct);
+  sa.demand_out = c->ws.demand; sa.stats_out = stats_dev;
   sa.dbg = nullptr;
   RouteArgs ra = {};
   ra.logits = c->ws.logits; ra.mask = c->ws.mask; ra.idx_out = c->ws.idx; ra.w_out = c->ws.w;
@@ -911,7 +930,8 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
   }
   if (activated_out)
     ACM_CUDA(cudaMemcpyAsync(activated_out, c->ws.act_mask, sizeof(uint32_t) * mask_words(E), cudaMemcpyDeviceToDevice, s));
-  if (stats) ACM_CUDA(cudaMemcpyAsync(stats, c->ws.stats, sizeof(acm_block_stats) * n_blocks, cudaMemcpyDefault, s));
+  if (stats && !stats_direct)
+    ACM_CUDA(cudaMemcpyAsync(stats, c->ws.stats, sizeof(acm_block_stats) * n_blocks, cudaMemcpyDefault, s));
   return ACM_OK;
 }
 
