@@ -47,6 +47,9 @@ def parse_args():
                     help="eligible-set policy of the restricted path: the paper's self-sizing selector (default), its "
                          "fixed-budget variant, or the fixed-budget baselines of Section 4.1 (votes / summed router mass)")
     ap.add_argument("--budget", type=int, default=22, help="B0 of the fixed-budget selectors")
+    ap.add_argument("--zipf", action="store_true",
+                    help="supplementary: give the configuration the Zipf(1.1) router bias that C3 has (skewed expert "
+                         "popularity), e.g. --config 5 --zipf")
     ap.add_argument("--batch", type=int, default=0,
                     help="supplementary run: B > 1 verification blocks per call (they share the config's nodes and "
                          "one pass over the expert weights) against the same blocks verified one call each")
@@ -310,6 +313,8 @@ def run_acm(args, world, rank, local):
         torch.cuda.synchronize()
 
     cfg = wl.CONFIGS[args.config]
+    if args.zipf and not cfg.zipf_bias:
+        cfg = wl.scaled(cfg, zipf_bias=True)
     L = args.layers or cfg.n_layers
     resident = cfg.resident_frac > 0
     if resident:
@@ -492,7 +497,7 @@ def run_acm(args, world, rank, local):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": f"C{cfg.index} {cfg.name}-shaped stack, {selector_name}",
+        "config": {"workload": f"C{cfg.index} {cfg.name}-shaped stack{' with Zipf(1.1) router bias' if args.zipf else ''}, {selector_name}",
                    "hidden": H, "n_experts": E, "top_k": k, "inter": cfg.inter, "n_shared": cfg.n_shared,
                    "n_nodes": T, "layers": L, "physical_layers": L_phys,
                    "l2": f"inputs larger than L2: {L_phys} distinct layers, "
