@@ -8,7 +8,7 @@
 //   warp 1      issues tcgen05.mma (M=128 weight rows, N=node columns, fp32 accumulators in TMEM)
 //   warps 2..5  epilogue: tcgen05.ld, SwiGLU / combine; only TMEM and shared memory are touched here
 //   warp 6      helper: waits for other CTAs' partial sums and copies them into shared memory ahead of
-//               need; adds the activation chunk to down stages once their expert group is complete
+//               need; adds the activation chunk to down stages once their experts are complete
 //   warp 7      publisher: moves staged fragments / activation tiles to global memory (bulk reduce-add,
 //               TMA store), waits for completion, then raises the counter other CTAs wait on
 // The weights are the M operand ("swap-AB"): every activated expert's weights are read from HBM
@@ -21,8 +21,9 @@
 //   down     tile = 128 output rows, K = (activated expert, intermediate) concatenated, cut evenly;
 //            experts complete early first.  Partial tiles are added to the output with fp32
 //            reductions in L2 (the caller zeroes the output).
-// The down phase reads activations written by other CTAs in the gate/up phase; two group counters
-// order them.  Every wait is bounded; on expiry the kernel raises a status and drains.
+// The down phase reads activations written by other CTAs in the gate/up phase; one finished-tile counter
+// per expert orders them (a CTA waits for the experts its share of the K range reads).  Every wait is
+// bounded; on expiry the kernel raises a status and drains.
 //
 // f32 path: plain FMA kernels (the fp32 toy configuration is a few MFLOP).
 #include <cuda_bf16.h>
@@ -605,7 +606,6 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   tc_fence_after();
   const Segment* seg = bars->plan.seg;
   const int n_seg = bars->plan.n_seg;
-  const int a_split = bars->plan.a_split;
   const uint32_t tmem_base = bars->tmem_base;
   if (threadIdx.x == 0) ACM_TRACE(0);
 
