@@ -684,3 +684,15 @@ def test_stage_times_come_from_device_stamps():
     with pytest.raises(acm.AcmError):
         ctx.stage_times()
     ctx.close()
+
+
+@pytest.mark.parametrize("T", [1, 2, 5, 17, 33, 63])
+def test_fused_call_on_ragged_block_sizes(T):
+    """Blocks of 1 to 63 nodes (padded accumulator columns, partial node tiles in the router kernel, trees
+    shallower than the commitment table) through the fused call, every output row against the oracle."""
+    cfg = wl.scaled(wl.CONFIGS[3], n_nodes=T, inter=256, n_layers=1)
+    ctx = _ctx(cfg)
+    st, rel = _verify_layer(cfg, 0, ctx, 0)
+    assert st["n_activated"] >= min(cfg.top_k, cfg.n_experts)
+    _verify_layer(cfg, 0, ctx, 0, natural=True)
+    ctx.close()
