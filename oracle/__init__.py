@@ -8,6 +8,7 @@ from .binding import (  # noqa: F401
     SelectParams,
     SelectStats,
     build,
+    dequantize_mxfp4,
     expf,
     expert_ffn,
     logf,

@@ -246,3 +246,19 @@ def moe_verify(x, w_router, bias, gate_up, down, alpha, k, params: SelectParams 
     return {"logits": logits, "probs": probs, "nat_idx": nat, "mask": sel["mask"],
             "unpruned_mask": sel["unpruned_mask"], "count": sel["count"], "demand": sel["demand"],
             "stats": sel["stats"], "idx": idx, "w": w, "out": out, "n_experts": E}
+
+
+# E2M1 code -> value (sign bit 3, exponent bits 2:1 with bias 1, mantissa bit 0; exponent 0 is subnormal)
+_E2M1 = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0], dtype=np.float64)
+
+
+def dequantize_mxfp4(codes, scales):
+    """MXFP4 -> float64: codes [..., K] uint8 (4-bit E2M1 codes), scales [..., K/32] uint8 (E8M0: 2^(s-127));
+    value = (-1)^sign * e2m1(code & 7) * 2^(s - 127).  Every result is exactly representable in bfloat16 as
+    long as it is in range, so an MXFP4 layer is the bf16 layer with these weights."""
+    codes = _np(codes).astype(np.int64)
+    scales = _np(scales).astype(np.int64)
+    mag = _E2M1[codes & 7]
+    sign = np.where(codes & 8, -1.0, 1.0)
+    factor = np.ldexp(1.0, scales - 127)
+    return sign * mag * np.repeat(factor, 32, axis=-1)

@@ -163,6 +163,50 @@ def pool_plan(n_experts, slot_expert, last_use, tick, activated):
     return se.tolist(), lu.tolist(), t.value, list(zip(le[:n].tolist(), ls[:n].tolist(), lw[:n].tolist())), n_hits.value
 
 
+# ---- MXFP4 expert weights: the library's tiled layout ------------------------------------------------
+# The FFN kernel fetches one pipeline stage of an MXFP4 weight tile -- 128 rows x 128 K -- with a single
+# contiguous copy, so the weights are stored tile by tile: per (expert, tile, stage) 8704 bytes =
+#   128 rows x 64 bytes of codes, then 128 rows x 4 scale bytes (one E8M0 byte per 32 K).
+# Inside each group of 8 consecutive K elements the codes sit in one 32-bit word with the even elements in
+# the low half and the odd ones in the high half (nibble j = element 2j, nibble 4+j = element 2j+1), which
+# is the order the kernel's expansion to bf16 pairs wants.  These functions only permute bytes.
+MX_STAGE_BYTES = 128 * 64 + 128 * 4
+
+
+def _mx_words(codes):
+    """codes [..., rows, 128] (4-bit values in uint8) -> [..., rows, 64] bytes in the word order above."""
+    c = codes.to(torch.int32).reshape(*codes.shape[:-1], 16, 4, 2)        # [group of 8][pair j][even, odd]
+    even, odd = c[..., 0], c[..., 1]                                           # [..., 16, 4]
+    lo = even[..., 0] | (even[..., 1] << 4) | (even[..., 2] << 8) | (even[..., 3] << 12)
+    hi = odd[..., 0] | (odd[..., 1] << 4) | (odd[..., 2] << 8) | (odd[..., 3] << 12)
+    b = torch.stack([lo & 0xff, lo >> 8, hi & 0xff, hi >> 8], dim=-1)          # little-endian bytes of the word
+    return b.to(torch.uint8).reshape(*codes.shape[:-1], 64)
+
+
+def pack_mxfp4_gate_up(codes, scales):
+    """codes [E, 2I, H], scales [E, 2I, H/32] (uint8; rows 0..I-1 gate, I..2I-1 up) ->
+    uint8 [E, I/64, H/128, 8704]: tile t = gate rows 64t..64t+63 followed by the matching up rows."""
+    E, R, H = codes.shape
+    I = R // 2
+    if I % 64 or H % 128:
+        raise ValueError("MXFP4 layers need inter % 64 == 0 and hidden % 128 == 0")
+    c = codes.reshape(E, 2, I // 64, 64, H // 128, 128).permute(0, 2, 4, 1, 3, 5)      # [E, tile, stage, g|u, 64, 128]
+    c = _mx_words(c.reshape(E, I // 64, H // 128, 128, 128)).reshape(E, I // 64, H // 128, 128 * 64)
+    s = scales.reshape(E, 2, I // 64, 64, H // 128, 4).permute(0, 2, 4, 1, 3, 5).reshape(E, I // 64, H // 128, 512)
+    return torch.cat([c, s], dim=-1).contiguous()
+
+
+def pack_mxfp4_down(codes, scales):
+    """codes [E, H, I], scales [E, H, I/32] (uint8) -> uint8 [E, H/128, I/128, 8704]."""
+    E, H, I = codes.shape
+    if H % 128 or I % 128:
+        raise ValueError("MXFP4 layers need hidden % 128 == 0 and inter % 128 == 0")
+    c = codes.reshape(E, H // 128, 128, I // 128, 128).permute(0, 1, 3, 2, 4)          # [E, tile, stage, 128 rows, 128]
+    c = _mx_words(c).reshape(E, H // 128, I // 128, 128 * 64)
+    s = scales.reshape(E, H // 128, 128, I // 128, 4).permute(0, 1, 3, 2, 4).reshape(E, H // 128, I // 128, 512)
+    return torch.cat([c, s], dim=-1).contiguous()
+
+
 def expert_ffn_f32_noalloc(x, idx, w, gate_up, down, out, stream=None):
     """acm_expert_ffn_f32_noalloc: the fp32 expert FFN for callers that may not allocate device memory at
     call time.  Every tensor, `out` included, is the caller's; nothing is allocated here or in the library

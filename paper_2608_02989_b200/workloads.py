@@ -187,3 +187,50 @@ def describe(cfg: BlockConfig) -> str:
             f"p_d={cfg.p_scale}*{cfg.p_decay}^d expert={cfg.expert_bytes / 1e6:.3f} MB "
             f"layer={weight_bytes_per_layer(cfg) / 1e9:.3f} GB"
             + (f" resident={math.floor(cfg.resident_frac * 100)}%" if cfg.resident_frac else ""))
+
+
+# ---- MXFP4 expert weights (the GPT-OSS-style storage the paper's offload table mentions) -------------
+# Microscaling FP4: blocks of 32 consecutive K elements share a power-of-two scale (one E8M0 byte: 2^(s-127));
+# an element is a 4-bit E2M1 code (sign, 2 exponent bits, 1 mantissa bit: 0, 0.5, 1, 1.5, 2, 3, 4, 6).
+# This is input preparation (how the synthetic weights are put into that storage), not the method.
+E2M1_VALUES = (0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0)
+
+
+def quantize_mxfp4(w: torch.Tensor):
+    """w [..., K] (K a multiple of 32) -> (codes uint8 [..., K] with the 4-bit code of every element,
+    scales uint8 [..., K/32]).  Per block: shared exponent = floor(log2(max|w|)) - 2 (2 = the largest E2M1
+    exponent), clamped to the E8M0 range; elements are rounded to the nearest E2M1 value (ties to the even
+    code) and saturate at +-6.  A block of zeros gets scale 2^-127."""
+    if w.shape[-1] % 32 != 0:
+        raise ValueError("the last dimension must be a multiple of 32")
+    wf = w.detach().to(torch.float32).reshape(*w.shape[:-1], w.shape[-1] // 32, 32)
+    amax = wf.abs().amax(dim=-1, keepdim=True)
+    exp = torch.floor(torch.log2(torch.clamp(amax, min=2.0 ** -126))) - 2.0
+    exp = torch.clamp(exp, -127.0, 127.0)
+    exp = torch.where(amax > 0, exp, torch.full_like(exp, -127.0))
+    scaled = wf / torch.exp2(exp)
+    grid = torch.tensor(E2M1_VALUES, dtype=torch.float32, device=w.device)
+    mag = scaled.abs().clamp(max=6.0)
+    # nearest grid point; at a midpoint take the even code (codes 0, 2, 4, 6 have mantissa bit 0)
+    d = (mag.unsqueeze(-1) - grid).abs()
+    best = d.argmin(dim=-1)
+    lo = torch.clamp(best - 1, min=0)
+    tie_lo = (d.gather(-1, lo.unsqueeze(-1)).squeeze(-1) == d.gather(-1, best.unsqueeze(-1)).squeeze(-1)) & (lo != best)
+    best = torch.where(tie_lo & (lo % 2 == 0), lo, best)
+    hi = torch.clamp(best + 1, max=7)
+    tie_hi = (d.gather(-1, hi.unsqueeze(-1)).squeeze(-1) == d.gather(-1, best.unsqueeze(-1)).squeeze(-1)) & (hi != best)
+    best = torch.where(tie_hi & (hi % 2 == 0), hi, best)
+    codes = (best + 8 * (scaled < 0).to(best.dtype)).to(torch.uint8).reshape(w.shape)
+    scales = (exp.squeeze(-1) + 127.0).to(torch.uint8)
+    return codes, scales
+
+
+def layer_weights_mxfp4(cfg: BlockConfig, layer: int, device="cpu") -> dict:
+    """The layer's weights with the routed experts in MXFP4: the bf16 draw of layer_weights, quantised.
+    Adds gate_up_codes [E,2I,H] / gate_up_scales [E,2I,H/32] and down_codes [E,H,I] / down_scales [E,H,I/32]
+    (uint8); gate_up / down are dropped."""
+    w = layer_weights(cfg, layer, device)
+    w["gate_up_codes"], w["gate_up_scales"] = quantize_mxfp4(w.pop("gate_up"))
+    w["down_codes"], w["down_scales"] = quantize_mxfp4(w.pop("down"))
+    w["gate_up"] = w["down"] = None
+    return w
