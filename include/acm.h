@@ -134,6 +134,23 @@ acm_status acm_set_layer_weights(acm_ctx* ctx, int layer, const void* w_router,
                                  const void* w_down, const void* shared_gate_up,
                                  const void* shared_down);
 
+/* The same for a layer whose routed experts are stored in MXFP4 (microscaling FP4 -- the storage the
+ * paper's offload measurements name for GPT-OSS, Section 4.4): 4-bit E2M1 codes, one E8M0 scale byte
+ * (2^(s-127)) per 32 consecutive K elements.  The FFN kernel expands the codes to bf16 on the way to the
+ * tensor cores -- every MXFP4 value is a bf16, so the layer computes exactly what a bf16 layer with the
+ * dequantised weights computes -- and streams a quarter of the bytes.  The tensors are in the library's
+ * tiled layout (one contiguous 8704-byte record per weight tile and pipeline stage):
+ *   gate_up_tiles [E][I/64][H/128][8704]: tile t = gate rows 64t..64t+63 then up rows I+64t..I+64t+63,
+ *   down_tiles    [E][H/128][I/128][8704]: tile t = rows 128t..128t+127,
+ *   record = 128 rows x 64 code bytes, then 128 rows x 4 scale bytes, for 128 consecutive K; each
+ *   32-bit word of code bytes holds 8 consecutive K elements, the even ones in the nibbles of its low
+ *   half, the odd ones in the nibbles of its high half (element 2j = nibble j, 2j+1 = nibble 4+j).
+ * Scale bytes above 128 (block scales above 2) are treated as 128.  bf16 contexts with n_shared == 0,
+ * hidden % 128 == 0 and inter % 128 == 0 only; no residency or pool on such a layer. */
+acm_status acm_set_layer_weights_mxfp4(acm_ctx* ctx, int layer, const void* w_router,
+                                       const float* router_bias, const void* gate_up_tiles,
+                                       const void* down_tiles);
+
 /* Eq. 3 on the host: alpha_t = p_table[depth_t]^beta * N_{depth_t}^{-1/2} (width factor
  * optional), evaluated in double and rounded once.  All pointers are HOST pointers.
  * ACM_ERR_INVALID if a depth lies outside the table. */

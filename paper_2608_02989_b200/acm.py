@@ -21,7 +21,7 @@ W_RENORM_TOPK, W_SOFTMAX_RAW, W_SOFTMAX_MASKED = 0, 1, 2
 DEMAND_TOPK_MASS, DEMAND_FULL_MASS, DEMAND_VOTES = 0, 1, 2
 
 EXPORTS = [
-    "acm_default_select_params", "acm_create", "acm_destroy", "acm_set_layer_weights",
+    "acm_default_select_params", "acm_create", "acm_destroy", "acm_set_layer_weights", "acm_set_layer_weights_mxfp4",
     "acm_node_weights", "acm_router", "acm_select_eligible", "acm_route_restricted",
     "acm_expert_ffn", "acm_moe_verify", "acm_moe_verify_batch", "acm_moe_verify_host", "acm_host_synchronize", "acm_set_resident",
     "acm_set_slot_pool", "acm_pool_stats", "acm_pool_plan",
@@ -80,6 +80,7 @@ def load_library():
     lib.acm_create.argtypes = [POINTER(ModelDesc), POINTER(c_void_p)]
     lib.acm_destroy.argtypes = [c_void_p]
     lib.acm_set_layer_weights.argtypes = [c_void_p, c_int] + [c_void_p] * 6
+    lib.acm_set_layer_weights_mxfp4.argtypes = [c_void_p, c_int] + [c_void_p] * 4
     lib.acm_node_weights.argtypes = [c_void_p, c_int, c_void_p, c_int, c_float, c_int, c_void_p]
     lib.acm_router.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.acm_select_eligible.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_int,
@@ -256,6 +257,12 @@ class Context:
         _check(self.lib.acm_set_layer_weights(self.handle, layer, _p(w_router), _p(router_bias), _p(gate_up),
                                               _p(down), _p(shared_gate_up), _p(shared_down)),
                "acm_set_layer_weights")
+
+    def set_layer_weights_mxfp4(self, layer, w_router, router_bias, gate_up_tiles, down_tiles):
+        """Routed experts in MXFP4, in the library's tiled layout (pack_mxfp4_gate_up / pack_mxfp4_down), on the device."""
+        self._keep[("w", layer)] = (w_router, router_bias, gate_up_tiles, down_tiles)
+        _check(self.lib.acm_set_layer_weights_mxfp4(self.handle, layer, _p(w_router), _p(router_bias), _p(gate_up_tiles),
+                                                    _p(down_tiles)), "acm_set_layer_weights_mxfp4")
 
     def set_resident(self, layer, resident_mask, host_gate_up, host_down):
         """resident_mask: host int32/uint32 words (or None to clear); host_*: pinned host tensors."""

@@ -9,7 +9,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libacm.so"
-SOURCES = ["api.cu", "routing.cu", "ffn.cu"]
+SOURCES = ["api.cu", "routing.cu", "ffn.cu", "ffn_mx.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "--fmad=true", "-Xptxas", "-v"]
 

@@ -163,12 +163,17 @@ struct FfnLaunch {
   int grid;
   int phase_mask;            // 1 = gate/up, 2 = down, 3 = both in one launch
   bool pdl;                  // launch with programmatic stream serialization
+  const void* mx_gate_up = nullptr;   // MXFP4 layers (launch_ffn_mxfp4): the tiled code + scale tensors
+  const void* mx_down = nullptr;
   unsigned long long* trace; // optional [grid][32] device timestamps (debugging aid) or null
 };
 cudaError_t ffn_configure();   // one-time function attributes
 size_t ffn_smem_bytes();
 cudaError_t launch_ffn_bf16(const FfnLaunch& p, const FfnMaps& maps, const CUtensorMap& x_map,
                             const CUtensorMap& h_map, const CUtensorMap& h_store_map, cudaStream_t s);
+cudaError_t ffn_mx_configure();
+cudaError_t launch_ffn_mxfp4(const FfnLaunch& p, const FfnMaps& maps, const CUtensorMap& x_map,
+                             const CUtensorMap& h_map, const CUtensorMap& h_store_map, cudaStream_t s);
 cudaError_t launch_ffn_f32(const float* x, const float* gate_up, const float* down,
                            const float* shared_gate_up, const float* shared_down, int n_shared,
                            const int32_t* idx, const float* w, float* hbuf, float* out, int T, int H,

@@ -22,6 +22,8 @@ struct Layer {
   const void* shared_down = nullptr;
   FfnMaps maps;
   bool set = false;
+  const void* mx_gate_up = nullptr;     // MXFP4 layer (acm_set_layer_weights_mxfp4): tiled codes + scales
+  const void* mx_down = nullptr;
   bool has_resident = false;
   const void* host_gate_up = nullptr;   // pinned host copies for on-demand loads
   const void* host_down = nullptr;
@@ -150,6 +152,7 @@ struct acm_ctx {
   uint64_t launches = 0;
   bool split_phases = false;             // ACM_FFN_SPLIT_PHASES=1 in the environment
   unsigned long long* trace = nullptr;   // ACM_FFN_TRACE=1|2: per-CTA timestamps of the last FFN launch
+  bool mx_configured = false;
   bool trace_light = false;              // =2: leave the launch sequence as it is (stale slots are not cleared)
 };
 
@@ -327,7 +330,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
     c->ev_used += 2;
     ACM_CUDA(cudaEventRecord(e0, s));
   }
-  if (c->split_phases) {
+  if (c->split_phases && !L.mx_gate_up) {
     // debugging aid: the two GEMM phases as separate launches (kernel boundary instead of flags)
     p.phase_mask = 1;
     ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
@@ -341,7 +344,12 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   // split changes -- and one late CTA delays every CTA that exchanges fragments with it.  Leave them out.
   const int routing_ctas = n_blocks > 0 ? n_blocks : route_ctas(T);   // a batch: one CTA per block
   if (pdl_ok && c->sm_count > 2 * routing_ctas) p.grid = c->sm_count - routing_ctas;
-  ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
+  if (L.mx_gate_up) {
+    p.mx_gate_up = L.mx_gate_up; p.mx_down = L.mx_down;
+    ACM_CUDA(launch_ffn_mxfp4(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
+  } else {
+    ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
+  }
   c->launches += 1;
   if (e1) ACM_CUDA(cudaEventRecord(e1, s));
   return ACM_OK;
@@ -583,6 +591,27 @@ acm_status acm_set_layer_weights(acm_ctx* c, int layer, const void* w_router, co
   return ACM_OK;
 }
 
+acm_status acm_set_layer_weights_mxfp4(acm_ctx* c, int layer, const void* w_router, const float* router_bias,
+                                       const void* gate_up_tiles, const void* down_tiles) {
+  if (!c || layer < 0 || layer >= c->desc.n_layers || !w_router || !gate_up_tiles || !down_tiles) return ACM_ERR_INVALID;
+  const acm_model_desc& d = c->desc;
+  if (d.dtype != ACM_BF16 || d.n_shared != 0 || d.inter % 128 != 0 || d.hidden % 128 != 0) return ACM_ERR_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(w_router) % 16 != 0 || reinterpret_cast<uintptr_t>(gate_up_tiles) % 16 != 0 ||
+      reinterpret_cast<uintptr_t>(down_tiles) % 16 != 0)
+    return ACM_ERR_INVALID;
+  if (!c->mx_configured) {
+    if (ffn_mx_configure() != cudaSuccess) return ACM_ERR_CUDA;
+    c->mx_configured = true;
+  }
+  Layer L;
+  L.w_router = w_router; L.bias = router_bias;
+  L.mx_gate_up = gate_up_tiles; L.mx_down = down_tiles;
+  std::memset(&L.maps, 0, sizeof L.maps);      // the MXFP4 kernel fetches its weights with plain bulk copies
+  L.set = true;
+  c->layers[layer] = L;
+  return ACM_OK;
+}
+
 acm_status acm_node_weights(const int32_t* depth, int T, const float* p_table, int n_depths, float beta,
                             int width_norm, float* alpha_out) {
   if (!depth || !p_table || !alpha_out || T < 1 || n_depths < 1) return ACM_ERR_INVALID;
@@ -652,7 +681,7 @@ acm_status acm_expert_ffn(acm_ctx* c, int layer, const void* x, int T, const int
   acm_status st = check_block_args(c, layer, T, true);
   if (st != ACM_OK) return st;
   const Layer& L = c->layers[layer];
-  if (!x || !idx || !w || !out || !L.gate_up) return ACM_ERR_INVALID;
+  if (!x || !idx || !w || !out || (!L.gate_up && !L.mx_gate_up)) return ACM_ERR_INVALID;
   if (reinterpret_cast<uintptr_t>(x) % 16 != 0 || reinterpret_cast<uintptr_t>(out) % 16 != 0) return ACM_ERR_INVALID;
   if (L.has_resident) return ACM_ERR_UNSUPPORTED;   // staging is driven by acm_moe_verify
   const acm_model_desc& d = c->desc;
@@ -678,7 +707,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   acm_status st = check_block_args(c, layer, T, true);
   if (st != ACM_OK) return st;
   const Layer& L = c->layers[layer];
-  if (!x || !out || (!L.gate_up && !L.has_pool)) return ACM_ERR_INVALID;
+  if (!x || !out || (!L.gate_up && !L.has_pool && !L.mx_gate_up)) return ACM_ERR_INVALID;
   if (reinterpret_cast<uintptr_t>(x) % 16 != 0 || reinterpret_cast<uintptr_t>(out) % 16 != 0) return ACM_ERR_INVALID;
   acm_select_params prm;
   if (eligible_mask_override) {
@@ -875,7 +904,7 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
   acm_status st = check_block_args(c, layer, T, true);
   if (st != ACM_OK) return st;
   const Layer& L = c->layers[layer];
-  if (!x || !out || !alpha || !L.gate_up) return ACM_ERR_INVALID;
+  if (!x || !out || !alpha || (!L.gate_up && !L.mx_gate_up)) return ACM_ERR_INVALID;
   if (reinterpret_cast<uintptr_t>(x) % 16 != 0 || reinterpret_cast<uintptr_t>(out) % 16 != 0) return ACM_ERR_INVALID;
   st = check_params(params);
   if (st != ACM_OK) return st;
@@ -1015,6 +1044,7 @@ acm_status acm_set_resident(acm_ctx* c, int layer, const uint32_t* resident_mask
     L.host_gate_up = L.host_down = nullptr;
     return ACM_OK;
   }
+  if (L.mx_gate_up) return ACM_ERR_UNSUPPORTED;   // MXFP4 layers are all-resident
   if (L.has_pool) return ACM_ERR_INVALID;      // clear the pool first (NULL mask)
   if (c->desc.dtype != ACM_BF16) return ACM_ERR_UNSUPPORTED;
   if (!host_gate_up || !host_down) return ACM_ERR_INVALID;
@@ -1032,6 +1062,7 @@ acm_status acm_set_resident(acm_ctx* c, int layer, const uint32_t* resident_mask
 acm_status acm_set_slot_pool(acm_ctx* c, int layer, int n_slots, void* pool_gate_up, void* pool_down,
                              const void* host_gate_up, const void* host_down, const int32_t* initial_experts,
                              int n_initial) {
+  if (c && layer >= 0 && layer < c->desc.n_layers && c->layers[layer].mx_gate_up) return ACM_ERR_UNSUPPORTED;
   if (!c || layer < 0 || layer >= c->desc.n_layers) return ACM_ERR_INVALID;
   const acm_model_desc& d = c->desc;
   if (d.dtype != ACM_BF16) return ACM_ERR_UNSUPPORTED;

@@ -55,7 +55,17 @@ constexpr int kOutStageBytes = kTileM * kMaxNodes * 4;   // 32 KB: outgoing frag
 constexpr int kHStageBytes = kMaxNodes * 64 * 2;         // 8 KB: one finished activation tile (64 features x nodes)
 constexpr int kAccCols = kMaxNodes;                      // TMEM columns per accumulator
 constexpr int kTmemCols = kAcc * kAccCols;
-constexpr int kThreads = 256;                            // producer, MMA, 4 epilogue warps, helper, publisher
+// ACM_FFN_MX = 1 (set by ffn_mx.cu, which includes this file) builds the same kernel for MXFP4 expert
+// weights: a pipeline stage of a weight tile arrives as 128 rows x 64 bytes of E2M1 codes + 128 x 4 E8M0
+// scale bytes (one contiguous 8704-byte copy into the stage's weight area), and four more warps expand it
+// there to the 32 KB bf16 tile the MMAs read -- every MXFP4 value is a bf16, so the arithmetic is the
+// bf16 path's.
+#ifndef ACM_FFN_MX
+#define ACM_FFN_MX 0
+#endif
+constexpr int kThreads = ACM_FFN_MX ? 384 : 256;         // producer, MMA, 4 epilogue warps, helper, publisher (+ 4 expanding warps)
+constexpr int kMxCodeBytes = kTileM * 64;                // 128 rows x 128 four-bit codes
+constexpr int kMxStageBytes = kMxCodeBytes + kTileM * 4; // + one scale byte per row and 32 K
 constexpr int kFragBytes = kTileM * kMaxNodes * 4;       // contributor fragments pre-summed in shared memory
 constexpr int kFragFloats = kTileM * kMaxNodes;
 constexpr unsigned long long kTimeoutNs = 1000ull * 1000ull * 1000ull;
@@ -133,6 +143,9 @@ struct __align__(8) Barriers {
   unsigned long long helper;         // completion of the helper warp's bulk copy
   unsigned long long ost_full, ost_free;   // epilogue <-> publisher: outgoing fragment staged / copied out
   unsigned long long hst_full[2], hst_free[2];   // epilogue <-> publisher: activation tile staged / stored
+#if ACM_FFN_MX
+  unsigned long long raw[kStages];   // the packed weight stage has landed (producer's copy -> expanding warps)
+#endif
   volatile uint32_t armed;           // stages whose barrier the weight producer has armed so far
   uint32_t tmem_base;
   int abort_flag;
@@ -227,6 +240,10 @@ __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_load_hint(uint32_t smem_dst, const void* gmem_src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+               ::"r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
 // Barrier over the 128 epilogue threads that also ANDs a predicate, so that all of them take the
@@ -373,6 +390,10 @@ struct FfnArgs {
   int32_t* status;
   int phase_mask;
   unsigned long long* trace;   // optional [grid][32] timestamps (debugging aid), may be null
+#if ACM_FFN_MX
+  const unsigned char* mx_gate_up;   // [E][I/64][H/128][8704]
+  const unsigned char* mx_down;      // [E][H/128][I/128][8704]
+#endif
 };
 
 __device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMap* routed, const CUtensorMap* shared,
@@ -449,8 +470,13 @@ __device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act
   }
 }
 
+#if ACM_FFN_MX
+#define ACM_FFN_KERNEL k_ffn_mxfp4
+#else
+#define ACM_FFN_KERNEL k_ffn_bf16
+#endif
 __global__ void __launch_bounds__(kThreads, 1)
-k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtensorMap x_map,
+ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtensorMap x_map,
            const __grid_constant__ CUtensorMap h_map, const __grid_constant__ CUtensorMap hs_map,
            const FfnArgs p) {
   extern __shared__ unsigned char smem_dyn[];
@@ -470,8 +496,11 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   if (threadIdx.x == 0) ACM_TRACE(12);     // kernel entry
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(smem_u32(&bars->full[s]), 1);
+      mbar_init(smem_u32(&bars->full[s]), ACM_FFN_MX ? 5 : 1);   // MXFP4: + one arrival per expanding warp
       mbar_init(smem_u32(&bars->empty[s]), 1);
+#if ACM_FFN_MX
+      mbar_init(smem_u32(&bars->raw[s]), 1);
+#endif
     }
     for (int b = 0; b < kAcc; ++b) {
       mbar_init(smem_u32(&bars->tfull[b]), 1);
@@ -493,8 +522,10 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
     fence_barrier_init();
   }
   if (warp == 0 && lane == 0) {
+#if !ACM_FFN_MX
     prefetch_tensormap(&maps.gate_up);
     prefetch_tensormap(&maps.down);
+#endif
     prefetch_tensormap(&x_map);
     prefetch_tensormap(&h_map);
   }
@@ -633,8 +664,18 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
               if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
               const uint32_t full = smem_u32(&bars->full[s]);
               const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
+#if ACM_FFN_MX
+              mbar_expect_tx(full, b_bytes);
+              {
+                const uint32_t rawb = smem_u32(&bars->raw[s]);
+                mbar_expect_tx(rawb, kMxStageBytes);
+                bulk_load_hint(sa, p.mx_gate_up + (static_cast<size_t>(eidx * tpe + (r0 >> 6)) * kc1 + kc) * kMxStageBytes,
+                               kMxStageBytes, rawb, pol_w);
+              }
+#else
               mbar_expect_tx(full, kABytes + b_bytes);
               tma_load_5d(sa, gu, full, 0, r0, 0, kc * kAtoms, eidx, pol_w);   // 64 gate + 64 up rows, 2 atoms
+#endif
               tma_load_3d(sa + kABytes, &x_map, full, 0, 0, kc * kAtoms, pol_x);
               if (!traced_first) { ACM_TRACE(1); traced_first = true; }
               ++n_armed;
@@ -655,8 +696,18 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
               if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
               const uint32_t full = smem_u32(&bars->full[s]);
               const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
+#if ACM_FFN_MX
+              mbar_expect_tx(full, b_bytes);
+              {
+                const uint32_t rawb = smem_u32(&bars->raw[s]);
+                mbar_expect_tx(rawb, kMxStageBytes);
+                bulk_load_hint(sa, p.mx_down + (static_cast<size_t>(eidx * h_tiles + ht) * kpe + ic) * kMxStageBytes,
+                               kMxStageBytes, rawb, pol_w);
+              }
+#else
               mbar_expect_tx(full, kABytes + b_bytes);
               tma_load_4d(sa, dn, full, 0, ht * kTileM, ic * kAtoms, eidx, pol_w);
+#endif
               bars->armed = ++n_armed;      // the helper warp may now add this stage's activation chunk
               if (++s == kStages) { s = 0; par ^= 1u; }
               if (++ic == kpe && kc + 1 < k1) {
@@ -903,6 +954,51 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
         }
       }
     }
+#if ACM_FFN_MX
+  } else if (warp >= 8) {
+    // ------------------------------------------------------------------ expanding warps (MXFP4 -> bf16)
+    // Thread r owns weight-tile row r.  Per stage: wait for the packed copy, take the row's 64 code bytes and 4
+    // scale bytes into registers, meet the other rows (the bf16 tile overwrites the packed one), write the row's
+    // 128 bf16 into the two 128-byte-swizzled atoms the MMA descriptors expect, then tell the stage's barrier.
+    // A code is sign | 2 exponent bits | 1 mantissa bit with subnormals: put at bits 15 | 8:7 | 6 of a bf16 it
+    // is the value times 2^-126 exactly, so one bf16 multiply by 2^(scale byte - 1) finishes the job.
+    const int r = threadIdx.x - 256;
+    unsigned total = 0;
+    for (int si = 0; si < n_seg; ++si) total += bars->plan.range[si].n_stages;
+    bool ok = true;
+    for (unsigned it = 0; it < total && ok; ++it) {
+      const uint32_t s = it % kStages, par = (it / kStages) & 1u;
+      if (!(ok = mbar_wait(smem_u32(&bars->raw[s]), par, abort_flag, p.status))) break;
+      unsigned char* A = stage_base + static_cast<size_t>(s) * kStageBytes;
+      uint4 q[4];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) q[b] = *reinterpret_cast<const uint4*>(A + r * 64 + 16 * b);
+      const uint32_t sc = *reinterpret_cast<const uint32_t*>(A + kMxCodeBytes + r * 4);
+      asm volatile("bar.sync 3, 128;" ::: "memory");
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {                     // 32 K = one scale
+        const uint32_t field = min(((sc >> (8 * b)) & 0xffu) + 126u, 254u) << 7;
+        const uint32_t c2 = field | (field << 16);
+        const uint32_t words[4] = {q[b].x, q[b].y, q[b].z, q[b].w};
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {                   // 8 K = one 16-byte chunk of the row
+          uint32_t o[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t t = (words[w] >> (4 * j)) & 0x000f000fu;       // elements 2j (low half) and 2j+1 (high half)
+            const uint32_t enc = (t * 0x1040u) & 0x81c081c0u;
+            asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(o[j]) : "r"(enc), "r"(c2));
+          }
+          const int chunk = 4 * b + w;                  // 16 chunks of 8 K; 8 per atom
+          unsigned char* dst = A + (chunk >> 3) * kAtomABytes + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+          *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->full[s]));
+    }
+#endif
   } else {
     // ------------------------------------------------------------------ epilogue (128 threads)
     // On-chip work only: accumulators -> registers -> shared memory.  Everything that has to reach
@@ -1068,6 +1164,7 @@ k_ffn_bf16(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtenso
   }
 }
 
+#if !ACM_FFN_MX
 // ---------------------------------------------------------------------------------- f32 path
 // h[t][j][i] = silu(g) * u for routed slot j < k (expert idx[t][j]) and shared slot j >= k.
 __global__ void k_ffn_f32_gate_up(const float* __restrict__ x, const float* __restrict__ gate_up,
@@ -1120,16 +1217,26 @@ __global__ void k_ffn_f32_down(const float* __restrict__ down, const float* __re
   if (lane == 0) out[static_cast<size_t>(t) * H + hh] = y;
 }
 
+#endif   // !ACM_FFN_MX
+
 }  // namespace
 
+#if ACM_FFN_MX
+cudaError_t ffn_mx_configure() {
+  return cudaFuncSetAttribute(ACM_FFN_KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+}
+cudaError_t launch_ffn_mxfp4(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
+                             const CUtensorMap& h_map, const CUtensorMap& hs_map, cudaStream_t s) {
+#else
 size_t ffn_smem_bytes() { return kSmemBytes; }
 
 cudaError_t ffn_configure() {
-  return cudaFuncSetAttribute(k_ffn_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  return cudaFuncSetAttribute(ACM_FFN_KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
 }
 
 cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
                             const CUtensorMap& h_map, const CUtensorMap& hs_map, cudaStream_t s) {
+#endif
   {
     // the schedules count (tile, K-chunk) units times the grid in 32 bits
     const unsigned long long u1 = static_cast<unsigned long long>(kMaxSlots) * (L.I / 64) * (L.H / (kBK * kAtoms));
@@ -1151,6 +1258,11 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag;
   a.sel_flag = L.sel_flag; a.sel_epoch = L.sel_epoch; a.sel_blocks = L.sel_blocks;
   a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask; a.trace = L.trace;
+#if ACM_FFN_MX
+  if (!L.mx_gate_up || !L.mx_down || L.I % 128 != 0 || L.n_shared != 0 || L.slot_of || L.resident) return cudaErrorInvalidValue;
+  a.mx_gate_up = static_cast<const unsigned char*>(L.mx_gate_up);
+  a.mx_down = static_cast<const unsigned char*>(L.mx_down);
+#endif
   void* args[] = {const_cast<FfnMaps*>(&maps), const_cast<CUtensorMap*>(&x_map), const_cast<CUtensorMap*>(&h_map),
                   const_cast<CUtensorMap*>(&hs_map), &a};
   cudaLaunchConfig_t cfg = {};
@@ -1172,9 +1284,10 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   cfg.attrs = attr;
   static const bool plain = [] { const char* e = std::getenv("ACM_FFN_PLAIN_LAUNCH"); return e && e[0] == '1'; }();
   cfg.numAttrs = (plain && !L.pdl) ? 0 : 1;
-  return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(k_ffn_bf16), args);
+  return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(ACM_FFN_KERNEL), args);
 }
 
+#if !ACM_FFN_MX
 cudaError_t launch_ffn_f32(const float* x, const float* gate_up, const float* down,
                            const float* shared_gate_up, const float* shared_down, int n_shared,
                            const int32_t* idx, const float* w, float* hbuf, float* out, int T, int H,
@@ -1191,8 +1304,11 @@ cudaError_t launch_ffn_f32(const float* x, const float* gate_up, const float* do
   return cudaGetLastError();
 }
 
+#endif   // !ACM_FFN_MX
+
 }  // namespace acm
 
+#if !ACM_FFN_MX
 // ------------------------------------------------------------------------------------------------
 // Allocation-free variant of the f32 expert FFN.  The per-(node, slot) intermediate activations that
 // the context-based call keeps in its cudaMalloc'ed workspace live here in a fixed array that is part
@@ -1234,3 +1350,4 @@ extern "C" acm_status acm_expert_ffn_f32_noalloc(const float* x, int T, int hidd
                                               inter, top_k, static_cast<cudaStream_t>(stream));
   return err == cudaSuccess ? ACM_OK : ACM_ERR_CUDA;
 }
+#endif   // !ACM_FFN_MX

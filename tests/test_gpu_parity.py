@@ -696,3 +696,45 @@ def test_fused_call_on_ragged_block_sizes(T):
     assert st["n_activated"] >= min(cfg.top_k, cfg.n_experts)
     _verify_layer(cfg, 0, ctx, 0, natural=True)
     ctx.close()
+
+
+def _mx_layer(cfg, layer=0):
+    """An MXFP4 layer: the config's bf16 draw quantised; returns the weights dict with the tiled device tensors and
+    the dequantised bf16 tensors (what the layer means)."""
+    w = wl.layer_weights_mxfp4(cfg, layer, DEV)
+    w["gate_up_tiles"] = acm.pack_mxfp4_gate_up(w["gate_up_codes"], w["gate_up_scales"]).to(DEV)
+    w["down_tiles"] = acm.pack_mxfp4_down(w["down_codes"], w["down_scales"]).to(DEV)
+    gu = torch.tensor(oracle.dequantize_mxfp4(w["gate_up_codes"], w["gate_up_scales"]))
+    dn = torch.tensor(oracle.dequantize_mxfp4(w["down_codes"], w["down_scales"]))
+    assert torch.equal(gu.to(torch.bfloat16).double(), gu) and torch.equal(dn.to(torch.bfloat16).double(), dn)
+    w["gate_up_deq"], w["down_deq"] = gu.to(torch.bfloat16).to(DEV), dn.to(torch.bfloat16).to(DEV)
+    return w
+
+
+@pytest.mark.parametrize("shape", [dict(inter=256, n_experts=32), dict(), dict(hidden=4096, inter=1536, n_nodes=33)])
+def test_mxfp4_layer_equals_the_bf16_layer_with_the_dequantised_weights(shape):
+    """Expert weights in MXFP4: sets and routes as always (the router is bf16); the FFN output against the oracle
+    run on the dequantised weights, and against the library's own bf16 kernel on them, which does the same
+    arithmetic in the same order."""
+    cfg = wl.scaled(wl.CONFIGS[3], n_layers=1, **shape)
+    ctx = _ctx(cfg, n_layers=2)
+    w = _mx_layer(cfg)
+    x = wl.hidden_states(cfg, 0, DEV)
+    alpha = acm.node_weights(wl.tree_depths(cfg), wl.commitment_table(cfg))
+    ctx.set_layer_weights_mxfp4(0, w["w_router"], w["router_bias"], w["gate_up_tiles"], w["down_tiles"])
+    ctx.set_layer_weights(1, w["w_router"], w["router_bias"], w["gate_up_deq"], w["down_deq"])
+    for natural in (False, True):
+        kw = dict(mask_override=torch.tensor(full_mask(cfg.n_experts).view(np.int32), device=DEV)) if natural else {}
+        a = None if natural else alpha.to(DEV)
+        out, idx, wt, mask, stats = ctx.moe_verify(0, x, a, None if natural else acm.SelectParams(), want=True, **kw)
+        ref_out, ref_idx, ref_wt, ref_mask, _ = ctx.moe_verify(1, x, a, None if natural else acm.SelectParams(), want=True, **kw)
+        assert ctx.device_status() == acm.OK
+        np.testing.assert_array_equal(idx.cpu().numpy(), ref_idx.cpu().numpy())
+        np.testing.assert_array_equal(_u32(mask), _u32(ref_mask))
+        rows = sorted({0, 1, cfg.n_nodes // 2, cfg.n_nodes - 1})
+        ffn = oracle.expert_ffn(_take(x, rows), idx.cpu().numpy()[rows], wt.cpu().numpy()[rows], w["gate_up_deq"], w["down_deq"])
+        _ffn_check(_take(out, rows), ffn, "MXFP4 layer")
+        # same tiles, same MMAs, same order of additions inside a tile; split-K partial sums meet in L2 in any order
+        rms = float(ref_out.double().pow(2).mean().sqrt())
+        assert float((out - ref_out).abs().max()) <= 1e-3 * rms
+    ctx.close()
