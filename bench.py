@@ -47,6 +47,9 @@ def parse_args():
                     help="eligible-set policy of the restricted path: the paper's self-sizing selector (default), its "
                          "fixed-budget variant, or the fixed-budget baselines of Section 4.1 (votes / summed router mass)")
     ap.add_argument("--budget", type=int, default=22, help="B0 of the fixed-budget selectors")
+    ap.add_argument("--mxfp4", action="store_true",
+                    help="supplementary: the routed experts stored in MXFP4 (the configuration's weights quantised), "
+                         "expanded to bf16 inside the FFN kernel")
     ap.add_argument("--zipf", action="store_true",
                     help="supplementary: give the configuration the Zipf(1.1) router bias that C3 has (skewed expert "
                          "popularity), e.g. --config 5 --zipf")
@@ -328,6 +331,13 @@ def run_acm(args, world, rank, local):
     ctx = acm.Context.for_config(cfg, n_layers=L_phys)
     keep = []
     for l in range(L_phys):
+        if args.mxfp4:
+            w = wl.layer_weights_mxfp4(cfg, l + 1000 * rank, dev)
+            gu = acm.pack_mxfp4_gate_up(w.pop("gate_up_codes"), w.pop("gate_up_scales"))
+            dn = acm.pack_mxfp4_down(w.pop("down_codes"), w.pop("down_scales"))
+            ctx.set_layer_weights_mxfp4(l, w["w_router"], w["router_bias"], gu, dn)
+            keep.append((w["w_router"], w["router_bias"], gu, dn))
+            continue
         w = wl.layer_weights(cfg, l + 1000 * rank, dev)
         ctx.set_layer_weights(l, w["w_router"], w["router_bias"], w["gate_up"], w["down"], w["shared_gate_up"],
                               w["shared_down"])
@@ -409,7 +419,8 @@ def run_acm(args, world, rank, local):
     ctx.check_device_status()
     st = stats.cpu().numpy()
     n_act = st[:, 4].astype(float)
-    expert_bytes = cfg.expert_bytes
+    # MXFP4: half a byte per weight plus one scale byte per 32
+    expert_bytes = 3 * H * cfg.inter * (0.5 + 1.0 / 32.0) if args.mxfp4 else cfg.expert_bytes
     # algorithmic bytes of one FFN launch: the activated experts' weights (+ shared), x in, y out
     alg_bytes = (n_act + cfg.n_shared) * expert_bytes + T * H * 2 + T * H * 4
     alg_per_launch = float(alg_bytes[sampled_layers(args.steps)].mean()) if not resident else float(alg_bytes.mean())
@@ -491,13 +502,13 @@ def run_acm(args, world, rank, local):
     achieved = alg_per_launch / (ffn_us * 1e-6) / 1e9 if ffn_n else None
     # DRAM bytes (read + write) of k_ffn_bf16 per activated expert, from the ncu capture summarised in
     # profiles/k_ffn_bf16_c3_layer.txt (4-layer case; traffic is proportional to the activated experts)
-    per_expert = DRAM_BYTES_PER_ACTIVATED_EXPERT.get(cfg.index)
+    per_expert = None if args.mxfp4 else DRAM_BYTES_PER_ACTIVATED_EXPERT.get(cfg.index)
     traffic = per_expert * (alg_per_launch - T * H * 6) / expert_bytes if per_expert else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": f"C{cfg.index} {cfg.name}-shaped stack{' with Zipf(1.1) router bias' if args.zipf else ''}, {selector_name}",
+        "config": {"workload": f"C{cfg.index} {cfg.name}-shaped stack{' with Zipf(1.1) router bias' if args.zipf else ''}{', MXFP4 expert weights' if args.mxfp4 else ''}, {selector_name}",
                    "hidden": H, "n_experts": E, "top_k": k, "inter": cfg.inter, "n_shared": cfg.n_shared,
                    "n_nodes": T, "layers": L, "physical_layers": L_phys,
                    "l2": f"inputs larger than L2: {L_phys} distinct layers, "
@@ -508,7 +519,7 @@ def run_acm(args, world, rank, local):
         "mean_natural_union": float(st[:, 5].mean()),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": (achieved / peak) if achieved else None, "traffic": traffic, "peak_kind": peak_kind,
-                     "kernel": "k_ffn_bf16", "us_per_launch": ffn_us, "launches_timed": ffn_n,
+                     "kernel": "k_ffn_mxfp4" if args.mxfp4 else "k_ffn_bf16", "us_per_launch": ffn_us, "launches_timed": ffn_n,
                      "timed_every": period,
                      "algorithmic_bytes_per_launch": alg_per_launch,
                      # context, not the headline: the same kernel inside the live pipeline (in-kernel stamps from its
@@ -521,7 +532,7 @@ def run_acm(args, world, rank, local):
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and not args.mxfp4:      # (the oracle's MXFP4 layer is its bf16 layer on the dequantised weights)
         line["cpu_baseline"] = cpu_baseline(cfg)
     print(json.dumps(line), flush=True)
     ctx.close()

@@ -209,18 +209,14 @@ def quantize_mxfp4(w: torch.Tensor):
     exp = torch.clamp(exp, -127.0, 127.0)
     exp = torch.where(amax > 0, exp, torch.full_like(exp, -127.0))
     scaled = wf / torch.exp2(exp)
-    grid = torch.tensor(E2M1_VALUES, dtype=torch.float32, device=w.device)
     mag = scaled.abs().clamp(max=6.0)
-    # nearest grid point; at a midpoint take the even code (codes 0, 2, 4, 6 have mantissa bit 0)
-    d = (mag.unsqueeze(-1) - grid).abs()
-    best = d.argmin(dim=-1)
-    lo = torch.clamp(best - 1, min=0)
-    tie_lo = (d.gather(-1, lo.unsqueeze(-1)).squeeze(-1) == d.gather(-1, best.unsqueeze(-1)).squeeze(-1)) & (lo != best)
-    best = torch.where(tie_lo & (lo % 2 == 0), lo, best)
-    hi = torch.clamp(best + 1, max=7)
-    tie_hi = (d.gather(-1, hi.unsqueeze(-1)).squeeze(-1) == d.gather(-1, best.unsqueeze(-1)).squeeze(-1)) & (hi != best)
-    best = torch.where(tie_hi & (hi % 2 == 0), hi, best)
-    codes = (best + 8 * (scaled < 0).to(best.dtype)).to(torch.uint8).reshape(w.shape)
+    # nearest grid point = the number of midpoints passed; at a midpoint take the even code (the midpoint
+    # between codes i and i+1 goes up only when i+1 is even)
+    best = torch.zeros_like(mag, dtype=torch.uint8)
+    for i in range(7):
+        mid = 0.5 * (E2M1_VALUES[i] + E2M1_VALUES[i + 1])
+        best += ((mag >= mid) if i % 2 == 1 else (mag > mid)).to(torch.uint8)
+    codes = (best + 8 * (scaled < 0).to(torch.uint8)).reshape(w.shape)
     scales = (exp.squeeze(-1) + 127.0).to(torch.uint8)
     return codes, scales
 
