@@ -145,6 +145,8 @@ acm_status acm_set_layer_weights(acm_ctx* ctx, int layer, const void* w_router,
  *   record = 128 rows x 64 code bytes, then 128 rows x 4 scale bytes, for 128 consecutive K; each
  *   32-bit word of code bytes holds 8 consecutive K elements, the even ones in the nibbles of its low
  *   half, the odd ones in the nibbles of its high half (element 2j = nibble j, 2j+1 = nibble 4+j).
+ *   The four 16-byte pieces of a row's code bytes (32 K each) are stored rotated by the row number:
+ *   piece p of row r (0..127 inside the record) at position p ^ ((r >> 1) & 3).
  * Scale bytes above 128 (block scales above 2) are treated as 128.  bf16 contexts with n_shared == 0,
  * hidden % 128 == 0 and inter % 128 == 0 only; no residency or pool on such a layer. */
 acm_status acm_set_layer_weights_mxfp4(acm_ctx* ctx, int layer, const void* w_router,

@@ -170,7 +170,9 @@ def pool_plan(n_experts, slot_expert, last_use, tick, activated):
 #   128 rows x 64 bytes of codes, then 128 rows x 4 scale bytes (one E8M0 byte per 32 K).
 # Inside each group of 8 consecutive K elements the codes sit in one 32-bit word with the even elements in
 # the low half and the odd ones in the high half (nibble j = element 2j, nibble 4+j = element 2j+1), which
-# is the order the kernel's expansion to bf16 pairs wants.  These functions only permute bytes.
+# is the order the kernel's expansion to bf16 pairs wants; the four 16-byte pieces of a row (32 K each) are
+# stored rotated by the row number (piece p of row r at position p ^ ((r >> 1) & 3)).  These functions only
+# permute bytes.
 MX_STAGE_BYTES = 128 * 64 + 128 * 4
 
 
@@ -181,7 +183,14 @@ def _mx_words(codes):
     lo = even[..., 0] | (even[..., 1] << 4) | (even[..., 2] << 8) | (even[..., 3] << 12)
     hi = odd[..., 0] | (odd[..., 1] << 4) | (odd[..., 2] << 8) | (odd[..., 3] << 12)
     b = torch.stack([lo & 0xff, lo >> 8, hi & 0xff, hi >> 8], dim=-1)          # little-endian bytes of the word
-    return b.to(torch.uint8).reshape(*codes.shape[:-1], 64)
+    b = b.to(torch.uint8).reshape(*codes.shape[:-1], 4, 16)                    # the row's four 16-byte pieces (32 K each)
+    # piece p of row r is stored at position p ^ ((r >> 1) & 3): a warp reading one piece per row then touches
+    # every shared-memory bank once
+    rows = codes.shape[-2]
+    pos = torch.arange(4, device=codes.device)[None, :] ^ ((torch.arange(rows, device=codes.device)[:, None] >> 1) & 3)
+    out = torch.empty_like(b)
+    out.scatter_(-2, pos[..., None].expand(*b.shape[:-3], rows, 4, 16).contiguous(), b)
+    return out.reshape(*codes.shape[:-1], 64)
 
 
 def pack_mxfp4_gate_up(codes, scales):

@@ -36,6 +36,9 @@
 namespace acm {
 namespace {
 
+#ifndef ACM_FFN_MX
+#define ACM_FFN_MX 0
+#endif
 #ifndef ACM_FFN_STAGES
 #define ACM_FFN_STAGES 3
 #endif
@@ -54,15 +57,14 @@ constexpr int kStageBytes = kABytes + kBBytesMax;
 constexpr int kOutStageBytes = kTileM * kMaxNodes * 4;   // 32 KB: outgoing fragment (also the gate/up exchange buffer)
 constexpr int kHStageBytes = kMaxNodes * 64 * 2;         // 8 KB: one finished activation tile (64 features x nodes)
 constexpr int kAccCols = kMaxNodes;                      // TMEM columns per accumulator
-constexpr int kTmemCols = kAcc * kAccCols;
+constexpr int kMxACols = 64;                             // MXFP4: one expanded weight stage in tensor memory = 128 K bf16 per row
+constexpr int kTmemCols = ACM_FFN_MX ? 512 : kAcc * kAccCols;   // MXFP4: accumulators, then kStages expanded weight stages
+static_assert(kAcc * kAccCols + kStages * kMxACols <= 512, "tensor memory: accumulators + expanded weight stages");
 // ACM_FFN_MX = 1 (set by ffn_mx.cu, which includes this file) builds the same kernel for MXFP4 expert
 // weights: a pipeline stage of a weight tile arrives as 128 rows x 64 bytes of E2M1 codes + 128 x 4 E8M0
 // scale bytes (one contiguous 8704-byte copy into the stage's weight area), and four more warps expand it
 // there to the 32 KB bf16 tile the MMAs read -- every MXFP4 value is a bf16, so the arithmetic is the
 // bf16 path's.
-#ifndef ACM_FFN_MX
-#define ACM_FFN_MX 0
-#endif
 constexpr int kThreads = ACM_FFN_MX ? 384 : 256;         // producer, MMA, 4 epilogue warps, helper, publisher (+ 4 expanding warps)
 constexpr int kMxCodeBytes = kTileM * 64;                // 128 rows x 128 four-bit codes
 constexpr int kMxStageBytes = kMxCodeBytes + kTileM * 4; // + one scale byte per row and 32 K
@@ -337,6 +339,22 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr) {
   return d;
 }
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+// The same MMA with the A operand (128 rows x 16 K bf16) in tensor memory: row = lane, two K elements per column.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 16 consecutive columns of this thread's lane
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ uint32_t umma_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
 }
@@ -770,9 +788,16 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
 #pragma unroll
             for (int at = 0; at < kAtoms; ++at) {
 #pragma unroll
-              for (int kk = 0; kk < kBK / 16; ++kk)
+              for (int kk = 0; kk < kBK / 16; ++kk) {
+#if ACM_FFN_MX
+                // the expanded weights are in tensor memory: stage s, 8 columns per 16 K
+                umma_bf16_ts(d_tmem, tmem_base + kAcc * kAccCols + s * kMxACols + (at * (kBK / 16) + kk) * 8,
+                             db0 + (at * (b_atom_bytes >> 4) + 2 * kk), idesc, (kc > k0 || at > 0 || kk > 0) ? 1u : 0u);
+#else
                 umma_bf16(d_tmem, da0 + (at * (kAtomABytes >> 4) + 2 * kk), db0 + (at * (b_atom_bytes >> 4) + 2 * kk), idesc,
                           (kc > k0 || at > 0 || kk > 0) ? 1u : 0u);
+#endif
+              }
             }
             umma_commit(smem_u32(&bars->empty[s]));
           }
@@ -957,44 +982,46 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
 #if ACM_FFN_MX
   } else if (warp >= 8) {
     // ------------------------------------------------------------------ expanding warps (MXFP4 -> bf16)
-    // Thread r owns weight-tile row r.  Per stage: wait for the packed copy, take the row's 64 code bytes and 4
-    // scale bytes into registers, meet the other rows (the bf16 tile overwrites the packed one), write the row's
-    // 128 bf16 into the two 128-byte-swizzled atoms the MMA descriptors expect, then tell the stage's barrier.
+    // Thread r owns weight-tile row r = lane r of tensor memory.  Per stage: wait for the packed copy, take
+    // the row's 64 code bytes and 4 scale bytes from shared memory, expand them to 128 bf16 in registers and
+    // store those into the stage's 64 columns of tensor memory, from where the MMAs take their A operand --
+    // the expanded tile never passes through shared memory.
     // A code is sign | 2 exponent bits | 1 mantissa bit with subnormals: put at bits 15 | 8:7 | 6 of a bf16 it
     // is the value times 2^-126 exactly, so one bf16 multiply by 2^(scale byte - 1) finishes the job.
     const int r = threadIdx.x - 256;
+    const uint32_t my_lane = static_cast<uint32_t>(r & ~31) << 16;          // this warp's quarter of the lanes
     unsigned total = 0;
     for (int si = 0; si < n_seg; ++si) total += bars->plan.range[si].n_stages;
     bool ok = true;
     for (unsigned it = 0; it < total && ok; ++it) {
       const uint32_t s = it % kStages, par = (it / kStages) & 1u;
       if (!(ok = mbar_wait(smem_u32(&bars->raw[s]), par, abort_flag, p.status))) break;
-      unsigned char* A = stage_base + static_cast<size_t>(s) * kStageBytes;
-      uint4 q[4];
-#pragma unroll
-      for (int b = 0; b < 4; ++b) q[b] = *reinterpret_cast<const uint4*>(A + r * 64 + 16 * b);
+      const unsigned char* A = stage_base + static_cast<size_t>(s) * kStageBytes;
       const uint32_t sc = *reinterpret_cast<const uint32_t*>(A + kMxCodeBytes + r * 4);
-      asm volatile("bar.sync 3, 128;" ::: "memory");
+      const uint32_t a_tmem = tmem_base + my_lane + kAcc * kAccCols + s * kMxACols;
+      tc_fence_after();
 #pragma unroll
-      for (int b = 0; b < 4; ++b) {                     // 32 K = one scale
+      for (int b = 0; b < 4; ++b) {                     // 32 K = one scale = 16 columns
+        // (the record keeps the row's four 16-byte pieces rotated by the row number, so that a warp's loads
+        // spread over all banks)
+        const uint4 q = *reinterpret_cast<const uint4*>(A + r * 64 + 16 * (b ^ ((r >> 1) & 3)));
         const uint32_t field = min(((sc >> (8 * b)) & 0xffu) + 126u, 254u) << 7;
         const uint32_t c2 = field | (field << 16);
-        const uint32_t words[4] = {q[b].x, q[b].y, q[b].z, q[b].w};
+        const uint32_t words[4] = {q.x, q.y, q.z, q.w};
+        uint32_t o[16];
 #pragma unroll
-        for (int w = 0; w < 4; ++w) {                   // 8 K = one 16-byte chunk of the row
-          uint32_t o[4];
+        for (int w = 0; w < 4; ++w) {
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const uint32_t t = (words[w] >> (4 * j)) & 0x000f000fu;       // elements 2j (low half) and 2j+1 (high half)
             const uint32_t enc = (t * 0x1040u) & 0x81c081c0u;
-            asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(o[j]) : "r"(enc), "r"(c2));
+            asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(o[4 * w + j]) : "r"(enc), "r"(c2));
           }
-          const int chunk = 4 * b + w;                  // 16 chunks of 8 K; 8 per atom
-          unsigned char* dst = A + (chunk >> 3) * kAtomABytes + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
-          *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
         }
+        tmem_st16(a_tmem + 16 * b, o);
       }
-      fence_proxy_async_smem();
+      tmem_st_wait();
+      tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->full[s]));
     }

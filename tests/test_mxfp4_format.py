@@ -60,7 +60,13 @@ def test_quantiser_is_the_nearest_representable_value_under_the_block_scale():
 
 def _unpack_words(tile_bytes):
     """Inverse of the word order: [rows, 64] bytes -> [rows, 128] codes."""
-    b = tile_bytes.astype(np.uint32).reshape(-1, 16, 4)
+    rows = tile_bytes.shape[0]
+    pieces = tile_bytes.reshape(rows, 4, 16)
+    unrot = np.empty_like(pieces)
+    for r in range(rows):
+        for piece in range(4):
+            unrot[r, piece] = pieces[r, piece ^ ((r >> 1) & 3)]
+    b = unrot.astype(np.uint32).reshape(-1, 16, 4)
     word = b[..., 0] | (b[..., 1] << 8) | (b[..., 2] << 16) | (b[..., 3] << 24)
     out = np.zeros(word.shape + (8,), dtype=np.uint8)
     for j in range(4):
