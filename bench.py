@@ -171,11 +171,21 @@ def run_pool(args):
     ctx = acm.Context.for_config(cfg, n_layers=L)
     keep = []
     for l in range(L):
-        w = wl.layer_weights(cfg, l, dev)
-        host_gu, host_dn = w["gate_up"].cpu().pin_memory(), w["down"].cpu().pin_memory()
-        pool_gu = torch.empty((X,) + tuple(w["gate_up"].shape[1:]), dtype=w["gate_up"].dtype, device=dev)
-        pool_dn = torch.empty((X,) + tuple(w["down"].shape[1:]), dtype=w["down"].dtype, device=dev)
-        ctx.set_layer_weights(l, w["w_router"], w["router_bias"], None, None)
+        if args.mxfp4:
+            w = wl.layer_weights_mxfp4(cfg, l, dev)
+            gu = acm.pack_mxfp4_gate_up(w.pop("gate_up_codes"), w.pop("gate_up_scales"))
+            dn = acm.pack_mxfp4_down(w.pop("down_codes"), w.pop("down_scales"))
+            host_gu, host_dn = gu.cpu().pin_memory(), dn.cpu().pin_memory()
+            pool_gu = torch.empty((X,) + tuple(gu.shape[1:]), dtype=torch.uint8, device=dev)
+            pool_dn = torch.empty((X,) + tuple(dn.shape[1:]), dtype=torch.uint8, device=dev)
+            del gu, dn
+            ctx.set_layer_weights_mxfp4(l, w["w_router"], w["router_bias"], None, None)
+        else:
+            w = wl.layer_weights(cfg, l, dev)
+            host_gu, host_dn = w["gate_up"].cpu().pin_memory(), w["down"].cpu().pin_memory()
+            pool_gu = torch.empty((X,) + tuple(w["gate_up"].shape[1:]), dtype=w["gate_up"].dtype, device=dev)
+            pool_dn = torch.empty((X,) + tuple(w["down"].shape[1:]), dtype=w["down"].dtype, device=dev)
+            ctx.set_layer_weights(l, w["w_router"], w["router_bias"], None, None)
         ctx.set_slot_pool(l, pool_gu, pool_dn, host_gu, host_dn, list(range(X)))     # starts full: experts 0..X-1
         keep.append((w["w_router"], w["router_bias"], host_gu, host_dn, pool_gu, pool_dn))
         del w
@@ -218,7 +228,7 @@ def run_pool(args):
                      "h2d_mib_per_layer_block": h2d / 2 ** 20 / (n_blocks * L)}
     line = {"metric": METRIC, "value": res["restricted_eq7"]["layer_blocks_per_s"], "unit": UNIT, "n_gpus": 1,
             "steps": n_blocks, "warmup": 0, "higher_is_better": True, "dtype": cfg.dtype, "data": "synthetic",
-            "config": {"workload": f"C5 {cfg.name}-shaped layers with Zipf-biased routing behind an LRU pool of {X} "
+            "config": {"workload": f"C5 {cfg.name}-shaped layers{' in MXFP4' if args.mxfp4 else ''} with Zipf-biased routing behind an LRU pool of {X} "
                                    f"expert slots per layer (offload variant); {L} layers, {n_blocks} distinct blocks",
                        "hidden": H, "n_experts": E, "top_k": cfg.top_k, "inter": cfg.inter, "n_nodes": T},
             "policies": res}

@@ -148,7 +148,10 @@ acm_status acm_set_layer_weights(acm_ctx* ctx, int layer, const void* w_router,
  *   The four 16-byte pieces of a row's code bytes (32 K each) are stored rotated by the row number:
  *   piece p of row r (0..127 inside the record) at position p ^ ((r >> 1) & 3).
  * Scale bytes above 128 (block scales above 2) are treated as 128.  bf16 contexts with n_shared == 0,
- * hidden % 128 == 0 and inter % 128 == 0 only; no residency or pool on such a layer. */
+ * hidden % 128 == 0 and inter % 128 == 0 only.  Both tile tensors may be NULL when the layer's experts
+ * live in a pool (acm_set_slot_pool, called next): its pool and host tensors are then in this tiled
+ * layout too ([n_slots][...] and [E][...]), and a loaded expert costs a quarter of the bf16 bytes.
+ * acm_set_resident (the static residency with staging slots) is not available on such a layer. */
 acm_status acm_set_layer_weights_mxfp4(acm_ctx* ctx, int layer, const void* w_router,
                                        const float* router_bias, const void* gate_up_tiles,
                                        const void* down_tiles);

@@ -22,7 +22,8 @@ struct Layer {
   const void* shared_down = nullptr;
   FfnMaps maps;
   bool set = false;
-  const void* mx_gate_up = nullptr;     // MXFP4 layer (acm_set_layer_weights_mxfp4): tiled codes + scales
+  bool mx = false;                      // MXFP4 layer (acm_set_layer_weights_mxfp4): expert tensors are tiled codes + scales
+  const void* mx_gate_up = nullptr;     // [E][I/64][H/128][8704] (null when the experts only live in a pool)
   const void* mx_down = nullptr;
   bool has_resident = false;
   const void* host_gate_up = nullptr;   // pinned host copies for on-demand loads
@@ -279,6 +280,18 @@ acm_block_stats* stats_target(acm_ctx* c, acm_block_stats* user, bool* direct) {
   return c->ws.stats;
 }
 
+// bytes of one expert's gate/up and down tensors as the layer stores them (bf16, or MXFP4 tile records)
+void expert_tensor_bytes(const acm_model_desc& d, bool mx, size_t* gu, size_t* dn) {
+  if (mx) {
+    const size_t rec = 128 * 64 + 128 * 4;
+    *gu = static_cast<size_t>(d.inter / 64) * (d.hidden / 128) * rec;
+    *dn = static_cast<size_t>(d.hidden / 128) * (d.inter / 128) * rec;
+  } else {
+    *gu = static_cast<size_t>(2) * d.inter * d.hidden * 2;
+    *dn = static_cast<size_t>(d.hidden) * d.inter * 2;
+  }
+}
+
 // One FFN launch over work list `li` (0 = resident + shared, 1 = staged).
 acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li, float* out, cudaStream_t s,
                         const uint32_t* res_dev = nullptr, acm_block_stats* stats_dev = nullptr, bool pdl_ok = false,
@@ -330,7 +343,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
     c->ev_used += 2;
     ACM_CUDA(cudaEventRecord(e0, s));
   }
-  if (c->split_phases && !L.mx_gate_up) {
+  if (c->split_phases && !L.mx) {
     // debugging aid: the two GEMM phases as separate launches (kernel boundary instead of flags)
     p.phase_mask = 1;
     ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
@@ -344,8 +357,9 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   // split changes -- and one late CTA delays every CTA that exchanges fragments with it.  Leave them out.
   const int routing_ctas = n_blocks > 0 ? n_blocks : route_ctas(T);   // a batch: one CTA per block
   if (pdl_ok && c->sm_count > 2 * routing_ctas) p.grid = c->sm_count - routing_ctas;
-  if (L.mx_gate_up) {
-    p.mx_gate_up = L.mx_gate_up; p.mx_down = L.mx_down;
+  if (L.mx) {
+    p.mx_gate_up = L.has_pool ? L.pool_gate_up : L.mx_gate_up;      // a pool: slot s of the pool tensors
+    p.mx_down = L.has_pool ? L.pool_down : L.mx_down;
     ACM_CUDA(launch_ffn_mxfp4(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
   } else {
     ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
@@ -593,7 +607,8 @@ acm_status acm_set_layer_weights(acm_ctx* c, int layer, const void* w_router, co
 
 acm_status acm_set_layer_weights_mxfp4(acm_ctx* c, int layer, const void* w_router, const float* router_bias,
                                        const void* gate_up_tiles, const void* down_tiles) {
-  if (!c || layer < 0 || layer >= c->desc.n_layers || !w_router || !gate_up_tiles || !down_tiles) return ACM_ERR_INVALID;
+  if (!c || layer < 0 || layer >= c->desc.n_layers || !w_router) return ACM_ERR_INVALID;
+  if ((gate_up_tiles == nullptr) != (down_tiles == nullptr)) return ACM_ERR_INVALID;
   const acm_model_desc& d = c->desc;
   if (d.dtype != ACM_BF16 || d.n_shared != 0 || d.inter % 128 != 0 || d.hidden % 128 != 0) return ACM_ERR_UNSUPPORTED;
   if (reinterpret_cast<uintptr_t>(w_router) % 16 != 0 || reinterpret_cast<uintptr_t>(gate_up_tiles) % 16 != 0 ||
@@ -605,6 +620,7 @@ acm_status acm_set_layer_weights_mxfp4(acm_ctx* c, int layer, const void* w_rout
   }
   Layer L;
   L.w_router = w_router; L.bias = router_bias;
+  L.mx = true;
   L.mx_gate_up = gate_up_tiles; L.mx_down = down_tiles;
   std::memset(&L.maps, 0, sizeof L.maps);      // the MXFP4 kernel fetches its weights with plain bulk copies
   L.set = true;
@@ -782,7 +798,8 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
     ACM_CUDA(cudaEventSynchronize(c->ev_lists));
     const int n_stage = c->host_stage_list[0];
     if (n_stage < 0 || n_stage > E) return ACM_ERR_CUDA;
-    const size_t gu = static_cast<size_t>(2) * d.inter * d.hidden * 2, dn = static_cast<size_t>(d.hidden) * d.inter * 2;
+    size_t gu, dn;
+    expert_tensor_bytes(d, L.mx, &gu, &dn);
     if (L.has_pool) {
       // LRU expert pool: the experts activated by this block that were resident are touched; the others
       // are loaded, synchronously with respect to their FFN, into the least recently used slots that this
@@ -1044,7 +1061,7 @@ acm_status acm_set_resident(acm_ctx* c, int layer, const uint32_t* resident_mask
     L.host_gate_up = L.host_down = nullptr;
     return ACM_OK;
   }
-  if (L.mx_gate_up) return ACM_ERR_UNSUPPORTED;   // MXFP4 layers are all-resident
+  if (L.mx) return ACM_ERR_UNSUPPORTED;   // MXFP4 layers: all-resident or behind a pool (acm_set_slot_pool)
   if (L.has_pool) return ACM_ERR_INVALID;      // clear the pool first (NULL mask)
   if (c->desc.dtype != ACM_BF16) return ACM_ERR_UNSUPPORTED;
   if (!host_gate_up || !host_down) return ACM_ERR_INVALID;
@@ -1062,7 +1079,6 @@ acm_status acm_set_resident(acm_ctx* c, int layer, const uint32_t* resident_mask
 acm_status acm_set_slot_pool(acm_ctx* c, int layer, int n_slots, void* pool_gate_up, void* pool_down,
                              const void* host_gate_up, const void* host_down, const int32_t* initial_experts,
                              int n_initial) {
-  if (c && layer >= 0 && layer < c->desc.n_layers && c->layers[layer].mx_gate_up) return ACM_ERR_UNSUPPORTED;
   if (!c || layer < 0 || layer >= c->desc.n_layers) return ACM_ERR_INVALID;
   const acm_model_desc& d = c->desc;
   if (d.dtype != ACM_BF16) return ACM_ERR_UNSUPPORTED;
@@ -1075,11 +1091,13 @@ acm_status acm_set_slot_pool(acm_ctx* c, int layer, int n_slots, void* pool_gate
     return ACM_ERR_INVALID;
   acm_status st = ensure_offload_common(c);
   if (st != ACM_OK) return st;
-  st = encode_gate_up(c, &L.pool_map_gu, pool_gate_up, n_slots);
-  if (st != ACM_OK) return st;
-  st = encode_down(c, &L.pool_map_dn, pool_down, n_slots);
-  if (st != ACM_OK) return st;
-  if (!L.gate_up) {          // no full device tensors: every descriptor the kernel is handed must still be valid
+  if (!L.mx) {                // (the MXFP4 kernel fetches its tile records with plain bulk copies)
+    st = encode_gate_up(c, &L.pool_map_gu, pool_gate_up, n_slots);
+    if (st != ACM_OK) return st;
+    st = encode_down(c, &L.pool_map_dn, pool_down, n_slots);
+    if (st != ACM_OK) return st;
+  }
+  if (!L.gate_up && !L.mx) {          // no full device tensors: every descriptor the kernel is handed must still be valid
     L.maps.gate_up = L.pool_map_gu;
     L.maps.down = L.pool_map_dn;
     if (d.n_shared == 0) {
@@ -1098,7 +1116,8 @@ acm_status acm_set_slot_pool(acm_ctx* c, int layer, int n_slots, void* pool_gate
   L.last_use.assign(n_slots, 0);
   L.tick = 0;
   L.pool_hits = L.pool_misses = L.pool_h2d = 0;
-  const size_t gu = static_cast<size_t>(2) * d.inter * d.hidden * 2, dn = static_cast<size_t>(d.hidden) * d.inter * 2;
+  size_t gu, dn;
+  expert_tensor_bytes(d, L.mx, &gu, &dn);
   for (int i = 0; i < n_initial; ++i) {
     const int e = initial_experts[i];
     if (e < 0 || e >= E || L.expert_slot[e] >= 0) return ACM_ERR_INVALID;

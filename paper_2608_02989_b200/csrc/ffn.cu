@@ -1286,7 +1286,7 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   a.sel_flag = L.sel_flag; a.sel_epoch = L.sel_epoch; a.sel_blocks = L.sel_blocks;
   a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask; a.trace = L.trace;
 #if ACM_FFN_MX
-  if (!L.mx_gate_up || !L.mx_down || L.I % 128 != 0 || L.n_shared != 0 || L.slot_of || L.resident) return cudaErrorInvalidValue;
+  if (!L.mx_gate_up || !L.mx_down || L.I % 128 != 0 || L.n_shared != 0) return cudaErrorInvalidValue;
   a.mx_gate_up = static_cast<const unsigned char*>(L.mx_gate_up);
   a.mx_down = static_cast<const unsigned char*>(L.mx_down);
 #endif

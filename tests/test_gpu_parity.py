@@ -503,8 +503,8 @@ def test_back_to_back_layers_without_host_synchronisation():
     ctx.close()
 
 
-@pytest.mark.parametrize("mode", [1, 0])
-def test_lru_expert_pool_over_a_sequence_of_blocks(mode):
+@pytest.mark.parametrize("mode,mx", [(1, False), (0, False), (1, True)])
+def test_lru_expert_pool_over_a_sequence_of_blocks(mode, mx):
     """Section 3.4's X-slot pool on a reduced config-5 layer: the expert tensors exist on the device only as pool
     slots; eight blocks in a row, each against the oracle run with the resident set an LRU model predicts, plus the
     model's hit / miss counts, loaded bytes and final slot contents."""
@@ -512,12 +512,25 @@ def test_lru_expert_pool_over_a_sequence_of_blocks(mode):
                     zipf_bias=True)            # skewed expert popularity: the activated set stays below the pool size
     w, _, alpha = _block(cfg, 3)
     E, X = cfg.n_experts, 24
-    host_gu, host_dn = w["gate_up"].cpu().pin_memory(), w["down"].cpu().pin_memory()
-    pool_gu = torch.full((X,) + tuple(w["gate_up"].shape[1:]), float("nan"), dtype=w["gate_up"].dtype, device=DEV)
-    pool_dn = torch.full((X,) + tuple(w["down"].shape[1:]), float("nan"), dtype=w["down"].dtype, device=DEV)
     initial = list(range(0, 24, 2))                 # 12 of the 20 slots start occupied
     ctx = _ctx(cfg)
-    ctx.set_layer_weights(0, w["w_router"], w["router_bias"], None, None)
+    expert_bytes = cfg.expert_bytes
+    if mx:
+        # the same layer with its experts in MXFP4: pool and host tensors hold tile records, the oracle sees the
+        # dequantised weights
+        m = _mx_layer(cfg, 3)
+        w["gate_up"], w["down"] = m["gate_up_deq"], m["down_deq"]
+        host_gu, host_dn = m["gate_up_tiles"].cpu().pin_memory(), m["down_tiles"].cpu().pin_memory()
+        pool_gu = torch.full((X,) + tuple(host_gu.shape[1:]), 0xFF, dtype=torch.uint8, device=DEV)
+        pool_dn = torch.full((X,) + tuple(host_dn.shape[1:]), 0xFF, dtype=torch.uint8, device=DEV)
+        ctx.set_layer_weights_mxfp4(0, w["w_router"], w["router_bias"], None, None)
+        expert_bytes = host_gu[0].numel() + host_dn[0].numel()
+        assert expert_bytes * 32 == cfg.expert_bytes // 2 * 17        # 4 bits + 1/32 byte per weight
+    else:
+        host_gu, host_dn = w["gate_up"].cpu().pin_memory(), w["down"].cpu().pin_memory()
+        pool_gu = torch.full((X,) + tuple(w["gate_up"].shape[1:]), float("nan"), dtype=w["gate_up"].dtype, device=DEV)
+        pool_dn = torch.full((X,) + tuple(w["down"].shape[1:]), float("nan"), dtype=w["down"].dtype, device=DEV)
+        ctx.set_layer_weights(0, w["w_router"], w["router_bias"], None, None)
     ctx.set_slot_pool(0, pool_gu, pool_dn, host_gu, host_dn, initial)
     model = _LruModel(X, initial)
     tot_hits = tot_misses = 0
@@ -542,7 +555,7 @@ def test_lru_expert_pool_over_a_sequence_of_blocks(mode):
         assert st["n_activated"] == len(activated) and st["n_staged"] == misses
     ps = ctx.pool_stats(0)
     assert (ps["hits"], ps["misses"]) == (tot_hits, tot_misses)
-    assert ps["h2d_bytes"] == tot_misses * cfg.expert_bytes
+    assert ps["h2d_bytes"] == tot_misses * expert_bytes
     assert ps["slot_expert"] == model.slot_expert
     assert tot_misses > 0 and tot_hits > 0
     ctx.close()
