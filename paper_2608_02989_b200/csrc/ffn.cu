@@ -993,30 +993,44 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     unsigned total = 0;
     for (int si = 0; si < n_seg; ++si) total += bars->plan.range[si].n_stages;
     bool ok = true;
-    for (unsigned it = 0; it < total && ok; ++it) {
+    // the row's packed data of the stage at hand
+    uint4 q[4];
+    uint32_t sc = 0;
+    auto fetch = [&](unsigned it) -> bool {
       const uint32_t s = it % kStages, par = (it / kStages) & 1u;
-      if (!(ok = mbar_wait(smem_u32(&bars->raw[s]), par, abort_flag, p.status))) break;
+      if (!mbar_wait(smem_u32(&bars->raw[s]), par, abort_flag, p.status)) return false;
       const unsigned char* A = stage_base + static_cast<size_t>(s) * kStageBytes;
-      const uint32_t sc = *reinterpret_cast<const uint32_t*>(A + kMxCodeBytes + r * 4);
+      // (the record keeps the row's four 16-byte pieces rotated by the row number, so that a warp's loads
+      // spread over all banks)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) q[b] = *reinterpret_cast<const uint4*>(A + r * 64 + 16 * (b ^ ((r >> 1) & 3)));
+      sc = *reinterpret_cast<const uint32_t*>(A + kMxCodeBytes + r * 4);
+      return true;
+    };
+    if (total > 0) ok = fetch(0);
+    for (unsigned it = 0; it < total && ok; ++it) {
+      const uint32_t s = it % kStages;
       const uint32_t a_tmem = tmem_base + my_lane + kAcc * kAccCols + s * kMxACols;
       tc_fence_after();
 #pragma unroll
       for (int b = 0; b < 4; ++b) {                     // 32 K = one scale = 16 columns
-        // (the record keeps the row's four 16-byte pieces rotated by the row number, so that a warp's loads
-        // spread over all banks)
-        const uint4 q = *reinterpret_cast<const uint4*>(A + r * 64 + 16 * (b ^ ((r >> 1) & 3)));
         const uint32_t field = min(((sc >> (8 * b)) & 0xffu) + 126u, 254u) << 7;
         const uint32_t c2 = field | (field << 16);
-        const uint32_t words[4] = {q.x, q.y, q.z, q.w};
+        const uint32_t words[4] = {q[b].x, q[b].y, q[b].z, q[b].w};
         uint32_t o[16];
 #pragma unroll
         for (int w = 0; w < 4; ++w) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t t = (words[w] >> (4 * j)) & 0x000f000fu;       // elements 2j (low half) and 2j+1 (high half)
-            const uint32_t enc = (t * 0x1040u) & 0x81c081c0u;
-            asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(o[4 * w + j]) : "r"(enc), "r"(c2));
-          }
+          // a word holds elements 2j (nibble j) and 2j+1 (nibble 4+j): pairs 0 and 1 are masked out where they
+          // sit -- the multiplier that moves magnitude and sign into place differs -- pairs 2 and 3 after one shift
+          const uint32_t w2 = words[w] >> 8;
+          const uint32_t e0 = ((words[w] & 0x000f000fu) * 0x1040u) & 0x81c081c0u;
+          const uint32_t e1 = ((words[w] & 0x00f000f0u) * 0x0104u) & 0x81c081c0u;
+          const uint32_t e2 = ((w2 & 0x000f000fu) * 0x1040u) & 0x81c081c0u;
+          const uint32_t e3 = ((w2 & 0x00f000f0u) * 0x0104u) & 0x81c081c0u;
+          asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(o[4 * w + 0]) : "r"(e0), "r"(c2));
+          asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(o[4 * w + 1]) : "r"(e1), "r"(c2));
+          asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(o[4 * w + 2]) : "r"(e2), "r"(c2));
+          asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(o[4 * w + 3]) : "r"(e3), "r"(c2));
         }
         tmem_st16(a_tmem + 16 * b, o);
       }
@@ -1024,6 +1038,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->full[s]));
+      if (it + 1 < total) ok = fetch(it + 1);
     }
 #endif
   } else {
