@@ -751,3 +751,28 @@ def test_mxfp4_layer_equals_the_bf16_layer_with_the_dequantised_weights(shape):
         rms = float(ref_out.double().pow(2).mean().sqrt())
         assert float((out - ref_out).abs().max()) <= 1e-3 * rms
     ctx.close()
+
+
+def test_multi_block_batch_on_an_mxfp4_layer():
+    """The batch call on an MXFP4 layer: per-block sets and routes as on the bf16 layer with the dequantised
+    weights, output rows within tolerance of the oracle."""
+    cfg = wl.scaled(wl.CONFIGS[3], n_layers=1, inter=256, n_experts=64)
+    ctx = _ctx(cfg, n_layers=2)
+    w = _mx_layer(cfg)
+    ctx.set_layer_weights_mxfp4(0, w["w_router"], w["router_bias"], w["gate_up_tiles"], w["down_tiles"])
+    x = wl.hidden_states(cfg, 0, DEV)
+    offsets, depths = wl.batch_tree_depths(cfg, 5)
+    p = wl.commitment_table(cfg)
+    alpha = torch.cat([acm.node_weights(depths[offsets[b]:offsets[b + 1]], p) for b in range(5)])
+    wq = dict(w, gate_up=w["gate_up_deq"], down=w["down_deq"])
+    _, refs = _batch_reference(cfg, wq, x, offsets, depths, {})
+    out, idx, wt, mask, act, stats = ctx.moe_verify_batch(0, x, offsets, alpha.to(DEV), want=True)
+    assert ctx.device_status() == acm.OK
+    for b, ref in enumerate(refs):
+        np.testing.assert_array_equal(_u32(mask[b]), ref["mask"])
+        np.testing.assert_array_equal(idx[offsets[b]:offsets[b + 1]].cpu().numpy(), ref["idx"])
+    ref_idx = np.concatenate([r["idx"] for r in refs])
+    ref_w = np.concatenate([r["w"] for r in refs])
+    ffn = oracle.expert_ffn(x, ref_idx, ref_w, w["gate_up_deq"], w["down_deq"])
+    _ffn_check(out, ffn, "MXFP4 batch")
+    ctx.close()
