@@ -225,7 +225,8 @@ def run_pool(args):
             hits += ps["hits"]; misses += ps["misses"]; h2d += ps["h2d_bytes"]
         res[name] = {"layer_blocks_per_s": n_blocks * L / dt, "hit_rate": hits / max(hits + misses, 1),
                      "activated_per_layer_block": (hits + misses) / (n_blocks * L),
-                     "h2d_mib_per_layer_block": h2d / 2 ** 20 / (n_blocks * L)}
+                     "h2d_mib_per_layer_block": h2d / 2 ** 20 / (n_blocks * L),
+                     "h2d_gbs": h2d / dt / 1e9}      # host->device rate over the whole run (the bound of this variant)
     line = {"metric": METRIC, "value": res["restricted_eq7"]["layer_blocks_per_s"], "unit": UNIT, "n_gpus": 1,
             "steps": n_blocks, "warmup": 0, "higher_is_better": True, "dtype": cfg.dtype, "data": "synthetic",
             "config": {"workload": f"C5 {cfg.name}-shaped layers{' in MXFP4' if args.mxfp4 else ''} with Zipf-biased routing behind an LRU pool of {X} "
