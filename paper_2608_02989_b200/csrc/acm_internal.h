@@ -52,6 +52,7 @@ struct Workspace {
   int32_t* tile_done;   // [64] router kernel: expert tiles finished per node tile (self-resetting)
   int32_t* ticket;      // [1] select/route kernel: finished CTAs (self-resetting)
   uint32_t* sel_words;  // [kMaxEarlyBlocks][8] the eligible masks as tagged 16-bit pieces (early start of the FFN kernel)
+  uint32_t* anc_words;  // [8] the anchor experts (the root's natural top-k) as tagged 16-bit pieces, published by the router kernel
 };
 
 struct SelectArgs {
@@ -114,7 +115,8 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
                                  float* logits, int T, int H, int E, float* zero_buf,
                                  size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status,
                                  float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k, int32_t* tile_done,
-                                 bool pdl, cudaStream_t s, long long* dbg = nullptr);
+                                 bool pdl, cudaStream_t s, long long* dbg = nullptr, uint32_t* anc_words = nullptr,
+                                 uint32_t anc_tag = 0);
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s);
 // select (unless mask_override) + route + the FFN kernel's routing inputs in ONE launch of ceil(T/4)
@@ -158,6 +160,8 @@ struct FfnLaunch {
   const uint32_t* sel_flag;
   int32_t sel_epoch;
   int sel_blocks;            // blocks of a batch (1..kMaxEarlyBlocks): eight words each, the work list is their union
+  const uint32_t* anc_flag = nullptr;   // with sel_flag: eight words tagged alike holding the anchor experts (published by the
+                             // router kernel, earlier): their gate/up tiles are streamed while the selection still runs
   float* out;                // [T,H], accumulated into (zeroed by the caller)
   int32_t* status;
   int grid;

@@ -153,6 +153,7 @@ struct acm_ctx {
   uint64_t launches = 0;
   bool split_phases = false;             // ACM_FFN_SPLIT_PHASES=1 in the environment
   unsigned long long* trace = nullptr;   // ACM_FFN_TRACE=1|2: per-CTA timestamps of the last FFN launch
+  bool anchor_start = true;              // ACM_NO_ANCHOR_START=1: the FFN kernel starts on the eligible set only
   bool mx_configured = false;
   bool trace_light = false;              // =2: leave the launch sequence as it is (stale slots are not cleared)
 };
@@ -295,7 +296,8 @@ void expert_tensor_bytes(const acm_model_desc& d, bool mx, size_t* gu, size_t* d
 // One FFN launch over work list `li` (0 = resident + shared, 1 = staged).
 acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li, float* out, cudaStream_t s,
                         const uint32_t* res_dev = nullptr, acm_block_stats* stats_dev = nullptr, bool pdl_ok = false,
-                        int32_t early_epoch = 0, const uint32_t* only = nullptr, int n_blocks = 0) {
+                        int32_t early_epoch = 0, const uint32_t* only = nullptr, int n_blocks = 0,
+                        bool anchors_first = false) {
   const acm_model_desc& d = c->desc;
   const int n_pad = (T + 15) / 16 * 16;
   acm_status st = ensure_h_maps(c, n_pad);
@@ -328,6 +330,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   if (early_epoch != 0) {
     p.sel_flag = c->ws.sel_words;
     p.sel_epoch = early_epoch;
+    if (anchors_first) p.anc_flag = c->ws.anc_words;
   }
   p.out = out; p.status = c->ws.status;
   p.grid = c->sm_count;
@@ -453,6 +456,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->split_phases = split && split[0] == '1';
   const char* no_pdl = std::getenv("ACM_NO_PDL");
   c->pdl = !(no_pdl && no_pdl[0] == '1');
+  const char* no_anc = std::getenv("ACM_NO_ANCHOR_START");
+  c->anchor_start = !(no_anc && no_anc[0] == '1');
   const char* no_early = std::getenv("ACM_NO_EARLY_START");
   c->early_start = !(no_early && no_early[0] == '1');
   const char* trace = std::getenv("ACM_FFN_TRACE");
@@ -502,6 +507,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_tile = carve(sizeof(int32_t) * kMaxNodes);
   const size_t o_ticket = carve(16);
   const size_t o_selw = carve(32 * kMaxEarlyBlocks);
+  const size_t o_ancw = carve(32);
   const size_t o_natmask = carve(sizeof(uint32_t) * Tm * kMaskWords);
   const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
   if (cudaMalloc(&c->ws_base, off) != cudaSuccess) return fail(ACM_ERR_NOMEM);
@@ -531,6 +537,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.tile_done = reinterpret_cast<int32_t*>(b + o_tile);
   c->ws.ticket = reinterpret_cast<int32_t*>(b + o_ticket);
   c->ws.sel_words = reinterpret_cast<uint32_t*>(b + o_selw);
+  c->ws.anc_words = reinterpret_cast<uint32_t*>(b + o_ancw);
   c->ws.nat_mask = reinterpret_cast<uint32_t*>(b + o_natmask);
   c->resident_dev = reinterpret_cast<uint32_t*>(b + o_res);
   if (want_trace && cudaMalloc(&c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 32)) != cudaSuccess)
@@ -741,6 +748,19 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   const bool f32 = d.dtype == ACM_F32;
   uint32_t* res_dev = L.has_resident ? c->resident_dev + 4 * layer : nullptr;
 
+  // Early start of the FFN kernel on the eligible set: when a selection runs (the eligible experts are
+  // then nearly always all activated; with an override mask they need not be) and every expert is resident.
+  const bool early = !f32 && !L.has_resident && !eligible_mask_override && !c->split_phases && c->early_start;
+  int32_t early_epoch = 0;
+  if (early) {
+    early_epoch = ++c->epoch;            // its low 16 bits tag the published words; 0 is never a valid tag
+    if ((early_epoch & 0xffff) == 0) early_epoch = ++c->epoch;
+    if (early_epoch <= 0) early_epoch = c->epoch = 1;
+  }
+  // ... and earlier still on the anchors (Eq. 5 with the default anchor, the root): the router kernel publishes
+  // the root's natural top-k as soon as that row is done, the FFN kernel streams their gate/up tiles while
+  // the selection runs.  They are in every eligible set the selection can return without a residency.
+  const bool anchors_first = early && c->anchor_start && c->pdl && prm.use_anchors != 0 && !L.mx;
   // stage 1 (also clears the output the FFN accumulates into and the FFN kernel's routing inputs)
   const bool need_probs = eligible_mask_override == nullptr;
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
@@ -748,7 +768,8 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
                                 c->ws.status,
                                 need_probs ? c->ws.probs : nullptr, need_probs ? c->ws.nat_idx : nullptr,
                                 need_probs ? c->ws.nat_mask : nullptr, k, c->ws.tile_done, c->pdl, s,
-                                c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr));
+                                c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr,
+                                anchors_first ? c->ws.anc_words : nullptr, static_cast<uint32_t>(early_epoch) & 0xffffu));
   // stages 2-3: one launch of a few small CTAs, which also fill the FFN kernel's routing inputs
   SelectArgs sa;
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
@@ -766,14 +787,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   ra.stats_out = stats_dev;
   // the bf16 FFN kernel counts the activated experts itself; otherwise the routing kernel's last CTA does
   ra.ticket = (f32 || L.has_resident) ? c->ws.ticket : nullptr;
-  // Early start of the FFN kernel on the eligible set: when a selection runs (the eligible experts are
-  // then nearly always all activated; with an override mask they need not be) and every expert is resident.
-  const bool early = !f32 && !L.has_resident && !eligible_mask_override && !c->split_phases && c->early_start;
-  int32_t early_epoch = 0;
   if (early) {
-    early_epoch = ++c->epoch;            // its low 16 bits tag the published words; 0 is never a valid tag
-    if ((early_epoch & 0xffff) == 0) early_epoch = ++c->epoch;
-    if (early_epoch <= 0) early_epoch = c->epoch = 1;
     ra.sel_flag = c->ws.sel_words;
     ra.sel_epoch = early_epoch;
   }
@@ -788,7 +802,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
                             static_cast<float*>(c->ws.hbuf), out, T, d.hidden, d.inter, k, s));
     c->launches += 2;
   } else if (!L.has_resident) {
-    st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, stats_dev, true, early_epoch);
+    st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, stats_dev, true, early_epoch, nullptr, 0, anchors_first);
     if (st != ACM_OK) return st;
   } else {
     // resident + shared experts run at once; the others are copied in from pinned host memory first
@@ -1286,6 +1300,7 @@ acm_status acm_device_status(acm_ctx* c, acm_stream stream) {
     ACM_CUDA(cudaMemset(c->ws.frag_flag, 0, c->flag_bytes));
     ACM_CUDA(cudaMemset(c->ws.ticket, 0, 16));
     ACM_CUDA(cudaMemset(c->ws.sel_words, 0, 32 * kMaxEarlyBlocks));
+    ACM_CUDA(cudaMemset(c->ws.anc_words, 0, 32));
     c->epoch = 0;
     ACM_CUDA(cudaMemset(c->ws.tile_done, 0, sizeof(int32_t) * kMaxNodes));
   }

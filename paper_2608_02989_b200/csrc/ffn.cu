@@ -128,9 +128,10 @@ struct SegRange {
   unsigned n_stages;     // pipeline stages this CTA runs in the segment
 };
 struct Plan {
-  Segment seg[4];
-  SegRange range[4];   // this CTA's share of each segment
-  int n_seg;
+  Segment seg[5];      // [0] may be the anchors' pre-segment (see the kernel's early start), then up to four
+  SegRange range[5];   // this CTA's share of each segment
+  volatile int n_seg;
+  int n_pre;      // experts whose gate/up tiles the pre-segment covers (the first slots of the work list)
   int a_split;    // experts [0, a_split) form group 0 (complete early), the rest group 1
 };
 
@@ -145,6 +146,7 @@ struct __align__(8) Barriers {
   unsigned long long helper;         // completion of the helper warp's bulk copy
   unsigned long long ost_full, ost_free;   // epilogue <-> publisher: outgoing fragment staged / copied out
   unsigned long long hst_full[2], hst_free[2];   // epilogue <-> publisher: activation tile staged / stored
+  unsigned long long plan_ready;     // anchors' pre-segment: the rest of the plan and of the work list is in place
 #if ACM_FFN_MX
   unsigned long long raw[kStages];   // the packed weight stage has landed (producer's copy -> expanding warps)
 #endif
@@ -154,6 +156,7 @@ struct __align__(8) Barriers {
   float wd[kMaxNodes];          // combine weights of the expert being finalised
   int32_t entry[kMaxSlots];     // this launch's work list: make_entry(source, index) of every activated slot
   int32_t expert[kMaxSlots];    // routed expert id of the slot (-1: shared expert)
+  uint32_t anc_half[2 * kMaskWords];   // early start on the anchors: their mask in 16-bit pieces
   uint32_t sel_half[4 * kMaskWords];   // early start: the eligible mask in 16-bit pieces (second half: blocks 4..7 of a batch)
   Plan plan;                    // this launch's work plan
 };
@@ -404,6 +407,7 @@ struct FfnArgs {
   const uint32_t* sel_flag;
   int32_t sel_epoch;
   int sel_blocks;
+  const uint32_t* anc_flag;    // non-null: eight tagged words with the anchor experts (Eq. 5), published before sel_flag
   float* out;
   int32_t* status;
   int phase_mask;
@@ -425,7 +429,7 @@ __device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMa
 // present or not -- and its own range in it, so nothing waits for a serial pass.
 __device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act, int tpe, int grid, int phase_mask,
                                           const FastDiv& d_kc1, int kpe, const FastDiv& d_grid, const FastDiv& d_tpe,
-                                          int h_tiles);
+                                          int h_tiles, int n_pre = 0, int base = 0);
 // Range of segment `si` for CTA `cta` (see SegRange).  (tiles * chunks * grid fits 32 bits: launcher.)
 __device__ __forceinline__ SegRange make_range(const Segment& sg, int cta, const FastDiv& d_grid, int h_tiles) {
   SegRange r;
@@ -449,10 +453,14 @@ __device__ __forceinline__ SegRange make_range(const Segment& sg, int cta, const
   return r;
 }
 
+// With a pre-segment (n_pre experts whose gate/up tiles are already being streamed as segment 0, base = 1) the
+// gate/up segments cover the other experts' tiles only; the down segments cover everyone, the pre-streamed experts
+// counting as complete early.
 __device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act, int tpe, int grid, int phase_mask,
                                           const FastDiv& d_kc1, int kpe, const FastDiv& d_grid, const FastDiv& d_tpe,
-                                          int h_tiles) {
-  const int n_t = n_act * tpe;
+                                          int h_tiles, int n_pre, int base) {
+  const int t_pre = n_pre * tpe;
+  const int n_t = (n_act - n_pre) * tpe;
   const int rounds = static_cast<int>(fdiv(static_cast<unsigned>(n_t), d_grid)), rem = n_t - rounds * grid;
   const bool p1 = (phase_mask & 1) != 0, p2 = (phase_mask & 2) != 0;
   // candidates in execution order: two gate/up segments, two down segments
@@ -460,14 +468,14 @@ __device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act
   bool h0, h1, h2, h3;
   int a_split;
   if (rounds == 0) {
-    const int nA = (n_act + 1) / 2;
-    a_split = nA;
-    c0 = Segment{1, 0, 0, nA * tpe, 0, 0, 0, d_kc1};                          h0 = p1 && nA > 0;
-    c1 = Segment{1, 0, nA * tpe, (n_act - nA) * tpe, 0, 0, 1, d_kc1};         h1 = p1 && n_act > nA;
+    const int n_rest = n_act - n_pre, nA = (n_rest + 1) / 2;
+    a_split = n_pre + nA;
+    c0 = Segment{1, 0, t_pre, nA * tpe, 0, 0, 0, d_kc1};                      h0 = p1 && nA > 0;
+    c1 = Segment{1, 0, t_pre + nA * tpe, (n_rest - nA) * tpe, 0, 0, 1, d_kc1};   h1 = p1 && n_rest > nA;
   } else {
-    a_split = static_cast<int>(fdiv(static_cast<unsigned>(rem + (rounds - 1) * grid), d_tpe));
-    c0 = Segment{1, 0, 0, rem, 0, 0, 0, d_kc1};                               h0 = p1 && rem > 0;
-    c1 = Segment{1, 1, rem, rounds * grid, 0, 0, 1, d_kc1};                   h1 = p1;
+    a_split = n_pre + static_cast<int>(fdiv(static_cast<unsigned>(rem + (rounds - 1) * grid), d_tpe));
+    c0 = Segment{1, 0, t_pre, rem, 0, 0, 0, d_kc1};                           h0 = p1 && rem > 0;
+    c1 = Segment{1, 1, t_pre + rem, rounds * grid, 0, 0, 1, d_kc1};           h1 = p1;
   }
   c2 = Segment{2, 0, 0, 0, 0, a_split, 0, plain_div(static_cast<unsigned>(a_split * kpe))};                 h2 = p2 && a_split > 0;
   c3 = Segment{2, 0, 0, 0, a_split, n_act, 1, plain_div(static_cast<unsigned>((n_act - a_split) * kpe))};   h3 = p2 && n_act > a_split;
@@ -479,13 +487,12 @@ __device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act
   if (h2 && i2 == lane) { mine = c2; have = true; }
   if (h3 && i3 == lane) { mine = c3; have = true; }
   if (have) {
-    pl.seg[lane] = mine;
-    pl.range[lane] = make_range(mine, cta, d_grid, h_tiles);
+    pl.seg[base + lane] = mine;
+    pl.range[base + lane] = make_range(mine, cta, d_grid, h_tiles);
   }
-  if (lane == 0) {
-    pl.n_seg = n;
-    pl.a_split = a_split;
-  }
+  if (lane == 0) pl.a_split = a_split;
+  __syncwarp(0xfu);            // (called by lanes 0..3: the segments are in place before their count is)
+  if (lane == 0) pl.n_seg = base + n;
 }
 
 #if ACM_FFN_MX
@@ -525,6 +532,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       mbar_init(smem_u32(&bars->tempty[b]), 128);
     }
     mbar_init(smem_u32(&bars->drained), 1);
+    mbar_init(smem_u32(&bars->plan_ready), 1);
     mbar_init(smem_u32(&bars->frag_full[0]), 1);
     mbar_init(smem_u32(&bars->frag_full[1]), 1);
     mbar_init(smem_u32(&bars->frag_free), 128);
@@ -554,8 +562,34 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   // Everything above touched only this CTA's own resources; global memory written by the kernels
   // before this one is read only from here on.  Early start: wait for the eligible set only.
   const bool early = p.sel_flag != nullptr;
+  // Early start on the ANCHORS (Eq. 5: the root's natural top-k, always eligible): the router kernel publishes
+  // them microseconds before the selection is done.  Their gate/up tiles become segment 0 of the plan, one
+  // whole tile per CTA, and the roles start on it at once; the helper warp meanwhile waits for the eligible
+  // set, completes the work list (the pre-streamed experts keep the first slots) and the plan, and opens
+  // `plan_ready`, which every other role passes before its second segment.
+  const bool pre = early && p.anc_flag != nullptr;
   if (threadIdx.x == 0) ACM_TRACE(29);
-  if (early) {
+  if (pre) {
+    bool timed_out = false;
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + 2 * kMaskWords) {
+      const int i = threadIdx.x - 64;
+      bool seen = false;
+      uint32_t v = 0;
+      const uint32_t tag = static_cast<uint32_t>(p.sel_epoch) & 0xffffu;
+      const unsigned long long t0 = global_timer();
+      do {
+        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.anc_flag + i) : "memory");
+        seen = (v >> 16) == tag;
+      } while (!seen && global_timer() - t0 < kTimeoutNs);
+      timed_out = !seen;
+      bars->anc_half[i] = seen ? (v & 0xffffu) : 0u;
+    }
+    __syncthreads();
+    if (timed_out) {
+      bars->abort_flag = 1;
+      atomicCAS(p.status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+    }
+  } else if (early) {
     // eight tagged words (16 mask bits under the 16-bit tag of this call), each polled by its own thread --
     // of warp 2, which has nothing else to do yet, so that the poll runs beside the set-up above
     bool timed_out = false;
@@ -611,7 +645,9 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
 #pragma unroll
   for (int wd = 0; wd < kMaskWords; ++wd) {
     uint32_t act;
-    if (early) {
+    if (pre) {
+      act = bars->anc_half[2 * wd] | (bars->anc_half[2 * wd + 1] << 16);      // for now: the anchors only
+    } else if (early) {
       act = bars->sel_half[2 * wd] | (bars->sel_half[2 * wd + 1] << 16);
       if (p.sel_blocks > 1) act |= bars->sel_half[2 * kMaskWords + 2 * wd] | (bars->sel_half[2 * kMaskWords + 2 * wd + 1] << 16);
     } else {
@@ -621,15 +657,42 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     am[wd] = (p.li == 0 ? act & res : act & ~res) & p.only[wd];
     n_routed += __popc(am[wd]);
   }
-  const int n_act = n_routed + (p.li == 0 ? p.n_shared : 0);
   const int tpe = p.I / 64;          // gate/up tiles per expert = K-chunks per expert in the down phase
+  // pre-segment: as many of the anchors (in ascending id) as give every CTA at most one whole tile
+  const int n_pre = pre ? min(n_routed, static_cast<int>(fdiv(static_cast<unsigned>(G), p.d_tpe))) : 0;
+  if (pre) {
+    // keep the first n_pre anchors only
+    int left = n_pre;
+#pragma unroll
+    for (int wd = 0; wd < kMaskWords; ++wd) {
+      uint32_t m = am[wd], kept = 0u;
+      while (m && left > 0) {
+        const uint32_t bit = m & (0u - m);
+        kept |= bit;
+        m ^= bit;
+        --left;
+      }
+      am[wd] = kept;
+    }
+    n_routed = n_pre;
+  }
+  const int n_act = n_routed + ((p.li == 0 && !pre) ? p.n_shared : 0);
   const int kc1 = p.H / (kBK * kAtoms);   // K-chunks (stages) of a gate/up tile
   const int kpe = (tpe + kAtoms - 1) / kAtoms;   // K-chunks (stages) per expert in the down phase
   const int h_tiles = p.H / kTileM;  // output tiles of the down phase
   const uint32_t b_atom_bytes = static_cast<uint32_t>(p.n_pad) * kBK * 2;   // one atom of the activation chunk
   const uint32_t b_bytes = kAtoms * b_atom_bytes;
-  if (warp == kThreads / 32 - 1 && lane < 4)      // (the publisher warp has nothing else to do yet)
+  if (pre) {
+    if (threadIdx.x == kThreads - 32) {            // segment 0: the pre-streamed experts' tiles, one whole tile per CTA
+      Segment sg0 = Segment{1, 1, 0, n_pre * tpe, 0, 0, 0, p.d_kc1};
+      bars->plan.seg[0] = sg0;
+      bars->plan.range[0] = make_range(sg0, cta, p.d_grid, h_tiles);
+      bars->plan.n_pre = n_pre;
+      bars->plan.n_seg = 1;
+    }
+  } else if (warp == kThreads / 32 - 1 && lane < 4) {      // (the publisher warp has nothing else to do yet)
     plan_lane(bars->plan, lane, cta, n_act, tpe, G, p.phase_mask, p.d_kc1, kpe, p.d_grid, p.d_tpe, h_tiles);
+  }
   int32_t* s_entry = bars->entry;
   if (threadIdx.x < kMaxExperts) {
     const int e = threadIdx.x, wd = e >> 5;
@@ -644,7 +707,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
                                 : p.li == 0 ? make_entry(kSrcRouted, e) : make_entry(kSrcStaged, slot);
       bars->expert[slot] = e;
     }
-  } else if (p.li == 0 && threadIdx.x - kMaxExperts < p.n_shared) {
+  } else if (p.li == 0 && !pre && threadIdx.x - kMaxExperts < p.n_shared) {
     const int i = threadIdx.x - kMaxExperts;
     s_entry[n_routed + i] = make_entry(kSrcShared, i);
     bars->expert[n_routed + i] = -1;
@@ -654,9 +717,14 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const Segment* seg = bars->plan.seg;
-  const int n_seg = bars->plan.n_seg;
   const uint32_t tmem_base = bars->tmem_base;
   if (threadIdx.x == 0) ACM_TRACE(0);
+  // Does segment si exist?  With a pre-segment the plan behind segment 0 arrives later (the helper warp opens
+  // plan_ready); n_seg is read from shared memory every time.
+  auto have_seg = [&](int si, bool wait_for_plan) -> bool {
+    if (pre && si == 1 && wait_for_plan && !mbar_wait(smem_u32(&bars->plan_ready), 0u, abort_flag, p.status)) return false;
+    return si < bars->plan.n_seg;
+  };
 
   if (warp == 0) {
     // ------------------------------------------------------------------ weight producer
@@ -668,7 +736,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
       uint32_t s = 0, par = 0, n_armed = 0;
       bool ok = true, traced_first = false;
-      for (int si = 0; si < n_seg && ok; ++si) {
+      for (int si = 0; ok && have_seg(si, true); ++si) {
         const Segment sg = seg[si];
         if (sg.phase == 1) {
           Sched sc(bars->plan.range[si]);
@@ -767,7 +835,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       uint32_t it = 0, f = 0;
       bool ok = true;
       unsigned long long acc_f[2] = {0, 0};
-      for (int si = 0; si < n_seg && ok; ++si) {
+      for (int si = 0; ok && have_seg(si, true); ++si) {
         const Segment sg = seg[si];
         Sched sc(bars->plan.range[si]);
         int tile, k0, k1;
@@ -824,7 +892,61 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     bool ok = true;
     int frag_uses = 0;
     uint32_t hs = 0, hidx = 0;   // ring slot and running index of the next stage, tracked through the gate/up stages too
-    for (int si = 0; si < n_seg && ok; ++si) {
+    if (pre) {
+      // While the others run the anchors' pre-segment: wait for the eligible set, give the other experts the
+      // slots behind the pre-streamed ones (ascending id), append the shared experts, work out the rest of the
+      // plan, and let everyone on.
+      uint32_t v = 0;
+      bool seen = true;
+      if (lane < 2 * kMaskWords) {
+        const uint32_t tag = static_cast<uint32_t>(p.sel_epoch) & 0xffffu;
+        const unsigned long long t0 = global_timer();
+        do {
+          asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.sel_flag + lane) : "memory");
+          seen = (v >> 16) == tag;
+        } while (!seen && global_timer() - t0 < kTimeoutNs);
+      }
+      const bool good = __all_sync(0xffffffffu, seen);
+      const uint32_t half = v & 0xffffu;
+      uint32_t rest[kMaskWords];
+      int n_rest = 0;
+#pragma unroll
+      for (int wd = 0; wd < kMaskWords; ++wd) {
+        const uint32_t lo = __shfl_sync(0xffffffffu, half, 2 * wd), hi = __shfl_sync(0xffffffffu, half, 2 * wd + 1);
+        rest[wd] = ((lo | (hi << 16)) & p.only[wd]) & ~am[wd];
+        n_rest += __popc(rest[wd]);
+      }
+      if (good) {
+        for (int e = lane; e < kMaxExperts; e += 32) {
+          const int wd = e >> 5;
+          const uint32_t mine = wd == 0 ? rest[0] : wd == 1 ? rest[1] : wd == 2 ? rest[2] : rest[3];
+          if ((mine >> (e & 31)) & 1u) {
+            int slot = n_pre + __popc(mine & ((1u << (e & 31)) - 1u));
+#pragma unroll
+            for (int w2 = 0; w2 < kMaskWords; ++w2) slot += w2 < wd ? __popc(rest[w2]) : 0;
+            s_entry[slot] = make_entry(kSrcRouted, e);
+            bars->expert[slot] = e;
+          }
+        }
+        if (lane < p.n_shared) {
+          s_entry[n_pre + n_rest + lane] = make_entry(kSrcShared, lane);
+          bars->expert[n_pre + n_rest + lane] = -1;
+        }
+        if (lane < 4)
+          plan_lane(bars->plan, lane, cta, n_pre + n_rest + p.n_shared, tpe, G, p.phase_mask, p.d_kc1, kpe, p.d_grid, p.d_tpe,
+                    h_tiles, n_pre, 1);
+      } else if (lane == 0) {
+        bars->abort_flag = 1;
+        atomicCAS(p.status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+      }
+      __syncwarp();
+      if (lane == 0) {
+        ACM_TRACE(30);
+        mbar_arrive(smem_u32(&bars->plan_ready));
+      }
+      ok = good;
+    }
+    for (int si = 0; ok && have_seg(si, false); ++si) {
       const Segment sg = seg[si];
       const int n_exp = sg.a1 - sg.a0;
       if (sg.phase == 1) {
@@ -937,7 +1059,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     if (lane == 0) {
       uint32_t ost_n = 0, fin_n = 0;
       bool ok = true;
-      for (int si = 0; si < n_seg && ok; ++si) {
+      for (int si = 0; ok && have_seg(si, true); ++si) {
         const Segment sg = seg[si];
         if (sg.phase != 1) continue;
         float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * kFragFloats;
@@ -991,7 +1113,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     const int r = threadIdx.x - 256;
     const uint32_t my_lane = static_cast<uint32_t>(r & ~31) << 16;          // this warp's quarter of the lanes
     unsigned total = 0;
-    for (int si = 0; si < n_seg; ++si) total += bars->plan.range[si].n_stages;
+    for (int si = 0; si < bars->plan.n_seg; ++si) total += bars->plan.range[si].n_stages;
     bool ok = true;
     // the row's packed data of the stage at hand
     uint4 q[4];
@@ -1066,7 +1188,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       if (ost_uses == 0) return true;
       return epi_vote_all(mbar_wait(smem_u32(&bars->ost_free), (ost_uses - 1) & 1u, abort_flag, p.status));
     };
-    for (int si = 0; si < n_seg && ok; ++si) {
+    for (int si = 0; ok && have_seg(si, true); ++si) {
       const Segment sg = seg[si];
       if (sg.phase == 1) {
         Sched sc(bars->plan.range[si]);
@@ -1299,6 +1421,7 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   a.stats = L.stats; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
   a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag;
   a.sel_flag = L.sel_flag; a.sel_epoch = L.sel_epoch; a.sel_blocks = L.sel_blocks;
+  a.anc_flag = (ACM_FFN_MX || L.sel_blocks != 1 || L.li != 0 || L.resident || L.slot_of || L.phase_mask != 3) ? nullptr : L.anc_flag;
   a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask; a.trace = L.trace;
 #if ACM_FFN_MX
   if (!L.mx_gate_up || !L.mx_down || L.I % 128 != 0 || L.n_shared != 0) return cudaErrorInvalidValue;
