@@ -330,7 +330,6 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   if (early_epoch != 0) {
     p.sel_flag = c->ws.sel_words;
     p.sel_epoch = early_epoch;
-    if (anchors_first) p.anc_flag = c->ws.anc_words;
   }
   p.out = out; p.status = c->ws.status;
   p.grid = c->sm_count;
@@ -355,6 +354,9 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   }
   // dependent launch only straight after the select/route kernel (no event, memset or copy between)
   p.pdl = pdl_ok && c->pdl && !e0 && (!c->trace || c->trace_light) && !c->split_phases;
+  // the anchors' pre-segment pays only when this launch overlaps the selection; a launch ordered after it (one
+  // bracketed by events) has the whole set at hand and takes the balanced plan
+  if (anchors_first && p.pdl && early_epoch != 0) p.anc_flag = c->ws.anc_words;
   // Straight after the routing kernel: the few SMs it ran on (or still holds, in an early start) take
   // microseconds longer to accept a CTA of this kernel -- an SM changes hands slowly when the shared-memory
   // split changes -- and one late CTA delays every CTA that exchanges fragments with it.  Leave them out.

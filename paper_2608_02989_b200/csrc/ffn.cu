@@ -146,7 +146,6 @@ struct __align__(8) Barriers {
   unsigned long long helper;         // completion of the helper warp's bulk copy
   unsigned long long ost_full, ost_free;   // epilogue <-> publisher: outgoing fragment staged / copied out
   unsigned long long hst_full[2], hst_free[2];   // epilogue <-> publisher: activation tile staged / stored
-  unsigned long long plan_ready;     // anchors' pre-segment: the rest of the plan and of the work list is in place
 #if ACM_FFN_MX
   unsigned long long raw[kStages];   // the packed weight stage has landed (producer's copy -> expanding warps)
 #endif
@@ -156,9 +155,10 @@ struct __align__(8) Barriers {
   float wd[kMaxNodes];          // combine weights of the expert being finalised
   int32_t entry[kMaxSlots];     // this launch's work list: make_entry(source, index) of every activated slot
   int32_t expert[kMaxSlots];    // routed expert id of the slot (-1: shared expert)
-  uint32_t anc_half[2 * kMaskWords];   // early start on the anchors: their mask in 16-bit pieces
   uint32_t sel_half[4 * kMaskWords];   // early start: the eligible mask in 16-bit pieces (second half: blocks 4..7 of a batch)
   Plan plan;                    // this launch's work plan
+  unsigned long long plan_ready;     // anchors' pre-segment: the rest of the plan and of the work list is in place
+  uint32_t anc_half[2 * kMaskWords];   // early start on the anchors: their mask in 16-bit pieces
 };
 
 static_assert(sizeof(Barriers) <= 232448 - 1024 - kStages * kStageBytes - kOutStageBytes - kFragBytes - 2 * kHStageBytes,
@@ -500,6 +500,9 @@ __device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act
 #else
 #define ACM_FFN_KERNEL k_ffn_bf16
 #endif
+// kPre: the variant that starts on the anchors' pre-segment (compiled apart, so that the plain variant's code is
+// exactly what it is without it)
+template <bool kPre>
 __global__ void __launch_bounds__(kThreads, 1)
 ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtensorMap x_map,
            const __grid_constant__ CUtensorMap h_map, const __grid_constant__ CUtensorMap hs_map,
@@ -567,7 +570,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   // whole tile per CTA, and the roles start on it at once; the helper warp meanwhile waits for the eligible
   // set, completes the work list (the pre-streamed experts keep the first slots) and the plan, and opens
   // `plan_ready`, which every other role passes before its second segment.
-  const bool pre = early && p.anc_flag != nullptr;
+  constexpr bool pre = kPre;
   if (threadIdx.x == 0) ACM_TRACE(29);
   if (pre) {
     bool timed_out = false;
@@ -721,9 +724,14 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   if (threadIdx.x == 0) ACM_TRACE(0);
   // Does segment si exist?  With a pre-segment the plan behind segment 0 arrives later (the helper warp opens
   // plan_ready); n_seg is read from shared memory every time.
+  const int n_seg_fixed = bars->plan.n_seg;
   auto have_seg = [&](int si, bool wait_for_plan) -> bool {
-    if (pre && si == 1 && wait_for_plan && !mbar_wait(smem_u32(&bars->plan_ready), 0u, abort_flag, p.status)) return false;
-    return si < bars->plan.n_seg;
+    if constexpr (kPre) {
+      if (si == 1 && wait_for_plan && !mbar_wait(smem_u32(&bars->plan_ready), 0u, abort_flag, p.status)) return false;
+      return si < bars->plan.n_seg;
+    } else {
+      return si < n_seg_fixed;
+    }
   };
 
   if (warp == 0) {
@@ -1387,7 +1395,7 @@ __global__ void k_ffn_f32_down(const float* __restrict__ down, const float* __re
 
 #if ACM_FFN_MX
 cudaError_t ffn_mx_configure() {
-  return cudaFuncSetAttribute(ACM_FFN_KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  return cudaFuncSetAttribute(ACM_FFN_KERNEL<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
 }
 cudaError_t launch_ffn_mxfp4(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
                              const CUtensorMap& h_map, const CUtensorMap& hs_map, cudaStream_t s) {
@@ -1395,7 +1403,9 @@ cudaError_t launch_ffn_mxfp4(const FfnLaunch& L, const FfnMaps& maps, const CUte
 size_t ffn_smem_bytes() { return kSmemBytes; }
 
 cudaError_t ffn_configure() {
-  return cudaFuncSetAttribute(ACM_FFN_KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  cudaError_t err = cudaFuncSetAttribute(ACM_FFN_KERNEL<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  if (err != cudaSuccess) return err;
+  return cudaFuncSetAttribute(ACM_FFN_KERNEL<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
 }
 
 cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
@@ -1449,7 +1459,12 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   cfg.attrs = attr;
   static const bool plain = [] { const char* e = std::getenv("ACM_FFN_PLAIN_LAUNCH"); return e && e[0] == '1'; }();
   cfg.numAttrs = (plain && !L.pdl) ? 0 : 1;
-  return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(ACM_FFN_KERNEL), args);
+#if ACM_FFN_MX
+  return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(ACM_FFN_KERNEL<false>), args);
+#else
+  return cudaLaunchKernelExC(&cfg, a.anc_flag && a.sel_flag ? reinterpret_cast<const void*>(ACM_FFN_KERNEL<true>)
+                                                            : reinterpret_cast<const void*>(ACM_FFN_KERNEL<false>), args);
+#endif
 }
 
 #if !ACM_FFN_MX
