@@ -503,8 +503,8 @@ def run_acm(args, world, rank, local):
         pipeline_gbs = acc.pop("_gbs")
         stage_us = {key: round(v, 2) for key, v in acc.items()}
         stage_us["note"] = ("in-kernel stamps, mean over %d layers: router = dependency release to selection start; "
-                            "select; route; ffn = first role start to last tile (it starts on the eligible set while "
-                            "the routes are made); whole = start of router to end of ffn" % n_samples)
+                            "select; route; ffn = first role start to last tile (it starts on the anchor experts while "
+                            "the selection runs); whole = start of router to end of ffn" % n_samples)
 
     if rank != 0:
         return
