@@ -776,3 +776,18 @@ def test_multi_block_batch_on_an_mxfp4_layer():
     ffn = oracle.expert_ffn(x, ref_idx, ref_w, w["gate_up_deq"], w["down_deq"])
     _ffn_check(out, ffn, "MXFP4 batch")
     ctx.close()
+
+
+@pytest.mark.parametrize("params_kw", [dict(fixed_budget=4), dict(fixed_budget=9), dict(use_anchors=0),
+                                       dict(use_anchors=0, fixed_budget=8), dict(demand=2, fixed_budget=30)])
+def test_fused_call_when_the_eligible_set_is_little_more_than_the_anchors(params_kw):
+    """The FFN kernel starts on the anchors before the eligible set is known: sets that hold nothing but the anchors
+    (a budget below k), one expert more, no anchors at all (the kernel then starts on the eligible set), and a large
+    fixed budget -- all rows against the oracle, on two layers back to back."""
+    cfg = wl.scaled(wl.CONFIGS[3], n_layers=2, inter=256)
+    ctx = _ctx(cfg, n_layers=2)
+    for layer in (0, 1):
+        st, _ = _verify_layer(cfg, layer, ctx, layer, params_kw=params_kw)
+        if params_kw.get("fixed_budget") == 4:
+            assert st["n_eligible_pruned"] == cfg.top_k == st["n_anchor"]
+    ctx.close()
