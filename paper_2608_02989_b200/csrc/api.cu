@@ -771,7 +771,8 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
                                 need_probs ? c->ws.probs : nullptr, need_probs ? c->ws.nat_idx : nullptr,
                                 need_probs ? c->ws.nat_mask : nullptr, k, c->ws.tile_done, c->pdl, s,
                                 c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr,
-                                anchors_first ? c->ws.anc_words : nullptr, static_cast<uint32_t>(early_epoch) & 0xffffu));
+                                // (published on every early call, used or not: the words never carry an old tag)
+                                early ? c->ws.anc_words : nullptr, static_cast<uint32_t>(early_epoch) & 0xffffu));
   // stages 2-3: one launch of a few small CTAs, which also fill the FFN kernel's routing inputs
   SelectArgs sa;
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
@@ -947,9 +948,19 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
   cudaStream_t s = static_cast<cudaStream_t>(stream);
 
   // stage 1 over all rows at once (it is per node); also clears `out` and the FFN kernel's routing inputs
+  // early start of the FFN kernel on the union of the blocks' eligible sets (it polls eight words per block)
+  const bool early = n_blocks <= kMaxEarlyBlocks && !c->split_phases && c->early_start;
+  int32_t early_epoch = 0;
+  if (early) {
+    early_epoch = ++c->epoch;
+    if ((early_epoch & 0xffff) == 0) early_epoch = ++c->epoch;
+    if (early_epoch <= 0) early_epoch = c->epoch = 1;
+  }
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, out,
                                 static_cast<size_t>(T) * d.hidden, c->ws.wtab, c->ffn_in_floats, c->ws.status,
-                                c->ws.probs, c->ws.nat_idx, c->ws.nat_mask, k, c->ws.tile_done, c->pdl, s, nullptr));
+                                c->ws.probs, c->ws.nat_idx, c->ws.nat_mask, k, c->ws.tile_done, c->pdl, s, nullptr,
+                                // (the anchor words follow every tag drawn, although this call does not use them)
+                                early ? c->ws.anc_words : nullptr, static_cast<uint32_t>(early_epoch) & 0xffffu));
   // stages 2-3: one CTA per block
   SelectArgs sa;
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
@@ -963,13 +974,7 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
   ra.logits = c->ws.logits; ra.mask = c->ws.mask; ra.idx_out = c->ws.idx; ra.w_out = c->ws.w;
   ra.weighting = d.weighting; ra.routed_scale = d.routed_scale;
   ra.act_mask = c->ws.act_mask; ra.wtab = c->ws.wtab;
-  // early start of the FFN kernel on the union of the blocks' eligible sets (it polls eight words per block)
-  const bool early = n_blocks <= kMaxEarlyBlocks && !c->split_phases && c->early_start;
-  int32_t early_epoch = 0;
   if (early) {
-    early_epoch = ++c->epoch;
-    if ((early_epoch & 0xffff) == 0) early_epoch = ++c->epoch;
-    if (early_epoch <= 0) early_epoch = c->epoch = 1;
     ra.sel_flag = c->ws.sel_words;
     ra.sel_epoch = early_epoch;
   }
