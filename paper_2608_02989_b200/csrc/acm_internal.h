@@ -52,7 +52,7 @@ struct Workspace {
   int32_t* tile_done;   // [64] router kernel: expert tiles finished per node tile (self-resetting)
   int32_t* ticket;      // [1] select/route kernel: finished CTAs (self-resetting)
   uint32_t* sel_words;  // [kMaxEarlyBlocks][8] the eligible masks as tagged 16-bit pieces (early start of the FFN kernel)
-  uint32_t* anc_words;  // [8] the anchor experts (the root's natural top-k) as tagged 16-bit pieces, published by the router kernel
+  uint32_t* anc_words;  // [kMaxEarlyBlocks][8] the anchor experts (each root's natural top-k) as tagged 16-bit pieces, published by the router kernel
 };
 
 struct SelectArgs {
@@ -76,7 +76,12 @@ struct BatchDesc {
   int n_blocks;
   int off[kMaxNodes + 1];
 };
-constexpr int kMaxEarlyBlocks = 8;   // blocks whose eligible sets the FFN kernel can poll for (8 tagged words each)
+constexpr int kMaxEarlyBlocks = 8;
+// The rows whose natural top-k the router kernel publishes as anchors (the blocks' roots; one for a single block).
+struct RootList {
+  int n;
+  int row[kMaxEarlyBlocks];
+};   // blocks whose eligible sets the FFN kernel can poll for (8 tagged words each)
 
 struct RouteArgs {
   const float* logits;
@@ -116,7 +121,7 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
                                  size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status,
                                  float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k, int32_t* tile_done,
                                  bool pdl, cudaStream_t s, long long* dbg = nullptr, uint32_t* anc_words = nullptr,
-                                 uint32_t anc_tag = 0);
+                                 uint32_t anc_tag = 0, const RootList* roots = nullptr);
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s);
 // select (unless mask_override) + route + the FFN kernel's routing inputs in ONE launch of ceil(T/4)

@@ -509,7 +509,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_tile = carve(sizeof(int32_t) * kMaxNodes);
   const size_t o_ticket = carve(16);
   const size_t o_selw = carve(32 * kMaxEarlyBlocks);
-  const size_t o_ancw = carve(32);
+  const size_t o_ancw = carve(32 * kMaxEarlyBlocks);
   const size_t o_natmask = carve(sizeof(uint32_t) * Tm * kMaskWords);
   const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
   if (cudaMalloc(&c->ws_base, off) != cudaSuccess) return fail(ACM_ERR_NOMEM);
@@ -956,11 +956,15 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
     if ((early_epoch & 0xffff) == 0) early_epoch = ++c->epoch;
     if (early_epoch <= 0) early_epoch = c->epoch = 1;
   }
+  // ... and on the union of the blocks' anchors (each block's first row is its root) while the selections run
+  const bool anchors_first = early && c->anchor_start && c->pdl && params->use_anchors != 0 && !L.mx;
+  RootList roots = {};
+  roots.n = early ? n_blocks : 0;
+  for (int b = 0; b < roots.n; ++b) roots.row[b] = bd.off[b];
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, out,
                                 static_cast<size_t>(T) * d.hidden, c->ws.wtab, c->ffn_in_floats, c->ws.status,
                                 c->ws.probs, c->ws.nat_idx, c->ws.nat_mask, k, c->ws.tile_done, c->pdl, s, nullptr,
-                                // (the anchor words follow every tag drawn, although this call does not use them)
-                                early ? c->ws.anc_words : nullptr, static_cast<uint32_t>(early_epoch) & 0xffffu));
+                                early ? c->ws.anc_words : nullptr, static_cast<uint32_t>(early_epoch) & 0xffffu, &roots));
   // stages 2-3: one CTA per block
   SelectArgs sa;
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
@@ -981,7 +985,7 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
   ACM_CUDA(launch_select_route_batch(c->ws.nat_mask, sa, ra, bd, E, k, c->pdl, s));
   c->launches += 2;
   // stage 4 once over all rows: an expert activated by several blocks is streamed once
-  st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, nullptr, true, early_epoch, nullptr, n_blocks);
+  st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, nullptr, true, early_epoch, nullptr, n_blocks, anchors_first);
   if (st != ACM_OK) return st;
 
   const size_t tk = static_cast<size_t>(T) * k;
@@ -1307,7 +1311,7 @@ acm_status acm_device_status(acm_ctx* c, acm_stream stream) {
     ACM_CUDA(cudaMemset(c->ws.frag_flag, 0, c->flag_bytes));
     ACM_CUDA(cudaMemset(c->ws.ticket, 0, 16));
     ACM_CUDA(cudaMemset(c->ws.sel_words, 0, 32 * kMaxEarlyBlocks));
-    ACM_CUDA(cudaMemset(c->ws.anc_words, 0, 32));
+    ACM_CUDA(cudaMemset(c->ws.anc_words, 0, 32 * kMaxEarlyBlocks));
     c->epoch = 0;
     ACM_CUDA(cudaMemset(c->ws.tile_done, 0, sizeof(int32_t) * kMaxNodes));
   }

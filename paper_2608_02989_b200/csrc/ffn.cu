@@ -154,11 +154,11 @@ struct __align__(8) Barriers {
   int abort_flag;
   float wd[kMaxNodes];          // combine weights of the expert being finalised
   int32_t entry[kMaxSlots];     // this launch's work list: make_entry(source, index) of every activated slot
-  int32_t expert[kMaxSlots];    // routed expert id of the slot (-1: shared expert)
+  int16_t expert[kMaxSlots];    // routed expert id of the slot (-1: shared expert)
   uint32_t sel_half[4 * kMaskWords];   // early start: the eligible mask in 16-bit pieces (second half: blocks 4..7 of a batch)
   Plan plan;                    // this launch's work plan
   unsigned long long plan_ready;     // anchors' pre-segment: the rest of the plan and of the work list is in place
-  uint32_t anc_half[2 * kMaskWords];   // early start on the anchors: their mask in 16-bit pieces
+  uint32_t anc_part[4 * kMaskWords];   // early start on the anchors: their mask in 16-bit pieces (by the two polling warps)
 };
 
 static_assert(sizeof(Barriers) <= 232448 - 1024 - kStages * kStageBytes - kOutStageBytes - kFragBytes - 2 * kHStageBytes,
@@ -573,19 +573,26 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   constexpr bool pre = kPre;
   if (threadIdx.x == 0) ACM_TRACE(29);
   if (pre) {
+    // eight words per block (a batch: the union of the blocks' anchors), one thread each, warps 2 and 3
     bool timed_out = false;
-    if (threadIdx.x >= 64 && threadIdx.x < 64 + 2 * kMaskWords) {
-      const int i = threadIdx.x - 64;
-      bool seen = false;
+    if (threadIdx.x >= 64 && threadIdx.x < 128) {
+      const int j = threadIdx.x - 64;
+      const bool mine = j < 2 * kMaskWords * p.sel_blocks;
+      bool seen = true;
       uint32_t v = 0;
-      const uint32_t tag = static_cast<uint32_t>(p.sel_epoch) & 0xffffu;
-      const unsigned long long t0 = global_timer();
-      do {
-        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.anc_flag + i) : "memory");
-        seen = (v >> 16) == tag;
-      } while (!seen && global_timer() - t0 < kTimeoutNs);
+      if (mine) {
+        const uint32_t tag = static_cast<uint32_t>(p.sel_epoch) & 0xffffu;
+        const unsigned long long t0 = global_timer();
+        do {
+          asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.anc_flag + j) : "memory");
+          seen = (v >> 16) == tag;
+        } while (!seen && global_timer() - t0 < kTimeoutNs);
+      }
       timed_out = !seen;
-      bars->anc_half[i] = seen ? (v & 0xffffu) : 0u;
+      uint32_t bits = (mine && seen) ? (v & 0xffffu) : 0u;
+      bits |= __shfl_xor_sync(0xffffffffu, bits, 8);
+      bits |= __shfl_xor_sync(0xffffffffu, bits, 16);
+      if (lane < 2 * kMaskWords) bars->anc_part[(j >> 5) * 2 * kMaskWords + lane] = bits;
     }
     __syncthreads();
     if (timed_out) {
@@ -649,7 +656,8 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   for (int wd = 0; wd < kMaskWords; ++wd) {
     uint32_t act;
     if (pre) {
-      act = bars->anc_half[2 * wd] | (bars->anc_half[2 * wd + 1] << 16);      // for now: the anchors only
+      act = (bars->anc_part[2 * wd] | bars->anc_part[2 * kMaskWords + 2 * wd]) |
+            ((bars->anc_part[2 * wd + 1] | bars->anc_part[2 * kMaskWords + 2 * wd + 1]) << 16);      // for now: the anchors only
     } else if (early) {
       act = bars->sel_half[2 * wd] | (bars->sel_half[2 * wd + 1] << 16);
       if (p.sel_blocks > 1) act |= bars->sel_half[2 * kMaskWords + 2 * wd] | (bars->sel_half[2 * kMaskWords + 2 * wd + 1] << 16);
@@ -904,18 +912,31 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       // While the others run the anchors' pre-segment: wait for the eligible set, give the other experts the
       // slots behind the pre-streamed ones (ascending id), append the shared experts, work out the rest of the
       // plan, and let everyone on.
-      uint32_t v = 0;
+      // eight words per block; lane l takes words l and l + 32 (blocks 0-3 and 4-7), the union goes to lanes 0..7
       bool seen = true;
-      if (lane < 2 * kMaskWords) {
+      uint32_t half = 0u;
+      {
         const uint32_t tag = static_cast<uint32_t>(p.sel_epoch) & 0xffffu;
-        const unsigned long long t0 = global_timer();
-        do {
-          asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.sel_flag + lane) : "memory");
-          seen = (v >> 16) == tag;
-        } while (!seen && global_timer() - t0 < kTimeoutNs);
+        const int n_words = 2 * kMaskWords * p.sel_blocks;
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+          const int j = lane + 32 * part;
+          if (j < n_words) {
+            uint32_t v = 0;
+            bool got = false;
+            const unsigned long long t0 = global_timer();
+            do {
+              asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.sel_flag + j) : "memory");
+              got = (v >> 16) == tag;
+            } while (!got && global_timer() - t0 < kTimeoutNs);
+            seen = seen && got;
+            half |= got ? (v & 0xffffu) : 0u;
+          }
+        }
+        half |= __shfl_xor_sync(0xffffffffu, half, 8);
+        half |= __shfl_xor_sync(0xffffffffu, half, 16);
       }
       const bool good = __all_sync(0xffffffffu, seen);
-      const uint32_t half = v & 0xffffu;
       uint32_t rest[kMaskWords];
       int n_rest = 0;
 #pragma unroll
@@ -1431,7 +1452,8 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   a.stats = L.stats; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
   a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag;
   a.sel_flag = L.sel_flag; a.sel_epoch = L.sel_epoch; a.sel_blocks = L.sel_blocks;
-  a.anc_flag = (ACM_FFN_MX || L.sel_blocks != 1 || L.li != 0 || L.resident || L.slot_of || L.phase_mask != 3) ? nullptr : L.anc_flag;
+  a.anc_flag = (ACM_FFN_MX || L.sel_blocks < 1 || L.sel_blocks > kMaxEarlyBlocks || L.li != 0 || L.resident || L.slot_of ||
+                L.phase_mask != 3) ? nullptr : L.anc_flag;
   a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask; a.trace = L.trace;
 #if ACM_FFN_MX
   if (!L.mx_gate_up || !L.mx_down || L.I % 128 != 0 || L.n_shared != 0) return cudaErrorInvalidValue;

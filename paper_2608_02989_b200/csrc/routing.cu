@@ -207,7 +207,7 @@ __global__ void __launch_bounds__(kRT * kRE * (32 / ElemTraits<Elem>::EPT))
 k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const float* __restrict__ bias,
                 float* logits, int T, int H, int E, int n_chunks, float* zero_buf,
                 size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status, float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k,
-                int32_t* tile_done, long long* dbg, uint32_t* anc_words, uint32_t anc_tag) {
+                int32_t* tile_done, long long* dbg, uint32_t* anc_words, uint32_t anc_tag, RootList roots) {
   constexpr int EPT = ElemTraits<Elem>::EPT;
   constexpr int Q = 32 / EPT;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -333,13 +333,19 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
           softmax_topk_row(logits + static_cast<size_t>(t) * E, probs ? probs + static_cast<size_t>(t) * E : nullptr,
                            nat_idx ? nat_idx + static_cast<size_t>(t) * k : nullptr,
                            nat_mask ? nat_mask + static_cast<size_t>(t) * kMaskWords : nullptr, E, k, lane);
-        if (t == 0 && anc_words && nat_mask) {
-          // The root's natural top-k are the anchors (Eq. 5), eligible whatever the selection decides: published
-          // at once, as eight words of 16 mask bits under the call's tag, for the FFN kernel to start on.
-          __syncwarp();
-          if (lane < 2 * kMaskWords) {
-            const uint32_t bits = (nat_mask[lane >> 1] >> (16 * (lane & 1))) & 0xffffu;
-            asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(anc_words + lane), "r"(bits | (anc_tag << 16)) : "memory");
+        if (anc_words && nat_mask && t < T) {
+          // A root's natural top-k are anchors (Eq. 5), eligible whatever the selection decides: published at
+          // once, as eight words of 16 mask bits under the call's tag, for the FFN kernel to start on (one group
+          // of eight words per block of a batch).
+          int which = -1;
+          for (int b = 0; b < roots.n; ++b) which = roots.row[b] == t ? b : which;
+          if (which >= 0) {
+            __syncwarp();
+            if (lane < 2 * kMaskWords) {
+              const uint32_t bits = (nat_mask[static_cast<size_t>(t) * kMaskWords + (lane >> 1)] >> (16 * (lane & 1))) & 0xffffu;
+              asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(anc_words + 2 * kMaskWords * which + lane),
+                           "r"(bits | (anc_tag << 16)) : "memory");
+            }
           }
         }
       }
@@ -866,8 +872,11 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
                                  float* logits, int T, int H, int E, float* zero_buf,
                                  size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status,
                                  float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k, int32_t* tile_done,
-                                 bool pdl, cudaStream_t s, long long* dbg, uint32_t* anc_words, uint32_t anc_tag) {
+                                 bool pdl, cudaStream_t s, long long* dbg, uint32_t* anc_words, uint32_t anc_tag,
+                                 const RootList* roots) {
   if (!probs && !nat_idx) tile_done = nullptr;
+  RootList rl = {};
+  if (roots) rl = *roots; else { rl.n = 1; rl.row[0] = 0; }
   cudaLaunchAttribute attr[1];
   set_pdl_attr(attr);
   cudaLaunchConfig_t cfg = {};
@@ -891,7 +900,7 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * 8); cfg.dynamicSmemBytes = smem;
     return cudaLaunchKernelEx(&cfg, kern, static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
                               logits, T, H, E, n_chunks, zero_buf, zero_floats, zero_buf2, zero_floats2, status, probs, nat_idx, nat_mask, k,
-                              tile_done, dbg, anc_words, anc_tag);
+                              tile_done, dbg, anc_words, anc_tag, rl);
   } else {
     auto kern = k_router_logits<__nv_bfloat16>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
@@ -899,7 +908,7 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * (32 / ElemTraits<__nv_bfloat16>::EPT)); cfg.dynamicSmemBytes = smem;
     return cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x),
                               static_cast<const __nv_bfloat16*>(w_router), bias, logits, T, H, E, n_chunks, zero_buf,
-                              zero_floats, zero_buf2, zero_floats2, status, probs, nat_idx, nat_mask, k, tile_done, dbg, anc_words, anc_tag);
+                              zero_floats, zero_buf2, zero_floats2, status, probs, nat_idx, nat_mask, k, tile_done, dbg, anc_words, anc_tag, rl);
   }
 }
 
