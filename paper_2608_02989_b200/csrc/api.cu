@@ -762,7 +762,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   // ... and earlier still on the anchors (Eq. 5 with the default anchor, the root): the router kernel publishes
   // the root's natural top-k as soon as that row is done, the FFN kernel streams their gate/up tiles while
   // the selection runs.  They are in every eligible set the selection can return without a residency.
-  const bool anchors_first = early && c->anchor_start && c->pdl && prm.use_anchors != 0 && !L.mx;
+  const bool anchors_first = early && c->anchor_start && c->pdl && prm.use_anchors != 0;
   // stage 1 (also clears the output the FFN accumulates into and the FFN kernel's routing inputs)
   const bool need_probs = eligible_mask_override == nullptr;
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
@@ -957,7 +957,7 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
     if (early_epoch <= 0) early_epoch = c->epoch = 1;
   }
   // ... and on the union of the blocks' anchors (each block's first row is its root) while the selections run
-  const bool anchors_first = early && c->anchor_start && c->pdl && params->use_anchors != 0 && !L.mx;
+  const bool anchors_first = early && c->anchor_start && c->pdl && params->use_anchors != 0;
   RootList roots = {};
   roots.n = early ? n_blocks : 0;
   for (int b = 0; b < roots.n; ++b) roots.row[b] = bd.off[b];

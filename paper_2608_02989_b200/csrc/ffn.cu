@@ -1141,8 +1141,6 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     // is the value times 2^-126 exactly, so one bf16 multiply by 2^(scale byte - 1) finishes the job.
     const int r = threadIdx.x - 256;
     const uint32_t my_lane = static_cast<uint32_t>(r & ~31) << 16;          // this warp's quarter of the lanes
-    unsigned total = 0;
-    for (int si = 0; si < bars->plan.n_seg; ++si) total += bars->plan.range[si].n_stages;
     bool ok = true;
     // the row's packed data of the stage at hand
     uint4 q[4];
@@ -1158,8 +1156,13 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       sc = *reinterpret_cast<const uint32_t*>(A + kMxCodeBytes + r * 4);
       return true;
     };
-    if (total > 0) ok = fetch(0);
-    for (unsigned it = 0; it < total && ok; ++it) {
+    // stage by stage through the segments (with the anchors' pre-segment the later ones arrive behind plan_ready)
+    unsigned it = 0, total = 0;
+    bool fetched = false;
+    for (int si = 0; ok && have_seg(si, true); ++si) {
+     total += bars->plan.range[si].n_stages;
+     if (!fetched && it < total) { ok = fetch(it); fetched = true; }
+     for (; it < total && ok; ++it) {
       const uint32_t s = it % kStages;
       const uint32_t a_tmem = tmem_base + my_lane + kAcc * kAccCols + s * kMxACols;
       tc_fence_after();
@@ -1189,7 +1192,8 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->full[s]));
-      if (it + 1 < total) ok = fetch(it + 1);
+      if (it + 1 < total) ok = fetch(it + 1); else fetched = false;
+     }
     }
 #endif
   } else {
@@ -1416,7 +1420,9 @@ __global__ void k_ffn_f32_down(const float* __restrict__ down, const float* __re
 
 #if ACM_FFN_MX
 cudaError_t ffn_mx_configure() {
-  return cudaFuncSetAttribute(ACM_FFN_KERNEL<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  cudaError_t err = cudaFuncSetAttribute(ACM_FFN_KERNEL<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  if (err != cudaSuccess) return err;
+  return cudaFuncSetAttribute(ACM_FFN_KERNEL<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
 }
 cudaError_t launch_ffn_mxfp4(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
                              const CUtensorMap& h_map, const CUtensorMap& hs_map, cudaStream_t s) {
@@ -1452,7 +1458,7 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   a.stats = L.stats; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
   a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag;
   a.sel_flag = L.sel_flag; a.sel_epoch = L.sel_epoch; a.sel_blocks = L.sel_blocks;
-  a.anc_flag = (ACM_FFN_MX || L.sel_blocks < 1 || L.sel_blocks > kMaxEarlyBlocks || L.li != 0 || L.resident || L.slot_of ||
+  a.anc_flag = (L.sel_blocks < 1 || L.sel_blocks > kMaxEarlyBlocks || L.li != 0 || L.resident || L.slot_of ||
                 L.phase_mask != 3) ? nullptr : L.anc_flag;
   a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask; a.trace = L.trace;
 #if ACM_FFN_MX
@@ -1481,12 +1487,8 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   cfg.attrs = attr;
   static const bool plain = [] { const char* e = std::getenv("ACM_FFN_PLAIN_LAUNCH"); return e && e[0] == '1'; }();
   cfg.numAttrs = (plain && !L.pdl) ? 0 : 1;
-#if ACM_FFN_MX
-  return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(ACM_FFN_KERNEL<false>), args);
-#else
   return cudaLaunchKernelExC(&cfg, a.anc_flag && a.sel_flag ? reinterpret_cast<const void*>(ACM_FFN_KERNEL<true>)
                                                             : reinterpret_cast<const void*>(ACM_FFN_KERNEL<false>), args);
-#endif
 }
 
 #if !ACM_FFN_MX
