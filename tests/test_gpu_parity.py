@@ -791,3 +791,66 @@ def test_fused_call_when_the_eligible_set_is_little_more_than_the_anchors(params
         if params_kw.get("fixed_budget") == 4:
             assert st["n_eligible_pruned"] == cfg.top_k == st["n_anchor"]
     ctx.close()
+
+
+def test_fused_call_on_random_shapes_and_selector_settings():
+    """A hundred seeded random layers -- hidden, experts, top-k, intermediate size, shared experts, nodes, weighting rule,
+    selector mode, budget, anchors on or off -- twice each through the fused call (the second call runs on what the
+    first left behind), everything against the oracle."""
+    rng = np.random.default_rng(2026)
+    for case in range(100):
+        H = int(rng.choice([256, 512, 1024]))
+        E = int(rng.integers(8, 129))
+        k = int(rng.integers(1, min(8, E) + 1))
+        I = int(rng.choice([64, 128, 192, 320]))
+        ns = int(rng.choice([0, 0, 1, 2]))
+        T = int(rng.integers(1, 65))
+        D = int(min(rng.integers(1, 9), max(T - 1, 1)))
+        cfg = wl.scaled(wl.CONFIGS[3], hidden=H, n_experts=E, top_k=k, inter=I, n_shared=ns, n_nodes=T, max_depth=D,
+                        n_layers=1, weighting=int(rng.integers(0, 3)), zipf_bias=bool(rng.integers(0, 2)))
+        kw = {}
+        if rng.random() < 0.4:
+            kw["fixed_budget"] = int(rng.integers(1, E + 1))
+        if rng.random() < 0.25:
+            kw["use_anchors"] = 0
+        if rng.random() < 0.3:
+            kw["demand"] = int(rng.integers(0, 3))
+        ctx = _ctx(cfg)
+        for rep in range(2):
+            _verify_layer(cfg, 0, ctx, 0, params_kw=kw)
+        ctx.close()
+
+
+def test_batch_call_on_random_block_partitions():
+    """Forty seeded random batches: 1 to 10 blocks of random sizes over random layers, against every block verified
+    alone by the oracle."""
+    rng = np.random.default_rng(77)
+    for case in range(40):
+        E = int(rng.integers(16, 129))
+        k = int(rng.integers(1, 9))
+        T = int(rng.integers(1, 65))
+        nb = int(rng.integers(1, min(T, 10) + 1))
+        cuts = sorted(rng.choice(np.arange(1, T), size=nb - 1, replace=False).tolist()) if nb > 1 else []
+        offsets = [0] + cuts + [T]
+        cfg = wl.scaled(wl.CONFIGS[3], hidden=int(rng.choice([256, 512])), n_experts=E, top_k=k, inter=int(rng.choice([64, 128, 256])),
+                        n_shared=int(rng.choice([0, 0, 1])), n_nodes=T, max_depth=4, n_layers=1, weighting=int(rng.integers(0, 3)))
+        kw = {"fixed_budget": int(rng.integers(1, E + 1))} if rng.random() < 0.3 else {}
+        w = wl.layer_weights(cfg, 0, DEV)
+        x = wl.hidden_states(cfg, 0, DEV)
+        depths = torch.cat([torch.sort(torch.cat([torch.zeros(1, dtype=torch.int32),
+                                                  torch.tensor(rng.integers(1, 5, size=offsets[b + 1] - offsets[b] - 1), dtype=torch.int32)])).values
+                            for b in range(nb)])
+        alpha_ref, refs = _batch_reference(cfg, w, x, offsets, depths, kw)
+        ctx = _ctx(cfg)
+        _set_weights(ctx, w, 0)
+        out, idx, wt, mask, act, stats = ctx.moe_verify_batch(0, x, offsets, torch.tensor(alpha_ref, device=DEV),
+                                                              acm.SelectParams(**kw), want=True)
+        assert ctx.device_status() == acm.OK
+        for b, ref in enumerate(refs):
+            np.testing.assert_array_equal(_u32(mask[b]), ref["mask"])
+            np.testing.assert_array_equal(idx[offsets[b]:offsets[b + 1]].cpu().numpy(), ref["idx"])
+        ref_idx = np.concatenate([r["idx"] for r in refs])
+        ref_w = np.concatenate([r["w"] for r in refs])
+        ffn = oracle.expert_ffn(x, ref_idx, ref_w, w["gate_up"], w["down"], w["shared_gate_up"], w["shared_down"])
+        _ffn_check(out, ffn, f"random batch {case}")
+        ctx.close()
