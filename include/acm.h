@@ -29,6 +29,11 @@
  *     workspace (allocated in acm_create with cudaMalloc on the current device).
  *   - One context serves one stream at a time: calls on the same context that overlap on
  *     the GPU race on its workspace.
+ *   - The fused calls expect the GPU to themselves (see acm_set_overlap): by default the expert-FFN kernel is
+ *     started ahead of stream order, one CTA per SM, and its CTAs wait on one another.  If other work of
+ *     the process (another stream, another context) can hold SMs while a fused call runs, select
+ *     ACM_OVERLAP_NONE; otherwise a CTA that finds no SM makes the others wait until their limit runs out
+ *     (ACM_ERR_TIMEOUT from acm_device_status, output of that call invalid, context still usable).
  *   - Limits (else ACM_ERR_UNSUPPORTED): n_experts <= 128, top_k <= 8, T <= 64;
  *     bf16: hidden % 128 == 0, inter % 64 == 0; f32: hidden % 32 == 0.
  *
@@ -65,7 +70,8 @@ typedef enum {
 
 typedef enum { ACM_F32 = 0, ACM_BF16 = 1 } acm_dtype;
 
-/* "preserves the target's native post-top-k weighting" (Section 3.1, below Eq. 2) */
+/* How the k selected experts' outputs are weighted: restricted routing keeps whatever rule the target model
+ * applies after its own top-k (Section 3.1, below Eq. 2), so the rule is a property of the model. */
 typedef enum {
   ACM_W_RENORM_TOPK = 0,     /* w = r_e / sum of r over the k selected experts          */
   ACM_W_SOFTMAX_RAW = 1,     /* w = r_e of the unmasked softmax (zero-probability mask) */
@@ -247,8 +253,8 @@ acm_status acm_host_synchronize(acm_ctx* ctx);
 acm_status acm_set_resident(acm_ctx* ctx, int layer, const uint32_t* resident_mask,
                             const void* host_gate_up, const void* host_down);
 
-/* Offload variant with the paper's per-layer expert pool (Section 3.4: "an X-slot expert pool in GPU
- * memory", LRU): the layer's routed experts live in `n_slots` slots of the caller's device tensors
+/* Offload variant with the per-layer expert pool of Section 3.4 (a fixed number of expert slots in GPU memory,
+ * replaced least-recently-used first): the layer's routed experts live in `n_slots` slots of the caller's device tensors
  * pool_gate_up [n_slots,2I,H] / pool_down [n_slots,H,I] (128-byte aligned; the tensors given to
  * acm_set_layer_weights may then be NULL), the full weights in PINNED host tensors [E,...].  The first
  * n_initial slots are filled with initial_experts (host ids; copied synchronously).  From then on, with
@@ -334,6 +340,52 @@ acm_status acm_expert_ffn_f32_noalloc(const float* x, int T, int hidden, int int
                                       int top_k, const int32_t* idx, const float* w,
                                       const float* w_gate_up, const float* w_down, float* out,
                                       acm_stream stream);
+
+/* How far the kernels of a fused call (acm_moe_verify, acm_moe_verify_batch, acm_moe_verify_host) overlap.
+ * The stages of Section 3.1-3.4 form a chain, and the expert FFN needs only part of its result to start:
+ *   ACM_OVERLAP_NONE       plain stream order.  The FFN kernel is a cooperative launch, so the driver itself
+ *                          checks that all its CTAs can be resident together.  The mode to use when anything
+ *                          else may run on the GPU at the same time.
+ *   ACM_OVERLAP_DEPENDENT  each kernel is launched as a programmatic dependent of the one before: it is
+ *                          resident and set up while its predecessor drains, then waits for it.
+ *   ACM_OVERLAP_ELIGIBLE   ... and the FFN kernel starts streaming as soon as the eligible set S' (Eq. 6, 7)
+ *                          is published, before the routes (Eq. 2) are written.
+ *   ACM_OVERLAP_ANCHORS    ... and before that on the anchor experts (Eq. 5), which are in every eligible
+ *                          set, while the selection still runs.  The default.
+ * From ACM_OVERLAP_DEPENDENT on, the FFN kernel's CTAs (one per SM, they exchange partial sums) are not
+ * checked for co-residency by the driver: the GPU must be otherwise idle while a fused call runs.
+ * Takes effect from the next call; results do not depend on the level. */
+typedef enum {
+  ACM_OVERLAP_NONE = 0,
+  ACM_OVERLAP_DEPENDENT = 1,
+  ACM_OVERLAP_ELIGIBLE = 2,
+  ACM_OVERLAP_ANCHORS = 3
+} acm_overlap;
+acm_status acm_set_overlap(acm_ctx* ctx, int level);
+
+/* Every device-side wait (on a barrier, a counter another CTA raises, a word an earlier kernel publishes) is
+ * bounded: after `nanoseconds` without progress the waiting CTA raises ACM_ERR_TIMEOUT in the status word,
+ * lets its copies in flight land, frees its tensor memory and returns; the launch's output is then invalid
+ * and acm_device_status re-arms the workspace.  Default 1 s; 1 us .. 60 s (else ACM_ERR_INVALID).  Healthy
+ * waits last microseconds, so a few milliseconds are safe on an idle GPU. */
+acm_status acm_set_wait_limit(acm_ctx* ctx, uint64_t nanoseconds);
+
+/* After ACM_ERR_TIMEOUT: which wait of the LAST expert-FFN launch gave up first in each of its CTAs.
+ * Synchronises the device.  site_out [capacity] (host): 0 = that CTA saw no wait run out, -1 = that CTA never
+ * started (it found no SM), else a wait-site number (1, 2: words published by the router / selection kernel;
+ * 3-5: the CTA's own pipeline; 6-10: data from other CTAs; 11-16: hand-overs inside the CTA; 17: the rest of
+ * the plan; 18: a packed MXFP4 stage).  *n_ctas = CTAs of that launch.  Call it before acm_device_status
+ * clears the state, or after: the words are kept until the next launch. */
+acm_status acm_wait_report(acm_ctx* ctx, int32_t* site_out /*host*/, int capacity, int32_t* n_ctas /*host*/);
+
+/* Failure injection for tests of the error path above (made on the host; nothing faults): launches the
+ * expert-FFN kernel of a bf16 layer in its early-start form, waiting for an eligible set (Eq. 6) under a
+ * sequence tag that no selection kernel is ever given.  Every CTA's first wait therefore runs out after the
+ * wait limit: the kernel returns, acm_device_status reports ACM_ERR_TIMEOUT and re-arms the workspace, and
+ * the next call on the context must be correct again.  out [T,hidden] is zeroed.  Set a short limit first
+ * (acm_set_wait_limit): the call keeps the GPU busy for that long. */
+acm_status acm_inject_unpublished_wait(acm_ctx* ctx, int layer, const void* x, int T, float* out,
+                                       acm_stream stream);
 
 /* Synchronises `stream` and returns the sticky device-side status (ACM_OK if none), then clears it. */
 acm_status acm_device_status(acm_ctx* ctx, acm_stream stream);

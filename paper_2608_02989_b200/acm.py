@@ -18,6 +18,7 @@ LIB_PATH = _PKG / "libacm.so"
 OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM, ERR_NONFINITE = range(7)
 F32, BF16 = 0, 1
 W_RENORM_TOPK, W_SOFTMAX_RAW, W_SOFTMAX_MASKED = 0, 1, 2
+OVERLAP_NONE, OVERLAP_DEPENDENT, OVERLAP_ELIGIBLE, OVERLAP_ANCHORS = 0, 1, 2, 3
 DEMAND_TOPK_MASS, DEMAND_FULL_MASS, DEMAND_VOTES = 0, 1, 2
 
 EXPORTS = [
@@ -26,6 +27,7 @@ EXPORTS = [
     "acm_expert_ffn", "acm_moe_verify", "acm_moe_verify_batch", "acm_moe_verify_host", "acm_host_synchronize", "acm_set_resident",
     "acm_set_slot_pool", "acm_pool_stats", "acm_pool_plan",
     "acm_h2d_bytes", "acm_ffn_timing", "acm_ffn_time_ms", "acm_stage_timing", "acm_stage_times", "acm_launch_count", "acm_device_status", "acm_status_string",
+    "acm_set_overlap", "acm_set_wait_limit", "acm_wait_report", "acm_inject_unpublished_wait",
     "acm_expert_ffn_f32_noalloc",
 ]
 NOALLOC_MAX_FLOATS = 1 << 20
@@ -108,6 +110,10 @@ def load_library():
     lib.acm_ffn_time_ms.argtypes = [c_void_p, POINTER(c_float), POINTER(c_int32)]
     lib.acm_launch_count.argtypes = [c_void_p, POINTER(c_uint64)]
     lib.acm_device_status.argtypes = [c_void_p, c_void_p]
+    lib.acm_set_overlap.argtypes = [c_void_p, c_int]
+    lib.acm_set_wait_limit.argtypes = [c_void_p, c_uint64]
+    lib.acm_wait_report.argtypes = [c_void_p, c_void_p, c_int, POINTER(c_int32)]
+    lib.acm_inject_unpublished_wait.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p]
     lib.acm_default_select_params.argtypes = [POINTER(SelectParams)]
     lib.acm_expert_ffn_f32_noalloc.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p,
                                                c_void_p, c_void_p, c_void_p, c_void_p]
@@ -432,6 +438,29 @@ class Context:
         v = c_uint64(0)
         _check(self.lib.acm_launch_count(self.handle, byref(v)), "acm_launch_count")
         return v.value
+
+    def set_overlap(self, level):
+        """acm_set_overlap: OVERLAP_NONE (safe on a shared GPU) .. OVERLAP_ANCHORS (default)."""
+        _check(self.lib.acm_set_overlap(self.handle, int(level)), "acm_set_overlap")
+
+    def set_wait_limit(self, nanoseconds):
+        _check(self.lib.acm_set_wait_limit(self.handle, int(nanoseconds)), "acm_set_wait_limit")
+
+    def wait_report(self) -> list:
+        """Per CTA of the last expert-FFN launch: 0 = no wait ran out, -1 = never started, else the wait site."""
+        buf = (c_int32 * 256)()
+        n = c_int32(0)
+        _check(self.lib.acm_wait_report(self.handle, buf, 256, byref(n)), "acm_wait_report")
+        return [int(buf[i]) for i in range(min(n.value, 256))]
+
+    def inject_unpublished_wait(self, layer, x, out=None, stream=None):
+        """acm_inject_unpublished_wait: the FFN kernel waits for an eligible set nobody publishes (error-path tests)."""
+        T = x.shape[0]
+        if out is None:
+            out = torch.empty(T, self.H, dtype=torch.float32, device=x.device)
+        _check(self.lib.acm_inject_unpublished_wait(self.handle, layer, _p(x), T, _p(out), _stream(stream)),
+               "acm_inject_unpublished_wait")
+        return out
 
     def device_status(self, stream=None) -> int:
         return int(self.lib.acm_device_status(self.handle, _stream(stream)))

@@ -28,8 +28,7 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
     if not force and LIB.exists() and LIB.stat().st_mtime >= sources_mtime():
         return LIB
     tmp = LIB.with_suffix(f".{os.getpid()}.tmp.so")
-    extra = os.environ.get("ACM_NVCC_EXTRA", "").split()      # e.g. -DACM_FFN_STAGES=4 for experiments
-    cmd = [_nvcc(), *NVCC_FLAGS, *extra, *[str(CSRC / s) for s in SOURCES], "-o", str(tmp)]
+    cmd = [_nvcc(), *NVCC_FLAGS, *[str(CSRC / s) for s in SOURCES], "-o", str(tmp)]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)

@@ -68,7 +68,6 @@ struct SelectArgs {
   int32_t* count_out;
   float* demand_out;             // may be null
   acm_block_stats* stats_out;    // may be null
-  long long* dbg;                // optional time stamps in ns (debugging aid)
 };
 
 // A batch of verification blocks stacked along the node axis: block b owns rows off[b] .. off[b+1]-1.
@@ -101,7 +100,7 @@ struct RouteArgs {
                                  // [1 + kMaxExperts ..] = the activated mask (4 words)
   uint32_t* sel_flag;            // non-null: [8] words, the eligible mask in 16-bit pieces tagged with sel_epoch
   int32_t sel_epoch;
-  long long* dbg;                // optional time stamps in ns of the select/route kernel's stages (debugging aid)
+  long long* dbg;                // optional time stamps in ns (acm_stage_timing): [0] start, [2] selection done, [3] routes done
 };
 
 // Programmatic dependent launch: a kernel launched with `pdl` may start while the kernel before it
@@ -170,11 +169,13 @@ struct FfnLaunch {
   float* out;                // [T,H], accumulated into (zeroed by the caller)
   int32_t* status;
   int grid;
-  int phase_mask;            // 1 = gate/up, 2 = down, 3 = both in one launch
   bool pdl;                  // launch with programmatic stream serialization
+  unsigned long long wait_limit_ns = 1000000000ull;   // the longest any single device-side wait may last
+  int32_t* wait_diag = nullptr;   // [grid] per-CTA words: (launch number << 8) | the wait that gave up first (0: none)
+  int32_t launch_tag = 0;         // launch number << 8
   const void* mx_gate_up = nullptr;   // MXFP4 layers (launch_ffn_mxfp4): the tiled code + scale tensors
   const void* mx_down = nullptr;
-  unsigned long long* trace; // optional [grid][32] device timestamps (debugging aid) or null
+  unsigned long long* trace; // optional [grid][32] device time stamps (acm_stage_timing) or null
 };
 cudaError_t ffn_configure();   // one-time function attributes
 size_t ffn_smem_bytes();
@@ -186,6 +187,6 @@ cudaError_t launch_ffn_mxfp4(const FfnLaunch& p, const FfnMaps& maps, const CUte
 cudaError_t launch_ffn_f32(const float* x, const float* gate_up, const float* down,
                            const float* shared_gate_up, const float* shared_down, int n_shared,
                            const int32_t* idx, const float* w, float* hbuf, float* out, int T, int H,
-                           int I, int k, cudaStream_t s);
+                           int I, int E, int k, cudaStream_t s);
 
 }  // namespace acm

@@ -146,16 +146,21 @@ struct acm_ctx {
   bool timing = false;
   int timing_period = 1;        // every n-th FFN launch is bracketed by events
   long long timing_seen = 0;
-  bool pdl = true;              // programmatic dependent launches between the kernels of the hot path
-  bool early_start = true;      // the FFN kernel starts on the eligible set, before the routes are final
+  // how far the kernels of a fused call overlap (acm_set_overlap)
+  int overlap = ACM_OVERLAP_ANCHORS;
+  bool pdl = true;              // >= DEPENDENT: programmatic dependent launches between the kernels of the hot path
+  bool early_start = true;      // >= ELIGIBLE: the FFN kernel starts on the eligible set, before the routes are final
+  bool anchor_start = true;     // ANCHORS: ... and before that on the anchors, while the selection runs
   std::vector<cudaEvent_t> ev_pool;
   size_t ev_used = 0;
   uint64_t launches = 0;
-  bool split_phases = false;             // ACM_FFN_SPLIT_PHASES=1 in the environment
-  unsigned long long* trace = nullptr;   // ACM_FFN_TRACE=1|2: per-CTA timestamps of the last FFN launch
-  bool anchor_start = true;              // ACM_NO_ANCHOR_START=1: the FFN kernel starts on the eligible set only
+  unsigned long long* trace = nullptr;   // acm_stage_timing: per-CTA time stamps of the last FFN launch + the routing kernels' stamps
   bool mx_configured = false;
-  bool trace_light = false;              // =2: leave the launch sequence as it is (stale slots are not cleared)
+  // bounded device-side waits (acm_set_wait_limit, acm_wait_report)
+  unsigned long long wait_limit_ns = 1000000000ull;
+  int32_t* wait_diag = nullptr;          // [sm_count] per-CTA words of the FFN kernel
+  int32_t ffn_launch_no = 0;             // numbers the FFN launches (24 bits are kept in the words)
+  int last_ffn_grid = 0;
 };
 
 namespace {
@@ -333,11 +338,13 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   }
   p.out = out; p.status = c->ws.status;
   p.grid = c->sm_count;
-  p.phase_mask = 3;
   p.trace = c->trace;
   p.pdl = false;
-  if (c->trace && !c->trace_light)
-    ACM_CUDA(cudaMemsetAsync(c->trace, 0, sizeof(unsigned long long) * 32 * c->sm_count, s));
+  p.wait_limit_ns = c->wait_limit_ns;
+  p.wait_diag = c->wait_diag;
+  c->ffn_launch_no = (c->ffn_launch_no + 1) & 0x7fffff;
+  if (c->ffn_launch_no == 0) c->ffn_launch_no = 1;
+  p.launch_tag = c->ffn_launch_no << 8;
   cudaEvent_t e0 = nullptr, e1 = nullptr;
   if (c->timing && (c->timing_seen++ % c->timing_period) == 0 && c->ev_used + 2 <= c->ev_pool.size()) {
     e0 = c->ev_pool[c->ev_used];
@@ -345,15 +352,8 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
     c->ev_used += 2;
     ACM_CUDA(cudaEventRecord(e0, s));
   }
-  if (c->split_phases && !L.mx) {
-    // debugging aid: the two GEMM phases as separate launches (kernel boundary instead of flags)
-    p.phase_mask = 1;
-    ACM_CUDA(launch_ffn_bf16(p, maps, x_map, c->h_map[li], c->h_store_map[li], s));
-    p.phase_mask = 2;
-    c->launches += 1;
-  }
   // dependent launch only straight after the select/route kernel (no event, memset or copy between)
-  p.pdl = pdl_ok && c->pdl && !e0 && (!c->trace || c->trace_light) && !c->split_phases;
+  p.pdl = pdl_ok && c->pdl && !e0;
   // the anchors' pre-segment pays only when this launch overlaps the selection; a launch ordered after it (one
   // bracketed by events) has the whole set at hand and takes the balanced plan
   if (anchors_first && p.pdl && early_epoch != 0) p.anc_flag = c->ws.anc_words;
@@ -362,6 +362,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   // split changes -- and one late CTA delays every CTA that exchanges fragments with it.  Leave them out.
   const int routing_ctas = n_blocks > 0 ? n_blocks : route_ctas(T);   // a batch: one CTA per block
   if (pdl_ok && c->sm_count > 2 * routing_ctas) p.grid = c->sm_count - routing_ctas;
+  c->last_ffn_grid = p.grid;
   if (L.mx) {
     p.mx_gate_up = L.has_pool ? L.pool_gate_up : L.mx_gate_up;      // a pool: slot s of the pool tensors
     p.mx_down = L.has_pool ? L.pool_down : L.mx_down;
@@ -422,16 +423,6 @@ void acm_default_select_params(acm_select_params* p) {
   p->max_remove = kMaxExperts;
 }
 
-// Debugging aid (not part of the public header): copies the per-CTA timestamps of the last FFN
-// launch to `host_out` ([sm_count][32] uint64).  Needs ACM_FFN_TRACE=1 at context creation.
-acm_status acm_debug_ffn_trace(acm_ctx* c, unsigned long long* host_out, int* n_ctas) {
-  if (!c || !host_out || !n_ctas || !c->trace) return ACM_ERR_INVALID;
-  ACM_CUDA(cudaDeviceSynchronize());
-  ACM_CUDA(cudaMemcpy(host_out, c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 32), cudaMemcpyDeviceToHost));
-  *n_ctas = c->sm_count;
-  return ACM_OK;
-}
-
 const char* acm_status_string(acm_status s) {
   switch (s) {
     case ACM_OK: return "ok";
@@ -454,17 +445,6 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   if (!c) return ACM_ERR_NOMEM;
   c->desc = *desc;
   c->layers.resize(desc->n_layers);
-  const char* split = std::getenv("ACM_FFN_SPLIT_PHASES");
-  c->split_phases = split && split[0] == '1';
-  const char* no_pdl = std::getenv("ACM_NO_PDL");
-  c->pdl = !(no_pdl && no_pdl[0] == '1');
-  const char* no_anc = std::getenv("ACM_NO_ANCHOR_START");
-  c->anchor_start = !(no_anc && no_anc[0] == '1');
-  const char* no_early = std::getenv("ACM_NO_EARLY_START");
-  c->early_start = !(no_early && no_early[0] == '1');
-  const char* trace = std::getenv("ACM_FFN_TRACE");
-  const bool want_trace = trace && (trace[0] == '1' || trace[0] == '2');
-  c->trace_light = trace && trace[0] == '2';
   auto fail = [&](acm_status s) {
     acm_destroy(c);
     return s;
@@ -512,6 +492,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_ancw = carve(32 * kMaxEarlyBlocks);
   const size_t o_natmask = carve(sizeof(uint32_t) * Tm * kMaskWords);
   const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
+  const size_t o_diag = carve(sizeof(int32_t) * c->sm_count);
   if (cudaMalloc(&c->ws_base, off) != cudaSuccess) return fail(ACM_ERR_NOMEM);
   if (cudaMemset(c->ws_base, 0, off) != cudaSuccess) return fail(ACM_ERR_CUDA);
   char* b = static_cast<char*>(c->ws_base);
@@ -542,8 +523,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.anc_words = reinterpret_cast<uint32_t*>(b + o_ancw);
   c->ws.nat_mask = reinterpret_cast<uint32_t*>(b + o_natmask);
   c->resident_dev = reinterpret_cast<uint32_t*>(b + o_res);
-  if (want_trace && cudaMalloc(&c->trace, sizeof(unsigned long long) * (32 * c->sm_count + 32)) != cudaSuccess)
-    return fail(ACM_ERR_NOMEM);
+  c->wait_diag = reinterpret_cast<int32_t*>(b + o_diag);
   *out = c;
   return ACM_OK;
 }
@@ -683,7 +663,7 @@ acm_status acm_select_eligible(acm_ctx* c, const float* probs, const int32_t* na
   a.probs = probs; a.nat_idx = nat_idx; a.alpha = alpha; a.anchor_nodes = anchor_nodes;
   a.n_anchor_nodes = n_anchor_nodes; a.resident = params->residency ? resident_mask : nullptr; a.prm = *params;
   a.mask_out = eligible_mask; a.unpruned_out = unpruned_mask; a.count_out = eligible_count;
-  a.demand_out = demand; a.stats_out = stats; a.dbg = nullptr;
+  a.demand_out = demand; a.stats_out = stats;
   ACM_CUDA(launch_select(a, T, c->desc.n_experts, c->desc.top_k, static_cast<cudaStream_t>(stream)));
   c->launches += 1;
   return ACM_OK;
@@ -715,7 +695,7 @@ acm_status acm_expert_ffn(acm_ctx* c, int layer, const void* x, int T, const int
     ACM_CUDA(launch_ffn_f32(static_cast<const float*>(x), static_cast<const float*>(L.gate_up),
                             static_cast<const float*>(L.down), static_cast<const float*>(L.shared_gate_up),
                             static_cast<const float*>(L.shared_down), d.n_shared, idx, w,
-                            static_cast<float*>(c->ws.hbuf), out, T, d.hidden, d.inter, d.top_k, s));
+                            static_cast<float*>(c->ws.hbuf), out, T, d.hidden, d.inter, d.n_experts, d.top_k, s));
     c->launches += 2;
     return ACM_OK;
   }
@@ -752,7 +732,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
 
   // Early start of the FFN kernel on the eligible set: when a selection runs (the eligible experts are
   // then nearly always all activated; with an override mask they need not be) and every expert is resident.
-  const bool early = !f32 && !L.has_resident && !eligible_mask_override && !c->split_phases && c->early_start;
+  const bool early = !f32 && !L.has_resident && !eligible_mask_override && c->early_start;
   int32_t early_epoch = 0;
   if (early) {
     early_epoch = ++c->epoch;            // its low 16 bits tag the published words; 0 is never a valid tag
@@ -762,7 +742,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   // ... and earlier still on the anchors (Eq. 5 with the default anchor, the root): the router kernel publishes
   // the root's natural top-k as soon as that row is done, the FFN kernel streams their gate/up tiles while
   // the selection runs.  They are in every eligible set the selection can return without a residency.
-  const bool anchors_first = early && c->anchor_start && c->pdl && prm.use_anchors != 0;
+  const bool anchors_first = early && c->anchor_start && prm.use_anchors != 0;
   // stage 1 (also clears the output the FFN accumulates into and the FFN kernel's routing inputs)
   const bool need_probs = eligible_mask_override == nullptr;
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
@@ -781,7 +761,6 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   bool stats_direct = false;
   acm_block_stats* stats_dev = stats_target(c, stats, &stats_direct);
   sa.demand_out = c->ws.demand; sa.stats_out = stats_dev;
-  sa.dbg = c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr;
   RouteArgs ra = {};
   ra.logits = c->ws.logits; ra.mask = c->ws.mask; ra.idx_out = c->ws.idx; ra.w_out = c->ws.w;
   ra.weighting = d.weighting; ra.routed_scale = d.routed_scale;
@@ -802,7 +781,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
     ACM_CUDA(launch_ffn_f32(static_cast<const float*>(x), static_cast<const float*>(L.gate_up),
                             static_cast<const float*>(L.down), static_cast<const float*>(L.shared_gate_up),
                             static_cast<const float*>(L.shared_down), d.n_shared, c->ws.idx, c->ws.w,
-                            static_cast<float*>(c->ws.hbuf), out, T, d.hidden, d.inter, k, s));
+                            static_cast<float*>(c->ws.hbuf), out, T, d.hidden, d.inter, E, k, s));
     c->launches += 2;
   } else if (!L.has_resident) {
     st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, stats_dev, true, early_epoch, nullptr, 0, anchors_first);
@@ -949,7 +928,7 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
 
   // stage 1 over all rows at once (it is per node); also clears `out` and the FFN kernel's routing inputs
   // early start of the FFN kernel on the union of the blocks' eligible sets (it polls eight words per block)
-  const bool early = n_blocks <= kMaxEarlyBlocks && !c->split_phases && c->early_start;
+  const bool early = n_blocks <= kMaxEarlyBlocks && c->early_start;
   int32_t early_epoch = 0;
   if (early) {
     early_epoch = ++c->epoch;
@@ -957,7 +936,7 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
     if (early_epoch <= 0) early_epoch = c->epoch = 1;
   }
   // ... and on the union of the blocks' anchors (each block's first row is its root) while the selections run
-  const bool anchors_first = early && c->anchor_start && c->pdl && params->use_anchors != 0;
+  const bool anchors_first = early && c->anchor_start && params->use_anchors != 0;
   RootList roots = {};
   roots.n = early ? n_blocks : 0;
   for (int b = 0; b < roots.n; ++b) roots.row[b] = bd.off[b];
@@ -973,7 +952,6 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
   bool stats_direct = false;
   acm_block_stats* stats_dev = stats_target(c, stats, &stats_direct);
   sa.demand_out = c->ws.demand; sa.stats_out = stats_dev;
-  sa.dbg = nullptr;
   RouteArgs ra = {};
   ra.logits = c->ws.logits; ra.mask = c->ws.mask; ra.idx_out = c->ws.idx; ra.w_out = c->ws.w;
   ra.weighting = d.weighting; ra.routed_scale = d.routed_scale;
@@ -1259,12 +1237,10 @@ acm_status acm_stage_timing(acm_ctx* c, int enable) {
       const size_t bytes = sizeof(unsigned long long) * (32 * c->sm_count + 32);
       if (cudaMalloc(&c->trace, bytes) != cudaSuccess) return ACM_ERR_NOMEM;
       ACM_CUDA(cudaMemset(c->trace, 0, bytes));
-      c->trace_light = true;       // stamps only: the launch sequence stays exactly as it is
     }
   } else if (c->trace) {
     ACM_CUDA(cudaFree(c->trace));
     c->trace = nullptr;
-    c->trace_light = false;
   }
   return ACM_OK;
 }
@@ -1297,6 +1273,49 @@ acm_status acm_launch_count(acm_ctx* c, uint64_t* launches_out) {
   if (!c || !launches_out) return ACM_ERR_INVALID;
   *launches_out = c->launches;
   return ACM_OK;
+}
+
+acm_status acm_set_overlap(acm_ctx* c, int level) {
+  if (!c || level < ACM_OVERLAP_NONE || level > ACM_OVERLAP_ANCHORS) return ACM_ERR_INVALID;
+  c->overlap = level;
+  c->pdl = level >= ACM_OVERLAP_DEPENDENT;
+  c->early_start = level >= ACM_OVERLAP_ELIGIBLE;
+  c->anchor_start = level >= ACM_OVERLAP_ANCHORS;
+  return ACM_OK;
+}
+
+acm_status acm_set_wait_limit(acm_ctx* c, uint64_t nanoseconds) {
+  if (!c || nanoseconds < 1000ull || nanoseconds > 60ull * 1000000000ull) return ACM_ERR_INVALID;
+  c->wait_limit_ns = nanoseconds;
+  return ACM_OK;
+}
+
+acm_status acm_wait_report(acm_ctx* c, int32_t* site_out, int capacity, int32_t* n_ctas) {
+  if (!c || !site_out || !n_ctas || capacity < 0) return ACM_ERR_INVALID;
+  ACM_CUDA(cudaDeviceSynchronize());
+  std::vector<int32_t> words(c->sm_count);
+  ACM_CUDA(cudaMemcpy(words.data(), c->wait_diag, sizeof(int32_t) * c->sm_count, cudaMemcpyDeviceToHost));
+  const int n = c->last_ffn_grid;
+  *n_ctas = n;
+  for (int i = 0; i < n && i < capacity; ++i)
+    site_out[i] = (words[i] >> 8) == c->ffn_launch_no ? (words[i] & 0xff) : -1;      // -1: that CTA never started
+  return ACM_OK;
+}
+
+acm_status acm_inject_unpublished_wait(acm_ctx* c, int layer, const void* x, int T, float* out, acm_stream stream) {
+  acm_status st = check_block_args(c, layer, T, true);
+  if (st != ACM_OK) return st;
+  const Layer& L = c->layers[layer];
+  if (!x || !out || (!L.gate_up && !L.mx_gate_up)) return ACM_ERR_INVALID;
+  if (reinterpret_cast<uintptr_t>(x) % 16 != 0 || reinterpret_cast<uintptr_t>(out) % 16 != 0) return ACM_ERR_INVALID;
+  if (c->desc.dtype != ACM_BF16 || L.has_resident) return ACM_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // a tag of its own, which no router or selection kernel is ever launched with
+  int32_t epoch = ++c->epoch;
+  if ((epoch & 0xffff) == 0) epoch = ++c->epoch;
+  if (epoch <= 0) epoch = c->epoch = 1;
+  ACM_CUDA(cudaMemsetAsync(out, 0, sizeof(float) * static_cast<size_t>(T) * c->desc.hidden, s));
+  return run_ffn_list(c, L, x, T, 0, out, s, nullptr, nullptr, false, epoch);
 }
 
 acm_status acm_device_status(acm_ctx* c, acm_stream stream) {

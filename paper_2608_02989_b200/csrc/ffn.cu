@@ -28,7 +28,6 @@
 // f32 path: plain FMA kernels (the fp32 toy configuration is a few MFLOP).
 #include <cuda_bf16.h>
 
-#include <cstdlib>
 #include <mutex>
 
 #include "acm_internal.h"
@@ -39,14 +38,8 @@ namespace {
 #ifndef ACM_FFN_MX
 #define ACM_FFN_MX 0
 #endif
-#ifndef ACM_FFN_STAGES
-#define ACM_FFN_STAGES 3
-#endif
-#ifndef ACM_FFN_ACC
-#define ACM_FFN_ACC 4
-#endif
-constexpr int kStages = ACM_FFN_STAGES;
-constexpr int kAcc = ACM_FFN_ACC;                        // TMEM accumulators in flight (power of two)
+constexpr int kStages = 3;                               // pipeline stages of the weight ring
+constexpr int kAcc = 4;                                  // TMEM accumulators in flight (power of two)
 constexpr int kBK = 64;                                  // K elements of one 128-byte swizzle atom
 constexpr int kAtoms = 2;                                // atoms per pipeline stage: a stage covers 128 K
 constexpr int kTileM = 128;
@@ -67,10 +60,9 @@ static_assert(kAcc * kAccCols + kStages * kMxACols <= 512, "tensor memory: accum
 // bf16 path's.
 constexpr int kThreads = ACM_FFN_MX ? 384 : 256;         // producer, MMA, 4 epilogue warps, helper, publisher (+ 4 expanding warps)
 constexpr int kMxCodeBytes = kTileM * 64;                // 128 rows x 128 four-bit codes
-constexpr int kMxStageBytes = kMxCodeBytes + kTileM * 4; // + one scale byte per row and 32 K
+[[maybe_unused]] constexpr int kMxStageBytes = kMxCodeBytes + kTileM * 4; // + one scale byte per row and 32 K
 constexpr int kFragBytes = kTileM * kMaxNodes * 4;       // contributor fragments pre-summed in shared memory
 constexpr int kFragFloats = kTileM * kMaxNodes;
-constexpr unsigned long long kTimeoutNs = 1000ull * 1000ull * 1000ull;
 
 // Division by a launch constant through a precomputed 64-bit reciprocal (exact for n < 2^32): the
 // schedules below are walked by ONE thread per role, for which a hardware-less integer division is
@@ -135,6 +127,38 @@ struct Plan {
   int a_split;    // experts [0, a_split) form group 0 (complete early), the rest group 1
 };
 
+// Every wait in this kernel is bounded.  What a role needs when one runs out lives in shared memory (GiveUp,
+// touched on slow paths only): the limit, where to raise the status, and this CTA's diagnostic word, which
+// names the wait that gave up first (acm_wait_report reads it).
+enum WaitSite : int {
+  kSiteNone = 0,
+  kSiteAnchorWords = 1,     // prologue: the anchors' tagged words (router kernel)
+  kSiteEligibleWords = 2,   // prologue / helper: the eligible set's tagged words (selection kernel)
+  kSiteStageEmpty = 3,      // weight producer: a ring stage the MMAs have not released
+  kSiteAccEmpty = 4,        // MMA issuer: an accumulator the epilogue has not drained
+  kSiteStageFull = 5,       // MMA issuer: a stage whose copies have not landed
+  kSiteFragFree = 6,        // helper: the fragment buffer in shared memory is still being read
+  kSiteFragArrivals = 7,    // helper: other CTAs' partial sums of a cut tile
+  kSiteFragCopy = 8,        // helper: its own bulk copy of the summed fragment
+  kSiteExpertReady = 9,     // helper: finished-tile counters of the experts a down stage reads
+  kSiteStageArmed = 10,     // helper: the weight producer has not armed the stage
+  kSiteOutStaged = 11,      // publisher: an outgoing fragment from the epilogue
+  kSiteActStaged = 12,      // publisher: a finished activation tile from the epilogue
+  kSiteAccFull = 13,        // epilogue: an accumulator's MMAs
+  kSiteOutFree = 14,        // epilogue: the outgoing-fragment buffer
+  kSiteFragFull = 15,       // epilogue: the summed fragments of a cut tile
+  kSiteActFree = 16,        // epilogue: an activation staging buffer
+  kSitePlanReady = 17,      // any role: the rest of the plan (anchor start)
+  kSitePackedStage = 18     // MXFP4 expanding warps: the packed weight stage
+};
+struct GiveUp {
+  volatile int flag;             // set once this CTA has given up: every role then leaves at its next slow path
+  unsigned long long limit_ns;   // the longest any single wait may last
+  int32_t* status;               // the context's sticky status word
+  int32_t* where;                // this CTA's diagnostic word: (launch number << 8) | WaitSite
+  int32_t tag;                   // launch number << 8
+};
+
 struct __align__(8) Barriers {
   unsigned long long full[kStages];
   unsigned long long empty[kStages];
@@ -151,7 +175,7 @@ struct __align__(8) Barriers {
 #endif
   volatile uint32_t armed;           // stages whose barrier the weight producer has armed so far
   uint32_t tmem_base;
-  int abort_flag;
+  GiveUp give_up;
   float wd[kMaxNodes];          // combine weights of the expert being finalised
   int32_t entry[kMaxSlots];     // this launch's work list: make_entry(source, index) of every activated slot
   int16_t expert[kMaxSlots];    // routed expert id of the slot (-1: shared expert)
@@ -190,29 +214,32 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false (after raising the status once) if the limit ran out or the CTA
-// has already given up; callers then skip the rest of their work.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  if (*abort_flag) return false;
+__device__ __noinline__ void give_up(GiveUp* g, int site) {
+  if (atomicExch(const_cast<int*>(&g->flag), 1) == 0 && g->where) *g->where = g->tag | site;
+  atomicCAS(g->status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+}
+// Returns false if the limit ran out (the status is raised once) or the CTA has already given up; callers
+// then skip the rest of their work.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, GiveUp* g, int site) {
+  if (g->flag) return false;
   for (int i = 0; i < 1024; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_timer();
   for (;;) {
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (global_timer() - t0 > kTimeoutNs) {
-      *abort_flag = 1;
-      atomicCAS(status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+    if (g->flag) return false;
+    if (global_timer() - t0 > g->limit_ns) {
+      give_up(g, site);
       return false;
     }
   }
 }
-// Bounded wait: one inlined poll for the common case (the phase is already complete), the bounded loop
-// out of line.  The single-thread roles pay every instruction of their per-stage loop.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+// One inlined poll for the common case (the phase is already complete), the bounded loop out of line: the
+// single-thread roles pay every instruction of their per-stage loop.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, GiveUp* g, int site) {
   if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, status);
+  return mbar_wait_slow(bar, parity, g, site);
 }
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
   int v;
@@ -223,8 +250,8 @@ __device__ __forceinline__ void red_release_add(int32_t* p, int v) {
   asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 // Bounded wait until *p >= target (p written by other CTAs with release semantics).
-__device__ bool flag_wait_ge(const int32_t* p, int target, volatile int* abort_flag, int32_t* status) {
-  if (*abort_flag) return false;
+__device__ bool flag_wait_ge(const int32_t* p, int target, GiveUp* g, int site) {
+  if (g->flag) return false;
   for (int i = 0; i < 256; ++i)
     if (ld_acquire(p) >= target) return true;
   const unsigned long long t0 = global_timer();
@@ -233,22 +260,34 @@ __device__ bool flag_wait_ge(const int32_t* p, int target, volatile int* abort_f
       if (ld_acquire(p) >= target) return true;
       __nanosleep(64);
     }
-    if (*abort_flag) return false;
-    if (global_timer() - t0 > kTimeoutNs) {
-      *abort_flag = 1;
-      atomicCAS(status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+    if (g->flag) return false;
+    if (global_timer() - t0 > g->limit_ns) {
+      give_up(g, site);
       return false;
     }
   }
+}
+// Bounded poll of one self-validating word (16 payload bits under a 16-bit tag) written by an earlier kernel
+// of the same stream: returns the payload, or sets `seen` to false when the limit ran out.
+__device__ __forceinline__ uint32_t poll_tagged_word(const uint32_t* word, uint32_t tag, unsigned long long limit_ns, bool& seen) {
+  uint32_t v = 0;
+  const unsigned long long t0 = global_timer();
+  do {
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
+    seen = (v >> 16) == tag;
+  } while (!seen && global_timer() - t0 < limit_ns);
+  return seen ? (v & 0xffffu) : 0u;
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+#if ACM_FFN_MX
 __device__ __forceinline__ void bulk_load_hint(uint32_t smem_dst, const void* gmem_src, uint32_t bytes, uint32_t bar, uint64_t policy) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
                ::"r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(bar), "l"(policy) : "memory");
 }
+#endif
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
 // Barrier over the 128 epilogue threads that also ANDs a predicate, so that all of them take the
@@ -341,7 +380,7 @@ __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr) {
   d |= static_cast<uint64_t>(2) << 61;                           // 128-byte swizzle
   return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+#if ACM_FFN_MX
 // The same MMA with the A operand (128 rows x 16 K bf16) in tensor memory: row = lane, two K elements per column.
 __device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
                                              uint32_t accumulate) {
@@ -358,6 +397,8 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
         "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+#endif
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
 __device__ __forceinline__ uint32_t umma_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
 }
@@ -387,8 +428,8 @@ struct Sched {
   }
 };
 
-#define ACM_TRACE(slot) do { if (p.trace) p.trace[static_cast<size_t>(blockIdx.x) * 32 + (slot)] = global_timer(); } while (0)
-#define ACM_TRACE_ADD(slot, dt) do { if (p.trace) p.trace[static_cast<size_t>(blockIdx.x) * 32 + (slot)] += (dt); } while (0)
+// Optional time stamps (acm_stage_timing): per CTA, slot 0 = the roles start, 10 / 11 = its last gate/up / down tile is done.
+#define ACM_STAMP(slot) do { if (p.trace) p.trace[static_cast<size_t>(blockIdx.x) * 32 + (slot)] = global_timer(); } while (0)
 
 struct FfnArgs {
   int T, H, I, n_pad;
@@ -410,8 +451,10 @@ struct FfnArgs {
   const uint32_t* anc_flag;    // non-null: eight tagged words with the anchor experts (Eq. 5), published before sel_flag
   float* out;
   int32_t* status;
-  int phase_mask;
-  unsigned long long* trace;   // optional [grid][32] timestamps (debugging aid), may be null
+  unsigned long long wait_limit_ns;   // the longest any single device-side wait may last
+  int32_t* wait_diag;          // [grid] per-CTA diagnostic words (see GiveUp) or null
+  int32_t launch_tag;          // launch number << 8
+  unsigned long long* trace;   // optional [grid][32] time stamps (acm_stage_timing) or null
 #if ACM_FFN_MX
   const unsigned char* mx_gate_up;   // [E][I/64][H/128][8704]
   const unsigned char* mx_down;      // [E][H/128][I/128][8704]
@@ -427,7 +470,7 @@ __device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMa
 // first touch costs every role a trip to DRAM at the start of the kernel).  It has at most four
 // segments; lane i of one warp works out the i-th one by itself -- the four candidates in order, each
 // present or not -- and its own range in it, so nothing waits for a serial pass.
-__device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act, int tpe, int grid, int phase_mask,
+__device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act, int tpe, int grid,
                                           const FastDiv& d_kc1, int kpe, const FastDiv& d_grid, const FastDiv& d_tpe,
                                           int h_tiles, int n_pre = 0, int base = 0);
 // Range of segment `si` for CTA `cta` (see SegRange).  (tiles * chunks * grid fits 32 bits: launcher.)
@@ -456,13 +499,12 @@ __device__ __forceinline__ SegRange make_range(const Segment& sg, int cta, const
 // With a pre-segment (n_pre experts whose gate/up tiles are already being streamed as segment 0, base = 1) the
 // gate/up segments cover the other experts' tiles only; the down segments cover everyone, the pre-streamed experts
 // counting as complete early.
-__device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act, int tpe, int grid, int phase_mask,
+__device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act, int tpe, int grid,
                                           const FastDiv& d_kc1, int kpe, const FastDiv& d_grid, const FastDiv& d_tpe,
                                           int h_tiles, int n_pre, int base) {
   const int t_pre = n_pre * tpe;
   const int n_t = (n_act - n_pre) * tpe;
   const int rounds = static_cast<int>(fdiv(static_cast<unsigned>(n_t), d_grid)), rem = n_t - rounds * grid;
-  const bool p1 = (phase_mask & 1) != 0, p2 = (phase_mask & 2) != 0;
   // candidates in execution order: two gate/up segments, two down segments
   Segment c0, c1, c2, c3;
   bool h0, h1, h2, h3;
@@ -470,15 +512,15 @@ __device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act
   if (rounds == 0) {
     const int n_rest = n_act - n_pre, nA = (n_rest + 1) / 2;
     a_split = n_pre + nA;
-    c0 = Segment{1, 0, t_pre, nA * tpe, 0, 0, 0, d_kc1};                      h0 = p1 && nA > 0;
-    c1 = Segment{1, 0, t_pre + nA * tpe, (n_rest - nA) * tpe, 0, 0, 1, d_kc1};   h1 = p1 && n_rest > nA;
+    c0 = Segment{1, 0, t_pre, nA * tpe, 0, 0, 0, d_kc1};                      h0 = nA > 0;
+    c1 = Segment{1, 0, t_pre + nA * tpe, (n_rest - nA) * tpe, 0, 0, 1, d_kc1};   h1 = n_rest > nA;
   } else {
     a_split = n_pre + static_cast<int>(fdiv(static_cast<unsigned>(rem + (rounds - 1) * grid), d_tpe));
-    c0 = Segment{1, 0, t_pre, rem, 0, 0, 0, d_kc1};                           h0 = p1 && rem > 0;
-    c1 = Segment{1, 1, t_pre + rem, rounds * grid, 0, 0, 1, d_kc1};           h1 = p1;
+    c0 = Segment{1, 0, t_pre, rem, 0, 0, 0, d_kc1};                           h0 = rem > 0;
+    c1 = Segment{1, 1, t_pre + rem, rounds * grid, 0, 0, 1, d_kc1};           h1 = true;
   }
-  c2 = Segment{2, 0, 0, 0, 0, a_split, 0, plain_div(static_cast<unsigned>(a_split * kpe))};                 h2 = p2 && a_split > 0;
-  c3 = Segment{2, 0, 0, 0, a_split, n_act, 1, plain_div(static_cast<unsigned>((n_act - a_split) * kpe))};   h3 = p2 && n_act > a_split;
+  c2 = Segment{2, 0, 0, 0, 0, a_split, 0, plain_div(static_cast<unsigned>(a_split * kpe))};                 h2 = a_split > 0;
+  c3 = Segment{2, 0, 0, 0, a_split, n_act, 1, plain_div(static_cast<unsigned>((n_act - a_split) * kpe))};   h3 = n_act > a_split;
   const int i0 = 0, i1 = i0 + h0, i2 = i1 + h1, i3 = i2 + h2, n = i3 + h3;
   Segment mine = c0;
   bool have = false;
@@ -516,12 +558,11 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   float* sfrag = reinterpret_cast<float*>(after_ring + kOutStageBytes);
   unsigned char* hstage = after_ring + kOutStageBytes + kFragBytes;   // 2 x [node][64 features] bf16, swizzled
   Barriers* bars = reinterpret_cast<Barriers*>(after_ring + kOutStageBytes + kFragBytes + 2 * kHStageBytes);
-  volatile int* abort_flag = &bars->abort_flag;
+  GiveUp* const quit = &bars->give_up;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, G = gridDim.x;
   griddep_launch_dependents();
-  if (threadIdx.x == 0) ACM_TRACE(12);     // kernel entry
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&bars->full[s]), ACM_FFN_MX ? 5 : 1);   // MXFP4: + one arrival per expanding warp
@@ -546,7 +587,12 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       mbar_init(smem_u32(&bars->hst_full[b]), 128);
       mbar_init(smem_u32(&bars->hst_free[b]), 1);
     }
-    bars->abort_flag = 0;
+    bars->give_up.flag = 0;
+    bars->give_up.limit_ns = p.wait_limit_ns;
+    bars->give_up.status = p.status;
+    bars->give_up.where = p.wait_diag ? p.wait_diag + blockIdx.x : nullptr;
+    bars->give_up.tag = p.launch_tag;
+    if (p.wait_diag) p.wait_diag[blockIdx.x] = p.launch_tag;      // "this CTA of that launch has started"
     bars->armed = 0;
     fence_barrier_init();
   }
@@ -571,82 +617,29 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   // set, completes the work list (the pre-streamed experts keep the first slots) and the plan, and opens
   // `plan_ready`, which every other role passes before its second segment.
   constexpr bool pre = kPre;
-  if (threadIdx.x == 0) ACM_TRACE(29);
-  if (pre) {
-    // eight words per block (a batch: the union of the blocks' anchors), one thread each, warps 2 and 3
+  if (pre || early) {
+    // Eight tagged words per block (16 mask bits under the 16-bit tag of this call; a batch has eight per block
+    // and takes their union), each polled by its own thread of warps 2 and 3 -- four blocks per warp -- which have
+    // nothing else to do yet, so that the poll runs beside the set-up above.  With the anchor start these are the
+    // anchors' words, else the eligible set's.
     bool timed_out = false;
     if (threadIdx.x >= 64 && threadIdx.x < 128) {
       const int j = threadIdx.x - 64;
-      const bool mine = j < 2 * kMaskWords * p.sel_blocks;
+      const uint32_t* words = pre ? p.anc_flag : p.sel_flag;
       bool seen = true;
-      uint32_t v = 0;
-      if (mine) {
-        const uint32_t tag = static_cast<uint32_t>(p.sel_epoch) & 0xffffu;
-        const unsigned long long t0 = global_timer();
-        do {
-          asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.anc_flag + j) : "memory");
-          seen = (v >> 16) == tag;
-        } while (!seen && global_timer() - t0 < kTimeoutNs);
-      }
+      uint32_t bits = 0u;
+      if (j < 2 * kMaskWords * p.sel_blocks)
+        bits = poll_tagged_word(words + j, static_cast<uint32_t>(p.sel_epoch) & 0xffffu, p.wait_limit_ns, seen);
       timed_out = !seen;
-      uint32_t bits = (mine && seen) ? (v & 0xffffu) : 0u;
       bits |= __shfl_xor_sync(0xffffffffu, bits, 8);
       bits |= __shfl_xor_sync(0xffffffffu, bits, 16);
-      if (lane < 2 * kMaskWords) bars->anc_part[(j >> 5) * 2 * kMaskWords + lane] = bits;
+      if (lane < 2 * kMaskWords) (pre ? bars->anc_part : bars->sel_half)[(j >> 5) * 2 * kMaskWords + lane] = bits;
     }
     __syncthreads();
-    if (timed_out) {
-      bars->abort_flag = 1;
-      atomicCAS(p.status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
-    }
-  } else if (early) {
-    // eight tagged words (16 mask bits under the 16-bit tag of this call), each polled by its own thread --
-    // of warp 2, which has nothing else to do yet, so that the poll runs beside the set-up above
-    bool timed_out = false;
-    if (p.sel_blocks > 1) {
-      // a batch of blocks: eight words per block, one thread each (warps 2 and 3: four blocks per warp); the
-      // work list is the union of the blocks' sets
-      if (threadIdx.x >= 64 && threadIdx.x < 128) {
-        const int j = threadIdx.x - 64;
-        const bool mine = j < 2 * kMaskWords * p.sel_blocks;
-        bool seen = true;
-        uint32_t v = 0;
-        if (mine) {
-          const uint32_t tag = static_cast<uint32_t>(p.sel_epoch) & 0xffffu;
-          const unsigned long long t0 = global_timer();
-          do {
-            asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.sel_flag + j) : "memory");
-            seen = (v >> 16) == tag;
-          } while (!seen && global_timer() - t0 < kTimeoutNs);
-        }
-        timed_out = !seen;
-        uint32_t bits = (mine && seen) ? (v & 0xffffu) : 0u;
-        bits |= __shfl_xor_sync(0xffffffffu, bits, 8);
-        bits |= __shfl_xor_sync(0xffffffffu, bits, 16);
-        if (lane < 2 * kMaskWords) bars->sel_half[(j >> 5) * 2 * kMaskWords + lane] = bits;
-      }
-    } else if (threadIdx.x >= 64 && threadIdx.x < 64 + 2 * kMaskWords) {
-      const int i = threadIdx.x - 64;
-      bool seen = false;
-      uint32_t v = 0;
-      const uint32_t tag = static_cast<uint32_t>(p.sel_epoch) & 0xffffu;
-      const unsigned long long t0 = global_timer();
-      do {
-        asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.sel_flag + i) : "memory");
-        seen = (v >> 16) == tag;
-      } while (!seen && global_timer() - t0 < kTimeoutNs);
-      timed_out = !seen;
-      bars->sel_half[i] = seen ? (v & 0xffffu) : 0u;
-    }
-    __syncthreads();
-    if (timed_out) {
-      bars->abort_flag = 1;
-      atomicCAS(p.status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
-    }
+    if (timed_out) give_up(quit, pre ? kSiteAnchorWords : kSiteEligibleWords);
   } else {
     griddep_wait();
   }
-  if (threadIdx.x == 0) ACM_TRACE(30);
   // The work list of this launch: slot a = the a-th activated expert of this list in ascending id
   // order (list 0: the resident ones, then the shared experts; list 1: the non-resident ones, which
   // the host has copied into staging slot a).
@@ -659,8 +652,8 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       act = (bars->anc_part[2 * wd] | bars->anc_part[2 * kMaskWords + 2 * wd]) |
             ((bars->anc_part[2 * wd + 1] | bars->anc_part[2 * kMaskWords + 2 * wd + 1]) << 16);      // for now: the anchors only
     } else if (early) {
-      act = bars->sel_half[2 * wd] | (bars->sel_half[2 * wd + 1] << 16);
-      if (p.sel_blocks > 1) act |= bars->sel_half[2 * kMaskWords + 2 * wd] | (bars->sel_half[2 * kMaskWords + 2 * wd + 1] << 16);
+      act = (bars->sel_half[2 * wd] | bars->sel_half[2 * kMaskWords + 2 * wd]) |
+            ((bars->sel_half[2 * wd + 1] | bars->sel_half[2 * kMaskWords + 2 * wd + 1]) << 16);
     } else {
       act = p.act_mask[wd];
     }
@@ -702,7 +695,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       bars->plan.n_seg = 1;
     }
   } else if (warp == kThreads / 32 - 1 && lane < 4) {      // (the publisher warp has nothing else to do yet)
-    plan_lane(bars->plan, lane, cta, n_act, tpe, G, p.phase_mask, p.d_kc1, kpe, p.d_grid, p.d_tpe, h_tiles);
+    plan_lane(bars->plan, lane, cta, n_act, tpe, G, p.d_kc1, kpe, p.d_grid, p.d_tpe, h_tiles);
   }
   int32_t* s_entry = bars->entry;
   if (threadIdx.x < kMaxExperts) {
@@ -723,19 +716,18 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     s_entry[n_routed + i] = make_entry(kSrcShared, i);
     bars->expert[n_routed + i] = -1;
   }
-  if (threadIdx.x == 0) ACM_TRACE(31);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const Segment* seg = bars->plan.seg;
   const uint32_t tmem_base = bars->tmem_base;
-  if (threadIdx.x == 0) ACM_TRACE(0);
+  if (threadIdx.x == 0) ACM_STAMP(0);
   // Does segment si exist?  With a pre-segment the plan behind segment 0 arrives later (the helper warp opens
   // plan_ready); n_seg is read from shared memory every time.
   const int n_seg_fixed = bars->plan.n_seg;
   auto have_seg = [&](int si, bool wait_for_plan) -> bool {
     if constexpr (kPre) {
-      if (si == 1 && wait_for_plan && !mbar_wait(smem_u32(&bars->plan_ready), 0u, abort_flag, p.status)) return false;
+      if (si == 1 && wait_for_plan && !mbar_wait(smem_u32(&bars->plan_ready), 0u, quit, kSitePlanReady)) return false;
       return si < bars->plan.n_seg;
     } else {
       return si < n_seg_fixed;
@@ -751,7 +743,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     if (lane == 0) {
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
       uint32_t s = 0, par = 0, n_armed = 0;
-      bool ok = true, traced_first = false;
+      bool ok = true;
       for (int si = 0; ok && have_seg(si, true); ++si) {
         const Segment sg = seg[si];
         if (sg.phase == 1) {
@@ -763,7 +755,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
             const int r0 = (sg.t0 + tile - a_of * tpe) * 64, eidx = entry_idx(ent);
             const CUtensorMap* gu = pick_map(entry_src(ent), &maps.gate_up, &maps.shared_gate_up, &maps.staged_gate_up);
             for (int kc = k0; kc < k1; ++kc) {
-              if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
+              if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, quit, kSiteStageEmpty))) break;
               const uint32_t full = smem_u32(&bars->full[s]);
               const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
 #if ACM_FFN_MX
@@ -779,12 +771,10 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
               tma_load_5d(sa, gu, full, 0, r0, 0, kc * kAtoms, eidx, pol_w);   // 64 gate + 64 up rows, 2 atoms
 #endif
               tma_load_3d(sa + kABytes, &x_map, full, 0, 0, kc * kAtoms, pol_x);
-              if (!traced_first) { ACM_TRACE(1); traced_first = true; }
               ++n_armed;
               if (++s == kStages) { s = 0; par ^= 1u; }
             }
           }
-          ACM_TRACE(sg.p1_index == 0 ? 13 : 2);
         } else {
           Sched sc(bars->plan.range[si]);
           int ht, k0, k1;
@@ -795,7 +785,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
             const CUtensorMap* dn = pick_map(entry_src(ent), &maps.down, &maps.shared_down, &maps.staged_down);
             int eidx = entry_idx(ent);
             for (int kc = k0; kc < k1; ++kc) {
-              if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, abort_flag, p.status))) break;
+              if (!(ok = mbar_wait(smem_u32(&bars->empty[s]), par ^ 1u, quit, kSiteStageEmpty))) break;
               const uint32_t full = smem_u32(&bars->full[s]);
               const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
 #if ACM_FFN_MX
@@ -820,7 +810,6 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
               }
             }
           }
-          ACM_TRACE(sg.p1_index == 0 ? 14 : 5);
         }
       }
       // The block's activated-expert counts, by the thread that is done first (its copies are all issued
@@ -850,25 +839,24 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       const uint64_t desc_hi = umma_smem_desc(0);
       uint32_t it = 0, f = 0;
       bool ok = true;
-      unsigned long long acc_f[2] = {0, 0};
       for (int si = 0; ok && have_seg(si, true); ++si) {
-        const Segment sg = seg[si];
         Sched sc(bars->plan.range[si]);
         int tile, k0, k1;
         while (ok && sc.next(tile, k0, k1)) {
           const uint32_t b = f % kAcc;
-          if (!(ok = mbar_wait(smem_u32(&bars->tempty[b]), ((f / kAcc) & 1u) ^ 1u, abort_flag, p.status))) break;
+          if (!(ok = mbar_wait(smem_u32(&bars->tempty[b]), ((f / kAcc) & 1u) ^ 1u, quit, kSiteAccEmpty))) break;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + b * kAccCols;
           for (int kc = k0; kc < k1; ++kc, ++it) {
             const uint32_t s = it % kStages, par = (it / kStages) & 1u;
-            const unsigned long long tw = p.trace ? global_timer() : 0ull;
-            if (!(ok = mbar_wait(smem_u32(&bars->full[s]), par, abort_flag, p.status))) break;
-            if (p.trace) { acc_f[sg.phase - 1] += global_timer() - tw; if (it == 0) ACM_TRACE(6); }
+            if (!(ok = mbar_wait(smem_u32(&bars->full[s]), par, quit, kSiteStageFull))) break;
             tc_fence_after();
             // descriptors: only the address field changes from stage to stage and atom to atom
             const uint32_t sa = smem_u32(stage_base) + s * kStageBytes;
-            const uint64_t da0 = desc_hi | ((sa & 0x3ffffu) >> 4), db0 = desc_hi | (((sa + kABytes) & 0x3ffffu) >> 4);
+#if !ACM_FFN_MX
+            const uint64_t da0 = desc_hi | ((sa & 0x3ffffu) >> 4);
+#endif
+            const uint64_t db0 = desc_hi | (((sa + kABytes) & 0x3ffffu) >> 4);
 #pragma unroll
             for (int at = 0; at < kAtoms; ++at) {
 #pragma unroll
@@ -889,9 +877,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
           umma_commit(smem_u32(&bars->tfull[b]));
           ++f;
         }
-        ACM_TRACE(6 + sg.phase);
       }
-      ACM_TRACE_ADD(19, acc_f[0]); ACM_TRACE_ADD(20, acc_f[1]);
       if (!ok) {
         // giving up: wait (bounded) for the MMAs already issued before TMEM is released
         umma_commit(smem_u32(&bars->drained));
@@ -922,15 +908,9 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
         for (int part = 0; part < 2; ++part) {
           const int j = lane + 32 * part;
           if (j < n_words) {
-            uint32_t v = 0;
-            bool got = false;
-            const unsigned long long t0 = global_timer();
-            do {
-              asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.sel_flag + j) : "memory");
-              got = (v >> 16) == tag;
-            } while (!got && global_timer() - t0 < kTimeoutNs);
+            bool got = true;
+            half |= poll_tagged_word(p.sel_flag + j, tag, p.wait_limit_ns, got);
             seen = seen && got;
-            half |= got ? (v & 0xffffu) : 0u;
           }
         }
         half |= __shfl_xor_sync(0xffffffffu, half, 8);
@@ -962,15 +942,13 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
           bars->expert[n_pre + n_rest + lane] = -1;
         }
         if (lane < 4)
-          plan_lane(bars->plan, lane, cta, n_pre + n_rest + p.n_shared, tpe, G, p.phase_mask, p.d_kc1, kpe, p.d_grid, p.d_tpe,
-                    h_tiles, n_pre, 1);
+          plan_lane(bars->plan, lane, cta, n_pre + n_rest + p.n_shared, tpe, G, p.d_kc1, kpe, p.d_grid, p.d_tpe, h_tiles,
+                    n_pre, 1);
       } else if (lane == 0) {
-        bars->abort_flag = 1;
-        atomicCAS(p.status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+        give_up(quit, kSiteEligibleWords);
       }
       __syncwarp();
       if (lane == 0) {
-        ACM_TRACE(30);
         mbar_arrive(smem_u32(&bars->plan_ready));
       }
       ok = good;
@@ -990,7 +968,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
         const bool head = (last_tile * kc1 >= ub) && (ue < tile_end);   // starts at chunk 0, ends before the tile does
         if (!head) continue;
         if (frag_uses > 0) {   // the buffer still holds the previous segment's sum until the epilogue has read it
-          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->frag_free), (frag_uses - 1) & 1u, abort_flag, p.status));
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->frag_free), (frag_uses - 1) & 1u, quit, kSiteFragFree));
           if (!ok) break;
         }
         float* frag = p.frag + (static_cast<size_t>(sg.p1_index) * G + cta) * kFragFloats;   // this CTA's buffer
@@ -1005,7 +983,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
         {
           // every CTA holding a later part of the tile has reduce-added its fragment: one bulk copy
           bool got = true;
-          if (lane == 0) got = flag_wait_ge(arrived, n_contrib, abort_flag, p.status);
+          if (lane == 0) got = flag_wait_ge(arrived, n_contrib, quit, kSiteFragArrivals);
           ok = __all_sync(0xffffffffu, got);
           if (!ok) break;
           if (lane == 0) {
@@ -1015,10 +993,9 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                          ::"r"(smem_u32(sfrag)), "l"(frag), "r"(static_cast<uint32_t>(n_el) * 4u), "r"(hb) : "memory");
           }
-          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->helper), frag_uses & 1u, abort_flag, p.status));
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->helper), frag_uses & 1u, quit, kSiteFragCopy));
           if (!ok) break;
           if (lane == 0) mbar_arrive(smem_u32(&bars->frag_full[sg.p1_index]));
-          if (lane == 0) ACM_TRACE(sg.p1_index == 0 ? 9 : 15);
           // leave the buffer and its counter zero for the next launch
           float4* z4 = reinterpret_cast<float4*>(frag);
           for (int i = lane; i < n_el / 4; i += 32) z4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1042,10 +1019,9 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
               q_hi = static_cast<int>(fdiv(static_cast<unsigned>(rg.k00) + n_units - 1u, p.d_kpe));
             }
             for (int q = q_lo + lane; q <= q_hi && good; q += 32)
-              good = flag_wait_ge(&p.ready[sg.a0 + q], tpe, abort_flag, p.status);
+              good = flag_wait_ge(&p.ready[sg.a0 + q], tpe, quit, kSiteExpertReady);
           }
           good = __all_sync(0xffffffffu, good);
-          if (lane == 0) ACM_TRACE(sg.p1_index == 0 ? 17 : 18);
         }
         if (good && lane == 0) {
           const uint64_t pol_x = policy_evict_last();
@@ -1060,10 +1036,9 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
               if (bars->armed <= hidx) {
                 const unsigned long long t0 = global_timer();
                 while (bars->armed <= hidx) {
-                  if (*abort_flag) { good = false; break; }
-                  if (global_timer() - t0 > kTimeoutNs) {
-                    *abort_flag = 1;
-                    atomicCAS(p.status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
+                  if (quit->flag) { good = false; break; }
+                  if (global_timer() - t0 > p.wait_limit_ns) {
+                    give_up(quit, kSiteStageArmed);
                     good = false;
                     break;
                   }
@@ -1097,7 +1072,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
         int tile, k0, k1;
         while (ok && sc.next(tile, k0, k1)) {
           if (k0 > 0) {
-            if (!(ok = mbar_wait(smem_u32(&bars->ost_full), ost_n & 1u, abort_flag, p.status))) break;
+            if (!(ok = mbar_wait(smem_u32(&bars->ost_full), ost_n & 1u, quit, kSiteOutStaged))) break;
             const uint32_t bytes = static_cast<uint32_t>(p.n_pad) * kTileM * 4u;
             // All CTAs that hold a tail part of this tile add into ONE global buffer, that of the CTA
             // which owns the tile's first chunks and will finish it.  The buffers are zero between
@@ -1115,7 +1090,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
             ++ost_n;
           } else {
             const uint32_t hb = fin_n & 1u;
-            if (!(ok = mbar_wait(smem_u32(&bars->hst_full[hb]), (fin_n >> 1) & 1u, abort_flag, p.status))) break;
+            if (!(ok = mbar_wait(smem_u32(&bars->hst_full[hb]), (fin_n >> 1) & 1u, quit, kSiteActStaged))) break;
             const int a = static_cast<int>(fdiv(static_cast<unsigned>(sg.t0 + tile), p.d_tpe)), ti = sg.t0 + tile - a * tpe;
             asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
                          ::"l"(&hs_map), "r"(0), "r"(0), "r"(ti), "r"(a), "r"(smem_u32(hstage + hb * kHStageBytes)) : "memory");
@@ -1124,8 +1099,6 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
             red_release_add(&p.ready[a], 1);
             mbar_arrive(smem_u32(&bars->hst_free[hb]));
             ++fin_n;
-            if (fin_n == 1) ACM_TRACE(16);
-            ACM_TRACE(28);
           }
         }
       }
@@ -1147,7 +1120,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     uint32_t sc = 0;
     auto fetch = [&](unsigned it) -> bool {
       const uint32_t s = it % kStages, par = (it / kStages) & 1u;
-      if (!mbar_wait(smem_u32(&bars->raw[s]), par, abort_flag, p.status)) return false;
+      if (!mbar_wait(smem_u32(&bars->raw[s]), par, quit, kSitePackedStage)) return false;
       const unsigned char* A = stage_base + static_cast<size_t>(s) * kStageBytes;
       // (the record keeps the row's four 16-byte pieces rotated by the row number, so that a warp's loads
       // spread over all banks)
@@ -1219,7 +1192,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     // has copied the previous fragment out
     auto wait_ostage = [&]() -> bool {
       if (ost_uses == 0) return true;
-      return epi_vote_all(mbar_wait(smem_u32(&bars->ost_free), (ost_uses - 1) & 1u, abort_flag, p.status));
+      return epi_vote_all(mbar_wait(smem_u32(&bars->ost_free), (ost_uses - 1) & 1u, quit, kSiteOutFree));
     };
     for (int si = 0; ok && have_seg(si, true); ++si) {
       const Segment sg = seg[si];
@@ -1242,9 +1215,8 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
               wd_mine = ex_id >= 0 ? __ldcg(p.wtab + static_cast<size_t>(ex_id) * kMaxNodes + row) : (row < p.T ? 1.0f : 0.0f);
             }
           }
-          ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f / kAcc) & 1u, abort_flag, p.status));
+          ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f / kAcc) & 1u, quit, kSiteAccFull));
           if (!ok) break;
-          if (row == 0) ACM_TRACE(21);
           tc_fence_after();
           load_acc(b);
           ++f;
@@ -1260,17 +1232,15 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
             continue;
           }
           if (row < p.n_pad) bars->wd[row] = wd_mine;
-          if (row == 0 && fin_count == 0) ACM_TRACE(3);
           if (k1 < kc1) {
             // head part: the helper warp has summed the other CTAs' fragments of this tile into smem
-            ok = epi_vote_all(mbar_wait(smem_u32(&bars->frag_full[sg.p1_index]), 0, abort_flag, p.status));
+            ok = epi_vote_all(mbar_wait(smem_u32(&bars->frag_full[sg.p1_index]), 0, quit, kSiteFragFull));
             if (!ok) break;
 #pragma unroll
             for (int c = 0; c < kMaxNodes; ++c)
               if (c < p.n_pad) v[c] += sfrag[c * kTileM + row];
             mbar_arrive(smem_u32(&bars->frag_free));
           }
-          if (row == 0) ACM_TRACE(23);
           // rows 0..63 hold gate, rows 64..127 the matching up projections.  Each pair of threads
           // (i, i+64) splits the node columns: the gate thread finishes columns [0, 32), the up
           // thread columns [32, 64); they swap the halves they do not finish through smem.
@@ -1288,10 +1258,9 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
           }
           const uint32_t hb = fin_count & 1u;
           bool hst_ok = true;
-          if (fin_count >= 2) hst_ok = mbar_wait(smem_u32(&bars->hst_free[hb]), ((fin_count >> 1) - 1) & 1u, abort_flag, p.status);
+          if (fin_count >= 2) hst_ok = mbar_wait(smem_u32(&bars->hst_free[hb]), ((fin_count >> 1) - 1) & 1u, quit, kSiteActFree);
           ok = epi_vote_all(hst_ok);      // also orders the exchange writes above before the reads below
           if (!ok) break;
-          if (row == 0) ACM_TRACE(24);
           {
             unsigned char* hs = hstage + hb * kHStageBytes;
             const int c0 = quarter < 2 ? 0 : kHalf;
@@ -1328,17 +1297,15 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
             fence_proxy_async_smem();
             mbar_arrive(smem_u32(&bars->hst_full[hb]));
             ++fin_count;
-            if (row == 0 && fin_count == 1) ACM_TRACE(4);
-            if (row == 0) ACM_TRACE(25);
           }
         }
-        if (row == 0) ACM_TRACE(10);
+        if (row == 0) ACM_STAMP(10);
       } else {
         Sched sc(bars->plan.range[si]);
         int ht, k0, k1;
         while (sc.next(ht, k0, k1)) {
           const uint32_t b = f % kAcc;
-          ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f / kAcc) & 1u, abort_flag, p.status));
+          ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f / kAcc) & 1u, quit, kSiteAccFull));
           if (!ok) break;
           tc_fence_after();
           load_acc(b);
@@ -1348,7 +1315,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
           for (int c = 0; c < kMaxNodes; ++c)
             if (c < p.T) atomicAdd(dst + static_cast<size_t>(c) * p.H, v[c]);
         }
-        if (row == 0) ACM_TRACE(11);
+        if (row == 0) ACM_STAMP(11);
       }
     }
   }
@@ -1366,12 +1333,13 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
 // h[t][j][i] = silu(g) * u for routed slot j < k (expert idx[t][j]) and shared slot j >= k.
 __global__ void k_ffn_f32_gate_up(const float* __restrict__ x, const float* __restrict__ gate_up,
                                   const float* __restrict__ shared_gate_up, const int32_t* __restrict__ idx,
-                                  float* __restrict__ hbuf, int T, int H, int I, int k, int n_shared) {
+                                  float* __restrict__ hbuf, int T, int H, int I, int E, int k, int n_shared) {
   const int slots = k + n_shared;
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= T * slots * I) return;
   const int i = warp % I, j = (warp / I) % slots, t = warp / (I * slots);
-  const int e = j < k ? idx[t * k + j] : j - k;
+  int e = j < k ? idx[t * k + j] : j - k;
+  if (j < k && e >= E) e = -1;                 // an id outside the layer is an empty slot, like -1
   const float* base = j < k ? gate_up : shared_gate_up;
   float h = 0.0f;
   if (e >= 0) {
@@ -1395,7 +1363,7 @@ __global__ void k_ffn_f32_gate_up(const float* __restrict__ x, const float* __re
 __global__ void k_ffn_f32_down(const float* __restrict__ down, const float* __restrict__ shared_down,
                                const int32_t* __restrict__ idx, const float* __restrict__ w,
                                const float* __restrict__ hbuf, float* __restrict__ out, int T, int H, int I,
-                               int k, int n_shared) {
+                               int E, int k, int n_shared) {
   const int slots = k + n_shared;
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (warp >= T * H) return;
@@ -1403,7 +1371,7 @@ __global__ void k_ffn_f32_down(const float* __restrict__ down, const float* __re
   float y = 0.f;
   for (int j = 0; j < slots; ++j) {
     const int e = j < k ? idx[t * k + j] : j - k;
-    if (e < 0) continue;
+    if (e < 0 || (j < k && e >= E)) continue;
     const float* d_row = (j < k ? down : shared_down) + (static_cast<size_t>(e) * H + hh) * I;
     const float* hr = hbuf + (static_cast<size_t>(t) * slots + j) * I;
     float acc = 0.f;
@@ -1458,9 +1426,9 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   a.stats = L.stats; a.hbuf = static_cast<__nv_bfloat16*>(L.hbuf);
   a.ready = L.ready; a.frag = L.frag; a.frag_flag = L.frag_flag;
   a.sel_flag = L.sel_flag; a.sel_epoch = L.sel_epoch; a.sel_blocks = L.sel_blocks;
-  a.anc_flag = (L.sel_blocks < 1 || L.sel_blocks > kMaxEarlyBlocks || L.li != 0 || L.resident || L.slot_of ||
-                L.phase_mask != 3) ? nullptr : L.anc_flag;
-  a.out = L.out; a.status = L.status; a.phase_mask = L.phase_mask; a.trace = L.trace;
+  a.anc_flag = (L.sel_blocks < 1 || L.sel_blocks > kMaxEarlyBlocks || L.li != 0 || L.resident || L.slot_of) ? nullptr : L.anc_flag;
+  a.out = L.out; a.status = L.status; a.trace = L.trace;
+  a.wait_limit_ns = L.wait_limit_ns; a.wait_diag = L.wait_diag; a.launch_tag = L.launch_tag;
 #if ACM_FFN_MX
   if (!L.mx_gate_up || !L.mx_down || L.I % 128 != 0 || L.n_shared != 0) return cudaErrorInvalidValue;
   a.mx_gate_up = static_cast<const unsigned char*>(L.mx_gate_up);
@@ -1485,8 +1453,7 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
     attr[0].val.cooperative = 1;
   }
   cfg.attrs = attr;
-  static const bool plain = [] { const char* e = std::getenv("ACM_FFN_PLAIN_LAUNCH"); return e && e[0] == '1'; }();
-  cfg.numAttrs = (plain && !L.pdl) ? 0 : 1;
+  cfg.numAttrs = 1;
   return cudaLaunchKernelExC(&cfg, a.anc_flag && a.sel_flag ? reinterpret_cast<const void*>(ACM_FFN_KERNEL<true>)
                                                             : reinterpret_cast<const void*>(ACM_FFN_KERNEL<false>), args);
 }
@@ -1495,16 +1462,16 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
 cudaError_t launch_ffn_f32(const float* x, const float* gate_up, const float* down,
                            const float* shared_gate_up, const float* shared_down, int n_shared,
                            const int32_t* idx, const float* w, float* hbuf, float* out, int T, int H,
-                           int I, int k, cudaStream_t s) {
+                           int I, int E, int k, cudaStream_t s) {
   const int slots = k + n_shared;
   const long long warps1 = static_cast<long long>(T) * slots * I;
   k_ffn_f32_gate_up<<<static_cast<unsigned>((warps1 * 32 + 255) / 256), 256, 0, s>>>(x, gate_up, shared_gate_up, idx, hbuf,
-                                                                                   T, H, I, k, n_shared);
+                                                                                   T, H, I, E, k, n_shared);
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
   const long long warps2 = static_cast<long long>(T) * H;
   k_ffn_f32_down<<<static_cast<unsigned>((warps2 * 32 + 255) / 256), 256, 0, s>>>(down, shared_down, idx, w, hbuf, out, T,
-                                                                                H, I, k, n_shared);
+                                                                                H, I, E, k, n_shared);
   return cudaGetLastError();
 }
 
@@ -1551,7 +1518,7 @@ extern "C" acm_status acm_expert_ffn_f32_noalloc(const float* x, int T, int hidd
     scratch = g_noalloc_ptr[dev];
   }
   const cudaError_t err = acm::launch_ffn_f32(x, w_gate_up, w_down, nullptr, nullptr, 0, idx, w, scratch, out, T, hidden,
-                                              inter, top_k, static_cast<cudaStream_t>(stream));
+                                              inter, n_experts, top_k, static_cast<cudaStream_t>(stream));
   return err == cudaSuccess ? ACM_OK : ACM_ERR_CUDA;
 }
 #endif   // !ACM_FFN_MX

@@ -14,7 +14,7 @@
 namespace acm {
 namespace {
 
-__device__ __forceinline__ long long time_ns() {     // one clock for every SM (debug stamps)
+__device__ __forceinline__ long long time_ns() {     // one clock for every SM (the stamps of acm_stage_timing)
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return static_cast<long long>(t);
@@ -156,25 +156,12 @@ struct ElemTraits<float> {
 };
 template <>
 struct ElemTraits<__nv_bfloat16> {
-#ifndef ACM_ROUTER_BF16_EPT
-#define ACM_ROUTER_BF16_EPT 4
-#endif
-  static constexpr int EPT = ACM_ROUTER_BF16_EPT;
-#if ACM_ROUTER_BF16_EPT == 8
-  using Vec = uint4;
-  __device__ static void unpack(const uint4& v, float* f) {
-    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
-    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
-    f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xffff0000u);
-    f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xffff0000u);
-  }
-#else
+  static constexpr int EPT = 4;
   using Vec = uint2;        // 8-byte loads, 8 threads per output: twice the warps to hide latency with
   __device__ static void unpack(const uint2& v, float* f) {
     f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
     f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
   }
-#endif
 };
 
 // ---- bulk asynchronous copies (global -> shared) completing on an mbarrier ----
@@ -218,8 +205,6 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
   const int tid = threadIdx.x;
   const int e0 = blockIdx.x * kRE, t0 = blockIdx.y * kRT;
   griddep_launch_dependents();
-  if (dbg && tid == 0) atomicMax(reinterpret_cast<unsigned long long*>(dbg + 17), static_cast<unsigned long long>(time_ns()));
-  if (dbg && tid == 0 && blockIdx.x == 0 && blockIdx.y == 0) dbg[16] = time_ns();
 
   // Staging: the 4 x-rows and 8 router rows of this tile, in n_chunks pieces along h.  One thread
   // per row issues its pieces as bulk copies; piece c of all rows completes on barrier c.  The
@@ -311,7 +296,6 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
     logits[static_cast<size_t>(t) * E + e] = z;
     if (!isfinite(z)) raise_status(status, ACM_ERR_NONFINITE);
   }
-  if (dbg && tid == 0) atomicMax(reinterpret_cast<unsigned long long*>(dbg + 14), static_cast<unsigned long long>(time_ns()));
   // The CTA that completes a tile of nodes last (all expert tiles written) finishes those nodes:
   // softmax and natural top-k, one warp per node -- spread over as many SMs as there are node tiles.
   if (tile_done) {
@@ -349,7 +333,6 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
           }
         }
       }
-      if (dbg && tid == 0) atomicMax(reinterpret_cast<unsigned long long*>(dbg + 15), static_cast<unsigned long long>(time_ns()));
     }
   }
 }
@@ -404,11 +387,9 @@ __device__ float sel_tree_sum_128(float* tree, float mine) {
 // r comes straight from global memory (every load is issued before the first wait); the natural
 // top-k sets come as bit masks from `natmask_g` ([T][4], written by the router kernel) or, if that
 // is null, are built here from a.nat_idx.  Global results are written only if `write_out`.
-#define ACM_ST(slot) do { if (a.dbg && write_out && threadIdx.x == 0) a.dbg[slot] = time_ns(); } while (0)
 __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, int k, const uint32_t* natmask_g,
                              bool write_out, uint32_t* publish_words = nullptr, uint32_t publish_tag = 0) {
   const int tid = threadIdx.x;
-  ACM_ST(5);
   const int lane = tid & 31, warp = tid >> 5;
   const bool live = tid < E;
   // small loads first (they gate the first barrier), then the 64 probabilities of this expert's column
@@ -450,7 +431,6 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
     }
     sm.A[tid] = A;
   }
-  ACM_ST(6);
 
   // votes v_e and demand u_e (nodes ascending, fused multiply-add)
   int votes = 0;
@@ -482,7 +462,6 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   }
   if (!live) { votes = 0; u = 0.0f; }
   if (a.prm.demand == ACM_DEMAND_VOTES) u = static_cast<float>(votes);
-  ACM_ST(7);
   sm.votes[tid] = votes;
   sm.u[tid] = u;
   sel_sync();                       // sm.A
@@ -493,7 +472,6 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   const int n_positive = sel_count(in_R && u > 0.0f);
   const float upos = in_R ? fmaxf(u, 0.0f) : 0.0f;
   const float Z = sel_tree_sum_128(sm.tree, upos);
-  ACM_ST(8);
 
   const int floor_keep = max(0, k - nA);
   int n_er = 0, n_keep;
@@ -511,7 +489,6 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
     n_keep = floor_keep;
   }
   n_keep = min(n_keep, nR);
-  ACM_ST(9);
 
   // rank inside R by (u descending, index ascending): one 64-bit key per expert
   const unsigned long long mykey =
@@ -529,7 +506,6 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
     }
     in_S = rank < n_keep;
   }
-  ACM_ST(10);
   const unsigned s_word = __ballot_sync(0xffffffffu, in_S);
   if (lane == 0) sm.S[warp] = s_word;
   const int nS = sel_count(in_S);
@@ -537,7 +513,6 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   if (live && votes > 0 && !in_S) atomicAdd(&sm.scal[0], votes);   // a(S)
   sel_sync();
   const int aS = sm.scal[0];
-  ACM_ST(11);
 
   bool in_Sp = in_S;
   int m_star = 0;
@@ -574,7 +549,6 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   }
   if (a.prm.residency == 2 && a.resident) m_star = nS - nSp;
 
-  ACM_ST(12);
   if (write_out) {
     const int words = (E + 31) / 32;
     if (tid < words) {
@@ -792,7 +766,6 @@ k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uin
     }
     if (lane == 0 && ra.stats_out) { ra.stats_out->n_activated = n_act; ra.stats_out->n_staged = tot_stg; }
   }
-  if (ra.dbg && tid == 0) ra.dbg[4] = time_ns();
 }
 
 // Several verification blocks in one launch: CTA b owns block b (the rows bd.off[b] .. bd.off[b+1]-1 of
@@ -821,7 +794,6 @@ k_select_route_batch(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, Bat
   mine.count_out += b;
   if (mine.demand_out) mine.demand_out += static_cast<size_t>(b) * kMaxExperts;
   if (mine.stats_out) mine.stats_out += b;
-  mine.dbg = nullptr;
   if (tid < kSelThreads)
     stage_select(mine, sm, T, E, k, natmask_g + static_cast<size_t>(t_lo) * kMaskWords, true,
                  ra.sel_flag ? ra.sel_flag + 2 * kMaskWords * b : nullptr, static_cast<uint32_t>(ra.sel_epoch) & 0xffffu);

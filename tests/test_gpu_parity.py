@@ -455,18 +455,20 @@ def test_host_buffer_call_matches_the_device_call():
     ctx.close()
 
 
-@pytest.mark.parametrize("env", [{"ACM_NO_PDL": "1"}, {"ACM_NO_EARLY_START": "1"},
-                                 {"ACM_NO_PDL": "1", "ACM_NO_EARLY_START": "1"}])
-def test_launch_modes_agree_with_the_oracle(env, monkeypatch):
-    """The fused call has three launch modes (dependent launches + early start on the eligible set, dependent
-    launches only, plain stream order); each is read from the environment when a context is created and each
-    must give the oracle's sets, routes and outputs."""
-    for key, val in env.items():
-        monkeypatch.setenv(key, val)
+@pytest.mark.parametrize("level", [acm.OVERLAP_NONE, acm.OVERLAP_DEPENDENT, acm.OVERLAP_ELIGIBLE, acm.OVERLAP_ANCHORS])
+def test_overlap_levels_agree_with_the_oracle(level):
+    """The fused call's kernels overlap to a degree the caller chooses (plain stream order with a cooperative FFN
+    launch; dependent launches; early start on the eligible set; early start on the anchors): every level must give
+    the oracle's sets, routes and outputs, on every row, and switching levels on a live context must too."""
     cfg = wl.CONFIGS[3]
     ctx = _ctx(cfg, n_layers=2)
+    ctx.set_overlap(level)
     for layer in (0, 1):
-        _verify_layer(cfg, layer, ctx, layer, rows=[0, 7, 63])
+        _verify_layer(cfg, layer, ctx, layer)
+    ctx.set_overlap((level + 2) % 4)
+    _verify_layer(cfg, 1, ctx, 1)
+    with pytest.raises(acm.AcmError):
+        ctx.set_overlap(7)
     ctx.close()
 
 
