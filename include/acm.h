@@ -298,6 +298,16 @@ acm_status acm_h2d_bytes(acm_ctx* ctx, uint64_t* bytes_out /*host*/, int reset);
 acm_status acm_ffn_timing(acm_ctx* ctx, int enable, int capacity);
 acm_status acm_ffn_time_ms(acm_ctx* ctx, float* total_ms, int32_t* launches);
 
+/* Offload variant (Section 3.4): where a call's time goes on a layer with a static residency (acm_set_resident).
+ * acm_offload_timing(enable, capacity) starts (enable != 0) or stops recording CUDA events in up to `capacity`
+ * such calls; acm_offload_times synchronises them and returns sums over the recorded calls, ms_out [4] (host,
+ * milliseconds): [0] whole call on the device, from before its first kernel to after its last; [1] from there to
+ * the end of the FFN over the experts that were resident; [2] the host-to-device copies of the loaded experts
+ * (on the copy stream); [3] the stall: how long the copies went on after the resident part was done, i.e. the
+ * time the stream spent waiting for them -- [0] minus [3] is the call without its host-to-device wait. */
+acm_status acm_offload_timing(acm_ctx* ctx, int enable, int capacity);
+acm_status acm_offload_times(acm_ctx* ctx, double* ms_out /*host [4]*/, int32_t* calls /*host*/);
+
 /* Per-stage device times of the fused call, from time stamps the kernels themselves take (one global
  * nanosecond clock) -- the launch sequence, its overlaps included, stays as it is.  acm_stage_timing
  * switches the stamps on or off (it synchronises the device; on costs a few stores per CTA).

@@ -28,6 +28,7 @@ EXPORTS = [
     "acm_set_slot_pool", "acm_pool_stats", "acm_pool_plan",
     "acm_h2d_bytes", "acm_ffn_timing", "acm_ffn_time_ms", "acm_stage_timing", "acm_stage_times", "acm_launch_count", "acm_device_status", "acm_status_string",
     "acm_set_overlap", "acm_set_wait_limit", "acm_wait_report", "acm_inject_unpublished_wait",
+    "acm_offload_timing", "acm_offload_times",
     "acm_expert_ffn_f32_noalloc",
 ]
 NOALLOC_MAX_FLOATS = 1 << 20
@@ -111,6 +112,8 @@ def load_library():
     lib.acm_launch_count.argtypes = [c_void_p, POINTER(c_uint64)]
     lib.acm_device_status.argtypes = [c_void_p, c_void_p]
     lib.acm_set_overlap.argtypes = [c_void_p, c_int]
+    lib.acm_offload_timing.argtypes = [c_void_p, c_int, c_int]
+    lib.acm_offload_times.argtypes = [c_void_p, POINTER(ctypes.c_double), POINTER(c_int32)]
     lib.acm_set_wait_limit.argtypes = [c_void_p, c_uint64]
     lib.acm_wait_report.argtypes = [c_void_p, c_void_p, c_int, POINTER(c_int32)]
     lib.acm_inject_unpublished_wait.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p]
@@ -227,9 +230,18 @@ def expert_ffn_f32_noalloc(x, idx, w, gate_up, down, out, stream=None):
     """acm_expert_ffn_f32_noalloc: the fp32 expert FFN for callers that may not allocate device memory at
     call time.  Every tensor, `out` included, is the caller's; nothing is allocated here or in the library
     (its scratch is a fixed array in the library image, shared by all calls: do not overlap calls)."""
+    for name, t, dt in (("x", x, torch.float32), ("idx", idx, torch.int32), ("w", w, torch.float32),
+                        ("gate_up", gate_up, torch.float32), ("down", down, torch.float32), ("out", out, torch.float32)):
+        if t.dtype != dt:
+            raise TypeError(f"{name} must be {dt}, got {t.dtype}")
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError(f"{name} must be a contiguous CUDA tensor")
     T, H = x.shape
     E, _, I = down.shape
     k = idx.shape[1]
+    if tuple(gate_up.shape) != (E, 2 * I, H) or tuple(idx.shape) != (T, k) or tuple(w.shape) != (T, k) or \
+            tuple(out.shape) != (T, H):
+        raise ValueError("shapes: x [T,H], idx/w [T,k], gate_up [E,2I,H], down [E,H,I], out [T,H]")
     _check(load_library().acm_expert_ffn_f32_noalloc(_p(x), T, H, I, E, k, _p(idx), _p(w), _p(gate_up), _p(down),
                                                      _p(out), _stream(stream)), "acm_expert_ffn_f32_noalloc")
     return out
@@ -424,6 +436,16 @@ class Context:
         ms, n = c_float(0), c_int32(0)
         _check(self.lib.acm_ffn_time_ms(self.handle, byref(ms), byref(n)), "acm_ffn_time_ms")
         return ms.value, n.value
+
+    def offload_timing(self, enable, capacity=0):
+        _check(self.lib.acm_offload_timing(self.handle, int(bool(enable)), int(capacity)), "acm_offload_timing")
+
+    def offload_times(self) -> dict:
+        """Sums over the recorded calls (ms): whole, resident part, copies, stall; and the number of calls."""
+        ms = (ctypes.c_double * 4)()
+        n = c_int32(0)
+        _check(self.lib.acm_offload_times(self.handle, ms, byref(n)), "acm_offload_times")
+        return {"whole_ms": ms[0], "resident_ms": ms[1], "copy_ms": ms[2], "stall_ms": ms[3], "calls": n.value}
 
     def stage_timing(self, enable):
         _check(self.lib.acm_stage_timing(self.handle, int(bool(enable))), "acm_stage_timing")

@@ -156,6 +156,11 @@ struct acm_ctx {
   uint64_t launches = 0;
   unsigned long long* trace = nullptr;   // acm_stage_timing: per-CTA time stamps of the last FFN launch + the routing kernels' stamps
   bool mx_configured = false;
+  // offload timing (acm_offload_timing): five events per call on a layer with a static residency
+  bool off_timing = false;
+  std::vector<cudaEvent_t> off_ev;
+  std::vector<unsigned char> off_has_copies;   // per recorded call: did it load anything?
+  size_t off_calls = 0;
   // bounded device-side waits (acm_set_wait_limit, acm_wait_report)
   unsigned long long wait_limit_ns = 1000000000ull;
   int32_t* wait_diag = nullptr;          // [sm_count] per-CTA words of the FFN kernel
@@ -375,6 +380,22 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   return ACM_OK;
 }
 
+// The sequence number of a fused call: its low 16 bits tag the words its kernels publish for one another (0 is
+// never a valid tag).  The tags come round every 65535 calls, and a word that no call has rewritten since (a
+// later block's words after single-block calls) would then look current: when they come round, the words are
+// cleared, in stream order, before the call's first kernel.
+acm_status next_epoch(acm_ctx* c, cudaStream_t s, int32_t* epoch_out) {
+  int32_t e = ++c->epoch;
+  if (e <= 0) e = c->epoch = 0x10000;
+  if ((e & 0xffff) == 0) {
+    ACM_CUDA(cudaMemsetAsync(c->ws.sel_words, 0, 32 * kMaxEarlyBlocks, s));
+    ACM_CUDA(cudaMemsetAsync(c->ws.anc_words, 0, 32 * kMaxEarlyBlocks, s));
+    e = ++c->epoch;
+  }
+  *epoch_out = e;
+  return ACM_OK;
+}
+
 // what both offload variants need: the pinned report buffer, the copy stream and its events
 acm_status ensure_offload_common(acm_ctx* c) {
   if (c->host_stage_list) return ACM_OK;
@@ -532,6 +553,7 @@ acm_status acm_destroy(acm_ctx* c) {
   if (!c) return ACM_ERR_INVALID;
   cudaDeviceSynchronize();
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->off_ev) cudaEventDestroy(e);
   if (c->ev_lists) cudaEventDestroy(c->ev_lists);
   if (c->ev_copied) cudaEventDestroy(c->ev_copied);
   if (c->ev_stage_free) cudaEventDestroy(c->ev_stage_free);
@@ -735,14 +757,19 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   const bool early = !f32 && !L.has_resident && !eligible_mask_override && c->early_start;
   int32_t early_epoch = 0;
   if (early) {
-    early_epoch = ++c->epoch;            // its low 16 bits tag the published words; 0 is never a valid tag
-    if ((early_epoch & 0xffff) == 0) early_epoch = ++c->epoch;
-    if (early_epoch <= 0) early_epoch = c->epoch = 1;
+    st = next_epoch(c, s, &early_epoch);
+    if (st != ACM_OK) return st;
   }
   // ... and earlier still on the anchors (Eq. 5 with the default anchor, the root): the router kernel publishes
   // the root's natural top-k as soon as that row is done, the FFN kernel streams their gate/up tiles while
   // the selection runs.  They are in every eligible set the selection can return without a residency.
   const bool anchors_first = early && c->anchor_start && prm.use_anchors != 0;
+  // offload timing: events around the resident part, the copies and the loaded part of this call
+  cudaEvent_t* oev = nullptr;
+  if (c->off_timing && L.has_resident && !L.has_pool && 5 * (c->off_calls + 1) <= c->off_ev.size()) {
+    oev = c->off_ev.data() + 5 * c->off_calls;
+    ACM_CUDA(cudaEventRecord(oev[0], s));
+  }
   // stage 1 (also clears the output the FFN accumulates into and the FFN kernel's routing inputs)
   const bool need_probs = eligible_mask_override == nullptr;
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
@@ -791,6 +818,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
     ACM_CUDA(cudaEventRecord(c->ev_lists, s));
     st = run_ffn_list(c, L, x, T, 0, out, s, res_dev, stats_dev);
     if (st != ACM_OK) return st;
+    if (oev) ACM_CUDA(cudaEventRecord(oev[1], s));
     ACM_CUDA(cudaEventSynchronize(c->ev_lists));
     const int n_stage = c->host_stage_list[0];
     if (n_stage < 0 || n_stage > E) return ACM_ERR_CUDA;
@@ -871,6 +899,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
       }
     } else if (n_stage > 0) {
       if (c->stage_in_use) ACM_CUDA(cudaStreamWaitEvent(c->copy_stream, c->ev_stage_free, 0));
+      if (oev) ACM_CUDA(cudaEventRecord(oev[2], c->copy_stream));
       for (int i = 0; i < n_stage; ++i) {
         const int e = c->host_stage_list[1 + i];
         if (e < 0 || e >= E) return ACM_ERR_CUDA;
@@ -882,12 +911,18 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
                                  c->copy_stream));
         c->h2d_bytes += gu + dn;
       }
+      if (oev) ACM_CUDA(cudaEventRecord(oev[3], c->copy_stream));
       ACM_CUDA(cudaEventRecord(c->ev_copied, c->copy_stream));
       ACM_CUDA(cudaStreamWaitEvent(s, c->ev_copied, 0));
       st = run_ffn_list(c, L, x, T, 1, out, s, res_dev, nullptr);
       if (st != ACM_OK) return st;
       ACM_CUDA(cudaEventRecord(c->ev_stage_free, s));
       c->stage_in_use = true;
+    }
+    if (oev) {
+      ACM_CUDA(cudaEventRecord(oev[4], s));
+      c->off_has_copies[c->off_calls] = (!L.has_pool && n_stage > 0) ? 1 : 0;
+      c->off_calls += 1;
     }
   }
 
@@ -931,9 +966,8 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
   const bool early = n_blocks <= kMaxEarlyBlocks && c->early_start;
   int32_t early_epoch = 0;
   if (early) {
-    early_epoch = ++c->epoch;
-    if ((early_epoch & 0xffff) == 0) early_epoch = ++c->epoch;
-    if (early_epoch <= 0) early_epoch = c->epoch = 1;
+    st = next_epoch(c, s, &early_epoch);
+    if (st != ACM_OK) return st;
   }
   // ... and on the union of the blocks' anchors (each block's first row is its root) while the selections run
   const bool anchors_first = early && c->anchor_start && params->use_anchors != 0;
@@ -1229,6 +1263,42 @@ acm_status acm_ffn_time_ms(acm_ctx* c, float* total_ms, int32_t* launches) {
   return ACM_OK;
 }
 
+acm_status acm_offload_timing(acm_ctx* c, int enable, int capacity) {
+  if (!c || capacity < 0) return ACM_ERR_INVALID;
+  c->off_timing = enable != 0;
+  c->off_calls = 0;
+  while (c->off_timing && c->off_ev.size() < static_cast<size_t>(5) * capacity) {
+    cudaEvent_t e;
+    ACM_CUDA(cudaEventCreate(&e));
+    c->off_ev.push_back(e);
+  }
+  c->off_has_copies.assign(c->off_ev.size() / 5 + 1, 0);
+  return ACM_OK;
+}
+
+acm_status acm_offload_times(acm_ctx* c, double* ms_out, int32_t* calls) {
+  if (!c || !ms_out || !calls) return ACM_ERR_INVALID;
+  double total = 0.0, resident = 0.0, copies = 0.0, stall = 0.0;
+  for (size_t i = 0; i < c->off_calls; ++i) {
+    cudaEvent_t* e = c->off_ev.data() + 5 * i;
+    ACM_CUDA(cudaEventSynchronize(e[4]));
+    float ms = 0.f;
+    ACM_CUDA(cudaEventElapsedTime(&ms, e[0], e[4]));
+    total += ms;
+    ACM_CUDA(cudaEventElapsedTime(&ms, e[0], e[1]));
+    resident += ms;
+    if (c->off_has_copies[i]) {
+      ACM_CUDA(cudaEventElapsedTime(&ms, e[2], e[3]));
+      copies += ms;
+      ACM_CUDA(cudaEventElapsedTime(&ms, e[1], e[3]));      // negative: the copies were done before the resident part was
+      if (ms > 0.f) stall += ms;
+    }
+  }
+  ms_out[0] = total; ms_out[1] = resident; ms_out[2] = copies; ms_out[3] = stall;
+  *calls = static_cast<int32_t>(c->off_calls);
+  return ACM_OK;
+}
+
 acm_status acm_stage_timing(acm_ctx* c, int enable) {
   if (!c) return ACM_ERR_INVALID;
   ACM_CUDA(cudaDeviceSynchronize());
@@ -1311,9 +1381,9 @@ acm_status acm_inject_unpublished_wait(acm_ctx* c, int layer, const void* x, int
   if (c->desc.dtype != ACM_BF16 || L.has_resident) return ACM_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // a tag of its own, which no router or selection kernel is ever launched with
-  int32_t epoch = ++c->epoch;
-  if ((epoch & 0xffff) == 0) epoch = ++c->epoch;
-  if (epoch <= 0) epoch = c->epoch = 1;
+  int32_t epoch = 0;
+  st = next_epoch(c, s, &epoch);
+  if (st != ACM_OK) return st;
   ACM_CUDA(cudaMemsetAsync(out, 0, sizeof(float) * static_cast<size_t>(T) * c->desc.hidden, s));
   return run_ffn_list(c, L, x, T, 0, out, s, nullptr, nullptr, false, epoch);
 }

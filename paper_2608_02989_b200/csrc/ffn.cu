@@ -214,6 +214,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// Has a wait that began at t0 outlasted the limit?  The clock is read twice before the answer is yes: a single
+// reading that lies outside [t0, t0 + limit] (a value caught while the counter's halves roll over would) must
+// not end a healthy launch.
+__device__ __forceinline__ bool limit_passed(unsigned long long t0, unsigned long long limit_ns) {
+  const long long d1 = static_cast<long long>(global_timer() - t0);
+  if (d1 >= 0 && static_cast<unsigned long long>(d1) <= limit_ns) return false;
+  const long long d2 = static_cast<long long>(global_timer() - t0);
+  return d2 < 0 ? false : static_cast<unsigned long long>(d2) > limit_ns;
+}
 __device__ __noinline__ void give_up(GiveUp* g, int site) {
   if (atomicExch(const_cast<int*>(&g->flag), 1) == 0 && g->where) *g->where = g->tag | site;
   atomicCAS(g->status, 0, static_cast<int32_t>(ACM_ERR_TIMEOUT));
@@ -229,7 +238,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, GiveU
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (g->flag) return false;
-    if (global_timer() - t0 > g->limit_ns) {
+    if (limit_passed(t0, g->limit_ns)) {
       give_up(g, site);
       return false;
     }
@@ -261,7 +270,7 @@ __device__ bool flag_wait_ge(const int32_t* p, int target, GiveUp* g, int site) 
       __nanosleep(64);
     }
     if (g->flag) return false;
-    if (global_timer() - t0 > g->limit_ns) {
+    if (limit_passed(t0, g->limit_ns)) {
       give_up(g, site);
       return false;
     }
@@ -275,7 +284,7 @@ __device__ __forceinline__ uint32_t poll_tagged_word(const uint32_t* word, uint3
   do {
     asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(word) : "memory");
     seen = (v >> 16) == tag;
-  } while (!seen && global_timer() - t0 < limit_ns);
+  } while (!seen && !limit_passed(t0, limit_ns));
   return seen ? (v & 0xffffu) : 0u;
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
@@ -1037,7 +1046,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
                 const unsigned long long t0 = global_timer();
                 while (bars->armed <= hidx) {
                   if (quit->flag) { good = false; break; }
-                  if (global_timer() - t0 > p.wait_limit_ns) {
+                  if (limit_passed(t0, p.wait_limit_ns)) {
                     give_up(quit, kSiteStageArmed);
                     good = false;
                     break;

@@ -211,7 +211,7 @@ def test_expert_ffn_against_oracle(T, H, I, E, k, ns):
     _set_weights(ctx, w)
     out = ctx.expert_ffn(0, x, torch.tensor(idx, device=DEV), torch.tensor(wt, device=DEV))
     assert ctx.device_status() == acm.OK
-    rows = np.arange(T) if T * E <= 2048 else np.array(sorted(rng.choice(T, 12, replace=False)))
+    rows = np.arange(T)
     ref = oracle.expert_ffn(_take(x, rows), idx[rows], wt[rows].astype(np.float64), w["gate_up"], w["down"],
                             w["shared_gate_up"], w["shared_down"])
     _ffn_check(_take(out, rows), ref, f"ffn {T}x{H}x{I}")
@@ -281,15 +281,14 @@ def test_config1_toy_fp32_end_to_end():
 @pytest.mark.parametrize("c", [2, 3, 4])
 def test_full_size_configs_end_to_end(c):
     """Full layer shapes of the OLMoE-, Qwen3-30B-A3B- and DeepSeek-V2-Lite-shaped configurations:
-    sets, routes and weights on every node; FFN outputs on sampled nodes the oracle computes one by one."""
+    sets, routes and weights on every node; FFN outputs on every node (all accumulator columns)."""
     cfg = wl.CONFIGS[c]
     ctx = _ctx(cfg, n_layers=2)
-    sample = [0, 1, cfg.n_nodes // 2, cfg.n_nodes - 1]
     sizes = []
     for layer in (0, cfg.n_layers - 1):
-        st, _ = _verify_layer(cfg, layer, ctx, layer % 2, rows=sample)
+        st, _ = _verify_layer(cfg, layer, ctx, layer % 2)
         sizes.append(st["n_eligible_pruned"])
-    _verify_layer(cfg, 1, ctx, 1, rows=sample, natural=True)
+    _verify_layer(cfg, 1, ctx, 1, natural=True)
     if c == 3:
         assert all(10 <= s <= 45 for s in sizes), sizes     # skewed routing: the set is far below E
     ctx.close()
@@ -352,13 +351,16 @@ def test_deterministic_selection_and_routing_across_runs():
     ctx.close()
 
 
-@pytest.mark.parametrize("mode", [1, 2])
-def test_offload_variant_residency_and_on_demand_loads(mode):
-    """Config-5 mechanism on a reduced layer: a seeded 40 % of the experts is GPU-resident, eligibility is
-    conditioned on residency (Eq. 7, or the strict resident-plus-anchors variant), and activated non-resident
-    experts are copied from pinned host memory.  The device copies of non-resident experts are poisoned with NaN:
-    a correct result proves they were never read."""
-    cfg = wl.scaled(wl.CONFIGS[5], hidden=512, inter=256, n_experts=32, top_k=4, n_nodes=32, max_depth=5, n_layers=1)
+@pytest.mark.parametrize("mode,full_shape", [(1, False), (2, False), (1, True), (2, True)])
+def test_offload_variant_residency_and_on_demand_loads(mode, full_shape):
+    """Config 5's mechanism, on a reduced layer and on the Qwen3-235B-A22B-shaped layer itself (hidden 4096,
+    intermediate 1536, 128 experts, 64 nodes: 37.7 MB per expert copy, staging slots and the second work list at
+    full extent): a seeded 40 % of the experts is GPU-resident, eligibility is conditioned on residency (Eq. 7, or the
+    strict resident-plus-anchors variant), and activated non-resident experts are copied from pinned host memory.
+    The device copies of non-resident experts are poisoned with NaN: a correct result proves they were never read.
+    Sets and routes bit for bit, every output row in tolerance, host-to-device bytes exact."""
+    cfg = wl.CONFIGS[5] if full_shape else \
+        wl.scaled(wl.CONFIGS[5], hidden=512, inter=256, n_experts=32, top_k=4, n_nodes=32, max_depth=5, n_layers=1)
     w, x, alpha = _block(cfg, 2)
     E = cfg.n_experts
     rmask = wl.resident_mask(cfg, 2)
@@ -406,10 +408,10 @@ def test_offload_variant_residency_and_on_demand_loads(mode):
 
 
 def test_config5_shape_one_layer():
-    """The Qwen3-235B-A22B-shaped layer at full size (4.8 GB of weights), restricted routing, all resident."""
+    """The Qwen3-235B-A22B-shaped layer at full size (4.8 GB of weights), restricted routing, all resident, every row."""
     cfg = wl.CONFIGS[5]
     ctx = _ctx(cfg)
-    st, _ = _verify_layer(cfg, 0, ctx, 0, rows=[0, 31, 63])
+    st, _ = _verify_layer(cfg, 0, ctx, 0)
     assert st["n_activated"] > cfg.top_k
     ctx.close()
 
@@ -499,9 +501,8 @@ def test_back_to_back_layers_without_host_synchronisation():
         np.testing.assert_array_equal(_u32(mask), ref["mask"])
         np.testing.assert_array_equal(idx.cpu().numpy(), ref["idx"])
         assert acm.stats_dict(stats)["n_activated"] == len(set(ref["idx"].ravel()) - {-1})
-        rows = [0, T - 1]
-        ffn = oracle.expert_ffn(_take(x, rows), ref["idx"][rows], ref["w"][rows], w["gate_up"], w["down"])
-        _ffn_check(_take(out, rows), ffn, f"call layer {layer} T {T}")
+        ffn = oracle.expert_ffn(x, ref["idx"], ref["w"], w["gate_up"], w["down"])
+        _ffn_check(out, ffn, f"call layer {layer} T {T}")
     ctx.close()
 
 
@@ -649,12 +650,11 @@ def test_multi_block_batch_equals_every_block_verified_alone(c, n_blocks, params
             assert st["n_activated"] == len(mine)
             union |= mine
         assert mask_to_set(_u32(act), cfg.n_experts) == union
-        rows = sorted({0, offsets[1] - 1, offsets[min(1, n_blocks - 1)], cfg.n_nodes // 2, cfg.n_nodes - 1})
         ref_idx = np.concatenate([r["idx"] for r in refs])
         ref_w = np.concatenate([r["w"] for r in refs])
-        ffn = oracle.expert_ffn(_take(x, rows), ref_idx[rows], ref_w[rows], w["gate_up"], w["down"],
-                                w["shared_gate_up"], w["shared_down"])
-        _ffn_check(_take(out, rows), ffn, f"C{c} batch of {n_blocks}")
+        if rep == 0:
+            ffn = oracle.expert_ffn(x, ref_idx, ref_w, w["gate_up"], w["down"], w["shared_gate_up"], w["shared_down"])
+        _ffn_check(out, ffn, f"C{c} batch of {n_blocks}")
     ctx.close()
 
 
@@ -746,9 +746,8 @@ def test_mxfp4_layer_equals_the_bf16_layer_with_the_dequantised_weights(shape):
         assert ctx.device_status() == acm.OK
         np.testing.assert_array_equal(idx.cpu().numpy(), ref_idx.cpu().numpy())
         np.testing.assert_array_equal(_u32(mask), _u32(ref_mask))
-        rows = sorted({0, 1, cfg.n_nodes // 2, cfg.n_nodes - 1})
-        ffn = oracle.expert_ffn(_take(x, rows), idx.cpu().numpy()[rows], wt.cpu().numpy()[rows], w["gate_up_deq"], w["down_deq"])
-        _ffn_check(_take(out, rows), ffn, "MXFP4 layer")
+        ffn = oracle.expert_ffn(x, idx.cpu().numpy(), wt.cpu().numpy(), w["gate_up_deq"], w["down_deq"])
+        _ffn_check(out, ffn, "MXFP4 layer")
         # same tiles, same MMAs, same order of additions inside a tile; split-K partial sums meet in L2 in any order
         rms = float(ref_out.double().pow(2).mean().sqrt())
         assert float((out - ref_out).abs().max()) <= 1e-3 * rms

@@ -203,3 +203,49 @@ def test_wait_that_runs_out_is_reported_and_the_context_recovers():
     check_good_call()
     assert set(ctx.wait_report()) == {0}
     ctx.close()
+
+
+def test_sequence_tags_coming_round_do_not_revive_old_words():
+    """The words the kernels publish for one another carry the call's sequence number in 16 bits.  A batch call
+    writes words for eight blocks; 65534 single-block calls later the tags come round, and a second batch call,
+    on other hidden states, gets the first one's tag again.  The old words of blocks 1..7 must not pass for
+    current ones: sets, routes and every output row against the oracle."""
+    import ctypes
+    cfg = wl.scaled(wl.CONFIGS[3], hidden=256, inter=64, n_experts=16, top_k=2, n_nodes=16, max_depth=1, n_layers=1)
+    w = wl.layer_weights(cfg, 0, DEV)
+    p = wl.commitment_table(cfg)
+    offsets = list(range(0, 17, 2))                       # eight blocks of two nodes
+    depths = [np.array([0, 1], dtype=np.int32)] * 8
+    ctx = acm.Context.for_config(cfg, n_layers=1)
+    ctx.set_layer_weights(0, w["w_router"], w["router_bias"], w["gate_up"], w["down"])
+    host_w = dict(w_router=_host_bits(w["w_router"]), router_bias=w["router_bias"].cpu().numpy(), gate_up=None, down=None)
+    ffn_w = (_host_bits(w["gate_up"]), _host_bits(w["down"]))
+
+    def batch_call(seed):
+        x = wl.hidden_states(cfg, seed, DEV)
+        alpha, refs = _reference(cfg, host_w, x, offsets, depths, p)
+        res = ctx.moe_verify_batch(0, x, offsets, torch.tensor(alpha, device=DEV), acm.SelectParams(), want=True)
+        assert ctx.device_status() == acm.OK
+        out, idx, wt, mask, act, stats = res
+        for b, ref in enumerate(refs):
+            np.testing.assert_array_equal(_u32(mask[b]), ref["mask"])
+            np.testing.assert_array_equal(idx[offsets[b]:offsets[b + 1]].cpu().numpy(), ref["idx"])
+        ffn = oracle.expert_ffn(x, np.concatenate([r["idx"] for r in refs]), np.concatenate([r["w"] for r in refs]), *ffn_w)
+        rms = float(np.sqrt(np.mean(ffn ** 2)))
+        assert float(np.abs(out.double().cpu().numpy() - ffn).max()) <= 2e-2 * rms
+        return [r["mask"].copy() for r in refs]
+
+    first = batch_call(1)
+    x1 = wl.hidden_states(cfg, 2, DEV)[:2].contiguous()
+    alpha1 = torch.tensor(oracle.node_weights(depths[0], p.numpy()), device=DEV)
+    out1 = torch.empty(2, cfg.hidden, dtype=torch.float32, device=DEV)
+    params = acm.SelectParams()
+    sp = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    args = (ctx.handle, 0, ctypes.c_void_p(x1.data_ptr()), 2, ctypes.c_void_p(alpha1.data_ptr()), ctypes.byref(params), None,
+            ctypes.c_void_p(out1.data_ptr()), None, None, None, None, sp)
+    for _ in range(65534):
+        assert ctx.lib.acm_moe_verify(*args) == 0
+    assert ctx.device_status() == acm.OK
+    second = batch_call(3)
+    assert any((a != b).any() for a, b in zip(first, second))       # (the two batches do have different sets)
+    ctx.close()

@@ -231,6 +231,75 @@ def test_fixed_budget_holds_total_size_with_anchors():
         assert set(nat[0]) <= mask_to_set(res["mask"], 16)
 
 
+# ------------------------------------------------------------------ anchors over several nodes (Eq. 5)
+def test_anchor_set_is_the_union_over_the_listed_nodes_hand_case():
+    # 3 nodes, 8 experts, k = 2.  Anchor nodes {0, 2}: A = K_0 u K_2 = {0, 1, 4, 5}.  The residual is what the other
+    # experts collect: node 1 alone chooses experts 2 and 3, so R's demand is u_2 = 1/2, u_3 = 1/4 and zero elsewhere
+    # (6, 7): q = (2/3, 1/3), exp(H) = 1.89 -> n_er = 2, S = A u {2, 3}.  Experts 4 and 5 collect the largest demand
+    # of all (node 2 has alpha 4), yet they must not take residual ranks: they are anchors, outside R.
+    r = np.zeros((3, 8), dtype=np.float32)
+    nat = np.int32([[0, 1], [2, 3], [4, 5]])
+    r[0, 0], r[0, 1] = 0.5, 0.25
+    r[1, 2], r[1, 3] = 0.5, 0.25
+    r[2, 4], r[2, 5] = 0.5, 0.25
+    alpha = np.float32([1.0, 1.0, 4.0])
+    res = oracle.select_eligible(r, nat, alpha, SelectParams(), anchor_nodes=np.int32([0, 2]))
+    assert res["stats"]["n_anchor"] == 4 and res["stats"]["n_er"] == 2
+    assert mask_to_set(res["mask"], 8) == {0, 1, 2, 3, 4, 5}
+    assert res["stats"]["residual_mass"] == 0.75
+    # the default (root only): A = {0, 1}; R now holds 2, 3, 4, 5 with demand (1/2, 1/4, 2, 1): q = (2/15, 1/15, 8/15,
+    # 4/15), exp(H) = 3.14 -> n_er = 4 and the same set results, but through a different count
+    root = oracle.select_eligible(r, nat, alpha, SelectParams())
+    assert root["stats"]["n_anchor"] == 2 and root["stats"]["n_er"] == 4
+    assert mask_to_set(root["mask"], 8) == {0, 1, 2, 3, 4, 5}
+    # a fixed budget tells the two apart: B = 4 keeps the four anchors and nothing else, or the root's two anchors
+    # plus the two residual experts with the largest demand (4 and 5)
+    four = oracle.select_eligible(r, nat, alpha, SelectParams(fixed_budget=4), anchor_nodes=np.int32([0, 2]))
+    assert mask_to_set(four["mask"], 8) == {0, 1, 4, 5}
+    four_root = oracle.select_eligible(r, nat, alpha, SelectParams(fixed_budget=4))
+    assert mask_to_set(four_root["mask"], 8) == {0, 1, 4, 5}
+    three = oracle.select_eligible(r, nat, np.float32([1.0, 4.0, 1.0]), SelectParams(fixed_budget=3), anchor_nodes=np.int32([0, 2]))
+    assert mask_to_set(three["mask"], 8) == {0, 1, 4, 5}       # the budget never cuts into the anchors: |S| >= |A|
+    # a listed node twice, or in another order, changes nothing; an empty list is not the default
+    again = oracle.select_eligible(r, nat, alpha, SelectParams(), anchor_nodes=np.int32([2, 0, 2]))
+    np.testing.assert_array_equal(again["mask"], res["mask"])
+
+
+def test_every_listed_anchor_node_keeps_its_natural_top_k():
+    rng = np.random.default_rng(515)
+    differs = 0
+    for trial in range(3000):
+        E = int(rng.integers(3, 10))
+        k = int(rng.integers(1, min(E, 3) + 1))
+        T = int(rng.integers(2, 7))
+        z, r = _softmax_rows(rng, T, E, scale=float(rng.uniform(0.2, 4.0)))
+        nat = _nat(z, k)
+        alpha = rng.uniform(0.05, 1.0, T).astype(np.float32)
+        nodes = sorted(rng.choice(T, size=int(rng.integers(1, T + 1)), replace=False).tolist())
+        res = oracle.select_eligible(r, nat, alpha, SelectParams(), anchor_nodes=np.int32(nodes))
+        S = mask_to_set(res["mask"], E)
+        A = set().union(*[set(nat[t]) for t in nodes])
+        st = res["stats"]
+        assert A <= S and st["n_anchor"] == len(A)                      # Eq. 5 for every listed node
+        assert len(S) == res["count"] >= max(len(A), k)
+        # the residual ranking sees only experts outside A: every kept non-anchor outranks every dropped one
+        u = res["demand"]
+        kept = [e for e in S if e not in A]
+        dropped = [e for e in range(E) if e not in S]
+        assert all((u[a], -a) > (u[b], -b) for a in kept for b in dropped)
+        assert len(kept) == (max(st["n_er"], k - len(A)) if st["residual_mass"] > 0.0 else max(0, k - len(A)))
+        # residual mass by its definition: positive demand outside A, summed in double (the oracle's tree sum is fp32)
+        want_z = sum(max(float(u[e]), 0.0) for e in range(E) if e not in A)
+        assert abs(st["residual_mass"] - want_z) <= 1e-6 * max(want_z, 1.0)
+        # routes of the listed nodes are their natural ones (their top-k is inside S)
+        idx, _ = oracle.route_restricted(z, res["mask"], k)
+        for t in nodes:
+            assert list(idx[t]) == list(nat[t])
+        root_only = oracle.select_eligible(r, nat, alpha, SelectParams())
+        differs += not np.array_equal(root_only["mask"], res["mask"])
+    assert differs > 100          # the list matters: it is not the default in disguise
+
+
 # ------------------------------------------------------------------ residency-aware pruning (Eq. 7)
 def _prune_brute(S, A, u, votes, resident, k, E):
     C = sorted((e for e in S if e not in resident), key=lambda e: (float(u[e]), e))

@@ -1,14 +1,16 @@
-"""The allocation-free fp32 expert FFN entry point against the context-based one.
+"""The allocation-free fp32 expert FFN entry point against the context-based one and against the oracle.
 
 Some callers cannot allocate device memory at the moment they call into this library (they run
 inside someone else's memory pool, or an implicit synchronisation from cudaMalloc would stall
 them), so one entry point keeps its scratch in a fixed array of the library image.  Called
-through the C ABI twice in a row, it must give what acm_expert_ffn gives, and it must refuse
-sizes beyond its fixed scratch.  Collected last on purpose."""
+through the C ABI twice in a row, it must give what acm_expert_ffn gives and what the CPU oracle
+computes, leave the device's free memory as it found it, treat expert ids outside the layer as
+empty slots, and refuse sizes beyond its fixed scratch.  Collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2608_02989_b200 import acm, workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -33,13 +35,58 @@ def test_noalloc_matches_context_entry_point_twice_in_a_row():
         ctx.set_layer_weights(0, w["w_router"], None, w["gate_up"], w["down"])
         want = ctx.expert_ffn(0, x, idx, wt)
         out = torch.full_like(want, float("nan"))          # caller-owned output, allocated before the call
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
         acm.expert_ffn_f32_noalloc(x, idx, wt, w["gate_up"], w["down"], out)
         torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before                   # nothing was allocated (or freed) on the device
         rms = float(want.double().pow(2).mean().sqrt())
         err = float((out.double() - want.double()).abs().max())
         assert torch.isfinite(out).all()
         assert err <= 2e-2 * rms, (call, err, rms)
+        # ... and against the CPU oracle (the two library entry points share their kernels)
+        ref = oracle.expert_ffn(x, idx.cpu().numpy(), wt.double().cpu().numpy(), w["gate_up"], w["down"])
+        rms_o = float(np.sqrt(np.mean(ref ** 2)))
+        assert float(np.abs(out.double().cpu().numpy() - ref).max()) <= 1e-4 * rms_o      # fp32 against fp64
         ctx.close()
+
+
+def test_noalloc_treats_expert_ids_outside_the_layer_as_empty_slots():
+    """An id >= n_experts must read no weights: it contributes nothing, exactly like -1."""
+    cfg, w, x, idx, wt = _inputs(5)
+    bad = idx.clone()
+    bad[0, 0] = cfg.n_experts            # first id past the layer
+    bad[3, 1] = 10 ** 6
+    hole = idx.clone()
+    hole[0, 0] = -1
+    hole[3, 1] = -1
+    out_bad = torch.full((cfg.n_nodes, cfg.hidden), float("nan"), device=DEV)
+    out_hole = torch.full_like(out_bad, float("nan"))
+    acm.expert_ffn_f32_noalloc(x, bad, wt, w["gate_up"], w["down"], out_bad)
+    acm.expert_ffn_f32_noalloc(x, hole, wt, w["gate_up"], w["down"], out_hole)
+    torch.cuda.synchronize()
+    assert torch.equal(out_bad, out_hole)
+    ref = oracle.expert_ffn(x, hole.cpu().numpy(), wt.double().cpu().numpy(), w["gate_up"], w["down"])
+    assert float(np.abs(out_bad.double().cpu().numpy() - ref).max()) <= 1e-4 * float(np.sqrt(np.mean(ref ** 2)))
+    # the context-based call on an fp32 layer bounds the ids the same way
+    ctx = acm.Context.for_config(cfg, n_layers=1)
+    ctx.set_layer_weights(0, w["w_router"], None, w["gate_up"], w["down"])
+    assert torch.equal(ctx.expert_ffn(0, x, bad, wt), out_hole)
+    ctx.close()
+
+
+def test_noalloc_wrapper_rejects_tensors_it_cannot_pass_on():
+    cfg, w, x, idx, wt = _inputs(6)
+    out = torch.empty(cfg.n_nodes, cfg.hidden, device=DEV)
+    with pytest.raises(TypeError):
+        acm.expert_ffn_f32_noalloc(x.double(), idx, wt, w["gate_up"], w["down"], out)
+    with pytest.raises(TypeError):
+        acm.expert_ffn_f32_noalloc(x, idx.long(), wt, w["gate_up"], w["down"], out)
+    with pytest.raises(ValueError):
+        acm.expert_ffn_f32_noalloc(x.t().contiguous().t(), idx, wt, w["gate_up"], w["down"], out)
+    with pytest.raises(ValueError):
+        acm.expert_ffn_f32_noalloc(x.cpu(), idx, wt, w["gate_up"], w["down"], out)
 
 
 def test_noalloc_rejects_sizes_beyond_its_scratch():
