@@ -351,6 +351,20 @@ acm_status acm_expert_ffn_f32_noalloc(const float* x, int T, int hidden, int int
                                       const float* w_gate_up, const float* w_down, float* out,
                                       acm_stream stream);
 
+/* The expert-FFN kernel's work plan, listed on the host (no GPU is touched): how one launch that streams
+ * n_experts_streamed experts of a bf16 layer (hidden, inter) on `grid` CTAs deals its weight tiles, for inspection
+ * and for tests of the plan's coverage.  n_anchor_first > 0 lists the plan of a launch that starts on that many
+ * anchor experts (Eq. 5) before the rest of the set is known (their tiles, one per CTA, are segment 0).
+ * pieces [capacity][8] (host) receives, in each
+ * CTA's execution order: CTA, segment, phase (1 = gate/up: 64 gate + 64 up rows x hidden; 2 = down: 128 output
+ * rows), for gate/up whether the tile is given whole (1) or cut along K (0) (down: 0), the tile (gate/up: slot *
+ * inter/64 + sub-tile; down: output tile), the piece's
+ * first and one-past-last K-chunk of 128 K (down: counted through the segment's expert group), and the cut
+ * segment's exchange buffer (gate/up) or the group's first expert slot (down).  ACM_ERR_NOMEM if capacity is too
+ * small (*n_pieces then tells how many there are). */
+acm_status acm_ffn_plan(int n_experts_streamed, int n_anchor_first, int hidden, int inter, int grid,
+                        int32_t* pieces /*host*/, int capacity, int32_t* n_pieces /*host*/, int32_t* n_segments /*host*/);
+
 /* How far the kernels of a fused call (acm_moe_verify, acm_moe_verify_batch, acm_moe_verify_host) overlap.
  * The stages of Section 3.1-3.4 form a chain, and the expert FFN needs only part of its result to start:
  *   ACM_OVERLAP_NONE       plain stream order.  The FFN kernel is a cooperative launch, so the driver itself

@@ -28,7 +28,7 @@ EXPORTS = [
     "acm_set_slot_pool", "acm_pool_stats", "acm_pool_plan",
     "acm_h2d_bytes", "acm_ffn_timing", "acm_ffn_time_ms", "acm_stage_timing", "acm_stage_times", "acm_launch_count", "acm_device_status", "acm_status_string",
     "acm_set_overlap", "acm_set_wait_limit", "acm_wait_report", "acm_inject_unpublished_wait",
-    "acm_offload_timing", "acm_offload_times",
+    "acm_offload_timing", "acm_offload_times", "acm_ffn_plan",
     "acm_expert_ffn_f32_noalloc",
 ]
 NOALLOC_MAX_FLOATS = 1 << 20
@@ -112,6 +112,7 @@ def load_library():
     lib.acm_launch_count.argtypes = [c_void_p, POINTER(c_uint64)]
     lib.acm_device_status.argtypes = [c_void_p, c_void_p]
     lib.acm_set_overlap.argtypes = [c_void_p, c_int]
+    lib.acm_ffn_plan.argtypes = [c_int] * 5 + [c_void_p, c_int, POINTER(c_int32), POINTER(c_int32)]
     lib.acm_offload_timing.argtypes = [c_void_p, c_int, c_int]
     lib.acm_offload_times.argtypes = [c_void_p, POINTER(ctypes.c_double), POINTER(c_int32)]
     lib.acm_set_wait_limit.argtypes = [c_void_p, c_uint64]
@@ -151,6 +152,22 @@ def node_weights(depth, p_table, beta=0.5, width_norm=True) -> torch.Tensor:
     _check(load_library().acm_node_weights(_p(depth), depth.numel(), _p(p_table), p_table.numel(),
                                            float(beta), int(bool(width_norm)), _p(alpha)), "acm_node_weights")
     return alpha
+
+
+def ffn_plan(n_experts_streamed, hidden, inter, grid, n_anchor_first=0):
+    """acm_ffn_plan on the host -> (pieces [n, 8] int32 numpy array, number of segments); see include/acm.h."""
+    import numpy as np
+    cap = 1 << 16
+    while True:
+        buf = np.zeros((cap, 8), dtype=np.int32)
+        n, nseg = c_int32(0), c_int32(0)
+        rc = load_library().acm_ffn_plan(n_experts_streamed, n_anchor_first, hidden, inter, grid,
+                                         buf.ctypes.data_as(c_void_p), cap, byref(n), byref(nseg))
+        if rc == ERR_NOMEM:
+            cap = n.value
+            continue
+        _check(rc, "acm_ffn_plan")
+        return buf[: n.value], nseg.value
 
 
 def pool_plan(n_experts, slot_expert, last_use, tick, activated):

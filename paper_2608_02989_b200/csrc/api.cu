@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "acm_internal.h"
+#include "ffn_plan.h"
 
 using namespace acm;
 
@@ -1343,6 +1344,48 @@ acm_status acm_launch_count(acm_ctx* c, uint64_t* launches_out) {
   if (!c || !launches_out) return ACM_ERR_INVALID;
   *launches_out = c->launches;
   return ACM_OK;
+}
+
+acm_status acm_ffn_plan(int n_experts_streamed, int n_anchor_first, int hidden, int inter, int grid, int32_t* pieces,
+                        int capacity, int32_t* n_pieces, int32_t* n_segments) {
+  if (!pieces || !n_pieces || !n_segments || capacity < 0) return ACM_ERR_INVALID;
+  if (n_experts_streamed < 1 || n_experts_streamed > kMaxSlots || n_anchor_first < 0 || n_anchor_first > n_experts_streamed ||
+      hidden < 128 || hidden % 128 != 0 || inter < 64 || inter % 64 != 0 || grid < 1 || grid > 1024)
+    return ACM_ERR_INVALID;
+  using namespace acm::plan;
+  const int tpe = inter / 64, kc1 = hidden / 128, kpe = (tpe + 1) / 2, h_tiles = hidden / 128;
+  if (n_anchor_first * tpe > grid) return ACM_ERR_INVALID;      // the pre-segment gives a CTA at most one tile
+  const FastDiv d_grid = make_fastdiv(grid), d_kc1 = make_fastdiv(kc1), d_tpe = make_fastdiv(tpe);
+  int n = 0, n_seg = 0;
+  for (int cta = 0; cta < grid; ++cta) {
+    Plan pl = {};
+    int base = 0;
+    if (n_anchor_first > 0) {
+      const Segment sg0 = Segment{1, 1, 0, n_anchor_first * tpe, 0, 0, 0, d_kc1, 0};
+      pl.seg[0] = sg0;
+      pl.range[0] = make_range(sg0, cta, d_grid, h_tiles);
+      base = 1;
+    }
+    for (int lane = 3; lane >= 0; --lane)
+      plan_lane(pl, lane, cta, n_experts_streamed, tpe, grid, d_kc1, kpe, d_grid, d_tpe, h_tiles, n_anchor_first, base);
+    n_seg = pl.n_seg;
+    for (int si = 0; si < pl.n_seg; ++si) {
+      const Segment& sg = pl.seg[si];
+      Sched sc(pl.range[si]);
+      int t, k0, k1;
+      while (sc.next(t, k0, k1)) {
+        if (n < capacity) {
+          int32_t* q = pieces + static_cast<size_t>(8) * n;
+          q[0] = cta; q[1] = si; q[2] = sg.phase; q[3] = sg.phase == 1 ? sg.whole : 0;
+          q[4] = sg.phase == 1 ? sg.t0 + t : t; q[5] = k0; q[6] = k1; q[7] = sg.phase == 1 ? sg.p1_index : sg.a0;
+        }
+        ++n;
+      }
+    }
+  }
+  *n_pieces = n;
+  *n_segments = n_seg;
+  return n <= capacity ? ACM_OK : ACM_ERR_NOMEM;
 }
 
 acm_status acm_set_overlap(acm_ctx* c, int level) {

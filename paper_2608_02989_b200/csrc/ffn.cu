@@ -31,6 +31,7 @@
 #include <mutex>
 
 #include "acm_internal.h"
+#include "ffn_plan.h"
 
 namespace acm {
 namespace {
@@ -64,68 +65,16 @@ constexpr int kMxCodeBytes = kTileM * 64;                // 128 rows x 128 four-
 constexpr int kFragBytes = kTileM * kMaxNodes * 4;       // contributor fragments pre-summed in shared memory
 constexpr int kFragFloats = kTileM * kMaxNodes;
 
-// Division by a launch constant through a precomputed 64-bit reciprocal (exact for n < 2^32): the
-// schedules below are walked by ONE thread per role, for which a hardware-less integer division is
-// a chain of dozens of dependent instructions.
-struct FastDiv {
-  unsigned long long M;   // ceil(2^64 / d) for d >= 2
-  unsigned d;
-};
-inline FastDiv make_fastdiv(unsigned d) {
-  FastDiv f;
-  f.d = d;
-  f.M = d > 1 ? 0xffffffffffffffffull / d + 1ull : 0ull;
-  return f;
-}
-// a divisor only known on the device (used a handful of times): M = 0 means "divide the plain way"
-__device__ __forceinline__ FastDiv plain_div(unsigned d) {
-  FastDiv f;
-  f.d = d;
-  f.M = 0ull;
-  return f;
-}
-__device__ __forceinline__ unsigned fdiv(unsigned n, const FastDiv& f) {
-  return f.M == 0ull ? (f.d == 1 ? n : n / f.d) : static_cast<unsigned>(__umul64hi(static_cast<unsigned long long>(n), f.M));
-}
-
-// The stream of one launch is cut into up to four segments, executed in this order by every CTA.
-// A gate/up tile (64 gate + 64 up rows over the whole hidden dimension) needs the complete sum before
-// its activation can be formed, so wherever possible a tile is given whole to one CTA:
-//   with at least one tile per CTA:
-//     1. the n_tiles mod G tiles that do not fill a round, cut evenly over all CTAs (their
-//        cross-CTA fragment exchange then hides behind the next segment)
-//     2. whole tiles, one per CTA and round
-//     3. down projection of the experts that were complete before the last round
-//     4. down projection of the rest -- by then their activations have been stored
-//   with fewer tiles than CTAs: gate/up of the first half of the experts, gate/up of the second
-//   half (both cut evenly), then down of the first half, down of the second half.
-// Down-projection work is linear in K and is always cut evenly.
-struct Segment {
-  int phase;      // 1 = gate/up, 2 = down
-  int whole;      // gate/up only: 1 = whole tiles dealt round-robin, 0 = tiles cut evenly over the CTAs
-  int t0, nt;     // gate/up: first tile and number of tiles (tile = slot * tiles_per_expert + sub-tile)
-  int a0, a1;     // down: activated-expert slots [a0, a1)
-  int p1_index;   // gate/up: which fragment buffer a cut segment uses; down: expert group it waits for
-  FastDiv chunks; // K-chunks per tile: the per-tile constant for gate/up, (a1 - a0) * chunks per expert for down
-};
-// This CTA's share of one segment of the plan.  Cut segments: equal contiguous ranges of (tile,
-// K-chunk) units, CTA c owns [c*U/G, (c+1)*U/G); whole-tile segments: tiles c, c+G, c+2G, ...
-// The divisions are done once per launch, by four lanes in parallel (fill_ranges), and every role
-// then walks its share with additions only: each role is a single thread that runs this code alone.
-struct SegRange {
-  unsigned u, u_end;     // cut: the CTA's unit range; whole: first tile and tile count of the segment
-  int tile0, k00;        // cut: tile and chunk of unit u
-  int kc;                // chunks per tile
-  int stride;            // whole: the grid size (tile step); 0 for a cut segment
-  unsigned n_stages;     // pipeline stages this CTA runs in the segment
-};
-struct Plan {
-  Segment seg[5];      // [0] may be the anchors' pre-segment (see the kernel's early start), then up to four
-  SegRange range[5];   // this CTA's share of each segment
-  volatile int n_seg;
-  int n_pre;      // experts whose gate/up tiles the pre-segment covers (the first slots of the work list)
-  int a_split;    // experts [0, a_split) form group 0 (complete early), the rest group 1
-};
+using plan::FastDiv;
+using plan::make_fastdiv;
+using plan::fdiv;
+using plan::Segment;
+using plan::SegRange;
+using plan::Plan;
+using plan::Sched;
+using plan::make_range;
+using plan::cut_begin;
+using plan::plan_lane;
 
 // Every wait in this kernel is bounded.  What a role needs when one runs out lives in shared memory (GiveUp,
 // touched on slow paths only): the limit, where to raise the status, and this CTA's diagnostic word, which
@@ -412,31 +361,6 @@ __device__ __forceinline__ uint32_t umma_idesc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
 }
 
-struct Sched {
-  unsigned u, u_end;
-  int tile, k0n, kc, stride;
-  __device__ explicit Sched(const SegRange& r) : u(r.u), u_end(r.u_end), tile(r.tile0), k0n(r.k00), kc(r.kc), stride(r.stride) {}
-  __device__ bool next(int& t, int& k0, int& k1) {
-    if (stride > 0) {            // whole tiles: u counts tiles
-      if (u >= u_end) return false;
-      t = static_cast<int>(u);
-      k0 = 0;
-      k1 = kc;
-      u += static_cast<unsigned>(stride);
-      return true;
-    }
-    if (u >= u_end) return false;
-    t = tile;
-    k0 = k0n;
-    const int rem = static_cast<int>(u_end - u);
-    k1 = rem < kc - k0 ? k0 + rem : kc;
-    u += static_cast<unsigned>(k1 - k0);
-    ++tile;
-    k0n = 0;
-    return true;
-  }
-};
-
 // Optional time stamps (acm_stage_timing): per CTA, slot 0 = the roles start, 10 / 11 = its last gate/up / down tile is done.
 #define ACM_STAMP(slot) do { if (p.trace) p.trace[static_cast<size_t>(blockIdx.x) * 32 + (slot)] = global_timer(); } while (0)
 
@@ -475,77 +399,8 @@ __device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMa
   return src == kSrcRouted ? routed : src == kSrcShared ? shared : staged;
 }
 
-// The plan lives in shared memory (a private copy indexed at run time would live in local memory, whose
-// first touch costs every role a trip to DRAM at the start of the kernel).  It has at most four
-// segments; lane i of one warp works out the i-th one by itself -- the four candidates in order, each
-// present or not -- and its own range in it, so nothing waits for a serial pass.
-__device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act, int tpe, int grid,
-                                          const FastDiv& d_kc1, int kpe, const FastDiv& d_grid, const FastDiv& d_tpe,
-                                          int h_tiles, int n_pre = 0, int base = 0);
-// Range of segment `si` for CTA `cta` (see SegRange).  (tiles * chunks * grid fits 32 bits: launcher.)
-__device__ __forceinline__ SegRange make_range(const Segment& sg, int cta, const FastDiv& d_grid, int h_tiles) {
-  SegRange r;
-  r.kc = static_cast<int>(sg.chunks.d);
-  if (sg.phase == 1 && sg.whole) {
-    r.u = static_cast<unsigned>(cta);
-    r.u_end = static_cast<unsigned>(sg.nt);
-    r.tile0 = 0; r.k00 = 0;
-    r.stride = static_cast<int>(d_grid.d);
-    r.n_stages = cta < sg.nt ? fdiv(static_cast<unsigned>(sg.nt - cta) + d_grid.d - 1u, d_grid) * sg.chunks.d : 0u;
-    return r;
-  }
-  const unsigned tiles = sg.phase == 1 ? static_cast<unsigned>(sg.nt) : static_cast<unsigned>(h_tiles);
-  const unsigned total = tiles * sg.chunks.d;
-  r.u = fdiv(total * static_cast<unsigned>(cta), d_grid);
-  r.u_end = fdiv(total * static_cast<unsigned>(cta + 1), d_grid);
-  r.tile0 = static_cast<int>(fdiv(tiles * static_cast<unsigned>(cta), d_grid));   // = floor(u / chunks): floors nest
-  r.k00 = static_cast<int>(r.u - static_cast<unsigned>(r.tile0) * sg.chunks.d);
-  r.stride = 0;
-  r.n_stages = r.u_end - r.u;
-  return r;
-}
-
-// With a pre-segment (n_pre experts whose gate/up tiles are already being streamed as segment 0, base = 1) the
-// gate/up segments cover the other experts' tiles only; the down segments cover everyone, the pre-streamed experts
-// counting as complete early.
-__device__ __forceinline__ void plan_lane(Plan& pl, int lane, int cta, int n_act, int tpe, int grid,
-                                          const FastDiv& d_kc1, int kpe, const FastDiv& d_grid, const FastDiv& d_tpe,
-                                          int h_tiles, int n_pre, int base) {
-  const int t_pre = n_pre * tpe;
-  const int n_t = (n_act - n_pre) * tpe;
-  const int rounds = static_cast<int>(fdiv(static_cast<unsigned>(n_t), d_grid)), rem = n_t - rounds * grid;
-  // candidates in execution order: two gate/up segments, two down segments
-  Segment c0, c1, c2, c3;
-  bool h0, h1, h2, h3;
-  int a_split;
-  if (rounds == 0) {
-    const int n_rest = n_act - n_pre, nA = (n_rest + 1) / 2;
-    a_split = n_pre + nA;
-    c0 = Segment{1, 0, t_pre, nA * tpe, 0, 0, 0, d_kc1};                      h0 = nA > 0;
-    c1 = Segment{1, 0, t_pre + nA * tpe, (n_rest - nA) * tpe, 0, 0, 1, d_kc1};   h1 = n_rest > nA;
-  } else {
-    a_split = n_pre + static_cast<int>(fdiv(static_cast<unsigned>(rem + (rounds - 1) * grid), d_tpe));
-    c0 = Segment{1, 0, t_pre, rem, 0, 0, 0, d_kc1};                           h0 = rem > 0;
-    c1 = Segment{1, 1, t_pre + rem, rounds * grid, 0, 0, 1, d_kc1};           h1 = true;
-  }
-  c2 = Segment{2, 0, 0, 0, 0, a_split, 0, plain_div(static_cast<unsigned>(a_split * kpe))};                 h2 = a_split > 0;
-  c3 = Segment{2, 0, 0, 0, a_split, n_act, 1, plain_div(static_cast<unsigned>((n_act - a_split) * kpe))};   h3 = n_act > a_split;
-  const int i0 = 0, i1 = i0 + h0, i2 = i1 + h1, i3 = i2 + h2, n = i3 + h3;
-  Segment mine = c0;
-  bool have = false;
-  if (h0 && i0 == lane) { mine = c0; have = true; }
-  if (h1 && i1 == lane) { mine = c1; have = true; }
-  if (h2 && i2 == lane) { mine = c2; have = true; }
-  if (h3 && i3 == lane) { mine = c3; have = true; }
-  if (have) {
-    pl.seg[base + lane] = mine;
-    pl.range[base + lane] = make_range(mine, cta, d_grid, h_tiles);
-  }
-  if (lane == 0) pl.a_split = a_split;
-  __syncwarp(0xfu);            // (called by lanes 0..3: the segments are in place before their count is)
-  if (lane == 0) pl.n_seg = base + n;
-}
-
+// The plan (ffn_plan.h) lives in shared memory: a private copy indexed at run time would live in local memory,
+// whose first touch costs every role a trip to DRAM at the start of the kernel.
 #if ACM_FFN_MX
 #define ACM_FFN_KERNEL k_ffn_mxfp4
 #else
@@ -625,7 +480,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   // whole tile per CTA, and the roles start on it at once; the helper warp meanwhile waits for the eligible
   // set, completes the work list (the pre-streamed experts keep the first slots) and the plan, and opens
   // `plan_ready`, which every other role passes before its second segment.
-  constexpr bool pre = kPre;
+  const bool pre = kPre && p.anc_flag != nullptr && p.sel_flag != nullptr;
   if (pre || early) {
     // Eight tagged words per block (16 mask bits under the 16-bit tag of this call; a batch has eight per block
     // and takes their union), each polled by its own thread of warps 2 and 3 -- four blocks per warp -- which have
@@ -697,7 +552,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   const uint32_t b_bytes = kAtoms * b_atom_bytes;
   if (pre) {
     if (threadIdx.x == kThreads - 32) {            // segment 0: the pre-streamed experts' tiles, one whole tile per CTA
-      Segment sg0 = Segment{1, 1, 0, n_pre * tpe, 0, 0, 0, p.d_kc1};
+      Segment sg0 = Segment{1, 1, 0, n_pre * tpe, 0, 0, 0, p.d_kc1, 0};
       bars->plan.seg[0] = sg0;
       bars->plan.range[0] = make_range(sg0, cta, p.d_grid, h_tiles);
       bars->plan.n_pre = n_pre;
@@ -735,7 +590,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   // plan_ready); n_seg is read from shared memory every time.
   const int n_seg_fixed = bars->plan.n_seg;
   auto have_seg = [&](int si, bool wait_for_plan) -> bool {
-    if constexpr (kPre) {
+    if (pre) {
       if (si == 1 && wait_for_plan && !mbar_wait(smem_u32(&bars->plan_ready), 0u, quit, kSitePlanReady)) return false;
       return si < bars->plan.n_seg;
     } else {
@@ -969,8 +824,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
         hidx += bars->plan.range[si].n_stages;
         hs = hidx % kStages;
         if (sg.whole) continue;          // whole tiles: nothing to exchange
-        const unsigned U1 = static_cast<unsigned>(sg.nt) * kc1;
-        const unsigned ub = fdiv(U1 * cta, p.d_grid), ue = fdiv(U1 * (cta + 1), p.d_grid);
+        const unsigned ub = cut_begin(sg, cta, p.d_grid), ue = cut_begin(sg, cta + 1, p.d_grid);
         if (ue <= ub) continue;
         const unsigned last_tile = fdiv(ue - 1, p.d_kc1);
         const unsigned tile_end = (last_tile + 1) * kc1;
@@ -985,7 +839,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
         const int n_el = p.n_pad * kTileM;
         int n_contrib = 0;
         for (int c2 = cta + 1; c2 < G; ++c2) {
-          const unsigned b2 = fdiv(U1 * c2, p.d_grid), e2 = fdiv(U1 * (c2 + 1), p.d_grid);
+          const unsigned b2 = cut_begin(sg, c2, p.d_grid), e2 = cut_begin(sg, c2 + 1, p.d_grid);
           if (b2 >= tile_end) break;
           if (e2 > b2) ++n_contrib;
         }
@@ -1086,10 +940,9 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
             // All CTAs that hold a tail part of this tile add into ONE global buffer, that of the CTA
             // which owns the tile's first chunks and will finish it.  The buffers are zero between
             // launches (the finishing CTA clears its own after reading), so nobody waits for anybody.
-            const unsigned U1 = static_cast<unsigned>(sg.nt) * kc1;            // (fits 32 bits: see the launcher)
             const unsigned tile_begin = static_cast<unsigned>(tile) * kc1;
             int c_head = cta - 1;
-            while (c_head > 0 && fdiv(U1 * c_head, p.d_grid) > tile_begin) --c_head;       // owner of the tile's first chunk
+            while (c_head > 0 && cut_begin(sg, c_head, p.d_grid) > tile_begin) --c_head;   // owner of the tile's first chunk
             asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
                          ::"l"(frag + static_cast<size_t>(c_head) * kFragFloats), "r"(smem_u32(ostage)), "r"(bytes) : "memory");
             bulk_commit();
@@ -1463,8 +1316,7 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   }
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelExC(&cfg, a.anc_flag && a.sel_flag ? reinterpret_cast<const void*>(ACM_FFN_KERNEL<true>)
-                                                            : reinterpret_cast<const void*>(ACM_FFN_KERNEL<false>), args);
+  return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(ACM_FFN_KERNEL<true>), args);
 }
 
 #if !ACM_FFN_MX
