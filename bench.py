@@ -27,7 +27,7 @@ ROOT = Path(__file__).resolve().parent
 if str(ROOT) not in sys.path:
     sys.path.insert(0, str(ROOT))
 
-DRAM_BYTES_PER_ACTIVATED_EXPERT = {3: (271304192 + 197928448 + 197003776) / 68.0}   # config -> bytes
+DRAM_BYTES_PER_ACTIVATED_EXPERT = {3: (273440512 + 193336832 + 193765376) / 68.0}   # config -> bytes (ncu, profiles/)
 METRIC = "verify_blocks_per_s_per_moe_layer"
 UNIT = "layer-blocks/s"
 
@@ -54,6 +54,11 @@ def parse_args():
     ap.add_argument("--zipf", action="store_true",
                     help="supplementary: give the configuration the Zipf(1.1) router bias that C3 has (skewed expert "
                          "popularity), e.g. --config 5 --zipf")
+    ap.add_argument("--overlap", type=int, default=3, choices=[0, 1, 2, 3],
+                    help="acm_set_overlap level: 0 plain stream order (cooperative FFN launch), 1 dependent launches, "
+                         "2 + FFN start on the eligible set, 3 + FFN start on the anchors (default)")
+    ap.add_argument("--bracket-every", type=int, default=11,
+                    help="bracket every n-th FFN launch with events for the roofline figure (0: none, the pure pipeline)")
     ap.add_argument("--all-resident", action="store_true",
                     help="config 5 only: every expert on the GPU (no offloading) instead of the configured 40 % residency")
     ap.add_argument("--batch", type=int, default=0,
@@ -372,6 +377,7 @@ def run_acm(args, world, rank, local):
     T, H, E, k = cfg.n_nodes, cfg.hidden, cfg.n_experts, cfg.top_k
 
     ctx = acm.Context.for_config(cfg, n_layers=L_phys)
+    ctx.set_overlap(args.overlap)
     keep = []
     for l in range(L_phys):
         if args.mxfp4:
@@ -426,9 +432,10 @@ def run_acm(args, world, rank, local):
     # measures).  The period is coprime with the layer count: over the steps every layer is sampled.
     period = 1
     if not resident:
-        period = 11
+        period = max(args.bracket_every, 1)
         while math.gcd(period, L) != 1:
             period += 1
+    bracket = args.bracket_every > 0
 
     def sampled_layers(steps):
         return np.arange(0, steps * L, period) % L
@@ -437,7 +444,7 @@ def run_acm(args, world, rank, local):
         for _ in range(warmup):
             step(calls)
         barrier()
-        if with_roofline:
+        if with_roofline and bracket:
             ctx.ffn_timing(period, steps * L * 2)
         n0 = ctx.launch_count()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -448,7 +455,7 @@ def run_acm(args, world, rank, local):
         barrier()
         ms = e0.elapsed_time(e1)
         launches = ctx.launch_count() - n0
-        ffn_ms, ffn_n = (ctx.ffn_time_ms() if with_roofline else (0.0, 0))
+        ffn_ms, ffn_n = (ctx.ffn_time_ms() if with_roofline and bracket else (0.0, 0))
         ctx.ffn_timing(False)
         if world > 1:
             ms, _ = aggregate_over_ranks(ms, float(L * steps), dist, dev)
@@ -556,14 +563,17 @@ def run_acm(args, world, rank, local):
                    "n_nodes": T, "layers": L, "physical_layers": L_phys,
                    "l2": f"inputs larger than L2: {L_phys} distinct layers, "
                          f"{alg_per_launch * L_phys / 1e9:.1f} GB of expert weights streamed per step",
+                   "overlap": args.overlap,
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "us_per_layer": 1e3 * ms / (args.steps * L),
         "mean_eligible": float(st[:, 3].mean()), "mean_activated": float(n_act.mean()),
         "mean_natural_union": float(st[:, 5].mean()),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": (achieved / peak) if achieved else None, "traffic": traffic, "peak_kind": peak_kind,
+                     "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+                     "traffic_kind": "scaled from the ncu capture in profiles/k_ffn_bf16_c3_layer.txt by this run's activated experts" if traffic else None,
+                     "peak_kind": peak_kind,
                      "kernel": "k_ffn_mxfp4" if args.mxfp4 else "k_ffn_bf16", "us_per_launch": ffn_us, "launches_timed": ffn_n,
-                     "timed_every": period,
+                     "timed_every": period if bracket else None,
                      "algorithmic_bytes_per_launch": alg_per_launch,
                      # context, not the headline: the same kernel inside the live pipeline (in-kernel stamps from its
                      # first role starting to its last tile; its set-up overlaps the kernels before it there)

@@ -406,9 +406,8 @@ __device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMa
 #else
 #define ACM_FFN_KERNEL k_ffn_bf16
 #endif
-// kPre: the variant that starts on the anchors' pre-segment (compiled apart, so that the plain variant's code is
-// exactly what it is without it)
-template <bool kPre>
+// One kernel for both starts (on the anchors' pre-segment, or with the whole work list at hand): a launch bracketed
+// by events then runs the same code as the launches around it, which keeps its instructions warm in the caches.
 __global__ void __launch_bounds__(kThreads, 1)
 ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtensorMap x_map,
            const __grid_constant__ CUtensorMap h_map, const __grid_constant__ CUtensorMap hs_map,
@@ -480,7 +479,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   // whole tile per CTA, and the roles start on it at once; the helper warp meanwhile waits for the eligible
   // set, completes the work list (the pre-streamed experts keep the first slots) and the plan, and opens
   // `plan_ready`, which every other role passes before its second segment.
-  const bool pre = kPre && p.anc_flag != nullptr && p.sel_flag != nullptr;
+  const bool pre = p.anc_flag != nullptr && p.sel_flag != nullptr;
   if (pre || early) {
     // Eight tagged words per block (16 mask bits under the 16-bit tag of this call; a batch has eight per block
     // and takes their union), each polled by its own thread of warps 2 and 3 -- four blocks per warp -- which have
@@ -1250,9 +1249,7 @@ __global__ void k_ffn_f32_down(const float* __restrict__ down, const float* __re
 
 #if ACM_FFN_MX
 cudaError_t ffn_mx_configure() {
-  cudaError_t err = cudaFuncSetAttribute(ACM_FFN_KERNEL<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
-  if (err != cudaSuccess) return err;
-  return cudaFuncSetAttribute(ACM_FFN_KERNEL<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  return cudaFuncSetAttribute(ACM_FFN_KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
 }
 cudaError_t launch_ffn_mxfp4(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
                              const CUtensorMap& h_map, const CUtensorMap& hs_map, cudaStream_t s) {
@@ -1260,9 +1257,7 @@ cudaError_t launch_ffn_mxfp4(const FfnLaunch& L, const FfnMaps& maps, const CUte
 size_t ffn_smem_bytes() { return kSmemBytes; }
 
 cudaError_t ffn_configure() {
-  cudaError_t err = cudaFuncSetAttribute(ACM_FFN_KERNEL<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
-  if (err != cudaSuccess) return err;
-  return cudaFuncSetAttribute(ACM_FFN_KERNEL<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  return cudaFuncSetAttribute(ACM_FFN_KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
 }
 
 cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
@@ -1316,7 +1311,7 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   }
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(ACM_FFN_KERNEL<true>), args);
+  return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(ACM_FFN_KERNEL), args);
 }
 
 #if !ACM_FFN_MX
