@@ -153,7 +153,8 @@ acm_status acm_set_layer_weights(acm_ctx* ctx, int layer, const void* w_router,
  *   half, the odd ones in the nibbles of its high half (element 2j = nibble j, 2j+1 = nibble 4+j).
  *   The four 16-byte pieces of a row's code bytes (32 K each) are stored rotated by the row number:
  *   piece p of row r (0..127 inside the record) at position p ^ ((r >> 1) & 3).
- * Scale bytes above 128 (block scales above 2) are treated as 128.  bf16 contexts with n_shared == 0,
+ * Scale bytes above 128 (block scales above 2) are not supported: the tensors are scanned when they are registered
+ * (here, and the host tensors in acm_set_slot_pool) and ACM_ERR_UNSUPPORTED is returned.  bf16 contexts with n_shared == 0,
  * hidden % 128 == 0 and inter % 128 == 0 only.  Both tile tensors may be NULL when the layer's experts
  * live in a pool (acm_set_slot_pool, called next): its pool and host tensors are then in this tiled
  * layout too ([n_slots][...] and [E][...]), and a loaded expert costs a quarter of the bf16 bytes.

@@ -11,7 +11,9 @@ namespace acm {
 
 constexpr int kMaxExperts = 128;   // E limit; also the padded length of expert-axis tree sums
 constexpr int kMaxTopK = 8;
-constexpr int kMaxNodes = 64;      // T limit = token columns of one FFN accumulator tile
+constexpr int kMaxNodes = 64;      // T limit of one verification block; the FFN kernel handles node columns 64 at a time
+constexpr int kWideNodes = 128;    // T limit of a batch of blocks = node columns of one wide FFN accumulator tile
+constexpr int kWtabStride = kWideNodes;   // row length of the combine-weight table [expert][node]
 constexpr int kMaxShared = 4;
 constexpr int kMaxSlots = kMaxExperts + kMaxShared;   // activated-expert slots of one work list
 constexpr int kMaskWords = 4;
@@ -43,10 +45,10 @@ struct Workspace {
   float* demand;        // [64][kMaxExperts]
   acm_block_stats* stats;   // [64]
   uint32_t* act_mask;   // [4] activated routed experts of the current block
-  float* wtab;          // [kMaxExperts][64] combine weight of (expert, node)
-  void* hbuf;           // [2][kMaxSlots][64][I] bf16 (f32 path: [T][k+ns][I] float)
-  float* frag;          // [2][grid][128*64] split-K partial sums, accumulated into the finishing CTA's buffer; zero between launches
-  int32_t* frag_flag;   // [2][grid] how many CTAs have added to that buffer; zero between launches
+  float* wtab;          // [kMaxExperts][kWtabStride] combine weight of (expert, node)
+  void* hbuf;           // [2][kMaxSlots][kWideNodes][I] bf16 (f32 path: [T][k+ns][I] float)
+  float* frag;          // [2][grid][2 column halves][128*64] split-K partial sums, accumulated into the finishing CTA's buffer; zero between launches
+  int32_t* frag_flag;   // [2][grid][2] how many CTAs have added to that buffer; zero between launches
   int32_t* ready;       // [2][kMaxSlots] finished gate/up tiles per activated slot
   int32_t* status;      // [1] sticky device-side status
   int32_t* tile_done;   // [64] router kernel: expert tiles finished per node tile (self-resetting)
@@ -73,7 +75,7 @@ struct SelectArgs {
 // A batch of verification blocks stacked along the node axis: block b owns rows off[b] .. off[b+1]-1.
 struct BatchDesc {
   int n_blocks;
-  int off[kMaxNodes + 1];
+  int off[kMaxNodes + 1];    // (at most 64 blocks, at most kWideNodes rows in all, at most kMaxNodes rows a block)
 };
 constexpr int kMaxEarlyBlocks = 8;
 // The rows whose natural top-k the router kernel publishes as anchors (the blocks' roots; one for a single block).
@@ -91,7 +93,7 @@ struct RouteArgs {
   float routed_scale;
   // inputs of the FFN kernel (all null when only the routes are wanted); zero on entry
   uint32_t* act_mask;            // [4] activated experts, OR-ed into
-  float* wtab;                   // [kMaxExperts][64] combine weights by (expert, node)
+  float* wtab;                   // [kMaxExperts][kWtabStride] combine weights by (expert, node)
   // The CTA that finishes last can also report on the whole block (it needs a ticket, so only when asked):
   int32_t* ticket;               // zero-initialised counter, left at zero; null: no report
   const uint32_t* resident;      // non-null: activated experts outside it are "staged"
@@ -150,9 +152,9 @@ struct FfnLaunch {
   uint32_t only[4];          // further restriction of this launch's experts (all ones: none); one wave of list 1
   int n_shared;
   const int32_t* slot_of;    // non-null: expert id -> slot of the layer's expert pool (the `staged` tensor maps)
-  const float* wtab;         // [kMaxExperts][64] combine weights by (expert, node)
+  const float* wtab;         // [kMaxExperts][kWtabStride] combine weights by (expert, node)
   acm_block_stats* stats;    // list 0 fills n_activated / n_staged (may be null)
-  void* hbuf;                // [kMaxSlots][64][I] bf16 of this list
+  void* hbuf;                // [kMaxSlots][kWideNodes][I] bf16 of this list
   int32_t* ready;            // [kMaxSlots] of this list (zero on entry)
   float* frag;
   int32_t* frag_flag;
@@ -178,7 +180,6 @@ struct FfnLaunch {
   unsigned long long* trace; // optional [grid][32] device time stamps (acm_stage_timing) or null
 };
 cudaError_t ffn_configure();   // one-time function attributes
-size_t ffn_smem_bytes();
 cudaError_t launch_ffn_bf16(const FfnLaunch& p, const FfnMaps& maps, const CUtensorMap& x_map,
                             const CUtensorMap& h_map, const CUtensorMap& h_store_map, cudaStream_t s);
 cudaError_t ffn_mx_configure();

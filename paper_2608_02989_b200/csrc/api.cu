@@ -98,6 +98,28 @@ bool plan_pool_block(int E, int n_slots, std::vector<int32_t>& slot_expert, std:
   return true;
 }
 
+// MXFP4 tile records: 128 x 64 code bytes, then 128 x 4 E8M0 scale bytes.  The FFN kernel applies a scale with one
+// bf16 multiply, which covers block scales up to 2 (scale byte 128); larger ones are refused at registration.
+constexpr size_t kMxRecordBytes = 128 * 64 + 128 * 4;
+constexpr int kMxMaxScaleByte = 128;
+__global__ void k_mx_max_scale(const unsigned char* tiles, size_t n_records, int* max_out) {
+  int m = 0;
+  for (size_t r = blockIdx.x; r < n_records; r += gridDim.x) {
+    const unsigned char* sc = tiles + r * kMxRecordBytes + 128 * 64;
+    for (int i = threadIdx.x; i < 512; i += blockDim.x) m = max(m, static_cast<int>(sc[i]));
+  }
+  m = __reduce_max_sync(0xffffffffu, m);
+  if ((threadIdx.x & 31) == 0 && m > 0) atomicMax(max_out, m);
+}
+int mx_max_scale_host(const unsigned char* tiles, size_t n_records) {
+  int m = 0;
+  for (size_t r = 0; r < n_records; ++r) {
+    const unsigned char* sc = tiles + r * kMxRecordBytes + 128 * 64;
+    for (int i = 0; i < 512; ++i) m = sc[i] > m ? sc[i] : m;
+  }
+  return m;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -250,19 +272,20 @@ acm_status encode_x(acm_ctx* c, CUtensorMap* m, const void* x, int T, int n_pad)
 // activations [slots, 64, I] as {k in atom, node, atom of I, slot}; one box = n_pad nodes x 2 atoms.
 acm_status encode_h(acm_ctx* c, CUtensorMap* m, const void* base, int n_pad, int atoms) {
   const uint64_t I = c->desc.inter;
-  const uint64_t dims[4] = {64, kMaxNodes, I / 64, kMaxSlots};
-  const uint64_t strides[3] = {I * 2, 128, kMaxNodes * I * 2};
+  const uint64_t dims[4] = {64, kWideNodes, I / 64, kMaxSlots};
+  const uint64_t strides[3] = {I * 2, 128, kWideNodes * I * 2};
   const uint32_t box[4] = {64, static_cast<uint32_t>(n_pad), static_cast<uint32_t>(atoms), 1};
   return encode_view(c, m, base, 4, dims, strides, box);
 }
 
 acm_status ensure_h_maps(acm_ctx* c, int n_pad) {
   if (c->h_map_npad == n_pad) return ACM_OK;
-  const size_t list_bytes = static_cast<size_t>(kMaxSlots) * kMaxNodes * c->desc.inter * 2;
+  const size_t list_bytes = static_cast<size_t>(kMaxSlots) * kWideNodes * c->desc.inter * 2;
   for (int l = 0; l < 2; ++l) {
     acm_status st = encode_h(c, &c->h_map[l], static_cast<char*>(c->ws.hbuf) + l * list_bytes, n_pad, 2);
     if (st != ACM_OK) return st;
-    st = encode_h(c, &c->h_store_map[l], static_cast<char*>(c->ws.hbuf) + l * list_bytes, n_pad, 1);
+    // (stored 64 node rows at a time: a wide tile in two halves)
+    st = encode_h(c, &c->h_store_map[l], static_cast<char*>(c->ws.hbuf) + l * list_bytes, n_pad < kMaxNodes ? n_pad : kMaxNodes, 1);
     if (st != ACM_OK) return st;
   }
   c->h_map_npad = n_pad;
@@ -334,7 +357,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   p.slot_of = L.has_pool ? L.slot_of_dev[L.slot_of_cur] : nullptr;
   p.wtab = c->ws.wtab;
   p.stats = stats_dev;
-  p.hbuf = static_cast<char*>(c->ws.hbuf) + static_cast<size_t>(li) * kMaxSlots * kMaxNodes * d.inter * 2;
+  p.hbuf = static_cast<char*>(c->ws.hbuf) + static_cast<size_t>(li) * kMaxSlots * kWideNodes * d.inter * 2;
   p.ready = c->ws.ready + li * kMaxSlots;
   p.frag = c->ws.frag; p.frag_flag = c->ws.frag_flag;
   p.sel_flag = nullptr; p.sel_epoch = 0; p.sel_blocks = n_blocks > 0 ? n_blocks : 1;
@@ -487,7 +510,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
     if (ffn_configure() != cudaSuccess) return fail(ACM_ERR_CUDA);
   }
 
-  const int Tm = kMaxNodes, E = desc->n_experts, k = desc->top_k, I = desc->inter;
+  const int Tm = kWideNodes, E = desc->n_experts, k = desc->top_k, I = desc->inter;
   size_t off = 0;
   auto carve = [&](size_t bytes) {
     const size_t at = off;
@@ -500,13 +523,13 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_dem = carve(sizeof(float) * kMaxExperts * Tm), o_stats = carve(sizeof(acm_block_stats) * Tm);
   // the FFN kernel's routing inputs, contiguous so that one pass clears them: weight table, finished-tile
   // counters, activated mask
-  const size_t ffn_in_bytes = sizeof(float) * kMaxExperts * kMaxNodes + sizeof(int32_t) * 2 * kMaxSlots + 16;
+  const size_t ffn_in_bytes = sizeof(float) * kMaxExperts * kWtabStride + sizeof(int32_t) * 2 * kMaxSlots + 16;
   const size_t o_ffn_in = carve(align_up(ffn_in_bytes, 16));
-  const size_t hbuf_bf16 = static_cast<size_t>(2) * kMaxSlots * kMaxNodes * I * 2;
+  const size_t hbuf_bf16 = static_cast<size_t>(2) * kMaxSlots * kWideNodes * I * 2;
   const size_t hbuf_f32 = static_cast<size_t>(Tm) * (k + desc->n_shared) * I * 4;
   const size_t o_h = carve(hbuf_bf16 > hbuf_f32 ? hbuf_bf16 : hbuf_f32);
-  const size_t o_frag = carve(sizeof(float) * 2 * static_cast<size_t>(c->sm_count) * 128 * kMaxNodes);
-  const size_t o_flag = carve(sizeof(int32_t) * 2 * c->sm_count);
+  const size_t o_frag = carve(sizeof(float) * 2 * 2 * static_cast<size_t>(c->sm_count) * 128 * kMaxNodes);
+  const size_t o_flag = carve(sizeof(int32_t) * 2 * 2 * c->sm_count);
   const size_t o_status = carve(16);
   const size_t o_tile = carve(sizeof(int32_t) * kMaxNodes);
   const size_t o_ticket = carve(16);
@@ -529,14 +552,14 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.demand = reinterpret_cast<float*>(b + o_dem);
   c->ws.stats = reinterpret_cast<acm_block_stats*>(b + o_stats);
   c->ws.wtab = reinterpret_cast<float*>(b + o_ffn_in);
-  c->ws.ready = reinterpret_cast<int32_t*>(b + o_ffn_in + sizeof(float) * kMaxExperts * kMaxNodes);
-  c->ws.act_mask = reinterpret_cast<uint32_t*>(b + o_ffn_in + sizeof(float) * kMaxExperts * kMaxNodes +
+  c->ws.ready = reinterpret_cast<int32_t*>(b + o_ffn_in + sizeof(float) * kMaxExperts * kWtabStride);
+  c->ws.act_mask = reinterpret_cast<uint32_t*>(b + o_ffn_in + sizeof(float) * kMaxExperts * kWtabStride +
                                                sizeof(int32_t) * 2 * kMaxSlots);
   c->ffn_in_floats = align_up(ffn_in_bytes, 16) / sizeof(float);
   c->ws.hbuf = b + o_h;
   c->ws.frag = reinterpret_cast<float*>(b + o_frag);
-  c->frag_bytes = sizeof(float) * 2 * static_cast<size_t>(c->sm_count) * 128 * kMaxNodes;
-  c->flag_bytes = sizeof(int32_t) * 2 * c->sm_count;
+  c->frag_bytes = sizeof(float) * 2 * 2 * static_cast<size_t>(c->sm_count) * 128 * kMaxNodes;
+  c->flag_bytes = sizeof(int32_t) * 2 * 2 * c->sm_count;
   c->ws.frag_flag = reinterpret_cast<int32_t*>(b + o_flag);
   c->ws.status = reinterpret_cast<int32_t*>(b + o_status);
   c->ws.tile_done = reinterpret_cast<int32_t*>(b + o_tile);
@@ -629,6 +652,19 @@ acm_status acm_set_layer_weights_mxfp4(acm_ctx* c, int layer, const void* w_rout
   if (!c->mx_configured) {
     if (ffn_mx_configure() != cudaSuccess) return ACM_ERR_CUDA;
     c->mx_configured = true;
+  }
+  if (gate_up_tiles) {
+    // every scale byte of both tensors, once, at registration (a small kernel and one synchronous read-back)
+    const size_t rec_gu = static_cast<size_t>(d.n_experts) * (d.inter / 64) * (d.hidden / 128);
+    const size_t rec_dn = static_cast<size_t>(d.n_experts) * (d.hidden / 128) * (d.inter / 128);
+    int* max_dev = reinterpret_cast<int*>(c->ws.ticket) + 2;      // (a spare word of the workspace)
+    ACM_CUDA(cudaMemset(max_dev, 0, sizeof(int)));
+    k_mx_max_scale<<<256, 256>>>(static_cast<const unsigned char*>(gate_up_tiles), rec_gu, max_dev);
+    k_mx_max_scale<<<256, 256>>>(static_cast<const unsigned char*>(down_tiles), rec_dn, max_dev);
+    int max_scale = 0;
+    ACM_CUDA(cudaMemcpy(&max_scale, max_dev, sizeof(int), cudaMemcpyDeviceToHost));
+    ACM_CUDA(cudaMemset(max_dev, 0, sizeof(int)));
+    if (max_scale > kMxMaxScaleByte) return ACM_ERR_UNSUPPORTED;
   }
   Layer L;
   L.w_router = w_router; L.bias = router_bias;
@@ -946,13 +982,15 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
   if (block_offsets[0] != 0) return ACM_ERR_INVALID;
   for (int b = 0; b <= n_blocks; ++b) {
     if (b > 0 && block_offsets[b] <= block_offsets[b - 1]) return ACM_ERR_INVALID;     // every block has a node
-    if (block_offsets[b] > kMaxNodes) return ACM_ERR_INVALID;
+    if (b > 0 && block_offsets[b] - block_offsets[b - 1] > c->desc.max_nodes) return ACM_ERR_INVALID;   // a block's own limit
+    if (block_offsets[b] > kWideNodes) return ACM_ERR_INVALID;
     bd.off[b] = block_offsets[b];
   }
   const int T = block_offsets[n_blocks];
-  acm_status st = check_block_args(c, layer, T, true);
+  acm_status st = check_block_args(c, layer, 1, true);
   if (st != ACM_OK) return st;
   const Layer& L = c->layers[layer];
+  if (T > kMaxNodes && L.mx) return ACM_ERR_UNSUPPORTED;      // (the MXFP4 kernel's tensor memory holds 64-column accumulators only)
   if (!x || !out || !alpha || (!L.gate_up && !L.mx_gate_up)) return ACM_ERR_INVALID;
   if (reinterpret_cast<uintptr_t>(x) % 16 != 0 || reinterpret_cast<uintptr_t>(out) % 16 != 0) return ACM_ERR_INVALID;
   st = check_params(params);
@@ -1129,6 +1167,13 @@ acm_status acm_set_slot_pool(acm_ctx* c, int layer, int n_slots, void* pool_gate
     return ACM_ERR_INVALID;
   acm_status st = ensure_offload_common(c);
   if (st != ACM_OK) return st;
+  if (L.mx) {                 // the pool is fed from the host tensors: their scale bytes must be in range
+    const size_t rec = static_cast<size_t>(d.n_experts) * ((d.inter / 64) * (d.hidden / 128));
+    const size_t rec_dn = static_cast<size_t>(d.n_experts) * ((d.hidden / 128) * (d.inter / 128));
+    if (mx_max_scale_host(static_cast<const unsigned char*>(host_gate_up), rec) > kMxMaxScaleByte ||
+        mx_max_scale_host(static_cast<const unsigned char*>(host_down), rec_dn) > kMxMaxScaleByte)
+      return ACM_ERR_UNSUPPORTED;
+  }
   if (!L.mx) {                // (the MXFP4 kernel fetches its tile records with plain bulk copies)
     st = encode_gate_up(c, &L.pool_map_gu, pool_gate_up, n_slots);
     if (st != ACM_OK) return st;

@@ -39,21 +39,19 @@ namespace {
 #ifndef ACM_FFN_MX
 #define ACM_FFN_MX 0
 #endif
-constexpr int kStages = 3;                               // pipeline stages of the weight ring
+constexpr int kMaxStages = 3;                            // pipeline stages of the weight ring (see Geo)
 constexpr int kAcc = 4;                                  // TMEM accumulators in flight (power of two)
 constexpr int kBK = 64;                                  // K elements of one 128-byte swizzle atom
 constexpr int kAtoms = 2;                                // atoms per pipeline stage: a stage covers 128 K
 constexpr int kTileM = 128;
 constexpr int kAtomABytes = kTileM * kBK * 2;            // 16 KB: 128 weight rows x one atom
 constexpr int kABytes = kAtoms * kAtomABytes;            // 32 KB weight tile, one TMA copy
-constexpr int kBBytesMax = kAtoms * kMaxNodes * kBK * 2; // 16 KB activation chunk, one TMA copy
-constexpr int kStageBytes = kABytes + kBBytesMax;
+// The epilogue handles node columns kMaxNodes = 64 at a time: one fragment, one activation tile.  A wide tile (a
+// batch of blocks with more than 64 nodes in all, up to kWideNodes = 128 accumulator columns) goes in two halves.
 constexpr int kOutStageBytes = kTileM * kMaxNodes * 4;   // 32 KB: outgoing fragment (also the gate/up exchange buffer)
-constexpr int kHStageBytes = kMaxNodes * 64 * 2;         // 8 KB: one finished activation tile (64 features x nodes)
-constexpr int kAccCols = kMaxNodes;                      // TMEM columns per accumulator
+constexpr int kHStageBytes = kMaxNodes * 64 * 2;         // 8 KB: one finished activation tile (64 features x 64 nodes)
 constexpr int kMxACols = 64;                             // MXFP4: one expanded weight stage in tensor memory = 128 K bf16 per row
-constexpr int kTmemCols = ACM_FFN_MX ? 512 : kAcc * kAccCols;   // MXFP4: accumulators, then kStages expanded weight stages
-static_assert(kAcc * kAccCols + kStages * kMxACols <= 512, "tensor memory: accumulators + expanded weight stages");
+static_assert(kAcc * kMaxNodes + kMaxStages * kMxACols <= 512, "tensor memory: accumulators + expanded weight stages");
 // ACM_FFN_MX = 1 (set by ffn_mx.cu, which includes this file) builds the same kernel for MXFP4 expert
 // weights: a pipeline stage of a weight tile arrives as 128 rows x 64 bytes of E2M1 codes + 128 x 4 E8M0
 // scale bytes (one contiguous 8704-byte copy into the stage's weight area), and four more warps expand it
@@ -108,24 +106,25 @@ struct GiveUp {
   int32_t tag;                   // launch number << 8
 };
 
-struct __align__(8) Barriers {
-  unsigned long long full[kStages];
-  unsigned long long empty[kStages];
+template <int kN>
+struct __align__(8) BarriersT {
+  unsigned long long full[kMaxStages];
+  unsigned long long empty[kMaxStages];
   unsigned long long tfull[kAcc];
   unsigned long long tempty[kAcc];
   unsigned long long drained;
-  unsigned long long frag_full[2];   // helper -> epilogue: pre-summed fragments of gate/up segment i are in smem
+  unsigned long long frag_full;      // helper -> epilogue: the pre-summed fragments of the next cut tile (half) are in smem
   unsigned long long frag_free;      // epilogue -> helper: the fragment buffer may be overwritten
   unsigned long long helper;         // completion of the helper warp's bulk copy
   unsigned long long ost_full, ost_free;   // epilogue <-> publisher: outgoing fragment staged / copied out
   unsigned long long hst_full[2], hst_free[2];   // epilogue <-> publisher: activation tile staged / stored
 #if ACM_FFN_MX
-  unsigned long long raw[kStages];   // the packed weight stage has landed (producer's copy -> expanding warps)
+  unsigned long long raw[kMaxStages];   // the packed weight stage has landed (producer's copy -> expanding warps)
 #endif
   volatile uint32_t armed;           // stages whose barrier the weight producer has armed so far
   uint32_t tmem_base;
   GiveUp give_up;
-  float wd[kMaxNodes];          // combine weights of the expert being finalised
+  float wd[kN];                 // combine weights of the expert being finalised
   int32_t entry[kMaxSlots];     // this launch's work list: make_entry(source, index) of every activated slot
   int16_t expert[kMaxSlots];    // routed expert id of the slot (-1: shared expert)
   uint32_t sel_half[4 * kMaskWords];   // early start: the eligible mask in 16-bit pieces (second half: blocks 4..7 of a batch)
@@ -134,9 +133,19 @@ struct __align__(8) Barriers {
   uint32_t anc_part[4 * kMaskWords];   // early start on the anchors: their mask in 16-bit pieces (by the two polling warps)
 };
 
-static_assert(sizeof(Barriers) <= 232448 - 1024 - kStages * kStageBytes - kOutStageBytes - kFragBytes - 2 * kHStageBytes,
-              "shared memory: ring + staging buffers + control block exceed 227 KB");
-constexpr size_t kSmemBytes = 1024 + static_cast<size_t>(kStages) * kStageBytes + kOutStageBytes + kFragBytes + 2 * kHStageBytes + sizeof(Barriers);
+// Geometry of the kernel for accumulator tiles of kN node columns: 64 (one block, three 48 KB stages) or 128 (a
+// batch, two 64 KB stages -- as many bytes in flight -- and all of tensor memory).
+template <int kN>
+struct Geo {
+  static constexpr int kStages = kN > kMaxNodes ? 2 : 3;
+  static constexpr int kBBytes = kAtoms * kN * kBK * 2;          // activation chunk of a stage, one TMA copy
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kTmemCols = ACM_FFN_MX ? 512 : kAcc * kN;    // MXFP4: accumulators, then the expanded weight stages
+  static constexpr size_t kSmemBytes =
+      1024 + static_cast<size_t>(kStages) * kStageBytes + kOutStageBytes + kFragBytes + 2 * kHStageBytes + sizeof(BarriersT<kN>);
+  static_assert(kSmemBytes <= 232448, "shared memory: ring + staging buffers + control block exceed 227 KB");
+  static_assert(kStages <= kMaxStages, "barrier arrays");
+};
 
 // ---------------------------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
@@ -408,10 +417,14 @@ __device__ __forceinline__ const CUtensorMap* pick_map(int src, const CUtensorMa
 #endif
 // One kernel for both starts (on the anchors' pre-segment, or with the whole work list at hand): a launch bracketed
 // by events then runs the same code as the launches around it, which keeps its instructions warm in the caches.
+// kN = node columns of an accumulator tile (see Geo).
+template <int kN>
 __global__ void __launch_bounds__(kThreads, 1)
 ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUtensorMap x_map,
            const __grid_constant__ CUtensorMap h_map, const __grid_constant__ CUtensorMap hs_map,
            const FfnArgs p) {
+  constexpr int kStages = Geo<kN>::kStages, kStageBytes = Geo<kN>::kStageBytes, kAccCols = kN, kTmemCols = Geo<kN>::kTmemCols;
+  using Barriers = BarriersT<kN>;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   unsigned char* stage_base = smem;
@@ -440,8 +453,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     }
     mbar_init(smem_u32(&bars->drained), 1);
     mbar_init(smem_u32(&bars->plan_ready), 1);
-    mbar_init(smem_u32(&bars->frag_full[0]), 1);
-    mbar_init(smem_u32(&bars->frag_full[1]), 1);
+    mbar_init(smem_u32(&bars->frag_full), 1);
     mbar_init(smem_u32(&bars->frag_free), 128);
     mbar_init(smem_u32(&bars->helper), 1);
     mbar_init(smem_u32(&bars->ost_full), 128);
@@ -525,6 +537,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     n_routed += __popc(am[wd]);
   }
   const int tpe = p.I / 64;          // gate/up tiles per expert = K-chunks per expert in the down phase
+  const int n_halves = (kN > kMaxNodes && p.n_pad > kMaxNodes) ? 2 : 1;   // the epilogue takes 64 node columns at a time
   // pre-segment: as many of the anchors (in ascending id) as give every CTA at most one whole tile
   const int n_pre = pre ? min(n_routed, static_cast<int>(fdiv(static_cast<unsigned>(G), p.d_tpe))) : 0;
   if (pre) {
@@ -829,20 +842,21 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
         const unsigned tile_end = (last_tile + 1) * kc1;
         const bool head = (last_tile * kc1 >= ub) && (ue < tile_end);   // starts at chunk 0, ends before the tile does
         if (!head) continue;
-        if (frag_uses > 0) {   // the buffer still holds the previous segment's sum until the epilogue has read it
-          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->frag_free), (frag_uses - 1) & 1u, quit, kSiteFragFree));
-          if (!ok) break;
-        }
-        float* frag = p.frag + (static_cast<size_t>(sg.p1_index) * G + cta) * kFragFloats;   // this CTA's buffer
-        int32_t* arrived = p.frag_flag + sg.p1_index * G + cta;
-        const int n_el = p.n_pad * kTileM;
         int n_contrib = 0;
         for (int c2 = cta + 1; c2 < G; ++c2) {
           const unsigned b2 = cut_begin(sg, c2, p.d_grid), e2 = cut_begin(sg, c2 + 1, p.d_grid);
           if (b2 >= tile_end) break;
           if (e2 > b2) ++n_contrib;
         }
-        {
+        // one fragment buffer and one arrival counter per column half of the tile (a wide tile has two)
+        for (int h = 0; h < n_halves && ok; ++h) {
+          if (frag_uses > 0) {   // the buffer in shared memory still holds the previous sum until the epilogue has read it
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->frag_free), (frag_uses - 1) & 1u, quit, kSiteFragFree));
+            if (!ok) break;
+          }
+          float* frag = p.frag + ((static_cast<size_t>(sg.p1_index) * G + cta) * 2 + h) * kFragFloats;   // this CTA's buffer
+          int32_t* arrived = p.frag_flag + (sg.p1_index * G + cta) * 2 + h;
+          const int n_el = min(p.n_pad - h * kMaxNodes, kMaxNodes) * kTileM;
           // every CTA holding a later part of the tile has reduce-added its fragment: one bulk copy
           bool got = true;
           if (lane == 0) got = flag_wait_ge(arrived, n_contrib, quit, kSiteFragArrivals);
@@ -857,13 +871,14 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
           }
           ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->helper), frag_uses & 1u, quit, kSiteFragCopy));
           if (!ok) break;
-          if (lane == 0) mbar_arrive(smem_u32(&bars->frag_full[sg.p1_index]));
+          if (lane == 0) mbar_arrive(smem_u32(&bars->frag_full));
           // leave the buffer and its counter zero for the next launch
           float4* z4 = reinterpret_cast<float4*>(frag);
           for (int i = lane; i < n_el / 4; i += 32) z4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
           if (lane == 0) *arrived = 0;
+          ++frag_uses;
         }
-        ++frag_uses;
+        if (!ok) break;
       } else {
         // activation producer: once every activation tile of this expert group is stored, add the
         // activation chunk of each down stage to the barrier the weight producer has armed (or will arm)
@@ -881,7 +896,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
               q_hi = static_cast<int>(fdiv(static_cast<unsigned>(rg.k00) + n_units - 1u, p.d_kpe));
             }
             for (int q = q_lo + lane; q <= q_hi && good; q += 32)
-              good = flag_wait_ge(&p.ready[sg.a0 + q], tpe, quit, kSiteExpertReady);
+              good = flag_wait_ge(&p.ready[sg.a0 + q], tpe * n_halves, quit, kSiteExpertReady);
           }
           good = __all_sync(0xffffffffu, good);
         }
@@ -928,14 +943,15 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       for (int si = 0; ok && have_seg(si, true); ++si) {
         const Segment sg = seg[si];
         if (sg.phase != 1) continue;
-        float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * kFragFloats;
-        int32_t* frag_flag = p.frag_flag + sg.p1_index * G;
+        float* frag = p.frag + static_cast<size_t>(sg.p1_index) * G * 2 * kFragFloats;
+        int32_t* frag_flag = p.frag_flag + sg.p1_index * G * 2;
         Sched sc(bars->plan.range[si]);
         int tile, k0, k1;
         while (ok && sc.next(tile, k0, k1)) {
+         for (int h = 0; h < n_halves && ok; ++h) {          // a wide tile comes in two column halves
           if (k0 > 0) {
             if (!(ok = mbar_wait(smem_u32(&bars->ost_full), ost_n & 1u, quit, kSiteOutStaged))) break;
-            const uint32_t bytes = static_cast<uint32_t>(p.n_pad) * kTileM * 4u;
+            const uint32_t bytes = static_cast<uint32_t>(min(p.n_pad - h * kMaxNodes, kMaxNodes)) * kTileM * 4u;
             // All CTAs that hold a tail part of this tile add into ONE global buffer, that of the CTA
             // which owns the tile's first chunks and will finish it.  The buffers are zero between
             // launches (the finishing CTA clears its own after reading), so nobody waits for anybody.
@@ -943,10 +959,10 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
             int c_head = cta - 1;
             while (c_head > 0 && cut_begin(sg, c_head, p.d_grid) > tile_begin) --c_head;   // owner of the tile's first chunk
             asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
-                         ::"l"(frag + static_cast<size_t>(c_head) * kFragFloats), "r"(smem_u32(ostage)), "r"(bytes) : "memory");
+                         ::"l"(frag + static_cast<size_t>(c_head * 2 + h) * kFragFloats), "r"(smem_u32(ostage)), "r"(bytes) : "memory");
             bulk_commit();
             bulk_wait_all();
-            red_release_add(&frag_flag[c_head], 1);
+            red_release_add(&frag_flag[c_head * 2 + h], 1);
             mbar_arrive(smem_u32(&bars->ost_free));
             ++ost_n;
           } else {
@@ -954,13 +970,14 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
             if (!(ok = mbar_wait(smem_u32(&bars->hst_full[hb]), (fin_n >> 1) & 1u, quit, kSiteActStaged))) break;
             const int a = static_cast<int>(fdiv(static_cast<unsigned>(sg.t0 + tile), p.d_tpe)), ti = sg.t0 + tile - a * tpe;
             asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
-                         ::"l"(&hs_map), "r"(0), "r"(0), "r"(ti), "r"(a), "r"(smem_u32(hstage + hb * kHStageBytes)) : "memory");
+                         ::"l"(&hs_map), "r"(0), "r"(h * kMaxNodes), "r"(ti), "r"(a), "r"(smem_u32(hstage + hb * kHStageBytes)) : "memory");
             bulk_commit();
             bulk_wait_all();
             red_release_add(&p.ready[a], 1);
             mbar_arrive(smem_u32(&bars->hst_free[hb]));
             ++fin_n;
           }
+         }
         }
       }
     }
@@ -1038,16 +1055,19 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
     const int quarter = warp & 3;               // TMEM lanes this warp may read
     const int row = quarter * 32 + lane;        // accumulator row = weight-tile row
     const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
-    uint32_t f = 0, ost_uses = 0, fin_count = 0;
+    uint32_t f = 0, ost_uses = 0, fin_count = 0, frag_reads = 0;
     bool ok = true, waited = !early;
     float v[kMaxNodes];
-    auto load_acc = [&](uint32_t b) {
+    // one half (up to 64 columns from column `cb` on) of accumulator b; the accumulator is released with its last half
+    auto load_half = [&](uint32_t b, int cb, int np, bool release) {
 #pragma unroll
       for (int c = 0; c < kMaxNodes; c += 16)
-        if (c < p.n_pad) tmem_ld16(tmem_base + lane_addr + b * kAccCols + c, v + c);
+        if (c < np) tmem_ld16(tmem_base + lane_addr + b * kAccCols + cb + c, v + c);
       tmem_ld_wait();
-      tc_fence_before();
-      mbar_arrive(smem_u32(&bars->tempty[b]));
+      if (release) {
+        tc_fence_before();
+        mbar_arrive(smem_u32(&bars->tempty[b]));
+      }
     };
     // the outgoing-fragment buffer (and the exchange buffer aliasing it) is free once the publisher
     // has copied the previous fragment out
@@ -1060,7 +1080,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       if (sg.phase == 1) {
         Sched sc(bars->plan.range[si]);
         int tile, k0, k1;
-        while (sc.next(tile, k0, k1)) {
+        while (ok && sc.next(tile, k0, k1)) {
           const uint32_t b = f % kAcc;
           // A tile this CTA will finish needs its expert's combine weights: fetch them (one L2 round
           // trip) while the tile's MMAs run, not after them.  They are the routing kernel's last output.
@@ -1073,108 +1093,116 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
             }
             if (row < p.n_pad) {
               const int ex_id = bars->expert[a];      // the table row of a routed expert, 1 for a shared one
-              wd_mine = ex_id >= 0 ? __ldcg(p.wtab + static_cast<size_t>(ex_id) * kMaxNodes + row) : (row < p.T ? 1.0f : 0.0f);
+              wd_mine = ex_id >= 0 ? __ldcg(p.wtab + static_cast<size_t>(ex_id) * kWtabStride + row) : (row < p.T ? 1.0f : 0.0f);
             }
           }
           ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f / kAcc) & 1u, quit, kSiteAccFull));
           if (!ok) break;
           tc_fence_after();
-          load_acc(b);
           ++f;
-          if (k0 > 0) {
-            // tail part of a tile whose first chunks belong to an earlier CTA: stage the fragment
+          if (k0 == 0 && row < p.n_pad) bars->wd[row] = wd_mine;
+          for (int h = 0; h < n_halves && ok; ++h) {
+            const int cb = h * kMaxNodes;                              // first node column of this half
+            const int np = min(p.n_pad - cb, kMaxNodes);               // its columns (a multiple of 16)
+            load_half(b, cb, np, h == n_halves - 1);
+            if (k0 > 0) {
+              // tail part of a tile whose first chunks belong to an earlier CTA: stage the fragment
+              if (!(ok = wait_ostage())) break;
+#pragma unroll
+              for (int c = 0; c < kMaxNodes; ++c)
+                if (c < np) ostage[c * kTileM + row] = v[c];
+              fence_proxy_async_smem();
+              mbar_arrive(smem_u32(&bars->ost_full));
+              ++ost_uses;
+              continue;
+            }
+            if (k1 < kc1) {
+              // head part: the helper warp has summed the other CTAs' fragments of this tile (half) into smem
+              ok = epi_vote_all(mbar_wait(smem_u32(&bars->frag_full), frag_reads & 1u, quit, kSiteFragFull));
+              if (!ok) break;
+#pragma unroll
+              for (int c = 0; c < kMaxNodes; ++c)
+                if (c < np) v[c] += sfrag[c * kTileM + row];
+              mbar_arrive(smem_u32(&bars->frag_free));
+              ++frag_reads;
+            }
+            // rows 0..63 hold gate, rows 64..127 the matching up projections.  Each pair of threads
+            // (i, i+64) splits the node columns: the gate thread finishes columns [0, 32), the up
+            // thread columns [32, 64); they swap the halves they do not finish through smem.
+            constexpr int kHalf = kMaxNodes / 2;
+            const int feat = row & 63;
             if (!(ok = wait_ostage())) break;
+            if (quarter >= 2) {
 #pragma unroll
-            for (int c = 0; c < kMaxNodes; ++c)
-              if (c < p.n_pad) ostage[c * kTileM + row] = v[c];
-            fence_proxy_async_smem();
-            mbar_arrive(smem_u32(&bars->ost_full));
-            ++ost_uses;
-            continue;
-          }
-          if (row < p.n_pad) bars->wd[row] = wd_mine;
-          if (k1 < kc1) {
-            // head part: the helper warp has summed the other CTAs' fragments of this tile into smem
-            ok = epi_vote_all(mbar_wait(smem_u32(&bars->frag_full[sg.p1_index]), 0, quit, kSiteFragFull));
+              for (int c = 0; c < kHalf; ++c)
+                if (c < np) ex[c * 64 + feat] = v[c];
+            } else {
+#pragma unroll
+              for (int c = kHalf; c < kMaxNodes; ++c)
+                if (c < np) ex[c * 64 + feat] = v[c];
+            }
+            const uint32_t hb = fin_count & 1u;
+            bool hst_ok = true;
+            if (fin_count >= 2) hst_ok = mbar_wait(smem_u32(&bars->hst_free[hb]), ((fin_count >> 1) - 1) & 1u, quit, kSiteActFree);
+            ok = epi_vote_all(hst_ok);      // also orders the exchange writes above before the reads below
             if (!ok) break;
+            {
+              unsigned char* hs = hstage + hb * kHStageBytes;
+              const int c0 = quarter < 2 ? 0 : kHalf;
 #pragma unroll
-            for (int c = 0; c < kMaxNodes; ++c)
-              if (c < p.n_pad) v[c] += sfrag[c * kTileM + row];
-            mbar_arrive(smem_u32(&bars->frag_free));
-          }
-          // rows 0..63 hold gate, rows 64..127 the matching up projections.  Each pair of threads
-          // (i, i+64) splits the node columns: the gate thread finishes columns [0, 32), the up
-          // thread columns [32, 64); they swap the halves they do not finish through smem.
-          constexpr int kHalf = kMaxNodes / 2;
-          const int feat = row & 63;
-          if (!(ok = wait_ostage())) break;
-          if (quarter >= 2) {
+              for (int j0 = 0; j0 < kHalf; j0 += 8) {
+                if (c0 + j0 < np) {           // np is a multiple of 16: a block of 8 columns is all in or all out
+                  float other[8], wgt[8], hval[8];
 #pragma unroll
-            for (int c = 0; c < kHalf; ++c)
-              if (c < p.n_pad) ex[c * 64 + feat] = v[c];
-          } else {
+                  for (int j = 0; j < 8; ++j) {
+                    other[j] = ex[(c0 + j0 + j) * 64 + feat];
+                    wgt[j] = bars->wd[cb + c0 + j0 + j];
+                  }
 #pragma unroll
-            for (int c = kHalf; c < kMaxNodes; ++c)
-              if (c < p.n_pad) ex[c * 64 + feat] = v[c];
-          }
-          const uint32_t hb = fin_count & 1u;
-          bool hst_ok = true;
-          if (fin_count >= 2) hst_ok = mbar_wait(smem_u32(&bars->hst_free[hb]), ((fin_count >> 1) - 1) & 1u, quit, kSiteActFree);
-          ok = epi_vote_all(hst_ok);      // also orders the exchange writes above before the reads below
-          if (!ok) break;
-          {
-            unsigned char* hs = hstage + hb * kHStageBytes;
-            const int c0 = quarter < 2 ? 0 : kHalf;
+                  for (int j = 0; j < 8; ++j) {
+                    const float mine = quarter < 2 ? v[j0 + j] : v[kHalf + j0 + j];
+                    const float g = quarter < 2 ? mine : other[j];
+                    const float u = quarter < 2 ? other[j] : mine;
+                    // w * u * silu(g), silu(g) = g/2 * (1 + tanh(g/2))
+                    const float hg = 0.5f * g;
+                    float th;
+                    asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(hg));
+                    const float q = wgt[j] * u * hg;
+                    hval[j] = fmaf(q, th, q);
+                  }
+                  // activation tile [node][64 features] bf16 in the 128-byte-swizzled layout of its TMA store
 #pragma unroll
-            for (int j0 = 0; j0 < kHalf; j0 += 8) {
-              if (c0 + j0 < p.n_pad) {           // n_pad is a multiple of 16: a block of 8 columns is all in or all out
-                float other[8], wgt[8], hval[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  other[j] = ex[(c0 + j0 + j) * 64 + feat];
-                  wgt[j] = bars->wd[c0 + j0 + j];
-                }
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  const float mine = quarter < 2 ? v[j0 + j] : v[kHalf + j0 + j];
-                  const float g = quarter < 2 ? mine : other[j];
-                  const float u = quarter < 2 ? other[j] : mine;
-                  // w * u * silu(g), silu(g) = g/2 * (1 + tanh(g/2))
-                  const float hg = 0.5f * g;
-                  float th;
-                  asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(hg));
-                  const float q = wgt[j] * u * hg;
-                  hval[j] = fmaf(q, th, q);
-                }
-                // activation tile [node][64 features] bf16 in the 128-byte-swizzled layout of its TMA store
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                  const int t = c0 + j0 + j;
-                  const int off = t * 128 + ((((feat >> 3) ^ (t & 7))) << 4) + ((feat & 7) << 1);
-                  *reinterpret_cast<__nv_bfloat16*>(hs + off) = __float2bfloat16_rn(hval[j]);
+                  for (int j = 0; j < 8; ++j) {
+                    const int t = c0 + j0 + j;
+                    const int off = t * 128 + ((((feat >> 3) ^ (t & 7))) << 4) + ((feat & 7) << 1);
+                    *reinterpret_cast<__nv_bfloat16*>(hs + off) = __float2bfloat16_rn(hval[j]);
+                  }
                 }
               }
+              fence_proxy_async_smem();
+              mbar_arrive(smem_u32(&bars->hst_full[hb]));
+              ++fin_count;
             }
-            fence_proxy_async_smem();
-            mbar_arrive(smem_u32(&bars->hst_full[hb]));
-            ++fin_count;
           }
         }
         if (row == 0) ACM_STAMP(10);
       } else {
         Sched sc(bars->plan.range[si]);
         int ht, k0, k1;
-        while (sc.next(ht, k0, k1)) {
+        while (ok && sc.next(ht, k0, k1)) {
           const uint32_t b = f % kAcc;
           ok = epi_vote_all(mbar_wait(smem_u32(&bars->tfull[b]), (f / kAcc) & 1u, quit, kSiteAccFull));
           if (!ok) break;
           tc_fence_after();
-          load_acc(b);
           ++f;
-          float* dst = p.out + static_cast<size_t>(ht) * kTileM + row;
+          for (int h = 0; h < n_halves; ++h) {
+            const int cb = h * kMaxNodes;
+            load_half(b, cb, min(p.n_pad - cb, kMaxNodes), h == n_halves - 1);
+            float* dst = p.out + static_cast<size_t>(cb) * p.H + static_cast<size_t>(ht) * kTileM + row;
 #pragma unroll
-          for (int c = 0; c < kMaxNodes; ++c)
-            if (c < p.T) atomicAdd(dst + static_cast<size_t>(c) * p.H, v[c]);
+            for (int c = 0; c < kMaxNodes; ++c)
+              if (cb + c < p.T) atomicAdd(dst + static_cast<size_t>(c) * p.H, v[c]);
+          }
         }
         if (row == 0) ACM_STAMP(11);
       }
@@ -1249,15 +1277,19 @@ __global__ void k_ffn_f32_down(const float* __restrict__ down, const float* __re
 
 #if ACM_FFN_MX
 cudaError_t ffn_mx_configure() {
-  return cudaFuncSetAttribute(ACM_FFN_KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  return cudaFuncSetAttribute(ACM_FFN_KERNEL<kMaxNodes>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(Geo<kMaxNodes>::kSmemBytes));
 }
 cudaError_t launch_ffn_mxfp4(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
                              const CUtensorMap& h_map, const CUtensorMap& hs_map, cudaStream_t s) {
 #else
-size_t ffn_smem_bytes() { return kSmemBytes; }
 
 cudaError_t ffn_configure() {
-  return cudaFuncSetAttribute(ACM_FFN_KERNEL, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes));
+  cudaError_t err = cudaFuncSetAttribute(ACM_FFN_KERNEL<kMaxNodes>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(Geo<kMaxNodes>::kSmemBytes));
+  if (err != cudaSuccess) return err;
+  return cudaFuncSetAttribute(ACM_FFN_KERNEL<kWideNodes>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(Geo<kWideNodes>::kSmemBytes));
 }
 
 cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUtensorMap& x_map,
@@ -1296,7 +1328,14 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(L.grid);
   cfg.blockDim = dim3(kThreads);
-  cfg.dynamicSmemBytes = kSmemBytes;
+#if ACM_FFN_MX
+  if (L.n_pad > kMaxNodes) return cudaErrorInvalidValue;
+  const bool wide = false;
+#else
+  const bool wide = L.n_pad > kMaxNodes;       // a batch with more than 64 nodes: 128-column accumulators
+  if (L.n_pad > kWideNodes) return cudaErrorInvalidValue;
+#endif
+  cfg.dynamicSmemBytes = wide ? Geo<kWideNodes>::kSmemBytes : Geo<kMaxNodes>::kSmemBytes;
   cfg.stream = s;
   // The CTAs wait on one another, so all of them must be resident: one CTA per SM on an otherwise
   // idle GPU is, and a cooperative launch makes the driver check it.  A dependent launch cannot be
@@ -1311,7 +1350,12 @@ cudaError_t launch_ffn_bf16(const FfnLaunch& L, const FfnMaps& maps, const CUten
   }
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(ACM_FFN_KERNEL), args);
+#if ACM_FFN_MX
+  return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(ACM_FFN_KERNEL<kMaxNodes>), args);
+#else
+  return cudaLaunchKernelExC(&cfg, wide ? reinterpret_cast<const void*>(ACM_FFN_KERNEL<kWideNodes>)
+                                        : reinterpret_cast<const void*>(ACM_FFN_KERNEL<kMaxNodes>), args);
+#endif
 }
 
 #if !ACM_FFN_MX

@@ -628,7 +628,7 @@ __device__ __forceinline__ void publish_routes(uint32_t* act_mask, float* wtab, 
     const unsigned bits = __reduce_or_sync(0xffffffffu, (has && (e >> 5) == wd) ? 1u << (e & 31) : 0u);
     if (lane == wd && bits) atomicOr(act_mask + wd, bits);
   }
-  if (has) wtab[static_cast<size_t>(e) * kMaxNodes + t] = w;
+  if (has) wtab[static_cast<size_t>(e) * kWtabStride + t] = w;
 }
 
 // the same sets OR-ed into a mask in shared memory (what one block of a batch activates by itself)
@@ -825,7 +825,7 @@ k_select_route_batch(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, Bat
 // Routes given by the caller (acm_expert_ffn) -> the FFN kernel's inputs.  One CTA.
 __global__ void __launch_bounds__(512) k_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask,
                                                          float* wtab, int32_t* ready, int T, int E, int k) {
-  for (int i = threadIdx.x; i < kMaxExperts * kMaxNodes; i += blockDim.x) wtab[i] = 0.0f;
+  for (int i = threadIdx.x; i < kMaxExperts * kWtabStride; i += blockDim.x) wtab[i] = 0.0f;
   for (int i = threadIdx.x; i < 2 * kMaxSlots; i += blockDim.x) ready[i] = 0;
   if (threadIdx.x < kMaskWords) act_mask[threadIdx.x] = 0u;
   __syncthreads();
@@ -833,7 +833,7 @@ __global__ void __launch_bounds__(512) k_routes_to_table(const int32_t* idx, con
     const int e = idx[i];
     if (e >= 0 && e < E) {
       atomicOr(act_mask + (e >> 5), 1u << (e & 31));
-      wtab[static_cast<size_t>(e) * kMaxNodes + i / k] = w[i];
+      wtab[static_cast<size_t>(e) * kWtabStride + i / k] = w[i];
     }
   }
 }

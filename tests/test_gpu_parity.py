@@ -754,6 +754,59 @@ def test_mxfp4_layer_equals_the_bf16_layer_with_the_dequantised_weights(shape):
     ctx.close()
 
 
+def test_mxfp4_scale_bytes_up_to_the_limit_and_beyond():
+    """E8M0 scale bytes up to 128 (block scale 2) are exact; a tensor with a larger one is refused when it is
+    registered, on the device path and on the pool's host path, instead of computing something else."""
+    cfg = wl.scaled(wl.CONFIGS[3], n_layers=1, inter=256, n_experts=32)
+    w = wl.layer_weights_mxfp4(cfg, 0, DEV)
+    rng = np.random.default_rng(3)
+    x = wl.hidden_states(cfg, 0, DEV)
+    alpha = acm.node_weights(wl.tree_depths(cfg), wl.commitment_table(cfg))
+    ctx = _ctx(cfg, n_layers=2)
+    for names in (("gate_up_scales",), ("gate_up_scales", "down_scales")):
+        for name in names:                                  # a few hundred blocks at the largest supported scales
+            sc = w[name].view(-1)
+            pick = torch.tensor(rng.choice(sc.numel(), 300, replace=False), device=sc.device)
+            sc[pick] = torch.tensor(rng.integers(126, 129, 300), dtype=torch.uint8, device=sc.device)
+        w["gate_up_tiles"] = acm.pack_mxfp4_gate_up(w["gate_up_codes"], w["gate_up_scales"]).to(DEV)
+        w["down_tiles"] = acm.pack_mxfp4_down(w["down_codes"], w["down_scales"]).to(DEV)
+        gu = torch.tensor(oracle.dequantize_mxfp4(w["gate_up_codes"], w["gate_up_scales"])).to(torch.bfloat16)
+        dn = torch.tensor(oracle.dequantize_mxfp4(w["down_codes"], w["down_scales"])).to(torch.bfloat16)
+        assert float(gu.abs().max()) >= 4.0                  # (the large scales are really in there)
+        ctx.set_layer_weights_mxfp4(0, w["w_router"], w["router_bias"], w["gate_up_tiles"], w["down_tiles"])
+        ctx.set_layer_weights(1, w["w_router"], w["router_bias"], gu.to(DEV), dn.to(DEV))
+        out, idx, wt, mask, stats = ctx.moe_verify(0, x, alpha.to(DEV), want=True)
+        ref_out = ctx.moe_verify(1, x, alpha.to(DEV))
+        assert ctx.device_status() == acm.OK
+        # the expansion is exact: the bf16 kernel on the dequantised weights does the same arithmetic
+        rms = float(ref_out.double().pow(2).mean().sqrt())
+        assert float((out - ref_out).abs().max()) <= 1e-3 * rms
+        if len(names) == 1:
+            # against the oracle where the sum is well conditioned (with huge down weights too, terms of +-10^4 cancel
+            # and the activations' rounding to bf16, which the tolerance allows for, is amplified)
+            # ... and row by row: a few hundred weights are 256 times the others, so a row's size depends on which of
+            # them its experts hold; each row within the tolerance of its own (or the layer's) RMS
+            ffn = oracle.expert_ffn(x, idx.cpu().numpy(), wt.cpu().numpy(), gu, dn)
+            got = out.double().cpu().numpy()
+            row_rms = np.maximum(np.sqrt(np.mean(ffn ** 2, axis=1)), float(np.sqrt(np.mean(ffn ** 2))))
+            assert (np.abs(got - ffn).max(axis=1) <= FFN_TOL * row_rms).all()
+    # one byte beyond the limit
+    bad = w["down_scales"].clone()
+    bad.view(-1)[12345] = 129
+    bad_tiles = acm.pack_mxfp4_down(w["down_codes"], bad).to(DEV)
+    with pytest.raises(acm.AcmError) as e:
+        ctx.set_layer_weights_mxfp4(0, w["w_router"], w["router_bias"], w["gate_up_tiles"], bad_tiles)
+    assert e.value.code == acm.ERR_UNSUPPORTED
+    ctx.set_layer_weights_mxfp4(0, w["w_router"], w["router_bias"], None, None)
+    X = 8
+    pool_gu = torch.zeros((X,) + tuple(w["gate_up_tiles"].shape[1:]), dtype=torch.uint8, device=DEV)
+    pool_dn = torch.zeros((X,) + tuple(w["down_tiles"].shape[1:]), dtype=torch.uint8, device=DEV)
+    with pytest.raises(acm.AcmError) as e:
+        ctx.set_slot_pool(0, pool_gu, pool_dn, w["gate_up_tiles"].cpu().pin_memory(), bad_tiles.cpu().pin_memory(), [0, 1])
+    assert e.value.code == acm.ERR_UNSUPPORTED
+    ctx.close()
+
+
 def test_multi_block_batch_on_an_mxfp4_layer():
     """The batch call on an MXFP4 layer: per-block sets and routes as on the bf16 layer with the dequantised
     weights, output rows within tolerance of the oracle."""
@@ -855,3 +908,48 @@ def test_batch_call_on_random_block_partitions():
         ffn = oracle.expert_ffn(x, ref_idx, ref_w, w["gate_up"], w["down"], w["shared_gate_up"], w["shared_down"])
         _ffn_check(out, ffn, f"random batch {case}")
         ctx.close()
+
+
+@pytest.mark.parametrize("c,sizes", [(3, [64, 64]), (3, [64, 37]), (4, [48, 48, 20]), (2, [32, 32, 32, 32]), (3, [50, 30])])
+def test_wide_batch_shares_one_pass_over_the_experts(c, sizes):
+    """More than 64 nodes in one batch call (up to 128: two full 64-node blocks): the FFN kernel then runs with
+    128-column accumulators, two 64 KB stages and an epilogue that takes the columns in two halves.  Every block's
+    set and routes are those of the oracle on that block alone, every output row is within tolerance, and each
+    activated expert is streamed once for all blocks.  Twice in a row on the same context."""
+    cfg = wl.CONFIGS[c]
+    ctx = _ctx(cfg)
+    w = wl.layer_weights(cfg, 0, DEV)
+    _set_weights(ctx, w, 0)
+    offsets = [0] + list(np.cumsum(sizes))
+    T = offsets[-1]
+    rng = np.random.default_rng(sum(sizes))
+    xs, depths = [], []
+    for b, n in enumerate(sizes):
+        xs.append(wl.hidden_states(wl.scaled(cfg, n_nodes=64), 70 + b, DEV)[:n])
+        d = np.sort(rng.integers(1, cfg.max_depth + 1, size=n - 1))
+        depths.append(torch.tensor(np.concatenate([[0], d]), dtype=torch.int32))
+    x = torch.cat(xs).contiguous()
+    alpha_ref, refs = _batch_reference(cfg, w, x, offsets, torch.cat(depths), {})
+    alpha = torch.tensor(alpha_ref, device=DEV)
+    ref_idx = np.concatenate([r["idx"] for r in refs])
+    ref_w = np.concatenate([r["w"] for r in refs])
+    ffn = oracle.expert_ffn(x, ref_idx, ref_w, w["gate_up"], w["down"], w["shared_gate_up"], w["shared_down"])
+    for rep in range(2):
+        out, idx, wt, mask, act, stats = ctx.moe_verify_batch(0, x, offsets, alpha, acm.SelectParams(), want=True)
+        assert ctx.device_status() == acm.OK, ctx.wait_report()
+        union = set()
+        for b, ref in enumerate(refs):
+            lo, hi = offsets[b], offsets[b + 1]
+            np.testing.assert_array_equal(_u32(mask[b]), ref["mask"])
+            np.testing.assert_array_equal(idx[lo:hi].cpu().numpy(), ref["idx"])
+            np.testing.assert_allclose(wt[lo:hi].cpu().numpy(), ref["w"], rtol=1e-5, atol=1e-7)
+            union |= set(ref["idx"].ravel().tolist()) - {-1}
+        assert mask_to_set(_u32(act), cfg.n_experts) == union
+        assert out.shape == (T, cfg.hidden)
+        _ffn_check(out, ffn, f"C{c} wide batch {sizes}")
+    # the limits: more than 128 rows in all, or a block beyond the context's own limit
+    with pytest.raises(acm.AcmError):
+        ctx.moe_verify_batch(0, torch.cat([x, x])[:130].contiguous(), [0, 64, 128, 130], torch.ones(130, device=DEV))
+    with pytest.raises(acm.AcmError):
+        ctx.moe_verify_batch(0, x[:70].contiguous(), [0, 70], torch.ones(70, device=DEV))
+    ctx.close()
