@@ -64,6 +64,9 @@ def parse_args():
     ap.add_argument("--batch", type=int, default=0,
                     help="supplementary run: B > 1 verification blocks per call (they share the config's nodes and "
                          "one pass over the expert weights) against the same blocks verified one call each")
+    ap.add_argument("--batch-nodes", type=int, default=0,
+                    help="with --batch: nodes of all blocks together (default: the configuration's; up to 128, e.g. "
+                         "--batch 2 --batch-nodes 128 = two full 64-node blocks per call)")
     ap.add_argument("--pool", type=int, default=0,
                     help="supplementary run: config-5-shaped layers (Zipf-biased routing) behind an LRU expert pool "
                          "of this many slots per layer; reports hit rate and host-to-device MiB per block")
@@ -745,8 +748,11 @@ def run_batch(args):
     torch.cuda.set_device(dev)
     cfg = wl.CONFIGS[args.config]
     L, B = args.layers or cfg.n_layers, args.batch
+    if args.batch_nodes:
+        cfg = wl.scaled(cfg, n_nodes=args.batch_nodes)        # the blocks' nodes together (each block at most 64)
     T, H, E, k = cfg.n_nodes, cfg.hidden, cfg.n_experts, cfg.top_k
     ctx = acm.Context.for_config(cfg, n_layers=L)
+    ctx.set_overlap(args.overlap)
     keep = []
     for l in range(L):
         w = wl.layer_weights(cfg, l, dev)

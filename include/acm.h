@@ -217,8 +217,9 @@ acm_status acm_moe_verify(acm_ctx* ctx, int layer, const void* x, int T, const f
  * same layer step for several verification blocks that share one pass over the expert weights).  The
  * blocks' nodes are stacked along the node axis: block b owns rows block_offsets[b] ..
  * block_offsets[b+1]-1 of x [T,hidden], alpha [T], out, idx_out, w_out (T = block_offsets[n_blocks] <=
- * 64; block_offsets is a HOST array of n_blocks+1 ascending entries starting at 0; every block has at
- * least one node and its first row is its root).  Stages 1-3 run per block exactly as in
+ * 128, every block at most max_nodes <= 64 rows -- two full blocks fit; block_offsets is a HOST array of
+ * n_blocks+1 ascending entries starting at 0; every block has at least one node and its first row is its
+ * root; MXFP4 layers: T <= 64).  Stages 1-3 run per block exactly as in
  * acm_moe_verify: block b's eligible set comes from its own nodes (Eq. 3-7) and its nodes are routed
  * inside it (Eq. 2), so every per-block result equals that of a single-block call on the block's rows.
  * Stage 4 runs once over all rows: an expert activated by several blocks is streamed from HBM once.
