@@ -2,7 +2,7 @@
 
 The kernels of a fused call hand data to one another through tagged words, counters and barriers, every wait
 on which is bounded.  The soak test drives hundreds of fused and batch calls -- fresh and reused contexts,
-1 to 32 blocks of ragged sizes, bursts without a host synchronisation, bf16 and MXFP4 layers -- and checks the
+1 to 32 blocks of ragged sizes, batches of up to 128 nodes, bursts without a host synchronisation, bf16 and MXFP4 layers -- and checks the
 device status and the oracle's eligible sets and routes on every call.  The failure test makes one wait run
 out on purpose (on the host side: a tag that nobody publishes) and checks that the library reports it,
 returns promptly and is correct again afterwards."""
@@ -29,16 +29,23 @@ def _host_bits(t):
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
-def _random_case(rng, cfg, many_blocks):
-    """A random batch: T nodes cut into nb blocks, per-block depths (root first), hidden states."""
-    if many_blocks:
-        nb = int(rng.integers(9, 33))
-        T = int(rng.integers(nb, 65))
-    else:
-        T = int(rng.integers(1, 65))
-        nb = int(rng.integers(1, min(T, 8) + 1))
-    cuts = sorted(rng.choice(np.arange(1, T), size=nb - 1, replace=False).tolist()) if nb > 1 else []
-    offsets = [0] + cuts + [T]
+def _random_case(rng, cfg, many_blocks, wide=False):
+    """A random batch: T nodes cut into nb blocks, per-block depths (root first), hidden states.  wide: more than 64
+    nodes in all (the FFN kernel's 128-column form), no block above 64."""
+    while True:
+        if wide:
+            T = int(rng.integers(65, 129))
+            nb = int(rng.integers(2, 9))
+        elif many_blocks:
+            nb = int(rng.integers(9, 33))
+            T = int(rng.integers(nb, 65))
+        else:
+            T = int(rng.integers(1, 65))
+            nb = int(rng.integers(1, min(T, 8) + 1))
+        cuts = sorted(rng.choice(np.arange(1, T), size=nb - 1, replace=False).tolist()) if nb > 1 else []
+        offsets = [0] + cuts + [T]
+        if max(np.diff(offsets)) <= 64:
+            break
     depths = []
     for b in range(nb):
         n = offsets[b + 1] - offsets[b]
@@ -86,7 +93,7 @@ def _check_burst(ctx, cfg, w_ffn, pending, what):
         assert np.isfinite(got).all() and float(np.abs(got - ffn).max()) <= 2e-2 * rms, what
 
 
-def _soak(cfg, layers, ffn_weights, set_weights, n_rounds, calls_per_round, seed):
+def _soak(cfg, layers, ffn_weights, set_weights, n_rounds, calls_per_round, seed, wide_ok=True):
     rng = np.random.default_rng(seed)
     p = wl.commitment_table(cfg)
     gen = torch.Generator(device=DEV).manual_seed(seed)
@@ -102,7 +109,8 @@ def _soak(cfg, layers, ffn_weights, set_weights, n_rounds, calls_per_round, seed
             cases = []
             for j in range(burst):            # inputs and references of the whole burst first ...
                 layer = int(rng.integers(0, len(layers)))
-                T, nb, offsets, depths = _random_case(rng, cfg, many_blocks=((i + j) % 4 == 3))
+                T, nb, offsets, depths = _random_case(rng, cfg, many_blocks=((i + j) % 4 == 3),
+                                                      wide=wide_ok and (i + j) % 4 == 1)
                 x = torch.randn(T, cfg.hidden, generator=gen, device=DEV).to(torch.bfloat16)
                 alpha, refs = _reference(cfg, layers[layer], x, offsets, depths, p)
                 single = nb == 1 and bool(rng.integers(0, 2))
@@ -157,7 +165,7 @@ def test_soak_fused_and_batch_calls_mxfp4():
 
     host_w = dict(w_router=_host_bits(w["w_router"]), router_bias=w["router_bias"].cpu().numpy(), gate_up=None, down=None)
     assert _soak(cfg, [host_w], [(_host_bits(gu), _host_bits(dn))], set_weights, n_rounds=1, calls_per_round=100,
-                 seed=12) == 100
+                 seed=12, wide_ok=False) == 100
 
 
 def test_wait_that_runs_out_is_reported_and_the_context_recovers():
