@@ -52,9 +52,9 @@ struct Workspace {
   int32_t* ready;       // [2][kMaxSlots] finished gate/up tiles per activated slot
   int32_t* status;      // [1] sticky device-side status
   int32_t* tile_done;   // [64] router kernel: expert tiles finished per node tile (self-resetting)
-  int32_t* ticket;      // [1] select/route kernel: finished CTAs (self-resetting)
+  int32_t* ticket;      // [4] spare words (the MXFP4 scale check keeps its maximum in one)
   uint32_t* sel_words;  // [kMaxEarlyBlocks][8] the eligible masks as tagged 16-bit pieces (early start of the FFN kernel)
-  uint32_t* anc_words;  // [kMaxEarlyBlocks][8] the anchor experts (each root's natural top-k) as tagged 16-bit pieces, published by the router kernel
+  uint32_t* anc_words;  // [kMaxEarlyBlocks][8] the anchor experts (each root's natural top-k) as tagged 16-bit pieces, published by the selection kernel first thing
 };
 
 struct SelectArgs {
@@ -77,12 +77,7 @@ struct BatchDesc {
   int n_blocks;
   int off[kMaxNodes + 1];    // (at most 64 blocks, at most kWideNodes rows in all, at most kMaxNodes rows a block)
 };
-constexpr int kMaxEarlyBlocks = 8;
-// The rows whose natural top-k the router kernel publishes as anchors (the blocks' roots; one for a single block).
-struct RootList {
-  int n;
-  int row[kMaxEarlyBlocks];
-};   // blocks whose eligible sets the FFN kernel can poll for (8 tagged words each)
+constexpr int kMaxEarlyBlocks = 8;   // blocks whose eligible sets the FFN kernel can poll for (8 tagged words each)
 
 struct RouteArgs {
   const float* logits;
@@ -94,10 +89,8 @@ struct RouteArgs {
   // inputs of the FFN kernel (all null when only the routes are wanted); zero on entry
   uint32_t* act_mask;            // [4] activated experts, OR-ed into
   float* wtab;                   // [kMaxExperts][kWtabStride] combine weights by (expert, node)
-  // The CTA that finishes last can also report on the whole block (it needs a ticket, so only when asked):
-  int32_t* ticket;               // zero-initialised counter, left at zero; null: no report
+  // the block's own report (single block):
   const uint32_t* resident;      // non-null: activated experts outside it are "staged"
-  acm_block_stats* stats_out;    // n_activated / n_staged are filled in
   int32_t* host_stage_list;      // mapped pinned memory (may be null): [0] = n_stage, [1..] = staged expert ids,
                                  // [1 + kMaxExperts ..] = the activated mask (4 words)
   uint32_t* sel_flag;            // non-null: [8] words, the eligible mask in 16-bit pieces tagged with sel_epoch
@@ -121,19 +114,19 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
                                  float* logits, int T, int H, int E, float* zero_buf,
                                  size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status,
                                  float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k, int32_t* tile_done,
-                                 bool pdl, cudaStream_t s, long long* dbg = nullptr, uint32_t* anc_words = nullptr,
-                                 uint32_t anc_tag = 0, const RootList* roots = nullptr);
+                                 bool pdl, cudaStream_t s, long long* dbg = nullptr);
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s);
-// select (unless mask_override) + route + the FFN kernel's routing inputs in ONE launch of ceil(T/4)
-// small CTAs; `nat_mask` = the natural top-k sets as bit masks [T][4] (from launch_router_logits)
-cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
-                                const uint32_t* mask_override, int T, int E, int k, bool pdl, cudaStream_t s);
-int route_ctas(int T);   // grid size of launch_select_route
-// the same for a batch of blocks: one CTA per block; the per-block outputs of `sa` (mask, unpruned, count,
-// demand [kMaxExperts each], stats) are arrays over the blocks, ra.sel_flag holds 8 words per block
-cudaError_t launch_select_route_batch(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
-                                      const BatchDesc& bd, int E, int k, bool pdl, cudaStream_t s);
+// The fused calls' stages 1b-3 in ONE launch, a cluster of select_ctas_per_block(widest block) CTAs per block of `bd`
+// (a single block: n_blocks = 1, off = {0, T}): softmax and natural top-k of the logits in ra.logits, selection
+// (unless mask_override, single block only), routes, the FFN kernel's routing inputs.  The per-block outputs of `sa`
+// (mask, unpruned, count, demand [kMaxExperts each], stats) are arrays over the blocks; ra.sel_flag and anc_words
+// (both may be null) hold 8 tagged words per block: the eligible set and, earlier, the anchors (the natural top-k
+// of the block's first row).
+int select_ctas_per_block(int widest);
+cudaError_t launch_softmax_select_route(const SelectArgs& sa, const RouteArgs& ra, const BatchDesc& bd,
+                                        const uint32_t* mask_override, uint32_t* anc_words, int E, int k, bool pdl,
+                                        cudaStream_t s);
 // routes given by the caller -> activated mask, weight table (both cleared first) and cleared `ready`
 cudaError_t launch_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask, float* wtab,
                                    int32_t* ready, int T, int E, int k, cudaStream_t s);
@@ -167,7 +160,7 @@ struct FfnLaunch {
   int32_t sel_epoch;
   int sel_blocks;            // blocks of a batch (1..kMaxEarlyBlocks): eight words each, the work list is their union
   const uint32_t* anc_flag = nullptr;   // with sel_flag: eight words tagged alike holding the anchor experts (published by the
-                             // router kernel, earlier): their gate/up tiles are streamed while the selection still runs
+                             // selection kernel, earlier): their gate/up tiles are streamed while the selection still runs
   float* out;                // [T,H], accumulated into (zeroed by the caller)
   int32_t* status;
   int grid;

@@ -331,7 +331,7 @@ void expert_tensor_bytes(const acm_model_desc& d, bool mx, size_t* gu, size_t* d
 acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li, float* out, cudaStream_t s,
                         const uint32_t* res_dev = nullptr, acm_block_stats* stats_dev = nullptr, bool pdl_ok = false,
                         int32_t early_epoch = 0, const uint32_t* only = nullptr, int n_blocks = 0,
-                        bool anchors_first = false) {
+                        bool anchors_first = false, int widest_block = 0) {
   const acm_model_desc& d = c->desc;
   const int n_pad = (T + 15) / 16 * 16;
   acm_status st = ensure_h_maps(c, n_pad);
@@ -389,7 +389,7 @@ acm_status run_ffn_list(acm_ctx* c, const Layer& L, const void* x, int T, int li
   // Straight after the routing kernel: the few SMs it ran on (or still holds, in an early start) take
   // microseconds longer to accept a CTA of this kernel -- an SM changes hands slowly when the shared-memory
   // split changes -- and one late CTA delays every CTA that exchanges fragments with it.  Leave them out.
-  const int routing_ctas = n_blocks > 0 ? n_blocks : route_ctas(T);   // a batch: one CTA per block
+  const int routing_ctas = (n_blocks > 0 ? n_blocks : 1) * select_ctas_per_block(widest_block > 0 ? widest_block : T);
   if (pdl_ok && c->sm_count > 2 * routing_ctas) p.grid = c->sm_count - routing_ctas;
   c->last_ffn_grid = p.grid;
   if (L.mx) {
@@ -797,9 +797,9 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
     st = next_epoch(c, s, &early_epoch);
     if (st != ACM_OK) return st;
   }
-  // ... and earlier still on the anchors (Eq. 5 with the default anchor, the root): the router kernel publishes
-  // the root's natural top-k as soon as that row is done, the FFN kernel streams their gate/up tiles while
-  // the selection runs.  They are in every eligible set the selection can return without a residency.
+  // ... and earlier still on the anchors (Eq. 5 with the default anchor, the root): the selection kernel publishes
+  // the root's natural top-k as soon as that row's softmax is done, the FFN kernel streams their gate/up tiles
+  // while the selection runs.  They are in every eligible set the selection can return without a residency.
   const bool anchors_first = early && c->anchor_start && prm.use_anchors != 0;
   // offload timing: events around the resident part, the copies and the loaded part of this call
   cudaEvent_t* oev = nullptr;
@@ -807,17 +807,13 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
     oev = c->off_ev.data() + 5 * c->off_calls;
     ACM_CUDA(cudaEventRecord(oev[0], s));
   }
-  // stage 1 (also clears the output the FFN accumulates into and the FFN kernel's routing inputs)
-  const bool need_probs = eligible_mask_override == nullptr;
+  // stage 1a: the logits (the kernel also clears the output the FFN accumulates into and the FFN kernel's
+  // routing inputs)
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
                                 f32 ? 0 : static_cast<size_t>(T) * d.hidden, c->ws.wtab, c->ffn_in_floats,
-                                c->ws.status,
-                                need_probs ? c->ws.probs : nullptr, need_probs ? c->ws.nat_idx : nullptr,
-                                need_probs ? c->ws.nat_mask : nullptr, k, c->ws.tile_done, c->pdl, s,
-                                c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr,
-                                // (published on every early call, used or not: the words never carry an old tag)
-                                early ? c->ws.anc_words : nullptr, static_cast<uint32_t>(early_epoch) & 0xffffu));
-  // stages 2-3: one launch of a few small CTAs, which also fill the FFN kernel's routing inputs
+                                c->ws.status, nullptr, nullptr, nullptr, k, nullptr, c->pdl, s,
+                                c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr));
+  // stages 1b-3: one cluster of CTAs, which also fills the FFN kernel's routing inputs
   SelectArgs sa;
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
   sa.n_anchor_nodes = 0; sa.resident = prm.residency ? res_dev : nullptr; sa.prm = prm;
@@ -830,15 +826,18 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   ra.weighting = d.weighting; ra.routed_scale = d.routed_scale;
   ra.act_mask = c->ws.act_mask; ra.wtab = c->ws.wtab; ra.resident = res_dev;
   ra.host_stage_list = L.has_resident ? c->host_stage_list_dev : nullptr;
-  ra.stats_out = stats_dev;
-  // the bf16 FFN kernel counts the activated experts itself; otherwise the routing kernel's last CTA does
-  ra.ticket = (f32 || L.has_resident) ? c->ws.ticket : nullptr;
   if (early) {
     ra.sel_flag = c->ws.sel_words;
     ra.sel_epoch = early_epoch;
   }
   ra.dbg = c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr;
-  ACM_CUDA(launch_select_route(c->ws.nat_mask, sa, ra, eligible_mask_override, T, E, k, c->pdl, s));
+  BatchDesc one = {};
+  one.n_blocks = 1;
+  one.off[0] = 0;
+  one.off[1] = T;
+  // (the anchors are published on every early call, used or not: the words never carry an old tag)
+  ACM_CUDA(launch_softmax_select_route(sa, ra, one, eligible_mask_override, early ? c->ws.anc_words : nullptr, E, k,
+                                       c->pdl, s));
   c->launches += 2;
 
   if (f32) {
@@ -1010,14 +1009,10 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
   }
   // ... and on the union of the blocks' anchors (each block's first row is its root) while the selections run
   const bool anchors_first = early && c->anchor_start && params->use_anchors != 0;
-  RootList roots = {};
-  roots.n = early ? n_blocks : 0;
-  for (int b = 0; b < roots.n; ++b) roots.row[b] = bd.off[b];
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, out,
                                 static_cast<size_t>(T) * d.hidden, c->ws.wtab, c->ffn_in_floats, c->ws.status,
-                                c->ws.probs, c->ws.nat_idx, c->ws.nat_mask, k, c->ws.tile_done, c->pdl, s, nullptr,
-                                early ? c->ws.anc_words : nullptr, static_cast<uint32_t>(early_epoch) & 0xffffu, &roots));
-  // stages 2-3: one CTA per block
+                                nullptr, nullptr, nullptr, k, nullptr, c->pdl, s, nullptr));
+  // stages 1b-3: one cluster of CTAs per block
   SelectArgs sa;
   sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
   sa.n_anchor_nodes = 0; sa.resident = nullptr; sa.prm = *params;
@@ -1033,10 +1028,12 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
     ra.sel_flag = c->ws.sel_words;
     ra.sel_epoch = early_epoch;
   }
-  ACM_CUDA(launch_select_route_batch(c->ws.nat_mask, sa, ra, bd, E, k, c->pdl, s));
+  ACM_CUDA(launch_softmax_select_route(sa, ra, bd, nullptr, early ? c->ws.anc_words : nullptr, E, k, c->pdl, s));
   c->launches += 2;
   // stage 4 once over all rows: an expert activated by several blocks is streamed once
-  st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, nullptr, true, early_epoch, nullptr, n_blocks, anchors_first);
+  int widest = 1;
+  for (int b = 0; b < n_blocks; ++b) widest = std::max(widest, bd.off[b + 1] - bd.off[b]);
+  st = run_ffn_list(c, L, x, T, 0, out, s, nullptr, nullptr, true, early_epoch, nullptr, n_blocks, anchors_first, widest);
   if (st != ACM_OK) return st;
 
   const size_t tk = static_cast<size_t>(T) * k;

@@ -7,6 +7,7 @@
 // (explicit round-to-nearest intrinsics, so the compiler can neither contract nor reorder):
 // 32 interleaved partial sums + halving tree for the logit dot product, a 128-slot halving
 // tree for sums over the expert axis, fixed polynomial recipes for exp and log.
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 
 #include "acm_internal.h"
@@ -69,19 +70,22 @@ __device__ __forceinline__ unsigned order_key(float z) {
 }
 // One round of a warp-wide top-k over 128 slots (slot e = lane + 32 c, key[c] == 0: not a candidate):
 // returns the slot with the largest key, ties to the lowest slot, or -1 if none is left; the
-// owning lane clears that key.  Two hardware warp reductions per round.
+// owning lane clears that key.  One hardware warp reduction (the maximum) and four independent votes per round: the
+// lowest slot that holds the maximum is in the lowest c that has it anywhere, at the lowest such lane.
 __device__ __forceinline__ int warp_take_best(unsigned (&key)[4], int lane) {
   const unsigned m01 = max(key[0], key[1]), m23 = max(key[2], key[3]);
   const unsigned best = __reduce_max_sync(0xffffffffu, max(m01, m23));
   if (best == 0u) return -1;
-  unsigned mine = 0xffffffffu;   // lowest slot of this lane that holds the best key
-  if (key[3] == best) mine = lane + 96;
-  if (key[2] == best) mine = lane + 64;
-  if (key[1] == best) mine = lane + 32;
-  if (key[0] == best) mine = lane;
-  const unsigned e = __reduce_min_sync(0xffffffffu, mine);
-  if ((e & 31u) == static_cast<unsigned>(lane)) key[e >> 5] = 0u;
-  return static_cast<int>(e);
+  const unsigned h0 = __ballot_sync(0xffffffffu, key[0] == best), h1 = __ballot_sync(0xffffffffu, key[1] == best);
+  const unsigned h2 = __ballot_sync(0xffffffffu, key[2] == best), h3 = __ballot_sync(0xffffffffu, key[3] == best);
+  const int c = h0 ? 0 : h1 ? 1 : h2 ? 2 : 3;
+  const unsigned h = h0 ? h0 : h1 ? h1 : h2 ? h2 : h3;
+  const int l = __ffs(h) - 1;
+  if (l == lane) {
+    key[0] = c == 0 ? 0u : key[0]; key[1] = c == 1 ? 0u : key[1];
+    key[2] = c == 2 ? 0u : key[2]; key[3] = c == 3 ? 0u : key[3];
+  }
+  return 32 * c + l;
 }
 
 // Sum of a 128-slot array held as 4 values per lane (slot = lane + 32 c): the halving tree
@@ -93,18 +97,14 @@ __device__ __forceinline__ float warp_tree_sum_128(float a0, float a1, float a2,
   return __shfl_sync(0xffffffffu, v, 0);
 }
 
-// Stage 1b for ONE node, by one warp: softmax over the expert axis (fixed recipe) and natural
-// top-k ranked on the logits.  `z_row` may have been written by other CTAs: read through L2.
-__device__ void softmax_topk_row(const float* z_row, float* probs_row, int32_t* nat_row, uint32_t* natmask_row,
-                                 int E, int k, int lane) {
-  float z[4], y[4];
+// Stage 1b for ONE node, by one warp, on a logit row held in registers (lane l holds experts l, l + 32, l + 64,
+// l + 96; -inf beyond E): softmax over the expert axis (fixed recipe) and natural top-k ranked on the logits.
+// Returns the probabilities in the same layout and the top-k set as a bit mask (warp-uniform); the ranked ids
+// go to `nat_row` if given.
+__device__ __forceinline__ void softmax_topk_regs(const float (&z)[4], int E, int k, int lane, float (&prob)[4],
+                                                  uint32_t (&bits)[kMaskWords], int32_t* nat_row, bool want_topk) {
+  float y[4];
   unsigned key[4];
-#pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    const int e = lane + 32 * c;
-    const float v = __ldcg(z_row + min(e, E - 1));
-    z[c] = e < E ? v : -INFINITY;
-  }
   float zmax = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
 #pragma unroll
   for (int s = 16; s >= 1; s >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, s));
@@ -115,24 +115,42 @@ __device__ void softmax_topk_row(const float* z_row, float* probs_row, int32_t* 
     key[c] = (lane + 32 * c < E) ? order_key(z[c]) : 0u;
   }
   const float denom = warp_tree_sum_128(y[0], y[1], y[2], y[3]);
-  if (probs_row) {
 #pragma unroll
-    for (int c = 0; c < 4; ++c)
-      if (lane + 32 * c < E) probs_row[lane + 32 * c] = __fdiv_rn(y[c], denom);
-  }
-  if (nat_row) {
-    uint32_t b0 = 0u, b1 = 0u, b2 = 0u, b3 = 0u;      // the same set as a bit mask (warp-uniform)
+  for (int c = 0; c < 4; ++c) prob[c] = __fdiv_rn(y[c], denom);
+  uint32_t b0 = 0u, b1 = 0u, b2 = 0u, b3 = 0u;
+  if (want_topk) {
     for (int j = 0; j < k; ++j) {
       const int e = warp_take_best(key, lane);
-      if (lane == 0) nat_row[j] = e;
+      if (nat_row && lane == 0) nat_row[j] = e;
       if (e >= 0) {
         const uint32_t bit = 1u << (e & 31);
         const int wd = e >> 5;
         b0 |= wd == 0 ? bit : 0u; b1 |= wd == 1 ? bit : 0u; b2 |= wd == 2 ? bit : 0u; b3 |= wd == 3 ? bit : 0u;
       }
     }
-    if (natmask_row && lane < kMaskWords) natmask_row[lane] = lane == 0 ? b0 : lane == 1 ? b1 : lane == 2 ? b2 : b3;
   }
+  bits[0] = b0; bits[1] = b1; bits[2] = b2; bits[3] = b3;
+}
+
+// The same for a row in global memory (`z_row` may have been written by other CTAs: read through L2).
+__device__ void softmax_topk_row(const float* z_row, float* probs_row, int32_t* nat_row, uint32_t* natmask_row,
+                                 int E, int k, int lane) {
+  float z[4], prob[4];
+  uint32_t bits[kMaskWords];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const int e = lane + 32 * c;
+    const float v = __ldcg(z_row + min(e, E - 1));
+    z[c] = e < E ? v : -INFINITY;
+  }
+  softmax_topk_regs(z, E, k, lane, prob, bits, nat_row, nat_row != nullptr);
+  if (probs_row) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+      if (lane + 32 * c < E) probs_row[lane + 32 * c] = prob[c];
+  }
+  if (nat_row && natmask_row && lane < kMaskWords)
+    natmask_row[lane] = lane == 0 ? bits[0] : lane == 1 ? bits[1] : lane == 2 ? bits[2] : bits[3];
 }
 
 // ------------------------------------------------------------------------------------------
@@ -194,7 +212,7 @@ __global__ void __launch_bounds__(kRT * kRE * (32 / ElemTraits<Elem>::EPT))
 k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const float* __restrict__ bias,
                 float* logits, int T, int H, int E, int n_chunks, float* zero_buf,
                 size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status, float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k,
-                int32_t* tile_done, long long* dbg, uint32_t* anc_words, uint32_t anc_tag, RootList roots) {
+                int32_t* tile_done, long long* dbg) {
   constexpr int EPT = ElemTraits<Elem>::EPT;
   constexpr int Q = 32 / EPT;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -317,21 +335,6 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
           softmax_topk_row(logits + static_cast<size_t>(t) * E, probs ? probs + static_cast<size_t>(t) * E : nullptr,
                            nat_idx ? nat_idx + static_cast<size_t>(t) * k : nullptr,
                            nat_mask ? nat_mask + static_cast<size_t>(t) * kMaskWords : nullptr, E, k, lane);
-        if (anc_words && nat_mask && t < T) {
-          // A root's natural top-k are anchors (Eq. 5), eligible whatever the selection decides: published at
-          // once, as eight words of 16 mask bits under the call's tag, for the FFN kernel to start on (one group
-          // of eight words per block of a batch).
-          int which = -1;
-          for (int b = 0; b < roots.n; ++b) which = roots.row[b] == t ? b : which;
-          if (which >= 0) {
-            __syncwarp();
-            if (lane < 2 * kMaskWords) {
-              const uint32_t bits = (nat_mask[static_cast<size_t>(t) * kMaskWords + (lane >> 1)] >> (16 * (lane & 1))) & 0xffffu;
-              asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(anc_words + 2 * kMaskWords * which + lane),
-                           "r"(bits | (anc_tag << 16)) : "memory");
-            }
-          }
-        }
       }
     }
   }
@@ -339,10 +342,9 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
 
 // ------------------------------------------------------------------------------------------
 // Stages 2 and 3.  The selection is a decision over the whole block (the demand sums over every
-// node), the routing is per node.  Rather than one CTA doing both for 64 nodes, a small grid runs
-// them: EVERY CTA repeats the selection on its 128 threads (it is deterministic, so all of them
-// hold the same S'), then routes its own four nodes, one warp each; the CTA that finishes last
-// gathers the routes into the FFN work lists.
+// node) taken by 128 threads, one per expert slot; the routing is per node, one warp each.  The stand-alone
+// entry points run them as kernels of their own; the fused calls run both behind the softmax in one CTA per
+// block (k_softmax_select_route).
 // ------------------------------------------------------------------------------------------
 constexpr int kNodesPerCta = 4;
 constexpr int kSelThreads = 128;
@@ -384,41 +386,47 @@ __device__ float sel_tree_sum_128(float* tree, float mine) {
 }
 
 // Stage 2: demand, anchors, self-sizing, pruning.  Called by threads 0..127; thread e owns expert e.
-// r comes straight from global memory (every load is issued before the first wait); the natural
+// kStaged = false: r comes straight from global memory (every load is issued before the first wait); the natural
 // top-k sets come as bit masks from `natmask_g` ([T][4], written by the router kernel) or, if that
-// is null, are built here from a.nat_idx.  Global results are written only if `write_out`.
+// is null, are built here from a.nat_idx.  kStaged = true: the caller has put the probabilities in shared memory
+// (`s_probs`, [T][E]) and filled sm.alpha and sm.natmask (rows >= T zero) before a CTA-wide barrier.
+// Global results are written only if `write_out`.
+template <bool kStaged>
 __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, int k, const uint32_t* natmask_g,
-                             bool write_out, uint32_t* publish_words = nullptr, uint32_t publish_tag = 0) {
+                             bool write_out, uint32_t* publish_words = nullptr, uint32_t publish_tag = 0,
+                             const float* s_probs = nullptr) {
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   const bool live = tid < E;
-  // small loads first (they gate the first barrier), then the 64 probabilities of this expert's column
-  const float my_alpha = tid < kMaxNodes ? a.alpha[min(tid, T - 1)] : 0.0f;
-  uint32_t my_nm[2] = {0u, 0u};
-  if (natmask_g) {
+  float pr[kStaged ? 1 : kMaxNodes];
+  if constexpr (!kStaged) {
+    // small loads first (they gate the first barrier), then the 64 probabilities of this expert's column
+    const float my_alpha = tid < kMaxNodes ? a.alpha[min(tid, T - 1)] : 0.0f;
+    uint32_t my_nm[2] = {0u, 0u};
+    if (natmask_g) {
 #pragma unroll
-    for (int i = 0; i < 2; ++i) my_nm[i] = __ldcg(natmask_g + min(tid + i * kSelThreads, T * kMaskWords - 1));
-  }
-  float pr[kMaxNodes];
-  {
-    const float* col = a.probs + min(tid, E - 1);
+      for (int i = 0; i < 2; ++i) my_nm[i] = __ldcg(natmask_g + min(tid + i * kSelThreads, T * kMaskWords - 1));
+    }
+    {
+      const float* col = a.probs + min(tid, E - 1);
 #pragma unroll
-    for (int t = 0; t < kMaxNodes; ++t) pr[t] = __ldcg(col + static_cast<size_t>(min(t, T - 1)) * E);
-  }
-  if (tid < kMaxNodes) sm.alpha[tid] = my_alpha;
-  if (tid < kMaskWords) sm.Hres[tid] = (tid < (E + 31) / 32) ? (a.resident ? a.resident[tid] : 0xffffffffu) : 0u;
-  if (tid < 8) sm.scal[tid] = 0;
-  if (natmask_g) {
+      for (int t = 0; t < kMaxNodes; ++t) pr[t] = __ldcg(col + static_cast<size_t>(min(t, T - 1)) * E);
+    }
+    if (tid < kMaxNodes) sm.alpha[tid] = my_alpha;
+    if (natmask_g) {
 #pragma unroll
-    for (int i = 0; i < 2; ++i) (&sm.natmask[0][0])[tid + i * kSelThreads] = my_nm[i];
-  } else {
-    for (int i = tid; i < kMaxNodes * kMaskWords; i += kSelThreads) (&sm.natmask[0][0])[i] = 0u;
-    sel_sync();
-    for (int i = tid; i < T * k; i += kSelThreads) {
-      const int e = a.nat_idx[i];
-      if (e >= 0 && e < E) atomicOr(&sm.natmask[i / k][e >> 5], 1u << (e & 31));
+      for (int i = 0; i < 2; ++i) (&sm.natmask[0][0])[tid + i * kSelThreads] = my_nm[i];
+    } else {
+      for (int i = tid; i < kMaxNodes * kMaskWords; i += kSelThreads) (&sm.natmask[0][0])[i] = 0u;
+      sel_sync();
+      for (int i = tid; i < T * k; i += kSelThreads) {
+        const int e = a.nat_idx[i];
+        if (e >= 0 && e < E) atomicOr(&sm.natmask[i / k][e >> 5], 1u << (e & 31));
+      }
     }
   }
+  if (tid < kMaskWords) sm.Hres[tid] = (tid < (E + 31) / 32) ? (a.resident ? a.resident[tid] : 0xffffffffu) : 0u;
+  if (tid < 8) sm.scal[tid] = 0;
   sel_sync();
   if (tid < kMaskWords) {           // anchors (Eq. 5): union of the anchor nodes' natural sets
     uint32_t A = 0u;
@@ -436,6 +444,33 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   int votes = 0;
   float u = 0.0f;
   const int demand_mode = a.prm.demand;
+  if constexpr (kStaged) {
+    // (a rolled loop of eight nodes a turn: in the fused kernel the code is fetched while the FFN kernel streams
+    // weights, and every further line of straight-line code is one more slow instruction fetch)
+    const float* pcol = s_probs + min(tid, E - 1);
+#pragma unroll 1
+    for (int t0 = 0; t0 < T; t0 += 8) {
+      float al[8], pj[8];
+      unsigned in_mask = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int t = min(t0 + j, T - 1);
+        al[j] = sm.alpha[t];
+        pj[j] = pcol[t * E];
+        in_mask |= ((sm.natmask[t][warp] >> lane) & 1u) << j;
+      }
+      const unsigned valid = t0 + 8 > T ? (1u << (T - t0)) - 1u : 0xffu;
+      in_mask &= valid;
+      votes += __popc(in_mask);
+      const unsigned take = demand_mode == ACM_DEMAND_FULL_MASS ? valid
+                          : demand_mode == ACM_DEMAND_TOPK_MASS ? in_mask : 0u;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float nu = __fmaf_rn(al[j], pj[j], u);
+        u = ((take >> j) & 1u) ? nu : u;
+      }
+    }
+  } else {
 #pragma unroll
   for (int t0 = 0; t0 < kMaxNodes; t0 += 16) {
     if (t0 < T) {
@@ -459,6 +494,7 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
         u = ((take >> j) & 1u) ? nu : u;
       }
     }
+  }
   }
   if (!live) { votes = 0; u = 0.0f; }
   if (a.prm.demand == ACM_DEMAND_VOTES) u = static_cast<float>(votes);
@@ -619,19 +655,7 @@ __device__ __forceinline__ void load_logit_row(const float* logits, int t, int E
   }
 }
 
-// Publishes one node's routes (lane j < k holds choice j) to the FFN kernel's inputs: the activated
-// mask (one OR per touched word) and the weight table.
-__device__ __forceinline__ void publish_routes(uint32_t* act_mask, float* wtab, int t, int k, int lane, int e, float w) {
-  const bool has = lane < k && e >= 0;
-#pragma unroll
-  for (int wd = 0; wd < kMaskWords; ++wd) {
-    const unsigned bits = __reduce_or_sync(0xffffffffu, (has && (e >> 5) == wd) ? 1u << (e & 31) : 0u);
-    if (lane == wd && bits) atomicOr(act_mask + wd, bits);
-  }
-  if (has) wtab[static_cast<size_t>(e) * kWtabStride + t] = w;
-}
-
-// the same sets OR-ed into a mask in shared memory (what one block of a batch activates by itself)
+// One node's routes (lane j < k holds choice j) OR-ed into a mask in shared memory (what one block activates)
 __device__ __forceinline__ void publish_routes_local(uint32_t* s_act, int k, int lane, int e) {
   const bool has = lane < k && e >= 0;
 #pragma unroll
@@ -643,7 +667,7 @@ __device__ __forceinline__ void publish_routes_local(uint32_t* s_act, int k, int
 
 __global__ void __launch_bounds__(kSelThreads) k_select(SelectArgs a, int T, int E, int k) {
   __shared__ StageSmem sm;
-  stage_select(a, sm, T, E, k, nullptr, true);
+  stage_select<false>(a, sm, T, E, k, nullptr, true);
 }
 
 // grid = ceil(T / 4) CTAs of four warps, one node per warp
@@ -676,71 +700,143 @@ __device__ __forceinline__ void publish_eligible(const RouteArgs& ra, const Stag
 }
 
 #define ACM_RT(slot) do { if (ra.dbg && blockIdx.x == 0 && threadIdx.x == 0) ra.dbg[slot] = time_ns(); } while (0)
-// Stages 2-3 and the FFN kernel's routing inputs in one launch of a few CTAs (see the note above):
-// one warp per node, up to 16 nodes per CTA; warps 0-3 of every CTA run the selection.  Few CTAs on
-// purpose: the FFN kernel, launched as a dependent, can take over an SM only once this kernel has left it.
-constexpr int kRouteNodesPerCta = 16;
-__global__ void __launch_bounds__(32 * kRouteNodesPerCta)
-k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uint32_t* mask_override, int T, int E,
-               int k) {
-  __shared__ StageSmem sm;
-  __shared__ int s_last;
+// Stages 1b-3 of the fused calls and the FFN kernel's routing inputs in ONE launch: a cluster of up to four CTAs
+// per verification block (block b = the rows bd.off[b] .. bd.off[b+1]-1 of every per-node array; a single block is a
+// batch of one), sixteen warps each, ONE ROW PER WARP -- softmax + top-k of a row is a chain of a few hundred
+// dependent instructions, so the rows are spread over as many warps and SMs as it takes to give each its own.  The
+// router kernel before it has written the logits only.  Every warp loads its row (the one trip through L2 of the
+// whole chain: with the FFN kernel already streaming weights, each further one would cost well over a microsecond),
+// then
+//   1b  softmax and natural top-k of the row (Eq. 1); the probabilities and the top-k mask go into the shared memory
+//       of EVERY CTA of the cluster (distributed shared memory), the logits stay in registers; the block's first row
+//       is its root, whose natural top-k are anchors (Eq. 5) and published at once as eight tagged words for the FFN
+//       kernel to start on;
+//   --  cluster barrier: every CTA now holds the whole block's probabilities and natural sets
+//   2   the selection (Eq. 3-7; it sees nothing of the other blocks), repeated by warps 0-3 of every CTA -- it is
+//       deterministic, so all hold the same S' and no second exchange is needed; the cluster's first CTA writes the
+//       outputs and publishes the eligible set as eight tagged words, ra.sel_flag + 8 b;
+//   3   the row's routes inside that set (Eq. 2).
+// The FFN kernel's inputs are shared by all blocks: the activated mask is OR-ed into by every CTA, the weight table
+// is indexed by the row in the stacked batch.  The CTAs ask for more shared memory than they use so that no CTA of
+// the FFN kernel (launched as a dependent while this one runs) fits beside them: its polling and streaming would
+// slow the selection by half.
+namespace cg = cooperative_groups;
+constexpr int kFusedWarps = 16;
+constexpr int kFusedMaxCtas = 4;
+constexpr size_t kFusedSmemRequest = 100u << 10;
+struct FusedSmem {
+  StageSmem st;
+  alignas(16) float probs[kMaxNodes * kMaxExperts];   // [T][E], every row written by the warp (of some CTA) that owns it
+  uint32_t act[kMaskWords];                             // experts this CTA's rows activate (first CTA: the block's)
+};
+static_assert(sizeof(FusedSmem) <= kFusedSmemRequest, "shared memory of the selection kernel");
+__global__ void __launch_bounds__(32 * kFusedWarps)
+k_softmax_select_route(SelectArgs sa, RouteArgs ra, BatchDesc bd, const uint32_t* mask_override, uint32_t* anc_words,
+                       int E, int k) {
+  extern __shared__ __align__(16) unsigned char fused_raw[];
+  FusedSmem& fs = *reinterpret_cast<FusedSmem*>(fused_raw);
+  StageSmem& sm = fs.st;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int C = static_cast<int>(cluster.num_blocks()), q = static_cast<int>(cluster.block_rank());
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int t_mine = blockIdx.x * (blockDim.x >> 5) + warp;
+  const int b = blockIdx.x / C, t_lo = bd.off[b], T = bd.off[b + 1] - t_lo;
+  const int r = q * kFusedWarps + warp;                 // this warp's row of the block
+  const bool first = q == 0;
+  const bool report = sa.stats_out != nullptr || ra.host_stage_list != nullptr;
+  const uint32_t tag = static_cast<uint32_t>(ra.sel_epoch) & 0xffffu;
   griddep_launch_dependents();
+  if (tid < kMaskWords) fs.act[tid] = 0u;
+  for (int i = tid; i < kMaxNodes * kMaskWords; i += blockDim.x) (&sm.natmask[0][0])[i] = 0u;
+  cluster.sync();                 // every CTA of the cluster is running and has cleared what the others write into
   griddep_wait();
   ACM_RT(0);
   float z[4];
-  load_logit_row(ra.logits, min(t_mine, T - 1), E, lane, z);      // in flight during the selection
-  if (mask_override) {
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const int e = lane + 32 * c;
+    const float v = __ldcg(ra.logits + static_cast<size_t>(t_lo + min(r, T - 1)) * E + min(e, E - 1));
+    z[c] = (r < T && e < E) ? v : -INFINITY;
+  }
+  if (!mask_override && tid < kMaxNodes) sm.alpha[tid] = sa.alpha[t_lo + min(tid, T - 1)];
+  if (r < T && !mask_override) {
+    float prob[4];
+    uint32_t bits[kMaskWords];
+    softmax_topk_regs(z, E, k, lane, prob, bits, nullptr, true);
+    if (r == 0 && anc_words && lane < 2 * kMaskWords) {
+      const uint32_t w = (lane >> 1) == 0 ? bits[0] : (lane >> 1) == 1 ? bits[1] : (lane >> 1) == 2 ? bits[2] : bits[3];
+      asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(anc_words + 2 * kMaskWords * b + lane),
+                   "r"(((w >> (16 * (lane & 1))) & 0xffffu) | (tag << 16)) : "memory");
+    }
+    const uint32_t my_bits = lane == 0 ? bits[0] : lane == 1 ? bits[1] : lane == 2 ? bits[2] : bits[3];
+    for (int p = 0; p < C; ++p) {
+      float* probs_p = cluster.map_shared_rank(fs.probs, p);
+      uint32_t* nat_p = cluster.map_shared_rank(&sm.natmask[0][0], p);
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+        if (lane + 32 * c < E) probs_p[r * E + lane + 32 * c] = prob[c];
+      if (lane < kMaskWords) nat_p[r * kMaskWords + lane] = my_bits;
+    }
+  }
+  cluster.sync();                 // the whole block's probabilities and natural sets are in every CTA
+
+  // 2
+  SelectArgs mine = sa;
+  mine.anchor_nodes = nullptr;
+  mine.n_anchor_nodes = 0;
+  mine.mask_out += b * kMaskWords;
+  if (mine.unpruned_out) mine.unpruned_out += b * kMaskWords;
+  mine.count_out += b;
+  if (mine.demand_out) mine.demand_out += static_cast<size_t>(b) * kMaxExperts;
+  if (mine.stats_out) mine.stats_out += b;
+  if (mask_override) {            // (single block) the caller's set instead of a selection
     if (tid < kMaskWords) {
       const uint32_t m = tid < (E + 31) / 32 ? mask_override[tid] : 0u;
       sm.Sp[tid] = m;
-      if (blockIdx.x == 0 && tid < (E + 31) / 32) sa.mask_out[tid] = m;
+      if (first && tid < (E + 31) / 32) mine.mask_out[tid] = m;
     }
-    if (blockIdx.x == 0 && tid == 0 && sa.stats_out) {
+    if (first && tid == 0 && mine.stats_out) {
       acm_block_stats st = {};
-      *sa.stats_out = st;
+      *mine.stats_out = st;
     }
     __syncthreads();
+    if (first && ra.sel_flag && tid < 2 * kMaskWords) publish_eligible(ra, sm, tid);
   } else {
-    if (tid < kSelThreads) {
-      stage_select(sa, sm, T, E, k, natmask_g, blockIdx.x == 0, blockIdx.x == 0 ? ra.sel_flag : nullptr,
-                   static_cast<uint32_t>(ra.sel_epoch) & 0xffffu);
-    }
+    if (tid < kSelThreads)
+      stage_select<true>(mine, sm, T, E, k, nullptr, first,
+                         (first && ra.sel_flag) ? ra.sel_flag + 2 * kMaskWords * b : nullptr, tag, fs.probs);
     __syncthreads();
   }
-  if (mask_override && ra.sel_flag && blockIdx.x == 0 && tid < 2 * kMaskWords) publish_eligible(ra, sm, tid);
   ACM_RT(2);
-  {
+
+  // 3
+  if (r < T) {
     uint32_t mask_w[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c) mask_w[c] = sm.Sp[c];
+    const int t = t_lo + r;
     int e;
     float w;
     route_node(z, mask_w, E, k, lane, ra.weighting, ra.routed_scale, e, w);
-    if (t_mine < T && lane < k) {
-      ra.idx_out[static_cast<size_t>(t_mine) * k + lane] = e;
-      ra.w_out[static_cast<size_t>(t_mine) * k + lane] = w;
+    if (lane < k) {
+      ra.idx_out[static_cast<size_t>(t) * k + lane] = e;
+      ra.w_out[static_cast<size_t>(t) * k + lane] = w;
+      if (e >= 0 && ra.wtab) ra.wtab[static_cast<size_t>(e) * kWtabStride + t] = w;
     }
-    if (ra.act_mask && t_mine < T) publish_routes(ra.act_mask, ra.wtab, t_mine, k, lane, e, w);
+    publish_routes_local(fs.act, k, lane, e);
   }
   ACM_RT(3);
-  if (!ra.ticket) return;
-  // Asked for a report on the whole block: the CTA that finishes last sees the complete mask.
-  __threadfence();
   __syncthreads();
-  if (tid == 0) {
-    const int prev = atomicAdd(ra.ticket, 1);
-    s_last = prev == static_cast<int>(gridDim.x) - 1;
-    if (s_last) *ra.ticket = 0;
+  if (tid < kMaskWords && fs.act[tid]) {
+    if (ra.act_mask) atomicOr(ra.act_mask + tid, fs.act[tid]);
+    if (report && !first) atomicOr(cluster.map_shared_rank(fs.act, 0) + tid, fs.act[tid]);
   }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  if (warp == 0) {
+  if (!report) return;
+  // the block's own report, by the cluster's first CTA: its activated experts and (single block, offloaded layer)
+  // which of them have to be copied in, in ascending id order = their staging slots
+  cluster.sync();
+  if (first && warp == 0) {
     const int words = (E + 31) / 32;
-    const uint32_t act = lane < words ? __ldcg(ra.act_mask + lane) : 0u;
+    const uint32_t act = lane < words ? fs.act[lane] : 0u;
     const uint32_t res = lane < words ? (ra.resident ? ra.resident[lane] : 0xffffffffu) : 0u;
     const uint32_t stg = act & ~res;
     int n_act = __popc(act), n_stg = __popc(stg), before = 0;
@@ -756,69 +852,18 @@ k_select_route(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, const uin
     if (ra.host_stage_list) {
       uint32_t m = stg;
       int pos = before;
-      while (m) {                        // staged experts in ascending id order = their staging slots
-        const int b = __ffs(m) - 1;
+      while (m) {
+        const int bit = __ffs(m) - 1;
         m &= m - 1;
-        ra.host_stage_list[1 + pos++] = lane * 32 + b;
+        ra.host_stage_list[1 + pos++] = lane * 32 + bit;
       }
       if (lane == 0) ra.host_stage_list[0] = tot_stg;
       if (lane < kMaskWords) ra.host_stage_list[1 + kMaxExperts + lane] = static_cast<int32_t>(act);   // the activated set
     }
-    if (lane == 0 && ra.stats_out) { ra.stats_out->n_activated = n_act; ra.stats_out->n_staged = tot_stg; }
-  }
-}
-
-// Several verification blocks in one launch: CTA b owns block b (the rows bd.off[b] .. bd.off[b+1]-1 of
-// every per-node array).  Its warps 0-3 run the selection on the block's own nodes (Eq. 3-7 see nothing
-// of the other blocks; the block's first row is its root), then all of its warps route the block's
-// nodes inside that set (Eq. 2).  The FFN kernel's inputs are shared by all blocks: the activated mask
-// is OR-ed into by everyone, the weight table is indexed by the row in the stacked batch.  Block b's
-// eligible set is published in its own eight tagged words, ra.sel_flag + 8 b.
-__global__ void __launch_bounds__(32 * kRouteNodesPerCta)
-k_select_route_batch(const uint32_t* natmask_g, SelectArgs sa, RouteArgs ra, BatchDesc bd, int E, int k) {
-  __shared__ StageSmem sm;
-  __shared__ uint32_t s_act[kMaskWords];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, n_warps = blockDim.x >> 5;
-  const int b = blockIdx.x;
-  const int t_lo = bd.off[b], T = bd.off[b + 1] - t_lo;
-  griddep_launch_dependents();
-  griddep_wait();
-  if (tid < kMaskWords) s_act[tid] = 0u;
-  SelectArgs mine = sa;
-  mine.probs += static_cast<size_t>(t_lo) * E;
-  mine.alpha += t_lo;
-  mine.anchor_nodes = nullptr;
-  mine.n_anchor_nodes = 0;
-  mine.mask_out += b * kMaskWords;
-  if (mine.unpruned_out) mine.unpruned_out += b * kMaskWords;
-  mine.count_out += b;
-  if (mine.demand_out) mine.demand_out += static_cast<size_t>(b) * kMaxExperts;
-  if (mine.stats_out) mine.stats_out += b;
-  if (tid < kSelThreads)
-    stage_select(mine, sm, T, E, k, natmask_g + static_cast<size_t>(t_lo) * kMaskWords, true,
-                 ra.sel_flag ? ra.sel_flag + 2 * kMaskWords * b : nullptr, static_cast<uint32_t>(ra.sel_epoch) & 0xffffu);
-  __syncthreads();
-  uint32_t mask_w[4];
-#pragma unroll
-  for (int c = 0; c < 4; ++c) mask_w[c] = sm.Sp[c];
-  for (int t = t_lo + warp; t < t_lo + T; t += n_warps) {
-    float z[4];
-    load_logit_row(ra.logits, t, E, lane, z);
-    int e;
-    float w;
-    route_node(z, mask_w, E, k, lane, ra.weighting, ra.routed_scale, e, w);
-    if (lane < k) {
-      ra.idx_out[static_cast<size_t>(t) * k + lane] = e;
-      ra.w_out[static_cast<size_t>(t) * k + lane] = w;
+    if (lane == 0 && mine.stats_out) {
+      mine.stats_out->n_activated = n_act;
+      mine.stats_out->n_staged = tot_stg;
     }
-    publish_routes(ra.act_mask, ra.wtab, t, k, lane, e, w);
-    publish_routes_local(s_act, k, lane, e);
-  }
-  __syncthreads();
-  if (tid == 0 && mine.stats_out) {      // this block's own activated experts (the batch's union is the mask)
-    int n = 0;
-    for (int wd = 0; wd < kMaskWords; ++wd) n += __popc(s_act[wd]);
-    mine.stats_out->n_activated = n;
   }
 }
 
@@ -844,11 +889,8 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
                                  float* logits, int T, int H, int E, float* zero_buf,
                                  size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status,
                                  float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k, int32_t* tile_done,
-                                 bool pdl, cudaStream_t s, long long* dbg, uint32_t* anc_words, uint32_t anc_tag,
-                                 const RootList* roots) {
+                                 bool pdl, cudaStream_t s, long long* dbg) {
   if (!probs && !nat_idx) tile_done = nullptr;
-  RootList rl = {};
-  if (roots) rl = *roots; else { rl.n = 1; rl.row[0] = 0; }
   cudaLaunchAttribute attr[1];
   set_pdl_attr(attr);
   cudaLaunchConfig_t cfg = {};
@@ -872,7 +914,7 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * 8); cfg.dynamicSmemBytes = smem;
     return cudaLaunchKernelEx(&cfg, kern, static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
                               logits, T, H, E, n_chunks, zero_buf, zero_floats, zero_buf2, zero_floats2, status, probs, nat_idx, nat_mask, k,
-                              tile_done, dbg, anc_words, anc_tag, rl);
+                              tile_done, dbg);
   } else {
     auto kern = k_router_logits<__nv_bfloat16>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
@@ -880,13 +922,8 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * (32 / ElemTraits<__nv_bfloat16>::EPT)); cfg.dynamicSmemBytes = smem;
     return cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x),
                               static_cast<const __nv_bfloat16*>(w_router), bias, logits, T, H, E, n_chunks, zero_buf,
-                              zero_floats, zero_buf2, zero_floats2, status, probs, nat_idx, nat_mask, k, tile_done, dbg, anc_words, anc_tag, rl);
+                              zero_floats, zero_buf2, zero_floats2, status, probs, nat_idx, nat_mask, k, tile_done, dbg);
   }
-}
-
-int route_ctas(int T) {
-  const int npc = T < kRouteNodesPerCta ? (T < 4 ? 4 : T) : kRouteNodesPerCta;
-  return (T + npc - 1) / npc;
 }
 
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s) {
@@ -899,34 +936,39 @@ cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s
   return cudaGetLastError();
 }
 
-cudaError_t launch_select_route(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
-                                const uint32_t* mask_override, int T, int E, int k, bool pdl, cudaStream_t s) {
-  cudaLaunchAttribute attr[1];
-  set_pdl_attr(attr);
-  cudaLaunchConfig_t cfg = {};
-  const int npc = T < kRouteNodesPerCta ? (T < 4 ? 4 : T) : kRouteNodesPerCta;     // at least the four selection warps
-  cfg.gridDim = dim3(route_ctas(T));
-  cfg.blockDim = dim3(32 * npc);
-  cfg.stream = s;
-  cfg.attrs = attr;
-  cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, k_select_route, nat_mask, sa, ra, mask_override, T, E, k);
+int select_ctas_per_block(int widest) {
+  const int c = (widest + kFusedWarps - 1) / kFusedWarps;
+  return c <= 1 ? 1 : c == 2 ? 2 : kFusedMaxCtas;
 }
 
-cudaError_t launch_select_route_batch(const uint32_t* nat_mask, const SelectArgs& sa, const RouteArgs& ra,
-                                      const BatchDesc& bd, int E, int k, bool pdl, cudaStream_t s) {
-  cudaLaunchAttribute attr[1];
-  set_pdl_attr(attr);
-  cudaLaunchConfig_t cfg = {};
+cudaError_t launch_softmax_select_route(const SelectArgs& sa, const RouteArgs& ra, const BatchDesc& bd,
+                                        const uint32_t* mask_override, uint32_t* anc_words, int E, int k, bool pdl,
+                                        cudaStream_t s) {
   int widest = 1;
   for (int b = 0; b < bd.n_blocks; ++b) widest = bd.off[b + 1] - bd.off[b] > widest ? bd.off[b + 1] - bd.off[b] : widest;
-  const int warps = widest < 4 ? 4 : widest > kRouteNodesPerCta ? kRouteNodesPerCta : widest;   // at least the four selection warps
-  cfg.gridDim = dim3(bd.n_blocks);
-  cfg.blockDim = dim3(32 * warps);
+  if (widest > kFusedMaxCtas * kFusedWarps) return cudaErrorInvalidValue;      // a warp per row
+  const int C = select_ctas_per_block(widest);
+  static bool configured = false;       // (the attribute is per device function; repeating it is harmless)
+  if (!configured) {
+    cudaError_t err = cudaFuncSetAttribute(k_softmax_select_route, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           static_cast<int>(kFusedSmemRequest));
+    if (err != cudaSuccess) return err;
+    configured = true;
+  }
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  set_pdl_attr(attr + 1);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(bd.n_blocks * C);
+  cfg.blockDim = dim3(32 * kFusedWarps);
+  cfg.dynamicSmemBytes = kFusedSmemRequest;
   cfg.stream = s;
   cfg.attrs = attr;
-  cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, k_select_route_batch, nat_mask, sa, ra, bd, E, k);
+  cfg.numAttrs = pdl ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, k_softmax_select_route, sa, ra, bd, mask_override, anc_words, E, k);
 }
 
 cudaError_t launch_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask, float* wtab,
