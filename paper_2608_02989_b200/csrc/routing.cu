@@ -97,6 +97,26 @@ __device__ __forceinline__ float warp_tree_sum_128(float a0, float a1, float a2,
   return __shfl_sync(0xffffffffu, v, 0);
 }
 
+// Natural top-k of one logit row held in registers (lane l holds experts l, l + 32, l + 64, l + 96), ranked on the
+// logits, ties to the lower index: the set as a bit mask (warp-uniform); the ranked ids go to `nat_row` if given.
+__device__ __forceinline__ void topk_bits(const float (&z)[4], int E, int k, int lane, uint32_t (&bits)[kMaskWords],
+                                          int32_t* nat_row) {
+  unsigned key[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) key[c] = (lane + 32 * c < E) ? order_key(z[c]) : 0u;
+  uint32_t b0 = 0u, b1 = 0u, b2 = 0u, b3 = 0u;
+  for (int j = 0; j < k; ++j) {
+    const int e = warp_take_best(key, lane);
+    if (nat_row && lane == 0) nat_row[j] = e;
+    if (e >= 0) {
+      const uint32_t bit = 1u << (e & 31);
+      const int wd = e >> 5;
+      b0 |= wd == 0 ? bit : 0u; b1 |= wd == 1 ? bit : 0u; b2 |= wd == 2 ? bit : 0u; b3 |= wd == 3 ? bit : 0u;
+    }
+  }
+  bits[0] = b0; bits[1] = b1; bits[2] = b2; bits[3] = b3;
+}
+
 // Stage 1b for ONE node, by one warp, on a logit row held in registers (lane l holds experts l, l + 32, l + 64,
 // l + 96; -inf beyond E): softmax over the expert axis (fixed recipe) and natural top-k ranked on the logits.
 // Returns the probabilities in the same layout and the top-k set as a bit mask (warp-uniform); the ranked ids
@@ -104,7 +124,6 @@ __device__ __forceinline__ float warp_tree_sum_128(float a0, float a1, float a2,
 __device__ __forceinline__ void softmax_topk_regs(const float (&z)[4], int E, int k, int lane, float (&prob)[4],
                                                   uint32_t (&bits)[kMaskWords], int32_t* nat_row, bool want_topk) {
   float y[4];
-  unsigned key[4];
   float zmax = fmaxf(fmaxf(z[0], z[1]), fmaxf(z[2], z[3]));
 #pragma unroll
   for (int s = 16; s >= 1; s >>= 1) zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, s));
@@ -112,24 +131,15 @@ __device__ __forceinline__ void softmax_topk_regs(const float (&z)[4], int E, in
   for (int c = 0; c < 4; ++c) {
     const float ex = exp_fixed(__fsub_rn(z[c], zmax));
     y[c] = (lane + 32 * c < E) ? ex : 0.0f;
-    key[c] = (lane + 32 * c < E) ? order_key(z[c]) : 0u;
   }
   const float denom = warp_tree_sum_128(y[0], y[1], y[2], y[3]);
 #pragma unroll
   for (int c = 0; c < 4; ++c) prob[c] = __fdiv_rn(y[c], denom);
-  uint32_t b0 = 0u, b1 = 0u, b2 = 0u, b3 = 0u;
   if (want_topk) {
-    for (int j = 0; j < k; ++j) {
-      const int e = warp_take_best(key, lane);
-      if (nat_row && lane == 0) nat_row[j] = e;
-      if (e >= 0) {
-        const uint32_t bit = 1u << (e & 31);
-        const int wd = e >> 5;
-        b0 |= wd == 0 ? bit : 0u; b1 |= wd == 1 ? bit : 0u; b2 |= wd == 2 ? bit : 0u; b3 |= wd == 3 ? bit : 0u;
-      }
-    }
+    topk_bits(z, E, k, lane, bits, nat_row);
+  } else {
+    bits[0] = bits[1] = bits[2] = bits[3] = 0u;
   }
-  bits[0] = b0; bits[1] = b1; bits[2] = b2; bits[3] = b3;
 }
 
 // The same for a row in global memory (`z_row` may have been written by other CTAs: read through L2).
@@ -354,7 +364,8 @@ struct StageSmem {
   uint32_t natmask[kMaxNodes][kMaskWords];
   int32_t votes[kMaxExperts];
   float u[kMaxExperts];
-  float tree[kMaxExperts + 4];
+  float tree[2][kMaxExperts];      // two sums over the expert axis in a row use one buffer each
+  int32_t rank[kMaxExperts];       // fused kernel: the experts' ranks, counted by four helper warps
   alignas(16) unsigned long long rkey[kMaxExperts];   // ranking keys of the experts (0 = not ranked)
   uint32_t A[kMaskWords], S[kMaskWords], Sp[kMaskWords], Hres[kMaskWords];
   int32_t scal[8];
@@ -370,19 +381,40 @@ __device__ __forceinline__ int sel_count(bool pred) {
       : "=r"(n) : "r"(static_cast<unsigned>(pred)) : "memory");
   return n;
 }
-// 128-slot halving tree (threads 0..127 hold one slot each): levels 64 and 32 are formed by warp 0
-// from shared memory, the remaining levels with shuffles -- the same additions in the same order
-// as a[i] += a[i+s], s = 64, 32, ..., 1.
+// 128-slot halving tree (threads 0..127 hold one slot each): every warp forms levels 64 and 32 from shared
+// memory and the remaining levels with shuffles -- the same additions in the same order as a[i] += a[i+s],
+// s = 64, 32, ..., 1, so all four warps hold the same sum and nothing has to be passed back.  (`tree` must not be
+// the buffer of the sum before: a slower warp may still be reading that.)
 __device__ float sel_tree_sum_128(float* tree, float mine) {
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31;
   tree[tid] = mine;
   sel_sync();
-  if (tid < 32) {
-    const float r = warp_tree_sum_128(tree[tid], tree[tid + 32], tree[tid + 64], tree[tid + 96]);
-    if (tid == 0) tree[kMaxExperts] = r;
+  return warp_tree_sum_128(tree[lane], tree[lane + 32], tree[lane + 64], tree[lane + 96]);
+}
+// Barriers between the four selection warps and the four helper warps of the fused kernel (256 threads): the side that
+// has produced something arrives, the side that needs it waits.
+__device__ __forceinline__ void pair_arrive(int id) { asm volatile("bar.arrive %0, 256;" ::"r"(id) : "memory"); }
+__device__ __forceinline__ void pair_wait(int id) { asm volatile("bar.sync %0, 256;" ::"r"(id) : "memory"); }
+constexpr int kBarKeys = 3, kBarRanks = 4;
+// Rank of an expert inside R by (u descending, index ascending) = the number of larger 64-bit keys.
+__device__ __forceinline__ int rank_of(const unsigned long long* rkey, unsigned long long mykey) {
+  int rank = 0;
+  const ulonglong2* keys2 = reinterpret_cast<const ulonglong2*>(rkey);
+#pragma unroll 8
+  for (int j = 0; j < kMaxExperts / 2; ++j) {
+    const ulonglong2 kk = keys2[j];
+    rank += (kk.x > mykey ? 1 : 0) + (kk.y > mykey ? 1 : 0);
   }
-  sel_sync();
-  return tree[kMaxExperts];
+  return rank;
+}
+// The helper warps' part (threads 128..255 of the fused kernel): the ranks, while the selection warps work out how
+// many experts to keep.
+__device__ void stage_select_helper(StageSmem& sm) {
+  const int h = threadIdx.x - kSelThreads;
+  pair_wait(kBarKeys);
+  sm.rank[h] = rank_of(sm.rkey, sm.rkey[h]);
+  __threadfence_block();
+  pair_arrive(kBarRanks);
 }
 
 // Stage 2: demand, anchors, self-sizing, pruning.  Called by threads 0..127; thread e owns expert e.
@@ -425,9 +457,11 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
       }
     }
   }
-  if (tid < kMaskWords) sm.Hres[tid] = (tid < (E + 31) / 32) ? (a.resident ? a.resident[tid] : 0xffffffffu) : 0u;
-  if (tid < 8) sm.scal[tid] = 0;
-  sel_sync();
+  if constexpr (!kStaged) {         // (the fused kernel has done this before its barrier)
+    if (tid < kMaskWords) sm.Hres[tid] = (tid < (E + 31) / 32) ? (a.resident ? a.resident[tid] : 0xffffffffu) : 0u;
+    if (tid < 8) sm.scal[tid] = 0;
+    sel_sync();
+  }
   if (tid < kMaskWords) {           // anchors (Eq. 5): union of the anchor nodes' natural sets
     uint32_t A = 0u;
     if (a.prm.use_anchors) {
@@ -445,27 +479,27 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   float u = 0.0f;
   const int demand_mode = a.prm.demand;
   if constexpr (kStaged) {
-    // (a rolled loop of eight nodes a turn: in the fused kernel the code is fetched while the FFN kernel streams
+    // (a rolled loop of sixteen nodes a turn: in the fused kernel the code is fetched while the FFN kernel streams
     // weights, and every further line of straight-line code is one more slow instruction fetch)
     const float* pcol = s_probs + min(tid, E - 1);
 #pragma unroll 1
-    for (int t0 = 0; t0 < T; t0 += 8) {
-      float al[8], pj[8];
+    for (int t0 = 0; t0 < T; t0 += 16) {
+      float al[16], pj[16];
       unsigned in_mask = 0;
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < 16; ++j) {
         const int t = min(t0 + j, T - 1);
         al[j] = sm.alpha[t];
         pj[j] = pcol[t * E];
         in_mask |= ((sm.natmask[t][warp] >> lane) & 1u) << j;
       }
-      const unsigned valid = t0 + 8 > T ? (1u << (T - t0)) - 1u : 0xffu;
+      const unsigned valid = t0 + 16 > T ? (1u << (T - t0)) - 1u : 0xffffu;
       in_mask &= valid;
       votes += __popc(in_mask);
       const unsigned take = demand_mode == ACM_DEMAND_FULL_MASS ? valid
                           : demand_mode == ACM_DEMAND_TOPK_MASS ? in_mask : 0u;
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
+      for (int j = 0; j < 16; ++j) {
         const float nu = __fmaf_rn(al[j], pj[j], u);
         u = ((take >> j) & 1u) ? nu : u;
       }
@@ -507,7 +541,15 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   const int nR = E - nA;
   const int n_positive = sel_count(in_R && u > 0.0f);
   const float upos = in_R ? fmaxf(u, 0.0f) : 0.0f;
-  const float Z = sel_tree_sum_128(sm.tree, upos);
+  // rank inside R by (u descending, index ascending): one 64-bit key per expert
+  const unsigned long long mykey =
+      in_R ? ((static_cast<unsigned long long>(order_key(u)) << 32) | (0xffffffffu - tid)) : 0ull;
+  sm.rkey[tid] = mykey;
+  if constexpr (kStaged) {
+    __threadfence_block();
+    pair_arrive(kBarKeys);          // the helper warps count the ranks meanwhile
+  }
+  const float Z = sel_tree_sum_128(sm.tree[0], upos);
 
   const int floor_keep = max(0, k - nA);
   int n_er = 0, n_keep;
@@ -516,7 +558,7 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   } else if (Z > 0.0f) {
     const float qv = __fdiv_rn(upos, Z);
     const float h = (qv >= 1.17549435e-38f) ? __fmul_rn(qv, log_fixed(qv)) : 0.0f;
-    const float entropy = -sel_tree_sum_128(sm.tree, h);
+    const float entropy = -sel_tree_sum_128(sm.tree[1], h);
     const float perp = exp_fixed(entropy);
     n_er = static_cast<int>(ceilf(__fsub_rn(perp, a.prm.ceil_guard)));
     n_er = min(max(n_er, 1), n_positive);
@@ -526,21 +568,13 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
   }
   n_keep = min(n_keep, nR);
 
-  // rank inside R by (u descending, index ascending): one 64-bit key per expert
-  const unsigned long long mykey =
-      in_R ? ((static_cast<unsigned long long>(order_key(u)) << 32) | (0xffffffffu - tid)) : 0ull;
-  sm.rkey[tid] = mykey;
-  sel_sync();
   bool in_S = in_A;
-  if (in_R) {
-    int rank = 0;
-    const ulonglong2* keys2 = reinterpret_cast<const ulonglong2*>(sm.rkey);
-#pragma unroll 8
-    for (int j = 0; j < kMaxExperts / 2; ++j) {
-      const ulonglong2 kk = keys2[j];
-      rank += (kk.x > mykey ? 1 : 0) + (kk.y > mykey ? 1 : 0);
-    }
-    in_S = rank < n_keep;
+  if constexpr (kStaged) {
+    pair_wait(kBarRanks);
+    if (in_R) in_S = sm.rank[tid] < n_keep;
+  } else {
+    sel_sync();
+    if (in_R) in_S = rank_of(sm.rkey, mykey) < n_keep;
   }
   const unsigned s_word = __ballot_sync(0xffffffffu, in_S);
   if (lane == 0) sm.S[warp] = s_word;
@@ -707,7 +741,7 @@ __device__ __forceinline__ void publish_eligible(const RouteArgs& ra, const Stag
 // router kernel before it has written the logits only.  Every warp loads its row (the one trip through L2 of the
 // whole chain: with the FFN kernel already streaming weights, each further one would cost well over a microsecond),
 // then
-//   1b  softmax and natural top-k of the row (Eq. 1); the probabilities and the top-k mask go into the shared memory
+//   1b  natural top-k and softmax of the row (Eq. 1); the probabilities and the top-k mask go into the shared memory
 //       of EVERY CTA of the cluster (distributed shared memory), the logits stay in registers; the block's first row
 //       is its root, whose natural top-k are anchors (Eq. 5) and published at once as eight tagged words for the FFN
 //       kernel to start on;
@@ -758,15 +792,19 @@ k_softmax_select_route(SelectArgs sa, RouteArgs ra, BatchDesc bd, const uint32_t
     z[c] = (r < T && e < E) ? v : -INFINITY;
   }
   if (!mask_override && tid < kMaxNodes) sm.alpha[tid] = sa.alpha[t_lo + min(tid, T - 1)];
+  if (tid < kMaskWords) sm.Hres[tid] = (tid < (E + 31) / 32) ? (sa.resident ? sa.resident[tid] : 0xffffffffu) : 0u;
+  if (tid < 8) sm.scal[tid] = 0;
   if (r < T && !mask_override) {
+    // (the top-k first: the root's are what the FFN kernel is waiting for)
     float prob[4];
-    uint32_t bits[kMaskWords];
-    softmax_topk_regs(z, E, k, lane, prob, bits, nullptr, true);
+    uint32_t bits[kMaskWords], none[kMaskWords];
+    topk_bits(z, E, k, lane, bits, nullptr);
     if (r == 0 && anc_words && lane < 2 * kMaskWords) {
       const uint32_t w = (lane >> 1) == 0 ? bits[0] : (lane >> 1) == 1 ? bits[1] : (lane >> 1) == 2 ? bits[2] : bits[3];
       asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(anc_words + 2 * kMaskWords * b + lane),
                    "r"(((w >> (16 * (lane & 1))) & 0xffffu) | (tag << 16)) : "memory");
     }
+    softmax_topk_regs(z, E, k, lane, prob, none, nullptr, false);
     const uint32_t my_bits = lane == 0 ? bits[0] : lane == 1 ? bits[1] : lane == 2 ? bits[2] : bits[3];
     for (int p = 0; p < C; ++p) {
       float* probs_p = cluster.map_shared_rank(fs.probs, p);
@@ -804,6 +842,8 @@ k_softmax_select_route(SelectArgs sa, RouteArgs ra, BatchDesc bd, const uint32_t
     if (tid < kSelThreads)
       stage_select<true>(mine, sm, T, E, k, nullptr, first,
                          (first && ra.sel_flag) ? ra.sel_flag + 2 * kMaskWords * b : nullptr, tag, fs.probs);
+    else if (tid < 2 * kSelThreads)
+      stage_select_helper(sm);
     __syncthreads();
   }
   ACM_RT(2);
