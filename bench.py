@@ -27,7 +27,7 @@ ROOT = Path(__file__).resolve().parent
 if str(ROOT) not in sys.path:
     sys.path.insert(0, str(ROOT))
 
-DRAM_BYTES_PER_ACTIVATED_EXPERT = {3: (273440512 + 193336832 + 193765376) / 68.0}   # config -> bytes (ncu, profiles/)
+DRAM_BYTES_PER_ACTIVATED_EXPERT = {3: (273970176 + 193497088 + 193248256) / 68.0}   # config -> bytes (ncu, profiles/)
 METRIC = "verify_blocks_per_s_per_moe_layer"
 UNIT = "layer-blocks/s"
 
@@ -57,7 +57,7 @@ def parse_args():
     ap.add_argument("--overlap", type=int, default=3, choices=[0, 1, 2, 3],
                     help="acm_set_overlap level: 0 plain stream order (cooperative FFN launch), 1 dependent launches, "
                          "2 + FFN start on the eligible set, 3 + FFN start on the anchors (default)")
-    ap.add_argument("--bracket-every", type=int, default=11,
+    ap.add_argument("--bracket-every", type=int, default=47,
                     help="bracket every n-th FFN launch with events for the roofline figure (0: none, the pure pipeline)")
     ap.add_argument("--all-resident", action="store_true",
                     help="config 5 only: every expert on the GPU (no offloading) instead of the configured 40 % residency")
@@ -544,9 +544,10 @@ def run_acm(args, world, rank, local):
         ctx.stage_timing(False)
         pipeline_gbs = acc.pop("_gbs")
         stage_us = {key: round(v, 2) for key, v in acc.items()}
-        stage_us["note"] = ("in-kernel stamps, mean over %d layers: router = dependency release to selection start; "
-                            "select; route; ffn = first role start to last tile (it starts on the anchor experts while "
-                            "the selection runs); whole = start of router to end of ffn" % n_samples)
+        stage_us["note"] = ("in-kernel stamps, mean over %d layers: router = dependency release of the logits kernel to "
+                            "the start of the selection kernel; select = softmax, natural top-k and selection; route; "
+                            "ffn = first role start to last tile (it starts on the anchor experts while the selection "
+                            "runs); whole = start of router to end of ffn" % n_samples)
 
     if rank != 0:
         return

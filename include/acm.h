@@ -316,8 +316,9 @@ acm_status acm_offload_times(acm_ctx* ctx, double* ms_out /*host [4]*/, int32_t*
  * acm_stage_times synchronises and reports, for the LAST acm_moe_verify call on a bf16 layer without a
  * residency, us_out [5] (host, microseconds):
  *   [0] stage 1: from the router kernel passing its dependency wait (everything before it in the
- *       stream is complete) to the start of the selection -- logits, softmax, natural top-k;
- *   [1] stage 2: the selection (Eq. 4-7), until the eligible set is published;
+ *       stream is complete) to the selection kernel passing its own -- the logits;
+ *   [1] stage 2: softmax and natural top-k (Eq. 1) and the selection (Eq. 4-7), until the eligible set
+ *       is published;
  *   [2] stage 3: the routes (Eq. 2) and the FFN kernel's routing inputs;
  *   [3] stage 4: the FFN kernel from its first CTA's roles starting to its last tile finished -- it
  *       starts on the anchor experts while stage 2 runs, so [0..3] overlap and do not add up to
