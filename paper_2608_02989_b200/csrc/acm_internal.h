@@ -124,6 +124,7 @@ cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s
 // (both may be null) hold 8 tagged words per block: the eligible set and, earlier, the anchors (the natural top-k
 // of the block's first row).
 int select_ctas_per_block(int widest);
+cudaError_t select_configure();   // the kernel's function attributes, once per device (when a context is created)
 cudaError_t launch_softmax_select_route(const SelectArgs& sa, const RouteArgs& ra, const BatchDesc& bd,
                                         const uint32_t* mask_override, uint32_t* anc_words, int E, int k, bool pdl,
                                         cudaStream_t s);

@@ -509,6 +509,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
     c->encode = reinterpret_cast<EncodeTiledFn>(fn);
     if (ffn_configure() != cudaSuccess) return fail(ACM_ERR_CUDA);
   }
+  if (select_configure() != cudaSuccess) return fail(ACM_ERR_CUDA);
 
   const int Tm = kWideNodes, E = desc->n_experts, k = desc->top_k, I = desc->inter;
   size_t off = 0;

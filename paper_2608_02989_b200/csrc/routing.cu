@@ -976,6 +976,11 @@ cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s
   return cudaGetLastError();
 }
 
+cudaError_t select_configure() {
+  return cudaFuncSetAttribute(k_softmax_select_route, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(kFusedSmemRequest));
+}
+
 int select_ctas_per_block(int widest) {
   const int c = (widest + kFusedWarps - 1) / kFusedWarps;
   return c <= 1 ? 1 : c == 2 ? 2 : kFusedMaxCtas;
@@ -988,13 +993,6 @@ cudaError_t launch_softmax_select_route(const SelectArgs& sa, const RouteArgs& r
   for (int b = 0; b < bd.n_blocks; ++b) widest = bd.off[b + 1] - bd.off[b] > widest ? bd.off[b + 1] - bd.off[b] : widest;
   if (widest > kFusedMaxCtas * kFusedWarps) return cudaErrorInvalidValue;      // a warp per row
   const int C = select_ctas_per_block(widest);
-  static bool configured = false;       // (the attribute is per device function; repeating it is harmless)
-  if (!configured) {
-    cudaError_t err = cudaFuncSetAttribute(k_softmax_select_route, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           static_cast<int>(kFusedSmemRequest));
-    if (err != cudaSuccess) return err;
-    configured = true;
-  }
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = C;
