@@ -33,9 +33,6 @@ __host__ __device__ inline int entry_idx(int32_t e) { return e & 0x0fffffff; }
 // Device workspace of one context (one allocation, carved on the host).
 struct Workspace {
   float* logits;        // [T,E]
-  float* probs;         // [T,E]
-  int32_t* nat_idx;     // [T,k]
-  uint32_t* nat_mask;   // [T,4] the same sets as bit masks
   int32_t* idx;         // [T,k]
   float* w;             // [T,k]
   // per block of a batch (a single block uses entry 0)

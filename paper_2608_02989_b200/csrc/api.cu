@@ -518,8 +518,8 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
     off = align_up(off + bytes, 1024);
     return at;
   };
-  const size_t o_logits = carve(sizeof(float) * Tm * E), o_probs = carve(sizeof(float) * Tm * E);
-  const size_t o_nat = carve(sizeof(int32_t) * Tm * k), o_idx = carve(sizeof(int32_t) * Tm * k);
+  const size_t o_logits = carve(sizeof(float) * Tm * E);
+  const size_t o_idx = carve(sizeof(int32_t) * Tm * k);
   const size_t o_w = carve(sizeof(float) * Tm * k), o_mask = carve(16 * Tm), o_unpr = carve(16 * Tm), o_cnt = carve(4 * Tm);
   const size_t o_dem = carve(sizeof(float) * kMaxExperts * Tm), o_stats = carve(sizeof(acm_block_stats) * Tm);
   // the FFN kernel's routing inputs, contiguous so that one pass clears them: weight table, finished-tile
@@ -536,15 +536,12 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_ticket = carve(16);
   const size_t o_selw = carve(32 * kMaxEarlyBlocks);
   const size_t o_ancw = carve(32 * kMaxEarlyBlocks);
-  const size_t o_natmask = carve(sizeof(uint32_t) * Tm * kMaskWords);
   const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
   const size_t o_diag = carve(sizeof(int32_t) * c->sm_count);
   if (cudaMalloc(&c->ws_base, off) != cudaSuccess) return fail(ACM_ERR_NOMEM);
   if (cudaMemset(c->ws_base, 0, off) != cudaSuccess) return fail(ACM_ERR_CUDA);
   char* b = static_cast<char*>(c->ws_base);
   c->ws.logits = reinterpret_cast<float*>(b + o_logits);
-  c->ws.probs = reinterpret_cast<float*>(b + o_probs);
-  c->ws.nat_idx = reinterpret_cast<int32_t*>(b + o_nat);
   c->ws.idx = reinterpret_cast<int32_t*>(b + o_idx);
   c->ws.w = reinterpret_cast<float*>(b + o_w);
   c->ws.mask = reinterpret_cast<uint32_t*>(b + o_mask);
@@ -567,7 +564,6 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.ticket = reinterpret_cast<int32_t*>(b + o_ticket);
   c->ws.sel_words = reinterpret_cast<uint32_t*>(b + o_selw);
   c->ws.anc_words = reinterpret_cast<uint32_t*>(b + o_ancw);
-  c->ws.nat_mask = reinterpret_cast<uint32_t*>(b + o_natmask);
   c->resident_dev = reinterpret_cast<uint32_t*>(b + o_res);
   c->wait_diag = reinterpret_cast<int32_t*>(b + o_diag);
   *out = c;
@@ -816,7 +812,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
                                 c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr));
   // stages 1b-3: one cluster of CTAs, which also fills the FFN kernel's routing inputs
   SelectArgs sa;
-  sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
+  sa.probs = nullptr; sa.nat_idx = nullptr; sa.alpha = alpha; sa.anchor_nodes = nullptr;   // (the fused kernel keeps both on chip)
   sa.n_anchor_nodes = 0; sa.resident = prm.residency ? res_dev : nullptr; sa.prm = prm;
   sa.mask_out = c->ws.mask; sa.unpruned_out = c->ws.unpruned; sa.count_out = c->ws.count;
   bool stats_direct = false;
@@ -1015,7 +1011,7 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
                                 nullptr, nullptr, nullptr, k, nullptr, c->pdl, s, nullptr));
   // stages 1b-3: one cluster of CTAs per block
   SelectArgs sa;
-  sa.probs = c->ws.probs; sa.nat_idx = c->ws.nat_idx; sa.alpha = alpha; sa.anchor_nodes = nullptr;
+  sa.probs = nullptr; sa.nat_idx = nullptr; sa.alpha = alpha; sa.anchor_nodes = nullptr;   // (the fused kernel keeps both on chip)
   sa.n_anchor_nodes = 0; sa.resident = nullptr; sa.prm = *params;
   sa.mask_out = c->ws.mask; sa.unpruned_out = c->ws.unpruned; sa.count_out = c->ws.count;
   bool stats_direct = false;
