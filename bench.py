@@ -36,7 +36,8 @@ def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None,
-                    help="timed steps (default 100; 3 for config 5 as configured, whose steps are bound by host-to-device copies)")
+                    help="timed steps (default 100; 3 for config 5 as configured, whose steps are bound by host-to-device "
+                         "copies; 20 for --impl reference)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=3, help="1..5; default 3 = Qwen3-30B-A3B-shaped stack")
     ap.add_argument("--layers", type=int, default=0, help="override the number of stacked layers (0 = the config's)")
@@ -72,7 +73,12 @@ def parse_args():
                          "of this many slots per layer; reports hit rate and host-to-device MiB per block")
     args = ap.parse_args()
     if args.steps is None:
-        args.steps = 3 if (args.config == 5 and not args.all_resident and not args.pool and args.impl == "acm") else 100
+        if args.impl == "reference":
+            args.steps = 20           # (each step of the oracle is a bounded sample of about half a second)
+        elif args.config == 5 and not args.all_resident and not args.pool:
+            args.steps = 3
+        else:
+            args.steps = 100
     return args
 
 
