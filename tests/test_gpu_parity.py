@@ -615,10 +615,10 @@ def _batch_reference(cfg, w, x, offsets, depths, params_kw):
 
 
 @pytest.mark.parametrize("c,n_blocks,params_kw", [(3, 4, {}), (3, 7, {}), (3, 2, {"fixed_budget": 12}), (4, 3, {}),
-                                                  (3, 12, {}), (2, 32, {}), (3, 1, {})])
+                                                  (3, 12, {}), (2, 32, {}), (3, 1, {}), (3, 64, {})])
 def test_multi_block_batch_equals_every_block_verified_alone(c, n_blocks, params_kw):
     """Several verification blocks in one call: each block's eligible set, routes and statistics are those of
-    the oracle run on that block alone (ragged block sizes, 1 to 32 blocks, with and without the FFN
+    the oracle run on that block alone (ragged block sizes, 1 to 64 blocks, with and without the FFN
     kernel's early start, shared experts), the FFN output rows match the oracle's, and the activated mask is
     the union over the blocks."""
     cfg = wl.CONFIGS[c]
@@ -711,6 +711,17 @@ def test_fused_call_on_ragged_block_sizes(T):
     assert st["n_activated"] >= min(cfg.top_k, cfg.n_experts)
     _verify_layer(cfg, 0, ctx, 0, natural=True)
     ctx.close()
+
+
+def test_fused_call_on_every_block_size():
+    """Every block size from 1 to 64 on one small layer shape: the selection kernel runs as a cluster of one, two or
+    four CTAs with one warp per row, the last of them partly or wholly without rows; sets, routes and every output
+    row against the oracle."""
+    for T in range(1, 65):
+        cfg = wl.scaled(wl.CONFIGS[3], n_nodes=T, hidden=256, inter=128, n_layers=1)
+        ctx = _ctx(cfg)
+        _verify_layer(cfg, 0, ctx, 0)
+        ctx.close()
 
 
 def _mx_layer(cfg, layer=0):
