@@ -886,6 +886,37 @@ def test_fused_call_on_random_shapes_and_selector_settings():
         ctx.close()
 
 
+@pytest.mark.parametrize("sizes", [[33, 1, 16, 14], [17, 17, 17, 13], [16, 16, 16, 16], [1] * 10 + [22], [32, 32], [64]])
+def test_batch_call_on_block_sizes_around_the_selection_clusters_steps(sizes):
+    """Partitions whose widest block sits on either side of 16 and 32 rows (the selection kernel gives every block a
+    cluster of one, two or four CTAs sized by the widest), with single-row blocks beside wide ones: every block
+    against the oracle run on it alone, every output row."""
+    rng = np.random.default_rng(len(sizes) * 1000 + sizes[0])
+    offsets = np.concatenate([[0], np.cumsum(sizes)]).astype(int).tolist()
+    T = offsets[-1]
+    cfg = wl.scaled(wl.CONFIGS[3], hidden=512, inter=128, n_nodes=T, max_depth=4, n_layers=1)
+    w = wl.layer_weights(cfg, 0, DEV)
+    x = wl.hidden_states(cfg, 0, DEV)
+    depths = torch.cat([torch.sort(torch.cat([torch.zeros(1, dtype=torch.int32),
+                                              torch.tensor(rng.integers(1, 5, size=n - 1), dtype=torch.int32)])).values
+                        for n in sizes])
+    alpha_ref, refs = _batch_reference(cfg, w, x, offsets, depths, {})
+    ctx = _ctx(cfg)
+    _set_weights(ctx, w, 0)
+    for rep in range(2):
+        out, idx, wt, mask, act, stats = ctx.moe_verify_batch(0, x, offsets, torch.tensor(alpha_ref, device=DEV),
+                                                              acm.SelectParams(), want=True)
+        assert ctx.device_status() == acm.OK
+        for b, ref in enumerate(refs):
+            np.testing.assert_array_equal(_u32(mask[b]), ref["mask"])
+            np.testing.assert_array_equal(idx[offsets[b]:offsets[b + 1]].cpu().numpy(), ref["idx"])
+        ref_idx = np.concatenate([r["idx"] for r in refs])
+        ref_w = np.concatenate([r["w"] for r in refs])
+        ffn = oracle.expert_ffn(x, ref_idx, ref_w, w["gate_up"], w["down"], w["shared_gate_up"], w["shared_down"])
+        _ffn_check(out, ffn, f"sizes {sizes}")
+    ctx.close()
+
+
 def test_batch_call_on_random_block_partitions():
     """Forty seeded random batches: 1 to 10 blocks of random sizes over random layers, against every block verified
     alone by the oracle."""
