@@ -51,6 +51,7 @@ struct Workspace {
   int32_t* tile_done;   // [64] router kernel: expert tiles finished per node tile (self-resetting)
   int32_t* ticket;      // [4] spare words (the MXFP4 scale check keeps its maximum in one)
   uint32_t* sel_words;  // [kMaxEarlyBlocks][8] the eligible masks as tagged 16-bit pieces (early start of the FFN kernel)
+  unsigned long long* root_words;   // [kMaxExperts] the root's logits under the call's 32-bit tag (router kernel, see RootArgs)
   uint32_t* anc_words;  // [kMaxEarlyBlocks][8] the anchor experts (each root's natural top-k) as tagged 16-bit pieces, published by the selection kernel first thing
 };
 
@@ -75,6 +76,18 @@ struct BatchDesc {
   int off[kMaxNodes + 1];    // (at most 64 blocks, at most kWideNodes rows in all, at most kMaxNodes rows a block)
 };
 constexpr int kMaxEarlyBlocks = 8;   // blocks whose eligible sets the FFN kernel can poll for (8 tagged words each)
+
+// Single-block fused call with an early start of the FFN kernel: the router kernel puts `rows` (0 or 1) rows of CTAs
+// in front of its grid that work out the root's logits ahead of everyone (published as 64-bit words, the value under
+// `tag`, in words[kMaxExperts]) and from them the anchors (Eq. 5), published as the eight tagged words anc_words.
+struct RootArgs {
+  int rows;
+  unsigned long long* words;
+  uint32_t tag;
+  uint32_t* anc_words;
+  uint32_t anc_tag;
+  unsigned long long wait_limit_ns;
+};
 
 struct RouteArgs {
   const float* logits;
@@ -111,7 +124,7 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
                                  float* logits, int T, int H, int E, float* zero_buf,
                                  size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status,
                                  float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k, int32_t* tile_done,
-                                 bool pdl, cudaStream_t s, long long* dbg = nullptr);
+                                 bool pdl, cudaStream_t s, long long* dbg = nullptr, const RootArgs* root = nullptr);
 cudaError_t launch_select(const SelectArgs& a, int T, int E, int k, cudaStream_t s);
 cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s);
 // The fused calls' stages 1b-3 in ONE launch, a cluster of select_ctas_per_block(widest block) CTAs per block of `bd`

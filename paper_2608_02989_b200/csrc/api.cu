@@ -536,6 +536,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_ticket = carve(16);
   const size_t o_selw = carve(32 * kMaxEarlyBlocks);
   const size_t o_ancw = carve(32 * kMaxEarlyBlocks);
+  const size_t o_rootw = carve(sizeof(unsigned long long) * kMaxExperts);
   const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
   const size_t o_diag = carve(sizeof(int32_t) * c->sm_count);
   if (cudaMalloc(&c->ws_base, off) != cudaSuccess) return fail(ACM_ERR_NOMEM);
@@ -564,6 +565,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   c->ws.ticket = reinterpret_cast<int32_t*>(b + o_ticket);
   c->ws.sel_words = reinterpret_cast<uint32_t*>(b + o_selw);
   c->ws.anc_words = reinterpret_cast<uint32_t*>(b + o_ancw);
+  c->ws.root_words = reinterpret_cast<unsigned long long*>(b + o_rootw);
   c->resident_dev = reinterpret_cast<uint32_t*>(b + o_res);
   c->wait_diag = reinterpret_cast<int32_t*>(b + o_diag);
   *out = c;
@@ -805,11 +807,20 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
     ACM_CUDA(cudaEventRecord(oev[0], s));
   }
   // stage 1a: the logits (the kernel also clears the output the FFN accumulates into and the FFN kernel's
-  // routing inputs)
+  // routing inputs); on an early call its first CTAs also work out the root's logits ahead of the rest and publish
+  // the anchors (on every early call, used or not: the words never carry an old tag)
+  RootArgs root = {};
+  root.rows = 1;
+  root.words = c->ws.root_words;
+  root.tag = static_cast<uint32_t>(early_epoch);
+  root.anc_words = c->ws.anc_words;
+  root.anc_tag = static_cast<uint32_t>(early_epoch) & 0xffffu;
+  root.wait_limit_ns = c->wait_limit_ns;
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, f32 ? nullptr : out,
                                 f32 ? 0 : static_cast<size_t>(T) * d.hidden, c->ws.wtab, c->ffn_in_floats,
                                 c->ws.status, nullptr, nullptr, nullptr, k, nullptr, c->pdl, s,
-                                c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr));
+                                c->trace ? reinterpret_cast<long long*>(c->trace) + 32 * c->sm_count : nullptr,
+                                early ? &root : nullptr));
   // stages 1b-3: one cluster of CTAs, which also fills the FFN kernel's routing inputs
   SelectArgs sa;
   sa.probs = nullptr; sa.nat_idx = nullptr; sa.alpha = alpha; sa.anchor_nodes = nullptr;   // (the fused kernel keeps both on chip)
@@ -832,9 +843,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   one.n_blocks = 1;
   one.off[0] = 0;
   one.off[1] = T;
-  // (the anchors are published on every early call, used or not: the words never carry an old tag)
-  ACM_CUDA(launch_softmax_select_route(sa, ra, one, eligible_mask_override, early ? c->ws.anc_words : nullptr, E, k,
-                                       c->pdl, s));
+  ACM_CUDA(launch_softmax_select_route(sa, ra, one, eligible_mask_override, nullptr, E, k, c->pdl, s));
   c->launches += 2;
 
   if (f32) {
@@ -1483,6 +1492,7 @@ acm_status acm_device_status(acm_ctx* c, acm_stream stream) {
     ACM_CUDA(cudaMemset(c->ws.ticket, 0, 16));
     ACM_CUDA(cudaMemset(c->ws.sel_words, 0, 32 * kMaxEarlyBlocks));
     ACM_CUDA(cudaMemset(c->ws.anc_words, 0, 32 * kMaxEarlyBlocks));
+    ACM_CUDA(cudaMemset(c->ws.root_words, 0, sizeof(unsigned long long) * kMaxExperts));
     c->epoch = 0;
     ACM_CUDA(cudaMemset(c->ws.tile_done, 0, sizeof(int32_t) * kMaxNodes));
   }

@@ -192,6 +192,9 @@ struct ElemTraits<__nv_bfloat16> {
   }
 };
 
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 v) { return __uint_as_float(static_cast<unsigned>(__bfloat16_as_ushort(v)) << 16); }
+
 // ---- bulk asynchronous copies (global -> shared) completing on an mbarrier ----
 __device__ __forceinline__ unsigned smem_addr(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ void mbar_init(unsigned long long* bar, int count) {
@@ -222,7 +225,7 @@ __global__ void __launch_bounds__(kRT * kRE * (32 / ElemTraits<Elem>::EPT))
 k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const float* __restrict__ bias,
                 float* logits, int T, int H, int E, int n_chunks, float* zero_buf,
                 size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status, float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k,
-                int32_t* tile_done, long long* dbg) {
+                int32_t* tile_done, long long* dbg, RootArgs ro) {
   constexpr int EPT = ElemTraits<Elem>::EPT;
   constexpr int Q = 32 / EPT;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -231,7 +234,10 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
   unsigned char* ws = smem_raw + static_cast<size_t>(kRT) * row_bytes;
 
   const int tid = threadIdx.x;
-  const int e0 = blockIdx.x * kRE, t0 = blockIdx.y * kRT;
+  // With ro.rows = 1 the first row of CTAs in the grid works on the block's root alone (see below); the node tiles
+  // follow from blockIdx.y = 1.
+  const bool for_root = ro.rows != 0 && blockIdx.y == 0;
+  const int e0 = blockIdx.x * kRE, t0 = for_root ? 0 : (static_cast<int>(blockIdx.y) - ro.rows) * kRT;
   griddep_launch_dependents();
 
   // Staging: the 4 x-rows and 8 router rows of this tile, in n_chunks pieces along h.  One thread
@@ -280,6 +286,83 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
       float4* z4 = reinterpret_cast<float4*>(zero_buf2);
       for (size_t i = b * blockDim.x + tid; i < zero_floats2 / 4; i += nb * blockDim.x) z4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
+  }
+
+  if (for_root) {
+    // The root's natural top-k are anchors (Eq. 5): eligible whatever the selection decides, and what the FFN kernel
+    // starts streaming on.  These CTAs come first in the grid, so they are resident (router rows on the way) before
+    // everyone else, and they give the root's eight logits of their tile a whole warp each -- one lane per partial
+    // sum, the same sums in the same order as below -- instead of eight threads: the root's logits are out a
+    // microsecond or two before the tile's.  They go out as 64-bit words, the value under the call's 32-bit tag;
+    // the first of these CTAs collects all E of them, ranks them by counting (rank = logits that are larger, or
+    // equal with a lower index: the order the top-k rounds take them in) and publishes the top-k as the eight
+    // tagged anchor words the FFN kernel polls.
+    for (int c = 0; c < n_chunks; ++c)
+      if (!mbar_wait_bounded(&chunk_bar[c], 0u)) raise_status(status, ACM_ERR_TIMEOUT);
+    const int w = tid >> 5, l = tid & 31;
+    const Elem* xr = reinterpret_cast<const Elem*>(xs);
+    const Elem* wrow = reinterpret_cast<const Elem*>(ws + static_cast<size_t>(w) * row_bytes);
+    float acc = 0.0f;
+#pragma unroll 8
+    for (int j = 0; j < H / 32; ++j) acc = __fmaf_rn(to_f32(xr[32 * j + l]), to_f32(wrow[32 * j + l]), acc);
+#pragma unroll
+    for (int s = 16; s >= 1; s >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, s));
+    const int e = e0 + w;
+    if (l == 0 && e < E) {
+      float z = acc;
+      if (bias) z = __fadd_rn(z, bias[e]);
+      const unsigned long long word = (static_cast<unsigned long long>(ro.tag) << 32) | __float_as_uint(z);
+      asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(ro.words + e), "l"(word) : "memory");
+    }
+    if (blockIdx.x != 0) return;
+    __shared__ unsigned s_key[kMaxExperts];
+    __shared__ int s_rank[kMaxExperts];
+    if (tid < kMaxExperts) {
+      unsigned key = 0u;
+      if (tid < E) {
+        unsigned long long v = 0ull;
+        const long long t_start = time_ns();
+        bool seen = false;
+        do {
+          asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(ro.words + tid) : "memory");
+          seen = static_cast<uint32_t>(v >> 32) == ro.tag;
+        } while (!seen && time_ns() - t_start < static_cast<long long>(ro.wait_limit_ns));
+        if (!seen) raise_status(status, ACM_ERR_TIMEOUT);
+        key = seen ? order_key(__uint_as_float(static_cast<uint32_t>(v))) : 0u;
+      }
+      s_key[tid] = key;
+      s_rank[tid] = 0;
+    }
+    __syncthreads();
+    {
+      const int mine_e = tid & (kMaxExperts - 1), half = tid >> 7;      // two threads per logit, 64 comparisons each
+      const unsigned mine = s_key[mine_e];
+      int cnt = 0;
+      const uint4* keys4 = reinterpret_cast<const uint4*>(s_key + 64 * half);
+#pragma unroll 4
+      for (int j = 0; j < 16; ++j) {
+        const uint4 kk = keys4[j];
+        const int b = 64 * half + 4 * j;
+        cnt += (kk.x > mine || (kk.x == mine && b + 0 < mine_e)) ? 1 : 0;
+        cnt += (kk.y > mine || (kk.y == mine && b + 1 < mine_e)) ? 1 : 0;
+        cnt += (kk.z > mine || (kk.z == mine && b + 2 < mine_e)) ? 1 : 0;
+        cnt += (kk.w > mine || (kk.w == mine && b + 3 < mine_e)) ? 1 : 0;
+      }
+      if (cnt) atomicAdd(&s_rank[mine_e], cnt);
+    }
+    __syncthreads();
+    if (tid < 32) {
+      uint32_t bits[kMaskWords];
+#pragma unroll
+      for (int c = 0; c < kMaskWords; ++c)
+        bits[c] = __ballot_sync(0xffffffffu, s_key[tid + 32 * c] != 0u && s_rank[tid + 32 * c] < k);
+      if (tid < 2 * kMaskWords) {
+        const uint32_t wd = (tid >> 1) == 0 ? bits[0] : (tid >> 1) == 1 ? bits[1] : (tid >> 1) == 2 ? bits[2] : bits[3];
+        asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(ro.anc_words + tid),
+                     "r"(((wd >> (16 * (tid & 1))) & 0xffffu) | (ro.anc_tag << 16)) : "memory");
+      }
+    }
+    return;
   }
 
   const int q = tid % Q;            // which EPT-wide group of the 32 partial sums
@@ -929,15 +1012,18 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
                                  float* logits, int T, int H, int E, float* zero_buf,
                                  size_t zero_floats, float* zero_buf2, size_t zero_floats2, int32_t* status,
                                  float* probs, int32_t* nat_idx, uint32_t* nat_mask, int k, int32_t* tile_done,
-                                 bool pdl, cudaStream_t s, long long* dbg) {
+                                 bool pdl, cudaStream_t s, long long* dbg, const RootArgs* root) {
   if (!probs && !nat_idx) tile_done = nullptr;
+  RootArgs ro = {};
+  if (root) ro = *root;
+  if (ro.rows != 0 && (!ro.words || !ro.anc_words || ro.rows != 1)) return cudaErrorInvalidValue;
   cudaLaunchAttribute attr[1];
   set_pdl_attr(attr);
   cudaLaunchConfig_t cfg = {};
   cfg.stream = s;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
-  const dim3 grid((E + kRE - 1) / kRE, (T + kRT - 1) / kRT);
+  const dim3 grid((E + kRE - 1) / kRE, (T + kRT - 1) / kRT + ro.rows);
   const int elt = dtype == ACM_F32 ? 4 : 2;
   size_t smem = static_cast<size_t>(kRT + kRE) * (static_cast<size_t>(H) * elt + 64);
   // At most two CTAs per SM (by asking for more shared memory than the tile needs): the grid then
@@ -954,7 +1040,7 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * 8); cfg.dynamicSmemBytes = smem;
     return cudaLaunchKernelEx(&cfg, kern, static_cast<const float*>(x), static_cast<const float*>(w_router), bias,
                               logits, T, H, E, n_chunks, zero_buf, zero_floats, zero_buf2, zero_floats2, status, probs, nat_idx, nat_mask, k,
-                              tile_done, dbg);
+                              tile_done, dbg, ro);
   } else {
     auto kern = k_router_logits<__nv_bfloat16>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
@@ -962,7 +1048,7 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
     cfg.gridDim = grid; cfg.blockDim = dim3(kRT * kRE * (32 / ElemTraits<__nv_bfloat16>::EPT)); cfg.dynamicSmemBytes = smem;
     return cudaLaunchKernelEx(&cfg, kern, static_cast<const __nv_bfloat16*>(x),
                               static_cast<const __nv_bfloat16*>(w_router), bias, logits, T, H, E, n_chunks, zero_buf,
-                              zero_floats, zero_buf2, zero_floats2, status, probs, nat_idx, nat_mask, k, tile_done, dbg);
+                              zero_floats, zero_buf2, zero_floats2, status, probs, nat_idx, nat_mask, k, tile_done, dbg, ro);
   }
 }
 
