@@ -51,8 +51,8 @@ struct Workspace {
   int32_t* tile_done;   // [64] router kernel: expert tiles finished per node tile (self-resetting)
   int32_t* ticket;      // [4] spare words (the MXFP4 scale check keeps its maximum in one)
   uint32_t* sel_words;  // [kMaxEarlyBlocks][8] the eligible masks as tagged 16-bit pieces (early start of the FFN kernel)
-  unsigned long long* root_words;   // [kMaxExperts] the root's logits under the call's 32-bit tag (router kernel, see RootArgs)
-  uint32_t* anc_words;  // [kMaxEarlyBlocks][8] the anchor experts (each root's natural top-k) as tagged 16-bit pieces, published by the selection kernel first thing
+  unsigned long long* root_words;   // [kMaxEarlyBlocks][kMaxExperts] the roots' logits under the call's 32-bit tag (router kernel, see RootArgs)
+  uint32_t* anc_words;  // [kMaxEarlyBlocks][8] the anchor experts (each root's natural top-k) as tagged 16-bit pieces, published by the router kernel's root CTAs
 };
 
 struct SelectArgs {
@@ -77,11 +77,13 @@ struct BatchDesc {
 };
 constexpr int kMaxEarlyBlocks = 8;   // blocks whose eligible sets the FFN kernel can poll for (8 tagged words each)
 
-// Single-block fused call with an early start of the FFN kernel: the router kernel puts `rows` (0 or 1) rows of CTAs
-// in front of its grid that work out the root's logits ahead of everyone (published as 64-bit words, the value under
-// `tag`, in words[kMaxExperts]) and from them the anchors (Eq. 5), published as the eight tagged words anc_words.
+// Fused calls with an early start of the FFN kernel: the router kernel puts `rows` rows of CTAs (one per block, at most
+// kMaxEarlyBlocks) in front of its grid; row b works out the logits of block b's root, the node row[b], ahead of
+// everyone (published as 64-bit words, the value under `tag`, in words[b][kMaxExperts]) and from them the block's
+// anchors (Eq. 5), published as the eight tagged words anc_words[b][8].
 struct RootArgs {
   int rows;
+  int row[kMaxEarlyBlocks];
   unsigned long long* words;
   uint32_t tag;
   uint32_t* anc_words;
@@ -130,14 +132,12 @@ cudaError_t launch_route(const RouteArgs& a, int T, int E, int k, cudaStream_t s
 // The fused calls' stages 1b-3 in ONE launch, a cluster of select_ctas_per_block(widest block) CTAs per block of `bd`
 // (a single block: n_blocks = 1, off = {0, T}): softmax and natural top-k of the logits in ra.logits, selection
 // (unless mask_override, single block only), routes, the FFN kernel's routing inputs.  The per-block outputs of `sa`
-// (mask, unpruned, count, demand [kMaxExperts each], stats) are arrays over the blocks; ra.sel_flag and anc_words
-// (both may be null) hold 8 tagged words per block: the eligible set and, earlier, the anchors (the natural top-k
-// of the block's first row).
+// (mask, unpruned, count, demand [kMaxExperts each], stats) are arrays over the blocks; ra.sel_flag (may be
+// null) holds 8 tagged words per block for the eligible set.
 int select_ctas_per_block(int widest);
 cudaError_t select_configure();   // the kernel's function attributes, once per device (when a context is created)
 cudaError_t launch_softmax_select_route(const SelectArgs& sa, const RouteArgs& ra, const BatchDesc& bd,
-                                        const uint32_t* mask_override, uint32_t* anc_words, int E, int k, bool pdl,
-                                        cudaStream_t s);
+                                        const uint32_t* mask_override, int E, int k, bool pdl, cudaStream_t s);
 // routes given by the caller -> activated mask, weight table (both cleared first) and cleared `ready`
 cudaError_t launch_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask, float* wtab,
                                    int32_t* ready, int T, int E, int k, cudaStream_t s);
@@ -171,7 +171,7 @@ struct FfnLaunch {
   int32_t sel_epoch;
   int sel_blocks;            // blocks of a batch (1..kMaxEarlyBlocks): eight words each, the work list is their union
   const uint32_t* anc_flag = nullptr;   // with sel_flag: eight words tagged alike holding the anchor experts (published by the
-                             // selection kernel, earlier): their gate/up tiles are streamed while the selection still runs
+                             // router kernel, earlier): their gate/up tiles are streamed while the selection still runs
   float* out;                // [T,H], accumulated into (zeroed by the caller)
   int32_t* status;
   int grid;

@@ -536,7 +536,7 @@ acm_status acm_create(const acm_model_desc* desc, acm_ctx** out) {
   const size_t o_ticket = carve(16);
   const size_t o_selw = carve(32 * kMaxEarlyBlocks);
   const size_t o_ancw = carve(32 * kMaxEarlyBlocks);
-  const size_t o_rootw = carve(sizeof(unsigned long long) * kMaxExperts);
+  const size_t o_rootw = carve(sizeof(unsigned long long) * kMaxExperts * kMaxEarlyBlocks);
   const size_t o_res = carve(sizeof(uint32_t) * 4 * desc->n_layers);
   const size_t o_diag = carve(sizeof(int32_t) * c->sm_count);
   if (cudaMalloc(&c->ws_base, off) != cudaSuccess) return fail(ACM_ERR_NOMEM);
@@ -796,9 +796,9 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
     st = next_epoch(c, s, &early_epoch);
     if (st != ACM_OK) return st;
   }
-  // ... and earlier still on the anchors (Eq. 5 with the default anchor, the root): the selection kernel publishes
-  // the root's natural top-k as soon as that row's softmax is done, the FFN kernel streams their gate/up tiles
-  // while the selection runs.  They are in every eligible set the selection can return without a residency.
+  // ... and earlier still on the anchors (Eq. 5 with the default anchor, the root): the router kernel's first CTAs
+  // work out the root's logits ahead of the rest and publish its natural top-k, the FFN kernel streams their gate/up
+  // tiles while the softmax and the selection run.  They are in every eligible set the selection can return without a residency.
   const bool anchors_first = early && c->anchor_start && prm.use_anchors != 0;
   // offload timing: events around the resident part, the copies and the loaded part of this call
   cudaEvent_t* oev = nullptr;
@@ -811,6 +811,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   // the anchors (on every early call, used or not: the words never carry an old tag)
   RootArgs root = {};
   root.rows = 1;
+  root.row[0] = 0;
   root.words = c->ws.root_words;
   root.tag = static_cast<uint32_t>(early_epoch);
   root.anc_words = c->ws.anc_words;
@@ -843,7 +844,7 @@ acm_status acm_moe_verify(acm_ctx* c, int layer, const void* x, int T, const flo
   one.n_blocks = 1;
   one.off[0] = 0;
   one.off[1] = T;
-  ACM_CUDA(launch_softmax_select_route(sa, ra, one, eligible_mask_override, nullptr, E, k, c->pdl, s));
+  ACM_CUDA(launch_softmax_select_route(sa, ra, one, eligible_mask_override, E, k, c->pdl, s));
   c->launches += 2;
 
   if (f32) {
@@ -1015,9 +1016,18 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
   }
   // ... and on the union of the blocks' anchors (each block's first row is its root) while the selections run
   const bool anchors_first = early && c->anchor_start && params->use_anchors != 0;
+  // (on an early call the router kernel's first CTAs work out every block's root ahead of the rest and publish the anchors)
+  RootArgs root = {};
+  root.rows = early ? n_blocks : 0;
+  for (int b = 0; b < root.rows; ++b) root.row[b] = bd.off[b];
+  root.words = c->ws.root_words;
+  root.tag = static_cast<uint32_t>(early_epoch);
+  root.anc_words = c->ws.anc_words;
+  root.anc_tag = static_cast<uint32_t>(early_epoch) & 0xffffu;
+  root.wait_limit_ns = c->wait_limit_ns;
   ACM_CUDA(launch_router_logits(d.dtype, x, L.w_router, L.bias, c->ws.logits, T, d.hidden, E, out,
                                 static_cast<size_t>(T) * d.hidden, c->ws.wtab, c->ffn_in_floats, c->ws.status,
-                                nullptr, nullptr, nullptr, k, nullptr, c->pdl, s, nullptr));
+                                nullptr, nullptr, nullptr, k, nullptr, c->pdl, s, nullptr, early ? &root : nullptr));
   // stages 1b-3: one cluster of CTAs per block
   SelectArgs sa;
   sa.probs = nullptr; sa.nat_idx = nullptr; sa.alpha = alpha; sa.anchor_nodes = nullptr;   // (the fused kernel keeps both on chip)
@@ -1034,7 +1044,7 @@ acm_status acm_moe_verify_batch(acm_ctx* c, int layer, const void* x, int n_bloc
     ra.sel_flag = c->ws.sel_words;
     ra.sel_epoch = early_epoch;
   }
-  ACM_CUDA(launch_softmax_select_route(sa, ra, bd, nullptr, early ? c->ws.anc_words : nullptr, E, k, c->pdl, s));
+  ACM_CUDA(launch_softmax_select_route(sa, ra, bd, nullptr, E, k, c->pdl, s));
   c->launches += 2;
   // stage 4 once over all rows: an expert activated by several blocks is streamed once
   int widest = 1;
@@ -1492,7 +1502,7 @@ acm_status acm_device_status(acm_ctx* c, acm_stream stream) {
     ACM_CUDA(cudaMemset(c->ws.ticket, 0, 16));
     ACM_CUDA(cudaMemset(c->ws.sel_words, 0, 32 * kMaxEarlyBlocks));
     ACM_CUDA(cudaMemset(c->ws.anc_words, 0, 32 * kMaxEarlyBlocks));
-    ACM_CUDA(cudaMemset(c->ws.root_words, 0, sizeof(unsigned long long) * kMaxExperts));
+    ACM_CUDA(cudaMemset(c->ws.root_words, 0, sizeof(unsigned long long) * kMaxExperts * kMaxEarlyBlocks));
     c->epoch = 0;
     ACM_CUDA(cudaMemset(c->ws.tile_done, 0, sizeof(int32_t) * kMaxNodes));
   }

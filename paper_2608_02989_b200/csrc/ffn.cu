@@ -79,7 +79,7 @@ using plan::plan_lane;
 // names the wait that gave up first (acm_wait_report reads it).
 enum WaitSite : int {
   kSiteNone = 0,
-  kSiteAnchorWords = 1,     // prologue: the anchors' tagged words (selection kernel, first thing)
+  kSiteAnchorWords = 1,     // prologue: the anchors' tagged words (router kernel's root CTAs)
   kSiteEligibleWords = 2,   // prologue / helper: the eligible set's tagged words (selection kernel)
   kSiteStageEmpty = 3,      // weight producer: a ring stage the MMAs have not released
   kSiteAccEmpty = 4,        // MMA issuer: an accumulator the epilogue has not drained
@@ -486,7 +486,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
   // Everything above touched only this CTA's own resources; global memory written by the kernels
   // before this one is read only from here on.  Early start: wait for the eligible set only.
   const bool early = p.sel_flag != nullptr;
-  // Early start on the ANCHORS (Eq. 5: the root's natural top-k, always eligible): the selection kernel publishes
+  // Early start on the ANCHORS (Eq. 5: the root's natural top-k, always eligible): the router kernel publishes
   // them microseconds before the selection is done.  Their gate/up tiles become segment 0 of the plan, one
   // whole tile per CTA, and the roles start on it at once; the helper warp meanwhile waits for the eligible
   // set, completes the work list (the pre-streamed experts keep the first slots) and the plan, and opens

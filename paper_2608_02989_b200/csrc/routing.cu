@@ -234,10 +234,12 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
   unsigned char* ws = smem_raw + static_cast<size_t>(kRT) * row_bytes;
 
   const int tid = threadIdx.x;
-  // With ro.rows = 1 the first row of CTAs in the grid works on the block's root alone (see below); the node tiles
-  // follow from blockIdx.y = 1.
-  const bool for_root = ro.rows != 0 && blockIdx.y == 0;
-  const int e0 = blockIdx.x * kRE, t0 = for_root ? 0 : (static_cast<int>(blockIdx.y) - ro.rows) * kRT;
+  // The first ro.rows rows of CTAs in the grid work on one block's root each (see below); the node tiles follow.
+  const bool for_root = static_cast<int>(blockIdx.y) < ro.rows;
+  int root_row = 0;
+#pragma unroll
+  for (int b = 0; b < kMaxEarlyBlocks; ++b) root_row = static_cast<int>(blockIdx.y) == b ? ro.row[b] : root_row;
+  const int e0 = blockIdx.x * kRE, t0 = for_root ? root_row : (static_cast<int>(blockIdx.y) - ro.rows) * kRT;
   griddep_launch_dependents();
 
   // Staging: the 4 x-rows and 8 router rows of this tile, in n_chunks pieces along h.  One thread
@@ -289,7 +291,7 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
   }
 
   if (for_root) {
-    // The root's natural top-k are anchors (Eq. 5): eligible whatever the selection decides, and what the FFN kernel
+    // A root's natural top-k are anchors (Eq. 5): eligible whatever the selection decides, and what the FFN kernel
     // starts streaming on.  These CTAs come first in the grid, so they are resident (router rows on the way) before
     // everyone else, and they give the root's eight logits of their tile a whole warp each -- one lane per partial
     // sum, the same sums in the same order as below -- instead of eight threads: the root's logits are out a
@@ -312,7 +314,7 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
       float z = acc;
       if (bias) z = __fadd_rn(z, bias[e]);
       const unsigned long long word = (static_cast<unsigned long long>(ro.tag) << 32) | __float_as_uint(z);
-      asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(ro.words + e), "l"(word) : "memory");
+      asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(ro.words + static_cast<size_t>(blockIdx.y) * kMaxExperts + e), "l"(word) : "memory");
     }
     if (blockIdx.x != 0) return;
     __shared__ unsigned s_key[kMaxExperts];
@@ -324,7 +326,7 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
         const long long t_start = time_ns();
         bool seen = false;
         do {
-          asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(ro.words + tid) : "memory");
+          asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(ro.words + static_cast<size_t>(blockIdx.y) * kMaxExperts + tid) : "memory");
           seen = static_cast<uint32_t>(v >> 32) == ro.tag;
         } while (!seen && time_ns() - t_start < static_cast<long long>(ro.wait_limit_ns));
         if (!seen) raise_status(status, ACM_ERR_TIMEOUT);
@@ -358,7 +360,7 @@ k_router_logits(const Elem* __restrict__ x, const Elem* __restrict__ wr, const f
         bits[c] = __ballot_sync(0xffffffffu, s_key[tid + 32 * c] != 0u && s_rank[tid + 32 * c] < k);
       if (tid < 2 * kMaskWords) {
         const uint32_t wd = (tid >> 1) == 0 ? bits[0] : (tid >> 1) == 1 ? bits[1] : (tid >> 1) == 2 ? bits[2] : bits[3];
-        asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(ro.anc_words + tid),
+        asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(ro.anc_words + 2 * kMaskWords * blockIdx.y + tid),
                      "r"(((wd >> (16 * (tid & 1))) & 0xffffu) | (ro.anc_tag << 16)) : "memory");
       }
     }
@@ -824,10 +826,8 @@ __device__ __forceinline__ void publish_eligible(const RouteArgs& ra, const Stag
 // router kernel before it has written the logits only.  Every warp loads its row (the one trip through L2 of the
 // whole chain: with the FFN kernel already streaming weights, each further one would cost well over a microsecond),
 // then
-//   1b  natural top-k and softmax of the row (Eq. 1); the probabilities and the top-k mask go into the shared memory
-//       of EVERY CTA of the cluster (distributed shared memory), the logits stay in registers; the block's first row
-//       is its root, whose natural top-k are anchors (Eq. 5) and published at once as eight tagged words for the FFN
-//       kernel to start on;
+//   1b  softmax and natural top-k of the row (Eq. 1); the probabilities and the top-k mask go into the shared memory
+//       of EVERY CTA of the cluster (distributed shared memory), the logits stay in registers;
 //   --  cluster barrier: every CTA now holds the whole block's probabilities and natural sets
 //   2   the selection (Eq. 3-7; it sees nothing of the other blocks), repeated by warps 0-3 of every CTA -- it is
 //       deterministic, so all hold the same S' and no second exchange is needed; the cluster's first CTA writes the
@@ -848,8 +848,7 @@ struct FusedSmem {
 };
 static_assert(sizeof(FusedSmem) <= kFusedSmemRequest, "shared memory of the selection kernel");
 __global__ void __launch_bounds__(32 * kFusedWarps)
-k_softmax_select_route(SelectArgs sa, RouteArgs ra, BatchDesc bd, const uint32_t* mask_override, uint32_t* anc_words,
-                       int E, int k) {
+k_softmax_select_route(SelectArgs sa, RouteArgs ra, BatchDesc bd, const uint32_t* mask_override, int E, int k) {
   extern __shared__ __align__(16) unsigned char fused_raw[];
   FusedSmem& fs = *reinterpret_cast<FusedSmem*>(fused_raw);
   StageSmem& sm = fs.st;
@@ -878,16 +877,9 @@ k_softmax_select_route(SelectArgs sa, RouteArgs ra, BatchDesc bd, const uint32_t
   if (tid < kMaskWords) sm.Hres[tid] = (tid < (E + 31) / 32) ? (sa.resident ? sa.resident[tid] : 0xffffffffu) : 0u;
   if (tid < 8) sm.scal[tid] = 0;
   if (r < T && !mask_override) {
-    // (the top-k first: the root's are what the FFN kernel is waiting for)
     float prob[4];
-    uint32_t bits[kMaskWords], none[kMaskWords];
-    topk_bits(z, E, k, lane, bits, nullptr);
-    if (r == 0 && anc_words && lane < 2 * kMaskWords) {
-      const uint32_t w = (lane >> 1) == 0 ? bits[0] : (lane >> 1) == 1 ? bits[1] : (lane >> 1) == 2 ? bits[2] : bits[3];
-      asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(anc_words + 2 * kMaskWords * b + lane),
-                   "r"(((w >> (16 * (lane & 1))) & 0xffffu) | (tag << 16)) : "memory");
-    }
-    softmax_topk_regs(z, E, k, lane, prob, none, nullptr, false);
+    uint32_t bits[kMaskWords];
+    softmax_topk_regs(z, E, k, lane, prob, bits, nullptr, true);
     const uint32_t my_bits = lane == 0 ? bits[0] : lane == 1 ? bits[1] : lane == 2 ? bits[2] : bits[3];
     for (int p = 0; p < C; ++p) {
       float* probs_p = cluster.map_shared_rank(fs.probs, p);
@@ -1016,7 +1008,7 @@ cudaError_t launch_router_logits(int dtype, const void* x, const void* w_router,
   if (!probs && !nat_idx) tile_done = nullptr;
   RootArgs ro = {};
   if (root) ro = *root;
-  if (ro.rows != 0 && (!ro.words || !ro.anc_words || ro.rows != 1)) return cudaErrorInvalidValue;
+  if (ro.rows != 0 && (!ro.words || !ro.anc_words || ro.rows < 0 || ro.rows > kMaxEarlyBlocks)) return cudaErrorInvalidValue;
   cudaLaunchAttribute attr[1];
   set_pdl_attr(attr);
   cudaLaunchConfig_t cfg = {};
@@ -1073,8 +1065,7 @@ int select_ctas_per_block(int widest) {
 }
 
 cudaError_t launch_softmax_select_route(const SelectArgs& sa, const RouteArgs& ra, const BatchDesc& bd,
-                                        const uint32_t* mask_override, uint32_t* anc_words, int E, int k, bool pdl,
-                                        cudaStream_t s) {
+                                        const uint32_t* mask_override, int E, int k, bool pdl, cudaStream_t s) {
   int widest = 1;
   for (int b = 0; b < bd.n_blocks; ++b) widest = bd.off[b + 1] - bd.off[b] > widest ? bd.off[b + 1] - bd.off[b] : widest;
   if (widest > kFusedMaxCtas * kFusedWarps) return cudaErrorInvalidValue;      // a warp per row
@@ -1092,7 +1083,7 @@ cudaError_t launch_softmax_select_route(const SelectArgs& sa, const RouteArgs& r
   cfg.stream = s;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 2 : 1;
-  return cudaLaunchKernelEx(&cfg, k_softmax_select_route, sa, ra, bd, mask_override, anc_words, E, k);
+  return cudaLaunchKernelEx(&cfg, k_softmax_select_route, sa, ra, bd, mask_override, E, k);
 }
 
 cudaError_t launch_routes_to_table(const int32_t* idx, const float* w, uint32_t* act_mask, float* wtab,
