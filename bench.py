@@ -27,7 +27,7 @@ ROOT = Path(__file__).resolve().parent
 if str(ROOT) not in sys.path:
     sys.path.insert(0, str(ROOT))
 
-DRAM_BYTES_PER_ACTIVATED_EXPERT = {3: (273970176 + 193497088 + 193248256) / 68.0}   # config -> bytes (ncu, profiles/)
+DRAM_BYTES_PER_ACTIVATED_EXPERT = {3: (273758464 + 193700864 + 193257216) / 68.0}   # config -> bytes (ncu, profiles/)
 METRIC = "verify_blocks_per_s_per_moe_layer"
 UNIT = "layer-blocks/s"
 
