@@ -321,7 +321,7 @@ acm_status acm_offload_times(acm_ctx* ctx, double* ms_out /*host [4]*/, int32_t*
  *       is published;
  *   [2] stage 3: the routes (Eq. 2) and the FFN kernel's routing inputs;
  *   [3] stage 4: the FFN kernel from its first CTA's roles starting to its last tile finished -- it
- *       starts on the anchor experts while stage 2 runs, so [0..3] overlap and do not add up to
+ *       starts on the anchor experts while stages 1 and 2 still run, so [0..3] overlap and do not add up to
  *   [4] the whole: from the start of [0] to the end of [3].
  * ACM_ERR_INVALID when the stamps are off or no such call has run. */
 acm_status acm_stage_timing(acm_ctx* ctx, int enable);
