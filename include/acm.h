@@ -117,7 +117,9 @@ typedef struct {
   int32_t displaced_aS;       /* a(S): natural assignments displaced by restricting to S */
   int32_t pruned_m;           /* m* of Eq. 7 */
   int32_t n_staged;           /* activated experts that were not GPU-resident */
-  int32_t reserved[3];
+  int32_t n_streamed;         /* routed experts whose weights the block's first FFN launch streamed: the activated ones,
+                                 or -- when it starts before the routes exist -- the eligible ones (anchors included) */
+  int32_t reserved[2];
 } acm_block_stats;
 
 /* Fills the paper's defaults: Eq. 4 demand, anchors on, self-sized, tau = 2^-10, no residency. */

@@ -54,9 +54,9 @@ class BlockStats(ctypes.Structure):
     _fields_ = [("n_anchor", c_int32), ("n_er", c_int32), ("n_eligible", c_int32),
                 ("n_eligible_pruned", c_int32), ("n_activated", c_int32), ("n_natural_union", c_int32),
                 ("displaced_aS", c_int32), ("pruned_m", c_int32), ("n_staged", c_int32),
-                ("reserved", c_int32 * 3)]
+                ("n_streamed", c_int32), ("reserved", c_int32 * 2)]
     NAMES = ["n_anchor", "n_er", "n_eligible", "n_eligible_pruned", "n_activated", "n_natural_union",
-             "displaced_aS", "pruned_m", "n_staged"]
+             "displaced_aS", "pruned_m", "n_staged", "n_streamed"]
 
 
 class AcmError(RuntimeError):

@@ -122,6 +122,7 @@ struct __align__(8) BarriersT {
   unsigned long long raw[kMaxStages];   // the packed weight stage has landed (producer's copy -> expanding warps)
 #endif
   volatile uint32_t armed;           // stages whose barrier the weight producer has armed so far
+  volatile int32_t n_routed_slots;   // routed experts in this launch's work list (known with the complete list)
   uint32_t tmem_base;
   GiveUp give_up;
   float wd[kN];                 // combine weights of the expert being finalised
@@ -571,6 +572,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
       bars->plan.n_seg = 1;
     }
   } else if (warp == kThreads / 32 - 1 && lane < 4) {      // (the publisher warp has nothing else to do yet)
+    if (lane == 0) bars->n_routed_slots = n_routed;
     plan_lane(bars->plan, lane, cta, n_act, tpe, G, p.d_kc1, kpe, p.d_grid, p.d_tpe, h_tiles);
   }
   int32_t* s_entry = bars->entry;
@@ -701,6 +703,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
         }
         p.stats->n_activated = n_all;
         p.stats->n_staged = n_stg;
+        p.stats->n_streamed = bars->n_routed_slots;
       }
       if (!ok) {
         // giving up: let copies already in flight land before the CTA exits
@@ -817,6 +820,7 @@ ACM_FFN_KERNEL(const __grid_constant__ FfnMaps maps, const __grid_constant__ CUt
           s_entry[n_pre + n_rest + lane] = make_entry(kSrcShared, lane);
           bars->expert[n_pre + n_rest + lane] = -1;
         }
+        if (lane == 0) bars->n_routed_slots = n_pre + n_rest;
         if (lane < 4)
           plan_lane(bars->plan, lane, cta, n_pre + n_rest + p.n_shared, tpe, G, p.d_kc1, kpe, p.d_grid, p.d_tpe, h_tiles,
                     n_pre, 1);

@@ -717,7 +717,7 @@ __device__ void stage_select(const SelectArgs& a, StageSmem& sm, int T, int E, i
         acm_block_stats st;
         st.n_anchor = nA; st.n_er = n_er; st.n_eligible = nS; st.n_eligible_pruned = nSp;
         st.n_activated = 0; st.n_natural_union = n_union; st.displaced_aS = aS; st.pruned_m = m_star;
-        st.n_staged = 0; st.reserved[0] = st.reserved[1] = st.reserved[2] = 0;
+        st.n_staged = 0; st.n_streamed = 0; st.reserved[0] = st.reserved[1] = 0;
         *a.stats_out = st;
       }
     }

@@ -262,6 +262,11 @@ def _verify_layer(cfg, layer, ctx, slot, params_kw=None, rows=None, natural=Fals
         for key in ("n_anchor", "n_er", "n_eligible", "n_natural_union", "displaced_aS"):
             assert st[key] == ref["stats"][key]
     assert st["n_activated"] == len(set(ref["idx"].ravel()) - {-1})
+    if cfg.dtype == "bf16":
+        # what the FFN launch streamed: with an early start every eligible expert -- the anchors it started on (ranked
+        # by the router kernel's root CTAs from their own copy of the root's logits) must all be among them -- else
+        # the activated ones
+        assert st["n_streamed"] == (st["n_activated"] if natural else st["n_eligible_pruned"])
     rows = np.arange(cfg.n_nodes) if rows is None else np.asarray(rows)
     ffn = oracle.expert_ffn(_take(x, rows), ref["idx"][rows], ref["w"][rows], w["gate_up"], w["down"],
                             w["shared_gate_up"], w["shared_down"])
